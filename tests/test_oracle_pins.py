@@ -1,0 +1,502 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix (no GPU).
+
+Each test is chosen so that a plausible slip in the oracle (a dropped term, a wrong sign or index,
+an off-by-one median, a swapped class) fails it.
+"""
+import json
+import os
+
+import numpy as np
+import pytest
+
+import oracle as orc
+from helpers import (ALLGATHER, ALLREDUCE, MiB, SENDRECV, frames_from, group_trace, make_cols)
+
+GOLD = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "paper_values.json")))
+
+
+def run(recs, comms, params=None, now=10**12, with_rates=True, frames=None, n_channels=0, windows=None):
+    o = orc.Oracle(params)
+    for cid, ranks, seq0 in comms:
+        assert o.comm_register(cid, ranks, seq0) == 0
+    if windows is None:
+        windows = [recs]
+    for w, r in enumerate(windows):
+        assert o.upload(w, make_cols(r, with_rates), frames if w == len(windows) - 1 else None, n_channels) == 0
+    assert o.analyze(0, len(windows), now) == 0
+    return o
+
+
+# ---------------------------------------------------------------- defaults the paper prints
+def test_defaults_match_paper():
+    p = orc.DEFAULT_PARAMS
+    assert p["alpha_milli"] == round(GOLD["alpha"]["value"] * 1000)
+    assert p["beta_milli"] == round(GOLD["beta"]["value"] * 1000)
+    assert p["theta_slow_milli"] == GOLD["theta_slow"]["value"] * 1000
+    assert p["m_max_rounds"] == GOLD["m_max_rounds"]["value"]
+    assert p["m_max_ns"] == GOLD["m_max_seconds"]["value"] * 10**9
+    assert p["hang_ns"] == GOLD["hang_threshold_seconds"]["value"] * 10**9
+    assert p["barrier_bytes"] == GOLD["barrier_bytes"]["value"]
+    f = GOLD["frame_bytes"]
+    assert f["header"] + f["body"] == f["total"]
+    # one block = Trace ID + channels x {SendCount, RecvCount} 8-byte slots
+    assert f["body"] // f["blocks"] == f["trace_id"] + f["channels"] * 2 * 8
+
+
+# ---------------------------------------------------------------- per-op quantities
+def test_identical_ranks_flag_nothing():
+    recs = group_trace([[2_000_000] * 8 for _ in range(20)])
+    o = run(recs, [(0, list(range(8)), 0)])
+    s = o.sizes(0)
+    assert s["n_groups"] == 20 and s["n_complete"] == 20 and s["n_analysed"] == 20
+    assert s["n_flag_skew"] == 0 and s["n_flag_dur"] == 0
+    flags, _ = o.slots(0)
+    assert (flags == 0).all()
+    g = o.groups(0)
+    assert (g["arrival_skew"] == 0).all() and (g["mad_dur"] == 0).all() and (g["med_dur"] == 2_000_000).all()
+    assert o.suspects()["n_total"] == 0
+
+
+def test_one_delayed_rank_is_the_only_one_flagged():
+    rng = np.random.default_rng(1)
+    durs, ents = [], []
+    for s in range(50):
+        durs.append([2_000_000 + int(x) for x in rng.integers(-1000, 1000, 8)])
+        e = [3000 * ((i + s) % 8) for i in range(8)]           # evenly spread arrivals: nobody is an outlier
+        e[5] += 2_000_000
+        ents.append(e)
+    o = run(group_trace(durs, ents), [(0, list(range(8)), 0)])
+    flags, _ = o.slots(0)
+    f = flags.reshape(50, 8)
+    assert ((f[:, 5] & 1) == 1).all() and ((f[:, 5] & 4) == 4).all()     # late and above the median
+    others = np.delete(f, 5, axis=1)
+    assert ((others & 1) == 0).all()
+    sus = o.suspects()
+    assert list(sus["rank"][sus["kind"] == 1]) == [5]
+    st = o.rank_stats(8)
+    assert st["votes"][5, 0] == 50 and st["ops"][5] == 50
+
+
+def test_hand_sets_median_mad():
+    # {1,2,3,4,100}: lower median 3, deviations {2,1,0,1,97} -> MAD 1, only 100 is an outlier
+    # {10,20,30,40}: lower median 20, deviations {10,0,10,20} -> sorted {0,10,10,20}, MAD 10, nobody flagged
+    a = [[1, 2, 3, 4, 100]]
+    b = [[10, 20, 30, 40]]
+    o = run(group_trace(a, comm=0) + group_trace(b, comm=1), [(0, list(range(5)), 0), (1, list(range(4)), 0)])
+    g = o.groups(0)
+    assert list(g["med_dur"]) == [3, 20] and list(g["mad_dur"]) == [1, 10]
+    assert list(g["t_max"]) == [100, 40] and list(g["t_min"]) == [1, 10]
+    assert list(g["rank_tmax"]) == [4, 3] and list(g["rank_tmin"]) == [0, 0]
+    flags, _ = o.slots(0)
+    assert list(flags & 2) == [0, 0, 0, 0, 2, 0, 0, 0, 0]
+    assert list(flags & 8) == [0, 0, 0, 8, 8, 0, 0, 8, 8]      # strictly above the median
+
+
+def test_threshold_is_exact_integer_test():
+    # n = 5 durations {0, 10, 20, 30, x}: median 20, deviations {20,10,0,10,x-20} -> MAD 10.
+    # flag <=> (x-20)*1000 > k_milli*10. With k_milli = 5189: x-20 = 51 -> 51000 < 51890 no; 52 -> 52000 > 51890 yes.
+    for x, want in ((71, 0), (72, 2)):
+        o = run(group_trace([[0, 10, 20, 30, x]]), [(0, list(range(5)), 0)])
+        flags, _ = o.slots(0)
+        assert (flags[4] & 2) == want
+    # equality is not an outlier: k_milli = 5000, deviation 50 -> 50000 > 50000 is false
+    o = run(group_trace([[0, 10, 20, 30, 70]]), [(0, list(range(5)), 0)], params=dict(k_milli=5000))
+    assert (o.slots(0)[0][4] & 2) == 0
+
+
+def test_mad_zero_flags_any_deviation():
+    o = run(group_trace([[7, 7, 7, 7, 7, 7, 7, 9]]), [(0, list(range(8)), 0)])
+    flags, _ = o.slots(0)
+    assert list(flags & 2) == [0] * 7 + [2]
+    assert o.groups(0)["mad_dur"][0] == 0
+
+
+def brute_order_stat(x, k):
+    """k-th smallest by counting: the v in x with #{x < v} <= k < #{x <= v}."""
+    for v in x:
+        if sum(1 for y in x if y < v) <= k < sum(1 for y in x if y <= v):
+            return v
+    raise AssertionError
+
+
+def test_median_mad_brute_force_by_counting():
+    rng = np.random.default_rng(7)
+    recs, comms = [], []
+    sets = []
+    for c, n in enumerate([4, 5, 6, 7, 8, 9, 13, 16, 31, 32, 33, 64, 100]):
+        durs = [[int(v) for v in rng.integers(1, 50, n)] for _ in range(3)]      # many ties
+        durs += [[int(v) for v in rng.integers(1, 2**40, n)] for _ in range(3)]
+        ents = [[int(v) for v in rng.integers(0, 10**6, n)] for _ in range(6)]
+        recs += group_trace(durs, ents, comm=c, ranks=list(range(1000 * c, 1000 * c + n)))
+        comms.append((c, list(range(1000 * c, 1000 * c + n)), 0))
+        sets += list(zip(durs, ents))
+    o = run(recs, comms)
+    g = o.groups(0)
+    assert len(sets) == len(g["med_dur"])
+    for i, (d, e) in enumerate(sets):
+        n = len(d); k = (n - 1) // 2
+        med = brute_order_stat(d, k)
+        assert g["med_dur"][i] == med
+        assert g["mad_dur"][i] == brute_order_stat([abs(v - med) for v in d], k)
+        sk = [v - min(e) for v in e]
+        meds = brute_order_stat(sk, k)
+        assert g["med_skew"][i] == meds
+        assert g["mad_skew"][i] == brute_order_stat([abs(v - meds) for v in sk], k)
+        assert g["arrival_skew"][i] == max(sk) and min(sk) == 0
+        assert g["t_min"][i] <= g["med_dur"][i] <= g["t_max"][i]
+
+
+def test_mad_of_normal_sample_is_0_6745_sigma():
+    rng = np.random.default_rng(3)
+    n = 4001
+    d = (10**9 + rng.normal(0, 10**6, n)).astype(np.int64)
+    o = run(group_trace([[int(v) for v in d]]), [(0, list(range(n)), 0)])
+    g = o.groups(0)
+    assert abs(g["mad_dur"][0] / 10**6 - 0.6745) < 0.03
+    assert abs(g["med_dur"][0] - 10**9) < 10**5
+
+
+def test_bus_bandwidth_closed_forms():
+    # allreduce, n = 8, 16 MiB: every rank enters at once and takes 2 ms -> 2(n-1)/n * bytes / t
+    o = run(group_trace([[2_000_000] * 8]), [(0, list(range(8)), 0)])
+    assert o.groups(0)["busbw"][0] == pytest.approx(16 * MiB * 14 / (2_000_000 * 8), rel=1e-15)
+    assert o.groups(0)["busbw"][0] == pytest.approx(14.680064, rel=1e-12)
+    # allgather (n-1)/n, sendrecv 1: span includes the arrival skew
+    recs = group_trace([[1_000_000] * 4], [[0, 0, 0, 1_000_000]], comm=0, op=ALLGATHER, bytes=4 * MiB)
+    recs += group_trace([[1_000_000] * 4], comm=1, ranks=[4, 5, 6, 7], op=SENDRECV, bytes=4 * MiB)
+    o = run(recs, [(0, [0, 1, 2, 3], 0), (1, [4, 5, 6, 7], 0)])
+    g = o.groups(0)
+    assert g["span"][0] == 2_000_000
+    assert g["busbw"][0] == pytest.approx(4 * MiB * 3 / (2_000_000 * 4), rel=1e-15)
+    assert g["busbw"][1] == pytest.approx(4 * MiB / 1_000_000, rel=1e-15)
+    st = o.rank_stats(8)
+    assert st["bw_sum"][0] == pytest.approx(4 * MiB * 3 / (1_000_000 * 4), rel=1e-15) and st["bw_cnt"][0] == 1
+
+
+def test_votes_total_equals_flag_total_and_invariants():
+    import tracegen as tg
+    spec = tg.cfg2(reps=40, n_windows=2, tp=4, pp=2, dp=4)
+    o = orc.Oracle()
+    for cid, ranks, seq0 in tg.registry(spec):
+        o.comm_register(cid, ranks, seq0)
+    tot_skew = tot_dur = 0
+    for w in range(2):
+        win = tg.gen_window(spec, w)
+        o.upload(w, win.cols)
+        o.analyze(w, 1, win.now_ns)
+        s = o.sizes(w)
+        flags, perm = o.slots(w)
+        assert int((flags & 1).sum()) == s["n_flag_skew"] and int(((flags & 2) >> 1).sum()) == s["n_flag_dur"]
+        assert s["n_groups"] == s["n_complete"] + s["n_incomplete"]
+        tot_skew += s["n_flag_skew"]; tot_dur += s["n_flag_dur"]
+        g = o.groups(w)
+        assert (g["arrival_skew"] >= 0).all() and (g["t_min"] <= g["t_max"]).all()
+        an = (g["gflags"] & 16) != 0                           # groups that went through the median test
+        assert an.any() and not an.all()
+        assert (g["t_min"][an] <= g["med_dur"][an]).all() and (g["med_dur"][an] <= g["t_max"][an]).all()
+        assert (g["med_skew"][an] <= g["arrival_skew"][an]).all() and (g["med_dur"][~an] == 0).all()
+        # e_min really is the smallest enter time of the group's records
+        te = win.cols["t_enter"].numpy()
+        for i in (0, 7, len(g["seq"]) - 1):
+            n = int(g["n_present"][i]); s0 = int(g["slot0"][i])
+            assert g["e_min"][i] == te[perm[s0:s0 + n]].min()
+    st = o.rank_stats(spec.n_ranks)
+    assert st["votes"][:, 0].sum() + st["votes"][:, 1].sum() == tot_skew
+    assert st["votes"][:, 2].sum() + st["votes"][:, 3].sum() == tot_dur
+
+
+# ---------------------------------------------------------------- grouping
+def test_input_order_and_window_split_invariance():
+    import tracegen as tg
+    spec = tg.cfg2(reps=30, n_windows=1, tp=4, pp=2, dp=2)
+    res = []
+    for order in ("rank_major", "arrival", "shuffled"):
+        o = orc.Oracle()
+        for cid, ranks, seq0 in tg.registry(spec):
+            o.comm_register(cid, ranks, seq0)
+        win = tg.gen_window(spec, 0, order=order)
+        o.upload(0, win.cols); o.analyze(0, 1, win.now_ns)
+        g = o.groups(0)
+        res.append((g, o.rank_stats(spec.n_ranks), o.slots(0)[0]))
+    for g, st, fl in res[1:]:
+        for k in g:
+            assert np.array_equal(g[k], res[0][0][k]), k
+        assert np.array_equal(st["votes"], res[0][1]["votes"]) and np.array_equal(fl, res[0][2])
+        assert np.allclose(st["bw_sum"], res[0][1]["bw_sum"], rtol=1e-12)
+    # splitting the same ops into two windows leaves the vote totals unchanged
+    spec2 = tg.cfg2(reps=15, n_windows=2, tp=4, pp=2, dp=2)
+    o = orc.Oracle()
+    for cid, ranks, seq0 in tg.registry(spec2):
+        o.comm_register(cid, ranks, seq0)
+    for w in range(2):
+        win = tg.gen_window(spec2, w)
+        o.upload(w, win.cols)
+    o.analyze(0, 2, win.now_ns)
+    assert np.array_equal(o.rank_stats(spec.n_ranks)["votes"], res[0][1]["votes"])
+    assert np.array_equal(o.rank_stats(spec.n_ranks)["ops"], res[0][1]["ops"])
+
+
+def test_rejected_records_and_incomplete_groups():
+    recs = group_trace([[5, 5, 5, 5], [5, 5, 5, 5], [5, 5, 5, 5]], seq0=10)
+    recs = [r for r in recs if not (r["seq"] == 11 and r["rank"] == 2)]          # missing member
+    recs.append(dict(rank=0, comm=99, seq=10, t_enter=1, t_exit=2))              # unknown communicator
+    recs.append(dict(rank=77, comm=0, seq=10, t_enter=1, t_exit=2))              # not a member
+    recs.append(dict(rank=1, comm=0, seq=3, t_enter=1, t_exit=2))                # before seq0
+    o = run(recs, [(0, [0, 1, 2, 3], 10)])
+    s = o.sizes(0)
+    assert s["n_rejected"] == 3 and s["error_bits"] == 1 | 2 | 4
+    assert s["n_groups"] == 3 and s["n_complete"] == 2 and s["n_incomplete"] == 1
+    g = o.groups(0)
+    assert list(g["n_present"]) == [4, 3, 4] and (g["gflags"][1] & 2) and g["t_max"][1] == 0
+    flags, perm = o.slots(0)
+    assert flags[6] == (64 | 128) and perm[6] == 0xFFFFFFFF and flags[5] == 128
+
+
+def test_barrier_and_small_groups_are_not_analysed():
+    recs = group_trace([[5, 5, 5, 900]], comm=0, bytes=3)                        # allreduce < 4 B: barrier
+    recs += group_trace([[5, 5, 5, 900]], comm=1, ranks=[4, 5, 6, 7], bytes=4)   # exactly 4 B is not
+    recs += group_trace([[5, 5, 900]], comm=2, ranks=[8, 9, 10])                 # below min_group
+    recs += group_trace([[5, 5, 5, 900]], comm=3, ranks=[12, 13, 14, 15], op=ALLGATHER, bytes=3)
+    o = run(recs, [(0, [0, 1, 2, 3], 0), (1, [4, 5, 6, 7], 0), (2, [8, 9, 10], 0), (3, [12, 13, 14, 15], 0)])
+    g = o.groups(0)
+    assert [int(f) & (4 | 16) for f in g["gflags"]] == [4, 16, 0, 16]
+    flags, _ = o.slots(0)
+    assert list(flags) == [128] * 4 + [0, 0, 0, 2 | 8] + [128] * 3 + [0, 0, 0, 2 | 8]
+    assert o.sizes(0)["n_barrier"] == 1
+    assert len(o.comm_rows(0)["comm"]) == 4 and o.comm_rows(0)["n_rounds"][0] == 0
+
+
+def test_opset_mismatch():
+    recs = group_trace([[5, 5, 5, 5]] * 2)
+    recs[5]["bytes"] = 8 * MiB
+    o = run(recs, [(0, [0, 1, 2, 3], 0)])
+    assert [int(f) & 8 for f in o.groups(0)["gflags"]] == [0, 8]
+
+
+# ---------------------------------------------------------------- Eq. 1-4 and slow location
+MS = 1_000_000
+
+
+def test_eq1_baseline_mean_of_first_m_rounds():
+    # m_max_rounds = 3: baseline stays the configured value while r <= m, then floor(mean(Tmax of first 3))
+    durs = [[10, 1], [21, 2], [30, 3], [40, 4]]
+    p = dict(m_max_rounds=3, tbase_init_ns=1000, min_group=2)
+    o = run(group_trace(durs[:3]), [(0, [0, 1], 0)], params=p)
+    r = o.comm_rows(0)
+    assert r["baseline_static"][0] == 1 and r["t_base"][0] == 1000 and r["m"][0] == 0
+    o = run(group_trace(durs), [(0, [0, 1], 0)], params=p)
+    r = o.comm_rows(0)
+    assert r["baseline_static"][0] == 0 and r["m"][0] == 3 and r["t_base"][0] == (10 + 21 + 30) // 3 == 20
+    # same rounds split over two windows: the state carries over
+    o = run(None, [(0, [0, 1], 0)], params=p, windows=[group_trace(durs[:2]), group_trace(durs[2:], seq0=2)])
+    assert o.comm_rows(0)["baseline_static"][0] == 1
+    assert o.comm_rows(1)["t_base"][0] == 20 and o.comm_rows(1)["rounds_total"][0] == 4
+
+
+def test_eq1_two_minute_rule():
+    # rounds start 0 s, 50 s, 130 s after the first: only the first two fall inside 120 s
+    recs = []
+    for s, (t, d) in enumerate([(0, 10), (50 * 10**9, 13), (130 * 10**9, 99)]):
+        for rk in (0, 1):
+            recs.append(dict(rank=rk, comm=0, seq=s, t_enter=10**9 + t, t_exit=10**9 + t + d))
+    o = run(recs, [(0, [0, 1], 0)])
+    r = o.comm_rows(0)
+    assert r["m"][0] == 2 and r["t_base"][0] == (10 + 13) // 2 and r["baseline_static"][0] == 0
+
+
+def test_eq2_selects_round_with_largest_range_not_largest_time():
+    # ranges: 100-90=10, 60-10=50, 60-10=50 (tie -> earliest), 200-199=1
+    durs = [[100, 90, 95, 95], [60, 10, 30, 30], [10, 60, 30, 30], [200, 199, 199, 199]]
+    o = run(group_trace(durs), [(0, [0, 1, 2, 3], 0)], params=dict(tbase_init_ns=10))
+    r = o.comm_rows(0)
+    assert r["sel_seq"][0] == 1 and r["t_max"][0] == 60 and r["t_min"][0] == 10
+    assert r["R"][0] == pytest.approx((60 - 10) / 10) and r["slow_detected"][0] == 1
+    assert r["n_rounds"][0] == 4
+
+
+def test_eq3_threshold_strict():
+    # T_base = 1000: R = 3.0 exactly is not slow, R just above is
+    for tmax, want in ((4000, 0), (4001, 1)):
+        o = run(group_trace([[tmax, 1000, 1000, 1000]]), [(0, [0, 1, 2, 3], 0)], params=dict(tbase_init_ns=1000))
+        r = o.comm_rows(0)
+        assert r["slow_detected"][0] == want and r["R"][0] == pytest.approx((tmax - 1000) / 1000)
+
+
+def coupled(enter_off, own_dur, chg=None, seq=0):
+    """Collective semantics: nobody leaves before the last rank arrived: t_exit = max enter + own duration."""
+    last = max(enter_off)
+    return [dict(rank=i, comm=0, seq=seq, t_enter=10**9 + seq * 10**9 + e, t_exit=10**9 + seq * 10**9 + last + d,
+                 send_chg=(chg[i] if chg else 1), recv_chg=1) for i, (e, d) in enumerate(zip(enter_off, own_dur))]
+
+
+def test_eq4_limits_of_p_and_root_ranks():
+    lim = GOLD["p_limits"]
+    p = dict(tbase_init_ns=2 * MS)
+    comms = [(0, [0, 1, 2, 3], 0)]
+    # computation-slow: rank 2 arrives 20 ms late -> the others wait; T_min -> T_base, P -> 1; root = min-duration rank
+    o = run(coupled([0, 0, 20 * MS, 0], [2 * MS] * 4), comms, params=p)
+    r = o.comm_rows(0)
+    assert (r["t_max"][0], r["t_min"][0]) == (22 * MS, 2 * MS)
+    assert r["P"][0] == pytest.approx(lim["comp_slow"]) and r["cls"][0] == 1 and r["root_comp"][0] == 2
+    assert r["R"][0] == pytest.approx(10.0) and r["slow_detected"][0] == 1 and r["located"][0] == 0
+    # communication-slow: everyone takes 5x as long, T_min -> T_max, P -> 0; root = most observed count changes
+    o = run(coupled([0, 0, 0, 0], [10 * MS] * 4, chg=[2, 2, 2, 7]), comms, params=p)
+    r = o.comm_rows(0)
+    assert r["P"][0] == pytest.approx(lim["comm_slow"]) and r["cls"][0] == 2 and r["root_comm"][0] == 3 and r["rate_source"][0] == 0
+    # equal contributions: T_max 18, T_min 10, T_base 2 -> P = 0.5 -> mixed, both roots reported
+    o = run(coupled([0, 8 * MS, 0, 0], [10 * MS] * 4, chg=[9, 2, 2, 2]), comms, params=p)
+    r = o.comm_rows(0)
+    assert r["P"][0] == pytest.approx(lim["equal"]) and r["cls"][0] == 3
+    assert r["root_comp"][0] == 1 and r["root_comm"][0] == 0
+
+
+def test_alpha_beta_boundaries_are_strict():
+    # T_base 1000, T_max 11000 -> den = 10000. P = 0.6 exactly -> mixed; 0.6001 -> comp; 0.4 -> mixed; 0.3999 -> comm
+    for tmin, cls in ((5000, 3), (4999, 1), (7000, 3), (7001, 2)):
+        o = run(group_trace([[11000, tmin, 8000, 8000]]), [(0, [0, 1, 2, 3], 0)], params=dict(tbase_init_ns=1000))
+        assert o.comm_rows(0)["cls"][0] == cls, tmin
+
+
+def test_send_rate_worked_example_and_duration_proxy():
+    ex = GOLD["send_rate_example"]
+    chg = [ex["normal_changes"]] * 3 + [ex["slow_changes"]]
+    recs = coupled([0, 0, 0, 0], [10 * MS] * 4, chg=chg)
+    o = run(recs, [(0, [0, 1, 2, 3], 0)], params=dict(tbase_init_ns=2 * MS))
+    assert o.groups(0)["max_chg"][0] == 7 and o.comm_rows(0)["root_comm"][0] == 3     # rate 1/7 < 1/2
+    # without rate columns the longest-duration rank stands in
+    recs = group_trace([[10 * MS, 10 * MS, 12 * MS, 10 * MS]])
+    o = run(recs, [(0, [0, 1, 2, 3], 0)], params=dict(tbase_init_ns=2 * MS), with_rates=False)
+    r = o.comm_rows(0)
+    assert r["rate_source"][0] == 1 and r["root_comm"][0] == 2
+
+
+def test_repetition_counter_triggers_location_on_second_detection():
+    p = dict(tbase_init_ns=2 * MS)
+    w0 = coupled([0, 0, 20 * MS, 0], [2 * MS] * 4, seq=0)
+    w1 = coupled([0, 0, 0, 0], [2 * MS] * 4, seq=1)            # a healthy window in between
+    w2 = coupled([0, 20 * MS, 0, 0], [2 * MS] * 4, seq=2)
+    o = run(None, [(0, [0, 1, 2, 3], 0)], params=p, windows=[w0, w1, w2])
+    assert [int(o.comm_rows(w)["slow_detected"][0]) for w in range(3)] == [1, 0, 1]
+    assert [int(o.comm_rows(w)["located"][0]) for w in range(3)] == [0, 0, 1]
+    assert [int(o.comm_rows(w)["slow_count"][0]) for w in range(3)] == [1, 1, 2]
+    assert o.comm_rows(2)["root_comp"][0] == 1
+
+
+# ---------------------------------------------------------------- hang detection and location
+def hang_records(n, seq, entered, done, t_enter=10**9):
+    recs = []
+    for s in range(seq):
+        recs += [dict(rank=i, comm=0, seq=s, t_enter=1000 + s, t_exit=2000 + s) for i in range(n)]
+    for i in range(n):
+        if i in entered:
+            recs.append(dict(rank=i, comm=0, seq=seq, t_enter=t_enter, t_exit=(t_enter + 5 if i in done else -1)))
+    return recs
+
+
+def test_hang_alert_threshold_and_barrier_filter():
+    now = 10**9 + 300 * 10**9
+    for extra, bytes_, want in ((1, 16 * MiB, 1), (0, 16 * MiB, 0), (1, 3, 0)):
+        recs = hang_records(4, 2, {0, 1, 2, 3}, set())
+        for r in recs:
+            r["bytes"] = bytes_
+        o = run(recs, [(0, [0, 1, 2, 3], 0)], now=now + extra)
+        a = o.alerts(0)
+        assert len(a["seq"]) == want
+        if want:
+            assert a["seq"][0] == 2 and a["age_ns"][0] == 300 * 10**9 + 1
+
+
+def test_hang_tree_h1_not_entered():
+    o = run(hang_records(6, 3, {0, 1, 2, 4}, set()), [(0, list(range(6)), 0)])
+    h = o.locate_hang(0, 0, 3)
+    assert h["cls"] == 1 and list(h["roots"]) == [3, 5] and h["n_not_entered"] == 2
+
+
+def test_hang_tree_h2_non_hung_ranks():
+    o = run(hang_records(6, 3, set(range(6)), {2}), [(0, list(range(6)), 0)])
+    h = o.locate_hang(0, 0, 3)
+    assert h["cls"] == 2 and list(h["roots"]) == [2] and h["n_hung"] == 5 and h["n_not_hung"] == 1
+
+
+def test_hang_tree_h3_fewest_counts_and_ring_tie_break():
+    n, C = 6, 2
+    recs = hang_records(n, 3, set(range(n)), set())
+    ranks = [10, 11, 12, 13, 14, 15]
+    for r in recs:
+        r["rank"] = ranks[r["rank"]]
+    # unique minimum at ring position 4
+    fr = frames_from([(ranks[i], 0, 3, [(9, 9), (9, 8)] if i != 4 else [(9, 7), (8, 6)]) for i in range(n)], C)
+    o = run(recs, [(0, ranks, 0)], frames=fr, n_channels=C)
+    h = o.locate_hang(0, 0, 3)
+    assert h["cls"] == 3 and list(h["roots"]) == [14] and h["stuck_step"] == 6 and h["min_total"] == 30
+    # a run of equal minima at positions 5,0,1 (wrapping): the most upstream one (5) is the root
+    tot = {5: 4, 0: 4, 1: 4}
+    fr = frames_from([(ranks[i], 0, 3, [(tot.get(i, 6), tot.get(i, 6))] * C) for i in range(n)], C)
+    o = run(recs, [(0, ranks, 0)], frames=fr, n_channels=C)
+    assert list(o.locate_hang(0, 0, 3)["roots"]) == [15]
+    # all equal: lowest position; a missing frame counts as zero progress
+    fr = frames_from([(ranks[i], 0, 3, [(5, 5)] * C) for i in range(n)], C)
+    o = run(recs, [(0, ranks, 0)], frames=fr, n_channels=C)
+    assert list(o.locate_hang(0, 0, 3)["roots"]) == [10]
+    fr = frames_from([(ranks[i], 0, 3, [(5, 5)] * C) for i in range(n) if i != 2], C)
+    o = run(recs, [(0, ranks, 0)], frames=fr, n_channels=C)
+    h = o.locate_hang(0, 0, 3)
+    assert list(h["roots"]) == [12] and h["n_missing_frames"] == 1 and h["min_total"] == 0
+
+
+# ---------------------------------------------------------------- the benchmark configurations
+def test_cfg1_rank5_is_the_sole_suspect():
+    import tracegen as tg
+    spec = tg.cfg1()
+    o = orc.Oracle()
+    for cid, ranks, seq0 in tg.registry(spec):
+        o.comm_register(cid, ranks, seq0)
+    win = tg.gen_window(spec, 0)
+    o.upload(0, win.cols); o.analyze(0, 1, win.now_ns)
+    s = o.sizes(0)
+    assert s["n_records"] == 8000 and s["n_groups"] == 1000 and s["n_complete"] == 1000 and s["n_alerts"] == 0
+    sus = o.suspects()
+    assert sorted(set(sus["rank"])) == [5] and list(sus["kind"]) == [1]
+    st = o.rank_stats(8)
+    assert 250 <= st["votes"][5, 0] <= 350
+
+
+def test_cfg3_hang_root_1793_step_23():
+    import tracegen as tg
+    spec = tg.cfg3()
+    o = orc.Oracle()
+    for cid, ranks, seq0 in tg.registry(spec):
+        o.comm_register(cid, ranks, seq0)
+    win = tg.gen_window(spec, 0)
+    o.upload(0, win.cols, win.frames, win.n_channels); o.analyze(0, 1, win.now_ns)
+    a = o.alerts(0)
+    assert list(a["comm"]) == [7] and list(a["seq"]) == [100]
+    h = o.locate_hang(0, 7, 100)
+    assert h["cls"] == 3 and list(h["roots"]) == [1793] and h["stuck_step"] == 23
+    assert h["min_total"] == 16 * 2 * 23 and h["n_hung"] == 256
+    # a ring that completed: every rank is "not hung", which the tree reads as H2 with all ranks
+    assert o.locate_hang(0, 3, 100)["cls"] == 2
+
+
+def test_scaled_cfg2_and_cfg5_recover_injected_ranks():
+    import tracegen as tg
+    for spec in (tg.cfg2(reps=60, n_windows=2), tg.cfg5(reps=2, n_windows=2, nodes=64, mid=32, hang_window=1)):
+        o = orc.Oracle()
+        for cid, ranks, seq0 in tg.registry(spec):
+            o.comm_register(cid, ranks, seq0)
+        alerts = []
+        for w in range(spec.n_windows):
+            win = tg.gen_window(spec, w)
+            o.upload(w, win.cols, win.frames, win.n_channels); o.analyze(w, 1, win.now_ns)
+            a = o.alerts(w)
+            alerts += [(w, int(c), int(s)) for c, s in zip(a["comm"], a["seq"])]
+        sus = o.suspects()
+        strag = sorted(set(int(r) for r in sus["rank"][sus["kind"] == 1]))
+        slow = sorted(set(int(r) for r in sus["rank"][sus["kind"] == 2]))
+        assert strag == spec.truth["stragglers"], (spec.name, strag)
+        assert slow == spec.truth["slow_links"], (spec.name, slow)
+        if spec.hang is not None:
+            assert len(alerts) == 1
+            w, c, s = alerts[0]
+            h = o.locate_hang(w, c, s)
+            assert h["cls"] == 3 and list(h["roots"]) == spec.truth["hang_root"] and h["stuck_step"] == 41
