@@ -134,6 +134,13 @@ void analyze_one(Oracle& o, Window& w, i64 now) {
     auto ci = o.comm_idx.find(w.comm[i]);
     if (ci == o.comm_idx.end()) { w.err |= E_UNKNOWN_COMM; ++w.n_rejected; continue; }
     Comm& c = o.comms[ci->second];
+    // the op counters a communicator covers in this window: every record that names it with a
+    // counter at or above its first one, whether or not the reporting rank turns out to be a member
+    if (w.seq[i] >= c.seq0) {
+      auto it = w.range.find(ci->second);
+      if (it == w.range.end()) w.range[ci->second] = {w.seq[i], w.seq[i]};
+      else { it->second.first = std::min(it->second.first, w.seq[i]); it->second.second = std::max(it->second.second, w.seq[i]); }
+    }
     auto pi = c.pos.find(w.rank[i]);
     if (pi == c.pos.end()) { w.err |= E_NOT_MEMBER; ++w.n_rejected; continue; }
     if (w.seq[i] < c.seq0) { w.err |= E_SEQ_RANGE; ++w.n_rejected; continue; }
@@ -144,11 +151,6 @@ void analyze_one(Oracle& o, Window& w, i64 now) {
     if (a.s != b.s) return a.s < b.s;
     return a.pos < b.pos;
   });
-  for (const Key& k : keys) {
-    auto it = w.range.find(k.c);
-    if (it == w.range.end()) w.range[k.c] = {k.s, k.s};
-    else { it->second.first = std::min(it->second.first, k.s); it->second.second = std::max(it->second.second, k.s); }
-  }
   u64 n_slots = 0;
   for (auto& r : w.range) {
     u32 n = (u32)o.comms[r.first].ranks.size();
