@@ -1,0 +1,276 @@
+/*
+ * ccld.h - C ABI of the CCL-D decision-analyzer hot path on one NVIDIA B200 (sm_100a).
+ *
+ * The library analyses batches ("windows") of rank-level collective-communication trace records
+ * the way the paper's centralized Decision Analysis Module does (Sec. 3, Sec. 4.2): it groups the
+ * records by (communicator, operation counter) - the Trace ID of Sec. 5.1 -, reduces each group
+ * across its ranks, tests every rank against the group with a robust median/MAD rule, keeps
+ * per-rank anomaly votes, applies the slow-detection and slow-location rules of Eq. 1-4 per
+ * communicator and window, raises hang alerts (Sec. 4.2.1) and locates the root rank of a hang
+ * with the decision tree of Sec. 4.2.2 / Fig. 6 from per-channel SendCount/RecvCount counters.
+ *
+ * Conventions
+ *   - Every function returns CCLD_OK (0) or a negative CCLD_ERR_* code; nothing throws or aborts.
+ *     ccld_last_error() returns a text for the last failure on that context.
+ *   - All compute runs in CUDA kernels on the context's device and stream. There is no CPU
+ *     fallback: without a usable CUDA device ccld_create fails with CCLD_ERR_CUDA.
+ *   - "host" / "device" is stated for every pointer. Output structs are caller-allocated PODs;
+ *     variable-length lists have a caller-supplied capacity and a *_total count so truncation
+ *     is visible.
+ *   - Times are int64 nanoseconds; thresholds are integers in milli-units (x1000).
+ *   - A context is not thread-safe; use one per thread or lock around it.
+ */
+#ifndef CCLD_H
+#define CCLD_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ccld_ctx ccld_ctx; /* opaque, library-owned */
+
+enum {
+  CCLD_OK = 0,
+  CCLD_ERR_ARG = -1,          /* bad argument (null pointer, zero size, unsupported option) */
+  CCLD_ERR_NOMEM = -2,        /* host or device allocation failed */
+  CCLD_ERR_CUDA = -3,         /* a CUDA call failed; see ccld_last_error */
+  CCLD_ERR_UNKNOWN_COMM = -4, /* a record names a communicator that was never registered */
+  CCLD_ERR_NOT_MEMBER = -5,   /* a record's rank is not a member of its communicator */
+  CCLD_ERR_SEQ_RANGE = -6,    /* a record's op counter is below the communicator's first one */
+  CCLD_ERR_NO_WINDOW = -7,    /* unknown window id, or window not analysed yet */
+  CCLD_ERR_CAPACITY = -8,     /* a size limit of the library was exceeded */
+  CCLD_ERR_STATE = -9,        /* call order violated (e.g. window analysed twice) */
+  CCLD_ERR_DUPLICATE = -10    /* two records with the same (communicator, op counter, rank) */
+};
+
+/* Operation types (the collectives of Sec. 2.1 plus point-to-point and broadcast). */
+enum { CCLD_OP_ALLREDUCE = 0, CCLD_OP_ALLGATHER = 1, CCLD_OP_REDUCESCATTER = 2, CCLD_OP_ALLTOALL = 3,
+       CCLD_OP_SENDRECV = 4, CCLD_OP_BROADCAST = 5 };
+
+/* Per-slot flag byte (one per member of every group, in group-major order). */
+enum { CCLD_F_SKEW_OUT = 1, CCLD_F_DUR_OUT = 2, CCLD_F_SKEW_HI = 4, CCLD_F_DUR_HI = 8,
+       CCLD_F_MISSING = 64, CCLD_F_NOT_ANALYSED = 128 };
+
+/* Per-group flag word. */
+enum { CCLD_G_COMPLETE = 1, CCLD_G_INCOMPLETE = 2, CCLD_G_BARRIER = 4, CCLD_G_OPSET_MISMATCH = 8,
+       CCLD_G_ANALYSED = 16, CCLD_G_HANG_ALERT = 32, CCLD_G_INFLIGHT = 64, CCLD_G_BAD_TIME = 128 };
+
+/* Input error bits reported in ccld_verdict.error_bits. */
+enum { CCLD_E_UNKNOWN_COMM = 1, CCLD_E_NOT_MEMBER = 2, CCLD_E_SEQ_RANGE = 4, CCLD_E_DUPLICATE = 8,
+       CCLD_E_CAPACITY = 16 };
+
+/* Limits. */
+#define CCLD_MAX_COMM_SIZE 8192u          /* ranks per communicator */
+#define CCLD_MAX_RANK_ID (1u << 22)       /* rank ids must be below this */
+#define CCLD_MAX_ALERTS_PER_WINDOW 1024u  /* hang alerts kept per window (the total is counted) */
+
+/*
+ * Analysis parameters. Defaults (ccld_params_default) are the values the paper quotes:
+ * theta_slow close to 3 (Sec. 4.2.1), alpha = 0.4 and beta = 0.6 (Sec. 4.2.2), m = min(100 rounds,
+ * rounds of the first two minutes) (Sec. 4.2.1, Eq. 1), 5-minute hang threshold (Sec. 6.1),
+ * barrier = AllReduce of fewer than 4 bytes (Sec. 4.2.1). tbase_init_ns is the administrator's
+ * T_base^(init) of Eq. 1 and must be > 0. The remaining fields belong to the rank-level
+ * median/MAD test, for which the paper gives no values.
+ */
+typedef struct {
+  int64_t tbase_init_ns;       /* T_base^(init), Eq. 1 */
+  uint32_t theta_slow_milli;   /* slow iff (T_max - T_base) * 1000 > theta_slow_milli * T_base, Eq. 3 */
+  uint32_t alpha_milli;        /* P < alpha: communication-slow, Eq. 4 */
+  uint32_t beta_milli;         /* P > beta: computation-slow, Eq. 4 */
+  uint32_t m_max_rounds;       /* Eq. 1: at most this many rounds feed the baseline */
+  int64_t m_max_ns;            /* Eq. 1: ... and only rounds that start within this time of the first */
+  int64_t hang_ns;             /* hang alert iff now - t_enter > hang_ns for an in-flight record */
+  uint64_t barrier_bytes;      /* AllReduce with bytes < barrier_bytes is a barrier */
+  uint32_t slow_rep_threshold; /* location is triggered once the cumulative slow count exceeds this */
+  uint32_t k_milli;            /* outlier iff |x - med| * 1000 > k_milli * MAD */
+  uint32_t min_group;          /* groups with fewer ranks get no median/MAD test */
+  uint32_t vote_rep_milli;     /* rank is a suspect iff votes * 1000 >= vote_rep_milli * ops */
+} ccld_params;
+
+void ccld_params_default(ccld_params* p /* host, out */);
+
+/*
+ * Lifecycle. `device` is a CUDA ordinal, `cuda_stream` a cudaStream_t (NULL = default stream) on
+ * which every copy and kernel of this context is enqueued. The context owns all device memory it
+ * allocates and frees it in ccld_destroy.
+ */
+int ccld_create(ccld_ctx** out, const ccld_params* params /* host */, int device, void* cuda_stream);
+int ccld_destroy(ccld_ctx* ctx);
+const char* ccld_last_error(ccld_ctx* ctx);
+
+/*
+ * Communicator registration (the "domain initialization" of Sec. 2.1): `ranks` (host, n entries,
+ * copied) lists the members in ring order - position p sends to position p+1 mod n -, which the
+ * hang localizer uses. `algo` 0 = ring; 1 = tree is not supported yet (CCLD_ERR_ARG). `seq0` is
+ * the communicator's first operation counter. All communicators must be registered before the
+ * first ccld_analyze_window (later calls return CCLD_ERR_STATE). 1 <= n <= CCLD_MAX_COMM_SIZE.
+ */
+int ccld_comm_register(ccld_ctx* ctx, uint32_t comm, const uint32_t* ranks, uint32_t n, uint8_t algo, uint32_t seq0);
+
+/*
+ * Hands one window of trace records to the analyzer - what the rank probes push on kernel
+ * completion (Sec. 5.2, step 4). SoA columns of length n_rec, any record order:
+ *   rank, comm, seq   uint32   reporting rank, communicator id, operation counter (Trace ID, Sec. 5.1)
+ *   op                uint8    CCLD_OP_*
+ *   bytes             uint64   message size (Operation Type Set, Sec. 4.1.2)
+ *   t_enter, t_exit   int64    ns; t_exit = -1 marks an operation still in flight
+ *   send_chg,recv_chg uint32   observed SendCount/RecvCount value changes during the op, i.e.
+ *                              1/SendRate and 1/RecvRate of Sec. 4.1.2; both may be NULL
+ * Optional progress frames (n_frames may be 0): for frame f, rank f_rank[f] reports for op
+ * (f_comm[f], f_seq[f]) the counters progress[f][channel][0] = SendCount and [1] = RecvCount
+ * (Probing Frame body, Sec. 5.1), n_channels channels per frame.
+ * mem_kind 0: every pointer is host memory; the data is copied to the device with asynchronous
+ * copies on the context's stream. Pageable buffers may be reused when the call returns; pinned
+ * buffers must stay unchanged until the stream has passed the copies (any synchronizing call of
+ * this library, e.g. ccld_get_verdict, guarantees that).
+ * mem_kind 1: every pointer is device memory on the context's device, borrowed until
+ * ccld_window_release or ccld_destroy; the caller keeps it alive and unchanged.
+ * At most one (comm, seq, rank) record per window (else CCLD_E_DUPLICATE at the verdict).
+ * n_rec < 2^32 - 1. A window id may be uploaded once until released.
+ */
+int ccld_trace_upload(ccld_ctx* ctx, uint32_t window_id, uint64_t n_rec, int mem_kind,
+                      const uint32_t* rank, const uint32_t* comm, const uint32_t* seq, const uint8_t* op,
+                      const uint64_t* bytes, const int64_t* t_enter_ns, const int64_t* t_exit_ns,
+                      const uint32_t* send_chg, const uint32_t* recv_chg,
+                      uint32_t n_frames, const uint32_t* f_rank, const uint32_t* f_comm, const uint32_t* f_seq,
+                      uint32_t n_channels, const uint32_t* progress);
+
+/* Drops a window: its records (if copied) and its results. */
+int ccld_window_release(ccld_ctx* ctx, uint32_t window_id);
+
+/*
+ * Analyses windows first_window .. first_window + n_windows - 1 (all uploaded, none analysed yet),
+ * in that order: grouping by (communicator, op counter) (Sec. 4.2.1), per-op cross-rank
+ * reductions, median/MAD flags, votes, then per communicator the window rules of Eq. 1-4 whose
+ * state (baseline rounds, slow counter) carries from window to window. `now_ns` is the analyzer's
+ * clock for the hang test. Work is enqueued on the context's stream; the call returns after
+ * one short device round trip that sizes the result buffers.
+ * A window is refused (CCLD_E_CAPACITY in its verdict, nothing analysed) if the op counters seen
+ * in it would need more than 2 * n_rec + (sum of communicator sizes) slots.
+ */
+int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows, int64_t now_ns);
+
+/* Clears votes, per-communicator state and all window results (records stay uploaded). */
+int ccld_reset(ccld_ctx* ctx);
+
+/* One suspect rank: kind 1 = straggler (late arrivals), 2 = slow link (long durations). */
+typedef struct {
+  uint32_t kind, rank, votes, ops;
+  double mean_busbw; /* bytes/ns = GB/s, mean over the rank's complete non-barrier ops */
+} ccld_suspect;
+
+/* Slow detection / location of one communicator in one window (Sec. 4.2.1-4.2.2). */
+typedef struct {
+  uint32_t comm;            /* communicator id */
+  uint32_t n_rounds;        /* complete non-barrier rounds of this window */
+  uint32_t sel_seq;         /* round selected by Eq. 2 (0xFFFFFFFF if none) */
+  uint32_t cls;             /* 0 none, 1 computation-slow, 2 communication-slow, 3 mixed */
+  uint32_t slow_detected;   /* R > theta_slow, Eq. 3 */
+  uint32_t located;         /* slow_detected and the repetition counter exceeded its threshold */
+  uint32_t baseline_static; /* 1: T_base is still the configured value (slow-at-start) */
+  uint32_t rate_source;     /* 0: root_comm from the rate columns, 1: longest duration stands in */
+  uint32_t root_comp;       /* rank with minimal duration in the selected round (0xFFFFFFFF if not slow) */
+  uint32_t root_comm;       /* rank with minimal Send/Recv rate in the selected round */
+  uint64_t slow_count;      /* cumulative slow detections of this communicator */
+  uint64_t rounds_total;    /* rounds seen so far (r of Eq. 1) */
+  uint64_t m;               /* m of Eq. 1, 0 while not fixed */
+  int64_t t_max, t_min, t_base;
+  double R, P;              /* Eq. 3, Eq. 4 (P = 0 when not slow) */
+} ccld_comm_verdict;
+
+typedef struct {
+  uint32_t comm, seq;
+  int64_t age_ns; /* now - t_enter of the oldest in-flight member */
+} ccld_hang_alert;
+
+/*
+ * Result of one analysed window plus the cumulative suspect list. The caller sets the three
+ * pointers (host memory, may be NULL with capacity 0) and capacities; the library fills the
+ * rest. comm_rows are ordered by registration order of the communicators, alerts by
+ * (communicator registration order, seq), suspects by (kind, votes descending, rank).
+ */
+typedef struct {
+  uint64_t n_records, n_groups, n_slots, n_rejected, n_complete, n_incomplete, n_barrier, n_analysed,
+      n_flag_skew, n_flag_dur, n_opset_mismatch;
+  uint32_t error_bits; /* CCLD_E_* seen in this window */
+  uint32_t n_comm_rows_total, n_alerts_total, n_suspects_total;
+  ccld_comm_verdict* comm_rows; uint32_t comm_rows_cap;
+  ccld_hang_alert* alerts;      uint32_t alerts_cap;
+  ccld_suspect* suspects;       uint32_t suspects_cap;
+} ccld_verdict;
+
+/*
+ * Synchronizes the stream and returns the verdict of an analysed window. Returns CCLD_OK, or the
+ * CCLD_ERR_* that corresponds to the lowest set bit of error_bits (the struct is filled either way).
+ */
+int ccld_get_verdict(ccld_ctx* ctx, uint32_t window_id, ccld_verdict* out /* host */);
+
+/*
+ * Hang location (Sec. 4.2.2, Fig. 6) for op (comm, seq) as seen in window `window_id`:
+ *   H1 (cls 1): members with no record of an op counter >= seq - they never entered; roots = those.
+ *   H2 (cls 2): all entered, some members' record of `seq` is complete - roots = those non-hung ranks.
+ *   H3 (cls 3): all hung - root = the member with the fewest SendCount+RecvCount summed over channels;
+ *       among equal minima the one whose ring predecessor has made more progress, then the lowest
+ *       ring position. A member without a frame counts as zero progress.
+ * roots (host, caller-allocated, may be NULL) receives up to roots_cap rank ids in ring order.
+ * Synchronizes the stream.
+ */
+typedef struct {
+  uint32_t cls, n_roots_total, n_not_entered, n_hung, n_not_hung, n_missing_frames;
+  uint32_t stuck_step; /* H3: the root's smallest RecvCount over channels */
+  uint32_t n_members;
+  uint64_t min_total;  /* H3: the root's summed counters */
+  uint32_t* roots; uint32_t roots_cap;
+} ccld_hang_verdict;
+
+int ccld_locate_hang(ccld_ctx* ctx, uint32_t window_id, uint32_t comm, uint32_t seq, ccld_hang_verdict* out /* host */);
+
+/*
+ * Parity / inspection access to the per-op table of an analysed window. Device pointers, valid
+ * until the window is released or the context reset. Groups are ordered by (communicator
+ * registration order, seq); group g of communicator row r covers slots
+ * [slot0_r + (g - group0_r) * n_r, ... + n_r). Column semantics (complete groups; zeros otherwise):
+ *   e_min = min t_enter; arrival_skew = max (t_enter - e_min); t_max, t_min = max, min duration;
+ *   span = max t_exit - e_min; med_x and mad_x = lower median and lower-median absolute deviation of
+ *   skew and duration (analysed groups); rank_tmin, rank_tmax = ranks of min, max duration (ties:
+ *   lowest ring position); max_chg, rank_max_chg = most observed count changes and its rank;
+ *   busbw = bytes * f / span in bytes per ns with f = 2(n-1)/n allreduce, (n-1)/n allgather,
+ *   reducescatter, alltoall, 1 otherwise.
+ * perm[slot] = index of the record in the uploaded columns, 0xFFFFFFFF if the member is missing.
+ */
+typedef struct {
+  uint64_t n_groups, n_slots;
+  const int64_t *e_min, *arrival_skew, *t_max, *t_min, *span, *med_skew, *mad_skew, *med_dur, *mad_dur;
+  const uint32_t *rank_tmin, *rank_tmax, *max_chg, *rank_max_chg, *n_present, *gflags;
+  const double* busbw;
+  const uint8_t* flags;  /* [n_slots] */
+  const uint32_t* perm;  /* [n_slots] */
+} ccld_optable;
+
+int ccld_get_optable(ccld_ctx* ctx, uint32_t window_id, ccld_optable* out /* host struct, device pointers */);
+
+/* Per communicator of a window: which op counters it covers and where its groups and slots start. */
+typedef struct {
+  uint32_t comm, n, seq_lo, n_seq;
+  uint64_t group0, slot0;
+} ccld_comm_range;
+
+/* Copies up to cap rows (host, registration order, only communicators with records); returns the total in *n_total. Synchronizes. */
+int ccld_get_ranges(ccld_ctx* ctx, uint32_t window_id, ccld_comm_range* rows /* host */, uint32_t cap, uint32_t* n_total);
+
+/*
+ * Cumulative per-rank statistics for ranks [0, n_ranks): votes[r][4] = {skew high, skew low,
+ * duration high, duration low}, ops = analysed ops, bw_cnt and bw_sum = count and fp64 sum of the
+ * rank's per-op bus bandwidth. Host arrays, caller-allocated. Synchronizes.
+ */
+int ccld_get_rank_stats(ccld_ctx* ctx, uint32_t n_ranks, uint32_t* votes, uint32_t* ops, uint32_t* bw_cnt, double* bw_sum);
+
+/* Utility for inspection tools: synchronous copy of `bytes` bytes from device memory of this context to host memory. */
+int ccld_copy_to_host(ccld_ctx* ctx, void* dst_host, const void* src_device, uint64_t bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CCLD_H */

@@ -1,0 +1,107 @@
+// Device-side data layout shared by the kernels and the host API of libccld (sm_100a).
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+#include "../../include/ccld.h"
+
+namespace ccld {
+
+typedef int64_t i64;
+typedef uint64_t u64;
+typedef uint32_t u32;
+typedef uint8_t u8;
+typedef unsigned long long ull;
+
+constexpr u32 NONE = 0xFFFFFFFFu;
+constexpr u64 U64_MAX_ = ~0ull;
+
+// ---- launch geometry ----
+constexpr int REC_THREADS = 256;       // record-streaming kernels: threads per CTA
+constexpr int REC_PER_THREAD = 8;
+constexpr int REC_PER_CTA = REC_THREADS * REC_PER_THREAD;
+constexpr int SMALL_N = 8;             // communicators of up to 8 ranks: one thread per group
+constexpr int SMALL_SEQS = 256;        //   seqs (= threads) per tile
+constexpr int MID_N = 1024;            // up to 1024 ranks: shared-memory bitonic sort, several groups per CTA
+constexpr int MID_THREADS = 256;
+constexpr int MID_ELEMS = 2048;        //   padded records per tile
+constexpr int LARGE_THREADS = 1024;    // above: one CTA walks a few consecutive groups, radix select
+constexpr int LARGE_SEQS = 8;
+constexpr int LARGE_MAXP = CCLD_MAX_COMM_SIZE / LARGE_THREADS;
+
+struct Params {
+  i64 tbase_init_ns, m_max_ns, hang_ns;
+  u64 barrier_bytes;
+  u32 theta_slow_milli, alpha_milli, beta_milli, m_max_rounds, slow_rep_threshold, k_milli, min_group, vote_rep_milli;
+};
+
+// Eq. 1 state of one communicator, carried from window to window.
+struct CommState { u64 rounds; i64 t_first; i64 sum_m; u64 m; u64 slow_count; };
+
+// Registered communicators (immutable after the first analysis) and cumulative per-rank statistics.
+struct Registry {
+  u32 n_comms, hash_mask, n_ranks, pad;
+  const uint2* hash;        // open addressing: (communicator id, index), index NONE = empty
+  const u32* comm_id;       // [n_comms]
+  const u32* comm_n;        // [n_comms] members
+  const u32* comm_seq0;     // [n_comms]
+  const u64* comm_moff;     // [n_comms] offset of the member list in `members`
+  const u32* members;       // rank ids, ring order
+  const u32* rank_ptr;      // [n_ranks+1] CSR over (communicator index, position) pairs of a rank
+  const u32* ent_comm;
+  const u32* ent_pos;
+  CommState* state;         // [n_comms]
+  u32* votes;               // [n_ranks][4] skew hi, skew lo, dur hi, dur lo
+  u32* ops;                 // [n_ranks]
+  u32* bw_cnt;              // [n_ranks]
+  double* bw_sum;           // [n_ranks]
+};
+
+// Which op counters a communicator covers in a window and where its groups / slots start.
+struct RangeRow { u32 seq_lo, n_seq, row_idx, n; u64 group0, slot0; };
+
+enum { C_REJECTED = 0, C_COMPLETE, C_INCOMPLETE, C_BARRIER, C_ANALYSED, C_FLAG_SKEW, C_FLAG_DUR, C_MISMATCH,
+       C_PRESENT, C_ALERTS, C_ERR, C_INTERNAL, C_COUNT = 16 };
+enum { T_GROUPS = 0, T_SLOTS, T_TILES0, T_TILES1, T_TILES2, T_ROWS, T_FAILED, T_COUNT = 8 };
+
+struct Tile { u32 w, c, seq_off, count; };
+
+// One window of a batch: input columns, scratch and result pointers (all device memory).
+struct WinDesc {
+  const u32 *rank, *comm, *seq;
+  const u8* op;
+  const u64* bytes;
+  const i64 *t_enter, *t_exit;
+  const u32 *send_chg, *recv_chg;   // may be null
+  u64 n_rec;
+  u64 slot_cap;                      // plan fails the window if it would need more slots
+  u32 cta0, n_cta;                   // this window's CTAs in the record-streaming grids
+  u32 *rmin, *rmax;                  // [n_comms] op counter range seen
+  RangeRow* ranges;                  // [n_comms]
+  u64* totals;                       // [T_COUNT]
+  u64* counters;                     // [C_COUNT]
+  // sized after the plan:
+  u64 n_groups, n_slots;
+  u32* perm;                         // [n_slots]
+  u8* flags;                         // [n_slots]
+  i64* gi64;                         // [9][n_groups]
+  u32* gu32;                         // [6][n_groups]
+  double* gbw;                       // [n_groups]
+  ccld_comm_verdict* comm_rows;      // [n_rows]
+  ccld_hang_alert* alerts;           // [CCLD_MAX_ALERTS_PER_WINDOW]
+  u32 tile0[3];                      // first tile of this window in each class list
+  u32 pad;
+};
+
+enum { GI_E_MIN = 0, GI_ARRIVAL_SKEW, GI_T_MAX, GI_T_MIN, GI_SPAN, GI_MED_SKEW, GI_MAD_SKEW, GI_MED_DUR, GI_MAD_DUR, GI_COUNT };
+enum { GU_RANK_TMIN = 0, GU_RANK_TMAX, GU_MAX_CHG, GU_RANK_MAX_CHG, GU_N_PRESENT, GU_GFLAGS, GU_COUNT };
+
+__host__ __device__ inline u32 next_pow2(u32 n) { u32 p = 1; while (p < n) p <<= 1; return p; }
+__host__ __device__ inline u32 comm_class(u32 n) { return n <= SMALL_N ? 0u : (n <= MID_N ? 1u : 2u); }
+__host__ __device__ inline u32 mid_npad(u32 n) { u32 p = next_pow2(n); return p < 16 ? 16 : p; }
+__host__ __device__ inline u32 tile_seqs(u32 n) {
+  u32 c = comm_class(n);
+  return c == 0 ? SMALL_SEQS : (c == 1 ? MID_ELEMS / mid_npad(n) : (u32)LARGE_SEQS);
+}
+
+}  // namespace ccld

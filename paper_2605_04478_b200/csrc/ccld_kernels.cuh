@@ -1,0 +1,1153 @@
+// Kernels of the CCL-D analyzer hot path for sm_100a. Everything the analysis computes runs here;
+// the host side only sizes buffers and launches.
+//
+//   k_seq_range     group-by, part 1: op-counter range per (window, communicator)
+//   k_plan          group-by, part 2: closed-form slot layout (prefix sums over communicators),
+//                   and the work list for the reduction kernels
+//   k_slot_scatter  group-by, part 3: perm[slot] = record index
+//   k_reduce_small  per-op reductions + median/MAD + flags + votes, n <= 8 (thread per group)
+//   k_reduce_mid    same, 9 <= n <= 1024 (shared-memory bitonic sort, several groups per CTA)
+//   k_reduce_large  same, n > 1024 (one CTA per group, radix select)
+//   k_window_decide Eq. 1-4 per communicator and window, slow location
+//   k_hang_locate   hang decision tree over presence / completion / progress counters
+//   k_suspects, k_rank_sort_*  suspect list and ordered output lists
+#pragma once
+#include "ccld_device.cuh"
+
+namespace ccld {
+
+// ------------------------------------------------------------------------------------------------
+// small helpers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ u32 comm_lookup(const Registry& R, u32 id) {
+  u32 h = (id * 2654435761u) & R.hash_mask;
+  for (u32 probe = 0; probe <= R.hash_mask; ++probe) {
+    uint2 e = R.hash[h];
+    if (e.y == NONE) return NONE;
+    if (e.x == id) return e.y;
+    h = (h + 1) & R.hash_mask;
+  }
+  return NONE;
+}
+
+__device__ __forceinline__ u32 pos_lookup(const Registry& R, u32 rank, u32 c) {
+  if (rank >= R.n_ranks) return NONE;
+  u32 b = R.rank_ptr[rank], e = R.rank_ptr[rank + 1];
+  for (u32 i = b; i < e; ++i)
+    if (R.ent_comm[i] == c) return R.ent_pos[i];
+  return NONE;
+}
+
+__device__ __forceinline__ u32 find_window(const WinDesc* wd, u32 nw, u32 cta) {
+  u32 lo = 0, hi = nw - 1;
+  while (lo < hi) {
+    u32 mid = (lo + hi + 1) >> 1;
+    if (wd[mid].cta0 <= cta) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+// a * ka > b * kb in exact 128-bit arithmetic
+__device__ __forceinline__ bool mul_gt(u64 a, u32 ka, u64 b, u32 kb) {
+  u64 alo = a * ka, ahi = __umul64hi(a, (u64)ka);
+  u64 blo = b * kb, bhi = __umul64hi(b, (u64)kb);
+  return ahi > bhi || (ahi == bhi && alo > blo);
+}
+__device__ __forceinline__ bool mul_lt(u64 a, u32 ka, u64 b, u32 kb) { return mul_gt(b, kb, a, ka); }
+
+// bus-bandwidth factor num/den of an op over n ranks
+__device__ __forceinline__ void bus_factor(u32 op, u32 n, double* num, double* den) {
+  if (op == CCLD_OP_ALLREDUCE) { *num = 2.0 * (double)(n - 1); *den = (double)n; }
+  else if (op == CCLD_OP_ALLGATHER || op == CCLD_OP_REDUCESCATTER || op == CCLD_OP_ALLTOALL) { *num = (double)(n - 1); *den = (double)n; }
+  else { *num = 1.0; *den = 1.0; }
+}
+__device__ __forceinline__ double busbw(double bytes_num, double den, i64 t) {
+  return t > 0 ? bytes_num / ((double)t * den) : 0.0;
+}
+
+__device__ __forceinline__ u64 absdiff(u64 a, u64 b) { return a >= b ? a - b : b - a; }
+
+__device__ __forceinline__ u64 shfl_xor64(u64 v, int m) { return __shfl_xor_sync(0xFFFFFFFFu, v, m); }
+
+__device__ __forceinline__ void count_add(u64* counters, int which, u32 v) {
+  if (v) atomicAdd((ull*)&counters[which], (ull)v);
+}
+
+__device__ __forceinline__ void raise_alert(const WinDesc& D, u32 comm_id, u32 seq, i64 age) {
+  ull k = atomicAdd((ull*)&D.counters[C_ALERTS], 1ull);
+  if (k < CCLD_MAX_ALERTS_PER_WINDOW) { ccld_hang_alert a; a.comm = comm_id; a.seq = seq; a.age_ns = age; D.alerts[k] = a; }
+}
+
+// ------------------------------------------------------------------------------------------------
+// group-by, part 1: which op counters does every communicator cover in every window
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __restrict__ wd, u32 nw, Registry R) {
+  const u32 w = find_window(wd, nw, blockIdx.x);
+  const WinDesc& D = wd[w];
+  const u64 base = (u64)(blockIdx.x - D.cta0) * REC_PER_CTA;
+  const u32 lane = threadIdx.x & 31;
+#pragma unroll
+  for (int k = 0; k < REC_PER_THREAD; ++k) {
+    const u64 i = base + (u64)k * REC_THREADS + threadIdx.x;
+    const bool in = i < D.n_rec;
+    const u32 cid = in ? D.comm[i] : 0u;
+    const u32 s = in ? D.seq[i] : 0u;
+    const u32 c = in ? comm_lookup(R, cid) : NONE;
+    const bool valid = c != NONE && s >= R.comm_seq0[c];
+    // one pair of atomics per distinct communicator in the warp, and only when it widens the range
+    const u32 m = __match_any_sync(0xFFFFFFFFu, valid ? c : NONE);
+    const u32 mn = __reduce_min_sync(m, s), mx = __reduce_max_sync(m, s);
+    if (valid && lane == (u32)(__ffs(m) - 1)) {
+      if (mn < D.rmin[c]) atomicMin(&D.rmin[c], mn);
+      if (mx > D.rmax[c]) atomicMax(&D.rmax[c], mx);
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// group-by, part 2: closed-form layout. One CTA per window scans the communicators.
+//   slot(comm, seq, pos) = slot0[comm] + (seq - seq_lo[comm]) * n[comm] + pos
+// ------------------------------------------------------------------------------------------------
+struct PlanAcc { u64 groups, slots; u32 rows, t0, t1, t2; };
+
+__device__ __forceinline__ PlanAcc plan_add(const PlanAcc& a, const PlanAcc& b) {
+  PlanAcc r; r.groups = a.groups + b.groups; r.slots = a.slots + b.slots; r.rows = a.rows + b.rows;
+  r.t0 = a.t0 + b.t0; r.t1 = a.t1 + b.t1; r.t2 = a.t2 + b.t2; return r;
+}
+__device__ __forceinline__ PlanAcc plan_shfl_up(const PlanAcc& a, int d) {
+  PlanAcc r;
+  r.groups = __shfl_up_sync(0xFFFFFFFFu, a.groups, d); r.slots = __shfl_up_sync(0xFFFFFFFFu, a.slots, d);
+  r.rows = __shfl_up_sync(0xFFFFFFFFu, a.rows, d); r.t0 = __shfl_up_sync(0xFFFFFFFFu, a.t0, d);
+  r.t1 = __shfl_up_sync(0xFFFFFFFFu, a.t1, d); r.t2 = __shfl_up_sync(0xFFFFFFFFu, a.t2, d);
+  return r;
+}
+
+__device__ __forceinline__ PlanAcc plan_item(const WinDesc& D, const Registry& R, u32 c) {
+  PlanAcc a = {0, 0, 0, 0, 0, 0};
+  if (c < R.n_comms) {
+    u32 lo = D.rmin[c], hi = D.rmax[c];
+    if (lo <= hi && lo != NONE) {
+      u64 ns = (u64)hi - lo + 1; u32 n = R.comm_n[c];
+      a.groups = ns; a.slots = ns * n; a.rows = 1;
+      u64 tiles = (ns + tile_seqs(n) - 1) / tile_seqs(n);
+      u32 t = tiles > 0x7FFFFFFFull ? 0x7FFFFFFFu : (u32)tiles;
+      u32 cls = comm_class(n);
+      a.t0 = cls == 0 ? t : 0; a.t1 = cls == 1 ? t : 0; a.t2 = cls == 2 ? t : 0;
+    }
+  }
+  return a;
+}
+
+// Exclusive prefix of `v` over the CTA's threads plus the CTA total, for PLAN_THREADS = 1024.
+constexpr int PLAN_THREADS = 1024;
+__device__ PlanAcc plan_block_scan(PlanAcc v, PlanAcc* total, PlanAcc* s_warp /*[33]*/) {
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  PlanAcc inc = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) { PlanAcc o = plan_shfl_up(inc, d); if (lane >= (u32)d) inc = plan_add(inc, o); }
+  if (lane == 31) s_warp[wid] = inc;
+  __syncthreads();
+  if (wid == 0) {
+    PlanAcc x = s_warp[lane], xi = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) { PlanAcc o = plan_shfl_up(xi, d); if (lane >= (u32)d) xi = plan_add(xi, o); }
+    PlanAcc ex = plan_shfl_up(xi, 1);
+    if (lane == 0) ex = PlanAcc{0, 0, 0, 0, 0, 0};
+    s_warp[lane] = ex;
+    if (lane == 31) s_warp[32] = xi;
+  }
+  __syncthreads();
+  PlanAcc ex = plan_shfl_up(inc, 1);
+  if (lane == 0) ex = PlanAcc{0, 0, 0, 0, 0, 0};
+  PlanAcc r = plan_add(s_warp[wid], ex);
+  *total = s_warp[32];
+  __syncthreads();
+  return r;
+}
+
+// emit == 0: write ranges and totals (and fail the window if it needs more than slot_cap slots).
+// emit == 1: write the tile lists (tile0[] filled by the host from the totals).
+__global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd, Registry R, Tile* __restrict__ tiles0,
+                                                       Tile* __restrict__ tiles1, Tile* __restrict__ tiles2, int emit) {
+  __shared__ PlanAcc s_warp[33];
+  __shared__ int s_failed;
+  WinDesc& D = wd[blockIdx.x];
+  if (emit && D.totals[T_FAILED]) return;
+  PlanAcc run = {0, 0, 0, 0, 0, 0};
+  for (u32 c0 = 0; c0 < R.n_comms; c0 += PLAN_THREADS) {
+    const u32 c = c0 + threadIdx.x;
+    PlanAcc it = plan_item(D, R, c), tot;
+    PlanAcc ex = plan_add(run, plan_block_scan(it, &tot, s_warp));
+    if (c < R.n_comms) {
+      if (!emit) {
+        RangeRow r;
+        r.seq_lo = it.rows ? D.rmin[c] : 0; r.n_seq = (u32)it.groups; r.row_idx = ex.rows; r.n = R.comm_n[c];
+        r.group0 = ex.groups; r.slot0 = ex.slots;
+        D.ranges[c] = r;
+      } else if (it.rows) {
+        const u32 n = R.comm_n[c], S = tile_seqs(n), cls = comm_class(n);
+        Tile* dst = cls == 0 ? tiles0 + D.tile0[0] + ex.t0 : (cls == 1 ? tiles1 + D.tile0[1] + ex.t1 : tiles2 + D.tile0[2] + ex.t2);
+        const u32 nt = it.t0 + it.t1 + it.t2;
+        for (u32 k = 0; k < nt; ++k) {
+          Tile t; t.w = blockIdx.x; t.c = c; t.seq_off = k * S;
+          u64 left = it.groups - (u64)k * S; t.count = left < S ? (u32)left : S;
+          dst[k] = t;
+        }
+      }
+    }
+    run = plan_add(run, tot);
+  }
+  if (emit) return;
+  if (threadIdx.x == 0) {
+    // op counters further apart than 2^31, or more slots than the cap: refuse the window
+    int failed = run.slots > D.slot_cap || run.groups > 0x7FFFFFFFull;
+    s_failed = failed;
+    D.totals[T_GROUPS] = failed ? 0 : run.groups; D.totals[T_SLOTS] = failed ? 0 : run.slots;
+    D.totals[T_TILES0] = failed ? 0 : run.t0; D.totals[T_TILES1] = failed ? 0 : run.t1; D.totals[T_TILES2] = failed ? 0 : run.t2;
+    D.totals[T_ROWS] = failed ? 0 : run.rows; D.totals[T_FAILED] = failed;
+    if (failed) atomicOr((unsigned*)&D.counters[C_ERR], (unsigned)CCLD_E_CAPACITY);
+  }
+  __syncthreads();
+  if (s_failed)
+    for (u32 c = threadIdx.x; c < R.n_comms; c += PLAN_THREADS) { RangeRow z = {0, 0, 0, R.comm_n[c], 0, 0}; D.ranges[c] = z; }
+}
+
+// ------------------------------------------------------------------------------------------------
+// group-by, part 3: every accepted record drops its index into its slot
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(REC_THREADS) k_slot_scatter(const WinDesc* __restrict__ wd, u32 nw, Registry R) {
+  const u32 w = find_window(wd, nw, blockIdx.x);
+  const WinDesc& D = wd[w];
+  const u64 base = (u64)(blockIdx.x - D.cta0) * REC_PER_CTA;
+  u32 err = 0, rej = 0, internal = 0;
+#pragma unroll
+  for (int k = 0; k < REC_PER_THREAD; ++k) {
+    const u64 i = base + (u64)k * REC_THREADS + threadIdx.x;
+    if (i >= D.n_rec) continue;
+    const u32 rk = D.rank[i], cid = D.comm[i], s = D.seq[i];
+    const u32 c = comm_lookup(R, cid);
+    if (c == NONE) { err |= CCLD_E_UNKNOWN_COMM; ++rej; continue; }
+    const u32 pos = pos_lookup(R, rk, c);
+    if (pos == NONE) { err |= CCLD_E_NOT_MEMBER; ++rej; continue; }
+    if (s < R.comm_seq0[c]) { err |= CCLD_E_SEQ_RANGE; ++rej; continue; }
+    const RangeRow r = D.ranges[c];
+    if (r.n_seq == 0) continue;                          // window refused by the plan
+    const u64 slot = r.slot0 + (u64)(s - r.seq_lo) * r.n + pos;
+    if (s < r.seq_lo || slot >= D.n_slots) { internal = 1; continue; }
+    D.perm[slot] = (u32)i;
+  }
+  err = __reduce_or_sync(0xFFFFFFFFu, err);
+  rej = __reduce_add_sync(0xFFFFFFFFu, rej);
+  internal = __reduce_or_sync(0xFFFFFFFFu, internal);
+  if ((threadIdx.x & 31) == 0) {
+    if (err) atomicOr((unsigned*)&D.counters[C_ERR], err);
+    count_add(D.counters, C_REJECTED, rej);
+    if (internal) atomicOr((unsigned*)&D.counters[C_INTERNAL], 1u);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// per-op reductions, n <= 8: one thread per group, lanes run along consecutive op counters so the
+// gathers of one member's records coalesce
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void cswap(u64& a, u64& b) { u64 lo = a < b ? a : b; u64 hi = a < b ? b : a; a = lo; b = hi; }
+
+// 19-exchange sorting network for 8 keys
+__device__ __forceinline__ void sort8(u64 (&v)[8]) {
+  cswap(v[0], v[2]); cswap(v[1], v[3]); cswap(v[4], v[6]); cswap(v[5], v[7]);
+  cswap(v[0], v[4]); cswap(v[1], v[5]); cswap(v[2], v[6]); cswap(v[3], v[7]);
+  cswap(v[0], v[1]); cswap(v[2], v[3]); cswap(v[4], v[5]); cswap(v[6], v[7]);
+  cswap(v[2], v[4]); cswap(v[3], v[5]);
+  cswap(v[1], v[4]); cswap(v[3], v[6]);
+  cswap(v[1], v[2]); cswap(v[3], v[4]); cswap(v[5], v[6]);
+}
+// bitonic merge: sorts 8 keys that first fall and then rise
+__device__ __forceinline__ void merge8(u64 (&v)[8]) {
+  cswap(v[0], v[4]); cswap(v[1], v[5]); cswap(v[2], v[6]); cswap(v[3], v[7]);
+  cswap(v[0], v[2]); cswap(v[1], v[3]); cswap(v[4], v[6]); cswap(v[5], v[7]);
+  cswap(v[0], v[1]); cswap(v[2], v[3]); cswap(v[4], v[5]); cswap(v[6], v[7]);
+}
+__device__ __forceinline__ u64 pick4(const u64 (&v)[8], u32 k) {
+  u64 r = v[0];
+  r = k == 1 ? v[1] : r; r = k == 2 ? v[2] : r; r = k == 3 ? v[3] : r;
+  return r;
+}
+
+// lower median and lower-median absolute deviation of x[0..n), n <= 8 (x[p] = U64_MAX for p >= n)
+__device__ __forceinline__ void median_mad8(const u64 (&x)[8], u32 n, u64* med, u64* mad) {
+  u64 s[8];
+#pragma unroll
+  for (int p = 0; p < 8; ++p) s[p] = x[p];
+  sort8(s);
+  const u32 k = (n - 1) >> 1;
+  const u64 m = pick4(s, k);
+#pragma unroll
+  for (int p = 0; p < 8; ++p) s[p] = (u32)p < n ? absdiff(s[p], m) : U64_MAX_;   // falls to 0 at k, then rises
+  merge8(s);
+  *med = m; *mad = pick4(s, k);
+}
+
+__global__ void __launch_bounds__(SMALL_SEQS) k_reduce_small(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles,
+                                                              Registry R, Params P, i64 now) {
+  __shared__ double s_bw[SMALL_SEQS / 32][SMALL_N];
+  const Tile t = tiles[blockIdx.x];
+  const WinDesc& D = wd[t.w];
+  const u32 c = t.c, n = R.comm_n[c];
+  const RangeRow row = D.ranges[c];
+  const u32* mem = R.members + R.comm_moff[c];
+  const u32 j = threadIdx.x;
+  const bool active = j < t.count;
+
+  double bw[SMALL_N];
+#pragma unroll
+  for (int p = 0; p < SMALL_N; ++p) bw[p] = 0.0;
+  bool complete = false, barrier = false, analysed = false, mismatch = false;
+  u32 n_present = 0, n_fs = 0, n_fd = 0;
+
+  if (active) {
+    const u64 g = row.group0 + t.seq_off + j;
+    const u64 slot = row.slot0 + (u64)(t.seq_off + j) * n;
+    u64 te[SMALL_N], du[SMALL_N];
+    i64 x_max = INT64_MIN, age = -1;
+    u64 gbytes = 0; u32 gop = 0; bool have_first = false, inflight = false, bad_time = false;
+    u32 max_chg = 0, pos_chg = 0; bool have_chg = false;
+    complete = true;
+#pragma unroll
+    for (int p = 0; p < SMALL_N; ++p) {
+      te[p] = U64_MAX_; du[p] = U64_MAX_;
+      if ((u32)p < n) {
+        const u32 idx = D.perm[slot + p];
+        if (idx == NONE) { complete = false; }
+        else {
+          ++n_present;
+          const i64 a = D.t_enter[idx], b = D.t_exit[idx];
+          const u64 by = D.bytes[idx]; const u32 o = D.op[idx];
+          u32 ch = 0;
+          if (D.send_chg != nullptr) { const u32 sc = D.send_chg[idx], rc = D.recv_chg[idx]; ch = sc > rc ? sc : rc; }
+          if (!have_first) { gbytes = by; gop = o; have_first = true; }
+          else if (o != gop || by != gbytes) mismatch = true;
+          if (b == -1) { inflight = true; complete = false; const i64 ag = now - a; age = ag > age ? ag : age; }
+          else if (a < 0 || b < a) { bad_time = true; complete = false; }
+          te[p] = (u64)a; du[p] = (u64)(b - a);
+          x_max = b > x_max ? b : x_max;
+          if (!have_chg || ch > max_chg) { max_chg = ch; pos_chg = p; have_chg = true; }
+        }
+      }
+    }
+    barrier = have_first && gop == CCLD_OP_ALLREDUCE && gbytes < P.barrier_bytes;
+    u32 gfl = (mismatch ? CCLD_G_OPSET_MISMATCH : 0) | (barrier ? CCLD_G_BARRIER : 0) | (inflight ? CCLD_G_INFLIGHT : 0) |
+              (bad_time ? CCLD_G_BAD_TIME : 0);
+    i64 out_i[GI_COUNT];
+#pragma unroll
+    for (int q = 0; q < GI_COUNT; ++q) out_i[q] = 0;
+    u32 r_tmin = 0, r_tmax = 0, r_chg = 0; double gbw = 0.0;
+    u8 fl[SMALL_N];
+#pragma unroll
+    for (int p = 0; p < SMALL_N; ++p) fl[p] = CCLD_F_NOT_ANALYSED;
+
+    if (!complete) {
+      gfl |= CCLD_G_INCOMPLETE;
+      max_chg = 0;
+      if (inflight && age > P.hang_ns && !barrier) { gfl |= CCLD_G_HANG_ALERT; raise_alert(D, R.comm_id[c], row.seq_lo + t.seq_off + j, age); }
+#pragma unroll
+      for (int p = 0; p < SMALL_N; ++p)
+        if ((u32)p < n && D.perm[slot + p] == NONE) fl[p] = CCLD_F_NOT_ANALYSED | CCLD_F_MISSING;
+    } else {
+      gfl |= CCLD_G_COMPLETE;
+      u64 e_min = U64_MAX_, tmax = 0, tmin = U64_MAX_; u32 pmax = 0, pmin = 0;
+#pragma unroll
+      for (int p = 0; p < SMALL_N; ++p) if ((u32)p < n) { e_min = te[p] < e_min ? te[p] : e_min; }
+      u64 sk[SMALL_N], askew = 0;
+#pragma unroll
+      for (int p = 0; p < SMALL_N; ++p) {
+        sk[p] = U64_MAX_;
+        if ((u32)p < n) {
+          sk[p] = te[p] - e_min; askew = sk[p] > askew ? sk[p] : askew;
+          if (p == 0 || du[p] > tmax) { tmax = du[p]; pmax = p; }
+          if (p == 0 || du[p] < tmin) { tmin = du[p]; pmin = p; }
+        }
+      }
+      const i64 span = x_max - (i64)e_min;
+      double num, den; bus_factor(gop, n, &num, &den);
+      const double bn = (double)gbytes * num;
+      gbw = busbw(bn, den, span);
+      out_i[GI_E_MIN] = (i64)e_min; out_i[GI_ARRIVAL_SKEW] = (i64)askew; out_i[GI_T_MAX] = (i64)tmax; out_i[GI_T_MIN] = (i64)tmin;
+      out_i[GI_SPAN] = span;
+      r_tmin = mem[pmin]; r_tmax = mem[pmax]; r_chg = mem[pos_chg];
+      if (!barrier) {
+#pragma unroll
+        for (int p = 0; p < SMALL_N; ++p) if ((u32)p < n) bw[p] = busbw(bn, den, (i64)du[p]);
+      }
+      analysed = !barrier && n >= P.min_group;
+      if (analysed) {
+        gfl |= CCLD_G_ANALYSED;
+        u64 med_s, mad_s, med_d, mad_d;
+        median_mad8(sk, n, &med_s, &mad_s);
+        median_mad8(du, n, &med_d, &mad_d);
+        out_i[GI_MED_SKEW] = (i64)med_s; out_i[GI_MAD_SKEW] = (i64)mad_s; out_i[GI_MED_DUR] = (i64)med_d; out_i[GI_MAD_DUR] = (i64)mad_d;
+#pragma unroll
+        for (int p = 0; p < SMALL_N; ++p) {
+          if ((u32)p < n) {
+            const bool so = mul_gt(absdiff(sk[p], med_s), 1000u, mad_s, P.k_milli), sh = sk[p] > med_s;
+            const bool dq = mul_gt(absdiff(du[p], med_d), 1000u, mad_d, P.k_milli), dh = du[p] > med_d;
+            fl[p] = (so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0);
+            if (so) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p] * 4 + (sh ? 0 : 1)], 1u); }
+            if (dq) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p] * 4 + (dh ? 2 : 3)], 1u); }
+          }
+        }
+      }
+    }
+    // ---- outputs ----
+    const u64 G = D.n_groups;
+#pragma unroll
+    for (int q = 0; q < GI_COUNT; ++q) D.gi64[(u64)q * G + g] = out_i[q];
+    D.gu32[(u64)GU_RANK_TMIN * G + g] = r_tmin; D.gu32[(u64)GU_RANK_TMAX * G + g] = r_tmax;
+    D.gu32[(u64)GU_MAX_CHG * G + g] = max_chg; D.gu32[(u64)GU_RANK_MAX_CHG * G + g] = r_chg;
+    D.gu32[(u64)GU_N_PRESENT * G + g] = n_present; D.gu32[(u64)GU_GFLAGS * G + g] = gfl;
+    D.gbw[g] = gbw;
+#pragma unroll
+    for (int p = 0; p < SMALL_N; ++p) if ((u32)p < n) D.flags[slot + p] = fl[p];
+  }
+
+  // ---- per-tile accumulation: counters and the per-rank bandwidth sums ----
+  const u32 n_comp = __syncthreads_count(active && complete);
+  const u32 n_inc = __syncthreads_count(active && !complete);
+  const u32 n_bar = __syncthreads_count(active && barrier);
+  const u32 n_an = __syncthreads_count(active && analysed);
+  const u32 n_mis = __syncthreads_count(active && mismatch);
+  const u32 n_bwc = __syncthreads_count(active && complete && !barrier);
+  u32 pres = __reduce_add_sync(0xFFFFFFFFu, n_present), fs = __reduce_add_sync(0xFFFFFFFFu, n_fs), fd = __reduce_add_sync(0xFFFFFFFFu, n_fd);
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+  for (int p = 0; p < SMALL_N; ++p) {
+    double v = bw[p];
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, d);
+    if (lane == 0) s_bw[wid][p] = v;
+  }
+  if (lane == 0) { count_add(D.counters, C_PRESENT, pres); count_add(D.counters, C_FLAG_SKEW, fs); count_add(D.counters, C_FLAG_DUR, fd); }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    count_add(D.counters, C_COMPLETE, n_comp); count_add(D.counters, C_INCOMPLETE, n_inc); count_add(D.counters, C_BARRIER, n_bar);
+    count_add(D.counters, C_ANALYSED, n_an); count_add(D.counters, C_MISMATCH, n_mis);
+  }
+  if (threadIdx.x < n && n_bwc) {
+    double v = 0.0;
+#pragma unroll
+    for (int q = 0; q < SMALL_SEQS / 32; ++q) v += s_bw[q][threadIdx.x];
+    atomicAdd(&R.bw_sum[mem[threadIdx.x]], v);
+    atomicAdd(&R.bw_cnt[mem[threadIdx.x]], n_bwc);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// per-op reductions, 9 <= n <= 1024: a tile of S groups is staged in shared memory ([group][member],
+// pitch n_pad + 1), reduced by one warp per group, sorted by a bitonic network over all groups at once
+// ------------------------------------------------------------------------------------------------
+struct MidGroup {
+  u64 e_min, gbytes, med_s, mad_s, med_d, mad_d;
+  u32 gfl, gop;
+  u32 complete, analysed;
+};
+
+// Sort phase: full bitonic sort (merge_only = false) or only the final merge of a sequence that
+// falls and then rises (merge_only = true); every group of the tile in parallel.
+__device__ void mid_bitonic(u64* key, u32 S, u32 n_pad, u32 pitch, bool merge_only) {
+  const u32 half = n_pad >> 1, lg_half = 31 - __clz(half);
+  const u32 total = S * half;
+  for (u32 k = merge_only ? n_pad : 2; k <= n_pad; k <<= 1) {
+    for (u32 jj = k >> 1; jj > 0; jj >>= 1) {
+      for (u32 e = threadIdx.x; e < total; e += MID_THREADS) {
+        const u32 grp = e >> lg_half, q = e & (half - 1);
+        const u32 i = ((q & ~(jj - 1)) << 1) | (q & (jj - 1)), l = i | jj;
+        const bool up = (i & k) == 0 || k == n_pad;
+        u64* a = key + grp * pitch + i; u64* b = key + grp * pitch + l;
+        const u64 va = *a, vb = *b;
+        if ((va > vb) == up) { *a = vb; *b = va; }
+      }
+      __syncthreads();
+    }
+  }
+}
+
+__global__ void __launch_bounds__(MID_THREADS) k_reduce_mid(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles,
+                                                            Registry R, Params P, i64 now) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const Tile t = tiles[blockIdx.x];
+  const WinDesc& D = wd[t.w];
+  const u32 c = t.c, n = R.comm_n[c];
+  const RangeRow row = D.ranges[c];
+  const u32* mem = R.members + R.comm_moff[c];
+  const u32 n_pad = mid_npad(n), pitch = n_pad + 1, S = t.count, S_max = MID_ELEMS / n_pad;
+  const u32 cap = S_max * pitch;
+  // shared-memory carve-up
+  u64* s_te = (u64*)smem_raw;            // enter time
+  u64* s_du = s_te + cap;                // duration
+  u64* s_key = s_du + cap;               // sort buffer
+  u64* s_by = s_key + cap;               // bytes
+  u32* s_idx = (u32*)(s_by + cap);       // record index
+  u32* s_ch = s_idx + cap;               // max(send_chg, recv_chg)
+  u8* s_op = (u8*)(s_ch + cap);
+  u8* s_st = s_op + cap;                 // 1 present, 2 in flight, 4 bad time
+  MidGroup* s_g = (MidGroup*)(((uintptr_t)(s_st + cap) + 15) & ~(uintptr_t)15);
+  __shared__ u32 s_cnt[8];
+
+  const u64 slot_t = row.slot0 + (u64)t.seq_off * n;      // first slot of the tile
+  const u64 g_t = row.group0 + t.seq_off;                  // first group of the tile
+  const u32 n_el = S * n;
+  if (threadIdx.x < 8) s_cnt[threadIdx.x] = 0;
+  // 1. record indices, coalesced along the slot order
+  for (u32 e = threadIdx.x; e < n_el; e += MID_THREADS) { const u32 jg = e / n, p = e - jg * n; s_idx[jg * pitch + p] = D.perm[slot_t + e]; }
+  __syncthreads();
+  // 2. gather: consecutive threads walk consecutive op counters of one member
+  for (u32 e = threadIdx.x; e < n_el; e += MID_THREADS) {
+    const u32 p = e / S, jg = e - p * S, a = jg * pitch + p;
+    const u32 idx = s_idx[a];
+    u64 te = 0, du = 0, by = 0; u32 ch = 0; u8 op = 0, st = 0;
+    if (idx != NONE) {
+      const i64 x = D.t_enter[idx], y = D.t_exit[idx];
+      by = D.bytes[idx]; op = D.op[idx];
+      if (D.send_chg != nullptr) { const u32 sc = D.send_chg[idx], rc = D.recv_chg[idx]; ch = sc > rc ? sc : rc; }
+      st = 1 | (y == -1 ? 2 : ((x < 0 || y < x) ? 4 : 0));
+      te = (u64)x; du = (u64)(y - x);
+    }
+    s_te[a] = te; s_du[a] = du; s_by[a] = by; s_ch[a] = ch; s_op[a] = op; s_st[a] = st;
+  }
+  __syncthreads();
+  // 3. one warp per group: cross-rank reductions
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  u32 c_comp = 0, c_inc = 0, c_bar = 0, c_an = 0, c_mis = 0, c_pres = 0;
+  for (u32 jg = wid; jg < S; jg += MID_THREADS / 32) {
+    const u32 b = jg * pitch;
+    u32 npres = 0, first = NONE, stor = 0;
+    for (u32 p = lane; p < n; p += 32) { const u32 st = s_st[b + p]; if (st & 1) { ++npres; first = first == NONE ? p : first; } stor |= st; }
+    npres = __reduce_add_sync(0xFFFFFFFFu, npres); first = __reduce_min_sync(0xFFFFFFFFu, first); stor = __reduce_or_sync(0xFFFFFFFFu, stor);
+    const bool have_first = first != NONE;
+    const u64 gbytes = have_first ? s_by[b + first] : 0; const u32 gop = have_first ? s_op[b + first] : 0;
+    const bool inflight = stor & 2, bad_time = stor & 4, complete = npres == n && !inflight && !bad_time;
+    const bool barrier = have_first && gop == CCLD_OP_ALLREDUCE && gbytes < P.barrier_bytes;
+    u32 mism = 0; i64 age = -1;
+    u64 e_min = U64_MAX_, tmax = 0, tmin = U64_MAX_; i64 x_max = INT64_MIN; u32 pmax = NONE, pmin = NONE; u64 chk = 0;
+    for (u32 p = lane; p < n; p += 32) {
+      const u32 st = s_st[b + p];
+      if (!(st & 1)) continue;
+      if (s_op[b + p] != gop || s_by[b + p] != gbytes) mism = 1;
+      const u64 te = s_te[b + p], du = s_du[b + p];
+      if (st & 2) { const i64 ag = now - (i64)te; age = ag > age ? ag : age; }
+      e_min = te < e_min ? te : e_min;
+      const i64 tx = (i64)(te + du); x_max = tx > x_max ? tx : x_max;
+      if (pmax == NONE || du > tmax) { tmax = du; pmax = p; }
+      if (pmin == NONE || du < tmin) { tmin = du; pmin = p; }
+      const u64 ck = ((u64)s_ch[b + p] << 32) | (u64)(NONE - p);        // most changes, then lowest position
+      chk = ck > chk ? ck : chk;
+    }
+    mism = __reduce_or_sync(0xFFFFFFFFu, mism);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      const i64 ag = (i64)shfl_xor64((u64)age, d); age = ag > age ? ag : age;
+      const u64 em = shfl_xor64(e_min, d); e_min = em < e_min ? em : e_min;
+      const i64 xm = (i64)shfl_xor64((u64)x_max, d); x_max = xm > x_max ? xm : x_max;
+      const u64 ck = shfl_xor64(chk, d); chk = ck > chk ? ck : chk;
+      const u64 tM = shfl_xor64(tmax, d); const u32 pM = __shfl_xor_sync(0xFFFFFFFFu, pmax, d);
+      if (pM != NONE && (pmax == NONE || tM > tmax || (tM == tmax && pM < pmax))) { tmax = tM; pmax = pM; }
+      const u64 tm = shfl_xor64(tmin, d); const u32 pm = __shfl_xor_sync(0xFFFFFFFFu, pmin, d);
+      if (pm != NONE && (pmin == NONE || tm < tmin || (tm == tmin && pm < pmin))) { tmin = tm; pmin = pm; }
+    }
+    u32 gfl = (mism ? CCLD_G_OPSET_MISMATCH : 0) | (barrier ? CCLD_G_BARRIER : 0) | (inflight ? CCLD_G_INFLIGHT : 0) |
+              (bad_time ? CCLD_G_BAD_TIME : 0) | (complete ? CCLD_G_COMPLETE : CCLD_G_INCOMPLETE);
+    const bool analysed = complete && !barrier && n >= P.min_group;
+    if (analysed) gfl |= CCLD_G_ANALYSED;
+    const bool hang = !complete && inflight && age > P.hang_ns && !barrier;
+    if (hang) gfl |= CCLD_G_HANG_ALERT;
+    if (lane == 0) {
+      const u64 g = g_t + jg, G = D.n_groups;
+      if (hang) raise_alert(D, R.comm_id[c], row.seq_lo + t.seq_off + jg, age);
+      MidGroup mg; mg.e_min = e_min; mg.gbytes = gbytes; mg.gop = gop; mg.gfl = gfl; mg.complete = complete; mg.analysed = analysed;
+      mg.med_s = mg.mad_s = mg.med_d = mg.mad_d = 0;
+      s_g[jg] = mg;
+      i64 span = 0; double gb = 0.0;
+      if (complete) {
+        span = x_max - (i64)e_min;
+        double num, den; bus_factor(gop, n, &num, &den);
+        gb = busbw((double)gbytes * num, den, span);
+      }
+      D.gi64[(u64)GI_E_MIN * G + g] = complete ? (i64)e_min : 0;
+      D.gi64[(u64)GI_T_MAX * G + g] = complete ? (i64)tmax : 0; D.gi64[(u64)GI_T_MIN * G + g] = complete ? (i64)tmin : 0;
+      D.gi64[(u64)GI_SPAN * G + g] = span;
+      D.gu32[(u64)GU_RANK_TMIN * G + g] = complete ? mem[pmin] : 0; D.gu32[(u64)GU_RANK_TMAX * G + g] = complete ? mem[pmax] : 0;
+      D.gu32[(u64)GU_MAX_CHG * G + g] = complete ? (u32)(chk >> 32) : 0;
+      D.gu32[(u64)GU_RANK_MAX_CHG * G + g] = complete ? mem[NONE - (u32)chk] : 0;
+      D.gu32[(u64)GU_N_PRESENT * G + g] = npres; D.gu32[(u64)GU_GFLAGS * G + g] = gfl;
+      D.gbw[g] = gb;
+      c_comp += complete; c_inc += !complete; c_bar += barrier; c_an += analysed; c_mis += mism; c_pres += npres;
+    }
+  }
+  __syncthreads();
+  const u32 k_med = (n - 1) >> 1;
+  // 4. arrival skew: sort, median, deviations, merge, MAD
+  for (u32 e = threadIdx.x; e < S * n_pad; e += MID_THREADS) {
+    const u32 jg = e / n_pad, i = e - jg * n_pad;
+    s_key[jg * pitch + i] = (i < n && s_g[jg].analysed) ? s_te[jg * pitch + i] - s_g[jg].e_min : U64_MAX_;
+  }
+  __syncthreads();
+  mid_bitonic(s_key, S, n_pad, pitch, false);
+  for (u32 jg = threadIdx.x; jg < S; jg += MID_THREADS) s_g[jg].med_s = s_key[jg * pitch + k_med];
+  __syncthreads();
+  for (u32 e = threadIdx.x; e < S * n_pad; e += MID_THREADS) {
+    const u32 jg = e / n_pad, i = e - jg * n_pad;
+    if (i < n) s_key[jg * pitch + i] = absdiff(s_key[jg * pitch + i], s_g[jg].med_s);
+  }
+  __syncthreads();
+  mid_bitonic(s_key, S, n_pad, pitch, true);
+  for (u32 jg = threadIdx.x; jg < S; jg += MID_THREADS) {
+    s_g[jg].mad_s = s_key[jg * pitch + k_med];
+    const u64 g = g_t + jg, G = D.n_groups; const bool an = s_g[jg].analysed;
+    D.gi64[(u64)GI_MED_SKEW * G + g] = an ? (i64)s_g[jg].med_s : 0; D.gi64[(u64)GI_MAD_SKEW * G + g] = an ? (i64)s_g[jg].mad_s : 0;
+  }
+  __syncthreads();
+  // 5. duration: the same
+  for (u32 e = threadIdx.x; e < S * n_pad; e += MID_THREADS) {
+    const u32 jg = e / n_pad, i = e - jg * n_pad;
+    s_key[jg * pitch + i] = (i < n && s_g[jg].analysed) ? s_du[jg * pitch + i] : U64_MAX_;
+  }
+  __syncthreads();
+  mid_bitonic(s_key, S, n_pad, pitch, false);
+  for (u32 jg = threadIdx.x; jg < S; jg += MID_THREADS) s_g[jg].med_d = s_key[jg * pitch + k_med];
+  __syncthreads();
+  for (u32 e = threadIdx.x; e < S * n_pad; e += MID_THREADS) {
+    const u32 jg = e / n_pad, i = e - jg * n_pad;
+    if (i < n) s_key[jg * pitch + i] = absdiff(s_key[jg * pitch + i], s_g[jg].med_d);
+  }
+  __syncthreads();
+  mid_bitonic(s_key, S, n_pad, pitch, true);
+  for (u32 jg = threadIdx.x; jg < S; jg += MID_THREADS) {
+    s_g[jg].mad_d = s_key[jg * pitch + k_med];
+    const u64 g = g_t + jg, G = D.n_groups; const bool an = s_g[jg].analysed;
+    D.gi64[(u64)GI_MED_DUR * G + g] = an ? (i64)s_g[jg].med_d : 0; D.gi64[(u64)GI_MAD_DUR * G + g] = an ? (i64)s_g[jg].mad_d : 0;
+  }
+  __syncthreads();
+  // 6. flags and votes, in slot order (coalesced byte stores)
+  u32 n_fs = 0, n_fd = 0;
+  for (u32 e = threadIdx.x; e < n_el; e += MID_THREADS) {
+    const u32 jg = e / n, p = e - jg * n, a = jg * pitch + p;
+    const MidGroup& mg = s_g[jg];
+    u8 f = CCLD_F_NOT_ANALYSED;
+    if (!(s_st[a] & 1)) f |= CCLD_F_MISSING;
+    else if (mg.analysed) {
+      const u64 sk = s_te[a] - mg.e_min, du = s_du[a];
+      const bool so = mul_gt(absdiff(sk, mg.med_s), 1000u, mg.mad_s, P.k_milli), sh = sk > mg.med_s;
+      const bool dq = mul_gt(absdiff(du, mg.med_d), 1000u, mg.mad_d, P.k_milli), dh = du > mg.med_d;
+      f = (so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0);
+      if (so) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p] * 4 + (sh ? 0 : 1)], 1u); }
+      if (dq) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p] * 4 + (dh ? 2 : 3)], 1u); }
+    }
+    D.flags[slot_t + e] = f;
+  }
+  // arrival skew = largest enter time minus the smallest, one warp per group
+  for (u32 jg = wid; jg < S; jg += MID_THREADS / 32) {
+    u64 mx = 0;
+    if (s_g[jg].complete) {
+      for (u32 p = lane; p < n; p += 32) { const u64 v = s_te[jg * pitch + p]; mx = v > mx ? v : mx; }
+#pragma unroll
+      for (int d = 16; d > 0; d >>= 1) { const u64 o = shfl_xor64(mx, d); mx = o > mx ? o : mx; }
+    }
+    if (lane == 0) D.gi64[(u64)GI_ARRIVAL_SKEW * D.n_groups + g_t + jg] = s_g[jg].complete ? (i64)(mx - s_g[jg].e_min) : 0;
+  }
+  // 7. per-rank bus bandwidth: thread p sums member p over the tile's groups
+  u32 n_bwc = 0;
+  for (u32 jg = 0; jg < S; ++jg) n_bwc += (s_g[jg].complete && !(s_g[jg].gfl & CCLD_G_BARRIER)) ? 1u : 0u;
+  if (n_bwc) {
+    for (u32 p = threadIdx.x; p < n; p += MID_THREADS) {
+      double v = 0.0;
+      for (u32 jg = 0; jg < S; ++jg) {
+        const MidGroup& mg = s_g[jg];
+        if (!mg.complete || (mg.gfl & CCLD_G_BARRIER)) continue;
+        double num, den; bus_factor(mg.gop, n, &num, &den);
+        v += busbw((double)mg.gbytes * num, den, (i64)s_du[jg * pitch + p]);
+      }
+      atomicAdd(&R.bw_sum[mem[p]], v);
+      atomicAdd(&R.bw_cnt[mem[p]], n_bwc);
+    }
+  }
+  // 8. counters
+  n_fs = __reduce_add_sync(0xFFFFFFFFu, n_fs); n_fd = __reduce_add_sync(0xFFFFFFFFu, n_fd);
+  if (lane == 0) {
+    atomicAdd(&s_cnt[0], c_comp); atomicAdd(&s_cnt[1], c_inc); atomicAdd(&s_cnt[2], c_bar); atomicAdd(&s_cnt[3], c_an);
+    atomicAdd(&s_cnt[4], c_mis); atomicAdd(&s_cnt[5], c_pres); atomicAdd(&s_cnt[6], n_fs); atomicAdd(&s_cnt[7], n_fd);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    count_add(D.counters, C_COMPLETE, s_cnt[0]); count_add(D.counters, C_INCOMPLETE, s_cnt[1]); count_add(D.counters, C_BARRIER, s_cnt[2]);
+    count_add(D.counters, C_ANALYSED, s_cnt[3]); count_add(D.counters, C_MISMATCH, s_cnt[4]); count_add(D.counters, C_PRESENT, s_cnt[5]);
+    count_add(D.counters, C_FLAG_SKEW, s_cnt[6]); count_add(D.counters, C_FLAG_DUR, s_cnt[7]);
+  }
+}
+
+inline size_t mid_smem_bytes(u32 n_pad_min) {
+  // cap = (MID_ELEMS / n_pad) * (n_pad + 1) is largest for the smallest n_pad
+  size_t cap = (size_t)(MID_ELEMS / n_pad_min) * (n_pad_min + 1);
+  return cap * (4 * 8 + 2 * 4 + 2) + 16 + (MID_ELEMS / n_pad_min) * sizeof(MidGroup);
+}
+
+// ------------------------------------------------------------------------------------------------
+// per-op reductions, n > 1024: one CTA per group; enter times and durations live in shared memory,
+// order statistics by most-significant-byte-first radix select
+// ------------------------------------------------------------------------------------------------
+template <class T, class Op>
+__device__ T block_reduce(T v, Op op, T* s_red /*[32]*/) {
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) { T o = __shfl_xor_sync(0xFFFFFFFFu, v, d); v = op(v, o); }
+  __syncthreads();
+  if (lane == 0) s_red[wid] = v;
+  __syncthreads();
+  T r = s_red[0];
+  for (u32 q = 1; q < blockDim.x / 32; ++q) r = op(r, s_red[q]);
+  return r;
+}
+struct OpMinU64 { __device__ u64 operator()(u64 a, u64 b) const { return a < b ? a : b; } };
+struct OpMaxU64 { __device__ u64 operator()(u64 a, u64 b) const { return a > b ? a : b; } };
+struct OpMaxI64 { __device__ i64 operator()(i64 a, i64 b) const { return a > b ? a : b; } };
+struct OpAddU32 { __device__ u32 operator()(u32 a, u32 b) const { return a + b; } };
+struct OpOrU32 { __device__ u32 operator()(u32 a, u32 b) const { return a | b; } };
+struct OpMinU32 { __device__ u32 operator()(u32 a, u32 b) const { return a < b ? a : b; } };
+
+// k-th smallest (0-based) of key(i), i < n; max_key bounds the keys. All threads of the CTA call it.
+template <class F>
+__device__ u64 radix_select(F key, u32 n, u32 k, u64 max_key, u32* hist /*[256]*/, u32* s_pick /*[2]*/) {
+  int top = max_key == 0 ? 0 : (63 - __clzll((long long)max_key)) >> 3;
+  u64 prefix = 0, mask = 0; u32 krem = k;
+  for (int b = top; b >= 0; --b) {
+    for (u32 i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+    __syncthreads();
+    for (u32 i = threadIdx.x; i < n; i += blockDim.x) {
+      const u64 v = key(i);
+      if ((v & mask) == prefix) {
+        const u32 bin = (u32)(v >> (8 * b)) & 255u;
+        const u32 m = __match_any_sync(__activemask(), bin);       // one atomic per distinct bin in the warp
+        if ((threadIdx.x & 31) == (u32)(__ffs(m) - 1)) atomicAdd(&hist[bin], (u32)__popc(m));
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      u32 loc[8], sum = 0;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) { loc[q] = hist[threadIdx.x * 8 + q]; sum += loc[q]; }
+      u32 inc = sum;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) { u32 o = __shfl_up_sync(0xFFFFFFFFu, inc, d); if ((threadIdx.x & 31) >= (u32)d) inc += o; }
+      u32 ex = inc - sum;
+      if (krem >= ex && krem < inc) {
+        u32 cum = ex;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          if (krem >= cum && krem < cum + loc[q]) { s_pick[0] = threadIdx.x * 8 + q; s_pick[1] = krem - cum; }
+          cum += loc[q];
+        }
+      }
+    }
+    __syncthreads();
+    prefix |= (u64)s_pick[0] << (8 * b); mask |= 0xFFull << (8 * b); krem = s_pick[1];
+    __syncthreads();
+  }
+  return prefix;
+}
+
+__global__ void __launch_bounds__(LARGE_THREADS) k_reduce_large(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles,
+                                                                 Registry R, Params P, i64 now) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ u64 s_red64[32];
+  __shared__ u32 s_red32[32];
+  __shared__ u32 s_hist[256];
+  __shared__ u32 s_pick[2];
+  const Tile t = tiles[blockIdx.x];
+  const WinDesc& D = wd[t.w];
+  const u32 c = t.c, n = R.comm_n[c];
+  const RangeRow row = D.ranges[c];
+  const u32* mem = R.members + R.comm_moff[c];
+  u64* s_te = (u64*)smem_raw;
+  u64* s_du = s_te + n;
+  const u64 G = D.n_groups;
+  double bwacc[LARGE_MAXP];               // member p = threadIdx.x + q * LARGE_THREADS
+#pragma unroll
+  for (int q = 0; q < LARGE_MAXP; ++q) bwacc[q] = 0.0;
+  u32 n_bwc = 0;
+
+  for (u32 jg = 0; jg < t.count; ++jg) {
+    __syncthreads();
+    const u64 g = row.group0 + t.seq_off + jg, slot = row.slot0 + (u64)(t.seq_off + jg) * n;
+    const u32 seq = row.seq_lo + t.seq_off + jg;
+    // pass 1: gather, presence, first present member
+    u32 npres = 0, first = NONE, stor = 0;
+    for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS) {
+      const u32 idx = D.perm[slot + p];
+      u64 te = 0, du = 0; u32 st = 0;
+      if (idx != NONE) {
+        const i64 x = D.t_enter[idx], y = D.t_exit[idx];
+        st = 1 | (y == -1 ? 2 : ((x < 0 || y < x) ? 4 : 0));
+        te = (u64)x; du = (u64)(y - x);
+        ++npres; first = first == NONE ? p : first;
+      }
+      stor |= st; s_te[p] = te; s_du[p] = du;
+    }
+    npres = block_reduce(npres, OpAddU32(), s_red32);
+    first = block_reduce(first, OpMinU32(), s_red32);
+    stor = block_reduce(stor, OpOrU32(), s_red32);
+    const bool have_first = first != NONE;
+    u64 gbytes = 0; u32 gop = 0;
+    if (have_first) { const u32 idx = D.perm[slot + first]; gbytes = D.bytes[idx]; gop = D.op[idx]; }
+    const bool inflight = stor & 2, bad_time = stor & 4, complete = npres == n && !inflight && !bad_time;
+    const bool barrier = have_first && gop == CCLD_OP_ALLREDUCE && gbytes < P.barrier_bytes;
+    // pass 2: op-set check, rate column, in-flight age, extrema
+    u32 mism = 0; i64 age = -1; u64 chk = 0;
+    u64 e_min = U64_MAX_, tmax = 0, tmin = U64_MAX_; i64 x_max = INT64_MIN;
+    for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS) {
+      const u32 idx = D.perm[slot + p];
+      if (idx == NONE) continue;
+      if (D.op[idx] != gop || D.bytes[idx] != gbytes) mism = 1;
+      u32 ch = 0;
+      if (D.send_chg != nullptr) { const u32 sc = D.send_chg[idx], rc = D.recv_chg[idx]; ch = sc > rc ? sc : rc; }
+      const u64 ck = ((u64)ch << 32) | (u64)(NONE - p); chk = ck > chk ? ck : chk;
+      const u64 te = s_te[p], du = s_du[p];
+      if (D.t_exit[idx] == -1) { const i64 ag = now - (i64)te; age = ag > age ? ag : age; }
+      e_min = te < e_min ? te : e_min; tmax = du > tmax ? du : tmax; tmin = du < tmin ? du : tmin;
+      const i64 tx = (i64)(te + du); x_max = tx > x_max ? tx : x_max;
+    }
+    mism = block_reduce(mism, OpOrU32(), s_red32);
+    age = block_reduce(age, OpMaxI64(), (i64*)s_red64);
+    chk = block_reduce(chk, OpMaxU64(), s_red64);
+    e_min = block_reduce(e_min, OpMinU64(), s_red64);
+    tmax = block_reduce(tmax, OpMaxU64(), s_red64);
+    tmin = block_reduce(tmin, OpMinU64(), s_red64);
+    x_max = block_reduce(x_max, OpMaxI64(), (i64*)s_red64);
+    u32 gfl = (mism ? CCLD_G_OPSET_MISMATCH : 0) | (barrier ? CCLD_G_BARRIER : 0) | (inflight ? CCLD_G_INFLIGHT : 0) |
+              (bad_time ? CCLD_G_BAD_TIME : 0) | (complete ? CCLD_G_COMPLETE : CCLD_G_INCOMPLETE);
+    const bool analysed = complete && !barrier && n >= P.min_group;
+    const bool hang = !complete && inflight && age > P.hang_ns && !barrier;
+    if (analysed) gfl |= CCLD_G_ANALYSED;
+    if (hang) gfl |= CCLD_G_HANG_ALERT;
+
+    if (!complete) {
+      for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS)
+        D.flags[slot + p] = D.perm[slot + p] == NONE ? (CCLD_F_NOT_ANALYSED | CCLD_F_MISSING) : CCLD_F_NOT_ANALYSED;
+      if (threadIdx.x == 0) {
+        if (hang) raise_alert(D, R.comm_id[c], seq, age);
+        for (int q = 0; q < GI_COUNT; ++q) D.gi64[(u64)q * G + g] = 0;
+        for (int q = 0; q < GU_COUNT; ++q) D.gu32[(u64)q * G + g] = 0;
+        D.gu32[(u64)GU_N_PRESENT * G + g] = npres; D.gu32[(u64)GU_GFLAGS * G + g] = gfl; D.gbw[g] = 0.0;
+        count_add(D.counters, C_INCOMPLETE, 1); count_add(D.counters, C_BARRIER, barrier); count_add(D.counters, C_MISMATCH, mism);
+        count_add(D.counters, C_PRESENT, npres);
+      }
+      continue;
+    }
+    // positions of the extrema: lowest ring position among equals
+    u32 pmax = NONE, pmin = NONE; u64 askew = 0;
+    for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS) {
+      if (s_du[p] == tmax && p < pmax) pmax = p;
+      if (s_du[p] == tmin && p < pmin) pmin = p;
+      const u64 sk = s_te[p] - e_min; askew = sk > askew ? sk : askew;
+    }
+    pmax = block_reduce(pmax, OpMinU32(), s_red32);
+    pmin = block_reduce(pmin, OpMinU32(), s_red32);
+    askew = block_reduce(askew, OpMaxU64(), s_red64);
+    const i64 span = x_max - (i64)e_min;
+    double num, den; bus_factor(gop, n, &num, &den);
+    const double bn = (double)gbytes * num;
+    if (!barrier) {
+      ++n_bwc;
+#pragma unroll
+      for (int q = 0; q < LARGE_MAXP; ++q) { const u32 p = threadIdx.x + q * LARGE_THREADS; if (p < n) bwacc[q] += busbw(bn, den, (i64)s_du[p]); }
+    }
+
+    u64 med_s = 0, mad_s = 0, med_d = 0, mad_d = 0; u32 n_fs = 0, n_fd = 0;
+    if (analysed) {
+      const u32 k = (n - 1) >> 1;
+      med_s = radix_select([&](u32 i) { return s_te[i] - e_min; }, n, k, askew, s_hist, s_pick);
+      { const u64 m = med_s, dmax = m > askew - m ? m : askew - m;
+        mad_s = radix_select([&](u32 i) { return absdiff(s_te[i] - e_min, m); }, n, k, dmax, s_hist, s_pick); }
+      med_d = tmin + radix_select([&](u32 i) { return s_du[i] - tmin; }, n, k, tmax - tmin, s_hist, s_pick);
+      { const u64 m = med_d, dmax = (m - tmin) > (tmax - m) ? (m - tmin) : (tmax - m);
+        mad_d = radix_select([&](u32 i) { return absdiff(s_du[i], m); }, n, k, dmax, s_hist, s_pick); }
+      for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS) {
+        const u64 sk = s_te[p] - e_min, du = s_du[p];
+        const bool so = mul_gt(absdiff(sk, med_s), 1000u, mad_s, P.k_milli), sh = sk > med_s;
+        const bool dq = mul_gt(absdiff(du, med_d), 1000u, mad_d, P.k_milli), dh = du > med_d;
+        D.flags[slot + p] = (so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0);
+        if (so) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p] * 4 + (sh ? 0 : 1)], 1u); }
+        if (dq) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p] * 4 + (dh ? 2 : 3)], 1u); }
+      }
+      n_fs = block_reduce(n_fs, OpAddU32(), s_red32);
+      n_fd = block_reduce(n_fd, OpAddU32(), s_red32);
+    } else {
+      for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS) D.flags[slot + p] = CCLD_F_NOT_ANALYSED;
+    }
+    if (threadIdx.x == 0) {
+      D.gi64[(u64)GI_E_MIN * G + g] = (i64)e_min; D.gi64[(u64)GI_ARRIVAL_SKEW * G + g] = (i64)askew;
+      D.gi64[(u64)GI_T_MAX * G + g] = (i64)tmax; D.gi64[(u64)GI_T_MIN * G + g] = (i64)tmin; D.gi64[(u64)GI_SPAN * G + g] = span;
+      D.gi64[(u64)GI_MED_SKEW * G + g] = (i64)med_s; D.gi64[(u64)GI_MAD_SKEW * G + g] = (i64)mad_s;
+      D.gi64[(u64)GI_MED_DUR * G + g] = (i64)med_d; D.gi64[(u64)GI_MAD_DUR * G + g] = (i64)mad_d;
+      D.gu32[(u64)GU_RANK_TMIN * G + g] = mem[pmin]; D.gu32[(u64)GU_RANK_TMAX * G + g] = mem[pmax];
+      D.gu32[(u64)GU_MAX_CHG * G + g] = (u32)(chk >> 32); D.gu32[(u64)GU_RANK_MAX_CHG * G + g] = mem[NONE - (u32)chk];
+      D.gu32[(u64)GU_N_PRESENT * G + g] = npres; D.gu32[(u64)GU_GFLAGS * G + g] = gfl;
+      D.gbw[g] = busbw(bn, den, span);
+      count_add(D.counters, C_COMPLETE, 1); count_add(D.counters, C_BARRIER, barrier); count_add(D.counters, C_ANALYSED, analysed);
+      count_add(D.counters, C_MISMATCH, mism); count_add(D.counters, C_PRESENT, npres);
+      count_add(D.counters, C_FLAG_SKEW, n_fs); count_add(D.counters, C_FLAG_DUR, n_fd);
+    }
+  }  // groups of the tile
+  if (n_bwc) {
+#pragma unroll
+    for (int q = 0; q < LARGE_MAXP; ++q) {
+      const u32 p = threadIdx.x + q * LARGE_THREADS;
+      if (p < n) { atomicAdd(&R.bw_sum[mem[p]], bwacc[q]); atomicAdd(&R.bw_cnt[mem[p]], n_bwc); }
+    }
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// window decision per communicator (Sec. 4.2.1 Eq. 1-3, Sec. 4.2.2 Eq. 4): one warp per
+// communicator walks the windows of the batch in order
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(128) k_window_decide(const WinDesc* __restrict__ wd, u32 nw, Registry R, Params P) {
+  const u32 c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (c >= R.n_comms) return;
+  const u32 n = R.comm_n[c];
+  const u32* mem = R.members + R.comm_moff[c];
+  CommState st = R.state[c];
+  for (u32 w = 0; w < nw; ++w) {
+    const WinDesc& D = wd[w];
+    const RangeRow row = D.ranges[c];
+    if (row.n_seq == 0) continue;
+    const u64 G = D.n_groups;
+    const u32* gfl = D.gu32 + (u64)GU_GFLAGS * G + row.group0;
+    const i64* e_min = D.gi64 + (u64)GI_E_MIN * G + row.group0;
+    const i64* t_max = D.gi64 + (u64)GI_T_MAX * G + row.group0;
+    const i64* t_min = D.gi64 + (u64)GI_T_MIN * G + row.group0;
+    u32 n_rounds = 0, n_an = 0;
+    u64 best_rng = 0; u32 best_k = NONE;
+    for (u32 k0 = 0; k0 < row.n_seq; k0 += 32) {
+      const u32 k = k0 + lane;
+      const u32 f = k < row.n_seq ? gfl[k] : 0;
+      const bool round = (f & CCLD_G_COMPLETE) && !(f & CCLD_G_BARRIER);
+      const u32 rmask = __ballot_sync(0xFFFFFFFFu, round);
+      n_rounds += __popc(rmask);
+      n_an += __popc(__ballot_sync(0xFFFFFFFFu, (f & CCLD_G_ANALYSED) != 0));
+      i64 em = 0, tM = 0, tm = 0;
+      if (round) { em = e_min[k]; tM = t_max[k]; tm = t_min[k]; }
+      // Eq. 1: rounds feed the baseline, in op-counter order, until m is fixed
+      if (st.m == 0) {
+        u32 rem = rmask;
+        while (rem && st.m == 0) {
+          const int src = __ffs(rem) - 1; rem &= rem - 1;
+          const i64 em_s = __shfl_sync(0xFFFFFFFFu, em, src), tM_s = __shfl_sync(0xFFFFFFFFu, tM, src);
+          if (st.rounds == 0) st.t_first = em_s;
+          if (st.rounds == (u64)P.m_max_rounds || (st.rounds > 0 && em_s - st.t_first >= P.m_max_ns)) st.m = st.rounds;
+          else st.sum_m += tM_s;
+          ++st.rounds;
+        }
+        st.rounds += __popc(rem);
+      } else {
+        st.rounds += __popc(rmask);
+      }
+      // Eq. 2: largest intra-round range, earliest op counter among equals
+      if (round) { const u64 rg = (u64)(tM - tm); if (best_k == NONE || rg > best_rng) { best_rng = rg; best_k = k; } }
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      const u64 orng = shfl_xor64(best_rng, d); const u32 ok = __shfl_xor_sync(0xFFFFFFFFu, best_k, d);
+      if (ok != NONE && (best_k == NONE || orng > best_rng || (orng == best_rng && ok < best_k))) { best_rng = orng; best_k = ok; }
+    }
+    // analysed ops of this window count towards every member's denominator
+    if (n_an) for (u32 p = lane; p < n; p += 32) atomicAdd(&R.ops[mem[p]], n_an);
+    if (lane == 0) {
+      ccld_comm_verdict v;
+      v.comm = R.comm_id[c]; v.n_rounds = n_rounds; v.sel_seq = NONE; v.cls = 0; v.slow_detected = 0; v.located = 0;
+      v.baseline_static = st.m == 0; v.rate_source = 0; v.root_comp = NONE; v.root_comm = NONE;
+      v.t_max = 0; v.t_min = 0; v.R = 0.0; v.P = 0.0;
+      v.t_base = st.m > 0 ? st.sum_m / (i64)st.m : P.tbase_init_ns;
+      v.rounds_total = st.rounds; v.m = st.m;
+      if (best_k != NONE) {
+        v.sel_seq = row.seq_lo + best_k; v.t_max = t_max[best_k]; v.t_min = t_min[best_k];
+        v.R = (double)(v.t_max - v.t_base) / (double)v.t_base;                                     // Eq. 3
+        const bool slow = v.t_max > v.t_base && mul_gt((u64)(v.t_max - v.t_base), 1000u, (u64)v.t_base, P.theta_slow_milli);
+        v.slow_detected = slow;
+        if (slow) {
+          ++st.slow_count;
+          v.located = st.slow_count > (u64)P.slow_rep_threshold;
+          const u64 num = (u64)(v.t_max - v.t_min), den = (u64)(v.t_max - v.t_base);
+          v.P = (double)num / (double)den;                                                         // Eq. 4
+          v.cls = mul_gt(num, 1000u, den, P.beta_milli) ? 1u : (mul_lt(num, 1000u, den, P.alpha_milli) ? 2u : 3u);
+          const u64 gq = row.group0 + best_k;
+          v.root_comp = D.gu32[(u64)GU_RANK_TMIN * G + gq];
+          const u32 mc = D.gu32[(u64)GU_MAX_CHG * G + gq];
+          if (mc > 0) { v.root_comm = D.gu32[(u64)GU_RANK_MAX_CHG * G + gq]; v.rate_source = 0; }
+          else { v.root_comm = D.gu32[(u64)GU_RANK_TMAX * G + gq]; v.rate_source = 1; }
+        }
+      }
+      v.slow_count = st.slow_count;
+      D.comm_rows[row.row_idx] = v;
+    }
+    st.slow_count = __shfl_sync(0xFFFFFFFFu, st.slow_count, 0);
+  }
+  if (lane == 0) R.state[c] = st;
+}
+
+// ------------------------------------------------------------------------------------------------
+// hang location (Sec. 4.2.2, Fig. 6): one CTA
+// ------------------------------------------------------------------------------------------------
+struct HangArgs {
+  u32 c, seq, n_frames, n_channels;
+  const u32 *f_rank, *f_comm, *f_seq, *progress;
+  u8* entered; u8* done;     // [n] scratch
+  u32* frame;                // [n] scratch
+  u64* tot;                  // [n] scratch
+  u32* roots; u32 roots_cap; // device list
+  ccld_hang_verdict* out;    // device copy of the struct (pointer fields unused)
+};
+
+__global__ void __launch_bounds__(1024) k_hang_locate(const WinDesc* __restrict__ wd, Registry R, HangArgs A) {
+  __shared__ u64 s_red64[32];
+  __shared__ u32 s_red32[32];
+  __shared__ u32 s_base;
+  const WinDesc& D = wd[0];
+  const u32 c = A.c, n = R.comm_n[c], cid = R.comm_id[c];
+  const u32* mem = R.members + R.comm_moff[c];
+  const RangeRow row = D.ranges[c];
+  for (u32 p = threadIdx.x; p < n; p += blockDim.x) { A.entered[p] = 0; A.done[p] = 0; A.frame[p] = NONE; A.tot[p] = 0; }
+  __syncthreads();
+  // a member has entered if it reported this or a later op counter
+  if (row.n_seq > 0 && A.seq <= row.seq_lo + (row.n_seq - 1)) {
+    const u32 s_first = A.seq > row.seq_lo ? A.seq - row.seq_lo : 0;
+    const u64 cnt = (u64)(row.n_seq - s_first) * n;
+    for (u64 e = threadIdx.x; e < cnt; e += blockDim.x) {
+      const u32 so = s_first + (u32)(e / n), p = (u32)(e % n);
+      const u32 idx = D.perm[row.slot0 + (u64)so * n + p];
+      if (idx != NONE) {
+        A.entered[p] = 1;
+        if (row.seq_lo + so == A.seq && D.t_exit[idx] != -1) A.done[p] = 1;
+      }
+    }
+  }
+  // progress frames of this op: the first frame uploaded for a member counts
+  for (u32 f = threadIdx.x; f < A.n_frames; f += blockDim.x) {
+    if (A.f_comm[f] != cid || A.f_seq[f] != A.seq) continue;
+    const u32 p = pos_lookup(R, A.f_rank[f], c);
+    if (p != NONE) atomicMin(&A.frame[p], f);
+  }
+  __syncthreads();
+  u32 n_ne = 0, n_ok = 0, n_missing = 0; u64 mn = U64_MAX_;
+  for (u32 p = threadIdx.x; p < n; p += blockDim.x) {
+    n_ne += !A.entered[p]; n_ok += A.done[p];
+    const u32 f = A.frame[p];
+    u64 tot = 0;
+    if (f == NONE) ++n_missing;
+    else for (u32 ch = 0; ch < A.n_channels; ++ch) tot += (u64)A.progress[((u64)f * A.n_channels + ch) * 2] + A.progress[((u64)f * A.n_channels + ch) * 2 + 1];
+    A.tot[p] = tot; mn = tot < mn ? tot : mn;
+  }
+  n_ne = block_reduce(n_ne, OpAddU32(), s_red32);
+  n_ok = block_reduce(n_ok, OpAddU32(), s_red32);
+  n_missing = block_reduce(n_missing, OpAddU32(), s_red32);
+  mn = block_reduce(mn, OpMinU64(), s_red64);
+  __syncthreads();
+  const u32 cls = n_ne > 0 ? 1u : (n_ok > 0 ? 2u : 3u);
+  u32 n_roots = 0, stuck = 0; u64 min_total = 0;
+  if (cls == 3) {
+    // fewest counters; among equals the most upstream of a run (predecessor ahead), then the lowest position
+    u32 up = NONE, any = NONE;
+    for (u32 p = threadIdx.x; p < n; p += blockDim.x) {
+      if (A.tot[p] != mn) continue;
+      any = p < any ? p : any;
+      if (A.tot[(p + n - 1) % n] > mn) up = p < up ? p : up;
+    }
+    up = block_reduce(up, OpMinU32(), s_red32);
+    any = block_reduce(any, OpMinU32(), s_red32);
+    const u32 root = up != NONE ? up : any;
+    n_roots = 1; min_total = mn;
+    if (threadIdx.x == 0) {
+      if (A.roots_cap > 0) A.roots[0] = mem[root];
+      const u32 f = A.frame[root];
+      if (f != NONE && A.n_channels > 0) {
+        u32 s = NONE;
+        for (u32 ch = 0; ch < A.n_channels; ++ch) { const u32 r = A.progress[((u64)f * A.n_channels + ch) * 2 + 1]; s = r < s ? r : s; }
+        stuck = s;
+      }
+    }
+  } else {
+    // ordered compaction of the not-entered (H1) or not-hung (H2) members
+    if (threadIdx.x == 0) s_base = 0;
+    __syncthreads();
+    for (u32 p0 = 0; p0 < n; p0 += blockDim.x) {
+      const u32 p = p0 + threadIdx.x;
+      const bool sel = p < n && (cls == 1 ? !A.entered[p] : A.done[p] != 0);
+      const u32 bal = __ballot_sync(0xFFFFFFFFu, sel);
+      const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+      __syncthreads();
+      if (lane == 0) s_red32[wid] = __popc(bal);
+      __syncthreads();
+      u32 off = s_base;
+      for (u32 q = 0; q < wid; ++q) off += s_red32[q];
+      off += __popc(bal & ((1u << lane) - 1));
+      if (sel && off < A.roots_cap) A.roots[off] = mem[p];
+      __syncthreads();
+      if (threadIdx.x == 0) { u32 tot = 0; for (u32 q = 0; q < blockDim.x / 32; ++q) tot += s_red32[q]; s_base += tot; }
+      __syncthreads();
+    }
+    n_roots = s_base;
+  }
+  if (threadIdx.x == 0) {
+    ccld_hang_verdict v;
+    v.cls = cls; v.n_roots_total = n_roots; v.n_not_entered = n_ne; v.n_hung = n - n_ok; v.n_not_hung = n_ok;
+    v.n_missing_frames = cls == 3 ? n_missing : 0; v.stuck_step = stuck; v.n_members = n; v.min_total = min_total;
+    v.roots = nullptr; v.roots_cap = 0;
+    *A.out = v;
+  }
+}
+
+// ------------------------------------------------------------------------------------------------
+// suspects and ordered lists
+// ------------------------------------------------------------------------------------------------
+__global__ void k_suspects(Registry R, Params P, ccld_suspect* __restrict__ out, u32 cap, u32* __restrict__ count) {
+  const u32 r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= R.n_ranks) return;
+  const u32 ops = R.ops[r];
+  if (ops == 0) return;
+  const u32 cnt = R.bw_cnt[r];
+  const double bw = cnt ? R.bw_sum[r] / (double)cnt : 0.0;
+  const u32 v[2] = {R.votes[(u64)r * 4 + 0], R.votes[(u64)r * 4 + 2]};
+  for (u32 kind = 1; kind <= 2; ++kind) {
+    if ((u64)v[kind - 1] * 1000u >= (u64)P.vote_rep_milli * ops) {
+      const u32 k = atomicAdd(count, 1u);
+      if (k < cap) { ccld_suspect s; s.kind = kind; s.rank = r; s.votes = v[kind - 1]; s.ops = ops; s.mean_busbw = bw; out[k] = s; }
+    }
+  }
+}
+
+// Rank-by-counting sort of short lists: element i goes to the number of elements that precede it.
+__global__ void k_rank_sort_suspects(const ccld_suspect* __restrict__ in, u32 n, ccld_suspect* __restrict__ out) {
+  const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const ccld_suspect a = in[i];
+  u32 before = 0;
+  for (u32 j = 0; j < n; ++j) {
+    const ccld_suspect b = in[j];
+    const bool lt = b.kind != a.kind ? b.kind < a.kind : (b.votes != a.votes ? b.votes > a.votes : b.rank < a.rank);
+    before += lt;
+  }
+  out[before] = a;
+}
+
+__global__ void k_rank_sort_alerts(const ccld_hang_alert* __restrict__ in, u32 n, ccld_hang_alert* __restrict__ out, Registry R) {
+  const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const ccld_hang_alert a = in[i];
+  const u32 ca = comm_lookup(R, a.comm);
+  u32 before = 0;
+  for (u32 j = 0; j < n; ++j) {
+    const ccld_hang_alert b = in[j];
+    const u32 cb = comm_lookup(R, b.comm);
+    before += cb != ca ? cb < ca : b.seq < a.seq;
+  }
+  out[before] = a;
+}
+
+}  // namespace ccld
