@@ -1,0 +1,575 @@
+// Host side of libccld: context, communicator registry, window upload, launch sequencing and result
+// read-back. No analysis arithmetic lives here; every step of the hot path is a kernel in
+// ccld_kernels.cuh.
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <memory>
+#include <new>
+#include <string>
+#include <unordered_map>
+#include <vector>
+
+#include "ccld_kernels.cuh"
+
+using namespace ccld;
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+
+struct Block { void* p = nullptr; size_t bytes = 0; };
+
+struct CommHost { u32 id, seq0; std::vector<u32> ranks; };
+
+// Device blocks are recycled through a free list so that steady-state analysis allocates nothing.
+struct Pool {
+  std::vector<Block> free_list;
+  Block get(size_t bytes, cudaError_t* err) {
+    bytes = align_up(std::max<size_t>(bytes, ALIGN));
+    int best = -1;
+    for (size_t i = 0; i < free_list.size(); ++i)
+      if (free_list[i].bytes >= bytes && free_list[i].bytes <= 2 * bytes + (1u << 20) && (best < 0 || free_list[i].bytes < free_list[best].bytes)) best = (int)i;
+    if (best >= 0) { Block b = free_list[best]; free_list.erase(free_list.begin() + best); *err = cudaSuccess; return b; }
+    Block b; b.bytes = bytes;
+    *err = cudaMalloc(&b.p, bytes);
+    if (*err != cudaSuccess) {                 // give cached blocks back to the driver and retry once
+      for (auto& f : free_list) cudaFree(f.p);
+      free_list.clear();
+      *err = cudaMalloc(&b.p, bytes);
+      if (*err != cudaSuccess) { b.p = nullptr; b.bytes = 0; }
+    }
+    return b;
+  }
+  void put(Block b) { if (b.p) free_list.push_back(b); }
+  void clear() { for (auto& f : free_list) cudaFree(f.p); free_list.clear(); }
+};
+
+struct Shared {                                 // a pooled block shared by the windows of one batch
+  Pool* pool; Block b;
+  Shared(Pool* p, Block blk) : pool(p), b(blk) {}
+  ~Shared() { pool->put(b); }
+};
+
+struct WindowHost {
+  u32 id = 0; u64 n_rec = 0; bool owns = false; Block own;
+  WinDesc d;                                    // device pointers
+  u32 n_frames = 0, n_channels = 0;
+  const u32 *f_rank = nullptr, *f_comm = nullptr, *f_seq = nullptr, *progress = nullptr;
+  bool analysed = false;
+  std::shared_ptr<Shared> plan_blk, res_blk;
+  WinDesc* d_desc = nullptr;                    // this window's descriptor on the device
+  u64 totals[T_COUNT];
+  WindowHost() { std::memset(&d, 0, sizeof d); std::memset(totals, 0, sizeof totals); }
+};
+
+}  // namespace
+
+struct ccld_ctx {
+  ccld_params params; Params dp; int device = 0; cudaStream_t stream = nullptr;
+  std::vector<CommHost> comms; std::unordered_map<u32, u32> comm_idx;
+  bool finalized = false; u32 n_ranks = 0, max_n = 0, max_large_n = 0; u64 sum_n = 0;
+  Block reg_blk, misc_blk; Registry reg; size_t stats_off = 0, stats_bytes = 0;
+  std::map<u32, WindowHost> windows;
+  Pool pool; std::string err;
+  u64* h_pinned = nullptr; size_t h_pinned_bytes = 0;
+  ccld_ctx() { std::memset(&reg, 0, sizeof reg); }
+};
+
+namespace {
+
+int fail(ccld_ctx* c, int code, const std::string& msg) { if (c) c->err = msg; return code; }
+
+#define CK(call)                                                                                   \
+  do { cudaError_t e_ = (call);                                                                    \
+       if (e_ != cudaSuccess) return fail(ctx, e_ == cudaErrorMemoryAllocation ? CCLD_ERR_NOMEM : CCLD_ERR_CUDA, \
+                                          std::string(#call) + ": " + cudaGetErrorString(e_)); } while (0)
+
+int ensure_pinned(ccld_ctx* ctx, size_t bytes) {
+  if (ctx->h_pinned_bytes >= bytes) return CCLD_OK;
+  if (ctx->h_pinned) cudaFreeHost(ctx->h_pinned);
+  ctx->h_pinned = nullptr; ctx->h_pinned_bytes = 0;
+  CK(cudaMallocHost((void**)&ctx->h_pinned, bytes));
+  ctx->h_pinned_bytes = bytes;
+  return CCLD_OK;
+}
+
+// Layout of the scratch block used by get_verdict and locate_hang.
+struct MiscLayout { size_t sus_a, sus_b, alerts, count, entered, done, frame, roots, tot, hang_out, total; };
+MiscLayout misc_layout(u32 n_ranks, u32 max_n) {
+  MiscLayout L; size_t off = 0;
+  auto take = [&](size_t b) { size_t o = off; off = align_up(off + std::max<size_t>(b, 1)); return o; };
+  L.sus_a = take(2ull * n_ranks * sizeof(ccld_suspect)); L.sus_b = take(2ull * n_ranks * sizeof(ccld_suspect));
+  L.alerts = take(CCLD_MAX_ALERTS_PER_WINDOW * sizeof(ccld_hang_alert)); L.count = take(16);
+  L.entered = take(max_n); L.done = take(max_n); L.frame = take(max_n * 4ull); L.roots = take(max_n * 4ull);
+  L.tot = take(max_n * 8ull); L.hang_out = take(sizeof(ccld_hang_verdict));
+  L.total = off;
+  return L;
+}
+
+// Builds the device tables of the communicator registry and the per-rank statistics.
+int finalize_registry(ccld_ctx* ctx) {
+  if (ctx->finalized) return CCLD_OK;
+  const u32 nc = (u32)ctx->comms.size();
+  if (nc == 0) return fail(ctx, CCLD_ERR_STATE, "no communicator registered");
+  u32 max_rank = 0; u64 sum_n = 0; u32 max_n = 0, max_large = 0;
+  for (auto& c : ctx->comms) {
+    for (u32 r : c.ranks) max_rank = std::max(max_rank, r);
+    sum_n += c.ranks.size(); max_n = std::max<u32>(max_n, (u32)c.ranks.size());
+    if (c.ranks.size() > MID_N) max_large = std::max<u32>(max_large, (u32)c.ranks.size());
+  }
+  const u32 nr = max_rank + 1;
+  u32 hsize = 16; while (hsize < 2 * nc) hsize <<= 1;
+  std::vector<uint2> hash(hsize, make_uint2(0, NONE));
+  std::vector<u32> comm_id(nc), comm_n(nc), comm_seq0(nc), members; std::vector<u64> moff(nc);
+  std::vector<u32> rank_ptr(nr + 1, 0);
+  members.reserve(sum_n);
+  for (u32 i = 0; i < nc; ++i) {
+    const CommHost& c = ctx->comms[i];
+    comm_id[i] = c.id; comm_n[i] = (u32)c.ranks.size(); comm_seq0[i] = c.seq0; moff[i] = members.size();
+    members.insert(members.end(), c.ranks.begin(), c.ranks.end());
+    u32 h = (c.id * 2654435761u) & (hsize - 1);
+    while (hash[h].y != NONE) h = (h + 1) & (hsize - 1);
+    hash[h] = make_uint2(c.id, i);
+    for (u32 r : c.ranks) ++rank_ptr[r + 1];
+  }
+  for (u32 r = 0; r < nr; ++r) rank_ptr[r + 1] += rank_ptr[r];
+  std::vector<u32> ent_comm(sum_n), ent_pos(sum_n), fill(rank_ptr.begin(), rank_ptr.end() - 1);
+  for (u32 i = 0; i < nc; ++i)
+    for (u32 p = 0; p < ctx->comms[i].ranks.size(); ++p) { u32 r = ctx->comms[i].ranks[p]; ent_comm[fill[r]] = i; ent_pos[fill[r]] = p; ++fill[r]; }
+
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
+  const size_t o_hash = take(hsize * sizeof(uint2)), o_id = take(nc * 4), o_n = take(nc * 4), o_s0 = take(nc * 4), o_moff = take(nc * 8),
+               o_mem = take(sum_n * 4), o_ptr = take((nr + 1) * 4ull), o_ec = take(sum_n * 4), o_ep = take(sum_n * 4);
+  const size_t o_stats = off;
+  const size_t o_state = take(nc * sizeof(CommState)), o_votes = take(nr * 16ull), o_ops = take(nr * 4ull), o_cnt = take(nr * 4ull), o_bw = take(nr * 8ull);
+  cudaError_t e;
+  ctx->reg_blk = ctx->pool.get(off, &e);
+  if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "registry allocation failed");
+  char* base = (char*)ctx->reg_blk.p;
+  cudaStream_t st = ctx->stream;
+  CK(cudaMemcpyAsync(base + o_hash, hash.data(), hsize * sizeof(uint2), cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(base + o_id, comm_id.data(), nc * 4, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(base + o_n, comm_n.data(), nc * 4, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(base + o_s0, comm_seq0.data(), nc * 4, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(base + o_moff, moff.data(), nc * 8, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(base + o_mem, members.data(), sum_n * 4, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(base + o_ptr, rank_ptr.data(), (nr + 1) * 4ull, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(base + o_ec, ent_comm.data(), sum_n * 4, cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(base + o_ep, ent_pos.data(), sum_n * 4, cudaMemcpyHostToDevice, st));
+  CK(cudaMemsetAsync(base + o_stats, 0, off - o_stats, st));
+  CK(cudaStreamSynchronize(st));              // the host vectors above go out of scope
+  Registry& R = ctx->reg;
+  R.n_comms = nc; R.hash_mask = hsize - 1; R.n_ranks = nr; R.pad = 0;
+  R.hash = (const uint2*)(base + o_hash); R.comm_id = (const u32*)(base + o_id); R.comm_n = (const u32*)(base + o_n);
+  R.comm_seq0 = (const u32*)(base + o_s0); R.comm_moff = (const u64*)(base + o_moff); R.members = (const u32*)(base + o_mem);
+  R.rank_ptr = (const u32*)(base + o_ptr); R.ent_comm = (const u32*)(base + o_ec); R.ent_pos = (const u32*)(base + o_ep);
+  R.state = (CommState*)(base + o_state); R.votes = (u32*)(base + o_votes); R.ops = (u32*)(base + o_ops);
+  R.bw_cnt = (u32*)(base + o_cnt); R.bw_sum = (double*)(base + o_bw);
+  ctx->stats_off = o_stats; ctx->stats_bytes = off - o_stats;
+  ctx->n_ranks = nr; ctx->max_n = max_n; ctx->max_large_n = max_large; ctx->sum_n = sum_n;
+
+  // scratch for suspects, alert ordering and hang location
+  ctx->misc_blk = ctx->pool.get(misc_layout(nr, max_n).total, &e);
+  if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "scratch allocation failed");
+
+  CK(cudaFuncSetAttribute(k_reduce_mid, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mid_smem_bytes(16)));
+  if (max_large) CK(cudaFuncSetAttribute(k_reduce_large, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(16ull * max_large)));
+  ctx->finalized = true;
+  return CCLD_OK;
+}
+
+void drop_results(WindowHost& w) {
+  w.analysed = false; w.plan_blk.reset(); w.res_blk.reset(); w.d_desc = nullptr;
+  std::memset(w.totals, 0, sizeof w.totals);
+}
+
+int find_analysed(ccld_ctx* ctx, u32 wid, WindowHost** out) {
+  auto it = ctx->windows.find(wid);
+  if (it == ctx->windows.end()) return fail(ctx, CCLD_ERR_NO_WINDOW, "unknown window id");
+  if (!it->second.analysed) return fail(ctx, CCLD_ERR_NO_WINDOW, "window not analysed");
+  *out = &it->second;
+  return CCLD_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+void ccld_params_default(ccld_params* p) {
+  if (!p) return;
+  p->tbase_init_ns = 2000000; p->theta_slow_milli = 3000; p->alpha_milli = 400; p->beta_milli = 600;
+  p->m_max_rounds = 100; p->m_max_ns = 120000000000ll; p->hang_ns = 300000000000ll; p->barrier_bytes = 4;
+  p->slow_rep_threshold = 1; p->k_milli = 5189; p->min_group = 4; p->vote_rep_milli = 100;
+}
+
+int ccld_create(ccld_ctx** out, const ccld_params* params, int device, void* cuda_stream) {
+  if (!out || !params) return CCLD_ERR_ARG;
+  *out = nullptr;
+  if (params->tbase_init_ns <= 0 || params->m_max_rounds == 0 || params->m_max_ns <= 0 || params->min_group == 0) return CCLD_ERR_ARG;
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device < 0 || device >= n_dev) return CCLD_ERR_CUDA;
+  if (cudaSetDevice(device) != cudaSuccess) return CCLD_ERR_CUDA;
+  ccld_ctx* ctx = new (std::nothrow) ccld_ctx();
+  if (!ctx) return CCLD_ERR_NOMEM;
+  ctx->params = *params; ctx->device = device; ctx->stream = (cudaStream_t)cuda_stream;
+  Params& d = ctx->dp;
+  d.tbase_init_ns = params->tbase_init_ns; d.m_max_ns = params->m_max_ns; d.hang_ns = params->hang_ns; d.barrier_bytes = params->barrier_bytes;
+  d.theta_slow_milli = params->theta_slow_milli; d.alpha_milli = params->alpha_milli; d.beta_milli = params->beta_milli;
+  d.m_max_rounds = params->m_max_rounds; d.slow_rep_threshold = params->slow_rep_threshold; d.k_milli = params->k_milli;
+  d.min_group = params->min_group; d.vote_rep_milli = params->vote_rep_milli;
+  *out = ctx;
+  return CCLD_OK;
+}
+
+int ccld_destroy(ccld_ctx* ctx) {
+  if (!ctx) return CCLD_ERR_ARG;
+  cudaSetDevice(ctx->device);
+  cudaStreamSynchronize(ctx->stream);
+  for (auto& kv : ctx->windows) { drop_results(kv.second); if (kv.second.owns) ctx->pool.put(kv.second.own); }
+  ctx->windows.clear();
+  ctx->pool.put(ctx->reg_blk); ctx->pool.put(ctx->misc_blk);
+  ctx->pool.clear();
+  if (ctx->h_pinned) cudaFreeHost(ctx->h_pinned);
+  delete ctx;
+  return CCLD_OK;
+}
+
+const char* ccld_last_error(ccld_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+int ccld_comm_register(ccld_ctx* ctx, uint32_t comm, const uint32_t* ranks, uint32_t n, uint8_t algo, uint32_t seq0) {
+  if (!ctx) return CCLD_ERR_ARG;
+  if (ctx->finalized) return fail(ctx, CCLD_ERR_STATE, "communicators must be registered before the first analysis");
+  if (!ranks || n == 0) return fail(ctx, CCLD_ERR_ARG, "empty communicator");
+  if (algo != 0) return fail(ctx, CCLD_ERR_ARG, "only ring communicators (algo 0) are supported");
+  if (n > CCLD_MAX_COMM_SIZE) return fail(ctx, CCLD_ERR_CAPACITY, "communicator larger than CCLD_MAX_COMM_SIZE");
+  if (ctx->comm_idx.count(comm)) return fail(ctx, CCLD_ERR_ARG, "communicator id registered twice");
+  CommHost c; c.id = comm; c.seq0 = seq0; c.ranks.assign(ranks, ranks + n);
+  std::vector<u32> sorted(c.ranks); std::sort(sorted.begin(), sorted.end());
+  if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return fail(ctx, CCLD_ERR_ARG, "rank listed twice in a communicator");
+  if (sorted.back() >= CCLD_MAX_RANK_ID) return fail(ctx, CCLD_ERR_CAPACITY, "rank id not below CCLD_MAX_RANK_ID");
+  ctx->comm_idx[comm] = (u32)ctx->comms.size();
+  ctx->comms.push_back(std::move(c));
+  return CCLD_OK;
+}
+
+int ccld_trace_upload(ccld_ctx* ctx, uint32_t window_id, uint64_t n_rec, int mem_kind,
+                      const uint32_t* rank, const uint32_t* comm, const uint32_t* seq, const uint8_t* op,
+                      const uint64_t* bytes, const int64_t* t_enter_ns, const int64_t* t_exit_ns,
+                      const uint32_t* send_chg, const uint32_t* recv_chg,
+                      uint32_t n_frames, const uint32_t* f_rank, const uint32_t* f_comm, const uint32_t* f_seq,
+                      uint32_t n_channels, const uint32_t* progress) {
+  if (!ctx) return CCLD_ERR_ARG;
+  if (mem_kind != 0 && mem_kind != 1) return fail(ctx, CCLD_ERR_ARG, "mem_kind must be 0 (host) or 1 (device)");
+  if (n_rec >= 0xFFFFFFFFull) return fail(ctx, CCLD_ERR_CAPACITY, "window of 2^32 - 1 or more records");
+  if (n_rec > 0 && (!rank || !comm || !seq || !op || !bytes || !t_enter_ns || !t_exit_ns)) return fail(ctx, CCLD_ERR_ARG, "null column");
+  if ((send_chg == nullptr) != (recv_chg == nullptr)) return fail(ctx, CCLD_ERR_ARG, "send_chg and recv_chg must both be given or both be null");
+  if (n_frames > 0 && (!f_rank || !f_comm || !f_seq || !progress || n_channels == 0)) return fail(ctx, CCLD_ERR_ARG, "incomplete progress frames");
+  if (ctx->windows.count(window_id)) return fail(ctx, CCLD_ERR_STATE, "window id already uploaded");
+  CK(cudaSetDevice(ctx->device));
+  WindowHost w; w.id = window_id; w.n_rec = n_rec; w.n_frames = n_frames; w.n_channels = n_channels;
+  WinDesc& d = w.d;
+  d.n_rec = n_rec;
+  if (mem_kind == 1) {
+    d.rank = rank; d.comm = comm; d.seq = seq; d.op = op; d.bytes = bytes; d.t_enter = t_enter_ns; d.t_exit = t_exit_ns;
+    d.send_chg = send_chg; d.recv_chg = recv_chg;
+    w.f_rank = f_rank; w.f_comm = f_comm; w.f_seq = f_seq; w.progress = progress;
+  } else {
+    size_t off = 0;
+    auto take = [&](size_t b) { size_t o = off; off = align_up(off + b); return o; };
+    const size_t o_rank = take(n_rec * 4), o_comm = take(n_rec * 4), o_seq = take(n_rec * 4), o_op = take(n_rec), o_bytes = take(n_rec * 8),
+                 o_te = take(n_rec * 8), o_tx = take(n_rec * 8), o_sc = take(send_chg ? n_rec * 4 : 0), o_rc = take(recv_chg ? n_rec * 4 : 0),
+                 o_fr = take(n_frames * 4ull), o_fc = take(n_frames * 4ull), o_fs = take(n_frames * 4ull), o_pr = take((size_t)n_frames * n_channels * 8);
+    cudaError_t e;
+    w.own = ctx->pool.get(off, &e);
+    if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "window allocation failed");
+    w.owns = true;
+    char* b = (char*)w.own.p; cudaStream_t st = ctx->stream;
+    auto up = [&](size_t o, const void* src, size_t nb) { return nb ? cudaMemcpyAsync(b + o, src, nb, cudaMemcpyHostToDevice, st) : cudaSuccess; };
+    cudaError_t ce = cudaSuccess;
+    auto acc = [&](cudaError_t x) { if (ce == cudaSuccess) ce = x; };
+    acc(up(o_rank, rank, n_rec * 4)); acc(up(o_comm, comm, n_rec * 4)); acc(up(o_seq, seq, n_rec * 4)); acc(up(o_op, op, n_rec));
+    acc(up(o_bytes, bytes, n_rec * 8)); acc(up(o_te, t_enter_ns, n_rec * 8)); acc(up(o_tx, t_exit_ns, n_rec * 8));
+    if (send_chg) { acc(up(o_sc, send_chg, n_rec * 4)); acc(up(o_rc, recv_chg, n_rec * 4)); }
+    if (n_frames) { acc(up(o_fr, f_rank, n_frames * 4ull)); acc(up(o_fc, f_comm, n_frames * 4ull)); acc(up(o_fs, f_seq, n_frames * 4ull));
+                    acc(up(o_pr, progress, (size_t)n_frames * n_channels * 8)); }
+    if (ce != cudaSuccess) { ctx->pool.put(w.own); return fail(ctx, CCLD_ERR_CUDA, std::string("upload copy: ") + cudaGetErrorString(ce)); }
+    d.rank = (const u32*)(b + o_rank); d.comm = (const u32*)(b + o_comm); d.seq = (const u32*)(b + o_seq); d.op = (const u8*)(b + o_op);
+    d.bytes = (const u64*)(b + o_bytes); d.t_enter = (const i64*)(b + o_te); d.t_exit = (const i64*)(b + o_tx);
+    d.send_chg = send_chg ? (const u32*)(b + o_sc) : nullptr; d.recv_chg = recv_chg ? (const u32*)(b + o_rc) : nullptr;
+    if (n_frames) { w.f_rank = (const u32*)(b + o_fr); w.f_comm = (const u32*)(b + o_fc); w.f_seq = (const u32*)(b + o_fs); w.progress = (const u32*)(b + o_pr); }
+  }
+  ctx->windows.emplace(window_id, std::move(w));
+  return CCLD_OK;
+}
+
+int ccld_window_release(ccld_ctx* ctx, uint32_t window_id) {
+  if (!ctx) return CCLD_ERR_ARG;
+  auto it = ctx->windows.find(window_id);
+  if (it == ctx->windows.end()) return fail(ctx, CCLD_ERR_NO_WINDOW, "unknown window id");
+  CK(cudaSetDevice(ctx->device));
+  CK(cudaStreamSynchronize(ctx->stream));     // nothing in flight may still read the blocks we recycle
+  drop_results(it->second);
+  if (it->second.owns) ctx->pool.put(it->second.own);
+  ctx->windows.erase(it);
+  return CCLD_OK;
+}
+
+int ccld_reset(ccld_ctx* ctx) {
+  if (!ctx) return CCLD_ERR_ARG;
+  CK(cudaSetDevice(ctx->device));
+  CK(cudaStreamSynchronize(ctx->stream));
+  for (auto& kv : ctx->windows) drop_results(kv.second);
+  if (ctx->finalized) CK(cudaMemsetAsync((char*)ctx->reg_blk.p + ctx->stats_off, 0, ctx->stats_bytes, ctx->stream));
+  return CCLD_OK;
+}
+
+int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows, int64_t now_ns) {
+  if (!ctx) return CCLD_ERR_ARG;
+  if (n_windows == 0) return fail(ctx, CCLD_ERR_ARG, "n_windows is zero");
+  CK(cudaSetDevice(ctx->device));
+  std::vector<WindowHost*> ws(n_windows);
+  for (u32 k = 0; k < n_windows; ++k) {
+    auto it = ctx->windows.find(first_window + k);
+    if (it == ctx->windows.end()) return fail(ctx, CCLD_ERR_NO_WINDOW, "window not uploaded");
+    if (it->second.analysed) return fail(ctx, CCLD_ERR_STATE, "window already analysed");
+    ws[k] = &it->second;
+  }
+  { int rc = finalize_registry(ctx); if (rc != CCLD_OK) return rc; }
+  const u32 B = n_windows, nc = ctx->reg.n_comms;
+  cudaStream_t st = ctx->stream;
+
+  // ---- plan block: descriptors, op-counter ranges, layout rows, totals, counters ----
+  size_t off = 0;
+  auto take = [&](size_t b) { size_t o = off; off = align_up(off + b); return o; };
+  const size_t o_desc = take(B * sizeof(WinDesc)), o_rmin = take((size_t)B * nc * 4), o_rmax = take((size_t)B * nc * 4),
+               o_rng = take((size_t)B * nc * sizeof(RangeRow)), o_tot = take((size_t)B * T_COUNT * 8), o_cnt = take((size_t)B * C_COUNT * 8);
+  cudaError_t e;
+  Block pb = ctx->pool.get(off, &e);
+  if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "plan allocation failed");
+  auto plan_blk = std::make_shared<Shared>(&ctx->pool, pb);
+  char* pbase = (char*)pb.p;
+  std::vector<WinDesc> hd(B);
+  u64 cta = 0;
+  for (u32 k = 0; k < B; ++k) {
+    WinDesc d = ws[k]->d;
+    d.slot_cap = 2 * d.n_rec + ctx->sum_n;
+    d.n_cta = (u32)((d.n_rec + REC_PER_CTA - 1) / REC_PER_CTA); d.cta0 = (u32)cta; cta += d.n_cta;
+    d.rmin = (u32*)(pbase + o_rmin) + (size_t)k * nc; d.rmax = (u32*)(pbase + o_rmax) + (size_t)k * nc;
+    d.ranges = (RangeRow*)(pbase + o_rng) + (size_t)k * nc;
+    d.totals = (u64*)(pbase + o_tot) + (size_t)k * T_COUNT; d.counters = (u64*)(pbase + o_cnt) + (size_t)k * C_COUNT;
+    d.n_groups = d.n_slots = 0; d.perm = nullptr; d.flags = nullptr; d.gi64 = nullptr; d.gu32 = nullptr; d.gbw = nullptr;
+    d.comm_rows = nullptr; d.alerts = nullptr; d.tile0[0] = d.tile0[1] = d.tile0[2] = 0; d.pad = 0;
+    hd[k] = d;
+  }
+  if (cta > 0x7FFFFFFFull) return fail(ctx, CCLD_ERR_CAPACITY, "batch too large for one launch");
+  WinDesc* d_desc = (WinDesc*)(pbase + o_desc);
+  CK(cudaMemsetAsync(pbase, 0, off, st));
+  CK(cudaMemsetAsync(pbase + o_rmin, 0xFF, (size_t)B * nc * 4, st));
+  CK(cudaMemcpyAsync(d_desc, hd.data(), B * sizeof(WinDesc), cudaMemcpyHostToDevice, st));
+  if (cta > 0) k_seq_range<<<(u32)cta, REC_THREADS, 0, st>>>(d_desc, B, ctx->reg);
+  k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, nullptr, nullptr, nullptr, 0);
+  CK(cudaGetLastError());
+  { int rc = ensure_pinned(ctx, (size_t)B * T_COUNT * 8); if (rc != CCLD_OK) return rc; }
+  CK(cudaMemcpyAsync(ctx->h_pinned, pbase + o_tot, (size_t)B * T_COUNT * 8, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+
+  // ---- result block: sized from the plan ----
+  off = 0;
+  u64 total_slots = 0, n_tiles[3] = {0, 0, 0};
+  for (u32 k = 0; k < B; ++k) { const u64* t = ctx->h_pinned + (size_t)k * T_COUNT; total_slots += t[T_SLOTS]; }
+  const size_t o_perm = take(total_slots * 4 + ALIGN);
+  std::vector<size_t> o_flags(B), o_gi(B), o_gu(B), o_gb(B), o_rows(B), o_al(B), perm_off(B);
+  { size_t po = 0;
+    for (u32 k = 0; k < B; ++k) {
+      const u64* t = ctx->h_pinned + (size_t)k * T_COUNT;
+      perm_off[k] = po; po += t[T_SLOTS] * 4;
+      o_flags[k] = take(t[T_SLOTS]); o_gi[k] = take(t[T_GROUPS] * 8 * GI_COUNT); o_gu[k] = take(t[T_GROUPS] * 4 * GU_COUNT);
+      o_gb[k] = take(t[T_GROUPS] * 8); o_rows[k] = take(t[T_ROWS] * sizeof(ccld_comm_verdict));
+      o_al[k] = take(CCLD_MAX_ALERTS_PER_WINDOW * sizeof(ccld_hang_alert));
+      hd[k].tile0[0] = (u32)n_tiles[0]; hd[k].tile0[1] = (u32)n_tiles[1]; hd[k].tile0[2] = (u32)n_tiles[2];
+      n_tiles[0] += t[T_TILES0]; n_tiles[1] += t[T_TILES1]; n_tiles[2] += t[T_TILES2];
+    } }
+  for (int q = 0; q < 3; ++q) if (n_tiles[q] > 0x7FFFFFFFull) return fail(ctx, CCLD_ERR_CAPACITY, "too many tiles in one batch");
+  const size_t o_t0 = take(n_tiles[0] * sizeof(Tile)), o_t1 = take(n_tiles[1] * sizeof(Tile)), o_t2 = take(n_tiles[2] * sizeof(Tile));
+  Block rb = ctx->pool.get(off, &e);
+  if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "result allocation failed");
+  auto res_blk = std::make_shared<Shared>(&ctx->pool, rb);
+  char* rbase = (char*)rb.p;
+  for (u32 k = 0; k < B; ++k) {
+    const u64* t = ctx->h_pinned + (size_t)k * T_COUNT;
+    WinDesc& d = hd[k];
+    d.n_groups = t[T_GROUPS]; d.n_slots = t[T_SLOTS];
+    d.perm = (u32*)(rbase + o_perm + perm_off[k]); d.flags = (u8*)(rbase + o_flags[k]);
+    d.gi64 = (i64*)(rbase + o_gi[k]); d.gu32 = (u32*)(rbase + o_gu[k]); d.gbw = (double*)(rbase + o_gb[k]);
+    d.comm_rows = (ccld_comm_verdict*)(rbase + o_rows[k]); d.alerts = (ccld_hang_alert*)(rbase + o_al[k]);
+  }
+  CK(cudaMemcpyAsync(d_desc, hd.data(), B * sizeof(WinDesc), cudaMemcpyHostToDevice, st));
+  if (total_slots) CK(cudaMemsetAsync(rbase + o_perm, 0xFF, total_slots * 4, st));
+  Tile *t0 = (Tile*)(rbase + o_t0), *t1 = (Tile*)(rbase + o_t1), *t2 = (Tile*)(rbase + o_t2);
+  k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, t0, t1, t2, 1);
+  if (cta > 0) k_slot_scatter<<<(u32)cta, REC_THREADS, 0, st>>>(d_desc, B, ctx->reg);
+  if (n_tiles[0]) k_reduce_small<<<(u32)n_tiles[0], SMALL_SEQS, 0, st>>>(d_desc, t0, ctx->reg, ctx->dp, now_ns);
+  if (n_tiles[1]) k_reduce_mid<<<(u32)n_tiles[1], MID_THREADS, mid_smem_bytes(16), st>>>(d_desc, t1, ctx->reg, ctx->dp, now_ns);
+  if (n_tiles[2]) k_reduce_large<<<(u32)n_tiles[2], LARGE_THREADS, 16ull * ctx->max_large_n, st>>>(d_desc, t2, ctx->reg, ctx->dp, now_ns);
+  k_window_decide<<<(nc + 3) / 4, 128, 0, st>>>(d_desc, B, ctx->reg, ctx->dp);
+  CK(cudaGetLastError());
+  for (u32 k = 0; k < B; ++k) {
+    WindowHost& w = *ws[k];
+    w.analysed = true; w.plan_blk = plan_blk; w.res_blk = res_blk; w.d_desc = d_desc + k; w.d = hd[k];
+    std::memcpy(w.totals, ctx->h_pinned + (size_t)k * T_COUNT, sizeof w.totals);
+  }
+  return CCLD_OK;
+}
+
+int ccld_get_verdict(ccld_ctx* ctx, uint32_t window_id, ccld_verdict* out) {
+  if (!ctx || !out) return CCLD_ERR_ARG;
+  WindowHost* w;
+  { int rc = find_analysed(ctx, window_id, &w); if (rc != CCLD_OK) return rc; }
+  CK(cudaSetDevice(ctx->device));
+  cudaStream_t st = ctx->stream;
+  u64 cnt[C_COUNT];
+  CK(cudaMemcpyAsync(cnt, w->d.counters, sizeof cnt, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  out->n_records = w->n_rec; out->n_groups = w->totals[T_GROUPS]; out->n_slots = w->totals[T_SLOTS];
+  out->n_rejected = w->n_rec - cnt[C_PRESENT]; out->n_complete = cnt[C_COMPLETE]; out->n_incomplete = cnt[C_INCOMPLETE];
+  out->n_barrier = cnt[C_BARRIER]; out->n_analysed = cnt[C_ANALYSED]; out->n_flag_skew = cnt[C_FLAG_SKEW]; out->n_flag_dur = cnt[C_FLAG_DUR];
+  out->n_opset_mismatch = cnt[C_MISMATCH];
+  u32 err = (u32)cnt[C_ERR];
+  if (!w->totals[T_FAILED] && w->n_rec - cnt[C_PRESENT] != cnt[C_REJECTED]) err |= CCLD_E_DUPLICATE;   // a slot was written twice
+  out->error_bits = err;
+  out->n_comm_rows_total = (u32)w->totals[T_ROWS];
+  const u32 n_rows = std::min<u32>(out->n_comm_rows_total, out->comm_rows ? out->comm_rows_cap : 0);
+  if (n_rows) CK(cudaMemcpyAsync(out->comm_rows, w->d.comm_rows, n_rows * sizeof(ccld_comm_verdict), cudaMemcpyDeviceToHost, st));
+  char* m = (char*)ctx->misc_blk.p;
+  const MiscLayout L = misc_layout(ctx->n_ranks, ctx->max_n);
+  ccld_suspect* sus_a = (ccld_suspect*)(m + L.sus_a); ccld_suspect* sus_b = (ccld_suspect*)(m + L.sus_b);
+  ccld_hang_alert* al_b = (ccld_hang_alert*)(m + L.alerts);
+  u32* d_count = (u32*)(m + L.count);
+  // hang alerts, ordered by (communicator, seq)
+  out->n_alerts_total = (u32)std::min<u64>(cnt[C_ALERTS], 0xFFFFFFFFull);
+  const u32 n_al_dev = std::min<u32>(out->n_alerts_total, CCLD_MAX_ALERTS_PER_WINDOW);
+  const u32 n_al = std::min<u32>(n_al_dev, out->alerts ? out->alerts_cap : 0);
+  if (n_al) {
+    k_rank_sort_alerts<<<(n_al_dev + 127) / 128, 128, 0, st>>>(w->d.alerts, n_al_dev, al_b, ctx->reg);
+    CK(cudaGetLastError());
+    CK(cudaMemcpyAsync(out->alerts, al_b, n_al * sizeof(ccld_hang_alert), cudaMemcpyDeviceToHost, st));
+  }
+  // cumulative suspects
+  const u32 sus_cap = 2 * ctx->n_ranks;
+  u32 n_sus = 0;
+  CK(cudaMemsetAsync(d_count, 0, 4, st));
+  k_suspects<<<(ctx->n_ranks + 255) / 256, 256, 0, st>>>(ctx->reg, ctx->dp, sus_a, sus_cap, d_count);
+  CK(cudaGetLastError());
+  CK(cudaMemcpyAsync(&n_sus, d_count, 4, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  out->n_suspects_total = n_sus;
+  const u32 n_out = std::min<u32>(n_sus, out->suspects ? out->suspects_cap : 0);
+  if (n_out) {
+    k_rank_sort_suspects<<<(n_sus + 127) / 128, 128, 0, st>>>(sus_a, n_sus, sus_b);
+    CK(cudaGetLastError());
+    CK(cudaMemcpyAsync(out->suspects, sus_b, n_out * sizeof(ccld_suspect), cudaMemcpyDeviceToHost, st));
+  }
+  CK(cudaStreamSynchronize(st));
+  if (cnt[C_INTERNAL]) return fail(ctx, CCLD_ERR_CUDA, "internal: slot index out of range");
+  if (err & CCLD_E_UNKNOWN_COMM) return fail(ctx, CCLD_ERR_UNKNOWN_COMM, "record of an unregistered communicator");
+  if (err & CCLD_E_NOT_MEMBER) return fail(ctx, CCLD_ERR_NOT_MEMBER, "record of a rank that is not a member of its communicator");
+  if (err & CCLD_E_SEQ_RANGE) return fail(ctx, CCLD_ERR_SEQ_RANGE, "record with an op counter below the communicator's first");
+  if (err & CCLD_E_DUPLICATE) return fail(ctx, CCLD_ERR_DUPLICATE, "duplicate (communicator, op counter, rank) record");
+  if (err & CCLD_E_CAPACITY) return fail(ctx, CCLD_ERR_CAPACITY, "op counters of the window span too many slots");
+  return CCLD_OK;
+}
+
+int ccld_locate_hang(ccld_ctx* ctx, uint32_t window_id, uint32_t comm, uint32_t seq, ccld_hang_verdict* out) {
+  if (!ctx || !out) return CCLD_ERR_ARG;
+  WindowHost* w;
+  { int rc = find_analysed(ctx, window_id, &w); if (rc != CCLD_OK) return rc; }
+  auto ci = ctx->comm_idx.find(comm);
+  if (ci == ctx->comm_idx.end()) return fail(ctx, CCLD_ERR_UNKNOWN_COMM, "unknown communicator");
+  CK(cudaSetDevice(ctx->device));
+  cudaStream_t st = ctx->stream;
+  const u32 n = (u32)ctx->comms[ci->second].ranks.size();
+  char* m = (char*)ctx->misc_blk.p;
+  const MiscLayout L = misc_layout(ctx->n_ranks, ctx->max_n);
+  HangArgs A;
+  A.c = ci->second; A.seq = seq; A.n_frames = w->n_frames; A.n_channels = w->n_channels;
+  A.f_rank = w->f_rank; A.f_comm = w->f_comm; A.f_seq = w->f_seq; A.progress = w->progress;
+  A.entered = (u8*)(m + L.entered); A.done = (u8*)(m + L.done); A.frame = (u32*)(m + L.frame); A.roots = (u32*)(m + L.roots);
+  A.tot = (u64*)(m + L.tot); A.out = (ccld_hang_verdict*)(m + L.hang_out);
+  A.roots_cap = n;
+  k_hang_locate<<<1, 1024, 0, st>>>(w->d_desc, ctx->reg, A);
+  CK(cudaGetLastError());
+  ccld_hang_verdict v;
+  CK(cudaMemcpyAsync(&v, A.out, sizeof v, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  u32* roots = out->roots; const u32 cap = roots ? out->roots_cap : 0;
+  *out = v; out->roots = roots; out->roots_cap = cap;
+  const u32 n_copy = std::min<u32>(std::min<u32>(v.n_roots_total, n), cap);
+  if (n_copy) { CK(cudaMemcpyAsync(roots, A.roots, n_copy * 4ull, cudaMemcpyDeviceToHost, st)); CK(cudaStreamSynchronize(st)); }
+  return CCLD_OK;
+}
+
+int ccld_get_optable(ccld_ctx* ctx, uint32_t window_id, ccld_optable* out) {
+  if (!ctx || !out) return CCLD_ERR_ARG;
+  WindowHost* w;
+  { int rc = find_analysed(ctx, window_id, &w); if (rc != CCLD_OK) return rc; }
+  const WinDesc& d = w->d; const u64 G = d.n_groups;
+  out->n_groups = G; out->n_slots = d.n_slots;
+  const i64* gi = d.gi64; const u32* gu = d.gu32;
+  out->e_min = gi + GI_E_MIN * G; out->arrival_skew = gi + GI_ARRIVAL_SKEW * G; out->t_max = gi + GI_T_MAX * G; out->t_min = gi + GI_T_MIN * G;
+  out->span = gi + GI_SPAN * G; out->med_skew = gi + GI_MED_SKEW * G; out->mad_skew = gi + GI_MAD_SKEW * G;
+  out->med_dur = gi + GI_MED_DUR * G; out->mad_dur = gi + GI_MAD_DUR * G;
+  out->rank_tmin = gu + GU_RANK_TMIN * G; out->rank_tmax = gu + GU_RANK_TMAX * G; out->max_chg = gu + GU_MAX_CHG * G;
+  out->rank_max_chg = gu + GU_RANK_MAX_CHG * G; out->n_present = gu + GU_N_PRESENT * G; out->gflags = gu + GU_GFLAGS * G;
+  out->busbw = d.gbw; out->flags = d.flags; out->perm = d.perm;
+  return CCLD_OK;
+}
+
+int ccld_get_ranges(ccld_ctx* ctx, uint32_t window_id, ccld_comm_range* rows, uint32_t cap, uint32_t* n_total) {
+  if (!ctx || !n_total) return CCLD_ERR_ARG;
+  WindowHost* w;
+  { int rc = find_analysed(ctx, window_id, &w); if (rc != CCLD_OK) return rc; }
+  CK(cudaSetDevice(ctx->device));
+  const u32 nc = ctx->reg.n_comms;
+  std::vector<RangeRow> rr(nc);
+  CK(cudaMemcpyAsync(rr.data(), w->d.ranges, nc * sizeof(RangeRow), cudaMemcpyDeviceToHost, ctx->stream));
+  CK(cudaStreamSynchronize(ctx->stream));
+  u32 k = 0;
+  for (u32 c = 0; c < nc; ++c) {
+    if (rr[c].n_seq == 0) continue;
+    if (rows && k < cap) { rows[k].comm = ctx->comms[c].id; rows[k].n = rr[c].n; rows[k].seq_lo = rr[c].seq_lo; rows[k].n_seq = rr[c].n_seq;
+                           rows[k].group0 = rr[c].group0; rows[k].slot0 = rr[c].slot0; }
+    ++k;
+  }
+  *n_total = k;
+  return CCLD_OK;
+}
+
+int ccld_get_rank_stats(ccld_ctx* ctx, uint32_t n_ranks, uint32_t* votes, uint32_t* ops, uint32_t* bw_cnt, double* bw_sum) {
+  if (!ctx || !votes || !ops || !bw_cnt || !bw_sum) return CCLD_ERR_ARG;
+  if (!ctx->finalized) return fail(ctx, CCLD_ERR_STATE, "nothing analysed yet");
+  CK(cudaSetDevice(ctx->device));
+  std::memset(votes, 0, (size_t)n_ranks * 16); std::memset(ops, 0, (size_t)n_ranks * 4);
+  std::memset(bw_cnt, 0, (size_t)n_ranks * 4); std::memset(bw_sum, 0, (size_t)n_ranks * 8);
+  const u32 n = std::min(n_ranks, ctx->reg.n_ranks);
+  cudaStream_t st = ctx->stream;
+  CK(cudaMemcpyAsync(votes, ctx->reg.votes, (size_t)n * 16, cudaMemcpyDeviceToHost, st));
+  CK(cudaMemcpyAsync(ops, ctx->reg.ops, (size_t)n * 4, cudaMemcpyDeviceToHost, st));
+  CK(cudaMemcpyAsync(bw_cnt, ctx->reg.bw_cnt, (size_t)n * 4, cudaMemcpyDeviceToHost, st));
+  CK(cudaMemcpyAsync(bw_sum, ctx->reg.bw_sum, (size_t)n * 8, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  return CCLD_OK;
+}
+
+int ccld_copy_to_host(ccld_ctx* ctx, void* dst_host, const void* src_device, uint64_t bytes) {
+  if (!ctx || (bytes && (!dst_host || !src_device))) return CCLD_ERR_ARG;
+  CK(cudaSetDevice(ctx->device));
+  if (bytes) CK(cudaMemcpyAsync(dst_host, src_device, bytes, cudaMemcpyDeviceToHost, ctx->stream));
+  CK(cudaStreamSynchronize(ctx->stream));
+  return CCLD_OK;
+}
+
+}  // extern "C"
