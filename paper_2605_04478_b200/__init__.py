@@ -24,7 +24,9 @@ MAX_ALERTS_PER_WINDOW = 1024
 
 EXPORTS = ("ccld_params_default", "ccld_create", "ccld_destroy", "ccld_last_error", "ccld_comm_register",
            "ccld_trace_upload", "ccld_window_release", "ccld_analyze_window", "ccld_reset", "ccld_get_verdict",
-           "ccld_locate_hang", "ccld_get_optable", "ccld_get_ranges", "ccld_get_rank_stats", "ccld_copy_to_host")
+           "ccld_locate_hang", "ccld_get_optable", "ccld_get_ranges", "ccld_get_rank_stats", "ccld_copy_to_host",
+           "ccld_timing_enable", "ccld_get_kernel_times")
+KERNEL_KINDS = ("k_seq_range", "k_plan", "k_slot_scatter", "k_reduce_small", "k_reduce_mid", "k_reduce_large", "k_window_decide")
 
 
 class CcldError(RuntimeError):
@@ -117,6 +119,8 @@ def load_library() -> C.CDLL:
         lib.ccld_get_ranges.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.POINTER(C.c_uint32)]
         lib.ccld_get_rank_stats.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.ccld_copy_to_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64]
+        lib.ccld_timing_enable.argtypes = [C.c_void_p, C.c_int]
+        lib.ccld_get_kernel_times.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         _lib = lib
     return _lib
 
@@ -298,6 +302,15 @@ class Analyzer:
         out["seq"] = (np.repeat(r["seq_lo"].astype(np.int64), ns) + within).astype(np.uint32)
         out["slot0"] = (np.repeat(r["slot0"].astype(np.int64), ns) + within * np.repeat(r["n"].astype(np.int64), ns)).astype(np.uint64)
         return out
+
+    def timing_enable(self, on: bool = True) -> None:
+        self._check(self.lib.ccld_timing_enable(self.h, 1 if on else 0))
+
+    def get_kernel_times(self) -> Dict[str, Dict[str, float]]:
+        """Per kernel kind: summed device milliseconds and launches since timing was enabled."""
+        ms = np.zeros(len(KERNEL_KINDS), np.float64); n = np.zeros(len(KERNEL_KINDS), np.uint64)
+        self._check(self.lib.ccld_get_kernel_times(self.h, ms.ctypes.data, n.ctypes.data))
+        return {k: {"ms": float(ms[i]), "launches": int(n[i])} for i, k in enumerate(KERNEL_KINDS)}
 
     def get_rank_stats(self, n_ranks: int) -> Dict[str, np.ndarray]:
         votes = np.zeros((n_ranks, 4), np.uint32); ops = np.zeros(n_ranks, np.uint32)

@@ -65,6 +65,10 @@ struct WindowHost {
   WindowHost() { std::memset(&d, 0, sizeof d); std::memset(totals, 0, sizeof totals); }
 };
 
+constexpr u32 TIMER_RING = 32;
+constexpr int TIMER_PAIRS = CCLD_K_KINDS + 1;          // the layout kernel runs twice per call
+struct TimerSlot { cudaEvent_t a[TIMER_PAIRS], b[TIMER_PAIRS]; int kind[TIMER_PAIRS]; int n = 0; };
+
 }  // namespace
 
 struct ccld_ctx {
@@ -75,7 +79,10 @@ struct ccld_ctx {
   std::map<u32, WindowHost> windows;
   Pool pool; std::string err;
   u64* h_pinned = nullptr; size_t h_pinned_bytes = 0;
-  ccld_ctx() { std::memset(&reg, 0, sizeof reg); }
+  // optional per-kernel timing: a ring of event pairs, harvested lazily
+  bool timing = false; std::vector<TimerSlot> ring; u32 ring_next = 0;
+  double t_ms[CCLD_K_KINDS]; u64 t_launches[CCLD_K_KINDS];
+  ccld_ctx() { std::memset(&reg, 0, sizeof reg); std::memset(t_ms, 0, sizeof t_ms); std::memset(t_launches, 0, sizeof t_launches); }
 };
 
 namespace {
@@ -95,6 +102,30 @@ int ensure_pinned(ccld_ctx* ctx, size_t bytes) {
   ctx->h_pinned_bytes = bytes;
   return CCLD_OK;
 }
+
+// Adds the elapsed times of a slot's finished event pairs to the sums (waits for the last one).
+void timer_harvest(ccld_ctx* ctx, TimerSlot& s) {
+  for (int i = 0; i < s.n; ++i) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(s.b[i]) == cudaSuccess && cudaEventElapsedTime(&ms, s.a[i], s.b[i]) == cudaSuccess) {
+      ctx->t_ms[s.kind[i]] += ms; ctx->t_launches[s.kind[i]] += 1;
+    }
+  }
+  s.n = 0;
+}
+TimerSlot* timer_begin(ccld_ctx* ctx) {
+  if (!ctx->timing) return nullptr;
+  TimerSlot& s = ctx->ring[ctx->ring_next++ % TIMER_RING];
+  timer_harvest(ctx, s);
+  return &s;
+}
+struct TimedLaunch {                                     // records an event pair around one launch
+  TimerSlot* s; cudaStream_t st; int i;
+  TimedLaunch(TimerSlot* slot, int kind, cudaStream_t stream) : s(slot), st(stream), i(-1) {
+    if (s && s->n < TIMER_PAIRS) { i = s->n++; s->kind[i] = kind; cudaEventRecord(s->a[i], st); }
+  }
+  ~TimedLaunch() { if (i >= 0) cudaEventRecord(s->b[i], st); }
+};
 
 // Layout of the scratch block used by get_verdict and locate_hang.
 struct MiscLayout { size_t sus_a, sus_b, alerts, count, entered, done, frame, roots, tot, hang_out, total; };
@@ -234,6 +265,7 @@ int ccld_destroy(ccld_ctx* ctx) {
   ctx->pool.put(ctx->reg_blk); ctx->pool.put(ctx->misc_blk);
   ctx->pool.clear();
   if (ctx->h_pinned) cudaFreeHost(ctx->h_pinned);
+  for (auto& sl : ctx->ring) for (int i = 0; i < TIMER_PAIRS; ++i) { cudaEventDestroy(sl.a[i]); cudaEventDestroy(sl.b[i]); }
   delete ctx;
   return CCLD_OK;
 }
@@ -370,8 +402,9 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   CK(cudaMemsetAsync(pbase, 0, off, st));
   CK(cudaMemsetAsync(pbase + o_rmin, 0xFF, (size_t)B * nc * 4, st));
   CK(cudaMemcpyAsync(d_desc, hd.data(), B * sizeof(WinDesc), cudaMemcpyHostToDevice, st));
-  if (cta > 0) k_seq_range<<<(u32)cta, REC_THREADS, 0, st>>>(d_desc, B, ctx->reg);
-  k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, nullptr, nullptr, nullptr, 0);
+  TimerSlot* ts = timer_begin(ctx);
+  if (cta > 0) { TimedLaunch tl(ts, 0, st); k_seq_range<<<(u32)cta, REC_THREADS, 0, st>>>(d_desc, B, ctx->reg); }
+  { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, nullptr, nullptr, nullptr, 0); }
   CK(cudaGetLastError());
   { int rc = ensure_pinned(ctx, (size_t)B * T_COUNT * 8); if (rc != CCLD_OK) return rc; }
   CK(cudaMemcpyAsync(ctx->h_pinned, pbase + o_tot, (size_t)B * T_COUNT * 8, cudaMemcpyDeviceToHost, st));
@@ -410,12 +443,12 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   CK(cudaMemcpyAsync(d_desc, hd.data(), B * sizeof(WinDesc), cudaMemcpyHostToDevice, st));
   if (total_slots) CK(cudaMemsetAsync(rbase + o_perm, 0xFF, total_slots * 4, st));
   Tile *t0 = (Tile*)(rbase + o_t0), *t1 = (Tile*)(rbase + o_t1), *t2 = (Tile*)(rbase + o_t2);
-  k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, t0, t1, t2, 1);
-  if (cta > 0) k_slot_scatter<<<(u32)cta, REC_THREADS, 0, st>>>(d_desc, B, ctx->reg);
-  if (n_tiles[0]) k_reduce_small<<<(u32)n_tiles[0], SMALL_SEQS, 0, st>>>(d_desc, t0, ctx->reg, ctx->dp, now_ns);
-  if (n_tiles[1]) k_reduce_mid<<<(u32)n_tiles[1], MID_THREADS, mid_smem_bytes(16), st>>>(d_desc, t1, ctx->reg, ctx->dp, now_ns);
-  if (n_tiles[2]) k_reduce_large<<<(u32)n_tiles[2], LARGE_THREADS, 16ull * ctx->max_large_n, st>>>(d_desc, t2, ctx->reg, ctx->dp, now_ns);
-  k_window_decide<<<(nc + 3) / 4, 128, 0, st>>>(d_desc, B, ctx->reg, ctx->dp);
+  { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, t0, t1, t2, 1); }
+  if (cta > 0) { TimedLaunch tl(ts, 2, st); k_slot_scatter<<<(u32)cta, REC_THREADS, 0, st>>>(d_desc, B, ctx->reg); }
+  if (n_tiles[0]) { TimedLaunch tl(ts, 3, st); k_reduce_small<<<(u32)n_tiles[0], SMALL_SEQS, 0, st>>>(d_desc, t0, ctx->reg, ctx->dp, now_ns); }
+  if (n_tiles[1]) { TimedLaunch tl(ts, 4, st); k_reduce_mid<<<(u32)n_tiles[1], MID_THREADS, mid_smem_bytes(16), st>>>(d_desc, t1, ctx->reg, ctx->dp, now_ns); }
+  if (n_tiles[2]) { TimedLaunch tl(ts, 5, st); k_reduce_large<<<(u32)n_tiles[2], LARGE_THREADS, 16ull * ctx->max_large_n, st>>>(d_desc, t2, ctx->reg, ctx->dp, now_ns); }
+  { TimedLaunch tl(ts, 6, st); k_window_decide<<<(nc + 3) / 4, 128, 0, st>>>(d_desc, B, ctx->reg, ctx->dp); }
   CK(cudaGetLastError());
   for (u32 k = 0; k < B; ++k) {
     WindowHost& w = *ws[k];
@@ -561,6 +594,29 @@ int ccld_get_rank_stats(ccld_ctx* ctx, uint32_t n_ranks, uint32_t* votes, uint32
   CK(cudaMemcpyAsync(bw_cnt, ctx->reg.bw_cnt, (size_t)n * 4, cudaMemcpyDeviceToHost, st));
   CK(cudaMemcpyAsync(bw_sum, ctx->reg.bw_sum, (size_t)n * 8, cudaMemcpyDeviceToHost, st));
   CK(cudaStreamSynchronize(st));
+  return CCLD_OK;
+}
+
+int ccld_timing_enable(ccld_ctx* ctx, int on) {
+  if (!ctx) return CCLD_ERR_ARG;
+  CK(cudaSetDevice(ctx->device));
+  CK(cudaStreamSynchronize(ctx->stream));
+  if (on && ctx->ring.empty()) {
+    ctx->ring.resize(TIMER_RING);
+    for (auto& sl : ctx->ring) for (int i = 0; i < TIMER_PAIRS; ++i) { CK(cudaEventCreate(&sl.a[i])); CK(cudaEventCreate(&sl.b[i])); }
+  }
+  for (auto& sl : ctx->ring) sl.n = 0;
+  std::memset(ctx->t_ms, 0, sizeof ctx->t_ms); std::memset(ctx->t_launches, 0, sizeof ctx->t_launches);
+  ctx->timing = on != 0;
+  return CCLD_OK;
+}
+
+int ccld_get_kernel_times(ccld_ctx* ctx, double* ms, uint64_t* launches) {
+  if (!ctx || !ms || !launches) return CCLD_ERR_ARG;
+  CK(cudaSetDevice(ctx->device));
+  CK(cudaStreamSynchronize(ctx->stream));
+  for (auto& sl : ctx->ring) timer_harvest(ctx, sl);
+  for (int k = 0; k < CCLD_K_KINDS; ++k) { ms[k] = ctx->t_ms[k]; launches[k] = ctx->t_launches[k]; }
   return CCLD_OK;
 }
 

@@ -1,0 +1,294 @@
+"""Parity of the CUDA library with the CPU oracle, through the C ABI, on the same seeded inputs.
+
+Integer quantities (skews, durations, medians, MADs, flags, votes, roots) must be identical;
+fp64 bandwidths, R and P within 1e-9 relative.
+"""
+import numpy as np
+import pytest
+import torch
+
+import tracegen as tg
+from helpers import ALLGATHER, MiB, frames_from, group_trace, make_cols
+from parity import compare_cumulative, compare_hang, compare_window, make_pair
+
+pytestmark = pytest.mark.gpu
+
+
+def run_spec(spec, windows=None, order="rank_major", batch=True, device="cpu", params=None):
+    """Uploads the given windows of `spec` to both sides, analyses them and compares everything."""
+    reg = tg.registry(spec)
+    an, o = make_pair(reg, params)
+    windows = list(range(spec.n_windows)) if windows is None else windows
+    wins = []
+    for w in windows:
+        win = tg.gen_window(spec, w, device=device, order=order)
+        wins.append(win)
+        an.trace_upload(w, win.cols, win.frames, win.n_channels)
+        assert o.upload(w, win.cols, win.frames, win.n_channels) == 0
+    now = wins[-1].now_ns
+    if batch:
+        an.analyze_window(windows[0], len(windows), now)
+    else:
+        for w in windows:
+            an.analyze_window(w, 1, now)
+    assert o.analyze(windows[0], len(windows), now) == 0
+    verdicts = [compare_window(an, o, w)[0] for w in windows]
+    sus = compare_cumulative(an, o, spec.n_ranks, windows[-1])
+    return an, o, verdicts, sus
+
+
+# ---------------------------------------------------------------- the benchmark configurations
+def test_cfg1_tiny_slow_case():
+    spec = tg.cfg1()
+    an, o, v, sus = run_spec(spec)
+    assert v[0]["n_records"] == 8000 and v[0]["n_groups"] == 1000
+    assert sorted(set(sus["rank"])) == [5] and list(sus["kind"]) == [1]
+
+
+def test_cfg2_full_size_512_ranks():
+    spec = tg.cfg2()
+    an, o, v, sus = run_spec(spec)
+    assert sum(x["n_records"] for x in v) == 15_360_000
+    assert sorted(set(int(r) for r in sus["rank"][sus["kind"] == 1])) == spec.truth["stragglers"]
+    assert sorted(set(int(r) for r in sus["rank"][sus["kind"] == 2])) == spec.truth["slow_links"]
+
+
+@pytest.mark.parametrize("order", ["arrival", "shuffled"])
+def test_cfg2_other_upload_orders(order):
+    spec = tg.cfg2(reps=100, n_windows=2)
+    run_spec(spec, order=order, batch=False)
+
+
+def test_cfg3_hang_case():
+    spec = tg.cfg3()
+    an, o, v, sus = run_spec(spec)
+    a = v[0]["alerts"]
+    assert list(a["comm"]) == [7] and list(a["seq"]) == [100]
+    h = compare_hang(an, o, 0, 7, 100)
+    assert h["cls"] == 3 and list(h["roots"]) == [1793] and h["stuck_step"] == 23
+    compare_hang(an, o, 0, 3, 100)       # a ring that completed
+    compare_hang(an, o, 0, 7, 101)       # an op nobody entered
+    compare_hang(an, o, 0, 7, 50)
+
+
+def test_cfg4_scaled_three_windows_device_resident():
+    # same structure as the streaming configuration (4,096 ranks, TP8 x PP8 x DP64), 100 ops per rank and window,
+    # generated on the GPU and borrowed by the library
+    spec = tg.cfg4(reps=20, n_windows=3)
+    an, o, v, sus = run_spec(spec, device="cuda")
+    assert v[0]["n_records"] == 409_600
+    assert sorted(set(int(r) for r in sus["rank"][sus["kind"] == 1])) == spec.truth["stragglers"]
+    assert sorted(set(int(r) for r in sus["rank"][sus["kind"] == 2])) == spec.truth["slow_links"]
+
+
+def test_cfg4w_one_4096_rank_communicator():
+    spec = tg.cfg4w(reps=21, n_windows=2)
+    an, o, v, sus = run_spec(spec)
+    assert v[0]["n_groups"] == 21 and v[0]["n_analysed"] == 21
+
+
+def test_cfg5_scaled_16384_ranks_with_hang():
+    # full rank count (groups of 8, 128, 2,048 and the hung 1,024-rank ring), one pattern repetition per window
+    spec = tg.cfg5(reps=1, n_windows=3, hang_window=1)
+    an, o, v, sus = run_spec(spec)
+    alerts = [(w, int(c), int(s)) for w, x in enumerate(v) for c, s in zip(x["alerts"]["comm"], x["alerts"]["seq"])]
+    assert len(alerts) == 1
+    w, c, s = alerts[0]
+    h = compare_hang(an, o, w, c, s)
+    assert h["cls"] == 3 and list(h["roots"]) == spec.truth["hang_root"] and h["stuck_step"] == 41
+
+
+# ---------------------------------------------------------------- group sizes across the three kernels
+def sized_spec(sizes, reps, seed=11, ties=False):
+    fams, r0, cid = [], 0, 0
+    for n in sizes:
+        m = torch.arange(r0, r0 + 2 * n, dtype=torch.int64).reshape(2, n)
+        m[1] = m[1].flip(0)                                  # ring order differs from rank order
+        fams.append(tg.Family(f"n{n}", m, (tg.OP_ALLREDUCE, tg.OP_ALLGATHER), cid,
+                              bytes_choices=(MiB,) if ties else None))
+        r0 += 2 * n; cid += 2
+    s = tg.Spec("sized", seed, r0, fams, list(range(len(sizes))), reps, 2)
+    s.faults = [tg.Fault(3, "delay_exp", 300, 400_000), tg.Fault(r0 - 2, "bw", factor_milli=500)]
+    if ties:
+        s.jitter_ns = 3                                       # enter times collide: many equal skews
+    return s
+
+
+@pytest.mark.parametrize("sizes,reps", [
+    ((1, 2, 3, 4, 5, 6, 7, 8), 300),                          # thread-per-group kernel, ragged tiles
+    ((9, 15, 16, 17, 31, 32, 33), 150),                       # bitonic kernel, small paddings
+    ((63, 64, 65, 100, 128, 255, 256, 257), 37),
+    ((511, 512, 1000, 1023, 1024), 5),
+    ((1025, 2048, 3000, 4096), 9),                            # radix-select kernel, tiles of 8 groups + tail
+    ((8192,), 3),                                             # the largest communicator the library takes
+])
+def test_group_sizes(sizes, reps):
+    run_spec(sized_spec(sizes, reps))
+
+
+def test_group_sizes_with_many_ties():
+    run_spec(sized_spec((4, 8, 24, 64, 200, 1500), 20, ties=True))
+
+
+# ---------------------------------------------------------------- edge cases
+def hand_pair(recs, comms, params=None, now=10**12, with_rates=True, frames=None, n_channels=0, expect_rc=0):
+    an, o = make_pair(comms, params)
+    cols = make_cols(recs, with_rates)
+    an.trace_upload(0, cols, frames, n_channels)
+    assert o.upload(0, cols, frames, n_channels) == 0
+    an.analyze_window(0, 1, now)
+    assert o.analyze(0, 1, now) == 0
+    compare_window(an, o, 0, expect_rc=expect_rc)
+    return an, o
+
+
+def test_rejected_records_and_incomplete_groups():
+    recs = group_trace([[5, 5, 5, 5], [5, 5, 5, 5], [5, 5, 5, 5]], seq0=10)
+    recs = [r for r in recs if not (r["seq"] == 11 and r["rank"] == 2)]
+    recs.append(dict(rank=0, comm=99, seq=10, t_enter=1, t_exit=2))
+    recs.append(dict(rank=77, comm=0, seq=10, t_enter=1, t_exit=2))
+    recs.append(dict(rank=77, comm=0, seq=14, t_enter=1, t_exit=2))      # non-member widens the op-counter range
+    recs.append(dict(rank=1, comm=0, seq=3, t_enter=1, t_exit=2))
+    hand_pair(recs, [(0, [0, 1, 2, 3], 10)], expect_rc=-4)
+    hand_pair(recs[:-4] + recs[-3:], [(0, [0, 1, 2, 3], 10)], expect_rc=-5)
+    hand_pair(recs[:-4] + recs[-1:], [(0, [0, 1, 2, 3], 10)], expect_rc=-6)
+
+
+def test_barrier_small_group_mismatch_bad_times_no_rates():
+    recs = group_trace([[5, 5, 5, 900]], comm=0, bytes=3)
+    recs += group_trace([[5, 5, 5, 900]], comm=1, ranks=[4, 5, 6, 7], bytes=4)
+    recs += group_trace([[5, 5, 900]], comm=2, ranks=[8, 9, 10])
+    recs += group_trace([[5, 5, 5, 900]], comm=3, ranks=[12, 13, 14, 15], op=ALLGATHER, bytes=3)
+    mism = group_trace([[5, 6, 7, 8]] * 2, comm=4, ranks=[16, 17, 18, 19])
+    mism[5]["bytes"] = 8 * MiB
+    bad = group_trace([[5, 6, 7, 8]] * 2, comm=5, ranks=[20, 21, 22, 23])
+    bad[1]["t_exit"] = bad[1]["t_enter"] - 3
+    bad[6]["t_enter"] = -5
+    comms = [(0, [0, 1, 2, 3], 0), (1, [4, 5, 6, 7], 0), (2, [8, 9, 10], 0), (3, [12, 13, 14, 15], 0),
+             (4, [16, 17, 18, 19], 0), (5, [20, 21, 22, 23], 0), (6, [30, 31], 0)]
+    hand_pair(recs + mism + bad, comms)
+    hand_pair(recs + mism + bad, comms, with_rates=False)
+
+
+def test_slow_location_classes_and_repetition():
+    MS = 1_000_000
+    comms = [(0, [0, 1, 2, 3], 0)]
+
+    def coupled(enter_off, own, chg, seq):
+        last = max(enter_off)
+        return [dict(rank=i, comm=0, seq=seq, t_enter=10**9 * (seq + 1) + e, t_exit=10**9 * (seq + 1) + last + d, send_chg=c, recv_chg=1)
+                for i, (e, d, c) in enumerate(zip(enter_off, own, chg))]
+    wins = [coupled([0, 0, 20 * MS, 0], [2 * MS] * 4, [1] * 4, 0), coupled([0] * 4, [10 * MS] * 4, [2, 2, 2, 7], 1),
+            coupled([0, 8 * MS, 0, 0], [10 * MS] * 4, [9, 2, 2, 2], 2), coupled([0] * 4, [2 * MS] * 4, [1] * 4, 3)]
+    an, o = make_pair(comms, dict(tbase_init_ns=2 * MS))
+    for w, r in enumerate(wins):
+        cols = make_cols(r)
+        an.trace_upload(w, cols); o.upload(w, cols)
+    an.analyze_window(0, 2, 10**12); an.analyze_window(2, 2, 10**12)
+    o.analyze(0, 4, 10**12)
+    rows = [compare_window(an, o, w)[0]["comm_rows"] for w in range(4)]
+    assert [int(r["cls"][0]) for r in rows] == [1, 2, 3, 0]
+    assert [int(r["located"][0]) for r in rows] == [0, 1, 1, 0]
+
+
+def test_baseline_becomes_dynamic_across_batches():
+    durs = [[1000 + 10 * s + i for i in range(4)] for s in range(260)]
+    durs[250][2] = 90_000
+    recs = group_trace(durs)
+    an, o = make_pair([(0, [0, 1, 2, 3], 0)], dict(tbase_init_ns=500))
+    for w in range(4):
+        cols = make_cols(recs[w * 260:(w + 1) * 260])
+        an.trace_upload(w, cols); o.upload(w, cols)
+    an.analyze_window(0, 1, 10**12); an.analyze_window(1, 3, 10**12)
+    o.analyze(0, 4, 10**12)
+    rows = [compare_window(an, o, w)[0]["comm_rows"] for w in range(4)]
+    assert [int(r["baseline_static"][0]) for r in rows] == [1, 0, 0, 0] and int(rows[3]["m"][0]) == 100
+
+
+def hang_records(n, seq, entered, done, ranks):
+    recs = []
+    for s in range(seq):
+        recs += [dict(rank=ranks[i], comm=0, seq=s, t_enter=1000 + s, t_exit=2000 + s) for i in range(n)]
+    for i in range(n):
+        if i in entered:
+            recs.append(dict(rank=ranks[i], comm=0, seq=seq, t_enter=10**9, t_exit=(10**9 + 5 if i in done else -1)))
+    return recs
+
+
+def test_hang_tree_leaves_and_tie_breaks():
+    n, C = 6, 2
+    ranks = [10, 11, 12, 13, 14, 15]
+    comms = [(0, ranks, 0)]
+    an, o = hand_pair(hang_records(n, 3, {0, 1, 2, 4}, set(), ranks), comms)
+    assert compare_hang(an, o, 0, 0, 3)["cls"] == 1
+    an, o = hand_pair(hang_records(n, 3, set(range(n)), {2}, ranks), comms)
+    assert compare_hang(an, o, 0, 0, 3)["cls"] == 2
+    recs = hang_records(n, 3, set(range(n)), set(), ranks)
+    tot = {5: 4, 0: 4, 1: 4}
+    cases = [
+        [(ranks[i], 0, 3, [(9, 9), (9, 8)] if i != 4 else [(9, 7), (8, 6)]) for i in range(n)],
+        [(ranks[i], 0, 3, [(tot.get(i, 6), tot.get(i, 6))] * C) for i in range(n)],
+        [(ranks[i], 0, 3, [(5, 5)] * C) for i in range(n)],
+        [(ranks[i], 0, 3, [(5, 5)] * C) for i in range(n) if i != 2],
+        [(ranks[i], 0, 3, [(5, 5)] * C) for i in range(n)] + [(ranks[1], 0, 3, [(1, 1)] * C), (99, 0, 3, [(0, 0)] * C), (ranks[0], 0, 2, [(0, 0)] * C)],
+    ]
+    for entries in cases:
+        an, o = hand_pair(recs, comms, frames=frames_from(entries, C), n_channels=C, now=10**9 + 400 * 10**9)
+        assert compare_hang(an, o, 0, 0, 3)["cls"] == 3
+    an, o = hand_pair(recs, comms)          # no frames at all
+    compare_hang(an, o, 0, 0, 3)
+
+
+def test_empty_window_capacity_and_call_order():
+    import paper_2605_04478_b200 as ccld
+    comms = [(0, [0, 1, 2, 3], 0), (1, [4, 5, 6, 7], 0)]
+    an, o = make_pair(comms)
+    empty = make_cols([])
+    an.trace_upload(0, empty); o.upload(0, empty)
+    cols = make_cols(group_trace([[5, 6, 7, 8]] * 3))
+    an.trace_upload(1, cols); o.upload(1, cols)
+    an.analyze_window(0, 2, 10**12); o.analyze(0, 2, 10**12)
+    compare_window(an, o, 0); compare_window(an, o, 1)
+    with pytest.raises(ccld.CcldError) as e:
+        an.analyze_window(1, 1, 10**12)
+    assert e.value.code == -9
+    with pytest.raises(ccld.CcldError) as e:
+        an.comm_register(5, [1, 2], 0, 0)
+    assert e.value.code == -9
+    with pytest.raises(ccld.CcldError) as e:
+        an.get_verdict(7)
+    assert e.value.code == -7
+    # op counters 0 and 4,000,000,000 in one window: the slot space would be absurd, the window is refused
+    far = group_trace([[5, 6, 7, 8]]) + group_trace([[5, 6, 7, 8]], seq0=4_000_000_000)
+    an.trace_upload(2, make_cols(far))
+    an.analyze_window(2, 1, 10**12)
+    v = an.get_verdict(2, check=False)
+    assert v["rc"] == -8 and v["error_bits"] == 16 and v["n_groups"] == 0
+    # the context still works afterwards
+    an.reset()
+    an.analyze_window(1, 1, 10**12)
+    assert an.get_verdict(1)["n_complete"] == 3
+    an2 = ccld.Analyzer()
+    with pytest.raises(ccld.CcldError) as e:
+        an2.comm_register(0, list(range(8193)))
+    assert e.value.code == -8
+
+
+def test_duplicate_record_is_reported():
+    recs = group_trace([[5, 6, 7, 8]] * 2)
+    recs.append(dict(recs[2]))
+    an, o = make_pair([(0, [0, 1, 2, 3], 0)])
+    an.trace_upload(0, make_cols(recs))
+    an.analyze_window(0, 1, 10**12)
+    v = an.get_verdict(0, check=False)
+    assert v["rc"] == -10 and v["error_bits"] & 8 and v["n_rejected"] == 1
+
+
+def test_reset_reproduces_the_same_results():
+    spec = tg.cfg2(reps=50, n_windows=2)
+    an, o, v, sus = run_spec(spec)
+    an.reset()
+    an.analyze_window(0, 2, 10**12)
+    for w in range(2):
+        compare_window(an, o, w)
+    compare_cumulative(an, o, spec.n_ranks, 1)
