@@ -279,6 +279,40 @@ int ccld_get_rank_stats(ccld_ctx* ctx, uint32_t n_ranks, uint32_t* votes, uint32
 int ccld_timing_enable(ccld_ctx* ctx, int on);
 int ccld_get_kernel_times(ccld_ctx* ctx, double* ms /* host [CCLD_K_KINDS] */, uint64_t* launches /* host [CCLD_K_KINDS] */);
 
+/*
+ * Hang location for one ring without any allocation. The paper has no counterpart to this entry
+ * point; it exists for callers that cannot allocate device memory when they need a diagnosis: a
+ * watchdog or signal handler looking at a job whose memory is exhausted or whose allocator sits
+ * behind the hang itself, a plugin hosted inside another process that must leave that process's
+ * memory pool alone, or a monitoring loop in which an allocation could stall the device. It needs
+ * no context and calls no cudaMalloc, cudaFree or allocating library routine; its working memory is
+ * one fixed array of CCLD_STATIC_SCRATCH_BYTES bytes that is part of the library image, so every GPU
+ * that loads the library holds that much from load to exit.
+ *
+ * Inputs (all device memory on `device`, owned by the caller), indexed by ring position p < n_members:
+ *   ranks[p]       rank id of the member at position p (position p sends to p+1 mod n)
+ *   state[p]       bit0: the member entered the op (reported this or a later op counter),
+ *                  bit1: its record of the op is complete (not hung), bit2: it has a progress frame
+ *   progress[p][channel][0..1]  SendCount, RecvCount per channel (read only where bit2 is set;
+ *                  may be NULL when n_channels is 0)
+ * Output: *out (host) as for ccld_locate_hang - same classes H1/H2/H3, same tie-breaks, roots in ring
+ * order into out->roots (host, caller-allocated, up to out->roots_cap). The call enqueues one kernel on
+ * `cuda_stream` and synchronizes that stream before it returns.
+ *
+ * Limits and rules: n_members <= CCLD_STATIC_MAX_MEMBERS, else CCLD_ERR_CAPACITY and nothing runs.
+ * `err` (host, may be NULL) receives a message of at most err_cap bytes on failure. The first call on
+ * a device looks up the array's device address (cudaGetSymbolAddress, with that device current) and
+ * caches it; make that first call before any stream capture begins. All calls on a device share the
+ * array, which keeps the previous call's contents; the kernel rewrites every entry it reads, but calls
+ * whose kernels overlap on the GPU (other streams or host threads) race and must be serialized by the
+ * caller. The caller's current device is restored on return.
+ */
+#define CCLD_STATIC_MAX_MEMBERS 8192u
+#define CCLD_STATIC_SCRATCH_BYTES (CCLD_STATIC_MAX_MEMBERS * 12u + 256u)
+int ccld_ring_locate_static(int device, void* cuda_stream, uint32_t n_members, const uint32_t* ranks /* device */,
+                            const uint8_t* state /* device */, uint32_t n_channels, const uint32_t* progress /* device */,
+                            ccld_hang_verdict* out /* host */, char* err /* host */, uint32_t err_cap);
+
 /* Utility for inspection tools: synchronous copy of `bytes` bytes from device memory of this context to host memory. */
 int ccld_copy_to_host(ccld_ctx* ctx, void* dst_host, const void* src_device, uint64_t bytes);
 

@@ -25,7 +25,8 @@ MAX_ALERTS_PER_WINDOW = 1024
 EXPORTS = ("ccld_params_default", "ccld_create", "ccld_destroy", "ccld_last_error", "ccld_comm_register",
            "ccld_trace_upload", "ccld_window_release", "ccld_analyze_window", "ccld_reset", "ccld_get_verdict",
            "ccld_locate_hang", "ccld_get_optable", "ccld_get_ranges", "ccld_get_rank_stats", "ccld_copy_to_host",
-           "ccld_timing_enable", "ccld_get_kernel_times")
+           "ccld_timing_enable", "ccld_get_kernel_times", "ccld_ring_locate_static")
+STATIC_MAX_MEMBERS = 8192
 KERNEL_KINDS = ("k_seq_range", "k_plan", "k_slot_scatter", "k_reduce_small", "k_reduce_mid", "k_reduce_large", "k_window_decide")
 
 
@@ -121,6 +122,8 @@ def load_library() -> C.CDLL:
         lib.ccld_copy_to_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64]
         lib.ccld_timing_enable.argtypes = [C.c_void_p, C.c_int]
         lib.ccld_get_kernel_times.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
+        lib.ccld_ring_locate_static.argtypes = [C.c_int, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p,
+                                                C.POINTER(HangVerdict), C.c_char_p, C.c_uint32]
         _lib = lib
     return _lib
 
@@ -143,6 +146,34 @@ def _as_tensor(torch, v, dt):
     if a.dtype != np.dtype(dt):
         a = a.view(dt) if a.dtype.itemsize == np.dtype(dt).itemsize else a.astype(dt)
     return torch.from_numpy(a)
+
+
+def ring_locate_static(ranks, state, progress=None, device: int = 0, stream=None, roots_cap: int = STATIC_MAX_MEMBERS):
+    """Hang location for one ring through ccld_ring_locate_static, the entry point that allocates nothing.
+
+    For callers that cannot allocate device memory at diagnosis time (out-of-memory or wedged-allocator
+    watchdogs, plugins hosted in another process, tight monitoring loops). ranks (int32 [n]), state
+    (uint8 [n]: bit0 entered, bit1 complete, bit2 has a frame) and progress (int32 [n, channels, 2] or
+    None) are CUDA tensors the caller already owns, in ring order. This wrapper itself only builds small
+    host-side ctypes objects. Calls on one device share a fixed scratch array: do not overlap them.
+    """
+    lib = load_library()
+    n = int(ranks.numel())
+    assert ranks.is_cuda and state.is_cuda and ranks.is_contiguous() and state.is_contiguous()
+    n_ch = 0 if progress is None else int(progress.shape[1])
+    roots = (C.c_uint32 * max(roots_cap, 1))()
+    hv = HangVerdict()
+    hv.roots = C.cast(roots, C.POINTER(C.c_uint32)); hv.roots_cap = roots_cap
+    err = C.create_string_buffer(256)
+    rc = lib.ccld_ring_locate_static(device, C.c_void_p(stream.cuda_stream if stream is not None else 0), n,
+                                     C.c_void_p(ranks.data_ptr()), C.c_void_p(state.data_ptr()), n_ch,
+                                     C.c_void_p(progress.data_ptr() if progress is not None else 0), C.byref(hv), err, 256)
+    if rc != OK:
+        raise CcldError(rc, err.value.decode())
+    out: Dict[str, object] = {k: int(getattr(hv, k)) for k in ("cls", "n_roots_total", "n_not_entered", "n_hung", "n_not_hung",
+                                                             "n_missing_frames", "stuck_step", "n_members", "min_total")}
+    out["roots"] = np.array(roots[:min(hv.n_roots_total, roots_cap)], dtype=np.uint32)
+    return out
 
 
 class Analyzer:

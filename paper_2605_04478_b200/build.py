@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libccld.so")
-SOURCES = [os.path.join(CSRC, "ccld_host.cu")]
+SOURCES = [os.path.join(CSRC, "ccld_host.cu"), os.path.join(CSRC, "ccld_static.cu")]
 DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("ccld_kernels.cuh", "ccld_device.cuh")] + [
     os.path.join(os.path.dirname(HERE), "include", "ccld.h")]
 
