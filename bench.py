@@ -50,12 +50,12 @@ def workload(n_windows, rank=0):
 
 
 def class_units(spec):
-    """Records and groups per window, split by the kernel that reduces them (n <= 8, <= 1024, larger)."""
-    out = {"small": [0, 0], "mid": [0, 0], "large": [0, 0]}
+    """Records and groups per window, split by the kernel that reduces them (n <= 8, <= 128, <= 1024, larger)."""
+    out = {"small": [0, 0], "warp": [0, 0], "mid": [0, 0], "large": [0, 0]}
     for f, fam in enumerate(spec.families):
         G, n = fam.members.shape
         ops = spec.pattern.count(f) * spec.reps
-        k = "small" if n <= 8 else ("mid" if n <= 1024 else "large")
+        k = "small" if n <= 8 else ("warp" if n <= 128 else ("mid" if n <= 1024 else "large"))
         out[k][0] += G * n * ops
         out[k][1] += G * ops
     return out
@@ -228,6 +228,7 @@ def run_ours(args, rank, world, local_rank):
         "k_seq_range": lambda: NW * 8 * sum(u[0] for u in units.values()),
         "k_slot_scatter": lambda: NW * (12 + 4) * sum(u[0] for u in units.values()),
         "k_reduce_small": lambda: NW * ((4 + 33 + 1) * units["small"][0] + ROW_BYTES * units["small"][1]),
+        "k_reduce_warp": lambda: NW * ((4 + 33 + 1) * units["warp"][0] + ROW_BYTES * units["warp"][1]),
         "k_reduce_mid": lambda: NW * ((4 + 33 + 1) * units["mid"][0] + ROW_BYTES * units["mid"][1]),
         "k_reduce_large": lambda: NW * ((4 + 33 + 1) * units["large"][0] + ROW_BYTES * units["large"][1]),
     }

@@ -22,6 +22,7 @@ constexpr int REC_PER_THREAD = 8;
 constexpr int REC_PER_CTA = REC_THREADS * REC_PER_THREAD;
 constexpr int SMALL_N = 8;             // communicators of up to 8 ranks: one thread per group
 constexpr int SMALL_SEQS = 256;        //   seqs (= threads) per tile
+constexpr int WARP_N = 128;            // up to 128 ranks: one warp per group, bitonic sort in registers
 constexpr int MID_N = 1024;            // up to 1024 ranks: shared-memory bitonic sort, several groups per CTA
 constexpr int MID_THREADS = 256;
 constexpr int MID_ELEMS = 2048;        //   padded records per tile
@@ -58,13 +59,17 @@ struct Registry {
 };
 
 // Which op counters a communicator covers in a window and where its groups / slots start.
-struct RangeRow { u32 seq_lo, n_seq, row_idx, n; u64 group0, slot0; };
+struct RangeRow { u32 seq_lo, n_seq, row_idx, n; u64 group0, slot0; u32 tile0, pad; };   // tile0: first tile in its class list
 
 enum { C_REJECTED = 0, C_COMPLETE, C_INCOMPLETE, C_BARRIER, C_ANALYSED, C_FLAG_SKEW, C_FLAG_DUR, C_MISMATCH,
        C_PRESENT, C_ALERTS, C_ERR, C_INTERNAL, C_COUNT = 16 };
-enum { T_GROUPS = 0, T_SLOTS, T_TILES0, T_TILES1, T_TILES2, T_ROWS, T_FAILED, T_COUNT = 8 };
+constexpr int N_CLASSES = 4;           // reduction kernels: n <= 8, <= 128, <= 1024, larger
+enum { T_GROUPS = 0, T_SLOTS, T_TILES0, T_TILES1, T_TILES2, T_TILES3, T_ROWS, T_FAILED, T_COUNT = 8 };
 
 struct Tile { u32 w, c, seq_off, count; };
+
+// What a tile contributes to its communicator's window decision (Eq. 2 and the round counts).
+struct TileSum { u64 best_rng; u32 best_k, n_rounds, n_an, pad; };   // best_k: op-counter offset in the range, NONE if no round
 
 // One window of a batch: input columns, scratch and result pointers (all device memory).
 struct WinDesc {
@@ -89,19 +94,19 @@ struct WinDesc {
   double* gbw;                       // [n_groups]
   ccld_comm_verdict* comm_rows;      // [n_rows]
   ccld_hang_alert* alerts;           // [CCLD_MAX_ALERTS_PER_WINDOW]
-  u32 tile0[3];                      // first tile of this window in each class list
-  u32 pad;
+  u32 tile0[N_CLASSES];              // first tile of this window in each class list
+  TileSum* tsum[N_CLASSES];          // per-class tile summaries of the whole batch
 };
 
 enum { GI_E_MIN = 0, GI_ARRIVAL_SKEW, GI_T_MAX, GI_T_MIN, GI_SPAN, GI_MED_SKEW, GI_MAD_SKEW, GI_MED_DUR, GI_MAD_DUR, GI_COUNT };
 enum { GU_RANK_TMIN = 0, GU_RANK_TMAX, GU_MAX_CHG, GU_RANK_MAX_CHG, GU_N_PRESENT, GU_GFLAGS, GU_COUNT };
 
 __host__ __device__ inline u32 next_pow2(u32 n) { u32 p = 1; while (p < n) p <<= 1; return p; }
-__host__ __device__ inline u32 comm_class(u32 n) { return n <= SMALL_N ? 0u : (n <= MID_N ? 1u : 2u); }
-__host__ __device__ inline u32 mid_npad(u32 n) { u32 p = next_pow2(n); return p < 16 ? 16 : p; }
+__host__ __device__ inline u32 comm_class(u32 n) { return n <= SMALL_N ? 0u : (n <= WARP_N ? 1u : (n <= MID_N ? 2u : 3u)); }
+__host__ __device__ inline u32 mid_npad(u32 n) { u32 p = next_pow2(n); return p < 32 ? 32 : p; }
 __host__ __device__ inline u32 tile_seqs(u32 n) {
   u32 c = comm_class(n);
-  return c == 0 ? SMALL_SEQS : (c == 1 ? MID_ELEMS / mid_npad(n) : (u32)LARGE_SEQS);
+  return c == 0 ? SMALL_SEQS : (c <= 2 ? MID_ELEMS / mid_npad(n) : (u32)LARGE_SEQS);
 }
 
 }  // namespace ccld

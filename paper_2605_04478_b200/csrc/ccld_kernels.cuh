@@ -6,7 +6,8 @@
 //                   and the work list for the reduction kernels
 //   k_slot_scatter  group-by, part 3: perm[slot] = record index
 //   k_reduce_small  per-op reductions + median/MAD + flags + votes, n <= 8 (thread per group)
-//   k_reduce_mid    same, 9 <= n <= 1024 (shared-memory bitonic sort, several groups per CTA)
+//   k_reduce_warp   same, 9 <= n <= 128 (warp per group, bitonic sort in registers)
+//   k_reduce_mid    same, 129 <= n <= 1024 (shared-memory bitonic sort, several groups per CTA)
 //   k_reduce_large  same, n > 1024 (one CTA per group, radix select)
 //   k_window_decide Eq. 1-4 per communicator and window, slow location
 //   k_hang_locate   hang decision tree over presence / completion / progress counters
@@ -78,6 +79,18 @@ __device__ __forceinline__ void raise_alert(const WinDesc& D, u32 comm_id, u32 s
   if (k < CCLD_MAX_ALERTS_PER_WINDOW) { ccld_hang_alert a; a.comm = comm_id; a.seq = seq; a.age_ns = age; D.alerts[k] = a; }
 }
 
+// Eq. 2 candidate merge: larger range wins, then the earlier op counter (k = NONE means "no round")
+__device__ __forceinline__ void best_merge(u64& rng, u32& k, u64 o_rng, u32 o_k) {
+  if (o_k != NONE && (k == NONE || o_rng > rng || (o_rng == rng && o_k < k))) { rng = o_rng; k = o_k; }
+}
+__device__ __forceinline__ void best_warp_reduce(u64& rng, u32& k) {
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) {
+    const u64 o_rng = shfl_xor64(rng, d); const u32 o_k = __shfl_xor_sync(0xFFFFFFFFu, k, d);
+    best_merge(rng, k, o_rng, o_k);
+  }
+}
+
 // ------------------------------------------------------------------------------------------------
 // group-by, part 1: which op counters does every communicator cover in every window
 // ------------------------------------------------------------------------------------------------
@@ -108,22 +121,25 @@ __global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __rest
 // group-by, part 2: closed-form layout. One CTA per window scans the communicators.
 //   slot(comm, seq, pos) = slot0[comm] + (seq - seq_lo[comm]) * n[comm] + pos
 // ------------------------------------------------------------------------------------------------
-struct PlanAcc { u64 groups, slots; u32 rows, t0, t1, t2; };
+struct PlanAcc { u64 groups, slots; u32 rows, t[N_CLASSES]; };
 
 __device__ __forceinline__ PlanAcc plan_add(const PlanAcc& a, const PlanAcc& b) {
   PlanAcc r; r.groups = a.groups + b.groups; r.slots = a.slots + b.slots; r.rows = a.rows + b.rows;
-  r.t0 = a.t0 + b.t0; r.t1 = a.t1 + b.t1; r.t2 = a.t2 + b.t2; return r;
+#pragma unroll
+  for (int q = 0; q < N_CLASSES; ++q) r.t[q] = a.t[q] + b.t[q];
+  return r;
 }
 __device__ __forceinline__ PlanAcc plan_shfl_up(const PlanAcc& a, int d) {
   PlanAcc r;
   r.groups = __shfl_up_sync(0xFFFFFFFFu, a.groups, d); r.slots = __shfl_up_sync(0xFFFFFFFFu, a.slots, d);
-  r.rows = __shfl_up_sync(0xFFFFFFFFu, a.rows, d); r.t0 = __shfl_up_sync(0xFFFFFFFFu, a.t0, d);
-  r.t1 = __shfl_up_sync(0xFFFFFFFFu, a.t1, d); r.t2 = __shfl_up_sync(0xFFFFFFFFu, a.t2, d);
+  r.rows = __shfl_up_sync(0xFFFFFFFFu, a.rows, d);
+#pragma unroll
+  for (int q = 0; q < N_CLASSES; ++q) r.t[q] = __shfl_up_sync(0xFFFFFFFFu, a.t[q], d);
   return r;
 }
 
 __device__ __forceinline__ PlanAcc plan_item(const WinDesc& D, const Registry& R, u32 c) {
-  PlanAcc a = {0, 0, 0, 0, 0, 0};
+  PlanAcc a = {0, 0, 0, {0, 0, 0, 0}};
   if (c < R.n_comms) {
     u32 lo = D.rmin[c], hi = D.rmax[c];
     if (lo <= hi && lo != NONE) {
@@ -131,8 +147,7 @@ __device__ __forceinline__ PlanAcc plan_item(const WinDesc& D, const Registry& R
       a.groups = ns; a.slots = ns * n; a.rows = 1;
       u64 tiles = (ns + tile_seqs(n) - 1) / tile_seqs(n);
       u32 t = tiles > 0x7FFFFFFFull ? 0x7FFFFFFFu : (u32)tiles;
-      u32 cls = comm_class(n);
-      a.t0 = cls == 0 ? t : 0; a.t1 = cls == 1 ? t : 0; a.t2 = cls == 2 ? t : 0;
+      a.t[comm_class(n)] = t;
     }
   }
   return a;
@@ -152,13 +167,13 @@ __device__ PlanAcc plan_block_scan(PlanAcc v, PlanAcc* total, PlanAcc* s_warp /*
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) { PlanAcc o = plan_shfl_up(xi, d); if (lane >= (u32)d) xi = plan_add(xi, o); }
     PlanAcc ex = plan_shfl_up(xi, 1);
-    if (lane == 0) ex = PlanAcc{0, 0, 0, 0, 0, 0};
+    if (lane == 0) ex = PlanAcc{0, 0, 0, {0, 0, 0, 0}};
     s_warp[lane] = ex;
     if (lane == 31) s_warp[32] = xi;
   }
   __syncthreads();
   PlanAcc ex = plan_shfl_up(inc, 1);
-  if (lane == 0) ex = PlanAcc{0, 0, 0, 0, 0, 0};
+  if (lane == 0) ex = PlanAcc{0, 0, 0, {0, 0, 0, 0}};
   PlanAcc r = plan_add(s_warp[wid], ex);
   *total = s_warp[32];
   __syncthreads();
@@ -167,13 +182,13 @@ __device__ PlanAcc plan_block_scan(PlanAcc v, PlanAcc* total, PlanAcc* s_warp /*
 
 // emit == 0: write ranges and totals (and fail the window if it needs more than slot_cap slots).
 // emit == 1: write the tile lists (tile0[] filled by the host from the totals).
-__global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd, Registry R, Tile* __restrict__ tiles0,
-                                                       Tile* __restrict__ tiles1, Tile* __restrict__ tiles2, int emit) {
+struct TileLists { Tile* t[N_CLASSES]; };
+__global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd, Registry R, TileLists lists, int emit) {
   __shared__ PlanAcc s_warp[33];
   __shared__ int s_failed;
   WinDesc& D = wd[blockIdx.x];
   if (emit && D.totals[T_FAILED]) return;
-  PlanAcc run = {0, 0, 0, 0, 0, 0};
+  PlanAcc run = {0, 0, 0, {0, 0, 0, 0}};
   for (u32 c0 = 0; c0 < R.n_comms; c0 += PLAN_THREADS) {
     const u32 c = c0 + threadIdx.x;
     PlanAcc it = plan_item(D, R, c), tot;
@@ -182,12 +197,14 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
       if (!emit) {
         RangeRow r;
         r.seq_lo = it.rows ? D.rmin[c] : 0; r.n_seq = (u32)it.groups; r.row_idx = ex.rows; r.n = R.comm_n[c];
-        r.group0 = ex.groups; r.slot0 = ex.slots;
+        r.group0 = ex.groups; r.slot0 = ex.slots; r.tile0 = 0; r.pad = 0;
         D.ranges[c] = r;
       } else if (it.rows) {
         const u32 n = R.comm_n[c], S = tile_seqs(n), cls = comm_class(n);
-        Tile* dst = cls == 0 ? tiles0 + D.tile0[0] + ex.t0 : (cls == 1 ? tiles1 + D.tile0[1] + ex.t1 : tiles2 + D.tile0[2] + ex.t2);
-        const u32 nt = it.t0 + it.t1 + it.t2;
+        const u32 first = D.tile0[cls] + ex.t[cls];
+        Tile* dst = lists.t[cls] + first;
+        D.ranges[c].tile0 = first;
+        const u32 nt = it.t[cls];
         for (u32 k = 0; k < nt; ++k) {
           Tile t; t.w = blockIdx.x; t.c = c; t.seq_off = k * S;
           u64 left = it.groups - (u64)k * S; t.count = left < S ? (u32)left : S;
@@ -203,13 +220,13 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
     int failed = run.slots > D.slot_cap || run.groups > 0x7FFFFFFFull;
     s_failed = failed;
     D.totals[T_GROUPS] = failed ? 0 : run.groups; D.totals[T_SLOTS] = failed ? 0 : run.slots;
-    D.totals[T_TILES0] = failed ? 0 : run.t0; D.totals[T_TILES1] = failed ? 0 : run.t1; D.totals[T_TILES2] = failed ? 0 : run.t2;
+    for (int q = 0; q < N_CLASSES; ++q) D.totals[T_TILES0 + q] = failed ? 0 : run.t[q];
     D.totals[T_ROWS] = failed ? 0 : run.rows; D.totals[T_FAILED] = failed;
     if (failed) atomicOr((unsigned*)&D.counters[C_ERR], (unsigned)CCLD_E_CAPACITY);
   }
   __syncthreads();
   if (s_failed)
-    for (u32 c = threadIdx.x; c < R.n_comms; c += PLAN_THREADS) { RangeRow z = {0, 0, 0, R.comm_n[c], 0, 0}; D.ranges[c] = z; }
+    for (u32 c = threadIdx.x; c < R.n_comms; c += PLAN_THREADS) { RangeRow z = {0, 0, 0, R.comm_n[c], 0, 0, 0, 0}; D.ranges[c] = z; }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -288,8 +305,10 @@ __device__ __forceinline__ void median_mad8(const u64 (&x)[8], u32 n, u64* med, 
 }
 
 __global__ void __launch_bounds__(SMALL_SEQS) k_reduce_small(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles,
-                                                              Registry R, Params P, i64 now) {
+                                                              TileSum* __restrict__ sums, Registry R, Params P, i64 now) {
   __shared__ double s_bw[SMALL_SEQS / 32][SMALL_N];
+  __shared__ u64 s_brng[SMALL_SEQS / 32];
+  __shared__ u32 s_bk[SMALL_SEQS / 32];
   const Tile t = tiles[blockIdx.x];
   const WinDesc& D = wd[t.w];
   const u32 c = t.c, n = R.comm_n[c];
@@ -303,6 +322,7 @@ __global__ void __launch_bounds__(SMALL_SEQS) k_reduce_small(const WinDesc* __re
   for (int p = 0; p < SMALL_N; ++p) bw[p] = 0.0;
   bool complete = false, barrier = false, analysed = false, mismatch = false;
   u32 n_present = 0, n_fs = 0, n_fd = 0;
+  u64 my_rng = 0;
 
   if (active) {
     const u64 g = row.group0 + t.seq_off + j;
@@ -373,6 +393,7 @@ __global__ void __launch_bounds__(SMALL_SEQS) k_reduce_small(const WinDesc* __re
       gbw = busbw(bn, den, span);
       out_i[GI_E_MIN] = (i64)e_min; out_i[GI_ARRIVAL_SKEW] = (i64)askew; out_i[GI_T_MAX] = (i64)tmax; out_i[GI_T_MIN] = (i64)tmin;
       out_i[GI_SPAN] = span;
+      my_rng = tmax - tmin;
       r_tmin = mem[pmin]; r_tmax = mem[pmax]; r_chg = mem[pos_chg];
       if (!barrier) {
 #pragma unroll
@@ -425,9 +446,19 @@ __global__ void __launch_bounds__(SMALL_SEQS) k_reduce_small(const WinDesc* __re
     for (int d = 16; d > 0; d >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, d);
     if (lane == 0) s_bw[wid][p] = v;
   }
+  {
+    const bool is_round = active && complete && !barrier;
+    u64 brng = is_round ? my_rng : 0; u32 bk = is_round ? t.seq_off + j : NONE;
+    best_warp_reduce(brng, bk);
+    if (lane == 0) { s_brng[wid] = brng; s_bk[wid] = bk; }
+  }
   if (lane == 0) { count_add(D.counters, C_PRESENT, pres); count_add(D.counters, C_FLAG_SKEW, fs); count_add(D.counters, C_FLAG_DUR, fd); }
   __syncthreads();
   if (threadIdx.x == 0) {
+    u64 brng = s_brng[0]; u32 bk = s_bk[0];
+    for (int q = 1; q < SMALL_SEQS / 32; ++q) best_merge(brng, bk, s_brng[q], s_bk[q]);
+    TileSum ts; ts.best_rng = brng; ts.best_k = bk; ts.n_rounds = n_bwc; ts.n_an = n_an; ts.pad = 0;
+    sums[blockIdx.x] = ts;
     count_add(D.counters, C_COMPLETE, n_comp); count_add(D.counters, C_INCOMPLETE, n_inc); count_add(D.counters, C_BARRIER, n_bar);
     count_add(D.counters, C_ANALYSED, n_an); count_add(D.counters, C_MISMATCH, n_mis);
   }
@@ -441,7 +472,7 @@ __global__ void __launch_bounds__(SMALL_SEQS) k_reduce_small(const WinDesc* __re
 }
 
 // ------------------------------------------------------------------------------------------------
-// per-op reductions, 9 <= n <= 1024: a tile of S groups is staged in shared memory ([group][member],
+// per-op reductions, 129 <= n <= 1024: a tile of S groups is staged in shared memory ([group][member],
 // pitch n_pad + 1), reduced by one warp per group, sorted by a bitonic network over all groups at once
 // ------------------------------------------------------------------------------------------------
 struct MidGroup {
@@ -471,7 +502,7 @@ __device__ void mid_bitonic(u64* key, u32 S, u32 n_pad, u32 pitch, bool merge_on
 }
 
 __global__ void __launch_bounds__(MID_THREADS) k_reduce_mid(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles,
-                                                            Registry R, Params P, i64 now) {
+                                                            TileSum* __restrict__ sums, Registry R, Params P, i64 now) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const Tile t = tiles[blockIdx.x];
   const WinDesc& D = wd[t.w];
@@ -491,6 +522,9 @@ __global__ void __launch_bounds__(MID_THREADS) k_reduce_mid(const WinDesc* __res
   u8* s_st = s_op + cap;                 // 1 present, 2 in flight, 4 bad time
   MidGroup* s_g = (MidGroup*)(((uintptr_t)(s_st + cap) + 15) & ~(uintptr_t)15);
   __shared__ u32 s_cnt[8];
+  __shared__ u64 s_brng[MID_THREADS / 32];
+  __shared__ u32 s_bk[MID_THREADS / 32], s_rounds[MID_THREADS / 32];
+  u64 w_brng = 0; u32 w_bk = NONE, w_rounds = 0;          // this warp's Eq. 2 candidate and round count (lane 0)
 
   const u64 slot_t = row.slot0 + (u64)t.seq_off * n;      // first slot of the tile
   const u64 g_t = row.group0 + t.seq_off;                  // first group of the tile
@@ -580,8 +614,10 @@ __global__ void __launch_bounds__(MID_THREADS) k_reduce_mid(const WinDesc* __res
       D.gu32[(u64)GU_N_PRESENT * G + g] = npres; D.gu32[(u64)GU_GFLAGS * G + g] = gfl;
       D.gbw[g] = gb;
       c_comp += complete; c_inc += !complete; c_bar += barrier; c_an += analysed; c_mis += mism; c_pres += npres;
+      if (complete && !barrier) { ++w_rounds; best_merge(w_brng, w_bk, tmax - tmin, t.seq_off + jg); }
     }
   }
+  if (lane == 0) { s_brng[wid] = w_brng; s_bk[wid] = w_bk; s_rounds[wid] = w_rounds; }
   __syncthreads();
   const u32 k_med = (n - 1) >> 1;
   // 4. arrival skew: sort, median, deviations, merge, MAD
@@ -677,6 +713,10 @@ __global__ void __launch_bounds__(MID_THREADS) k_reduce_mid(const WinDesc* __res
   }
   __syncthreads();
   if (threadIdx.x == 0) {
+    u64 brng = s_brng[0]; u32 bk = s_bk[0], rounds = s_rounds[0];
+    for (int q = 1; q < MID_THREADS / 32; ++q) { best_merge(brng, bk, s_brng[q], s_bk[q]); rounds += s_rounds[q]; }
+    TileSum ts; ts.best_rng = brng; ts.best_k = bk; ts.n_rounds = rounds; ts.n_an = s_cnt[3]; ts.pad = 0;
+    sums[blockIdx.x] = ts;
     count_add(D.counters, C_COMPLETE, s_cnt[0]); count_add(D.counters, C_INCOMPLETE, s_cnt[1]); count_add(D.counters, C_BARRIER, s_cnt[2]);
     count_add(D.counters, C_ANALYSED, s_cnt[3]); count_add(D.counters, C_MISMATCH, s_cnt[4]); count_add(D.counters, C_PRESENT, s_cnt[5]);
     count_add(D.counters, C_FLAG_SKEW, s_cnt[6]); count_add(D.counters, C_FLAG_DUR, s_cnt[7]);
@@ -687,6 +727,266 @@ inline size_t mid_smem_bytes(u32 n_pad_min) {
   // cap = (MID_ELEMS / n_pad) * (n_pad + 1) is largest for the smallest n_pad
   size_t cap = (size_t)(MID_ELEMS / n_pad_min) * (n_pad_min + 1);
   return cap * (4 * 8 + 2 * 4 + 2) + 16 + (MID_ELEMS / n_pad_min) * sizeof(MidGroup);
+}
+
+// ------------------------------------------------------------------------------------------------
+// per-op reductions, 9 <= n <= 128: a tile of S groups is staged in shared memory as in k_reduce_mid,
+// then one warp owns a group end to end: cross-rank reductions by shuffles, order statistics by a
+// bitonic network over E = n_pad / 32 registers per lane (32-bit keys whenever the group's value
+// range fits), flags straight to global memory. No block-wide barrier inside the sort.
+// ------------------------------------------------------------------------------------------------
+template <class K> struct KeyMax;
+template <> struct KeyMax<u32> { static __device__ __forceinline__ u32 v() { return 0xFFFFFFFFu; } };
+template <> struct KeyMax<u64> { static __device__ __forceinline__ u64 v() { return U64_MAX_; } };
+
+// Element i = r * 32 + lane of the warp's 32 E keys. Full sort, or (MERGE) the last merge phase only,
+// which sorts a sequence that falls and then rises.
+template <int E, class K, bool MERGE>
+__device__ __forceinline__ void warp_bitonic(K (&v)[E], u32 lane) {
+  constexpr int NP = 32 * E;
+#pragma unroll
+  for (int k = MERGE ? NP : 2; k <= NP; k <<= 1) {
+#pragma unroll
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      if (j >= 32) {
+        const int dr = j >> 5;
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+          if ((r & dr) == 0) {
+            const int r2 = r | dr;
+            const bool up = k == NP || (((r * 32) & k) == 0);
+            const K a = v[r], b = v[r2];
+            const K lo = a < b ? a : b, hi = a < b ? b : a;
+            v[r] = up ? lo : hi; v[r2] = up ? hi : lo;
+          }
+        }
+      } else {
+        const bool lower = (lane & j) == 0;
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+          const K o = __shfl_xor_sync(0xFFFFFFFFu, v[r], j);
+          const bool up = k == NP || (((r * 32 + lane) & k) == 0);
+          const K lo = v[r] < o ? v[r] : o, hi = v[r] < o ? o : v[r];
+          v[r] = (lower == up) ? lo : hi;
+        }
+      }
+    }
+  }
+}
+
+template <int E, class K>
+__device__ __forceinline__ K warp_pick(const K (&v)[E], u32 idx) {
+  K x = v[0];
+#pragma unroll
+  for (int r = 1; r < E; ++r) x = (idx >> 5) == (u32)r ? v[r] : x;
+  return __shfl_sync(0xFFFFFFFFu, x, idx & 31);
+}
+
+// lower median and lower-median absolute deviation of key(p), p < n <= 32 E
+template <int E, class K, class F>
+__device__ __forceinline__ void warp_median_mad(F key, u32 n, u32 lane, K* med, K* mad) {
+  K v[E];
+#pragma unroll
+  for (int r = 0; r < E; ++r) { const u32 p = r * 32 + lane; v[r] = p < n ? key(p) : KeyMax<K>::v(); }
+  warp_bitonic<E, K, false>(v, lane);
+  const u32 k = (n - 1) >> 1;
+  const K m = warp_pick<E, K>(v, k);
+#pragma unroll
+  for (int r = 0; r < E; ++r) { const u32 p = r * 32 + lane; v[r] = p < n ? (v[r] >= m ? v[r] - m : m - v[r]) : KeyMax<K>::v(); }
+  warp_bitonic<E, K, true>(v, lane);
+  *med = m; *mad = warp_pick<E, K>(v, k);
+}
+
+template <int E>
+__device__ __forceinline__ void warp_group_stats(const u64* te, const u64* du, u32 n, u32 lane, u64 e_min, u64 askew, u64 tmin, u64 tmax,
+                                                 u64* med_s, u64* mad_s, u64* med_d, u64* mad_d) {
+  if (askew < 0xFFFFFFFFull) { u32 m, d; warp_median_mad<E, u32>([&](u32 p) { return (u32)(te[p] - e_min); }, n, lane, &m, &d); *med_s = m; *mad_s = d; }
+  else { u64 m, d; warp_median_mad<E, u64>([&](u32 p) { return te[p] - e_min; }, n, lane, &m, &d); *med_s = m; *mad_s = d; }
+  if (tmax - tmin < 0xFFFFFFFFull) { u32 m, d; warp_median_mad<E, u32>([&](u32 p) { return (u32)(du[p] - tmin); }, n, lane, &m, &d); *med_d = tmin + m; *mad_d = d; }
+  else { u64 m, d; warp_median_mad<E, u64>([&](u32 p) { return du[p] - tmin; }, n, lane, &m, &d); *med_d = tmin + m; *mad_d = d; }
+}
+
+constexpr int WARP_EMAX = WARP_N / 32;
+
+inline size_t warp_smem_bytes() {
+  // cap = (MID_ELEMS / n_pad) * (n_pad + 1) is largest for n_pad = 32
+  const size_t cap = (size_t)(MID_ELEMS / 32) * 33;
+  return cap * (3 * 8 + 4 + 2) + 16 + (MID_THREADS / 32) * WARP_N * sizeof(double);
+}
+
+__global__ void __launch_bounds__(MID_THREADS) k_reduce_warp(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles,
+                                                             TileSum* __restrict__ sums, Registry R, Params P, i64 now) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const Tile t = tiles[blockIdx.x];
+  const WinDesc& D = wd[t.w];
+  const u32 c = t.c, n = R.comm_n[c];
+  const RangeRow row = D.ranges[c];
+  const u32* mem = R.members + R.comm_moff[c];
+  const u32 n_pad = mid_npad(n), pitch = n_pad + 1, S = t.count, S_max = MID_ELEMS / n_pad;
+  const u32 cap = S_max * pitch;
+  u64* s_te = (u64*)smem_raw;            // enter time
+  u64* s_du = s_te + cap;                // duration
+  u64* s_by = s_du + cap;                // bytes
+  u32* s_idx = (u32*)(s_by + cap);       // record index ...
+  u32* s_ch = s_idx;                     // ... replaced in place by max(send_chg, recv_chg) once the record is gathered
+  u8* s_op = (u8*)(s_idx + cap);
+  u8* s_st = s_op + cap;                 // 1 present, 2 in flight, 4 bad time
+  double* s_bw = (double*)(((uintptr_t)(s_st + cap) + 15) & ~(uintptr_t)15);   // [warps][n_pad]
+  __shared__ u32 s_cnt[8];
+  __shared__ u64 s_brng[MID_THREADS / 32];
+  __shared__ u32 s_bk[MID_THREADS / 32], s_rounds[MID_THREADS / 32];
+
+  const u64 slot_t = row.slot0 + (u64)t.seq_off * n;
+  const u64 g_t = row.group0 + t.seq_off;
+  const u32 n_el = S * n;
+  if (threadIdx.x < 8) s_cnt[threadIdx.x] = 0;
+  // 1. record indices, coalesced along the slot order
+  for (u32 e = threadIdx.x; e < n_el; e += MID_THREADS) { const u32 jg = e / n, p = e - jg * n; s_idx[jg * pitch + p] = D.perm[slot_t + e]; }
+  __syncthreads();
+  // 2. gather: consecutive threads walk consecutive op counters of one member
+  for (u32 e = threadIdx.x; e < n_el; e += MID_THREADS) {
+    const u32 p = e / S, jg = e - p * S, a = jg * pitch + p;
+    const u32 idx = s_idx[a];
+    u64 te = 0, du = 0, by = 0; u32 ch = 0; u8 op = 0, st = 0;
+    if (idx != NONE) {
+      const i64 x = D.t_enter[idx], y = D.t_exit[idx];
+      by = D.bytes[idx]; op = D.op[idx];
+      if (D.send_chg != nullptr) { const u32 sc = D.send_chg[idx], rc = D.recv_chg[idx]; ch = sc > rc ? sc : rc; }
+      st = 1 | (y == -1 ? 2 : ((x < 0 || y < x) ? 4 : 0));
+      te = (u64)x; du = (u64)(y - x);
+    }
+    s_te[a] = te; s_du[a] = du; s_by[a] = by; s_ch[a] = ch; s_op[a] = op; s_st[a] = st;
+  }
+  __syncthreads();
+  // 3. one warp per group, end to end
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const u32 k_milli = P.k_milli;
+  u32 c_comp = 0, c_inc = 0, c_bar = 0, c_an = 0, c_mis = 0, c_pres = 0, n_fs = 0, n_fd = 0, n_bwc = 0;
+  u64 w_brng = 0; u32 w_bk = NONE;
+  double bwacc[WARP_EMAX];
+#pragma unroll
+  for (int r = 0; r < WARP_EMAX; ++r) bwacc[r] = 0.0;
+  for (u32 jg = wid; jg < S; jg += MID_THREADS / 32) {
+    const u32 b = jg * pitch;
+    u32 npres = 0, first = NONE, stor = 0;
+    for (u32 p = lane; p < n; p += 32) { const u32 st = s_st[b + p]; if (st & 1) { ++npres; first = first == NONE ? p : first; } stor |= st; }
+    npres = __reduce_add_sync(0xFFFFFFFFu, npres); first = __reduce_min_sync(0xFFFFFFFFu, first); stor = __reduce_or_sync(0xFFFFFFFFu, stor);
+    const bool have_first = first != NONE;
+    const u64 gbytes = have_first ? s_by[b + first] : 0; const u32 gop = have_first ? s_op[b + first] : 0;
+    const bool inflight = stor & 2, bad_time = stor & 4, complete = npres == n && !inflight && !bad_time;
+    const bool barrier = have_first && gop == CCLD_OP_ALLREDUCE && gbytes < P.barrier_bytes;
+    u32 mism = 0; i64 age = -1;
+    u64 e_min = U64_MAX_, e_max = 0, tmax = 0, tmin = U64_MAX_; i64 x_max = INT64_MIN; u32 pmax = NONE, pmin = NONE; u64 chk = 0;
+    for (u32 p = lane; p < n; p += 32) {
+      const u32 st = s_st[b + p];
+      if (!(st & 1)) continue;
+      if (s_op[b + p] != gop || s_by[b + p] != gbytes) mism = 1;
+      const u64 te = s_te[b + p], du = s_du[b + p];
+      if (st & 2) { const i64 ag = now - (i64)te; age = ag > age ? ag : age; }
+      e_min = te < e_min ? te : e_min; e_max = te > e_max ? te : e_max;
+      const i64 tx = (i64)(te + du); x_max = tx > x_max ? tx : x_max;
+      if (pmax == NONE || du > tmax) { tmax = du; pmax = p; }
+      if (pmin == NONE || du < tmin) { tmin = du; pmin = p; }
+      const u64 ck = ((u64)s_ch[b + p] << 32) | (u64)(NONE - p);        // most changes, then lowest position
+      chk = ck > chk ? ck : chk;
+    }
+    mism = __reduce_or_sync(0xFFFFFFFFu, mism);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+      const i64 ag = (i64)shfl_xor64((u64)age, d); age = ag > age ? ag : age;
+      const u64 em = shfl_xor64(e_min, d); e_min = em < e_min ? em : e_min;
+      const u64 eM = shfl_xor64(e_max, d); e_max = eM > e_max ? eM : e_max;
+      const i64 xm = (i64)shfl_xor64((u64)x_max, d); x_max = xm > x_max ? xm : x_max;
+      const u64 ck = shfl_xor64(chk, d); chk = ck > chk ? ck : chk;
+      const u64 tM = shfl_xor64(tmax, d); const u32 pM = __shfl_xor_sync(0xFFFFFFFFu, pmax, d);
+      if (pM != NONE && (pmax == NONE || tM > tmax || (tM == tmax && pM < pmax))) { tmax = tM; pmax = pM; }
+      const u64 tm = shfl_xor64(tmin, d); const u32 pm = __shfl_xor_sync(0xFFFFFFFFu, pmin, d);
+      if (pm != NONE && (pmin == NONE || tm < tmin || (tm == tmin && pm < pmin))) { tmin = tm; pmin = pm; }
+    }
+    u32 gfl = (mism ? CCLD_G_OPSET_MISMATCH : 0) | (barrier ? CCLD_G_BARRIER : 0) | (inflight ? CCLD_G_INFLIGHT : 0) |
+              (bad_time ? CCLD_G_BAD_TIME : 0) | (complete ? CCLD_G_COMPLETE : CCLD_G_INCOMPLETE);
+    const bool analysed = complete && !barrier && n >= P.min_group;
+    if (analysed) gfl |= CCLD_G_ANALYSED;
+    const bool hang = !complete && inflight && age > P.hang_ns && !barrier;
+    if (hang) gfl |= CCLD_G_HANG_ALERT;
+    const u64 askew = complete ? e_max - e_min : 0;
+    u64 med_s = 0, mad_s = 0, med_d = 0, mad_d = 0;
+    if (analysed) {
+      if (n_pad == 32) warp_group_stats<1>(s_te + b, s_du + b, n, lane, e_min, askew, tmin, tmax, &med_s, &mad_s, &med_d, &mad_d);
+      else if (n_pad == 64) warp_group_stats<2>(s_te + b, s_du + b, n, lane, e_min, askew, tmin, tmax, &med_s, &mad_s, &med_d, &mad_d);
+      else warp_group_stats<4>(s_te + b, s_du + b, n, lane, e_min, askew, tmin, tmax, &med_s, &mad_s, &med_d, &mad_d);
+    }
+    // flags and votes, in slot order
+    double num = 1.0, den = 1.0; bus_factor(gop, n, &num, &den);
+    const double bn = (double)gbytes * num;
+    const bool add_bw = complete && !barrier;
+#pragma unroll
+    for (int r = 0; r < WARP_EMAX; ++r) {
+      const u32 p = r * 32 + lane;
+      if (p < n) {
+        const u32 st = s_st[b + p];
+        u8 f = CCLD_F_NOT_ANALYSED;
+        if (!(st & 1)) f |= CCLD_F_MISSING;
+        else if (analysed) {
+          const u64 sk = s_te[b + p] - e_min, du = s_du[b + p];
+          const bool so = mul_gt(absdiff(sk, med_s), 1000u, mad_s, k_milli), sh = sk > med_s;
+          const bool dq = mul_gt(absdiff(du, med_d), 1000u, mad_d, k_milli), dh = du > med_d;
+          f = (so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0);
+          if (so) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p] * 4 + (sh ? 0 : 1)], 1u); }
+          if (dq) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p] * 4 + (dh ? 2 : 3)], 1u); }
+        }
+        D.flags[slot_t + (u64)jg * n + p] = f;
+        if (add_bw) bwacc[r] += busbw(bn, den, (i64)s_du[b + p]);
+      }
+    }
+    if (lane == 0) {
+      const u64 g = g_t + jg, G = D.n_groups;
+      if (hang) raise_alert(D, R.comm_id[c], row.seq_lo + t.seq_off + jg, age);
+      const i64 span = complete ? x_max - (i64)e_min : 0;
+      D.gi64[(u64)GI_E_MIN * G + g] = complete ? (i64)e_min : 0; D.gi64[(u64)GI_ARRIVAL_SKEW * G + g] = (i64)askew;
+      D.gi64[(u64)GI_T_MAX * G + g] = complete ? (i64)tmax : 0; D.gi64[(u64)GI_T_MIN * G + g] = complete ? (i64)tmin : 0;
+      D.gi64[(u64)GI_SPAN * G + g] = span;
+      D.gi64[(u64)GI_MED_SKEW * G + g] = (i64)med_s; D.gi64[(u64)GI_MAD_SKEW * G + g] = (i64)mad_s;
+      D.gi64[(u64)GI_MED_DUR * G + g] = (i64)med_d; D.gi64[(u64)GI_MAD_DUR * G + g] = (i64)mad_d;
+      D.gu32[(u64)GU_RANK_TMIN * G + g] = complete ? mem[pmin] : 0; D.gu32[(u64)GU_RANK_TMAX * G + g] = complete ? mem[pmax] : 0;
+      D.gu32[(u64)GU_MAX_CHG * G + g] = complete ? (u32)(chk >> 32) : 0;
+      D.gu32[(u64)GU_RANK_MAX_CHG * G + g] = complete ? mem[NONE - (u32)chk] : 0;
+      D.gu32[(u64)GU_N_PRESENT * G + g] = npres; D.gu32[(u64)GU_GFLAGS * G + g] = gfl;
+      D.gbw[g] = complete ? busbw(bn, den, span) : 0.0;
+      c_comp += complete; c_inc += !complete; c_bar += barrier; c_an += analysed; c_mis += mism; c_pres += npres;
+      if (add_bw) best_merge(w_brng, w_bk, tmax - tmin, t.seq_off + jg);
+    }
+    n_bwc += add_bw ? 1u : 0u;
+  }
+  // 4. per-rank bus bandwidth: warps -> shared memory -> one atomic per member and tile
+#pragma unroll
+  for (int r = 0; r < WARP_EMAX; ++r) { const u32 p = r * 32 + lane; if (p < n_pad) s_bw[wid * n_pad + p] = bwacc[r]; }
+  n_fs = __reduce_add_sync(0xFFFFFFFFu, n_fs); n_fd = __reduce_add_sync(0xFFFFFFFFu, n_fd);
+  if (lane == 0) {
+    atomicAdd(&s_cnt[0], c_comp); atomicAdd(&s_cnt[1], c_inc); atomicAdd(&s_cnt[2], c_bar); atomicAdd(&s_cnt[3], c_an);
+    atomicAdd(&s_cnt[4], c_mis); atomicAdd(&s_cnt[5], c_pres); atomicAdd(&s_cnt[6], n_fs); atomicAdd(&s_cnt[7], n_fd);
+    s_brng[wid] = w_brng; s_bk[wid] = w_bk; s_rounds[wid] = n_bwc;
+  }
+  __syncthreads();
+  u32 rounds = 0;
+  for (int q = 0; q < MID_THREADS / 32; ++q) rounds += s_rounds[q];
+  if (rounds) {
+    for (u32 p = threadIdx.x; p < n; p += MID_THREADS) {
+      double v = 0.0;
+      for (int q = 0; q < MID_THREADS / 32; ++q) v += s_bw[q * n_pad + p];
+      atomicAdd(&R.bw_sum[mem[p]], v);
+      atomicAdd(&R.bw_cnt[mem[p]], rounds);
+    }
+  }
+  if (threadIdx.x == 0) {
+    u64 brng = s_brng[0]; u32 bk = s_bk[0];
+    for (int q = 1; q < MID_THREADS / 32; ++q) best_merge(brng, bk, s_brng[q], s_bk[q]);
+    TileSum ts; ts.best_rng = brng; ts.best_k = bk; ts.n_rounds = rounds; ts.n_an = s_cnt[3]; ts.pad = 0;
+    sums[blockIdx.x] = ts;
+    count_add(D.counters, C_COMPLETE, s_cnt[0]); count_add(D.counters, C_INCOMPLETE, s_cnt[1]); count_add(D.counters, C_BARRIER, s_cnt[2]);
+    count_add(D.counters, C_ANALYSED, s_cnt[3]); count_add(D.counters, C_MISMATCH, s_cnt[4]); count_add(D.counters, C_PRESENT, s_cnt[5]);
+    count_add(D.counters, C_FLAG_SKEW, s_cnt[6]); count_add(D.counters, C_FLAG_DUR, s_cnt[7]);
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -754,7 +1054,7 @@ __device__ u64 radix_select(F key, u32 n, u32 k, u64 max_key, u32* hist /*[256]*
 }
 
 __global__ void __launch_bounds__(LARGE_THREADS) k_reduce_large(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles,
-                                                                 Registry R, Params P, i64 now) {
+                                                                 TileSum* __restrict__ sums, Registry R, Params P, i64 now) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   __shared__ u64 s_red64[32];
   __shared__ u32 s_red32[32];
@@ -771,7 +1071,8 @@ __global__ void __launch_bounds__(LARGE_THREADS) k_reduce_large(const WinDesc* _
   double bwacc[LARGE_MAXP];               // member p = threadIdx.x + q * LARGE_THREADS
 #pragma unroll
   for (int q = 0; q < LARGE_MAXP; ++q) bwacc[q] = 0.0;
-  u32 n_bwc = 0;
+  u32 n_bwc = 0, n_an_tile = 0;
+  u64 t_brng = 0; u32 t_bk = NONE;
 
   for (u32 jg = 0; jg < t.count; ++jg) {
     __syncthreads();
@@ -854,7 +1155,8 @@ __global__ void __launch_bounds__(LARGE_THREADS) k_reduce_large(const WinDesc* _
     double num, den; bus_factor(gop, n, &num, &den);
     const double bn = (double)gbytes * num;
     if (!barrier) {
-      ++n_bwc;
+      ++n_bwc; n_an_tile += analysed ? 1u : 0u;
+      best_merge(t_brng, t_bk, tmax - tmin, t.seq_off + jg);
 #pragma unroll
       for (int q = 0; q < LARGE_MAXP; ++q) { const u32 p = threadIdx.x + q * LARGE_THREADS; if (p < n) bwacc[q] += busbw(bn, den, (i64)s_du[p]); }
     }
@@ -895,6 +1197,7 @@ __global__ void __launch_bounds__(LARGE_THREADS) k_reduce_large(const WinDesc* _
       count_add(D.counters, C_FLAG_SKEW, n_fs); count_add(D.counters, C_FLAG_DUR, n_fd);
     }
   }  // groups of the tile
+  if (threadIdx.x == 0) { TileSum ts; ts.best_rng = t_brng; ts.best_k = t_bk; ts.n_rounds = n_bwc; ts.n_an = n_an_tile; ts.pad = 0; sums[blockIdx.x] = ts; }
   if (n_bwc) {
 #pragma unroll
     for (int q = 0; q < LARGE_MAXP; ++q) {
@@ -911,7 +1214,7 @@ __global__ void __launch_bounds__(LARGE_THREADS) k_reduce_large(const WinDesc* _
 __global__ void __launch_bounds__(128) k_window_decide(const WinDesc* __restrict__ wd, u32 nw, Registry R, Params P) {
   const u32 c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (c >= R.n_comms) return;
-  const u32 n = R.comm_n[c];
+  const u32 n = R.comm_n[c], cls = comm_class(n), S_tile = tile_seqs(n);
   const u32* mem = R.members + R.comm_moff[c];
   CommState st = R.state[c];
   for (u32 w = 0; w < nw; ++w) {
@@ -919,44 +1222,43 @@ __global__ void __launch_bounds__(128) k_window_decide(const WinDesc* __restrict
     const RangeRow row = D.ranges[c];
     if (row.n_seq == 0) continue;
     const u64 G = D.n_groups;
-    const u32* gfl = D.gu32 + (u64)GU_GFLAGS * G + row.group0;
-    const i64* e_min = D.gi64 + (u64)GI_E_MIN * G + row.group0;
     const i64* t_max = D.gi64 + (u64)GI_T_MAX * G + row.group0;
     const i64* t_min = D.gi64 + (u64)GI_T_MIN * G + row.group0;
+    // round counts and the Eq. 2 candidate come from the tile summaries the reduce kernels left behind
+    const TileSum* ts = D.tsum[cls] + row.tile0;
+    const u32 nt = (row.n_seq + S_tile - 1) / S_tile;
     u32 n_rounds = 0, n_an = 0;
     u64 best_rng = 0; u32 best_k = NONE;
-    for (u32 k0 = 0; k0 < row.n_seq; k0 += 32) {
-      const u32 k = k0 + lane;
-      const u32 f = k < row.n_seq ? gfl[k] : 0;
-      const bool round = (f & CCLD_G_COMPLETE) && !(f & CCLD_G_BARRIER);
-      const u32 rmask = __ballot_sync(0xFFFFFFFFu, round);
-      n_rounds += __popc(rmask);
-      n_an += __popc(__ballot_sync(0xFFFFFFFFu, (f & CCLD_G_ANALYSED) != 0));
-      i64 em = 0, tM = 0, tm = 0;
-      if (round) { em = e_min[k]; tM = t_max[k]; tm = t_min[k]; }
-      // Eq. 1: rounds feed the baseline, in op-counter order, until m is fixed
-      if (st.m == 0) {
-        u32 rem = rmask;
+    for (u32 q = lane; q < nt; q += 32) {
+      const TileSum x = ts[q];
+      n_rounds += x.n_rounds; n_an += x.n_an;
+      best_merge(best_rng, best_k, x.best_rng, x.best_k);
+    }
+    n_rounds = __reduce_add_sync(0xFFFFFFFFu, n_rounds); n_an = __reduce_add_sync(0xFFFFFFFFu, n_an);
+    best_warp_reduce(best_rng, best_k);
+    // Eq. 1: rounds feed the baseline, in op-counter order, until m is fixed
+    u32 walked = 0;
+    if (st.m == 0 && n_rounds > 0) {
+      const u32* gfl = D.gu32 + (u64)GU_GFLAGS * G + row.group0;
+      const i64* e_min = D.gi64 + (u64)GI_E_MIN * G + row.group0;
+      for (u32 k0 = 0; k0 < row.n_seq && st.m == 0; k0 += 32) {
+        const u32 k = k0 + lane;
+        const u32 f = k < row.n_seq ? gfl[k] : 0;
+        const bool round = (f & CCLD_G_COMPLETE) && !(f & CCLD_G_BARRIER);
+        u32 rem = __ballot_sync(0xFFFFFFFFu, round);
+        i64 em = 0, tM = 0;
+        if (round) { em = e_min[k]; tM = t_max[k]; }
         while (rem && st.m == 0) {
           const int src = __ffs(rem) - 1; rem &= rem - 1;
           const i64 em_s = __shfl_sync(0xFFFFFFFFu, em, src), tM_s = __shfl_sync(0xFFFFFFFFu, tM, src);
           if (st.rounds == 0) st.t_first = em_s;
           if (st.rounds == (u64)P.m_max_rounds || (st.rounds > 0 && em_s - st.t_first >= P.m_max_ns)) st.m = st.rounds;
           else st.sum_m += tM_s;
-          ++st.rounds;
+          ++st.rounds; ++walked;
         }
-        st.rounds += __popc(rem);
-      } else {
-        st.rounds += __popc(rmask);
       }
-      // Eq. 2: largest intra-round range, earliest op counter among equals
-      if (round) { const u64 rg = (u64)(tM - tm); if (best_k == NONE || rg > best_rng) { best_rng = rg; best_k = k; } }
     }
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
-      const u64 orng = shfl_xor64(best_rng, d); const u32 ok = __shfl_xor_sync(0xFFFFFFFFu, best_k, d);
-      if (ok != NONE && (best_k == NONE || orng > best_rng || (orng == best_rng && ok < best_k))) { best_rng = orng; best_k = ok; }
-    }
+    st.rounds += n_rounds - walked;
     // analysed ops of this window count towards every member's denominator
     if (n_an) for (u32 p = lane; p < n; p += 32) atomicAdd(&R.ops[mem[p]], n_an);
     if (lane == 0) {
