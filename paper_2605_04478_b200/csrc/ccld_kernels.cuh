@@ -267,10 +267,10 @@ __global__ void __launch_bounds__(REC_THREADS) k_slot_scatter(const WinDesc* __r
 // per-op reductions, n <= 8: one thread per group, lanes run along consecutive op counters so the
 // gathers of one member's records coalesce
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ void cswap(u64& a, u64& b) { u64 lo = a < b ? a : b; u64 hi = a < b ? b : a; a = lo; b = hi; }
+template <class K> __device__ __forceinline__ void cswap(K& a, K& b) { const K lo = a < b ? a : b; const K hi = a < b ? b : a; a = lo; b = hi; }
 
 // 19-exchange sorting network for 8 keys
-__device__ __forceinline__ void sort8(u64 (&v)[8]) {
+template <class K> __device__ __forceinline__ void sort8(K (&v)[8]) {
   cswap(v[0], v[2]); cswap(v[1], v[3]); cswap(v[4], v[6]); cswap(v[5], v[7]);
   cswap(v[0], v[4]); cswap(v[1], v[5]); cswap(v[2], v[6]); cswap(v[3], v[7]);
   cswap(v[0], v[1]); cswap(v[2], v[3]); cswap(v[4], v[5]); cswap(v[6], v[7]);
@@ -279,43 +279,110 @@ __device__ __forceinline__ void sort8(u64 (&v)[8]) {
   cswap(v[1], v[2]); cswap(v[3], v[4]); cswap(v[5], v[6]);
 }
 // bitonic merge: sorts 8 keys that first fall and then rise
-__device__ __forceinline__ void merge8(u64 (&v)[8]) {
+template <class K> __device__ __forceinline__ void merge8(K (&v)[8]) {
   cswap(v[0], v[4]); cswap(v[1], v[5]); cswap(v[2], v[6]); cswap(v[3], v[7]);
   cswap(v[0], v[2]); cswap(v[1], v[3]); cswap(v[4], v[6]); cswap(v[5], v[7]);
   cswap(v[0], v[1]); cswap(v[2], v[3]); cswap(v[4], v[5]); cswap(v[6], v[7]);
 }
-__device__ __forceinline__ u64 pick4(const u64 (&v)[8], u32 k) {
-  u64 r = v[0];
+template <class K> __device__ __forceinline__ K pick4(const K (&v)[8], u32 k) {
+  K r = v[0];
   r = k == 1 ? v[1] : r; r = k == 2 ? v[2] : r; r = k == 3 ? v[3] : r;
   return r;
 }
 
-// lower median and lower-median absolute deviation of x[0..n), n <= 8 (x[p] = U64_MAX for p >= n)
-__device__ __forceinline__ void median_mad8(const u64 (&x)[8], u32 n, u64* med, u64* mad) {
-  u64 s[8];
+template <class K> struct KeyMax;
+template <> struct KeyMax<u32> { static __device__ __forceinline__ u32 v() { return 0xFFFFFFFFu; } };
+template <> struct KeyMax<u64> { static __device__ __forceinline__ u64 v() { return U64_MAX_; } };
+
+// lower median and lower-median absolute deviation of x[0..n), n <= 8 (x[p] = maximum key for p >= n)
+template <class K> __device__ __forceinline__ void median_mad8(const K (&x)[8], u32 n, K* med, K* mad) {
+  K s[8];
 #pragma unroll
   for (int p = 0; p < 8; ++p) s[p] = x[p];
   sort8(s);
   const u32 k = (n - 1) >> 1;
-  const u64 m = pick4(s, k);
+  const K m = pick4(s, k);
 #pragma unroll
-  for (int p = 0; p < 8; ++p) s[p] = (u32)p < n ? absdiff(s[p], m) : U64_MAX_;   // falls to 0 at k, then rises
+  for (int p = 0; p < 8; ++p) s[p] = (u32)p < n ? (s[p] >= m ? s[p] - m : m - s[p]) : KeyMax<K>::v();   // falls to 0 at k, then rises
   merge8(s);
   *med = m; *mad = pick4(s, k);
 }
 
-__global__ void __launch_bounds__(SMALL_SEQS) k_reduce_small(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles,
-                                                              TileSum* __restrict__ sums, Registry R, Params P, i64 now) {
-  __shared__ double s_bw[SMALL_SEQS / 32][SMALL_N];
-  __shared__ u64 s_brng[SMALL_SEQS / 32];
-  __shared__ u32 s_bk[SMALL_SEQS / 32];
-  const Tile t = tiles[blockIdx.x];
-  const WinDesc& D = wd[t.w];
-  const u32 c = t.c, n = R.comm_n[c];
+// 1 / x for x >= 1 to within a few ulp: single-precision seed and two Newton steps
+__device__ __forceinline__ double rcp_newton(double x) {
+  double r = (double)__frcp_rn((float)x);
+  double e = fma(-x, r, 1.0); r = fma(r, e, r);
+  e = fma(-x, r, 1.0); r = fma(r, e, r);
+  return r;
+}
+__device__ __forceinline__ double busbw_fast(double bytes_num, double den, i64 t) {
+  return t > 0 ? bytes_num * rcp_newton((double)t * den) : 0.0;
+}
+
+// Sums v[m] over the warp for m = 0..7 with 9 shuffles; lane l ends up with the total of member
+// m = 4 * bit4(l) + 2 * bit3(l) + bit2(l).
+__device__ __forceinline__ double warp_sum8(double (&v)[8], u32 lane) {
+#pragma unroll
+  for (int w = 4, bit = 16; w >= 1; w >>= 1, bit >>= 1) {
+    const bool hi = (lane & bit) != 0;
+#pragma unroll
+    for (int i = 0; i < w; ++i) {
+      const double send = hi ? v[i] : v[i + w], keep = hi ? v[i + w] : v[i];
+      v[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, bit);
+    }
+  }
+  v[0] += __shfl_xor_sync(0xFFFFFFFFu, v[0], 2);
+  v[0] += __shfl_xor_sync(0xFFFFFFFFu, v[0], 1);
+  return v[0];
+}
+
+// A complete group whose skews or durations do not fit 32-bit keys (a spread of more than 4.29 s inside
+// one op): gathered again and handled here, out of line, so that the common path stays in 32 bits.
+// Returns the four order statistics, the packed flag bytes, and adds the members' bus bandwidths.
+__device__ __noinline__ u64 small_group64(const WinDesc& D, const Registry& R, const u32* mem, u64 slot, u32 n, u64 e_min, u32 k_milli,
+                                          bool analysed, bool add_bw, double bn, double den, u64* out4) {
+  u64 sk[8], du[8];
+#pragma unroll
+  for (int p = 0; p < 8; ++p) {
+    sk[p] = U64_MAX_; du[p] = U64_MAX_;
+    if ((u32)p < n) { const u32 idx = D.perm[slot + p]; const i64 a = D.t_enter[idx], b = D.t_exit[idx]; sk[p] = (u64)a - e_min; du[p] = (u64)(b - a); }
+  }
+  if (add_bw)
+    for (u32 p = 0; p < n; ++p) atomicAdd(&R.bw_sum[mem[p]], busbw_fast(bn, den, (i64)du[p]));
+  u64 packed = 0;
+  out4[0] = out4[1] = out4[2] = out4[3] = 0;
+  if (analysed) {
+    u64 med_s, mad_s, med_d, mad_d;
+    median_mad8<u64>(sk, n, &med_s, &mad_s);
+    median_mad8<u64>(du, n, &med_d, &mad_d);
+    out4[0] = med_s; out4[1] = mad_s; out4[2] = med_d; out4[3] = mad_d;
+#pragma unroll
+    for (int p = 0; p < 8; ++p) {
+      if ((u32)p < n) {
+        const bool so = mul_gt(absdiff(sk[p], med_s), 1000u, mad_s, k_milli), sh = sk[p] > med_s;
+        const bool dq = mul_gt(absdiff(du[p], med_d), 1000u, mad_d, k_milli), dh = du[p] > med_d;
+        const u32 f = (so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0);
+        packed |= (u64)f << (8 * p);
+      }
+    }
+  } else {
+    for (u32 p = 0; p < n; ++p) packed |= (u64)CCLD_F_NOT_ANALYSED << (8 * p);
+  }
+  return packed;
+}
+
+enum { SC_COMP = 0, SC_INC, SC_BAR, SC_AN, SC_MIS, SC_BWC, SC_PRES, SC_FS, SC_FD, SC_COUNT };
+
+template <bool FULL>
+__device__ __forceinline__ void reduce_small_tile(const WinDesc& D, const Tile& t, TileSum* __restrict__ sums, const Registry& R, const Params& P,
+                                                  i64 now, u32 n_rt, double (*s_bw)[SMALL_N], u64* s_brng, u32* s_bk, u32* s_cnt) {
+  const u32 n = FULL ? (u32)SMALL_N : n_rt;
+  const u32 c = t.c;
   const RangeRow row = D.ranges[c];
   const u32* mem = R.members + R.comm_moff[c];
-  const u32 j = threadIdx.x;
+  const u32 j = threadIdx.x, lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const bool active = j < t.count;
+  const u32 k_milli = P.k_milli;
 
   double bw[SMALL_N];
 #pragma unroll
@@ -327,23 +394,32 @@ __global__ void __launch_bounds__(SMALL_SEQS) k_reduce_small(const WinDesc* __re
   if (active) {
     const u64 g = row.group0 + t.seq_off + j;
     const u64 slot = row.slot0 + (u64)(t.seq_off + j) * n;
+    u32 idx[SMALL_N];
+    if (FULL && (slot & 3) == 0) {
+      const uint4 a = *reinterpret_cast<const uint4*>(D.perm + slot), b = *reinterpret_cast<const uint4*>(D.perm + slot + 4);
+      idx[0] = a.x; idx[1] = a.y; idx[2] = a.z; idx[3] = a.w; idx[4] = b.x; idx[5] = b.y; idx[6] = b.z; idx[7] = b.w;
+    } else {
+#pragma unroll
+      for (int p = 0; p < SMALL_N; ++p) idx[p] = (FULL || (u32)p < n) ? D.perm[slot + p] : NONE;
+    }
     u64 te[SMALL_N], du[SMALL_N];
     i64 x_max = INT64_MIN, age = -1;
     u64 gbytes = 0; u32 gop = 0; bool have_first = false, inflight = false, bad_time = false;
     u32 max_chg = 0, pos_chg = 0; bool have_chg = false;
+    u32 miss = 0;
     complete = true;
 #pragma unroll
     for (int p = 0; p < SMALL_N; ++p) {
       te[p] = U64_MAX_; du[p] = U64_MAX_;
-      if ((u32)p < n) {
-        const u32 idx = D.perm[slot + p];
-        if (idx == NONE) { complete = false; }
+      if (FULL || (u32)p < n) {
+        const u32 ix = idx[p];
+        if (ix == NONE) { complete = false; miss |= 1u << p; }
         else {
           ++n_present;
-          const i64 a = D.t_enter[idx], b = D.t_exit[idx];
-          const u64 by = D.bytes[idx]; const u32 o = D.op[idx];
+          const i64 a = D.t_enter[ix], b = D.t_exit[ix];
+          const u64 by = D.bytes[ix]; const u32 o = D.op[ix];
           u32 ch = 0;
-          if (D.send_chg != nullptr) { const u32 sc = D.send_chg[idx], rc = D.recv_chg[idx]; ch = sc > rc ? sc : rc; }
+          if (D.send_chg != nullptr) { const u32 sc = D.send_chg[ix], rc = D.recv_chg[ix]; ch = sc > rc ? sc : rc; }
           if (!have_first) { gbytes = by; gop = o; have_first = true; }
           else if (o != gop || by != gbytes) mismatch = true;
           if (b == -1) { inflight = true; complete = false; const i64 ag = now - a; age = ag > age ? ag : age; }
@@ -357,110 +433,135 @@ __global__ void __launch_bounds__(SMALL_SEQS) k_reduce_small(const WinDesc* __re
     barrier = have_first && gop == CCLD_OP_ALLREDUCE && gbytes < P.barrier_bytes;
     u32 gfl = (mismatch ? CCLD_G_OPSET_MISMATCH : 0) | (barrier ? CCLD_G_BARRIER : 0) | (inflight ? CCLD_G_INFLIGHT : 0) |
               (bad_time ? CCLD_G_BAD_TIME : 0);
-    i64 out_i[GI_COUNT];
-#pragma unroll
-    for (int q = 0; q < GI_COUNT; ++q) out_i[q] = 0;
+    u64 o_emin = 0, o_askew = 0, o_tmax = 0, o_tmin = 0, med_s = 0, mad_s = 0, med_d = 0, mad_d = 0; i64 o_span = 0;
     u32 r_tmin = 0, r_tmax = 0, r_chg = 0; double gbw = 0.0;
-    u8 fl[SMALL_N];
+    u64 packed = 0;                                        // the group's flag bytes, member p in byte p
 #pragma unroll
-    for (int p = 0; p < SMALL_N; ++p) fl[p] = CCLD_F_NOT_ANALYSED;
+    for (int p = 0; p < SMALL_N; ++p)
+      if (FULL || (u32)p < n) packed |= (u64)(CCLD_F_NOT_ANALYSED | ((miss >> p) & 1u ? CCLD_F_MISSING : 0)) << (8 * p);
 
     if (!complete) {
       gfl |= CCLD_G_INCOMPLETE;
       max_chg = 0;
       if (inflight && age > P.hang_ns && !barrier) { gfl |= CCLD_G_HANG_ALERT; raise_alert(D, R.comm_id[c], row.seq_lo + t.seq_off + j, age); }
-#pragma unroll
-      for (int p = 0; p < SMALL_N; ++p)
-        if ((u32)p < n && D.perm[slot + p] == NONE) fl[p] = CCLD_F_NOT_ANALYSED | CCLD_F_MISSING;
     } else {
       gfl |= CCLD_G_COMPLETE;
-      u64 e_min = U64_MAX_, tmax = 0, tmin = U64_MAX_; u32 pmax = 0, pmin = 0;
+      u64 e_min = te[0], e_max = te[0], tmax = du[0], tmin = du[0]; u32 pmax = 0, pmin = 0;
 #pragma unroll
-      for (int p = 0; p < SMALL_N; ++p) if ((u32)p < n) { e_min = te[p] < e_min ? te[p] : e_min; }
-      u64 sk[SMALL_N], askew = 0;
-#pragma unroll
-      for (int p = 0; p < SMALL_N; ++p) {
-        sk[p] = U64_MAX_;
-        if ((u32)p < n) {
-          sk[p] = te[p] - e_min; askew = sk[p] > askew ? sk[p] : askew;
-          if (p == 0 || du[p] > tmax) { tmax = du[p]; pmax = p; }
-          if (p == 0 || du[p] < tmin) { tmin = du[p]; pmin = p; }
+      for (int p = 1; p < SMALL_N; ++p) {
+        if (FULL || (u32)p < n) {
+          e_min = te[p] < e_min ? te[p] : e_min; e_max = te[p] > e_max ? te[p] : e_max;
+          if (du[p] > tmax) { tmax = du[p]; pmax = p; }
+          if (du[p] < tmin) { tmin = du[p]; pmin = p; }
         }
       }
+      const u64 askew = e_max - e_min;
       const i64 span = x_max - (i64)e_min;
       double num, den; bus_factor(gop, n, &num, &den);
       const double bn = (double)gbytes * num;
-      gbw = busbw(bn, den, span);
-      out_i[GI_E_MIN] = (i64)e_min; out_i[GI_ARRIVAL_SKEW] = (i64)askew; out_i[GI_T_MAX] = (i64)tmax; out_i[GI_T_MIN] = (i64)tmin;
-      out_i[GI_SPAN] = span;
+      gbw = busbw_fast(bn, den, span);
+      o_emin = e_min; o_askew = askew; o_tmax = tmax; o_tmin = tmin; o_span = span;
       my_rng = tmax - tmin;
       r_tmin = mem[pmin]; r_tmax = mem[pmax]; r_chg = mem[pos_chg];
-      if (!barrier) {
-#pragma unroll
-        for (int p = 0; p < SMALL_N; ++p) if ((u32)p < n) bw[p] = busbw(bn, den, (i64)du[p]);
-      }
       analysed = !barrier && n >= P.min_group;
-      if (analysed) {
-        gfl |= CCLD_G_ANALYSED;
-        u64 med_s, mad_s, med_d, mad_d;
-        median_mad8(sk, n, &med_s, &mad_s);
-        median_mad8(du, n, &med_d, &mad_d);
-        out_i[GI_MED_SKEW] = (i64)med_s; out_i[GI_MAD_SKEW] = (i64)mad_s; out_i[GI_MED_DUR] = (i64)med_d; out_i[GI_MAD_DUR] = (i64)mad_d;
+      if (analysed) gfl |= CCLD_G_ANALYSED;
+      if (askew < 0xFFFFFFFFull && my_rng < 0xFFFFFFFFull) {
+        // 32-bit keys from here on: skew, and duration minus the shortest duration
+        u32 sk[SMALL_N], dd[SMALL_N];
 #pragma unroll
         for (int p = 0; p < SMALL_N; ++p) {
-          if ((u32)p < n) {
-            const bool so = mul_gt(absdiff(sk[p], med_s), 1000u, mad_s, P.k_milli), sh = sk[p] > med_s;
-            const bool dq = mul_gt(absdiff(du[p], med_d), 1000u, mad_d, P.k_milli), dh = du[p] > med_d;
-            fl[p] = (so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0);
-            if (so) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p] * 4 + (sh ? 0 : 1)], 1u); }
-            if (dq) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p] * 4 + (dh ? 2 : 3)], 1u); }
+          const bool in = FULL || (u32)p < n;
+          sk[p] = in ? (u32)(te[p] - e_min) : 0xFFFFFFFFu; dd[p] = in ? (u32)(du[p] - tmin) : 0xFFFFFFFFu;
+        }
+        if (analysed) {
+          u32 ms, ds, md, dm;
+          median_mad8<u32>(sk, n, &ms, &ds);
+          median_mad8<u32>(dd, n, &md, &dm);
+          med_s = ms; mad_s = ds; med_d = tmin + md; mad_d = dm;
+          const u64 ts = (u64)ds * k_milli, td = (u64)dm * k_milli;
+          packed = 0;
+#pragma unroll
+          for (int p = 0; p < SMALL_N; ++p) {
+            if (FULL || (u32)p < n) {
+              const u32 a = sk[p] >= ms ? sk[p] - ms : ms - sk[p], b = dd[p] >= md ? dd[p] - md : md - dd[p];
+              const bool so = (u64)a * 1000u > ts, sh = sk[p] > ms, dq = (u64)b * 1000u > td, dh = dd[p] > md;
+              packed |= (u64)((so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0)) << (8 * p);
+            }
+          }
+        }
+        if (!barrier) {
+#pragma unroll
+          for (int p = 0; p < SMALL_N; ++p) if (FULL || (u32)p < n) bw[p] = busbw_fast(bn, den, (i64)(tmin + dd[p]));
+        }
+      } else {
+        u64 o4[4];
+        packed = small_group64(D, R, mem, slot, n, e_min, k_milli, analysed, !barrier, bn, den, o4);
+        med_s = o4[0]; mad_s = o4[1]; med_d = o4[2]; mad_d = o4[3];
+      }
+      if (analysed) {
+#pragma unroll
+        for (int p = 0; p < SMALL_N; ++p) {
+          if (FULL || (u32)p < n) {
+            const u32 f = (u32)(packed >> (8 * p));
+            if (f & CCLD_F_SKEW_OUT) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p] * 4 + ((f & CCLD_F_SKEW_HI) ? 0 : 1)], 1u); }
+            if (f & CCLD_F_DUR_OUT) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p] * 4 + ((f & CCLD_F_DUR_HI) ? 2 : 3)], 1u); }
           }
         }
       }
     }
     // ---- outputs ----
     const u64 G = D.n_groups;
-#pragma unroll
-    for (int q = 0; q < GI_COUNT; ++q) D.gi64[(u64)q * G + g] = out_i[q];
+    D.gi64[(u64)GI_E_MIN * G + g] = (i64)o_emin; D.gi64[(u64)GI_ARRIVAL_SKEW * G + g] = (i64)o_askew;
+    D.gi64[(u64)GI_T_MAX * G + g] = (i64)o_tmax; D.gi64[(u64)GI_T_MIN * G + g] = (i64)o_tmin; D.gi64[(u64)GI_SPAN * G + g] = o_span;
+    D.gi64[(u64)GI_MED_SKEW * G + g] = (i64)med_s; D.gi64[(u64)GI_MAD_SKEW * G + g] = (i64)mad_s;
+    D.gi64[(u64)GI_MED_DUR * G + g] = (i64)med_d; D.gi64[(u64)GI_MAD_DUR * G + g] = (i64)mad_d;
     D.gu32[(u64)GU_RANK_TMIN * G + g] = r_tmin; D.gu32[(u64)GU_RANK_TMAX * G + g] = r_tmax;
     D.gu32[(u64)GU_MAX_CHG * G + g] = max_chg; D.gu32[(u64)GU_RANK_MAX_CHG * G + g] = r_chg;
     D.gu32[(u64)GU_N_PRESENT * G + g] = n_present; D.gu32[(u64)GU_GFLAGS * G + g] = gfl;
     D.gbw[g] = gbw;
+    if (FULL && (slot & 7) == 0) {
+      *reinterpret_cast<u64*>(D.flags + slot) = packed;
+    } else {
 #pragma unroll
-    for (int p = 0; p < SMALL_N; ++p) if ((u32)p < n) D.flags[slot + p] = fl[p];
+      for (int p = 0; p < SMALL_N; ++p) if (FULL || (u32)p < n) D.flags[slot + p] = (u8)(packed >> (8 * p));
+    }
   }
 
-  // ---- per-tile accumulation: counters and the per-rank bandwidth sums ----
-  const u32 n_comp = __syncthreads_count(active && complete);
-  const u32 n_inc = __syncthreads_count(active && !complete);
-  const u32 n_bar = __syncthreads_count(active && barrier);
-  const u32 n_an = __syncthreads_count(active && analysed);
-  const u32 n_mis = __syncthreads_count(active && mismatch);
-  const u32 n_bwc = __syncthreads_count(active && complete && !barrier);
-  u32 pres = __reduce_add_sync(0xFFFFFFFFu, n_present), fs = __reduce_add_sync(0xFFFFFFFFu, n_fs), fd = __reduce_add_sync(0xFFFFFFFFu, n_fd);
-  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-#pragma unroll
-  for (int p = 0; p < SMALL_N; ++p) {
-    double v = bw[p];
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, d);
-    if (lane == 0) s_bw[wid][p] = v;
-  }
+  // ---- per-tile accumulation: counters, Eq. 2 candidate and the per-rank bandwidth sums ----
+  const bool is_round = active && complete && !barrier;
   {
-    const bool is_round = active && complete && !barrier;
+    const u32 b_comp = __ballot_sync(0xFFFFFFFFu, active && complete), b_inc = __ballot_sync(0xFFFFFFFFu, active && !complete);
+    const u32 b_bar = __ballot_sync(0xFFFFFFFFu, active && barrier), b_an = __ballot_sync(0xFFFFFFFFu, active && analysed);
+    const u32 b_mis = __ballot_sync(0xFFFFFFFFu, active && mismatch), b_bwc = __ballot_sync(0xFFFFFFFFu, is_round);
+    const u32 pres = __reduce_add_sync(0xFFFFFFFFu, n_present), fs = __reduce_add_sync(0xFFFFFFFFu, n_fs), fd = __reduce_add_sync(0xFFFFFFFFu, n_fd);
     u64 brng = is_round ? my_rng : 0; u32 bk = is_round ? t.seq_off + j : NONE;
     best_warp_reduce(brng, bk);
-    if (lane == 0) { s_brng[wid] = brng; s_bk[wid] = bk; }
+    const double tot = warp_sum8(bw, lane);
+    if ((lane & 3) == 0) s_bw[wid][lane >> 2] = tot;
+    if (lane == 0) {
+      s_brng[wid] = brng; s_bk[wid] = bk;
+      if (b_comp) atomicAdd(&s_cnt[SC_COMP], (u32)__popc(b_comp));
+      if (b_inc) atomicAdd(&s_cnt[SC_INC], (u32)__popc(b_inc));
+      if (b_bar) atomicAdd(&s_cnt[SC_BAR], (u32)__popc(b_bar));
+      if (b_an) atomicAdd(&s_cnt[SC_AN], (u32)__popc(b_an));
+      if (b_mis) atomicAdd(&s_cnt[SC_MIS], (u32)__popc(b_mis));
+      if (b_bwc) atomicAdd(&s_cnt[SC_BWC], (u32)__popc(b_bwc));
+      if (pres) atomicAdd(&s_cnt[SC_PRES], pres);
+      if (fs) atomicAdd(&s_cnt[SC_FS], fs);
+      if (fd) atomicAdd(&s_cnt[SC_FD], fd);
+    }
   }
-  if (lane == 0) { count_add(D.counters, C_PRESENT, pres); count_add(D.counters, C_FLAG_SKEW, fs); count_add(D.counters, C_FLAG_DUR, fd); }
   __syncthreads();
+  const u32 n_bwc = s_cnt[SC_BWC];
   if (threadIdx.x == 0) {
     u64 brng = s_brng[0]; u32 bk = s_bk[0];
     for (int q = 1; q < SMALL_SEQS / 32; ++q) best_merge(brng, bk, s_brng[q], s_bk[q]);
-    TileSum ts; ts.best_rng = brng; ts.best_k = bk; ts.n_rounds = n_bwc; ts.n_an = n_an; ts.pad = 0;
+    TileSum ts; ts.best_rng = brng; ts.best_k = bk; ts.n_rounds = n_bwc; ts.n_an = s_cnt[SC_AN]; ts.pad = 0;
     sums[blockIdx.x] = ts;
-    count_add(D.counters, C_COMPLETE, n_comp); count_add(D.counters, C_INCOMPLETE, n_inc); count_add(D.counters, C_BARRIER, n_bar);
-    count_add(D.counters, C_ANALYSED, n_an); count_add(D.counters, C_MISMATCH, n_mis);
+    count_add(D.counters, C_COMPLETE, s_cnt[SC_COMP]); count_add(D.counters, C_INCOMPLETE, s_cnt[SC_INC]);
+    count_add(D.counters, C_BARRIER, s_cnt[SC_BAR]); count_add(D.counters, C_ANALYSED, s_cnt[SC_AN]);
+    count_add(D.counters, C_MISMATCH, s_cnt[SC_MIS]); count_add(D.counters, C_PRESENT, s_cnt[SC_PRES]);
+    count_add(D.counters, C_FLAG_SKEW, s_cnt[SC_FS]); count_add(D.counters, C_FLAG_DUR, s_cnt[SC_FD]);
   }
   if (threadIdx.x < n && n_bwc) {
     double v = 0.0;
@@ -469,6 +570,21 @@ __global__ void __launch_bounds__(SMALL_SEQS) k_reduce_small(const WinDesc* __re
     atomicAdd(&R.bw_sum[mem[threadIdx.x]], v);
     atomicAdd(&R.bw_cnt[mem[threadIdx.x]], n_bwc);
   }
+}
+
+__global__ void __launch_bounds__(SMALL_SEQS) k_reduce_small(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles,
+                                                                 TileSum* __restrict__ sums, Registry R, Params P, i64 now) {
+  __shared__ double s_bw[SMALL_SEQS / 32][SMALL_N];
+  __shared__ u64 s_brng[SMALL_SEQS / 32];
+  __shared__ u32 s_bk[SMALL_SEQS / 32];
+  __shared__ u32 s_cnt[SC_COUNT];
+  if (threadIdx.x < SC_COUNT) s_cnt[threadIdx.x] = 0;
+  __syncthreads();
+  const Tile t = tiles[blockIdx.x];
+  const WinDesc& D = wd[t.w];
+  const u32 n = R.comm_n[t.c];
+  if (n == SMALL_N) reduce_small_tile<true>(D, t, sums, R, P, now, n, s_bw, s_brng, s_bk, s_cnt);
+  else reduce_small_tile<false>(D, t, sums, R, P, now, n, s_bw, s_brng, s_bk, s_cnt);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -735,9 +851,6 @@ inline size_t mid_smem_bytes(u32 n_pad_min) {
 // bitonic network over E = n_pad / 32 registers per lane (32-bit keys whenever the group's value
 // range fits), flags straight to global memory. No block-wide barrier inside the sort.
 // ------------------------------------------------------------------------------------------------
-template <class K> struct KeyMax;
-template <> struct KeyMax<u32> { static __device__ __forceinline__ u32 v() { return 0xFFFFFFFFu; } };
-template <> struct KeyMax<u64> { static __device__ __forceinline__ u64 v() { return U64_MAX_; } };
 
 // Element i = r * 32 + lane of the warp's 32 E keys. Full sort, or (MERGE) the last merge phase only,
 // which sorts a sequence that falls and then rises.
