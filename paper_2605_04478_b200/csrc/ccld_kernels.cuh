@@ -402,6 +402,16 @@ __device__ __forceinline__ void reduce_small_tile(const WinDesc& D, const Tile& 
 #pragma unroll
       for (int p = 0; p < SMALL_N; ++p) idx[p] = (FULL || (u32)p < n) ? D.perm[slot + p] : NONE;
     }
+    // every gather is issued before any is used: a missing member reads record 0 and is masked out below
+    i64 ld_a[SMALL_N], ld_b[SMALL_N]; u64 ld_by[SMALL_N]; u32 ld_op[SMALL_N], ld_ch[SMALL_N];
+    const bool have_rates = D.send_chg != nullptr;
+#pragma unroll
+    for (int p = 0; p < SMALL_N; ++p) {
+      const u32 ix = idx[p] == NONE ? 0u : idx[p];
+      ld_a[p] = D.t_enter[ix]; ld_b[p] = D.t_exit[ix]; ld_by[p] = D.bytes[ix]; ld_op[p] = D.op[ix];
+      ld_ch[p] = 0;
+      if (have_rates) { const u32 sc = D.send_chg[ix], rc = D.recv_chg[ix]; ld_ch[p] = sc > rc ? sc : rc; }
+    }
     u64 te[SMALL_N], du[SMALL_N];
     i64 x_max = INT64_MIN, age = -1;
     u64 gbytes = 0; u32 gop = 0; bool have_first = false, inflight = false, bad_time = false;
@@ -412,14 +422,12 @@ __device__ __forceinline__ void reduce_small_tile(const WinDesc& D, const Tile& 
     for (int p = 0; p < SMALL_N; ++p) {
       te[p] = U64_MAX_; du[p] = U64_MAX_;
       if (FULL || (u32)p < n) {
-        const u32 ix = idx[p];
-        if (ix == NONE) { complete = false; miss |= 1u << p; }
+        if (idx[p] == NONE) { complete = false; miss |= 1u << p; }
         else {
           ++n_present;
-          const i64 a = D.t_enter[ix], b = D.t_exit[ix];
-          const u64 by = D.bytes[ix]; const u32 o = D.op[ix];
-          u32 ch = 0;
-          if (D.send_chg != nullptr) { const u32 sc = D.send_chg[ix], rc = D.recv_chg[ix]; ch = sc > rc ? sc : rc; }
+          const i64 a = ld_a[p], b = ld_b[p];
+          const u64 by = ld_by[p]; const u32 o = ld_op[p];
+          const u32 ch = ld_ch[p];
           if (!have_first) { gbytes = by; gop = o; have_first = true; }
           else if (o != gop || by != gbytes) mismatch = true;
           if (b == -1) { inflight = true; complete = false; const i64 ag = now - a; age = ag > age ? ag : age; }
@@ -960,14 +968,15 @@ __global__ void __launch_bounds__(MID_THREADS) k_reduce_warp(const WinDesc* __re
   for (u32 e = threadIdx.x; e < n_el; e += MID_THREADS) {
     const u32 p = e / S, jg = e - p * S, a = jg * pitch + p;
     const u32 idx = s_idx[a];
-    u64 te = 0, du = 0, by = 0; u32 ch = 0; u8 op = 0, st = 0;
+    const u32 ix = idx == NONE ? 0u : idx;                  // a missing member reads record 0 and is masked out
+    const i64 x = D.t_enter[ix], y = D.t_exit[ix];
+    u64 by = D.bytes[ix]; u32 ch = 0; u8 op = D.op[ix], st = 0;
+    if (D.send_chg != nullptr) { const u32 sc = D.send_chg[ix], rc = D.recv_chg[ix]; ch = sc > rc ? sc : rc; }
+    u64 te = 0, du = 0;
     if (idx != NONE) {
-      const i64 x = D.t_enter[idx], y = D.t_exit[idx];
-      by = D.bytes[idx]; op = D.op[idx];
-      if (D.send_chg != nullptr) { const u32 sc = D.send_chg[idx], rc = D.recv_chg[idx]; ch = sc > rc ? sc : rc; }
       st = 1 | (y == -1 ? 2 : ((x < 0 || y < x) ? 4 : 0));
       te = (u64)x; du = (u64)(y - x);
-    }
+    } else { by = 0; ch = 0; op = 0; }
     s_te[a] = te; s_du[a] = du; s_by[a] = by; s_ch[a] = ch; s_op[a] = op; s_st[a] = st;
   }
   __syncthreads();
