@@ -42,7 +42,8 @@ struct CommState { u64 rounds; i64 t_first; i64 sum_m; u64 m; u64 slow_count; };
 // Registered communicators (immutable after the first analysis) and cumulative per-rank statistics.
 struct Registry {
   u32 n_comms, hash_mask, n_ranks, pad;
-  const uint2* hash;        // open addressing: (communicator id, index), index NONE = empty
+  const uint4* hash;        // open addressing: (communicator id, index, seq0, n), index NONE = empty
+  const uint4* rank_tab;    // [n_ranks][2]: up to RANK_TAB_K inline (communicator id, index << 13 | position) pairs of a rank
   const u32* comm_id;       // [n_comms]
   const u32* comm_n;        // [n_comms] members
   const u32* comm_seq0;     // [n_comms]
@@ -57,6 +58,12 @@ struct Registry {
   u32* bw_cnt;              // [n_ranks]
   double* bw_sum;           // [n_ranks]
 };
+
+// rank_tab: pairs beyond RANK_TAB_K do not fit inline; the last pair then holds (NONE, RANK_TAB_OVERFLOW) and the
+// CSR lists are searched instead. Empty pairs are (NONE, NONE).
+constexpr int RANK_TAB_K = 4;
+constexpr u32 RANK_TAB_OVERFLOW = 0xFFFFFFFEu;
+constexpr u32 RANK_TAB_POS_BITS = 13;  // positions < CCLD_MAX_COMM_SIZE = 8192
 
 // Which op counters a communicator covers in a window and where its groups / slots start.
 struct RangeRow { u32 seq_lo, n_seq, row_idx, n; u64 group0, slot0; u32 tile0, pad; };   // tile0: first tile in its class list
@@ -83,6 +90,7 @@ struct WinDesc {
   u32 cta0, n_cta;                   // this window's CTAs in the record-streaming grids
   u32 *rmin, *rmax;                  // [n_comms] op counter range seen
   RangeRow* ranges;                  // [n_comms]
+  uint4* srow;                       // [n_comms] scatter rows: (slot0 - seq_lo * n) low, high, n (0 = nothing to place), seq_lo
   u64* totals;                       // [T_COUNT]
   u64* counters;                     // [C_COUNT]
   // sized after the plan:

@@ -153,7 +153,8 @@ int finalize_registry(ccld_ctx* ctx) {
   }
   const u32 nr = max_rank + 1;
   u32 hsize = 16; while (hsize < 2 * nc) hsize <<= 1;
-  std::vector<uint2> hash(hsize, make_uint2(0, NONE));
+  if (nc >= (1u << (32 - RANK_TAB_POS_BITS))) return fail(ctx, CCLD_ERR_CAPACITY, "too many communicators");
+  std::vector<uint4> hash(hsize, make_uint4(0, NONE, 0, 0));
   std::vector<u32> comm_id(nc), comm_n(nc), comm_seq0(nc), members; std::vector<u64> moff(nc);
   std::vector<u32> rank_ptr(nr + 1, 0);
   members.reserve(sum_n);
@@ -163,17 +164,29 @@ int finalize_registry(ccld_ctx* ctx) {
     members.insert(members.end(), c.ranks.begin(), c.ranks.end());
     u32 h = (c.id * 2654435761u) & (hsize - 1);
     while (hash[h].y != NONE) h = (h + 1) & (hsize - 1);
-    hash[h] = make_uint2(c.id, i);
+    hash[h] = make_uint4(c.id, i, c.seq0, (u32)c.ranks.size());
     for (u32 r : c.ranks) ++rank_ptr[r + 1];
   }
   for (u32 r = 0; r < nr; ++r) rank_ptr[r + 1] += rank_ptr[r];
   std::vector<u32> ent_comm(sum_n), ent_pos(sum_n), fill(rank_ptr.begin(), rank_ptr.end() - 1);
   for (u32 i = 0; i < nc; ++i)
     for (u32 p = 0; p < ctx->comms[i].ranks.size(); ++p) { u32 r = ctx->comms[i].ranks[p]; ent_comm[fill[r]] = i; ent_pos[fill[r]] = p; ++fill[r]; }
+  // inline (communicator id, index << 13 | position) pairs per rank, RANK_TAB_K of them in two uint4
+  std::vector<u32> rank_tab((size_t)nr * 2 * RANK_TAB_K, NONE);
+  for (u32 r = 0; r < nr; ++r) {
+    const u32 cnt = rank_ptr[r + 1] - rank_ptr[r];
+    const u32 inl = cnt <= (u32)RANK_TAB_K ? cnt : (u32)RANK_TAB_K - 1;
+    for (u32 k = 0; k < inl; ++k) {
+      const u32 ci = ent_comm[rank_ptr[r] + k];
+      rank_tab[((size_t)r * RANK_TAB_K + k) * 2] = ctx->comms[ci].id;
+      rank_tab[((size_t)r * RANK_TAB_K + k) * 2 + 1] = (ci << RANK_TAB_POS_BITS) | ent_pos[rank_ptr[r] + k];
+    }
+    if (cnt > (u32)RANK_TAB_K) rank_tab[((size_t)r * RANK_TAB_K + RANK_TAB_K - 1) * 2 + 1] = RANK_TAB_OVERFLOW;
+  }
 
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
-  const size_t o_hash = take(hsize * sizeof(uint2)), o_id = take(nc * 4), o_n = take(nc * 4), o_s0 = take(nc * 4), o_moff = take(nc * 8),
+  const size_t o_hash = take(hsize * sizeof(uint4)), o_rtab = take(rank_tab.size() * 4), o_id = take(nc * 4), o_n = take(nc * 4), o_s0 = take(nc * 4), o_moff = take(nc * 8),
                o_mem = take(sum_n * 4), o_ptr = take((nr + 1) * 4ull), o_ec = take(sum_n * 4), o_ep = take(sum_n * 4);
   const size_t o_stats = off;
   const size_t o_state = take(nc * sizeof(CommState)), o_votes = take(nr * 16ull), o_ops = take(nr * 4ull), o_cnt = take(nr * 4ull), o_bw = take(nr * 8ull);
@@ -182,7 +195,8 @@ int finalize_registry(ccld_ctx* ctx) {
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "registry allocation failed");
   char* base = (char*)ctx->reg_blk.p;
   cudaStream_t st = ctx->stream;
-  CK(cudaMemcpyAsync(base + o_hash, hash.data(), hsize * sizeof(uint2), cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(base + o_hash, hash.data(), hsize * sizeof(uint4), cudaMemcpyHostToDevice, st));
+  CK(cudaMemcpyAsync(base + o_rtab, rank_tab.data(), rank_tab.size() * 4, cudaMemcpyHostToDevice, st));
   CK(cudaMemcpyAsync(base + o_id, comm_id.data(), nc * 4, cudaMemcpyHostToDevice, st));
   CK(cudaMemcpyAsync(base + o_n, comm_n.data(), nc * 4, cudaMemcpyHostToDevice, st));
   CK(cudaMemcpyAsync(base + o_s0, comm_seq0.data(), nc * 4, cudaMemcpyHostToDevice, st));
@@ -195,7 +209,7 @@ int finalize_registry(ccld_ctx* ctx) {
   CK(cudaStreamSynchronize(st));              // the host vectors above go out of scope
   Registry& R = ctx->reg;
   R.n_comms = nc; R.hash_mask = hsize - 1; R.n_ranks = nr; R.pad = 0;
-  R.hash = (const uint2*)(base + o_hash); R.comm_id = (const u32*)(base + o_id); R.comm_n = (const u32*)(base + o_n);
+  R.hash = (const uint4*)(base + o_hash); R.rank_tab = (const uint4*)(base + o_rtab); R.comm_id = (const u32*)(base + o_id); R.comm_n = (const u32*)(base + o_n);
   R.comm_seq0 = (const u32*)(base + o_s0); R.comm_moff = (const u64*)(base + o_moff); R.members = (const u32*)(base + o_mem);
   R.rank_ptr = (const u32*)(base + o_ptr); R.ent_comm = (const u32*)(base + o_ec); R.ent_pos = (const u32*)(base + o_ep);
   R.state = (CommState*)(base + o_state); R.votes = (u32*)(base + o_votes); R.ops = (u32*)(base + o_ops);
@@ -379,7 +393,7 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   size_t off = 0;
   auto take = [&](size_t b) { size_t o = off; off = align_up(off + b); return o; };
   const size_t o_desc = take(B * sizeof(WinDesc)), o_rmin = take((size_t)B * nc * 4), o_rmax = take((size_t)B * nc * 4),
-               o_rng = take((size_t)B * nc * sizeof(RangeRow)), o_tot = take((size_t)B * T_COUNT * 8), o_cnt = take((size_t)B * C_COUNT * 8);
+               o_rng = take((size_t)B * nc * sizeof(RangeRow)), o_srow = take((size_t)B * nc * sizeof(uint4)), o_tot = take((size_t)B * T_COUNT * 8), o_cnt = take((size_t)B * C_COUNT * 8);
   cudaError_t e;
   Block pb = ctx->pool.get(off, &e);
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "plan allocation failed");
@@ -392,7 +406,7 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
     d.slot_cap = 2 * d.n_rec + ctx->sum_n;
     d.n_cta = (u32)((d.n_rec + REC_PER_CTA - 1) / REC_PER_CTA); d.cta0 = (u32)cta; cta += d.n_cta;
     d.rmin = (u32*)(pbase + o_rmin) + (size_t)k * nc; d.rmax = (u32*)(pbase + o_rmax) + (size_t)k * nc;
-    d.ranges = (RangeRow*)(pbase + o_rng) + (size_t)k * nc;
+    d.ranges = (RangeRow*)(pbase + o_rng) + (size_t)k * nc; d.srow = (uint4*)(pbase + o_srow) + (size_t)k * nc;
     d.totals = (u64*)(pbase + o_tot) + (size_t)k * T_COUNT; d.counters = (u64*)(pbase + o_cnt) + (size_t)k * C_COUNT;
     d.n_groups = d.n_slots = 0; d.perm = nullptr; d.flags = nullptr; d.gi64 = nullptr; d.gu32 = nullptr; d.gbw = nullptr;
     d.comm_rows = nullptr; d.alerts = nullptr;

@@ -20,16 +20,20 @@ namespace ccld {
 // ------------------------------------------------------------------------------------------------
 // small helpers
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ u32 comm_lookup(const Registry& R, u32 id) {
-  u32 h = (id * 2654435761u) & R.hash_mask;
+__device__ __forceinline__ u32 hash_home(const Registry& R, u32 id) { return (id * 2654435761u) & R.hash_mask; }
+
+// Continues a probe sequence whose first entry (at the home slot) the caller already holds.
+__device__ __forceinline__ uint4 comm_find(const Registry& R, u32 id, uint4 e) {
+  u32 h = hash_home(R, id);
   for (u32 probe = 0; probe <= R.hash_mask; ++probe) {
-    uint2 e = R.hash[h];
-    if (e.y == NONE) return NONE;
-    if (e.x == id) return e.y;
+    if (e.y == NONE || e.x == id) return e;
     h = (h + 1) & R.hash_mask;
+    e = R.hash[h];
   }
-  return NONE;
+  return make_uint4(0, NONE, 0, 0);
 }
+
+__device__ __forceinline__ u32 comm_lookup(const Registry& R, u32 id) { return comm_find(R, id, R.hash[hash_home(R, id)]).y; }
 
 __device__ __forceinline__ u32 pos_lookup(const Registry& R, u32 rank, u32 c) {
   if (rank >= R.n_ranks) return NONE;
@@ -92,29 +96,69 @@ __device__ __forceinline__ void best_warp_reduce(u64& rng, u32& k) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// group-by, part 1: which op counters does every communicator cover in every window
+// group-by, part 1: which op counters does every communicator cover in every window.
+// The dependent lookups of a thread's eight records are issued stage by stage (all hash probes, then
+// all range checks) so that their latencies overlap instead of adding up.
 // ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void range_widen(const WinDesc& D, u32 c, u32 mn, u32 mx) {
+  if (mn < __ldcg(&D.rmin[c])) atomicMin(&D.rmin[c], mn);
+  if (mx > __ldcg(&D.rmax[c])) atomicMax(&D.rmax[c], mx);
+}
+
+constexpr u32 RANGE_TAB = 64;           // per-CTA table of the communicators met; overflow goes straight to global memory
+
+__device__ __forceinline__ void range_note(const WinDesc& D, u32* t_key, u32* t_mn, u32* t_mx, u32 c, u32 mn, u32 mx) {
+  u32 h = c & (RANGE_TAB - 1);
+  for (u32 probe = 0; probe < RANGE_TAB; ++probe) {
+    const u32 old = atomicCAS(&t_key[h], NONE, c);
+    if (old == NONE || old == c) { atomicMin(&t_mn[h], mn); atomicMax(&t_mx[h], mx); return; }
+    h = (h + 1) & (RANGE_TAB - 1);
+  }
+  range_widen(D, c, mn, mx);
+}
+
 __global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __restrict__ wd, u32 nw, Registry R) {
+  __shared__ u32 t_key[RANGE_TAB], t_mn[RANGE_TAB], t_mx[RANGE_TAB];
+  if (threadIdx.x < RANGE_TAB) { t_key[threadIdx.x] = NONE; t_mn[threadIdx.x] = NONE; t_mx[threadIdx.x] = 0; }
+  __syncthreads();
   const u32 w = find_window(wd, nw, blockIdx.x);
   const WinDesc& D = wd[w];
   const u64 base = (u64)(blockIdx.x - D.cta0) * REC_PER_CTA;
-  const u32 lane = threadIdx.x & 31;
+  u32 cid[REC_PER_THREAD], sq[REC_PER_THREAD]; uint4 he[REC_PER_THREAD];
 #pragma unroll
   for (int k = 0; k < REC_PER_THREAD; ++k) {
     const u64 i = base + (u64)k * REC_THREADS + threadIdx.x;
     const bool in = i < D.n_rec;
-    const u32 cid = in ? D.comm[i] : 0u;
-    const u32 s = in ? D.seq[i] : 0u;
-    const u32 c = in ? comm_lookup(R, cid) : NONE;
-    const bool valid = c != NONE && s >= R.comm_seq0[c];
-    // one pair of atomics per distinct communicator in the warp, and only when it widens the range
-    const u32 m = __match_any_sync(0xFFFFFFFFu, valid ? c : NONE);
-    const u32 mn = __reduce_min_sync(m, s), mx = __reduce_max_sync(m, s);
-    if (valid && lane == (u32)(__ffs(m) - 1)) {
-      if (mn < D.rmin[c]) atomicMin(&D.rmin[c], mn);
-      if (mx > D.rmax[c]) atomicMax(&D.rmax[c], mx);
+    cid[k] = in ? D.comm[i] : NONE; sq[k] = in ? D.seq[i] : 0u;
+  }
+#pragma unroll
+  for (int k = 0; k < REC_PER_THREAD; ++k) he[k] = R.hash[hash_home(R, cid[k])];
+  // the thread's records are 256 apart: in a rank-major upload they cycle through a few communicators,
+  // so fold them into at most four (communicator, min, max) triples, then into the CTA's table
+  u32 uc[4], umn[4], umx[4]; int cnt = 0;
+#pragma unroll
+  for (int k = 0; k < REC_PER_THREAD; ++k) {
+    const u64 i = base + (u64)k * REC_THREADS + threadIdx.x;
+    const uint4 e = comm_find(R, cid[k], he[k]);
+    if (i < D.n_rec && e.y != NONE && sq[k] >= e.z) {
+      bool found = false;
+#pragma unroll
+      for (int q = 0; q < 4; ++q)
+        if (q < cnt && uc[q] == e.y) { umn[q] = sq[k] < umn[q] ? sq[k] : umn[q]; umx[q] = sq[k] > umx[q] ? sq[k] : umx[q]; found = true; }
+      if (!found) {
+        if (cnt == 4) range_note(D, t_key, t_mn, t_mx, e.y, sq[k], sq[k]);
+        else {
+#pragma unroll
+          for (int q = 0; q < 4; ++q) if (q == cnt) { uc[q] = e.y; umn[q] = sq[k]; umx[q] = sq[k]; }
+          ++cnt;
+        }
+      }
     }
   }
+#pragma unroll
+  for (int q = 0; q < 4; ++q) if (q < cnt) range_note(D, t_key, t_mn, t_mx, uc[q], umn[q], umx[q]);
+  __syncthreads();
+  if (threadIdx.x < RANGE_TAB && t_key[threadIdx.x] != NONE) range_widen(D, t_key[threadIdx.x], t_mn[threadIdx.x], t_mx[threadIdx.x]);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -199,6 +243,8 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
         r.seq_lo = it.rows ? D.rmin[c] : 0; r.n_seq = (u32)it.groups; r.row_idx = ex.rows; r.n = R.comm_n[c];
         r.group0 = ex.groups; r.slot0 = ex.slots; r.tile0 = 0; r.pad = 0;
         D.ranges[c] = r;
+        const u64 sb = r.slot0 - (u64)r.seq_lo * r.n;
+        D.srow[c] = make_uint4((u32)sb, (u32)(sb >> 32), it.rows ? r.n : 0u, r.seq_lo);
       } else if (it.rows) {
         const u32 n = R.comm_n[c], S = tile_seqs(n), cls = comm_class(n);
         const u32 first = D.tile0[cls] + ex.t[cls];
@@ -226,32 +272,78 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
   }
   __syncthreads();
   if (s_failed)
-    for (u32 c = threadIdx.x; c < R.n_comms; c += PLAN_THREADS) { RangeRow z = {0, 0, 0, R.comm_n[c], 0, 0, 0, 0}; D.ranges[c] = z; }
+    for (u32 c = threadIdx.x; c < R.n_comms; c += PLAN_THREADS) { RangeRow z = {0, 0, 0, R.comm_n[c], 0, 0, 0, 0}; D.ranges[c] = z; D.srow[c] = make_uint4(0, 0, 0, 0); }
 }
 
 // ------------------------------------------------------------------------------------------------
-// group-by, part 3: every accepted record drops its index into its slot
+// group-by, part 3: every accepted record drops its index into its slot. Two dependent loads per
+// record in the common case - the rank's inline (communicator, index, position) pairs, then the
+// communicator's scatter row - issued for four records at a time.
 // ------------------------------------------------------------------------------------------------
+// Registry walk for a record whose (rank, communicator) pair is not inline: returns index << 13 | position in the
+// low word, or NONE there with the rejecting CCLD_E_* bit in the high word.
+__device__ __noinline__ u64 resolve_slow(const Registry& R, u32 rank, u32 cid) {
+  const u32 c = comm_lookup(R, cid);
+  if (c == NONE) return ((u64)CCLD_E_UNKNOWN_COMM << 32) | NONE;
+  const u32 pos = pos_lookup(R, rank, c);
+  if (pos == NONE) return ((u64)CCLD_E_NOT_MEMBER << 32) | NONE;
+  return (c << RANK_TAB_POS_BITS) | pos;
+}
+
 __global__ void __launch_bounds__(REC_THREADS) k_slot_scatter(const WinDesc* __restrict__ wd, u32 nw, Registry R) {
   const u32 w = find_window(wd, nw, blockIdx.x);
   const WinDesc& D = wd[w];
   const u64 base = (u64)(blockIdx.x - D.cta0) * REC_PER_CTA;
   u32 err = 0, rej = 0, internal = 0;
+  constexpr int HALF = REC_PER_THREAD / 2;
 #pragma unroll
-  for (int k = 0; k < REC_PER_THREAD; ++k) {
-    const u64 i = base + (u64)k * REC_THREADS + threadIdx.x;
-    if (i >= D.n_rec) continue;
-    const u32 rk = D.rank[i], cid = D.comm[i], s = D.seq[i];
-    const u32 c = comm_lookup(R, cid);
-    if (c == NONE) { err |= CCLD_E_UNKNOWN_COMM; ++rej; continue; }
-    const u32 pos = pos_lookup(R, rk, c);
-    if (pos == NONE) { err |= CCLD_E_NOT_MEMBER; ++rej; continue; }
-    if (s < R.comm_seq0[c]) { err |= CCLD_E_SEQ_RANGE; ++rej; continue; }
-    const RangeRow r = D.ranges[c];
-    if (r.n_seq == 0) continue;                          // window refused by the plan
-    const u64 slot = r.slot0 + (u64)(s - r.seq_lo) * r.n + pos;
-    if (s < r.seq_lo || slot >= D.n_slots) { internal = 1; continue; }
-    D.perm[slot] = (u32)i;
+  for (int h = 0; h < 2; ++h) {
+    u32 rk[HALF], cid[HALF], sq[HALF]; bool in[HALF];
+#pragma unroll
+    for (int k = 0; k < HALF; ++k) {
+      const u64 i = base + (u64)(h * HALF + k) * REC_THREADS + threadIdx.x;
+      in[k] = i < D.n_rec;
+      rk[k] = in[k] ? D.rank[i] : 0u; cid[k] = in[k] ? D.comm[i] : 0u; sq[k] = in[k] ? D.seq[i] : 0u;
+    }
+    uint4 ta[HALF], tb[HALF];
+#pragma unroll
+    for (int k = 0; k < HALF; ++k) {
+      const u32 r = rk[k] < R.n_ranks ? rk[k] : 0u;
+      ta[k] = R.rank_tab[(u64)r * 2]; tb[k] = R.rank_tab[(u64)r * 2 + 1];
+    }
+    u32 cp[HALF];                              // index << 13 | position, NONE if the record is rejected
+#pragma unroll
+    for (int k = 0; k < HALF; ++k) {
+      u32 v = NONE;
+      if (rk[k] < R.n_ranks) {
+        v = ta[k].x == cid[k] ? ta[k].y : v; v = ta[k].z == cid[k] ? ta[k].w : v;
+        v = tb[k].x == cid[k] ? tb[k].y : v; v = tb[k].z == cid[k] ? tb[k].w : v;
+      }
+      if (in[k] && (v == NONE || cid[k] == NONE)) {
+        const u64 rs = resolve_slow(R, rk[k], cid[k]);
+        v = (u32)rs;
+        if (rs >> 32) { err |= (u32)(rs >> 32); ++rej; }
+      }
+      cp[k] = in[k] ? v : NONE;
+    }
+    uint4 sr[HALF];
+#pragma unroll
+    for (int k = 0; k < HALF; ++k) sr[k] = cp[k] != NONE ? D.srow[cp[k] >> RANK_TAB_POS_BITS] : make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int k = 0; k < HALF; ++k) {
+      if (cp[k] != NONE) {
+        const u32 n = sr[k].z, lo = sr[k].w;
+        if (n == 0 || sq[k] < lo) {
+          if (sq[k] < R.comm_seq0[cp[k] >> RANK_TAB_POS_BITS]) { err |= CCLD_E_SEQ_RANGE; ++rej; }
+          else if (n != 0) internal = 1;
+        } else {
+          const u64 sb = (u64)sr[k].x | ((u64)sr[k].y << 32);
+          const u64 slot = sb + (u64)sq[k] * n + (cp[k] & ((1u << RANK_TAB_POS_BITS) - 1));
+          if (slot >= D.n_slots) internal = 1;
+          else D.perm[slot] = (u32)(base + (u64)(h * HALF + k) * REC_THREADS + threadIdx.x);
+        }
+      }
+    }
   }
   err = __reduce_or_sync(0xFFFFFFFFu, err);
   rej = __reduce_add_sync(0xFFFFFFFFu, rej);
