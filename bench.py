@@ -227,8 +227,7 @@ def run_ours(args, rank, world, local_rank):
     alg = {   # algorithmic bytes one launch moves (per window: records, groups of the class)
         "k_seq_range": lambda: NW * 8 * sum(u[0] for u in units.values()),
         "k_slot_scatter": lambda: NW * (12 + 4) * sum(u[0] for u in units.values()),
-        "k_reduce_small": lambda: NW * ((4 + 33 + 1) * units["small"][0] + ROW_BYTES * units["small"][1]),
-        "k_reduce_warp": lambda: NW * ((4 + 33 + 1) * units["warp"][0] + ROW_BYTES * units["warp"][1]),
+        "k_reduce_fused": lambda: NW * ((4 + 33 + 1) * (units["small"][0] + units["warp"][0]) + ROW_BYTES * (units["small"][1] + units["warp"][1])),
         "k_reduce_mid": lambda: NW * ((4 + 33 + 1) * units["mid"][0] + ROW_BYTES * units["mid"][1]),
         "k_reduce_large": lambda: NW * ((4 + 33 + 1) * units["large"][0] + ROW_BYTES * units["large"][1]),
     }

@@ -271,12 +271,11 @@ int ccld_get_rank_stats(ccld_ctx* ctx, uint32_t n_ranks, uint32_t* votes, uint32
  * Per-kernel device timing for benchmarks. While enabled, ccld_analyze_window brackets each of its
  * kernel launches with CUDA events on the context's stream. ccld_get_kernel_times synchronizes the
  * stream and returns, per kernel kind, the summed device time in milliseconds and the number of
- * launches since timing was last enabled. Kinds: 0 op-counter range, 1 slot layout and tile list
- * (two launches per call), 2 slot scatter, 3 reductions n <= 8, 4 reductions n <= 128, 5 reductions
- * n <= 1024, 6 reductions n > 1024, 7 window decision. Enabling (on = 1) clears the sums; on = 0
- * stops timing.
+ * launches since timing was last enabled. Kinds: 0 op-counter range, 1 slot layout and work lists
+ * (two launches per call), 2 slot scatter, 3 reductions n <= 128 (fused), 4 reductions n <= 1024,
+ * 5 reductions n > 1024, 6 window decision. Enabling (on = 1) clears the sums; on = 0 stops timing.
  */
-#define CCLD_K_KINDS 8
+#define CCLD_K_KINDS 7
 int ccld_timing_enable(ccld_ctx* ctx, int on);
 int ccld_get_kernel_times(ccld_ctx* ctx, double* ms /* host [CCLD_K_KINDS] */, uint64_t* launches /* host [CCLD_K_KINDS] */);
 

@@ -27,8 +27,7 @@ EXPORTS = ("ccld_params_default", "ccld_create", "ccld_destroy", "ccld_last_erro
            "ccld_locate_hang", "ccld_get_optable", "ccld_get_ranges", "ccld_get_rank_stats", "ccld_copy_to_host",
            "ccld_timing_enable", "ccld_get_kernel_times", "ccld_ring_locate_static")
 STATIC_MAX_MEMBERS = 8192
-KERNEL_KINDS = ("k_seq_range", "k_plan", "k_slot_scatter", "k_reduce_small", "k_reduce_warp", "k_reduce_mid", "k_reduce_large",
-                "k_window_decide")
+KERNEL_KINDS = ("k_seq_range", "k_plan", "k_slot_scatter", "k_reduce_fused", "k_reduce_mid", "k_reduce_large", "k_window_decide")
 
 
 class CcldError(RuntimeError):

@@ -21,7 +21,7 @@ constexpr int REC_THREADS = 256;       // record-streaming kernels: threads per 
 constexpr int REC_PER_THREAD = 8;
 constexpr int REC_PER_CTA = REC_THREADS * REC_PER_THREAD;
 constexpr int SMALL_N = 8;             // communicators of up to 8 ranks: one thread per group
-constexpr int SMALL_SEQS = 256;        //   seqs (= threads) per tile
+constexpr int SMALL_SEQS = 256;        //   threads per CTA: eight warp-tiles of up to 32 op counters
 constexpr int WARP_N = 128;            // up to 128 ranks: one warp per group, bitonic sort in registers
 constexpr int MID_N = 1024;            // up to 1024 ranks: shared-memory bitonic sort, several groups per CTA
 constexpr int MID_THREADS = 256;
@@ -66,14 +66,23 @@ constexpr u32 RANK_TAB_OVERFLOW = 0xFFFFFFFEu;
 constexpr u32 RANK_TAB_POS_BITS = 13;  // positions < CCLD_MAX_COMM_SIZE = 8192
 
 // Which op counters a communicator covers in a window and where its groups / slots start.
-struct RangeRow { u32 seq_lo, n_seq, row_idx, n; u64 group0, slot0; u32 tile0, pad; };   // tile0: first tile in its class list
+// tile0 / n_units: where the communicator's TileSum entries start (index into its summary array) and how many it has.
+struct RangeRow { u32 seq_lo, n_seq, row_idx, n; u64 group0, slot0; u32 tile0, n_units; };
 
 enum { C_REJECTED = 0, C_COMPLETE, C_INCOMPLETE, C_BARRIER, C_ANALYSED, C_FLAG_SKEW, C_FLAG_DUR, C_MISMATCH,
        C_PRESENT, C_ALERTS, C_ERR, C_INTERNAL, C_COUNT = 16 };
-constexpr int N_CLASSES = 4;           // reduction kernels: n <= 8, <= 128, <= 1024, larger
-enum { T_GROUPS = 0, T_SLOTS, T_TILES0, T_TILES1, T_TILES2, T_TILES3, T_ROWS, T_FAILED, T_COUNT = 8 };
+constexpr int N_CLASSES = 4;           // reduction code paths: n <= 8, <= 128, <= 1024, larger
+// Classes 0 and 1 run in one fused kernel whose work list is ordered by (window, time chunk): a window's op
+// counters are cut into T chunks per communicator, so that the tiles of one chunk - which gather from the same
+// stretch of every rank's records - run together and share the fetched sectors in L2.
+constexpr u32 CHUNK_REF = 96;          // op counters per chunk of the busiest communicator of a window
+constexpr u32 CHUNK_MAX = 64;          // at most this many chunks per window (longer chunks beyond)
+enum { T_GROUPS = 0, T_SLOTS, T_FCTA, T_FWT, T_FSUM, T_TILES2, T_TILES3, T_ROWS, T_FAILED, T_CHUNKS, T_COUNT = 12 };
+enum { B_FCTA = 0, B_FWT, B_FSUM, B_T2, B_T3, B_COUNT };
 
-struct Tile { u32 w, c, seq_off, count; };
+struct Tile { u32 w, c, seq_off, count; };                 // classes 2 and 3: one CTA each; summary index = tile index
+struct WarpTile { u32 c, seq_off, count, sum_idx; };      // class 0: up to 32 consecutive op counters of one communicator
+struct FusedCta { u32 w, cls, c, seq_off, count, sum_idx, wt_first, wt_count; };   // class 0: wt_*; class 1: c .. sum_idx
 
 // What a tile contributes to its communicator's window decision (Eq. 2 and the round counts).
 struct TileSum { u64 best_rng; u32 best_k, n_rounds, n_an, pad; };   // best_k: op-counter offset in the range, NONE if no round
@@ -102,8 +111,9 @@ struct WinDesc {
   double* gbw;                       // [n_groups]
   ccld_comm_verdict* comm_rows;      // [n_rows]
   ccld_hang_alert* alerts;           // [CCLD_MAX_ALERTS_PER_WINDOW]
-  u32 tile0[N_CLASSES];              // first tile of this window in each class list
-  TileSum* tsum[N_CLASSES];          // per-class tile summaries of the whole batch
+  u32 base[B_COUNT];                 // this window's first entry in the batch-wide lists (B_*)
+  u32 pad;
+  TileSum* tsum[3];                  // tile summaries of the whole batch: fused classes, class 2, class 3
 };
 
 enum { GI_E_MIN = 0, GI_ARRIVAL_SKEW, GI_T_MAX, GI_T_MIN, GI_SPAN, GI_MED_SKEW, GI_MAD_SKEW, GI_MED_DUR, GI_MAD_DUR, GI_COUNT };
@@ -112,9 +122,18 @@ enum { GU_RANK_TMIN = 0, GU_RANK_TMAX, GU_MAX_CHG, GU_RANK_MAX_CHG, GU_N_PRESENT
 __host__ __device__ inline u32 next_pow2(u32 n) { u32 p = 1; while (p < n) p <<= 1; return p; }
 __host__ __device__ inline u32 comm_class(u32 n) { return n <= SMALL_N ? 0u : (n <= WARP_N ? 1u : (n <= MID_N ? 2u : 3u)); }
 __host__ __device__ inline u32 mid_npad(u32 n) { u32 p = next_pow2(n); return p < 32 ? 32 : p; }
+// op counters per work unit: a warp-tile (class 0) or a CTA tile (classes 1 to 3)
 __host__ __device__ inline u32 tile_seqs(u32 n) {
   u32 c = comm_class(n);
-  return c == 0 ? SMALL_SEQS : (c <= 2 ? MID_ELEMS / mid_npad(n) : (u32)LARGE_SEQS);
+  return c == 0 ? 32u : (c <= 2 ? MID_ELEMS / mid_npad(n) : (u32)LARGE_SEQS);
+}
+__host__ __device__ inline u32 ceil_div(u32 a, u32 b) { return (a + b - 1) / b; }
+// chunking of a fused-class communicator with n_seq op counters in a window of T chunks
+__host__ __device__ inline u32 chunk_len(u32 n_seq, u32 T) { return ceil_div(n_seq, T); }
+__host__ __device__ inline u32 chunk_count(u32 n_seq, u32 T) { return n_seq ? ceil_div(n_seq, chunk_len(n_seq, T)) : 0u; }
+__host__ __device__ inline u32 chunk_size(u32 n_seq, u32 T, u32 tau) {    // op counters in chunk tau (0 beyond the last)
+  const u32 S = chunk_len(n_seq, T);
+  return (u64)tau * S >= n_seq ? 0u : (n_seq - tau * S < S ? n_seq - tau * S : S);
 }
 
 }  // namespace ccld

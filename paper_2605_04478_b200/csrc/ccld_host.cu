@@ -221,7 +221,7 @@ int finalize_registry(ccld_ctx* ctx) {
   ctx->misc_blk = ctx->pool.get(misc_layout(nr, max_n).total, &e);
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "scratch allocation failed");
 
-  CK(cudaFuncSetAttribute(k_reduce_warp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)warp_smem_bytes()));
+  CK(cudaFuncSetAttribute(k_reduce_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)warp_smem_bytes()));
   CK(cudaFuncSetAttribute(k_reduce_mid, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mid_smem_bytes(2 * WARP_N)));
   if (max_large) CK(cudaFuncSetAttribute(k_reduce_large, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(16ull * max_large)));
   ctx->finalized = true;
@@ -410,7 +410,8 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
     d.totals = (u64*)(pbase + o_tot) + (size_t)k * T_COUNT; d.counters = (u64*)(pbase + o_cnt) + (size_t)k * C_COUNT;
     d.n_groups = d.n_slots = 0; d.perm = nullptr; d.flags = nullptr; d.gi64 = nullptr; d.gu32 = nullptr; d.gbw = nullptr;
     d.comm_rows = nullptr; d.alerts = nullptr;
-    for (int q = 0; q < N_CLASSES; ++q) { d.tile0[q] = 0; d.tsum[q] = nullptr; }
+    for (int q = 0; q < B_COUNT; ++q) d.base[q] = 0;
+    d.pad = 0; d.tsum[0] = d.tsum[1] = d.tsum[2] = nullptr;
     hd[k] = d;
   }
   if (cta > 0x7FFFFFFFull) return fail(ctx, CCLD_ERR_CAPACITY, "batch too large for one launch");
@@ -420,7 +421,7 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   CK(cudaMemcpyAsync(d_desc, hd.data(), B * sizeof(WinDesc), cudaMemcpyHostToDevice, st));
   TimerSlot* ts = timer_begin(ctx);
   if (cta > 0) { TimedLaunch tl(ts, 0, st); k_seq_range<<<(u32)cta, REC_THREADS, 0, st>>>(d_desc, B, ctx->reg); }
-  { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, TileLists{{nullptr, nullptr, nullptr, nullptr}}, 0); }
+  { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, PlanLists{nullptr, nullptr, nullptr, nullptr}, 0); }
   CK(cudaGetLastError());
   { int rc = ensure_pinned(ctx, (size_t)B * T_COUNT * 8); if (rc != CCLD_OK) return rc; }
   CK(cudaMemcpyAsync(ctx->h_pinned, pbase + o_tot, (size_t)B * T_COUNT * 8, cudaMemcpyDeviceToHost, st));
@@ -428,7 +429,8 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
 
   // ---- result block: sized from the plan ----
   off = 0;
-  u64 total_slots = 0, n_tiles[N_CLASSES] = {0, 0, 0, 0};
+  u64 total_slots = 0, n_list[B_COUNT] = {0, 0, 0, 0, 0};       // batch-wide list lengths (B_*)
+  const int t_of[B_COUNT] = {T_FCTA, T_FWT, T_FSUM, T_TILES2, T_TILES3};
   for (u32 k = 0; k < B; ++k) { const u64* t = ctx->h_pinned + (size_t)k * T_COUNT; total_slots += t[T_SLOTS]; }
   const size_t o_perm = take(total_slots * 4 + ALIGN);
   std::vector<size_t> o_flags(B), o_gi(B), o_gu(B), o_gb(B), o_rows(B), o_al(B), perm_off(B);
@@ -439,13 +441,12 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
       o_flags[k] = take(t[T_SLOTS]); o_gi[k] = take(t[T_GROUPS] * 8 * GI_COUNT); o_gu[k] = take(t[T_GROUPS] * 4 * GU_COUNT);
       o_gb[k] = take(t[T_GROUPS] * 8); o_rows[k] = take(t[T_ROWS] * sizeof(ccld_comm_verdict));
       o_al[k] = take(CCLD_MAX_ALERTS_PER_WINDOW * sizeof(ccld_hang_alert));
-      for (int q = 0; q < N_CLASSES; ++q) { hd[k].tile0[q] = (u32)n_tiles[q]; n_tiles[q] += t[T_TILES0 + q]; }
+      for (int q = 0; q < B_COUNT; ++q) { hd[k].base[q] = (u32)n_list[q]; n_list[q] += t[t_of[q]]; }
     } }
-  size_t o_tl[N_CLASSES], o_ts[N_CLASSES];
-  for (int q = 0; q < N_CLASSES; ++q) {
-    if (n_tiles[q] > 0x7FFFFFFFull) return fail(ctx, CCLD_ERR_CAPACITY, "too many tiles in one batch");
-    o_tl[q] = take(n_tiles[q] * sizeof(Tile)); o_ts[q] = take(n_tiles[q] * sizeof(TileSum));
-  }
+  for (int q = 0; q < B_COUNT; ++q) if (n_list[q] > 0x7FFFFFFFull) return fail(ctx, CCLD_ERR_CAPACITY, "too many tiles in one batch");
+  const size_t o_fcta = take(n_list[B_FCTA] * sizeof(FusedCta)), o_fwt = take(n_list[B_FWT] * sizeof(WarpTile)),
+               o_fsum = take(n_list[B_FSUM] * sizeof(TileSum)), o_t2 = take(n_list[B_T2] * sizeof(Tile)), o_s2 = take(n_list[B_T2] * sizeof(TileSum)),
+               o_t3 = take(n_list[B_T3] * sizeof(Tile)), o_s3 = take(n_list[B_T3] * sizeof(TileSum));
   Block rb = ctx->pool.get(off, &e);
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "result allocation failed");
   auto res_blk = std::make_shared<Shared>(&ctx->pool, rb);
@@ -457,19 +458,17 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
     d.perm = (u32*)(rbase + o_perm + perm_off[k]); d.flags = (u8*)(rbase + o_flags[k]);
     d.gi64 = (i64*)(rbase + o_gi[k]); d.gu32 = (u32*)(rbase + o_gu[k]); d.gbw = (double*)(rbase + o_gb[k]);
     d.comm_rows = (ccld_comm_verdict*)(rbase + o_rows[k]); d.alerts = (ccld_hang_alert*)(rbase + o_al[k]);
-    for (int q = 0; q < N_CLASSES; ++q) d.tsum[q] = (TileSum*)(rbase + o_ts[q]);
+    d.tsum[0] = (TileSum*)(rbase + o_fsum); d.tsum[1] = (TileSum*)(rbase + o_s2); d.tsum[2] = (TileSum*)(rbase + o_s3);
   }
   CK(cudaMemcpyAsync(d_desc, hd.data(), B * sizeof(WinDesc), cudaMemcpyHostToDevice, st));
   if (total_slots) CK(cudaMemsetAsync(rbase + o_perm, 0xFF, total_slots * 4, st));
-  TileLists tl_all; TileSum* tsum[N_CLASSES];
-  for (int q = 0; q < N_CLASSES; ++q) { tl_all.t[q] = (Tile*)(rbase + o_tl[q]); tsum[q] = (TileSum*)(rbase + o_ts[q]); }
-  { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, tl_all, 1); }
+  PlanLists pl; pl.fcta = (FusedCta*)(rbase + o_fcta); pl.fwt = (WarpTile*)(rbase + o_fwt); pl.t2 = (Tile*)(rbase + o_t2); pl.t3 = (Tile*)(rbase + o_t3);
+  { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, pl, 1); }
   if (cta > 0) { TimedLaunch tl(ts, 2, st); k_slot_scatter<<<(u32)cta, REC_THREADS, 0, st>>>(d_desc, B, ctx->reg); }
-  if (n_tiles[0]) { TimedLaunch tl(ts, 3, st); k_reduce_small<<<(u32)n_tiles[0], SMALL_SEQS, 0, st>>>(d_desc, tl_all.t[0], tsum[0], ctx->reg, ctx->dp, now_ns); }
-  if (n_tiles[1]) { TimedLaunch tl(ts, 4, st); k_reduce_warp<<<(u32)n_tiles[1], MID_THREADS, warp_smem_bytes(), st>>>(d_desc, tl_all.t[1], tsum[1], ctx->reg, ctx->dp, now_ns); }
-  if (n_tiles[2]) { TimedLaunch tl(ts, 5, st); k_reduce_mid<<<(u32)n_tiles[2], MID_THREADS, mid_smem_bytes(2 * WARP_N), st>>>(d_desc, tl_all.t[2], tsum[2], ctx->reg, ctx->dp, now_ns); }
-  if (n_tiles[3]) { TimedLaunch tl(ts, 6, st); k_reduce_large<<<(u32)n_tiles[3], LARGE_THREADS, 16ull * ctx->max_large_n, st>>>(d_desc, tl_all.t[3], tsum[3], ctx->reg, ctx->dp, now_ns); }
-  { TimedLaunch tl(ts, 7, st); k_window_decide<<<(nc + 3) / 4, 128, 0, st>>>(d_desc, B, ctx->reg, ctx->dp); }
+  if (n_list[B_FCTA]) { TimedLaunch tl(ts, 3, st); k_reduce_fused<<<(u32)n_list[B_FCTA], SMALL_SEQS, warp_smem_bytes(), st>>>(d_desc, pl.fcta, pl.fwt, (TileSum*)(rbase + o_fsum), ctx->reg, ctx->dp, now_ns); }
+  if (n_list[B_T2]) { TimedLaunch tl(ts, 4, st); k_reduce_mid<<<(u32)n_list[B_T2], MID_THREADS, mid_smem_bytes(2 * WARP_N), st>>>(d_desc, pl.t2, (TileSum*)(rbase + o_s2), ctx->reg, ctx->dp, now_ns); }
+  if (n_list[B_T3]) { TimedLaunch tl(ts, 5, st); k_reduce_large<<<(u32)n_list[B_T3], LARGE_THREADS, 16ull * ctx->max_large_n, st>>>(d_desc, pl.t3, (TileSum*)(rbase + o_s3), ctx->reg, ctx->dp, now_ns); }
+  { TimedLaunch tl(ts, 6, st); k_window_decide<<<(nc + 3) / 4, 128, 0, st>>>(d_desc, B, ctx->reg, ctx->dp); }
   CK(cudaGetLastError());
   for (u32 k = 0; k < B; ++k) {
     WindowHost& w = *ws[k];

@@ -5,8 +5,8 @@
 //   k_plan          group-by, part 2: closed-form slot layout (prefix sums over communicators),
 //                   and the work list for the reduction kernels
 //   k_slot_scatter  group-by, part 3: perm[slot] = record index
-//   k_reduce_small  per-op reductions + median/MAD + flags + votes, n <= 8 (thread per group)
-//   k_reduce_warp   same, 9 <= n <= 128 (warp per group, bitonic sort in registers)
+//   k_reduce_fused  per-op reductions + median/MAD + flags + votes for n <= 128, chunk-major work list:
+//                   n <= 8 one thread per group (warp-tiles), 9 <= n <= 128 one warp per group (register bitonic sort)
 //   k_reduce_mid    same, 129 <= n <= 1024 (shared-memory bitonic sort, several groups per CTA)
 //   k_reduce_large  same, n > 1024 (one CTA per group, radix select)
 //   k_window_decide Eq. 1-4 per communicator and window, slow location
@@ -162,37 +162,40 @@ __global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __rest
 }
 
 // ------------------------------------------------------------------------------------------------
-// group-by, part 2: closed-form layout. One CTA per window scans the communicators.
+// group-by, part 2: closed-form layout and work lists. One CTA per window scans the communicators.
 //   slot(comm, seq, pos) = slot0[comm] + (seq - seq_lo[comm]) * n[comm] + pos
 // ------------------------------------------------------------------------------------------------
-struct PlanAcc { u64 groups, slots; u32 rows, t[N_CLASSES]; };
+struct PlanAcc { u64 groups, slots; u32 rows, t2, t3, pad; };
 
 __device__ __forceinline__ PlanAcc plan_add(const PlanAcc& a, const PlanAcc& b) {
   PlanAcc r; r.groups = a.groups + b.groups; r.slots = a.slots + b.slots; r.rows = a.rows + b.rows;
-#pragma unroll
-  for (int q = 0; q < N_CLASSES; ++q) r.t[q] = a.t[q] + b.t[q];
-  return r;
+  r.t2 = a.t2 + b.t2; r.t3 = a.t3 + b.t3; r.pad = 0; return r;
 }
 __device__ __forceinline__ PlanAcc plan_shfl_up(const PlanAcc& a, int d) {
   PlanAcc r;
   r.groups = __shfl_up_sync(0xFFFFFFFFu, a.groups, d); r.slots = __shfl_up_sync(0xFFFFFFFFu, a.slots, d);
-  r.rows = __shfl_up_sync(0xFFFFFFFFu, a.rows, d);
-#pragma unroll
-  for (int q = 0; q < N_CLASSES; ++q) r.t[q] = __shfl_up_sync(0xFFFFFFFFu, a.t[q], d);
+  r.rows = __shfl_up_sync(0xFFFFFFFFu, a.rows, d); r.t2 = __shfl_up_sync(0xFFFFFFFFu, a.t2, d);
+  r.t3 = __shfl_up_sync(0xFFFFFFFFu, a.t3, d); r.pad = 0;
   return r;
 }
 
+// op counters communicator c covers in the window (0 if none; clamped to 2^32 - 1)
+__device__ __forceinline__ u32 plan_nseq(const WinDesc& D, const Registry& R, u32 c) {
+  if (c >= R.n_comms) return 0;
+  const u32 lo = D.rmin[c], hi = D.rmax[c];
+  if (!(lo <= hi && lo != NONE)) return 0;
+  const u64 ns = (u64)hi - lo + 1;
+  return ns > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)ns;
+}
+
 __device__ __forceinline__ PlanAcc plan_item(const WinDesc& D, const Registry& R, u32 c) {
-  PlanAcc a = {0, 0, 0, {0, 0, 0, 0}};
-  if (c < R.n_comms) {
-    u32 lo = D.rmin[c], hi = D.rmax[c];
-    if (lo <= hi && lo != NONE) {
-      u64 ns = (u64)hi - lo + 1; u32 n = R.comm_n[c];
-      a.groups = ns; a.slots = ns * n; a.rows = 1;
-      u64 tiles = (ns + tile_seqs(n) - 1) / tile_seqs(n);
-      u32 t = tiles > 0x7FFFFFFFull ? 0x7FFFFFFFu : (u32)tiles;
-      a.t[comm_class(n)] = t;
-    }
+  PlanAcc a = {0, 0, 0, 0, 0, 0};
+  const u32 ns = plan_nseq(D, R, c);
+  if (ns) {
+    const u32 n = R.comm_n[c], cls = comm_class(n);
+    a.groups = ns; a.slots = (u64)ns * n; a.rows = 1;
+    const u32 t = ceil_div(ns, tile_seqs(n));
+    a.t2 = cls == 2 ? t : 0; a.t3 = cls == 3 ? t : 0;
   }
   return a;
 }
@@ -211,68 +214,200 @@ __device__ PlanAcc plan_block_scan(PlanAcc v, PlanAcc* total, PlanAcc* s_warp /*
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) { PlanAcc o = plan_shfl_up(xi, d); if (lane >= (u32)d) xi = plan_add(xi, o); }
     PlanAcc ex = plan_shfl_up(xi, 1);
-    if (lane == 0) ex = PlanAcc{0, 0, 0, {0, 0, 0, 0}};
+    if (lane == 0) ex = PlanAcc{0, 0, 0, 0, 0, 0};
     s_warp[lane] = ex;
     if (lane == 31) s_warp[32] = xi;
   }
   __syncthreads();
   PlanAcc ex = plan_shfl_up(inc, 1);
-  if (lane == 0) ex = PlanAcc{0, 0, 0, {0, 0, 0, 0}};
+  if (lane == 0) ex = PlanAcc{0, 0, 0, 0, 0, 0};
   PlanAcc r = plan_add(s_warp[wid], ex);
   *total = s_warp[32];
   __syncthreads();
   return r;
 }
 
-// emit == 0: write ranges and totals (and fail the window if it needs more than slot_cap slots).
-// emit == 1: write the tile lists (tile0[] filled by the host from the totals).
-struct TileLists { Tile* t[N_CLASSES]; };
-__global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd, Registry R, TileLists lists, int emit) {
+// The same for a pair of 32-bit counters.
+__device__ uint2 plan_scan2(uint2 v, uint2* total, uint2* s_pair /*[33]*/) {
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  uint2 inc = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    const u32 ox = __shfl_up_sync(0xFFFFFFFFu, inc.x, d), oy = __shfl_up_sync(0xFFFFFFFFu, inc.y, d);
+    if (lane >= (u32)d) { inc.x += ox; inc.y += oy; }
+  }
+  if (lane == 31) s_pair[wid] = inc;
+  __syncthreads();
+  if (wid == 0) {
+    const uint2 x = s_pair[lane]; uint2 xi = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      const u32 ox = __shfl_up_sync(0xFFFFFFFFu, xi.x, d), oy = __shfl_up_sync(0xFFFFFFFFu, xi.y, d);
+      if (lane >= (u32)d) { xi.x += ox; xi.y += oy; }
+    }
+    s_pair[lane] = make_uint2(xi.x - x.x, xi.y - x.y);
+    if (lane == 31) s_pair[32] = xi;
+  }
+  __syncthreads();
+  const uint2 r = make_uint2(s_pair[wid].x + inc.x - v.x, s_pair[wid].y + inc.y - v.y);
+  *total = s_pair[32];
+  __syncthreads();
+  return r;
+}
+
+// Work units (warp-tiles of class 0, CTA tiles of class 1) of communicator c in chunk tau; 0 for other classes.
+__device__ __forceinline__ u32 chunk_units(u32 ns, u32 n, u32 T, u32 tau) {
+  if (ns == 0 || comm_class(n) > 1) return 0;
+  return ceil_div(chunk_size(ns, T, tau), tile_seqs(n));
+}
+// All units of communicator c in the window (its TileSum entries): full chunks plus the last one.
+__device__ __forceinline__ u32 comm_units(u32 ns, u32 n, u32 T) {
+  if (ns == 0 || comm_class(n) > 1) return 0;
+  const u32 S = chunk_len(ns, T), nch = ceil_div(ns, S), U = tile_seqs(n);
+  return (nch - 1) * ceil_div(S, U) + ceil_div(ns - (nch - 1) * S, U);
+}
+
+struct PlanLists { FusedCta* fcta; WarpTile* fwt; Tile* t2; Tile* t3; };
+
+// emit == 0: ranges, scatter rows and totals (the window is refused if it needs more than slot_cap slots).
+// emit == 1: the work lists (base[] filled by the host from the totals).
+__global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd, Registry R, PlanLists L, int emit) {
   __shared__ PlanAcc s_warp[33];
+  __shared__ uint2 s_pair[33];
+  __shared__ u32 s_red[32];
   __shared__ int s_failed;
   WinDesc& D = wd[blockIdx.x];
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   if (emit && D.totals[T_FAILED]) return;
-  PlanAcc run = {0, 0, 0, {0, 0, 0, 0}};
-  for (u32 c0 = 0; c0 < R.n_comms; c0 += PLAN_THREADS) {
-    const u32 c = c0 + threadIdx.x;
-    PlanAcc it = plan_item(D, R, c), tot;
-    PlanAcc ex = plan_add(run, plan_block_scan(it, &tot, s_warp));
-    if (c < R.n_comms) {
-      if (!emit) {
+
+  if (!emit) {
+    // 1. layout: groups, slots, rows; tiles of the two big classes; busiest fused-class communicator
+    PlanAcc run = {0, 0, 0, 0, 0, 0};
+    u32 mx = 0;
+    for (u32 c0 = 0; c0 < R.n_comms; c0 += PLAN_THREADS) {
+      const u32 c = c0 + threadIdx.x;
+      PlanAcc it = plan_item(D, R, c), tot;
+      PlanAcc ex = plan_add(run, plan_block_scan(it, &tot, s_warp));
+      if (c < R.n_comms) {
         RangeRow r;
         r.seq_lo = it.rows ? D.rmin[c] : 0; r.n_seq = (u32)it.groups; r.row_idx = ex.rows; r.n = R.comm_n[c];
-        r.group0 = ex.groups; r.slot0 = ex.slots; r.tile0 = 0; r.pad = 0;
+        r.group0 = ex.groups; r.slot0 = ex.slots; r.tile0 = 0; r.n_units = 0;
         D.ranges[c] = r;
         const u64 sb = r.slot0 - (u64)r.seq_lo * r.n;
         D.srow[c] = make_uint4((u32)sb, (u32)(sb >> 32), it.rows ? r.n : 0u, r.seq_lo);
-      } else if (it.rows) {
+        if (it.rows && comm_class(r.n) <= 1) mx = r.n_seq > mx ? r.n_seq : mx;
+      }
+      run = plan_add(run, tot);
+    }
+    mx = __reduce_max_sync(0xFFFFFFFFu, mx);
+    if (lane == 0) s_red[wid] = mx;
+    __syncthreads();
+    mx = 0;
+    for (int q = 0; q < PLAN_THREADS / 32; ++q) mx = s_red[q] > mx ? s_red[q] : mx;
+    u32 T = mx ? ceil_div(mx, CHUNK_REF) : 1u;
+    T = T > CHUNK_MAX ? CHUNK_MAX : T;
+    __syncthreads();
+    // 2. summary entries of the fused classes
+    u32 urun = 0;
+    for (u32 c0 = 0; c0 < R.n_comms; c0 += PLAN_THREADS) {
+      const u32 c = c0 + threadIdx.x;
+      const u32 ns = plan_nseq(D, R, c), n = c < R.n_comms ? R.comm_n[c] : 1u;
+      const u32 u = comm_units(ns, n, T);
+      uint2 tot; const uint2 ex = plan_scan2(make_uint2(u, 0), &tot, s_pair);
+      if (c < R.n_comms && u) { D.ranges[c].tile0 = urun + ex.x; D.ranges[c].n_units = u; }
+      urun += tot.x;
+    }
+    // 3. CTAs and warp-tiles of the fused kernel, chunk by chunk
+    u64 n_cta = 0, n_wt = 0;
+    for (u32 tau = 0; tau < T; ++tau) {
+      u32 wt = 0, c1 = 0;
+      for (u32 c = threadIdx.x; c < R.n_comms; c += PLAN_THREADS) {
+        const u32 n = R.comm_n[c], u = chunk_units(plan_nseq(D, R, c), n, T, tau);
+        if (comm_class(n) == 0) wt += u; else c1 += u;
+      }
+      uint2 tot; plan_scan2(make_uint2(wt, c1), &tot, s_pair);
+      n_cta += ceil_div(tot.x, 8) + tot.y; n_wt += tot.x;
+    }
+    if (threadIdx.x == 0) {
+      // op counters further apart than 2^31, or more slots than the cap: refuse the window
+      const int failed = run.slots > D.slot_cap || run.groups > 0x7FFFFFFFull || n_cta > 0x7FFFFFFFull || n_wt > 0x7FFFFFFFull;
+      s_failed = failed;
+      D.totals[T_GROUPS] = failed ? 0 : run.groups; D.totals[T_SLOTS] = failed ? 0 : run.slots;
+      D.totals[T_FCTA] = failed ? 0 : n_cta; D.totals[T_FWT] = failed ? 0 : n_wt; D.totals[T_FSUM] = failed ? 0 : urun;
+      D.totals[T_TILES2] = failed ? 0 : run.t2; D.totals[T_TILES3] = failed ? 0 : run.t3;
+      D.totals[T_ROWS] = failed ? 0 : run.rows; D.totals[T_FAILED] = failed; D.totals[T_CHUNKS] = T;
+      if (failed) atomicOr((unsigned*)&D.counters[C_ERR], (unsigned)CCLD_E_CAPACITY);
+    }
+    __syncthreads();
+    if (s_failed)
+      for (u32 c = threadIdx.x; c < R.n_comms; c += PLAN_THREADS) { RangeRow z = {0, 0, 0, R.comm_n[c], 0, 0, 0, 0}; D.ranges[c] = z; D.srow[c] = make_uint4(0, 0, 0, 0); }
+    return;
+  }
+
+  // ---- emit ----
+  const u32 T = (u32)D.totals[T_CHUNKS];
+  // tiles of classes 2 and 3, communicator by communicator; summary indices of every communicator become batch-wide
+  {
+    PlanAcc run = {0, 0, 0, 0, 0, 0};
+    for (u32 c0 = 0; c0 < R.n_comms; c0 += PLAN_THREADS) {
+      const u32 c = c0 + threadIdx.x;
+      PlanAcc it = plan_item(D, R, c), tot;
+      PlanAcc ex = plan_add(run, plan_block_scan(it, &tot, s_warp));
+      if (c < R.n_comms && it.rows) {
         const u32 n = R.comm_n[c], S = tile_seqs(n), cls = comm_class(n);
-        const u32 first = D.tile0[cls] + ex.t[cls];
-        Tile* dst = lists.t[cls] + first;
-        D.ranges[c].tile0 = first;
-        const u32 nt = it.t[cls];
-        for (u32 k = 0; k < nt; ++k) {
-          Tile t; t.w = blockIdx.x; t.c = c; t.seq_off = k * S;
-          u64 left = it.groups - (u64)k * S; t.count = left < S ? (u32)left : S;
-          dst[k] = t;
+        if (cls <= 1) D.ranges[c].tile0 += D.base[B_FSUM];
+        else {
+          const u32 first = cls == 2 ? D.base[B_T2] + ex.t2 : D.base[B_T3] + ex.t3, nt = cls == 2 ? it.t2 : it.t3;
+          Tile* dst = (cls == 2 ? L.t2 : L.t3) + first;
+          D.ranges[c].tile0 = first; D.ranges[c].n_units = nt;
+          for (u32 k = 0; k < nt; ++k) {
+            Tile t; t.w = blockIdx.x; t.c = c; t.seq_off = k * S;
+            const u64 left = it.groups - (u64)k * S; t.count = left < S ? (u32)left : S;
+            dst[k] = t;
+          }
         }
       }
+      run = plan_add(run, tot);
     }
-    run = plan_add(run, tot);
-  }
-  if (emit) return;
-  if (threadIdx.x == 0) {
-    // op counters further apart than 2^31, or more slots than the cap: refuse the window
-    int failed = run.slots > D.slot_cap || run.groups > 0x7FFFFFFFull;
-    s_failed = failed;
-    D.totals[T_GROUPS] = failed ? 0 : run.groups; D.totals[T_SLOTS] = failed ? 0 : run.slots;
-    for (int q = 0; q < N_CLASSES; ++q) D.totals[T_TILES0 + q] = failed ? 0 : run.t[q];
-    D.totals[T_ROWS] = failed ? 0 : run.rows; D.totals[T_FAILED] = failed;
-    if (failed) atomicOr((unsigned*)&D.counters[C_ERR], (unsigned)CCLD_E_CAPACITY);
   }
   __syncthreads();
-  if (s_failed)
-    for (u32 c = threadIdx.x; c < R.n_comms; c += PLAN_THREADS) { RangeRow z = {0, 0, 0, R.comm_n[c], 0, 0, 0, 0}; D.ranges[c] = z; D.srow[c] = make_uint4(0, 0, 0, 0); }
+  // fused classes: chunk-major list of CTAs; a class-0 CTA takes eight consecutive warp-tiles
+  u32 cta_base = D.base[B_FCTA], wt_base = D.base[B_FWT];
+  for (u32 tau = 0; tau < T; ++tau) {
+    u32 wt_run = 0, c1_run = 0;
+    // class-1 CTAs come after the chunk's class-0 CTAs, whose number needs the chunk's warp-tile total first
+    u32 wt_total = 0;
+    {
+      u32 wt = 0;
+      for (u32 c = threadIdx.x; c < R.n_comms; c += PLAN_THREADS) { const u32 n = R.comm_n[c]; if (comm_class(n) == 0) wt += chunk_units(plan_nseq(D, R, c), n, T, tau); }
+      uint2 tot; plan_scan2(make_uint2(wt, 0), &tot, s_pair);
+      wt_total = tot.x;
+    }
+    const u32 n0 = ceil_div(wt_total, 8);
+    for (u32 c0 = 0; c0 < R.n_comms; c0 += PLAN_THREADS) {
+      const u32 c = c0 + threadIdx.x;
+      const u32 ns = plan_nseq(D, R, c), n = c < R.n_comms ? R.comm_n[c] : 1u, cls = comm_class(n);
+      const u32 u = chunk_units(ns, n, T, tau);
+      uint2 tot; const uint2 ex = plan_scan2(make_uint2(cls == 0 ? u : 0, cls == 1 ? u : 0), &tot, s_pair);
+      if (u) {
+        const u32 S = chunk_len(ns, T), U = tile_seqs(n), cnt = chunk_size(ns, T, tau);
+        const u32 sum0 = D.ranges[c].tile0 + tau * ceil_div(S, U);
+        for (u32 k = 0; k < u; ++k) {
+          const u32 off = tau * S + k * U, len = cnt - k * U < U ? cnt - k * U : U;
+          if (cls == 0) { WarpTile x; x.c = c; x.seq_off = off; x.count = len; x.sum_idx = sum0 + k; L.fwt[wt_base + wt_run + ex.x + k] = x; }
+          else { FusedCta x; x.w = blockIdx.x; x.cls = 1; x.c = c; x.seq_off = off; x.count = len; x.sum_idx = sum0 + k; x.wt_first = 0; x.wt_count = 0;
+                 L.fcta[cta_base + n0 + c1_run + ex.y + k] = x; }
+        }
+      }
+      wt_run += tot.x; c1_run += tot.y;
+    }
+    for (u32 j = threadIdx.x; j < n0; j += PLAN_THREADS) {
+      FusedCta x; x.w = blockIdx.x; x.cls = 0; x.c = 0; x.seq_off = 0; x.count = 0; x.sum_idx = 0;
+      x.wt_first = wt_base + 8 * j; x.wt_count = wt_total - 8 * j < 8 ? wt_total - 8 * j : 8;
+      L.fcta[cta_base + j] = x;
+    }
+    cta_base += n0 + c1_run; wt_base += wt_total;
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -465,14 +600,15 @@ __device__ __noinline__ u64 small_group64(const WinDesc& D, const Registry& R, c
 
 enum { SC_COMP = 0, SC_INC, SC_BAR, SC_AN, SC_MIS, SC_BWC, SC_PRES, SC_FS, SC_FD, SC_COUNT };
 
+// One warp-tile: up to 32 consecutive op counters of one communicator, one lane per group.
 template <bool FULL>
-__device__ __forceinline__ void reduce_small_tile(const WinDesc& D, const Tile& t, TileSum* __restrict__ sums, const Registry& R, const Params& P,
-                                                  i64 now, u32 n_rt, double (*s_bw)[SMALL_N], u64* s_brng, u32* s_bk, u32* s_cnt) {
+__device__ __forceinline__ void reduce_small_warp(const WinDesc& D, const WarpTile& t, TileSum* __restrict__ sums, const Registry& R, const Params& P,
+                                                  i64 now, u32 n_rt, double (*s_bw)[SMALL_N], u32* s_rounds, u32* s_cnt) {
   const u32 n = FULL ? (u32)SMALL_N : n_rt;
   const u32 c = t.c;
   const RangeRow row = D.ranges[c];
   const u32* mem = R.members + R.comm_moff[c];
-  const u32 j = threadIdx.x, lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5, j = lane;
   const bool active = j < t.count;
   const u32 k_milli = P.k_milli;
 
@@ -627,64 +763,67 @@ __device__ __forceinline__ void reduce_small_tile(const WinDesc& D, const Tile& 
     }
   }
 
-  // ---- per-tile accumulation: counters, Eq. 2 candidate and the per-rank bandwidth sums ----
+  // ---- per-warp accumulation: counters (CTA shared memory), Eq. 2 candidate, per-rank bandwidth sums ----
   const bool is_round = active && complete && !barrier;
-  {
-    const u32 b_comp = __ballot_sync(0xFFFFFFFFu, active && complete), b_inc = __ballot_sync(0xFFFFFFFFu, active && !complete);
-    const u32 b_bar = __ballot_sync(0xFFFFFFFFu, active && barrier), b_an = __ballot_sync(0xFFFFFFFFu, active && analysed);
-    const u32 b_mis = __ballot_sync(0xFFFFFFFFu, active && mismatch), b_bwc = __ballot_sync(0xFFFFFFFFu, is_round);
-    const u32 pres = __reduce_add_sync(0xFFFFFFFFu, n_present), fs = __reduce_add_sync(0xFFFFFFFFu, n_fs), fd = __reduce_add_sync(0xFFFFFFFFu, n_fd);
-    u64 brng = is_round ? my_rng : 0; u32 bk = is_round ? t.seq_off + j : NONE;
-    best_warp_reduce(brng, bk);
-    const double tot = warp_sum8(bw, lane);
-    if ((lane & 3) == 0) s_bw[wid][lane >> 2] = tot;
-    if (lane == 0) {
-      s_brng[wid] = brng; s_bk[wid] = bk;
-      if (b_comp) atomicAdd(&s_cnt[SC_COMP], (u32)__popc(b_comp));
-      if (b_inc) atomicAdd(&s_cnt[SC_INC], (u32)__popc(b_inc));
-      if (b_bar) atomicAdd(&s_cnt[SC_BAR], (u32)__popc(b_bar));
-      if (b_an) atomicAdd(&s_cnt[SC_AN], (u32)__popc(b_an));
-      if (b_mis) atomicAdd(&s_cnt[SC_MIS], (u32)__popc(b_mis));
-      if (b_bwc) atomicAdd(&s_cnt[SC_BWC], (u32)__popc(b_bwc));
-      if (pres) atomicAdd(&s_cnt[SC_PRES], pres);
-      if (fs) atomicAdd(&s_cnt[SC_FS], fs);
-      if (fd) atomicAdd(&s_cnt[SC_FD], fd);
-    }
+  const u32 b_comp = __ballot_sync(0xFFFFFFFFu, active && complete), b_inc = __ballot_sync(0xFFFFFFFFu, active && !complete);
+  const u32 b_bar = __ballot_sync(0xFFFFFFFFu, active && barrier), b_an = __ballot_sync(0xFFFFFFFFu, active && analysed);
+  const u32 b_mis = __ballot_sync(0xFFFFFFFFu, active && mismatch), b_bwc = __ballot_sync(0xFFFFFFFFu, is_round);
+  const u32 pres = __reduce_add_sync(0xFFFFFFFFu, n_present), fs = __reduce_add_sync(0xFFFFFFFFu, n_fs), fd = __reduce_add_sync(0xFFFFFFFFu, n_fd);
+  u64 brng = is_round ? my_rng : 0; u32 bk = is_round ? t.seq_off + j : NONE;
+  best_warp_reduce(brng, bk);
+  const double tot = warp_sum8(bw, lane);
+  if ((lane & 3) == 0) s_bw[wid][lane >> 2] = tot;
+  if (lane == 0) {
+    s_rounds[wid] = (u32)__popc(b_bwc);
+    TileSum ts; ts.best_rng = brng; ts.best_k = bk; ts.n_rounds = (u32)__popc(b_bwc); ts.n_an = (u32)__popc(b_an); ts.pad = 0;
+    sums[t.sum_idx] = ts;
+    if (b_comp) atomicAdd(&s_cnt[SC_COMP], (u32)__popc(b_comp));
+    if (b_inc) atomicAdd(&s_cnt[SC_INC], (u32)__popc(b_inc));
+    if (b_bar) atomicAdd(&s_cnt[SC_BAR], (u32)__popc(b_bar));
+    if (b_an) atomicAdd(&s_cnt[SC_AN], (u32)__popc(b_an));
+    if (b_mis) atomicAdd(&s_cnt[SC_MIS], (u32)__popc(b_mis));
+    if (pres) atomicAdd(&s_cnt[SC_PRES], pres);
+    if (fs) atomicAdd(&s_cnt[SC_FS], fs);
+    if (fd) atomicAdd(&s_cnt[SC_FD], fd);
+  }
+}
+
+// Class-0 CTA of the fused kernel: eight warp-tiles of one window and one time chunk.
+__device__ __forceinline__ void reduce_small_cta(const WinDesc& D, const FusedCta& t, const WarpTile* __restrict__ wts, TileSum* __restrict__ sums,
+                                                 const Registry& R, const Params& P, i64 now) {
+  __shared__ double s_bw[SMALL_SEQS / 32][SMALL_N];
+  __shared__ u32 s_comm[SMALL_SEQS / 32], s_rounds[SMALL_SEQS / 32];
+  __shared__ u32 s_cnt[SC_COUNT];
+  const u32 wid = threadIdx.x >> 5;
+  if (threadIdx.x < SC_COUNT) s_cnt[threadIdx.x] = 0;
+  if (threadIdx.x < SMALL_SEQS / 32) { s_comm[threadIdx.x] = NONE; s_rounds[threadIdx.x] = 0; }
+  __syncthreads();
+  if (wid < t.wt_count) {
+    const WarpTile wt = wts[t.wt_first + wid];
+    const u32 n = R.comm_n[wt.c];
+    if ((threadIdx.x & 31) == 0) s_comm[wid] = wt.c;
+    if (n == SMALL_N) reduce_small_warp<true>(D, wt, sums, R, P, now, n, s_bw, s_rounds, s_cnt);
+    else reduce_small_warp<false>(D, wt, sums, R, P, now, n, s_bw, s_rounds, s_cnt);
   }
   __syncthreads();
-  const u32 n_bwc = s_cnt[SC_BWC];
   if (threadIdx.x == 0) {
-    u64 brng = s_brng[0]; u32 bk = s_bk[0];
-    for (int q = 1; q < SMALL_SEQS / 32; ++q) best_merge(brng, bk, s_brng[q], s_bk[q]);
-    TileSum ts; ts.best_rng = brng; ts.best_k = bk; ts.n_rounds = n_bwc; ts.n_an = s_cnt[SC_AN]; ts.pad = 0;
-    sums[blockIdx.x] = ts;
     count_add(D.counters, C_COMPLETE, s_cnt[SC_COMP]); count_add(D.counters, C_INCOMPLETE, s_cnt[SC_INC]);
     count_add(D.counters, C_BARRIER, s_cnt[SC_BAR]); count_add(D.counters, C_ANALYSED, s_cnt[SC_AN]);
     count_add(D.counters, C_MISMATCH, s_cnt[SC_MIS]); count_add(D.counters, C_PRESENT, s_cnt[SC_PRES]);
     count_add(D.counters, C_FLAG_SKEW, s_cnt[SC_FS]); count_add(D.counters, C_FLAG_DUR, s_cnt[SC_FD]);
   }
-  if (threadIdx.x < n && n_bwc) {
-    double v = 0.0;
-#pragma unroll
-    for (int q = 0; q < SMALL_SEQS / 32; ++q) v += s_bw[q][threadIdx.x];
-    atomicAdd(&R.bw_sum[mem[threadIdx.x]], v);
-    atomicAdd(&R.bw_cnt[mem[threadIdx.x]], n_bwc);
+  // per-rank bandwidth: consecutive warp-tiles of one communicator are summed before the atomics
+  if (threadIdx.x < (SMALL_SEQS / 32) * SMALL_N) {
+    const u32 q0 = threadIdx.x >> 3, m = threadIdx.x & 7, c = s_comm[q0];
+    if (c != NONE && (q0 == 0 || s_comm[q0 - 1] != c) && m < R.comm_n[c]) {
+      double v = 0.0; u32 rounds = 0;
+      for (u32 q = q0; q < SMALL_SEQS / 32 && s_comm[q] == c; ++q) { v += s_bw[q][m]; rounds += s_rounds[q]; }
+      if (rounds) {
+        const u32 rank = R.members[R.comm_moff[c] + m];
+        atomicAdd(&R.bw_sum[rank], v); atomicAdd(&R.bw_cnt[rank], rounds);
+      }
+    }
   }
-}
-
-__global__ void __launch_bounds__(SMALL_SEQS) k_reduce_small(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles,
-                                                                 TileSum* __restrict__ sums, Registry R, Params P, i64 now) {
-  __shared__ double s_bw[SMALL_SEQS / 32][SMALL_N];
-  __shared__ u64 s_brng[SMALL_SEQS / 32];
-  __shared__ u32 s_bk[SMALL_SEQS / 32];
-  __shared__ u32 s_cnt[SC_COUNT];
-  if (threadIdx.x < SC_COUNT) s_cnt[threadIdx.x] = 0;
-  __syncthreads();
-  const Tile t = tiles[blockIdx.x];
-  const WinDesc& D = wd[t.w];
-  const u32 n = R.comm_n[t.c];
-  if (n == SMALL_N) reduce_small_tile<true>(D, t, sums, R, P, now, n, s_bw, s_brng, s_bk, s_cnt);
-  else reduce_small_tile<false>(D, t, sums, R, P, now, n, s_bw, s_brng, s_bk, s_cnt);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1027,11 +1166,9 @@ inline size_t warp_smem_bytes() {
   return cap * (3 * 8 + 4 + 2) + 16 + (MID_THREADS / 32) * WARP_N * sizeof(double);
 }
 
-__global__ void __launch_bounds__(MID_THREADS) k_reduce_warp(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles,
-                                                             TileSum* __restrict__ sums, Registry R, Params P, i64 now) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  const Tile t = tiles[blockIdx.x];
-  const WinDesc& D = wd[t.w];
+// Class-1 CTA of the fused kernel: one tile of S groups of one communicator.
+__device__ __forceinline__ void reduce_warp_cta(const WinDesc& D, const FusedCta& t, TileSum* __restrict__ sums, const Registry& R, const Params& P,
+                                                i64 now, unsigned char* smem_raw) {
   const u32 c = t.c, n = R.comm_n[c];
   const RangeRow row = D.ranges[c];
   const u32* mem = R.members + R.comm_moff[c];
@@ -1196,11 +1333,24 @@ __global__ void __launch_bounds__(MID_THREADS) k_reduce_warp(const WinDesc* __re
     u64 brng = s_brng[0]; u32 bk = s_bk[0];
     for (int q = 1; q < MID_THREADS / 32; ++q) best_merge(brng, bk, s_brng[q], s_bk[q]);
     TileSum ts; ts.best_rng = brng; ts.best_k = bk; ts.n_rounds = rounds; ts.n_an = s_cnt[3]; ts.pad = 0;
-    sums[blockIdx.x] = ts;
+    sums[t.sum_idx] = ts;
     count_add(D.counters, C_COMPLETE, s_cnt[0]); count_add(D.counters, C_INCOMPLETE, s_cnt[1]); count_add(D.counters, C_BARRIER, s_cnt[2]);
     count_add(D.counters, C_ANALYSED, s_cnt[3]); count_add(D.counters, C_MISMATCH, s_cnt[4]); count_add(D.counters, C_PRESENT, s_cnt[5]);
     count_add(D.counters, C_FLAG_SKEW, s_cnt[6]); count_add(D.counters, C_FLAG_DUR, s_cnt[7]);
   }
+}
+
+// ------------------------------------------------------------------------------------------------
+// fused reduce kernel for communicators of up to 128 ranks: the work list is chunk-major, so CTAs that
+// run together gather from the same stretch of every rank's records
+// ------------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(SMALL_SEQS) k_reduce_fused(const WinDesc* __restrict__ wd, const FusedCta* __restrict__ ctas,
+                                                             const WarpTile* __restrict__ wts, TileSum* __restrict__ sums, Registry R, Params P, i64 now) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  const FusedCta t = ctas[blockIdx.x];
+  const WinDesc& D = wd[t.w];
+  if (t.cls == 0) reduce_small_cta(D, t, wts, sums, R, P, now);
+  else reduce_warp_cta(D, t, sums, R, P, now, smem_raw);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -1428,7 +1578,7 @@ __global__ void __launch_bounds__(LARGE_THREADS) k_reduce_large(const WinDesc* _
 __global__ void __launch_bounds__(128) k_window_decide(const WinDesc* __restrict__ wd, u32 nw, Registry R, Params P) {
   const u32 c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (c >= R.n_comms) return;
-  const u32 n = R.comm_n[c], cls = comm_class(n), S_tile = tile_seqs(n);
+  const u32 n = R.comm_n[c], cls = comm_class(n);
   const u32* mem = R.members + R.comm_moff[c];
   CommState st = R.state[c];
   for (u32 w = 0; w < nw; ++w) {
@@ -1439,8 +1589,8 @@ __global__ void __launch_bounds__(128) k_window_decide(const WinDesc* __restrict
     const i64* t_max = D.gi64 + (u64)GI_T_MAX * G + row.group0;
     const i64* t_min = D.gi64 + (u64)GI_T_MIN * G + row.group0;
     // round counts and the Eq. 2 candidate come from the tile summaries the reduce kernels left behind
-    const TileSum* ts = D.tsum[cls] + row.tile0;
-    const u32 nt = (row.n_seq + S_tile - 1) / S_tile;
+    const TileSum* ts = D.tsum[cls <= 1 ? 0 : cls - 1] + row.tile0;
+    const u32 nt = row.n_units;
     u32 n_rounds = 0, n_an = 0;
     u64 best_rng = 0; u32 best_k = NONE;
     for (u32 q = lane; q < nt; q += 32) {
