@@ -17,8 +17,8 @@ constexpr u32 NONE = 0xFFFFFFFFu;
 constexpr u64 U64_MAX_ = ~0ull;
 
 // ---- launch geometry ----
-constexpr int REC_THREADS = 256;       // record-streaming kernels: threads per CTA
-constexpr int REC_PER_THREAD = 8;
+constexpr int REC_THREADS = 128;       // record-streaming kernels: threads per CTA
+constexpr int REC_PER_THREAD = 16;     //   each walks a run of consecutive records
 constexpr int REC_PER_CTA = REC_THREADS * REC_PER_THREAD;
 constexpr int SMALL_N = 8;             // communicators of up to 8 ranks: one thread per group
 constexpr int SMALL_SEQS = 256;        //   threads per CTA: eight warp-tiles of up to 32 op counters

@@ -96,10 +96,34 @@ __device__ __forceinline__ void best_warp_reduce(u64& rng, u32& k) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// group-by, part 1: which op counters does every communicator cover in every window.
-// The dependent lookups of a thread's eight records are issued stage by stage (all hash probes, then
-// all range checks) so that their latencies overlap instead of adding up.
+// record-streaming kernels (group-by parts 1 and 3). A CTA stages the key columns of REC_PER_CTA
+// consecutive records in shared memory with coalesced 128-bit loads; each thread then walks a run of
+// REC_RUN consecutive records. In rank-major or arrival-ordered uploads a run cycles through a handful
+// of (rank, communicator) pairs, which the thread keeps in registers, so the registry is consulted a
+// few times per run instead of once per record. Any order is handled: a full cache is flushed.
 // ------------------------------------------------------------------------------------------------
+constexpr int REC_RUN = REC_PER_CTA / REC_THREADS;       // consecutive records per thread
+constexpr int REC_PITCH = REC_RUN + 1;                   // shared-memory pitch of a run (conflict-free walks)
+constexpr int RC = 4;                                    // cached pairs per thread
+
+// Copies n_valid <= REC_PER_CTA elements of a u32 column, starting at record `first`, into s[(i / RUN) * PITCH + i % RUN].
+__device__ __forceinline__ void stage_column(const u32* __restrict__ col, u64 first, u32 n_valid, u32* s) {
+  if ((((uintptr_t)(col + first)) & 15) == 0) {
+    for (u32 q = threadIdx.x; q < REC_PER_CTA / 4; q += REC_THREADS) {
+      const u32 i = q * 4;
+      if (i + 4 <= n_valid) {
+        const uint4 v = *reinterpret_cast<const uint4*>(col + first + i);
+        u32* d = s + (i / REC_RUN) * REC_PITCH + (i % REC_RUN);      // REC_RUN is a multiple of 4: the four stay in one run
+        d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+      } else {
+        for (u32 k = i; k < n_valid; ++k) s[(k / REC_RUN) * REC_PITCH + (k % REC_RUN)] = col[first + k];
+      }
+    }
+  } else {
+    for (u32 i = threadIdx.x; i < n_valid; i += REC_THREADS) s[(i / REC_RUN) * REC_PITCH + (i % REC_RUN)] = col[first + i];
+  }
+}
+
 __device__ __forceinline__ void range_widen(const WinDesc& D, u32 c, u32 mn, u32 mx) {
   if (mn < __ldcg(&D.rmin[c])) atomicMin(&D.rmin[c], mn);
   if (mx > __ldcg(&D.rmax[c])) atomicMax(&D.rmax[c], mx);
@@ -117,46 +141,48 @@ __device__ __forceinline__ void range_note(const WinDesc& D, u32* t_key, u32* t_
   range_widen(D, c, mn, mx);
 }
 
+// ---- group-by, part 1: which op counters does every communicator cover in every window ----
 __global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __restrict__ wd, u32 nw, Registry R) {
+  __shared__ u32 s_comm[REC_THREADS * REC_PITCH], s_seq[REC_THREADS * REC_PITCH];
   __shared__ u32 t_key[RANGE_TAB], t_mn[RANGE_TAB], t_mx[RANGE_TAB];
   if (threadIdx.x < RANGE_TAB) { t_key[threadIdx.x] = NONE; t_mn[threadIdx.x] = NONE; t_mx[threadIdx.x] = 0; }
-  __syncthreads();
   const u32 w = find_window(wd, nw, blockIdx.x);
   const WinDesc& D = wd[w];
-  const u64 base = (u64)(blockIdx.x - D.cta0) * REC_PER_CTA;
-  u32 cid[REC_PER_THREAD], sq[REC_PER_THREAD]; uint4 he[REC_PER_THREAD];
+  const u64 first = (u64)(blockIdx.x - D.cta0) * REC_PER_CTA;
+  const u32 n_valid = D.n_rec - first < REC_PER_CTA ? (u32)(D.n_rec - first) : (u32)REC_PER_CTA;
+  stage_column(D.comm, first, n_valid, s_comm);
+  stage_column(D.seq, first, n_valid, s_seq);
+  __syncthreads();
+  // cached communicators: id, index (NONE = unregistered), seq0, smallest / largest counter seen (empty: mn > mx)
+  u32 e_cid[RC], e_c[RC], e_s0[RC], e_mn[RC], e_mx[RC]; int cn = 0;
+  const u32 r0 = threadIdx.x * REC_RUN;
+  const u32 len = r0 >= n_valid ? 0u : (n_valid - r0 < REC_RUN ? n_valid - r0 : (u32)REC_RUN);
+  const u32* pc = s_comm + threadIdx.x * REC_PITCH; const u32* ps = s_seq + threadIdx.x * REC_PITCH;
+  for (u32 k = 0; k < len; ++k) {
+    const u32 cid = pc[k], sq = ps[k];
+    bool hit = false;
 #pragma unroll
-  for (int k = 0; k < REC_PER_THREAD; ++k) {
-    const u64 i = base + (u64)k * REC_THREADS + threadIdx.x;
-    const bool in = i < D.n_rec;
-    cid[k] = in ? D.comm[i] : NONE; sq[k] = in ? D.seq[i] : 0u;
-  }
-#pragma unroll
-  for (int k = 0; k < REC_PER_THREAD; ++k) he[k] = R.hash[hash_home(R, cid[k])];
-  // the thread's records are 256 apart: in a rank-major upload they cycle through a few communicators,
-  // so fold them into at most four (communicator, min, max) triples, then into the CTA's table
-  u32 uc[4], umn[4], umx[4]; int cnt = 0;
-#pragma unroll
-  for (int k = 0; k < REC_PER_THREAD; ++k) {
-    const u64 i = base + (u64)k * REC_THREADS + threadIdx.x;
-    const uint4 e = comm_find(R, cid[k], he[k]);
-    if (i < D.n_rec && e.y != NONE && sq[k] >= e.z) {
-      bool found = false;
-#pragma unroll
-      for (int q = 0; q < 4; ++q)
-        if (q < cnt && uc[q] == e.y) { umn[q] = sq[k] < umn[q] ? sq[k] : umn[q]; umx[q] = sq[k] > umx[q] ? sq[k] : umx[q]; found = true; }
-      if (!found) {
-        if (cnt == 4) range_note(D, t_key, t_mn, t_mx, e.y, sq[k], sq[k]);
-        else {
-#pragma unroll
-          for (int q = 0; q < 4; ++q) if (q == cnt) { uc[q] = e.y; umn[q] = sq[k]; umx[q] = sq[k]; }
-          ++cnt;
-        }
+    for (int e = 0; e < RC; ++e) {
+      if (e < cn && e_cid[e] == cid) {
+        hit = true;
+        if (e_c[e] != NONE && sq >= e_s0[e]) { e_mn[e] = sq < e_mn[e] ? sq : e_mn[e]; e_mx[e] = sq > e_mx[e] ? sq : e_mx[e]; }
       }
+    }
+    if (!hit) {
+      if (cn == RC) {
+#pragma unroll
+        for (int e = 0; e < RC; ++e) if (e_c[e] != NONE && e_mn[e] <= e_mx[e]) range_note(D, t_key, t_mn, t_mx, e_c[e], e_mn[e], e_mx[e]);
+        cn = 0;
+      }
+      const uint4 h = comm_find(R, cid, R.hash[hash_home(R, cid)]);
+      const bool ok = h.y != NONE && sq >= h.z;
+#pragma unroll
+      for (int e = 0; e < RC; ++e) if (e == cn) { e_cid[e] = cid; e_c[e] = h.y; e_s0[e] = h.z; e_mn[e] = ok ? sq : NONE; e_mx[e] = ok ? sq : 0u; }
+      ++cn;
     }
   }
 #pragma unroll
-  for (int q = 0; q < 4; ++q) if (q < cnt) range_note(D, t_key, t_mn, t_mx, uc[q], umn[q], umx[q]);
+  for (int e = 0; e < RC; ++e) if (e < cn && e_c[e] != NONE && e_mn[e] <= e_mx[e]) range_note(D, t_key, t_mn, t_mx, e_c[e], e_mn[e], e_mx[e]);
   __syncthreads();
   if (threadIdx.x < RANGE_TAB && t_key[threadIdx.x] != NONE) range_widen(D, t_key[threadIdx.x], t_mn[threadIdx.x], t_mx[threadIdx.x]);
 }
@@ -417,6 +443,9 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
 // ------------------------------------------------------------------------------------------------
 // Registry walk for a record whose (rank, communicator) pair is not inline: returns index << 13 | position in the
 // low word, or NONE there with the rejecting CCLD_E_* bit in the high word.
+constexpr int SCAT_THREADS = 256;     // lanes on consecutive records: the stores of a warp land close together
+constexpr int SCAT_PER_THREAD = REC_PER_CTA / SCAT_THREADS;
+
 __device__ __noinline__ u64 resolve_slow(const Registry& R, u32 rank, u32 cid) {
   const u32 c = comm_lookup(R, cid);
   if (c == NONE) return ((u64)CCLD_E_UNKNOWN_COMM << 32) | NONE;
@@ -425,20 +454,23 @@ __device__ __noinline__ u64 resolve_slow(const Registry& R, u32 rank, u32 cid) {
   return (c << RANK_TAB_POS_BITS) | pos;
 }
 
-__global__ void __launch_bounds__(REC_THREADS) k_slot_scatter(const WinDesc* __restrict__ wd, u32 nw, Registry R) {
+__global__ void __launch_bounds__(SCAT_THREADS) k_slot_scatter(const WinDesc* __restrict__ wd, u32 nw, Registry R) {
   const u32 w = find_window(wd, nw, blockIdx.x);
   const WinDesc& D = wd[w];
   const u64 base = (u64)(blockIdx.x - D.cta0) * REC_PER_CTA;
   u32 err = 0, rej = 0, internal = 0;
-  constexpr int HALF = REC_PER_THREAD / 2;
+  // descriptor fields in registers: the stores below could alias the descriptor as far as the compiler knows
+  u32* const perm = D.perm; const u64 n_slots = D.n_slots; const uint4* const srow = D.srow; const u64 n_rec = D.n_rec;
+  const u32 *c_rank = D.rank, *c_comm = D.comm, *c_seq = D.seq;
+  constexpr int HALF = SCAT_PER_THREAD / 2;
 #pragma unroll
   for (int h = 0; h < 2; ++h) {
     u32 rk[HALF], cid[HALF], sq[HALF]; bool in[HALF];
 #pragma unroll
     for (int k = 0; k < HALF; ++k) {
-      const u64 i = base + (u64)(h * HALF + k) * REC_THREADS + threadIdx.x;
-      in[k] = i < D.n_rec;
-      rk[k] = in[k] ? D.rank[i] : 0u; cid[k] = in[k] ? D.comm[i] : 0u; sq[k] = in[k] ? D.seq[i] : 0u;
+      const u64 i = base + (u64)(h * HALF + k) * SCAT_THREADS + threadIdx.x;
+      in[k] = i < n_rec;
+      rk[k] = in[k] ? c_rank[i] : 0u; cid[k] = in[k] ? c_comm[i] : 0u; sq[k] = in[k] ? c_seq[i] : 0u;
     }
     uint4 ta[HALF], tb[HALF];
 #pragma unroll
@@ -463,7 +495,7 @@ __global__ void __launch_bounds__(REC_THREADS) k_slot_scatter(const WinDesc* __r
     }
     uint4 sr[HALF];
 #pragma unroll
-    for (int k = 0; k < HALF; ++k) sr[k] = cp[k] != NONE ? D.srow[cp[k] >> RANK_TAB_POS_BITS] : make_uint4(0, 0, 0, 0);
+    for (int k = 0; k < HALF; ++k) sr[k] = cp[k] != NONE ? srow[cp[k] >> RANK_TAB_POS_BITS] : make_uint4(0, 0, 0, 0);
 #pragma unroll
     for (int k = 0; k < HALF; ++k) {
       if (cp[k] != NONE) {
@@ -474,8 +506,8 @@ __global__ void __launch_bounds__(REC_THREADS) k_slot_scatter(const WinDesc* __r
         } else {
           const u64 sb = (u64)sr[k].x | ((u64)sr[k].y << 32);
           const u64 slot = sb + (u64)sq[k] * n + (cp[k] & ((1u << RANK_TAB_POS_BITS) - 1));
-          if (slot >= D.n_slots) internal = 1;
-          else D.perm[slot] = (u32)(base + (u64)(h * HALF + k) * REC_THREADS + threadIdx.x);
+          if (slot >= n_slots) internal = 1;
+          else perm[slot] = (u32)(base + (u64)(h * HALF + k) * SCAT_THREADS + threadIdx.x);
         }
       }
     }
