@@ -69,6 +69,17 @@ def peak_hbm():
         return HBM_FALLBACK_GBS, "fallback"
 
 
+def max_over_ranks(ms, device):
+    """The slowest rank's elapsed time (all-reduce MAX over the default process group; identity for one rank)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
@@ -209,10 +220,7 @@ def run_ours(args, rank, world, local_rank):
     ms = ev0.elapsed_time(ev1)
     kt = an.get_kernel_times()
     an.timing_enable(False)
-    if world > 1:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, dev)
     value = world * n_rec * args.steps / (ms * 1e-3)
 
     # sanity: the injected ranks are the suspects
@@ -285,10 +293,7 @@ def run_ours(args, rank, world, local_rank):
         e1.record()
         torch.cuda.synchronize()
         e_ms = e0.elapsed_time(e1)
-        if world > 1:
-            t = torch.tensor([e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
+        e_ms = max_over_ranks(e_ms, dev)
         e2e = {"value": world * e_rec * e_steps / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "windows_per_step": NE, "steps": e_steps, "ms_per_step": e_ms / e_steps}
         an_e.close()

@@ -662,39 +662,73 @@ __device__ __forceinline__ void reduce_small_warp(const WinDesc& D, const WarpTi
 #pragma unroll
       for (int p = 0; p < SMALL_N; ++p) idx[p] = (FULL || (u32)p < n) ? D.perm[slot + p] : NONE;
     }
-    // every gather is issued before any is used: a missing member reads record 0 and is masked out below
-    i64 ld_a[SMALL_N], ld_b[SMALL_N]; u64 ld_by[SMALL_N]; u32 ld_op[SMALL_N], ld_ch[SMALL_N];
-    const bool have_rates = D.send_chg != nullptr;
+    // Two batches of gathers, each issued in full before any of it is used (a missing member reads record 0 and
+    // is masked out): first the times, which are reduced to 32-bit keys, then the op-set and rate columns.
+    u32 safe[SMALL_N];
 #pragma unroll
-    for (int p = 0; p < SMALL_N; ++p) {
-      const u32 ix = idx[p] == NONE ? 0u : idx[p];
-      ld_a[p] = D.t_enter[ix]; ld_b[p] = D.t_exit[ix]; ld_by[p] = D.bytes[ix]; ld_op[p] = D.op[ix];
-      ld_ch[p] = 0;
-      if (have_rates) { const u32 sc = D.send_chg[ix], rc = D.recv_chg[ix]; ld_ch[p] = sc > rc ? sc : rc; }
-    }
-    u64 te[SMALL_N], du[SMALL_N];
+    for (int p = 0; p < SMALL_N; ++p) safe[p] = idx[p] == NONE ? 0u : idx[p];
     i64 x_max = INT64_MIN, age = -1;
-    u64 gbytes = 0; u32 gop = 0; bool have_first = false, inflight = false, bad_time = false;
-    u32 max_chg = 0, pos_chg = 0; bool have_chg = false;
+    bool inflight = false, bad_time = false;
     u32 miss = 0;
-    complete = true;
+    u64 e_min = 0, e_max = 0, tmax = 0, tmin = 0; u32 pmax = 0, pmin = 0;
+    u32 sk[SMALL_N], dd[SMALL_N];
+    bool fast = false;
+    {
+      const i64* __restrict__ c_te = D.t_enter; const i64* __restrict__ c_tx = D.t_exit;
+      i64 ld_a[SMALL_N], ld_b[SMALL_N];
 #pragma unroll
-    for (int p = 0; p < SMALL_N; ++p) {
-      te[p] = U64_MAX_; du[p] = U64_MAX_;
-      if (FULL || (u32)p < n) {
-        if (idx[p] == NONE) { complete = false; miss |= 1u << p; }
-        else {
-          ++n_present;
-          const i64 a = ld_a[p], b = ld_b[p];
-          const u64 by = ld_by[p]; const u32 o = ld_op[p];
-          const u32 ch = ld_ch[p];
-          if (!have_first) { gbytes = by; gop = o; have_first = true; }
-          else if (o != gop || by != gbytes) mismatch = true;
-          if (b == -1) { inflight = true; complete = false; const i64 ag = now - a; age = ag > age ? ag : age; }
-          else if (a < 0 || b < a) { bad_time = true; complete = false; }
-          te[p] = (u64)a; du[p] = (u64)(b - a);
-          x_max = b > x_max ? b : x_max;
-          if (!have_chg || ch > max_chg) { max_chg = ch; pos_chg = p; have_chg = true; }
+      for (int p = 0; p < SMALL_N; ++p) { ld_a[p] = c_te[safe[p]]; ld_b[p] = c_tx[safe[p]]; }
+#pragma unroll
+      for (int p = 0; p < SMALL_N; ++p) {
+        if (FULL || (u32)p < n) {
+          if (idx[p] == NONE) miss |= 1u << p;
+          else {
+            ++n_present;
+            const i64 a = ld_a[p], b = ld_b[p];
+            if (b == -1) { inflight = true; const i64 ag = now - a; age = ag > age ? ag : age; }
+            else if (a < 0 || b < a) bad_time = true;
+            x_max = b > x_max ? b : x_max;
+          }
+        }
+      }
+      complete = miss == 0 && !inflight && !bad_time;
+      if (complete) {
+        e_min = (u64)ld_a[0]; e_max = e_min; tmax = (u64)(ld_b[0] - ld_a[0]); tmin = tmax;
+#pragma unroll
+        for (int p = 1; p < SMALL_N; ++p) {
+          if (FULL || (u32)p < n) {
+            const u64 te = (u64)ld_a[p], du = (u64)(ld_b[p] - ld_a[p]);
+            e_min = te < e_min ? te : e_min; e_max = te > e_max ? te : e_max;
+            if (du > tmax) { tmax = du; pmax = p; }
+            if (du < tmin) { tmin = du; pmin = p; }
+          }
+        }
+        fast = e_max - e_min < 0xFFFFFFFFull && tmax - tmin < 0xFFFFFFFFull;
+#pragma unroll
+        for (int p = 0; p < SMALL_N; ++p) {
+          const bool in = FULL || (u32)p < n;
+          sk[p] = in ? (u32)((u64)ld_a[p] - e_min) : 0xFFFFFFFFu; dd[p] = in ? (u32)((u64)(ld_b[p] - ld_a[p]) - tmin) : 0xFFFFFFFFu;
+        }
+      }
+    }
+    asm volatile("" ::: "memory");                           // keep the second batch behind the first
+    u64 gbytes = 0; u32 gop = 0; bool have_first = false;
+    u32 max_chg = 0, pos_chg = 0; bool have_chg = false;
+    {
+      const u64* __restrict__ c_by = D.bytes; const u8* __restrict__ c_op = D.op;
+      const u32* __restrict__ c_sc = D.send_chg; const u32* __restrict__ c_rc = D.recv_chg;
+      u64 ld_by[SMALL_N]; u32 ld_op[SMALL_N], ld_ch[SMALL_N];
+#pragma unroll
+      for (int p = 0; p < SMALL_N; ++p) {
+        ld_by[p] = c_by[safe[p]]; ld_op[p] = c_op[safe[p]]; ld_ch[p] = 0;
+        if (c_sc != nullptr) { const u32 sc = c_sc[safe[p]], rc = c_rc[safe[p]]; ld_ch[p] = sc > rc ? sc : rc; }
+      }
+#pragma unroll
+      for (int p = 0; p < SMALL_N; ++p) {
+        if ((FULL || (u32)p < n) && idx[p] != NONE) {
+          if (!have_first) { gbytes = ld_by[p]; gop = ld_op[p]; have_first = true; }
+          else if (ld_op[p] != gop || ld_by[p] != gbytes) mismatch = true;
+          if (!have_chg || ld_ch[p] > max_chg) { max_chg = ld_ch[p]; pos_chg = p; have_chg = true; }
         }
       }
     }
@@ -714,15 +748,6 @@ __device__ __forceinline__ void reduce_small_warp(const WinDesc& D, const WarpTi
       if (inflight && age > P.hang_ns && !barrier) { gfl |= CCLD_G_HANG_ALERT; raise_alert(D, R.comm_id[c], row.seq_lo + t.seq_off + j, age); }
     } else {
       gfl |= CCLD_G_COMPLETE;
-      u64 e_min = te[0], e_max = te[0], tmax = du[0], tmin = du[0]; u32 pmax = 0, pmin = 0;
-#pragma unroll
-      for (int p = 1; p < SMALL_N; ++p) {
-        if (FULL || (u32)p < n) {
-          e_min = te[p] < e_min ? te[p] : e_min; e_max = te[p] > e_max ? te[p] : e_max;
-          if (du[p] > tmax) { tmax = du[p]; pmax = p; }
-          if (du[p] < tmin) { tmin = du[p]; pmin = p; }
-        }
-      }
       const u64 askew = e_max - e_min;
       const i64 span = x_max - (i64)e_min;
       double num, den; bus_factor(gop, n, &num, &den);
@@ -733,26 +758,22 @@ __device__ __forceinline__ void reduce_small_warp(const WinDesc& D, const WarpTi
       r_tmin = mem[pmin]; r_tmax = mem[pmax]; r_chg = mem[pos_chg];
       analysed = !barrier && n >= P.min_group;
       if (analysed) gfl |= CCLD_G_ANALYSED;
-      if (askew < 0xFFFFFFFFull && my_rng < 0xFFFFFFFFull) {
-        // 32-bit keys from here on: skew, and duration minus the shortest duration
-        u32 sk[SMALL_N], dd[SMALL_N];
-#pragma unroll
-        for (int p = 0; p < SMALL_N; ++p) {
-          const bool in = FULL || (u32)p < n;
-          sk[p] = in ? (u32)(te[p] - e_min) : 0xFFFFFFFFu; dd[p] = in ? (u32)(du[p] - tmin) : 0xFFFFFFFFu;
-        }
+      if (fast) {
+        // 32-bit keys: skew, and duration minus the shortest duration
         if (analysed) {
           u32 ms, ds, md, dm;
           median_mad8<u32>(sk, n, &ms, &ds);
           median_mad8<u32>(dd, n, &md, &dm);
           med_s = ms; mad_s = ds; med_d = tmin + md; mad_d = dm;
-          const u64 ts = (u64)ds * k_milli, td = (u64)dm * k_milli;
+          // |x - med| * 1000 > k * MAD  <=>  |x - med| > floor(k * MAD / 1000); deviations are below 2^32
+          const u64 qs = (u64)ds * k_milli / 1000u, qd = (u64)dm * k_milli / 1000u;
+          const u32 ts = qs > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)qs, td = qd > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)qd;
           packed = 0;
 #pragma unroll
           for (int p = 0; p < SMALL_N; ++p) {
             if (FULL || (u32)p < n) {
               const u32 a = sk[p] >= ms ? sk[p] - ms : ms - sk[p], b = dd[p] >= md ? dd[p] - md : md - dd[p];
-              const bool so = (u64)a * 1000u > ts, sh = sk[p] > ms, dq = (u64)b * 1000u > td, dh = dd[p] > md;
+              const bool so = a > ts, sh = sk[p] > ms, dq = b > td, dh = dd[p] > md;
               packed |= (u64)((so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0)) << (8 * p);
             }
           }

@@ -1,0 +1,85 @@
+"""Parity at the benchmark's full size and launch configuration.
+
+The streaming slow-mix workload (4,096 ranks, 100 windows of 1,000 ops per rank, 409.6 M records) is
+generated on the GPU and analysed in ONE call, exactly as bench.py does. The oracle then recomputes
+sampled windows one by one (each on a fresh oracle: the per-op table, flags, slot permutation and
+counts do not depend on earlier windows), and the first two windows in sequence for the stateful
+outputs. Properties that hold at any size are checked on every window.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle as orc
+import tracegen as tg
+from parity import compare_window, same, close
+
+pytestmark = pytest.mark.gpu
+
+
+def test_cfg4_full_size_in_the_bench_configuration():
+    import paper_2605_04478_b200 as ccld
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * 2**30:
+        pytest.skip("needs about 30 GB of device memory")
+    spec = tg.cfg4()
+    NW = spec.n_windows
+    assert NW == 100 and tg.records_per_window(spec) == 4_096_000
+    an = ccld.Analyzer()
+    reg = tg.registry(spec)
+    for cid, ranks, seq0 in reg:
+        an.comm_register(cid, ranks, 0, seq0)
+    sample = [0, 1, 37, 99]
+    kept = {}
+    for w in range(NW):
+        win = tg.gen_window(spec, w, device="cuda")
+        an.trace_upload(w, win.cols)
+        if w in sample:
+            kept[w] = {k: v.cpu() for k, v in win.cols.items()}
+        now = win.now_ns
+    an.analyze_window(0, NW, now)
+
+    # properties on every window
+    tot_flags = 0
+    for w in range(NW):
+        v = an.get_verdict(w)
+        assert v["n_records"] == 4_096_000 and v["n_groups"] == 422_400 and v["n_slots"] == 4_096_000
+        assert v["n_complete"] == 422_400 and v["n_incomplete"] == 0 and v["n_rejected"] == 0 and v["error_bits"] == 0
+        assert v["n_analysed"] == 422_400 and v["n_comm_rows_total"] == 1088 and v["n_alerts_total"] == 0
+        tot_flags += v["n_flag_skew"] + v["n_flag_dur"]
+    st = an.get_rank_stats(spec.n_ranks)
+    assert int(st["votes"].sum()) == tot_flags                       # vote total = flag total
+    assert (st["ops"] == 100_000).all() and (st["bw_cnt"] == 100_000).all()
+    sus = v["suspects"]
+    assert sorted(set(int(r) for r in sus["rank"][sus["kind"] == 1])) == spec.truth["stragglers"]
+    assert sorted(set(int(r) for r in sus["rank"][sus["kind"] == 2])) == spec.truth["slow_links"]
+
+    # sampled windows against the oracle, element by element (stateless outputs)
+    for w in sample[2:]:
+        o = orc.Oracle()
+        for cid, ranks, seq0 in reg:
+            o.comm_register(cid, ranks, seq0)
+        o.upload(w, kept[w]); o.analyze(w, 1, now)
+        compare_window(an, o, w, stateless_only=True)
+        t = an.get_optable(w)
+        assert (t["arrival_skew"] >= 0).all() and (t["t_min"] <= t["med_dur"]).all() and (t["med_dur"] <= t["t_max"]).all()
+    # the first two windows in sequence: communicator rows and cumulative state too
+    o = orc.Oracle()
+    for cid, ranks, seq0 in reg:
+        o.comm_register(cid, ranks, seq0)
+    for w in (0, 1):
+        o.upload(w, kept[w])
+    o.analyze(0, 2, now)
+    for w in (0, 1):
+        compare_window(an, o, w)
+    # per-rank votes after two windows: analyse the same two windows alone on a second context
+    an2 = ccld.Analyzer()
+    for cid, ranks, seq0 in reg:
+        an2.comm_register(cid, ranks, 0, seq0)
+    for w in (0, 1):
+        an2.trace_upload(w, {k: v.cuda() for k, v in kept[w].items()})
+    an2.analyze_window(0, 2, now)
+    a, b = an2.get_rank_stats(spec.n_ranks), o.rank_stats(spec.n_ranks)
+    for k in ("votes", "ops", "bw_cnt"):
+        same(a[k], b[k], k)
+    close(a["bw_sum"], b["bw_sum"], "bw_sum")
