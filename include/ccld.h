@@ -238,7 +238,9 @@ int ccld_locate_hang(ccld_ctx* ctx, uint32_t window_id, uint32_t comm, uint32_t 
  *   lowest ring position); max_chg, rank_max_chg = most observed count changes and its rank;
  *   busbw = bytes * f / span in bytes per ns with f = 2(n-1)/n allreduce, (n-1)/n allgather,
  *   reducescatter, alltoall, 1 otherwise.
- * perm[slot] = index of the record in the uploaded columns, 0xFFFFFFFF if the member is missing.
+ * perm holds, per slot, the index of the record in the uploaded columns (0xFFFFFFFF if the member is
+ * missing). Unlike flags it is member-major inside a communicator: the record of ring position p and op
+ * counter s of communicator row r is perm[slot0_r + p * n_seq_r + (s - seq_lo_r)].
  */
 typedef struct {
   uint64_t n_groups, n_slots;

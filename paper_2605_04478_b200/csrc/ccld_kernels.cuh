@@ -72,6 +72,12 @@ __device__ __forceinline__ double busbw(double bytes_num, double den, i64 t) {
 
 __device__ __forceinline__ u64 absdiff(u64 a, u64 b) { return a >= b ? a - b : b - a; }
 
+// Where the record index of (communicator row, op-counter offset, ring position) sits in `perm`. The permutation
+// is member-major inside a communicator - [position][op counter] - so that consecutive records of one rank, which
+// carry consecutive op counters, scatter to consecutive entries, and so that a warp reading 32 consecutive op
+// counters of one member reads 128 contiguous bytes. Flags and per-op rows stay group-major.
+__device__ __forceinline__ u64 perm_at(const RangeRow& row, u32 seq_off, u32 pos) { return row.slot0 + (u64)pos * row.n_seq + seq_off; }
+
 __device__ __forceinline__ u64 shfl_xor64(u64 v, int m) { return __shfl_xor_sync(0xFFFFFFFFu, v, m); }
 
 __device__ __forceinline__ void count_add(u64* counters, int which, u32 v) {
@@ -319,8 +325,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
         r.seq_lo = it.rows ? D.rmin[c] : 0; r.n_seq = (u32)it.groups; r.row_idx = ex.rows; r.n = R.comm_n[c];
         r.group0 = ex.groups; r.slot0 = ex.slots; r.tile0 = 0; r.n_units = 0;
         D.ranges[c] = r;
-        const u64 sb = r.slot0 - (u64)r.seq_lo * r.n;
-        D.srow[c] = make_uint4((u32)sb, (u32)(sb >> 32), it.rows ? r.n : 0u, r.seq_lo);
+        D.srow[c] = make_uint4((u32)r.slot0, (u32)(r.slot0 >> 32), r.n_seq, r.seq_lo);
         if (it.rows && comm_class(r.n) <= 1) mx = r.n_seq > mx ? r.n_seq : mx;
       }
       run = plan_add(run, tot);
@@ -499,14 +504,14 @@ __global__ void __launch_bounds__(SCAT_THREADS) k_slot_scatter(const WinDesc* __
 #pragma unroll
     for (int k = 0; k < HALF; ++k) {
       if (cp[k] != NONE) {
-        const u32 n = sr[k].z, lo = sr[k].w;
-        if (n == 0 || sq[k] < lo) {
+        const u32 ns = sr[k].z, lo = sr[k].w;
+        if (ns == 0 || sq[k] < lo) {
           if (sq[k] < R.comm_seq0[cp[k] >> RANK_TAB_POS_BITS]) { err |= CCLD_E_SEQ_RANGE; ++rej; }
-          else if (n != 0) internal = 1;
+          else if (ns != 0) internal = 1;
         } else {
           const u64 sb = (u64)sr[k].x | ((u64)sr[k].y << 32);
-          const u64 slot = sb + (u64)sq[k] * n + (cp[k] & ((1u << RANK_TAB_POS_BITS) - 1));
-          if (slot >= n_slots) internal = 1;
+          const u64 slot = sb + (u64)(cp[k] & ((1u << RANK_TAB_POS_BITS) - 1)) * ns + (sq[k] - lo);
+          if (sq[k] - lo >= ns || slot >= n_slots) internal = 1;
           else perm[slot] = (u32)(base + (u64)(h * HALF + k) * SCAT_THREADS + threadIdx.x);
         }
       }
@@ -598,13 +603,13 @@ __device__ __forceinline__ double warp_sum8(double (&v)[8], u32 lane) {
 // A complete group whose skews or durations do not fit 32-bit keys (a spread of more than 4.29 s inside
 // one op): gathered again and handled here, out of line, so that the common path stays in 32 bits.
 // Returns the four order statistics, the packed flag bytes, and adds the members' bus bandwidths.
-__device__ __noinline__ u64 small_group64(const WinDesc& D, const Registry& R, const u32* mem, u64 slot, u32 n, u64 e_min, u32 k_milli,
+__device__ __noinline__ u64 small_group64(const WinDesc& D, const Registry& R, const u32* mem, u64 pslot, u32 pstride, u32 n, u64 e_min, u32 k_milli,
                                           bool analysed, bool add_bw, double bn, double den, u64* out4) {
   u64 sk[8], du[8];
 #pragma unroll
   for (int p = 0; p < 8; ++p) {
     sk[p] = U64_MAX_; du[p] = U64_MAX_;
-    if ((u32)p < n) { const u32 idx = D.perm[slot + p]; const i64 a = D.t_enter[idx], b = D.t_exit[idx]; sk[p] = (u64)a - e_min; du[p] = (u64)(b - a); }
+    if ((u32)p < n) { const u32 idx = D.perm[pslot + (u64)p * pstride]; const i64 a = D.t_enter[idx], b = D.t_exit[idx]; sk[p] = (u64)a - e_min; du[p] = (u64)(b - a); }
   }
   if (add_bw)
     for (u32 p = 0; p < n; ++p) atomicAdd(&R.bw_sum[mem[p]], busbw_fast(bn, den, (i64)du[p]));
@@ -655,12 +660,10 @@ __device__ __forceinline__ void reduce_small_warp(const WinDesc& D, const WarpTi
     const u64 g = row.group0 + t.seq_off + j;
     const u64 slot = row.slot0 + (u64)(t.seq_off + j) * n;
     u32 idx[SMALL_N];
-    if (FULL && (slot & 3) == 0) {
-      const uint4 a = *reinterpret_cast<const uint4*>(D.perm + slot), b = *reinterpret_cast<const uint4*>(D.perm + slot + 4);
-      idx[0] = a.x; idx[1] = a.y; idx[2] = a.z; idx[3] = a.w; idx[4] = b.x; idx[5] = b.y; idx[6] = b.z; idx[7] = b.w;
-    } else {
+    {
+      const u32* __restrict__ pm = D.perm + perm_at(row, t.seq_off + j, 0);
 #pragma unroll
-      for (int p = 0; p < SMALL_N; ++p) idx[p] = (FULL || (u32)p < n) ? D.perm[slot + p] : NONE;
+      for (int p = 0; p < SMALL_N; ++p) idx[p] = (FULL || (u32)p < n) ? pm[(u64)p * row.n_seq] : NONE;
     }
     // Two batches of gathers, each issued in full before any of it is used (a missing member reads record 0 and
     // is masked out): first the times, which are reduced to 32-bit keys, then the op-set and rate columns.
@@ -784,7 +787,7 @@ __device__ __forceinline__ void reduce_small_warp(const WinDesc& D, const WarpTi
         }
       } else {
         u64 o4[4];
-        packed = small_group64(D, R, mem, slot, n, e_min, k_milli, analysed, !barrier, bn, den, o4);
+        packed = small_group64(D, R, mem, perm_at(row, t.seq_off + j, 0), row.n_seq, n, e_min, k_milli, analysed, !barrier, bn, den, o4);
         med_s = o4[0]; mad_s = o4[1]; med_d = o4[2]; mad_d = o4[3];
       }
       if (analysed) {
@@ -939,7 +942,10 @@ __global__ void __launch_bounds__(MID_THREADS) k_reduce_mid(const WinDesc* __res
   const u32 n_el = S * n;
   if (threadIdx.x < 8) s_cnt[threadIdx.x] = 0;
   // 1. record indices, coalesced along the slot order
-  for (u32 e = threadIdx.x; e < n_el; e += MID_THREADS) { const u32 jg = e / n, p = e - jg * n; s_idx[jg * pitch + p] = D.perm[slot_t + e]; }
+  for (u32 p = threadIdx.x >> 5; p < n; p += MID_THREADS / 32) {
+    const u32* __restrict__ pm = D.perm + perm_at(row, t.seq_off, p);
+    for (u32 jg = threadIdx.x & 31; jg < S; jg += 32) s_idx[jg * pitch + p] = pm[jg];
+  }
   __syncthreads();
   // 2. gather: consecutive threads walk consecutive op counters of one member
   for (u32 e = threadIdx.x; e < n_el; e += MID_THREADS) {
@@ -1244,7 +1250,10 @@ __device__ __forceinline__ void reduce_warp_cta(const WinDesc& D, const FusedCta
   const u32 n_el = S * n;
   if (threadIdx.x < 8) s_cnt[threadIdx.x] = 0;
   // 1. record indices, coalesced along the slot order
-  for (u32 e = threadIdx.x; e < n_el; e += MID_THREADS) { const u32 jg = e / n, p = e - jg * n; s_idx[jg * pitch + p] = D.perm[slot_t + e]; }
+  for (u32 p = threadIdx.x >> 5; p < n; p += MID_THREADS / 32) {
+    const u32* __restrict__ pm = D.perm + perm_at(row, t.seq_off, p);
+    for (u32 jg = threadIdx.x & 31; jg < S; jg += 32) s_idx[jg * pitch + p] = pm[jg];
+  }
   __syncthreads();
   // 2. gather: consecutive threads walk consecutive op counters of one member
   for (u32 e = threadIdx.x; e < n_el; e += MID_THREADS) {
@@ -1493,12 +1502,14 @@ __global__ void __launch_bounds__(LARGE_THREADS) k_reduce_large(const WinDesc* _
 
   for (u32 jg = 0; jg < t.count; ++jg) {
     __syncthreads();
-    const u64 g = row.group0 + t.seq_off + jg, slot = row.slot0 + (u64)(t.seq_off + jg) * n;
+    const u64 g = row.group0 + t.seq_off + jg, slot = row.slot0 + (u64)(t.seq_off + jg) * n;      // slot: flags, group-major
     const u32 seq = row.seq_lo + t.seq_off + jg;
+    const u32* __restrict__ pm = D.perm + perm_at(row, t.seq_off + jg, 0);                          // member p at pm[p * n_seq]
+    const u64 pst = row.n_seq;
     // pass 1: gather, presence, first present member
     u32 npres = 0, first = NONE, stor = 0;
     for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS) {
-      const u32 idx = D.perm[slot + p];
+      const u32 idx = pm[p * pst];
       u64 te = 0, du = 0; u32 st = 0;
       if (idx != NONE) {
         const i64 x = D.t_enter[idx], y = D.t_exit[idx];
@@ -1513,14 +1524,14 @@ __global__ void __launch_bounds__(LARGE_THREADS) k_reduce_large(const WinDesc* _
     stor = block_reduce(stor, OpOrU32(), s_red32);
     const bool have_first = first != NONE;
     u64 gbytes = 0; u32 gop = 0;
-    if (have_first) { const u32 idx = D.perm[slot + first]; gbytes = D.bytes[idx]; gop = D.op[idx]; }
+    if (have_first) { const u32 idx = pm[first * pst]; gbytes = D.bytes[idx]; gop = D.op[idx]; }
     const bool inflight = stor & 2, bad_time = stor & 4, complete = npres == n && !inflight && !bad_time;
     const bool barrier = have_first && gop == CCLD_OP_ALLREDUCE && gbytes < P.barrier_bytes;
     // pass 2: op-set check, rate column, in-flight age, extrema
     u32 mism = 0; i64 age = -1; u64 chk = 0;
     u64 e_min = U64_MAX_, tmax = 0, tmin = U64_MAX_; i64 x_max = INT64_MIN;
     for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS) {
-      const u32 idx = D.perm[slot + p];
+      const u32 idx = pm[p * pst];
       if (idx == NONE) continue;
       if (D.op[idx] != gop || D.bytes[idx] != gbytes) mism = 1;
       u32 ch = 0;
@@ -1547,7 +1558,7 @@ __global__ void __launch_bounds__(LARGE_THREADS) k_reduce_large(const WinDesc* _
 
     if (!complete) {
       for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS)
-        D.flags[slot + p] = D.perm[slot + p] == NONE ? (CCLD_F_NOT_ANALYSED | CCLD_F_MISSING) : CCLD_F_NOT_ANALYSED;
+        D.flags[slot + p] = pm[p * pst] == NONE ? (CCLD_F_NOT_ANALYSED | CCLD_F_MISSING) : CCLD_F_NOT_ANALYSED;
       if (threadIdx.x == 0) {
         if (hang) raise_alert(D, R.comm_id[c], seq, age);
         for (int q = 0; q < GI_COUNT; ++q) D.gi64[(u64)q * G + g] = 0;
@@ -1740,7 +1751,7 @@ __global__ void __launch_bounds__(1024) k_hang_locate(const WinDesc* __restrict_
     const u64 cnt = (u64)(row.n_seq - s_first) * n;
     for (u64 e = threadIdx.x; e < cnt; e += blockDim.x) {
       const u32 so = s_first + (u32)(e / n), p = (u32)(e % n);
-      const u32 idx = D.perm[row.slot0 + (u64)so * n + p];
+      const u32 idx = D.perm[perm_at(row, so, p)];
       if (idx != NONE) {
         A.entered[p] = 1;
         if (row.seq_lo + so == A.seq && D.t_exit[idx] != -1) A.done[p] = 1;
