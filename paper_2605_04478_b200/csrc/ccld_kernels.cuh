@@ -1236,9 +1236,8 @@ __device__ __forceinline__ void reduce_warp_cta(const WinDesc& D, const FusedCta
   u64* s_te = (u64*)smem_raw;            // enter time
   u64* s_du = s_te + cap;                // duration
   u64* s_by = s_du + cap;                // bytes
-  u32* s_idx = (u32*)(s_by + cap);       // record index ...
-  u32* s_ch = s_idx;                     // ... replaced in place by max(send_chg, recv_chg) once the record is gathered
-  u8* s_op = (u8*)(s_idx + cap);
+  u32* s_ch = (u32*)(s_by + cap);        // max(send_chg, recv_chg)
+  u8* s_op = (u8*)(s_ch + cap);
   u8* s_st = s_op + cap;                 // 1 present, 2 in flight, 4 bad time
   double* s_bw = (double*)(((uintptr_t)(s_st + cap) + 15) & ~(uintptr_t)15);   // [warps][n_pad]
   __shared__ u32 s_cnt[8];
@@ -1249,26 +1248,26 @@ __device__ __forceinline__ void reduce_warp_cta(const WinDesc& D, const FusedCta
   const u64 g_t = row.group0 + t.seq_off;
   const u32 n_el = S * n;
   if (threadIdx.x < 8) s_cnt[threadIdx.x] = 0;
-  // 1. record indices, coalesced along the slot order
-  for (u32 p = threadIdx.x >> 5; p < n; p += MID_THREADS / 32) {
-    const u32* __restrict__ pm = D.perm + perm_at(row, t.seq_off, p);
-    for (u32 jg = threadIdx.x & 31; jg < S; jg += 32) s_idx[jg * pitch + p] = pm[jg];
-  }
-  __syncthreads();
-  // 2. gather: consecutive threads walk consecutive op counters of one member
-  for (u32 e = threadIdx.x; e < n_el; e += MID_THREADS) {
-    const u32 p = e / S, jg = e - p * S, a = jg * pitch + p;
-    const u32 idx = s_idx[a];
-    const u32 ix = idx == NONE ? 0u : idx;                  // a missing member reads record 0 and is masked out
-    const i64 x = D.t_enter[ix], y = D.t_exit[ix];
-    u64 by = D.bytes[ix]; u32 ch = 0; u8 op = D.op[ix], st = 0;
-    if (D.send_chg != nullptr) { const u32 sc = D.send_chg[ix], rc = D.recv_chg[ix]; ch = sc > rc ? sc : rc; }
-    u64 te = 0, du = 0;
-    if (idx != NONE) {
-      st = 1 | (y == -1 ? 2 : ((x < 0 || y < x) ? 4 : 0));
-      te = (u64)x; du = (u64)(y - x);
-    } else { by = 0; ch = 0; op = 0; }
-    s_te[a] = te; s_du[a] = du; s_by[a] = by; s_ch[a] = ch; s_op[a] = op; s_st[a] = st;
+  // 1. gather: a warp walks consecutive op counters of one member (its slice of perm is contiguous)
+  {
+    const bool have_rates = D.send_chg != nullptr;
+    for (u32 p = threadIdx.x >> 5; p < n; p += MID_THREADS / 32) {
+      const u32* __restrict__ pm = D.perm + perm_at(row, t.seq_off, p);
+      for (u32 jg = threadIdx.x & 31; jg < S; jg += 32) {
+        const u32 a = jg * pitch + p;
+        const u32 idx = pm[jg];
+        const u32 ix = idx == NONE ? 0u : idx;                  // a missing member reads record 0 and is masked out
+        const i64 x = D.t_enter[ix], y = D.t_exit[ix];
+        u64 by = D.bytes[ix]; u32 ch = 0; u8 op = D.op[ix], st = 0;
+        if (have_rates) { const u32 sc = D.send_chg[ix], rc = D.recv_chg[ix]; ch = sc > rc ? sc : rc; }
+        u64 te = 0, du = 0;
+        if (idx != NONE) {
+          st = 1 | (y == -1 ? 2 : ((x < 0 || y < x) ? 4 : 0));
+          te = (u64)x; du = (u64)(y - x);
+        } else { by = 0; ch = 0; op = 0; }
+        s_te[a] = te; s_du[a] = du; s_by[a] = by; s_ch[a] = ch; s_op[a] = op; s_st[a] = st;
+      }
+    }
   }
   __syncthreads();
   // 3. one warp per group, end to end
@@ -1349,7 +1348,7 @@ __device__ __forceinline__ void reduce_warp_cta(const WinDesc& D, const FusedCta
           if (dq) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p] * 4 + (dh ? 2 : 3)], 1u); }
         }
         D.flags[slot_t + (u64)jg * n + p] = f;
-        if (add_bw) bwacc[r] += busbw(bn, den, (i64)s_du[b + p]);
+        if (add_bw) bwacc[r] += busbw_fast(bn, den, (i64)s_du[b + p]);
       }
     }
     if (lane == 0) {
@@ -1365,7 +1364,7 @@ __device__ __forceinline__ void reduce_warp_cta(const WinDesc& D, const FusedCta
       D.gu32[(u64)GU_MAX_CHG * G + g] = complete ? (u32)(chk >> 32) : 0;
       D.gu32[(u64)GU_RANK_MAX_CHG * G + g] = complete ? mem[NONE - (u32)chk] : 0;
       D.gu32[(u64)GU_N_PRESENT * G + g] = npres; D.gu32[(u64)GU_GFLAGS * G + g] = gfl;
-      D.gbw[g] = complete ? busbw(bn, den, span) : 0.0;
+      D.gbw[g] = complete ? busbw_fast(bn, den, span) : 0.0;
       c_comp += complete; c_inc += !complete; c_bar += barrier; c_an += analysed; c_mis += mism; c_pres += npres;
       if (add_bw) best_merge(w_brng, w_bk, tmax - tmin, t.seq_off + jg);
     }
