@@ -81,8 +81,10 @@ enum { T_GROUPS = 0, T_SLOTS, T_FCTA, T_FWT, T_FSUM, T_TILES2, T_TILES3, T_ROWS,
 enum { B_FCTA = 0, B_FWT, B_FSUM, B_T2, B_T3, B_COUNT };
 
 struct Tile { u32 w, c, seq_off, count; };                 // classes 2 and 3: one CTA each; summary index = tile index
-struct WarpTile { u32 c, seq_off, count, sum_idx; };      // class 0: up to 32 consecutive op counters of one communicator
-struct FusedCta { u32 w, cls, c, seq_off, count, sum_idx, wt_first, wt_count; };   // class 0: wt_*; class 1: c .. sum_idx
+// Work-list entries of the fused kernel carry a copy of the communicator's range row and member-list offset, so that a
+// tile needs no further lookups before its first gather.
+struct WarpTile { u32 c, seq_off, count, sum_idx; RangeRow row; u64 moff; };      // class 0: up to 32 consecutive op counters of one communicator
+struct FusedCta { u32 w, cls, c, seq_off, count, sum_idx, wt_first, wt_count; RangeRow row; u64 moff; };   // class 0: wt_*; class 1: c .. sum_idx, row, moff
 
 // What a tile contributes to its communicator's window decision (Eq. 2 and the round counts).
 struct TileSum { u64 best_rng; u32 best_k, n_rounds, n_an, pad; };   // best_k: op-counter offset in the range, NONE if no round

@@ -422,18 +422,20 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
       uint2 tot; const uint2 ex = plan_scan2(make_uint2(cls == 0 ? u : 0, cls == 1 ? u : 0), &tot, s_pair);
       if (u) {
         const u32 S = chunk_len(ns, T), U = tile_seqs(n), cnt = chunk_size(ns, T, tau);
-        const u32 sum0 = D.ranges[c].tile0 + tau * ceil_div(S, U);
+        const RangeRow crow = D.ranges[c]; const u64 cmoff = R.comm_moff[c];
+        const u32 sum0 = crow.tile0 + tau * ceil_div(S, U);
         for (u32 k = 0; k < u; ++k) {
           const u32 off = tau * S + k * U, len = cnt - k * U < U ? cnt - k * U : U;
-          if (cls == 0) { WarpTile x; x.c = c; x.seq_off = off; x.count = len; x.sum_idx = sum0 + k; L.fwt[wt_base + wt_run + ex.x + k] = x; }
+          if (cls == 0) { WarpTile x; x.c = c; x.seq_off = off; x.count = len; x.sum_idx = sum0 + k; x.row = crow; x.moff = cmoff; L.fwt[wt_base + wt_run + ex.x + k] = x; }
           else { FusedCta x; x.w = blockIdx.x; x.cls = 1; x.c = c; x.seq_off = off; x.count = len; x.sum_idx = sum0 + k; x.wt_first = 0; x.wt_count = 0;
-                 L.fcta[cta_base + n0 + c1_run + ex.y + k] = x; }
+                 x.row = crow; x.moff = cmoff; L.fcta[cta_base + n0 + c1_run + ex.y + k] = x; }
         }
       }
       wt_run += tot.x; c1_run += tot.y;
     }
     for (u32 j = threadIdx.x; j < n0; j += PLAN_THREADS) {
-      FusedCta x; x.w = blockIdx.x; x.cls = 0; x.c = 0; x.seq_off = 0; x.count = 0; x.sum_idx = 0;
+      FusedCta x; x.w = blockIdx.x; x.cls = 0; x.c = 0; x.seq_off = 0; x.count = 0; x.sum_idx = 0; x.moff = 0;
+      x.row = RangeRow{0, 0, 0, 0, 0, 0, 0, 0};
       x.wt_first = wt_base + 8 * j; x.wt_count = wt_total - 8 * j < 8 ? wt_total - 8 * j : 8;
       L.fcta[cta_base + j] = x;
     }
@@ -643,8 +645,8 @@ __device__ __forceinline__ void reduce_small_warp(const WinDesc& D, const WarpTi
                                                   i64 now, u32 n_rt, double (*s_bw)[SMALL_N], u32* s_rounds, u32* s_cnt) {
   const u32 n = FULL ? (u32)SMALL_N : n_rt;
   const u32 c = t.c;
-  const RangeRow row = D.ranges[c];
-  const u32* mem = R.members + R.comm_moff[c];
+  const RangeRow& row = t.row;
+  const u32* mem = R.members + t.moff;
   const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5, j = lane;
   const bool active = j < t.count;
   const u32 k_milli = P.k_milli;
@@ -714,7 +716,6 @@ __device__ __forceinline__ void reduce_small_warp(const WinDesc& D, const WarpTi
         }
       }
     }
-    asm volatile("" ::: "memory");                           // keep the second batch behind the first
     u64 gbytes = 0; u32 gop = 0; bool have_first = false;
     u32 max_chg = 0, pos_chg = 0; bool have_chg = false;
     {
@@ -856,7 +857,7 @@ __device__ __forceinline__ void reduce_small_cta(const WinDesc& D, const FusedCt
   __syncthreads();
   if (wid < t.wt_count) {
     const WarpTile wt = wts[t.wt_first + wid];
-    const u32 n = R.comm_n[wt.c];
+    const u32 n = wt.row.n;
     if ((threadIdx.x & 31) == 0) s_comm[wid] = wt.c;
     if (n == SMALL_N) reduce_small_warp<true>(D, wt, sums, R, P, now, n, s_bw, s_rounds, s_cnt);
     else reduce_small_warp<false>(D, wt, sums, R, P, now, n, s_bw, s_rounds, s_cnt);
@@ -1228,9 +1229,9 @@ inline size_t warp_smem_bytes() {
 // Class-1 CTA of the fused kernel: one tile of S groups of one communicator.
 __device__ __forceinline__ void reduce_warp_cta(const WinDesc& D, const FusedCta& t, TileSum* __restrict__ sums, const Registry& R, const Params& P,
                                                 i64 now, unsigned char* smem_raw) {
-  const u32 c = t.c, n = R.comm_n[c];
-  const RangeRow row = D.ranges[c];
-  const u32* mem = R.members + R.comm_moff[c];
+  const u32 c = t.c, n = t.row.n;
+  const RangeRow& row = t.row;
+  const u32* mem = R.members + t.moff;
   const u32 n_pad = mid_npad(n), pitch = n_pad + 1, S = t.count, S_max = MID_ELEMS / n_pad;
   const u32 cap = S_max * pitch;
   u64* s_te = (u64*)smem_raw;            // enter time
@@ -1248,24 +1249,38 @@ __device__ __forceinline__ void reduce_warp_cta(const WinDesc& D, const FusedCta
   const u64 g_t = row.group0 + t.seq_off;
   const u32 n_el = S * n;
   if (threadIdx.x < 8) s_cnt[threadIdx.x] = 0;
-  // 1. gather: a warp walks consecutive op counters of one member (its slice of perm is contiguous)
+  // 1. gather: a warp walks consecutive op counters of one member (its slice of perm is contiguous); four members
+  //    are in flight per lane so that the two dependent loads (index, then record) overlap across members
   {
     const bool have_rates = D.send_chg != nullptr;
-    for (u32 p = threadIdx.x >> 5; p < n; p += MID_THREADS / 32) {
-      const u32* __restrict__ pm = D.perm + perm_at(row, t.seq_off, p);
-      for (u32 jg = threadIdx.x & 31; jg < S; jg += 32) {
-        const u32 a = jg * pitch + p;
-        const u32 idx = pm[jg];
-        const u32 ix = idx == NONE ? 0u : idx;                  // a missing member reads record 0 and is masked out
-        const i64 x = D.t_enter[ix], y = D.t_exit[ix];
-        u64 by = D.bytes[ix]; u32 ch = 0; u8 op = D.op[ix], st = 0;
-        if (have_rates) { const u32 sc = D.send_chg[ix], rc = D.recv_chg[ix]; ch = sc > rc ? sc : rc; }
-        u64 te = 0, du = 0;
-        if (idx != NONE) {
-          st = 1 | (y == -1 ? 2 : ((x < 0 || y < x) ? 4 : 0));
-          te = (u64)x; du = (u64)(y - x);
-        } else { by = 0; ch = 0; op = 0; }
-        s_te[a] = te; s_du[a] = du; s_by[a] = by; s_ch[a] = ch; s_op[a] = op; s_st[a] = st;
+    constexpr int GU = 4;
+    const u32 lane_g = threadIdx.x & 31, wid_g = threadIdx.x >> 5;
+    const i64* __restrict__ c_te = D.t_enter; const i64* __restrict__ c_tx = D.t_exit; const u64* __restrict__ c_by = D.bytes;
+    const u8* __restrict__ c_op = D.op; const u32* __restrict__ c_sc = D.send_chg; const u32* __restrict__ c_rc = D.recv_chg;
+    const u32* __restrict__ pm0 = D.perm + perm_at(row, t.seq_off, 0);
+    for (u32 pb = wid_g; pb < n; pb += (MID_THREADS / 32) * GU) {
+      for (u32 jg = lane_g; jg < S; jg += 32) {
+        u32 idx[GU];
+#pragma unroll
+        for (int u = 0; u < GU; ++u) { const u32 p = pb + u * (MID_THREADS / 32); idx[u] = p < n ? pm0[(u64)p * row.n_seq + jg] : NONE; }
+        i64 x[GU], y[GU]; u64 by[GU]; u32 ch[GU], op[GU];
+#pragma unroll
+        for (int u = 0; u < GU; ++u) {
+          const u32 ix = idx[u] == NONE ? 0u : idx[u];          // a missing member reads record 0 and is masked out
+          x[u] = c_te[ix]; y[u] = c_tx[ix]; by[u] = c_by[ix]; op[u] = c_op[ix]; ch[u] = 0;
+          if (have_rates) { const u32 sc = c_sc[ix], rc = c_rc[ix]; ch[u] = sc > rc ? sc : rc; }
+        }
+#pragma unroll
+        for (int u = 0; u < GU; ++u) {
+          const u32 p = pb + u * (MID_THREADS / 32);
+          if (p < n) {
+            const u32 a = jg * pitch + p;
+            const bool have = idx[u] != NONE;
+            const u8 st = have ? (u8)(1 | (y[u] == -1 ? 2 : ((x[u] < 0 || y[u] < x[u]) ? 4 : 0))) : (u8)0;
+            s_te[a] = have ? (u64)x[u] : 0; s_du[a] = have ? (u64)(y[u] - x[u]) : 0; s_by[a] = have ? by[u] : 0;
+            s_ch[a] = have ? ch[u] : 0; s_op[a] = have ? (u8)op[u] : (u8)0; s_st[a] = st;
+          }
+        }
       }
     }
   }
