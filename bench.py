@@ -28,6 +28,10 @@ UNIT = "records/s"
 REC_BYTES = 45            # 3 x u32 keys, u8 op, u64 bytes, 2 x i64 times, 2 x u32 rate columns
 ROW_BYTES = 104           # one per-op row
 HBM_FALLBACK_GBS = 6650.0
+# DRAM traffic per record (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture divided by the records of the
+# captured launch; 5-window case, 20.48 M records, see profiles/). Traffic grows in proportion to the records, so a
+# launch's traffic is this figure times its records. Set an entry to None whenever its kernel changes.
+NCU_TRAFFIC_PER_RECORD = {"k_reduce_fused": (782.503424e6 + 228.286208e6) / 20.48e6}
 
 
 def parse():
@@ -246,8 +250,10 @@ def run_ours(args, rank, world, local_rank):
     achieved = d_bytes / (d_ms * 1e-3) / 1e9 if d_ms > 0 else 0.0
     path_bytes = REC_BYTES * n_rec + n_rec + ROW_BYTES * NW * sum(u[1] for u in units.values())
     path_gbs = path_bytes * args.steps / (ms * 1e-3) / 1e9
+    tpr = NCU_TRAFFIC_PER_RECORD.get(dom)
+    traffic = tpr * n_rec if tpr is not None else None
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "peak_source": peak_kind, "ms_per_launch": d_ms, "algorithmic_bytes_per_launch": d_bytes,
+                "traffic": traffic, "peak_source": peak_kind, "ms_per_launch": d_ms, "algorithmic_bytes_per_launch": d_bytes,
                 "kernels_ms_per_step": {k: kt[k]["ms"] / args.steps for k in kt},
                 "whole_path": {"algorithmic_bytes_per_step": path_bytes, "achieved": path_gbs, "frac": path_gbs / peak}}
     launches = sum(x["launches"] for x in kt.values())
