@@ -251,7 +251,7 @@ def run_ours(args, rank, world, local_rank):
     path_bytes = REC_BYTES * n_rec + n_rec + ROW_BYTES * NW * sum(u[1] for u in units.values())
     path_gbs = path_bytes * args.steps / (ms * 1e-3) / 1e9
     tpr = NCU_TRAFFIC_PER_RECORD.get(dom)
-    traffic = tpr * n_rec if tpr is not None else None
+    traffic = tpr * NW * (units["small"][0] + units["warp"][0]) if tpr is not None else None   # records of the kernel's classes
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": traffic, "peak_source": peak_kind, "ms_per_launch": d_ms, "algorithmic_bytes_per_launch": d_bytes,
                 "kernels_ms_per_step": {k: kt[k]["ms"] / args.steps for k in kt},
