@@ -221,7 +221,6 @@ int finalize_registry(ccld_ctx* ctx) {
   ctx->misc_blk = ctx->pool.get(misc_layout(nr, max_n).total, &e);
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "scratch allocation failed");
 
-  CK(cudaFuncSetAttribute(k_reduce_fused, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)warp_smem_bytes()));
   CK(cudaFuncSetAttribute(k_reduce_mid, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mid_smem_bytes(2 * WARP_N)));
   if (max_large) CK(cudaFuncSetAttribute(k_reduce_large, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(16ull * max_large)));
   ctx->finalized = true;
@@ -465,7 +464,7 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   PlanLists pl; pl.fcta = (FusedCta*)(rbase + o_fcta); pl.fwt = (WarpTile*)(rbase + o_fwt); pl.t2 = (Tile*)(rbase + o_t2); pl.t3 = (Tile*)(rbase + o_t3);
   { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, pl, 1); }
   if (cta > 0) { TimedLaunch tl(ts, 2, st); k_slot_scatter<<<(u32)cta, SCAT_THREADS, 0, st>>>(d_desc, B, ctx->reg); }
-  if (n_list[B_FCTA]) { TimedLaunch tl(ts, 3, st); k_reduce_fused<<<(u32)n_list[B_FCTA], SMALL_SEQS, warp_smem_bytes(), st>>>(d_desc, pl.fcta, pl.fwt, (TileSum*)(rbase + o_fsum), ctx->reg, ctx->dp, now_ns); }
+  if (n_list[B_FCTA]) { TimedLaunch tl(ts, 3, st); k_reduce_fused<<<(u32)n_list[B_FCTA], SMALL_SEQS, 0, st>>>(d_desc, pl.fcta, pl.fwt, (TileSum*)(rbase + o_fsum), ctx->reg, ctx->dp, now_ns); }
   if (n_list[B_T2]) { TimedLaunch tl(ts, 4, st); k_reduce_mid<<<(u32)n_list[B_T2], MID_THREADS, mid_smem_bytes(2 * WARP_N), st>>>(d_desc, pl.t2, (TileSum*)(rbase + o_s2), ctx->reg, ctx->dp, now_ns); }
   if (n_list[B_T3]) { TimedLaunch tl(ts, 5, st); k_reduce_large<<<(u32)n_list[B_T3], LARGE_THREADS, 16ull * ctx->max_large_n, st>>>(d_desc, pl.t3, (TileSum*)(rbase + o_s3), ctx->reg, ctx->dp, now_ns); }
   { TimedLaunch tl(ts, 6, st); k_window_decide<<<(nc + 3) / 4, 128, 0, st>>>(d_desc, B, ctx->reg, ctx->dp); }

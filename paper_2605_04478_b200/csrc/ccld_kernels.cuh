@@ -1145,274 +1145,367 @@ inline size_t mid_smem_bytes(u32 n_pad_min) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// per-op reductions, 9 <= n <= 128: a tile of S groups is staged in shared memory as in k_reduce_mid,
-// then one warp owns a group end to end: cross-rank reductions by shuffles, order statistics by a
-// bitonic network over E = n_pad / 32 registers per lane (32-bit keys whenever the group's value
-// range fits), flags straight to global memory. No block-wide barrier inside the sort.
+// per-op reductions, 9 <= n <= 128: L = n_pad / 8 lanes per group, eight ring positions per lane
+// (lane s of a group holds positions 8 s .. 8 s + 7), 32 / L consecutive op counters per warp. Each
+// lane gathers, reduces and sorts its eight values in registers exactly like the n <= 8 path; the
+// lanes of a group meet through xor shuffles: log2 L rounds for the extrema, and a merge network
+// whose cross-lane steps move eight independent keys each. 32-bit keys whenever the group's value
+// range fits; other groups go through an out-of-line 64-bit routine. No shared-memory staging.
 // ------------------------------------------------------------------------------------------------
-
-// Element i = r * 32 + lane of the warp's 32 E keys. Full sort, or (MERGE) the last merge phase only,
-// which sorts a sequence that falls and then rises.
-template <int E, class K, bool MERGE>
-__device__ __forceinline__ void warp_bitonic(K (&v)[E], u32 lane) {
-  constexpr int NP = 32 * E;
-#pragma unroll
-  for (int k = MERGE ? NP : 2; k <= NP; k <<= 1) {
-#pragma unroll
-    for (int j = k >> 1; j > 0; j >>= 1) {
-      if (j >= 32) {
-        const int dr = j >> 5;
-#pragma unroll
-        for (int r = 0; r < E; ++r) {
-          if ((r & dr) == 0) {
-            const int r2 = r | dr;
-            const bool up = k == NP || (((r * 32) & k) == 0);
-            const K a = v[r], b = v[r2];
-            const K lo = a < b ? a : b, hi = a < b ? b : a;
-            v[r] = up ? lo : hi; v[r2] = up ? hi : lo;
-          }
-        }
-      } else {
-        const bool lower = (lane & j) == 0;
-#pragma unroll
-        for (int r = 0; r < E; ++r) {
-          const K o = __shfl_xor_sync(0xFFFFFFFFu, v[r], j);
-          const bool up = k == NP || (((r * 32 + lane) & k) == 0);
-          const K lo = v[r] < o ? v[r] : o, hi = v[r] < o ? o : v[r];
-          v[r] = (lower == up) ? lo : hi;
-        }
-      }
-    }
-  }
-}
-
-template <int E, class K>
-__device__ __forceinline__ K warp_pick(const K (&v)[E], u32 idx) {
+template <class K> __device__ __forceinline__ K pick8(const K (&v)[8], u32 r) {
   K x = v[0];
 #pragma unroll
-  for (int r = 1; r < E; ++r) x = (idx >> 5) == (u32)r ? v[r] : x;
-  return __shfl_sync(0xFFFFFFFFu, x, idx & 31);
+  for (int i = 1; i < 8; ++i) x = r == (u32)i ? v[i] : x;
+  return x;
 }
 
-// lower median and lower-median absolute deviation of key(p), p < n <= 32 E
-template <int E, class K, class F>
-__device__ __forceinline__ void warp_median_mad(F key, u32 n, u32 lane, K* med, K* mad) {
-  K v[E];
+// One cross-lane step of a merge network: element r of this lane against element r (MIRROR: 7 - r) of lane ^ mask;
+// the lane with keep_low set keeps the smaller key of each pair.
+template <class K, bool MIRROR>
+__device__ __forceinline__ void sub_exchange(K (&v)[8], int mask, bool keep_low) {
+  K o[8];
 #pragma unroll
-  for (int r = 0; r < E; ++r) { const u32 p = r * 32 + lane; v[r] = p < n ? key(p) : KeyMax<K>::v(); }
-  warp_bitonic<E, K, false>(v, lane);
-  const u32 k = (n - 1) >> 1;
-  const K m = warp_pick<E, K>(v, k);
+  for (int r = 0; r < 8; ++r) o[r] = __shfl_xor_sync(0xFFFFFFFFu, v[MIRROR ? 7 - r : r], mask);
 #pragma unroll
-  for (int r = 0; r < E; ++r) { const u32 p = r * 32 + lane; v[r] = p < n ? (v[r] >= m ? v[r] - m : m - v[r]) : KeyMax<K>::v(); }
-  warp_bitonic<E, K, true>(v, lane);
-  *med = m; *mad = warp_pick<E, K>(v, k);
+  for (int r = 0; r < 8; ++r) { const bool lt = v[r] < o[r]; v[r] = (lt == keep_low) ? v[r] : o[r]; }
 }
 
-template <int E>
-__device__ __forceinline__ void warp_group_stats(const u64* te, const u64* du, u32 n, u32 lane, u64 e_min, u64 askew, u64 tmin, u64 tmax,
-                                                 u64* med_s, u64* mad_s, u64* med_d, u64* mad_d) {
-  if (askew < 0xFFFFFFFFull) { u32 m, d; warp_median_mad<E, u32>([&](u32 p) { return (u32)(te[p] - e_min); }, n, lane, &m, &d); *med_s = m; *mad_s = d; }
-  else { u64 m, d; warp_median_mad<E, u64>([&](u32 p) { return te[p] - e_min; }, n, lane, &m, &d); *med_s = m; *mad_s = d; }
-  if (tmax - tmin < 0xFFFFFFFFull) { u32 m, d; warp_median_mad<E, u32>([&](u32 p) { return (u32)(du[p] - tmin); }, n, lane, &m, &d); *med_d = tmin + m; *mad_d = d; }
-  else { u64 m, d; warp_median_mad<E, u64>([&](u32 p) { return du[p] - tmin; }, n, lane, &m, &d); *med_d = tmin + m; *mad_d = d; }
+// Sorts the 8 L keys of a group ascending; element i lives in lane i / 8 (of the group), register i % 8.
+template <int L, class K>
+__device__ __forceinline__ void sub_sort(K (&v)[8], u32 s) {
+  sort8(v);
+#pragma unroll
+  for (int m = 1; m < L; m <<= 1) {
+    // two ascending runs of m lanes each: the mirror step leaves every key of the low run <= every key of the high
+    // run and both runs bitonic; half-cleaners across lanes and then inside the lane finish the merge
+    sub_exchange<K, true>(v, 2 * m - 1, (s & m) == 0);
+#pragma unroll
+    for (int h = m >> 1; h >= 1; h >>= 1) sub_exchange<K, false>(v, h, (s & h) == 0);
+    merge8(v);
+  }
+}
+// Sorts 8 L keys that fall and then rise.
+template <int L, class K>
+__device__ __forceinline__ void sub_merge(K (&v)[8], u32 s) {
+#pragma unroll
+  for (int h = L >> 1; h >= 1; h >>= 1) sub_exchange<K, false>(v, h, (s & h) == 0);
+  merge8(v);
 }
 
-constexpr int WARP_EMAX = WARP_N / 32;
-
-inline size_t warp_smem_bytes() {
-  // cap = (MID_ELEMS / n_pad) * (n_pad + 1) is largest for n_pad = 32
-  const size_t cap = (size_t)(MID_ELEMS / 32) * 33;
-  return cap * (3 * 8 + 4 + 2) + 16 + (MID_THREADS / 32) * WARP_N * sizeof(double);
+// Lower median and lower-median absolute deviation of a group's keys (x[q] = maximum key where the position does
+// not exist or the group is not sorted at all). Every lane of the warp must call it.
+template <int L, class K>
+__device__ __forceinline__ void sub_median_mad(const K (&x)[8], u32 n, u32 s, u32 lane, K* med, K* mad) {
+  K v[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) v[q] = x[q];
+  sub_sort<L, K>(v, s);
+  const u32 k = (n - 1) >> 1, src = (lane & ~(u32)(L - 1)) | (k >> 3);
+  const K m = __shfl_sync(0xFFFFFFFFu, pick8(v, k & 7), src);
+#pragma unroll
+  for (int r = 0; r < 8; ++r) v[r] = s * 8 + r < n ? (v[r] >= m ? v[r] - m : m - v[r]) : KeyMax<K>::v();   // falls to 0 at k, then rises
+  sub_merge<L, K>(v, s);
+  *med = m; *mad = __shfl_sync(0xFFFFFFFFu, pick8(v, k & 7), src);
 }
 
-// Class-1 CTA of the fused kernel: one tile of S groups of one communicator.
-__device__ __forceinline__ void reduce_warp_cta(const WinDesc& D, const FusedCta& t, TileSum* __restrict__ sums, const Registry& R, const Params& P,
-                                                i64 now, unsigned char* smem_raw) {
-  const u32 c = t.c, n = t.row.n;
+// Groups whose skews or durations do not fit 32-bit keys: the whole warp comes here (shuffles), lanes with `mine`
+// set gather their times again and get the order statistics and flag bytes of their group in 64 bits; their
+// members' bus bandwidths are added straight to the per-rank sums.
+template <int L>
+__device__ __noinline__ void sub_group64(const WinDesc& D, const Registry& R, const u32* mem, u64 pslot, u32 pstride, u32 n, u32 s, u32 lane, bool mine,
+                                         u64 e_min, u32 k_milli, bool analysed, bool add_bw, double bn, double den, u64* out4, u64* packed_io) {
+  u64 sk[8], du[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    sk[q] = U64_MAX_; du[q] = U64_MAX_;
+    if (mine && s * 8 + q < n) { const u32 idx = D.perm[pslot + (u64)q * pstride]; const i64 a = D.t_enter[idx], b = D.t_exit[idx]; sk[q] = (u64)a - e_min; du[q] = (u64)(b - a); }
+  }
+  if (mine && add_bw)
+    for (u32 q = 0; q < 8 && s * 8 + q < n; ++q) atomicAdd(&R.bw_sum[mem[s * 8 + q]], busbw_fast(bn, den, (i64)du[q]));
+  u64 med_s, mad_s, med_d, mad_d;
+  sub_median_mad<L, u64>(sk, n, s, lane, &med_s, &mad_s);
+  sub_median_mad<L, u64>(du, n, s, lane, &med_d, &mad_d);
+  if (mine && analysed) {
+    out4[0] = med_s; out4[1] = mad_s; out4[2] = med_d; out4[3] = mad_d;
+    u64 packed = 0;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      if (s * 8 + q < n) {
+        const bool so = mul_gt(absdiff(sk[q], med_s), 1000u, mad_s, k_milli), sh = sk[q] > med_s;
+        const bool dq = mul_gt(absdiff(du[q], med_d), 1000u, mad_d, k_milli), dh = du[q] > med_d;
+        packed |= (u64)((so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0)) << (8 * q);
+      }
+    }
+    *packed_io = packed;
+  }
+}
+
+struct SubShared {
+  double bw[MID_THREADS / 32][WARP_N];
+  u64 brng[MID_THREADS / 32];
+  u32 bk[MID_THREADS / 32], rounds[MID_THREADS / 32], n_an[MID_THREADS / 32];
+  u32 cnt[SC_COUNT];
+};
+
+// One warp: 32 / L consecutive op counters of the tile, L lanes each.
+template <int L>
+__device__ __forceinline__ void reduce_sub_warp(const WinDesc& D, const FusedCta& t, const Registry& R, const Params& P, i64 now, SubShared& sh) {
+  constexpr int GW = 32 / L;                                  // groups per warp
+  constexpr u32 FULLM = 0xFFFFFFFFu;
   const RangeRow& row = t.row;
+  const u32 n = row.n, c = t.c;
   const u32* mem = R.members + t.moff;
-  const u32 n_pad = mid_npad(n), pitch = n_pad + 1, S = t.count, S_max = MID_ELEMS / n_pad;
-  const u32 cap = S_max * pitch;
-  u64* s_te = (u64*)smem_raw;            // enter time
-  u64* s_du = s_te + cap;                // duration
-  u64* s_by = s_du + cap;                // bytes
-  u32* s_ch = (u32*)(s_by + cap);        // max(send_chg, recv_chg)
-  u8* s_op = (u8*)(s_ch + cap);
-  u8* s_st = s_op + cap;                 // 1 present, 2 in flight, 4 bad time
-  double* s_bw = (double*)(((uintptr_t)(s_st + cap) + 15) & ~(uintptr_t)15);   // [warps][n_pad]
-  __shared__ u32 s_cnt[8];
-  __shared__ u64 s_brng[MID_THREADS / 32];
-  __shared__ u32 s_bk[MID_THREADS / 32], s_rounds[MID_THREADS / 32];
-
-  const u64 slot_t = row.slot0 + (u64)t.seq_off * n;
-  const u64 g_t = row.group0 + t.seq_off;
-  const u32 n_el = S * n;
-  if (threadIdx.x < 8) s_cnt[threadIdx.x] = 0;
-  // 1. gather: a warp walks consecutive op counters of one member (its slice of perm is contiguous); four members
-  //    are in flight per lane so that the two dependent loads (index, then record) overlap across members
-  {
-    const bool have_rates = D.send_chg != nullptr;
-    constexpr int GU = 4;
-    const u32 lane_g = threadIdx.x & 31, wid_g = threadIdx.x >> 5;
-    const i64* __restrict__ c_te = D.t_enter; const i64* __restrict__ c_tx = D.t_exit; const u64* __restrict__ c_by = D.bytes;
-    const u8* __restrict__ c_op = D.op; const u32* __restrict__ c_sc = D.send_chg; const u32* __restrict__ c_rc = D.recv_chg;
-    const u32* __restrict__ pm0 = D.perm + perm_at(row, t.seq_off, 0);
-    for (u32 pb = wid_g; pb < n; pb += (MID_THREADS / 32) * GU) {
-      for (u32 jg = lane_g; jg < S; jg += 32) {
-        u32 idx[GU];
-#pragma unroll
-        for (int u = 0; u < GU; ++u) { const u32 p = pb + u * (MID_THREADS / 32); idx[u] = p < n ? pm0[(u64)p * row.n_seq + jg] : NONE; }
-        i64 x[GU], y[GU]; u64 by[GU]; u32 ch[GU], op[GU];
-#pragma unroll
-        for (int u = 0; u < GU; ++u) {
-          const u32 ix = idx[u] == NONE ? 0u : idx[u];          // a missing member reads record 0 and is masked out
-          x[u] = c_te[ix]; y[u] = c_tx[ix]; by[u] = c_by[ix]; op[u] = c_op[ix]; ch[u] = 0;
-          if (have_rates) { const u32 sc = c_sc[ix], rc = c_rc[ix]; ch[u] = sc > rc ? sc : rc; }
-        }
-#pragma unroll
-        for (int u = 0; u < GU; ++u) {
-          const u32 p = pb + u * (MID_THREADS / 32);
-          if (p < n) {
-            const u32 a = jg * pitch + p;
-            const bool have = idx[u] != NONE;
-            const u8 st = have ? (u8)(1 | (y[u] == -1 ? 2 : ((x[u] < 0 || y[u] < x[u]) ? 4 : 0))) : (u8)0;
-            s_te[a] = have ? (u64)x[u] : 0; s_du[a] = have ? (u64)(y[u] - x[u]) : 0; s_by[a] = have ? by[u] : 0;
-            s_ch[a] = have ? ch[u] : 0; s_op[a] = have ? (u8)op[u] : (u8)0; s_st[a] = st;
-          }
-        }
-      }
-    }
-  }
-  __syncthreads();
-  // 3. one warp per group, end to end
   const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const u32 s = lane % L, j = wid * GW + lane / L, p0 = s * 8;
+  const bool active = j < t.count, lead = active && s == 0;
+  const u32 gmask = ((1u << L) - 1u) << (lane & ~(u32)(L - 1));   // the lanes of my group
   const u32 k_milli = P.k_milli;
-  u32 c_comp = 0, c_inc = 0, c_bar = 0, c_an = 0, c_mis = 0, c_pres = 0, n_fs = 0, n_fd = 0, n_bwc = 0;
-  u64 w_brng = 0; u32 w_bk = NONE;
-  double bwacc[WARP_EMAX];
+
+  // ---- batch 0: record indices of my eight positions (member-major permutation: stride n_seq) ----
+  u32 idx[8];
+  const u64 pslot = perm_at(row, t.seq_off + (active ? j : 0u), p0);
+  {
+    const u32* __restrict__ pm = D.perm + pslot;
 #pragma unroll
-  for (int r = 0; r < WARP_EMAX; ++r) bwacc[r] = 0.0;
-  for (u32 jg = wid; jg < S; jg += MID_THREADS / 32) {
-    const u32 b = jg * pitch;
-    u32 npres = 0, first = NONE, stor = 0;
-    for (u32 p = lane; p < n; p += 32) { const u32 st = s_st[b + p]; if (st & 1) { ++npres; first = first == NONE ? p : first; } stor |= st; }
-    npres = __reduce_add_sync(0xFFFFFFFFu, npres); first = __reduce_min_sync(0xFFFFFFFFu, first); stor = __reduce_or_sync(0xFFFFFFFFu, stor);
-    const bool have_first = first != NONE;
-    const u64 gbytes = have_first ? s_by[b + first] : 0; const u32 gop = have_first ? s_op[b + first] : 0;
-    const bool inflight = stor & 2, bad_time = stor & 4, complete = npres == n && !inflight && !bad_time;
-    const bool barrier = have_first && gop == CCLD_OP_ALLREDUCE && gbytes < P.barrier_bytes;
-    u32 mism = 0; i64 age = -1;
-    u64 e_min = U64_MAX_, e_max = 0, tmax = 0, tmin = U64_MAX_; i64 x_max = INT64_MIN; u32 pmax = NONE, pmin = NONE; u64 chk = 0;
-    for (u32 p = lane; p < n; p += 32) {
-      const u32 st = s_st[b + p];
-      if (!(st & 1)) continue;
-      if (s_op[b + p] != gop || s_by[b + p] != gbytes) mism = 1;
-      const u64 te = s_te[b + p], du = s_du[b + p];
-      if (st & 2) { const i64 ag = now - (i64)te; age = ag > age ? ag : age; }
-      e_min = te < e_min ? te : e_min; e_max = te > e_max ? te : e_max;
-      const i64 tx = (i64)(te + du); x_max = tx > x_max ? tx : x_max;
-      if (pmax == NONE || du > tmax) { tmax = du; pmax = p; }
-      if (pmin == NONE || du < tmin) { tmin = du; pmin = p; }
-      const u64 ck = ((u64)s_ch[b + p] << 32) | (u64)(NONE - p);        // most changes, then lowest position
-      chk = ck > chk ? ck : chk;
-    }
-    mism = __reduce_or_sync(0xFFFFFFFFu, mism);
+    for (int q = 0; q < 8; ++q) idx[q] = (active && p0 + q < n) ? pm[(u64)q * row.n_seq] : NONE;
+  }
+  // ---- batch 1: times (a missing member reads record 0 and is masked out) ----
+  u32 npres = 0, miss = 0, stb = 0;                           // stb: 1 in flight, 2 bad time
+  i64 x_max = INT64_MIN, age = -1;
+  u64 e_min = U64_MAX_, e_max = 0, tmax = 0, tmin = U64_MAX_; u32 pmax = NONE, pmin = NONE;
+  i64 ld_a[8], ld_b[8];
+  {
+    const i64* __restrict__ c_te = D.t_enter; const i64* __restrict__ c_tx = D.t_exit;
 #pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
-      const i64 ag = (i64)shfl_xor64((u64)age, d); age = ag > age ? ag : age;
-      const u64 em = shfl_xor64(e_min, d); e_min = em < e_min ? em : e_min;
-      const u64 eM = shfl_xor64(e_max, d); e_max = eM > e_max ? eM : e_max;
-      const i64 xm = (i64)shfl_xor64((u64)x_max, d); x_max = xm > x_max ? xm : x_max;
-      const u64 ck = shfl_xor64(chk, d); chk = ck > chk ? ck : chk;
-      const u64 tM = shfl_xor64(tmax, d); const u32 pM = __shfl_xor_sync(0xFFFFFFFFu, pmax, d);
-      if (pM != NONE && (pmax == NONE || tM > tmax || (tM == tmax && pM < pmax))) { tmax = tM; pmax = pM; }
-      const u64 tm = shfl_xor64(tmin, d); const u32 pm = __shfl_xor_sync(0xFFFFFFFFu, pmin, d);
-      if (pm != NONE && (pmin == NONE || tm < tmin || (tm == tmin && pm < pmin))) { tmin = tm; pmin = pm; }
-    }
-    u32 gfl = (mism ? CCLD_G_OPSET_MISMATCH : 0) | (barrier ? CCLD_G_BARRIER : 0) | (inflight ? CCLD_G_INFLIGHT : 0) |
-              (bad_time ? CCLD_G_BAD_TIME : 0) | (complete ? CCLD_G_COMPLETE : CCLD_G_INCOMPLETE);
-    const bool analysed = complete && !barrier && n >= P.min_group;
-    if (analysed) gfl |= CCLD_G_ANALYSED;
-    const bool hang = !complete && inflight && age > P.hang_ns && !barrier;
-    if (hang) gfl |= CCLD_G_HANG_ALERT;
-    const u64 askew = complete ? e_max - e_min : 0;
-    u64 med_s = 0, mad_s = 0, med_d = 0, mad_d = 0;
-    if (analysed) {
-      if (n_pad == 32) warp_group_stats<1>(s_te + b, s_du + b, n, lane, e_min, askew, tmin, tmax, &med_s, &mad_s, &med_d, &mad_d);
-      else if (n_pad == 64) warp_group_stats<2>(s_te + b, s_du + b, n, lane, e_min, askew, tmin, tmax, &med_s, &mad_s, &med_d, &mad_d);
-      else warp_group_stats<4>(s_te + b, s_du + b, n, lane, e_min, askew, tmin, tmax, &med_s, &mad_s, &med_d, &mad_d);
-    }
-    // flags and votes, in slot order
-    double num = 1.0, den = 1.0; bus_factor(gop, n, &num, &den);
-    const double bn = (double)gbytes * num;
-    const bool add_bw = complete && !barrier;
+    for (int q = 0; q < 8; ++q) { const u32 ix = idx[q] == NONE ? 0u : idx[q]; ld_a[q] = c_te[ix]; ld_b[q] = c_tx[ix]; }
 #pragma unroll
-    for (int r = 0; r < WARP_EMAX; ++r) {
-      const u32 p = r * 32 + lane;
-      if (p < n) {
-        const u32 st = s_st[b + p];
-        u8 f = CCLD_F_NOT_ANALYSED;
-        if (!(st & 1)) f |= CCLD_F_MISSING;
-        else if (analysed) {
-          const u64 sk = s_te[b + p] - e_min, du = s_du[b + p];
-          const bool so = mul_gt(absdiff(sk, med_s), 1000u, mad_s, k_milli), sh = sk > med_s;
-          const bool dq = mul_gt(absdiff(du, med_d), 1000u, mad_d, k_milli), dh = du > med_d;
-          f = (so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0);
-          if (so) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p] * 4 + (sh ? 0 : 1)], 1u); }
-          if (dq) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p] * 4 + (dh ? 2 : 3)], 1u); }
-        }
-        D.flags[slot_t + (u64)jg * n + p] = f;
-        if (add_bw) bwacc[r] += busbw_fast(bn, den, (i64)s_du[b + p]);
+    for (int q = 0; q < 8; ++q) {
+      if (idx[q] != NONE) {
+        ++npres;
+        const i64 a = ld_a[q], b = ld_b[q];
+        if (b == -1) { stb |= 1; const i64 ag = now - a; age = ag > age ? ag : age; }
+        else if (a < 0 || b < a) stb |= 2;
+        x_max = b > x_max ? b : x_max;
+        const u64 te = (u64)a, du = (u64)(b - a);
+        e_min = te < e_min ? te : e_min; e_max = te > e_max ? te : e_max;
+        if (pmax == NONE || du > tmax) { tmax = du; pmax = p0 + q; }
+        if (pmin == NONE || du < tmin) { tmin = du; pmin = p0 + q; }
+      } else if (active && p0 + q < n) miss = 1;
+    }
+  }
+  // ---- the lanes of a group meet ----
+  const u32 b_miss = __ballot_sync(FULLM, miss != 0), b_if = __ballot_sync(FULLM, (stb & 1) != 0), b_bt = __ballot_sync(FULLM, (stb & 2) != 0);
+  const bool inflight = (b_if & gmask) != 0, bad_time = (b_bt & gmask) != 0;
+  const bool complete = active && (b_miss & gmask) == 0 && !inflight && !bad_time;
+  if (b_miss) {
+#pragma unroll
+    for (int h = 1; h < L; h <<= 1) npres += __shfl_xor_sync(FULLM, npres, h);
+  } else npres = active ? n : 0u;
+  if (b_if) {
+#pragma unroll
+    for (int h = 1; h < L; h <<= 1) { const i64 o = (i64)shfl_xor64((u64)age, h); age = o > age ? o : age; }
+  }
+#pragma unroll
+  for (int h = 1; h < L; h <<= 1) {
+    { const i64 o = (i64)shfl_xor64((u64)x_max, h); x_max = o > x_max ? o : x_max; }
+    { const u64 o = shfl_xor64(e_min, h); e_min = o < e_min ? o : e_min; }
+    { const u64 o = shfl_xor64(e_max, h); e_max = o > e_max ? o : e_max; }
+    { const u64 ot = shfl_xor64(tmax, h); const u32 op = __shfl_xor_sync(FULLM, pmax, h);
+      if (op != NONE && (pmax == NONE || ot > tmax || (ot == tmax && op < pmax))) { tmax = ot; pmax = op; } }
+    { const u64 ot = shfl_xor64(tmin, h); const u32 op = __shfl_xor_sync(FULLM, pmin, h);
+      if (op != NONE && (pmin == NONE || ot < tmin || (ot == tmin && op < pmin))) { tmin = ot; pmin = op; } }
+  }
+  const bool fast = complete && e_max - e_min < 0xFFFFFFFFull && tmax - tmin < 0xFFFFFFFFull;
+  // 32-bit keys: skew, and duration minus the shortest duration (maximum key where there is nothing to sort)
+  u32 sk[8], dd[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) {
+    const bool in = fast && p0 + q < n;
+    sk[q] = in ? (u32)((u64)ld_a[q] - e_min) : 0xFFFFFFFFu; dd[q] = in ? (u32)((u64)(ld_b[q] - ld_a[q]) - tmin) : 0xFFFFFFFFu;
+  }
+  // ---- batch 2: op-set and rate columns ----
+  u64 gbytes = 0, chk = 0; u32 gop = 0; bool have_first = false, mismatch = false;
+  {
+    const u64* __restrict__ c_by = D.bytes; const u8* __restrict__ c_op = D.op;
+    const u32* __restrict__ c_sc = D.send_chg; const u32* __restrict__ c_rc = D.recv_chg;
+    u64 ld_by[8]; u32 ld_op[8], ld_ch[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const u32 ix = idx[q] == NONE ? 0u : idx[q];
+      ld_by[q] = c_by[ix]; ld_op[q] = c_op[ix]; ld_ch[q] = 0;
+      if (c_sc != nullptr) { const u32 sc = c_sc[ix], rc = c_rc[ix]; ld_ch[q] = sc > rc ? sc : rc; }
+    }
+    // the group's first present member: mine, then the lowest lane that has one
+    u64 fby = 0; u32 fop = 0; bool fhave = false;
+#pragma unroll
+    for (int q = 7; q >= 0; --q) if (idx[q] != NONE) { fby = ld_by[q]; fop = ld_op[q]; fhave = true; }
+    const u32 b_have = __ballot_sync(FULLM, fhave) & gmask;
+    have_first = b_have != 0;
+    const u32 src = have_first ? (u32)__ffs(b_have) - 1u : lane;
+    gbytes = __shfl_sync(FULLM, fby, src); gop = __shfl_sync(FULLM, fop, src);
+    bool mism = false;
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      if (idx[q] != NONE) {
+        if (ld_op[q] != gop || ld_by[q] != gbytes) mism = true;
+        const u64 ck = ((u64)ld_ch[q] << 32) | (u64)(NONE - (p0 + q));     // most changes, then lowest position
+        chk = ck > chk ? ck : chk;
       }
     }
-    if (lane == 0) {
-      const u64 g = g_t + jg, G = D.n_groups;
-      if (hang) raise_alert(D, R.comm_id[c], row.seq_lo + t.seq_off + jg, age);
-      const i64 span = complete ? x_max - (i64)e_min : 0;
-      D.gi64[(u64)GI_E_MIN * G + g] = complete ? (i64)e_min : 0; D.gi64[(u64)GI_ARRIVAL_SKEW * G + g] = (i64)askew;
-      D.gi64[(u64)GI_T_MAX * G + g] = complete ? (i64)tmax : 0; D.gi64[(u64)GI_T_MIN * G + g] = complete ? (i64)tmin : 0;
-      D.gi64[(u64)GI_SPAN * G + g] = span;
-      D.gi64[(u64)GI_MED_SKEW * G + g] = (i64)med_s; D.gi64[(u64)GI_MAD_SKEW * G + g] = (i64)mad_s;
-      D.gi64[(u64)GI_MED_DUR * G + g] = (i64)med_d; D.gi64[(u64)GI_MAD_DUR * G + g] = (i64)mad_d;
-      D.gu32[(u64)GU_RANK_TMIN * G + g] = complete ? mem[pmin] : 0; D.gu32[(u64)GU_RANK_TMAX * G + g] = complete ? mem[pmax] : 0;
-      D.gu32[(u64)GU_MAX_CHG * G + g] = complete ? (u32)(chk >> 32) : 0;
-      D.gu32[(u64)GU_RANK_MAX_CHG * G + g] = complete ? mem[NONE - (u32)chk] : 0;
-      D.gu32[(u64)GU_N_PRESENT * G + g] = npres; D.gu32[(u64)GU_GFLAGS * G + g] = gfl;
-      D.gbw[g] = complete ? busbw_fast(bn, den, span) : 0.0;
-      c_comp += complete; c_inc += !complete; c_bar += barrier; c_an += analysed; c_mis += mism; c_pres += npres;
-      if (add_bw) best_merge(w_brng, w_bk, tmax - tmin, t.seq_off + jg);
-    }
-    n_bwc += add_bw ? 1u : 0u;
-  }
-  // 4. per-rank bus bandwidth: warps -> shared memory -> one atomic per member and tile
+    mismatch = (__ballot_sync(FULLM, mism) & gmask) != 0;
 #pragma unroll
-  for (int r = 0; r < WARP_EMAX; ++r) { const u32 p = r * 32 + lane; if (p < n_pad) s_bw[wid * n_pad + p] = bwacc[r]; }
-  n_fs = __reduce_add_sync(0xFFFFFFFFu, n_fs); n_fd = __reduce_add_sync(0xFFFFFFFFu, n_fd);
-  if (lane == 0) {
-    atomicAdd(&s_cnt[0], c_comp); atomicAdd(&s_cnt[1], c_inc); atomicAdd(&s_cnt[2], c_bar); atomicAdd(&s_cnt[3], c_an);
-    atomicAdd(&s_cnt[4], c_mis); atomicAdd(&s_cnt[5], c_pres); atomicAdd(&s_cnt[6], n_fs); atomicAdd(&s_cnt[7], n_fd);
-    s_brng[wid] = w_brng; s_bk[wid] = w_bk; s_rounds[wid] = n_bwc;
+    for (int h = 1; h < L; h <<= 1) { const u64 o = shfl_xor64(chk, h); chk = o > chk ? o : chk; }
   }
+  const bool barrier = have_first && gop == CCLD_OP_ALLREDUCE && gbytes < P.barrier_bytes;
+  const bool analysed = complete && !barrier && n >= P.min_group;
+  const bool add_bw = complete && !barrier;
+  const bool hang = active && !complete && inflight && age > P.hang_ns && !barrier;
+  u32 gfl = (mismatch ? CCLD_G_OPSET_MISMATCH : 0) | (barrier ? CCLD_G_BARRIER : 0) | (inflight ? CCLD_G_INFLIGHT : 0) |
+            (bad_time ? CCLD_G_BAD_TIME : 0) | (complete ? CCLD_G_COMPLETE : CCLD_G_INCOMPLETE) | (analysed ? CCLD_G_ANALYSED : 0) |
+            (hang ? CCLD_G_HANG_ALERT : 0);
+
+  // ---- order statistics, flags, bandwidths ----
+  u64 med_s = 0, mad_s = 0, med_d = 0, mad_d = 0;
+  u64 packed = 0;                                            // my eight flag bytes
+#pragma unroll
+  for (int q = 0; q < 8; ++q)
+    if (p0 + q < n) packed |= (u64)(CCLD_F_NOT_ANALYSED | (idx[q] == NONE ? CCLD_F_MISSING : 0)) << (8 * q);
+  double bw[8];
+#pragma unroll
+  for (int q = 0; q < 8; ++q) bw[q] = 0.0;
+  double num = 1.0, den = 1.0; bus_factor(gop, n, &num, &den);
+  const double bn = (double)gbytes * num;
+  if (__any_sync(FULLM, analysed && fast)) {
+    u32 ms, ds, md, dm;
+    sub_median_mad<L, u32>(sk, n, s, lane, &ms, &ds);
+    sub_median_mad<L, u32>(dd, n, s, lane, &md, &dm);
+    if (analysed && fast) {
+      med_s = ms; mad_s = ds; med_d = tmin + md; mad_d = dm;
+      // |x - med| * 1000 > k * MAD  <=>  |x - med| > floor(k * MAD / 1000); deviations are below 2^32
+      const u64 qs = (u64)ds * k_milli / 1000u, qd = (u64)dm * k_milli / 1000u;
+      const u32 ts = qs > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)qs, td = qd > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)qd;
+      packed = 0;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        if (p0 + q < n) {
+          const u32 a = sk[q] >= ms ? sk[q] - ms : ms - sk[q], b = dd[q] >= md ? dd[q] - md : md - dd[q];
+          const bool so = a > ts, sh = sk[q] > ms, dq = b > td, dh = dd[q] > md;
+          packed |= (u64)((so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0)) << (8 * q);
+        }
+      }
+    }
+  }
+  if (add_bw && fast) {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) if (p0 + q < n) bw[q] = busbw_fast(bn, den, (i64)(tmin + dd[q]));
+  }
+  if (__any_sync(FULLM, complete && !fast)) {
+    u64 o4[4] = {0, 0, 0, 0};
+    sub_group64<L>(D, R, mem, pslot, row.n_seq, n, s, lane, complete && !fast, e_min, k_milli, analysed, add_bw, bn, den, o4, &packed);
+    if (analysed && !fast) { med_s = o4[0]; mad_s = o4[1]; med_d = o4[2]; mad_d = o4[3]; }
+  }
+  u32 n_fs = 0, n_fd = 0;
+  if (analysed) {
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      if (p0 + q < n) {
+        const u32 f = (u32)(packed >> (8 * q));
+        if (f & CCLD_F_SKEW_OUT) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p0 + q] * 4 + ((f & CCLD_F_SKEW_HI) ? 0 : 1)], 1u); }
+        if (f & CCLD_F_DUR_OUT) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p0 + q] * 4 + ((f & CCLD_F_DUR_HI) ? 2 : 3)], 1u); }
+      }
+    }
+  }
+  // ---- outputs: every lane its flag bytes, the group's first lane the row ----
+  if (active) {
+    const u64 slot = row.slot0 + (u64)(t.seq_off + j) * n + p0;
+    if (p0 + 8 <= n && (slot & 7) == 0) *reinterpret_cast<u64*>(D.flags + slot) = packed;
+    else {
+#pragma unroll
+      for (int q = 0; q < 8; ++q) if (p0 + q < n) D.flags[slot + q] = (u8)(packed >> (8 * q));
+    }
+  }
+  if (lead) {
+    const u64 g = row.group0 + t.seq_off + j, G = D.n_groups;
+    if (hang) raise_alert(D, R.comm_id[c], row.seq_lo + t.seq_off + j, age);
+    const i64 span = complete ? x_max - (i64)e_min : 0;
+    D.gi64[(u64)GI_E_MIN * G + g] = complete ? (i64)e_min : 0; D.gi64[(u64)GI_ARRIVAL_SKEW * G + g] = complete ? (i64)(e_max - e_min) : 0;
+    D.gi64[(u64)GI_T_MAX * G + g] = complete ? (i64)tmax : 0; D.gi64[(u64)GI_T_MIN * G + g] = complete ? (i64)tmin : 0;
+    D.gi64[(u64)GI_SPAN * G + g] = span;
+    D.gi64[(u64)GI_MED_SKEW * G + g] = (i64)med_s; D.gi64[(u64)GI_MAD_SKEW * G + g] = (i64)mad_s;
+    D.gi64[(u64)GI_MED_DUR * G + g] = (i64)med_d; D.gi64[(u64)GI_MAD_DUR * G + g] = (i64)mad_d;
+    D.gu32[(u64)GU_RANK_TMIN * G + g] = complete ? mem[pmin] : 0; D.gu32[(u64)GU_RANK_TMAX * G + g] = complete ? mem[pmax] : 0;
+    D.gu32[(u64)GU_MAX_CHG * G + g] = complete ? (u32)(chk >> 32) : 0;
+    D.gu32[(u64)GU_RANK_MAX_CHG * G + g] = complete ? mem[NONE - (u32)chk] : 0;
+    D.gu32[(u64)GU_N_PRESENT * G + g] = npres; D.gu32[(u64)GU_GFLAGS * G + g] = gfl;
+    D.gbw[g] = complete ? busbw_fast(bn, den, span) : 0.0;
+  }
+
+  // ---- per-warp accumulation ----
+  const bool is_round = lead && add_bw;
+  const u32 b_comp = __ballot_sync(FULLM, lead && complete), b_inc = __ballot_sync(FULLM, lead && !complete);
+  const u32 b_bar = __ballot_sync(FULLM, lead && barrier), b_an = __ballot_sync(FULLM, lead && analysed);
+  const u32 b_mis = __ballot_sync(FULLM, lead && mismatch), b_bwc = __ballot_sync(FULLM, is_round);
+  const u32 pres = __reduce_add_sync(FULLM, lead ? npres : 0u), fs = __reduce_add_sync(FULLM, n_fs), fd = __reduce_add_sync(FULLM, n_fd);
+  u64 brng = is_round ? tmax - tmin : 0; u32 bk = is_round ? t.seq_off + j : NONE;
+  best_warp_reduce(brng, bk);
+  // bandwidth sums over the warp's groups: each round halves the values a lane carries
+  u32 off = 0;
+#pragma unroll
+  for (int bit = 16, w = 4; bit >= L; bit >>= 1, w >>= 1) {
+    const bool hi = (lane & bit) != 0;
+#pragma unroll
+    for (int i = 0; i < w; ++i) {
+      const double send = hi ? bw[i] : bw[i + w], keep = hi ? bw[i + w] : bw[i];
+      bw[i] = keep + __shfl_xor_sync(FULLM, send, bit);
+    }
+    off += hi ? (u32)w : 0u;
+  }
+#pragma unroll
+  for (int i = 0; i < 8 / GW; ++i) sh.bw[wid][p0 + off + i] = bw[i];
+  if (lane == 0) {
+    sh.brng[wid] = brng; sh.bk[wid] = bk; sh.rounds[wid] = (u32)__popc(b_bwc); sh.n_an[wid] = (u32)__popc(b_an);
+    if (b_comp) atomicAdd(&sh.cnt[SC_COMP], (u32)__popc(b_comp));
+    if (b_inc) atomicAdd(&sh.cnt[SC_INC], (u32)__popc(b_inc));
+    if (b_bar) atomicAdd(&sh.cnt[SC_BAR], (u32)__popc(b_bar));
+    if (b_an) atomicAdd(&sh.cnt[SC_AN], (u32)__popc(b_an));
+    if (b_mis) atomicAdd(&sh.cnt[SC_MIS], (u32)__popc(b_mis));
+    if (pres) atomicAdd(&sh.cnt[SC_PRES], pres);
+    if (fs) atomicAdd(&sh.cnt[SC_FS], fs);
+    if (fd) atomicAdd(&sh.cnt[SC_FD], fd);
+  }
+}
+
+// Class-1 CTA of the fused kernel: one tile of 2048 / n_pad consecutive op counters of one communicator.
+__device__ __forceinline__ void reduce_sub_cta(const WinDesc& D, const FusedCta& t, TileSum* __restrict__ sums, const Registry& R, const Params& P, i64 now) {
+  __shared__ SubShared sh;
+  const u32 n = t.row.n, n_pad = mid_npad(n);
+  if (threadIdx.x < SC_COUNT) sh.cnt[threadIdx.x] = 0;
+  __syncthreads();
+  if (n_pad == 32) reduce_sub_warp<4>(D, t, R, P, now, sh);
+  else if (n_pad == 64) reduce_sub_warp<8>(D, t, R, P, now, sh);
+  else reduce_sub_warp<16>(D, t, R, P, now, sh);
   __syncthreads();
   u32 rounds = 0;
-  for (int q = 0; q < MID_THREADS / 32; ++q) rounds += s_rounds[q];
+#pragma unroll
+  for (int q = 0; q < MID_THREADS / 32; ++q) rounds += sh.rounds[q];
   if (rounds) {
+    const u32* mem = R.members + t.moff;
     for (u32 p = threadIdx.x; p < n; p += MID_THREADS) {
       double v = 0.0;
-      for (int q = 0; q < MID_THREADS / 32; ++q) v += s_bw[q * n_pad + p];
+#pragma unroll
+      for (int q = 0; q < MID_THREADS / 32; ++q) v += sh.bw[q][p];
       atomicAdd(&R.bw_sum[mem[p]], v);
       atomicAdd(&R.bw_cnt[mem[p]], rounds);
     }
   }
   if (threadIdx.x == 0) {
-    u64 brng = s_brng[0]; u32 bk = s_bk[0];
-    for (int q = 1; q < MID_THREADS / 32; ++q) best_merge(brng, bk, s_brng[q], s_bk[q]);
-    TileSum ts; ts.best_rng = brng; ts.best_k = bk; ts.n_rounds = rounds; ts.n_an = s_cnt[3]; ts.pad = 0;
+    u64 brng = sh.brng[0]; u32 bk = sh.bk[0], n_an = sh.n_an[0];
+    for (int q = 1; q < MID_THREADS / 32; ++q) { best_merge(brng, bk, sh.brng[q], sh.bk[q]); n_an += sh.n_an[q]; }
+    TileSum ts; ts.best_rng = brng; ts.best_k = bk; ts.n_rounds = rounds; ts.n_an = n_an; ts.pad = 0;
     sums[t.sum_idx] = ts;
-    count_add(D.counters, C_COMPLETE, s_cnt[0]); count_add(D.counters, C_INCOMPLETE, s_cnt[1]); count_add(D.counters, C_BARRIER, s_cnt[2]);
-    count_add(D.counters, C_ANALYSED, s_cnt[3]); count_add(D.counters, C_MISMATCH, s_cnt[4]); count_add(D.counters, C_PRESENT, s_cnt[5]);
-    count_add(D.counters, C_FLAG_SKEW, s_cnt[6]); count_add(D.counters, C_FLAG_DUR, s_cnt[7]);
+    count_add(D.counters, C_COMPLETE, sh.cnt[SC_COMP]); count_add(D.counters, C_INCOMPLETE, sh.cnt[SC_INC]); count_add(D.counters, C_BARRIER, sh.cnt[SC_BAR]);
+    count_add(D.counters, C_ANALYSED, sh.cnt[SC_AN]); count_add(D.counters, C_MISMATCH, sh.cnt[SC_MIS]); count_add(D.counters, C_PRESENT, sh.cnt[SC_PRES]);
+    count_add(D.counters, C_FLAG_SKEW, sh.cnt[SC_FS]); count_add(D.counters, C_FLAG_DUR, sh.cnt[SC_FD]);
   }
 }
 
@@ -1420,13 +1513,12 @@ __device__ __forceinline__ void reduce_warp_cta(const WinDesc& D, const FusedCta
 // fused reduce kernel for communicators of up to 128 ranks: the work list is chunk-major, so CTAs that
 // run together gather from the same stretch of every rank's records
 // ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(SMALL_SEQS) k_reduce_fused(const WinDesc* __restrict__ wd, const FusedCta* __restrict__ ctas,
+__global__ void __launch_bounds__(SMALL_SEQS, 2) k_reduce_fused(const WinDesc* __restrict__ wd, const FusedCta* __restrict__ ctas,
                                                              const WarpTile* __restrict__ wts, TileSum* __restrict__ sums, Registry R, Params P, i64 now) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
   const FusedCta t = ctas[blockIdx.x];
   const WinDesc& D = wd[t.w];
   if (t.cls == 0) reduce_small_cta(D, t, wts, sums, R, P, now);
-  else reduce_warp_cta(D, t, sums, R, P, now, smem_raw);
+  else reduce_sub_cta(D, t, sums, R, P, now);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -130,6 +130,32 @@ def test_group_sizes_with_many_ties():
     run_spec(sized_spec((4, 8, 24, 64, 200, 1500), 20, ties=True))
 
 
+def test_wide_value_ranges_and_damaged_groups_in_every_class():
+    """Skews and durations more than 2^32 ns apart (64-bit keys), and missing / in-flight / mismatched / barrier
+    groups, for group sizes of every kernel and every lanes-per-group layout."""
+    rng = np.random.default_rng(5)
+    recs, comms, r0 = [], [], 0
+    for cid, n in enumerate((5, 8, 12, 24, 40, 64, 100, 128, 200, 1100)):
+        ranks = list(range(r0, r0 + n)); r0 += n
+        comms.append((cid, ranks, 0))
+        n_seq = 70 if n <= 128 else 6
+        durs = rng.integers(1_000_000, 1_200_000, size=(n_seq, n)).tolist()
+        ents = rng.integers(0, 40_000, size=(n_seq, n)).tolist()
+        durs[1][n // 2] = 7_000_000_000                       # duration spread above 2^32 ns
+        ents[2][n - 1] = 5_000_000_000                        # skew spread above 2^32 ns
+        durs[3][0] = 6_000_000_000; ents[3][n // 3] = 4_400_000_000
+        durs[n_seq - 1][n - 1] = 2**33                        # in the last (ragged) tile
+        g = group_trace(durs, ents, comm=cid, ranks=ranks, spacing=10_000_000_000, bytes=MiB)
+        by_key = {(r["seq"], r["rank"]): r for r in g}
+        del by_key[(4, ranks[n - 1])]                         # missing member
+        by_key[(5, ranks[1])]["t_exit"] = -1                  # in flight
+        by_key[(n_seq - 2, ranks[n // 2])]["bytes"] = 2 * MiB  # op-set mismatch
+        for r in g:
+            if r["seq"] == 0: r["bytes"] = 3                  # barrier
+        recs += list(by_key.values())
+    hand_pair(recs, comms, now=10**13)
+
+
 # ---------------------------------------------------------------- edge cases
 def hand_pair(recs, comms, params=None, now=10**12, with_rates=True, frames=None, n_channels=0, expect_rc=0):
     an, o = make_pair(comms, params)
