@@ -45,6 +45,7 @@ def _load():
                      "orc_copy_groups", "orc_copy_slots", "orc_copy_comm_rows", "orc_copy_alerts",
                      "orc_copy_rank_stats", "orc_suspects", "orc_locate_hang"):
             getattr(_lib, name).restype = C.c_int
+        _lib.orc_derive_rates.restype = None
     return _lib
 
 
@@ -165,3 +166,15 @@ class Oracle:
         d["min_total"] = int(mn[0])
         d["roots"] = roots[:min(d["n_roots"], cap)].copy()
         return d
+
+
+def derive_rates(rank, t_enter, t_exit, tick_off, tick_ns, send_count, recv_count):
+    """Counter changes per record from raw probe samples (Sec. 4.1.2); returns (send_chg, recv_chg) as uint32 arrays."""
+    lib = _load()
+    rank = _np(rank, np.uint32); te = _np(t_enter, np.int64); tx = _np(t_exit, np.int64)
+    off = _np(tick_off, np.uint64); tn = _np(tick_ns, np.int64); sc = _np(send_count, np.uint32); rc = _np(recv_count, np.uint32)
+    n = len(rank)
+    out_s = np.zeros(n, np.uint32); out_r = np.zeros(n, np.uint32)
+    lib.orc_derive_rates(C.c_uint64(n), _p(rank), _p(te), _p(tx), C.c_uint32(len(off) - 1), _p(off), _p(tn), _p(sc), _p(rc),
+                         _p(out_s), _p(out_r))
+    return out_s, out_r

@@ -13,6 +13,8 @@
 // Pins (tests/test_oracle_*.py): hand-built traces with known answers, the paper's limits of P
 // (Sec. 4.2.2), the SendRate worked example (Sec. 4.1.2, Fig. 5), one trace per leaf of the hang
 // decision tree, brute-force order statistics by counting, and invariants.
+// orc_derive_rates (counter changes per op from raw probe samples) is pinned to the same worked example, to closed
+// forms for a counter that advances every tick, to additivity over adjacent ops and to a numpy restatement.
 // "Parity unpinned" against the paper: the bus-bandwidth factor and the median/MAD convention,
 // because the paper defines neither (they are this repository's conventions, pinned only to
 // closed forms and hand values).
@@ -484,6 +486,27 @@ int orc_locate_hang(void* h, u32 wid, u32 comm, u32 seq, u32* out, u64* min_tota
   out[0] = cls; out[1] = (u32)r.size(); out[2] = n_ne; out[3] = n_hung; out[4] = n_ok; out[5] = n_missing; out[6] = stuck; out[7] = n;
   for (size_t i = 0; i < r.size() && i < cap; ++i) roots[i] = r[i];
   return 0;
+}
+
+// SendRate / RecvRate inputs from raw probe samples (Sec. 4.1.2: the rate is the reciprocal of the number of changes
+// of SendCount / RecvCount seen by a probe that samples at a fixed period; Sec. 5.2 step 2: the diagnostic thread
+// derives it from the counters). Rank r's samples are ticks [tick_off[r], tick_off[r+1]) in time order. For every
+// record, the number of that rank's ticks k (not the rank's first) with t_enter < t_k <= t_end whose counter differs
+// from the previous tick's; t_end = t_exit, or unbounded while the op is in flight (t_exit = -1).
+void orc_derive_rates(u64 n_rec, const u32* rank, const i64* t_enter, const i64* t_exit, u32 n_ranks, const u64* tick_off,
+                      const i64* tick_ns, const u32* send_count, const u32* recv_count, u32* send_chg, u32* recv_chg) {
+  for (u64 i = 0; i < n_rec; ++i) {
+    u32 s = 0, r = 0;
+    if (rank[i] < n_ranks) {
+      for (u64 k = tick_off[rank[i]] + 1; k < tick_off[rank[i] + 1]; ++k) {
+        if (tick_ns[k] <= t_enter[i]) continue;
+        if (t_exit[i] != -1 && tick_ns[k] > t_exit[i]) continue;
+        if (send_count[k] != send_count[k - 1]) ++s;
+        if (recv_count[k] != recv_count[k - 1]) ++r;
+      }
+    }
+    send_chg[i] = s; recv_chg[i] = r;
+  }
 }
 
 }  // extern "C"

@@ -500,3 +500,73 @@ def test_scaled_cfg2_and_cfg5_recover_injected_ranks():
             w, c, s = alerts[0]
             h = o.locate_hang(w, c, s)
             assert h["cls"] == 3 and list(h["roots"]) == spec.truth["hang_root"] and h["stuck_step"] == 41
+
+
+# ---------------------------------------------------------------- counter changes from raw probe samples (Sec. 4.1.2)
+MS = 1_000_000
+
+
+def _ticks(series):
+    """series: per rank a list of (t_ns, send_count, recv_count) -> CSR arrays."""
+    off = np.cumsum([0] + [len(s) for s in series]).astype(np.uint64)
+    flat = [x for s in series for x in s]
+    return (off, np.array([x[0] for x in flat], np.int64), np.array([x[1] for x in flat], np.uint32),
+            np.array([x[2] for x in flat], np.uint32))
+
+
+def test_derived_rates_reproduce_the_papers_worked_example():
+    """Sec. 4.1.2, Fig. 5: probed every 1 ms, 8 sends show as 2 value changes on a normal rank and as 7 on a slow one."""
+    ex = GOLD["send_rate_example"]
+    normal = [(k * MS, min(8, 4 * k), 0) for k in range(11)]                      # 0, 4, 8, 8, ...
+    slow_vals = [0, 1, 2, 3, 4, 6, 7, 8, 8, 8, 8]                                 # seven changes to reach 8
+    slow = [(k * MS, slow_vals[k], 0) for k in range(11)]
+    off, tn, sc, rc = _ticks([normal, slow])
+    s, r = orc.derive_rates([0, 1], [0, 0], [10 * MS, 10 * MS], off, tn, sc, rc)
+    assert list(s) == [ex["normal_changes"], ex["slow_changes"]] and list(r) == [0, 0]
+    # the rate is the reciprocal of the count: 1/2 against 1/7
+    assert [1, int(s[0])] == ex["normal_rate"] and [1, int(s[1])] == ex["slow_rate"]
+
+
+def test_derived_rates_closed_form_boundaries_and_additivity():
+    # a counter that advances at every tick: changes = ticks in (t_enter, t_exit]; recv advances every second tick
+    T = 200
+    ser = [(1000 + k * MS, k, k // 2) for k in range(T)]
+    off, tn, sc, rc = _ticks([ser])
+    rng = np.random.default_rng(11)
+    a = rng.integers(0, T * MS, 64); b = a + rng.integers(0, 30 * MS, 64)
+    s, r = orc.derive_rates(np.zeros(64, np.uint32), a, b, off, tn, sc, rc)
+    tick = lambda t: np.clip((t - 1000) // MS + 1, 0, T)                           # ticks at or before t
+    assert np.array_equal(s, np.maximum(tick(b), 1) - np.maximum(tick(a), 1))      # the rank's first tick never counts
+    # a tick exactly at t_enter is outside, exactly at t_exit inside
+    s2, _ = orc.derive_rates([0, 0], [1000 + 5 * MS, 1000 + 5 * MS - 1], [1000 + 7 * MS, 1000 + 7 * MS - 1], off, tn, sc, rc)
+    assert list(s2) == [2, 2]
+    # adjacent ops add up to the enclosing one
+    cuts = np.sort(rng.integers(0, T * MS, 9))
+    s3, r3 = orc.derive_rates(np.zeros(8, np.uint32), cuts[:-1], cuts[1:], off, tn, sc, rc)
+    s4, r4 = orc.derive_rates([0], [cuts[0]], [cuts[-1]], off, tn, sc, rc)
+    assert s3.sum() == s4[0] and r3.sum() == r4[0]
+    # constant counters, an op in flight (counts to the end of the samples), a rank without samples, an unknown rank
+    off2, tn2, sc2, rc2 = _ticks([[(k * MS, 5, 9) for k in range(50)], ser, []])
+    s5, r5 = orc.derive_rates([0, 1, 2, 7], [0, 1000 + 150 * MS, 0, 0], [40 * MS, -1, 40 * MS, 40 * MS], off2, tn2, sc2, rc2)
+    assert list(s5) == [0, T - 1 - 150, 0, 0] and list(r5) == [0, (T - 1) // 2 - 150 // 2, 0, 0]
+
+
+def test_derived_rates_against_a_numpy_restatement():
+    rng = np.random.default_rng(12)
+    series = []
+    for _ in range(9):
+        n = int(rng.integers(0, 300))
+        t = np.sort(rng.choice(400 * MS, size=n, replace=False))
+        series.append(list(zip(t.tolist(), np.cumsum(rng.integers(0, 3, n)).tolist(), np.cumsum(rng.integers(0, 2, n)).tolist())))
+    off, tn, sc, rc = _ticks(series)
+    n_rec = 500
+    rank = rng.integers(0, 9, n_rec).astype(np.uint32)
+    te = rng.integers(0, 400 * MS, n_rec); tx = te + rng.integers(0, 50 * MS, n_rec)
+    tx[rng.random(n_rec) < 0.05] = -1
+    s, r = orc.derive_rates(rank, te, tx, off, tn, sc, rc)
+    for i in range(n_rec):
+        lo, hi = int(off[rank[i]]), int(off[rank[i] + 1])
+        t = tn[lo:hi]
+        inside = (t[1:] > te[i]) & ((t[1:] <= tx[i]) | (tx[i] == -1))
+        assert s[i] == int((np.diff(sc[lo:hi].astype(np.int64))[inside] != 0).sum())
+        assert r[i] == int((np.diff(rc[lo:hi].astype(np.int64))[inside] != 0).sum())
