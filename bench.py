@@ -43,6 +43,7 @@ def parse():
     ap.add_argument("--windows", type=int, default=100, help="windows of 1,000 ops per rank resident on the GPU")
     ap.add_argument("--e2e-windows", type=int, default=10, help="windows per end-to-end step (host buffers)")
     ap.add_argument("--cpu-windows", type=int, default=10, help="windows the CPU oracle is timed on")
+    ap.add_argument("--rate-windows", type=int, default=2, help="windows whose raw probe samples are turned into rate columns (0 = skip)")
     return ap.parse_args()
 
 
@@ -304,6 +305,30 @@ def run_ours(args, rank, world, local_rank):
                "windows_per_step": NE, "steps": e_steps, "ms_per_step": e_ms / e_steps}
         an_e.close()
 
+    # ---- counter changes per op from raw probe samples (the step before the path), timed on its own ----
+    rates = None
+    NR = min(args.rate_windows, NW)
+    if NR > 0:
+        win = tg.gen_window(spec, 0, device=dev)
+        ticks = tg.gen_ticks(win.cols, spec.n_ranks)
+        call = lambda: an.derive_rates(win.cols["rank"], win.cols["t_enter"], win.cols["t_exit"], ticks["tick_off"], ticks["tick_ns"],
+                                       ticks["send_count"], ticks["recv_count"])
+        for _ in range(3):
+            call()
+        torch.cuda.synchronize()
+        r0, r1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        r0.record()
+        for _ in range(NR * 5):
+            call()
+        r1.record()
+        torch.cuda.synchronize()
+        r_ms = r0.elapsed_time(r1) / (NR * 5)
+        n_t = int(ticks["tick_ns"].numel())
+        r_bytes = 16 * n_t + 28 * win.n_rec              # ticks read once (time, two counters); rank and times read, two counts written
+        rates = {"records": win.n_rec, "ticks": n_t, "ms_per_window": r_ms, "algorithmic_bytes": r_bytes,
+                 "achieved": r_bytes / (r_ms * 1e-3) / 1e9, "unit": "GB/s", "frac": r_bytes / (r_ms * 1e-3) / 1e9 / peak, "launches_per_window": 4}
+        del win, ticks
+
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -313,6 +338,7 @@ def run_ours(args, rank, world, local_rank):
                        "records_per_gpu": n_rec, "bytes_per_record": REC_BYTES, "l2": "inputs larger than L2 (%.1f GB of columns per GPU)" % (n_rec * REC_BYTES / 1e9),
                        "injected_ranks_recovered": recovered},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu_base,
+            "derive_rates": rates,
         }
         print(json.dumps(line), flush=True)
     if world > 1:

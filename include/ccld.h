@@ -270,6 +270,27 @@ int ccld_get_ranges(ccld_ctx* ctx, uint32_t window_id, ccld_comm_range* rows /* 
 int ccld_get_rank_stats(ccld_ctx* ctx, uint32_t n_ranks, uint32_t* votes, uint32_t* ops, uint32_t* bw_cnt, double* bw_sum);
 
 /*
+ * SendRate / RecvRate inputs from raw probe samples (Sec. 4.1.2: the rate is the reciprocal of the number of changes of
+ * SendCount / RecvCount seen by a probe that samples at a fixed period; Sec. 5.2 step 2 has the host's diagnostic
+ * thread derive it). This call does that step on the GPU and produces the send_chg / recv_chg columns that
+ * ccld_trace_upload takes.
+ *   Samples: rank r < n_ranks owns ticks [tick_off[r], tick_off[r + 1]) of tick_ns / send_count / recv_count, in time
+ *   order; tick_off has n_ranks + 1 entries, tick_off[0] = 0, tick_off[n_ranks] = n_ticks.
+ *   Result: for record i of rank r, send_chg[i] = the number of r's ticks k, other than r's first, with
+ *   t_enter_ns[i] < tick_ns[k] <= t_end whose send_count differs from the previous tick's; t_end = t_exit_ns[i], or
+ *   unbounded while the op is in flight (t_exit_ns[i] = -1). recv_chg likewise. A rank without ticks, or a rank id
+ *   >= n_ranks, gets 0.
+ * Every pointer is device memory of the context's device, owned by the caller and left untouched except for the two
+ * outputs (n_rec entries each). The kernels are enqueued on the context's stream and the call returns without
+ * synchronizing; scratch (8 bytes per tick) comes from the context's block pool. Counts are 32-bit:
+ * n_ticks >= 2^32 - 1 is refused with CCLD_ERR_CAPACITY. Other errors: CCLD_ERR_ARG (null pointers, n_ranks = 0),
+ * CCLD_ERR_NOMEM, CCLD_ERR_CUDA.
+ */
+int ccld_derive_rates(ccld_ctx* ctx, uint64_t n_rec, const uint32_t* rank, const int64_t* t_enter_ns, const int64_t* t_exit_ns,
+                      uint32_t n_ranks, uint64_t n_ticks, const uint64_t* tick_off, const int64_t* tick_ns,
+                      const uint32_t* send_count, const uint32_t* recv_count, uint32_t* send_chg, uint32_t* recv_chg);
+
+/*
  * Per-kernel device timing for benchmarks. While enabled, ccld_analyze_window brackets each of its
  * kernel launches with CUDA events on the context's stream. ccld_get_kernel_times synchronizes the
  * stream and returns, per kernel kind, the summed device time in milliseconds and the number of

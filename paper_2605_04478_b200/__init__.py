@@ -25,7 +25,7 @@ MAX_ALERTS_PER_WINDOW = 1024
 EXPORTS = ("ccld_params_default", "ccld_create", "ccld_destroy", "ccld_last_error", "ccld_comm_register",
            "ccld_trace_upload", "ccld_window_release", "ccld_analyze_window", "ccld_reset", "ccld_get_verdict",
            "ccld_locate_hang", "ccld_get_optable", "ccld_get_ranges", "ccld_get_rank_stats", "ccld_copy_to_host",
-           "ccld_timing_enable", "ccld_get_kernel_times", "ccld_ring_locate_static")
+           "ccld_timing_enable", "ccld_get_kernel_times", "ccld_ring_locate_static", "ccld_derive_rates")
 STATIC_MAX_MEMBERS = 8192
 KERNEL_KINDS = ("k_seq_range", "k_plan", "k_slot_scatter", "k_reduce_fused", "k_reduce_mid", "k_reduce_large", "k_window_decide")
 
@@ -120,6 +120,7 @@ def load_library() -> C.CDLL:
         lib.ccld_get_ranges.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.POINTER(C.c_uint32)]
         lib.ccld_get_rank_stats.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         lib.ccld_copy_to_host.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint64]
+        lib.ccld_derive_rates.argtypes = [C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint64] + [C.c_void_p] * 6
         lib.ccld_timing_enable.argtypes = [C.c_void_p, C.c_int]
         lib.ccld_get_kernel_times.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p]
         lib.ccld_ring_locate_static.argtypes = [C.c_int, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p,
@@ -342,6 +343,24 @@ class Analyzer:
         ms = np.zeros(len(KERNEL_KINDS), np.float64); n = np.zeros(len(KERNEL_KINDS), np.uint64)
         self._check(self.lib.ccld_get_kernel_times(self.h, ms.ctypes.data, n.ctypes.data))
         return {k: {"ms": float(ms[i]), "launches": int(n[i])} for i, k in enumerate(KERNEL_KINDS)}
+
+    def derive_rates(self, rank, t_enter, t_exit, tick_off, tick_ns, send_count, recv_count):
+        """ccld_derive_rates: counter changes per record from raw probe samples (Sec. 4.1.2). All inputs are tensors on
+        this GPU; returns (send_chg, recv_chg) as int32 tensors on this GPU (bit pattern uint32), written asynchronously on
+        the analyzer's stream."""
+        torch = self.torch
+        cols = [_as_tensor(torch, rank, "int32"), _as_tensor(torch, t_enter, "int64"), _as_tensor(torch, t_exit, "int64"),
+                _as_tensor(torch, tick_off, "int64"), _as_tensor(torch, tick_ns, "int64"), _as_tensor(torch, send_count, "int32"),
+                _as_tensor(torch, recv_count, "int32")]
+        assert all(c.device.type == "cuda" for c in cols), "ccld_derive_rates takes device memory"
+        cols = [c.contiguous() for c in cols]
+        n = int(cols[0].numel()); n_ranks = int(cols[3].numel()) - 1; n_ticks = int(cols[4].numel())
+        out_s = torch.empty(n, dtype=torch.int32, device=cols[0].device); out_r = torch.empty_like(out_s)
+        ptr = lambda v: C.c_void_p(v.data_ptr()) if v.numel() else C.c_void_p(0)
+        self._check(self.lib.ccld_derive_rates(self.h, n, ptr(cols[0]), ptr(cols[1]), ptr(cols[2]), n_ranks, n_ticks, ptr(cols[3]),
+                                               ptr(cols[4]), ptr(cols[5]), ptr(cols[6]), ptr(out_s), ptr(out_r)))
+        self._rate_keep = cols                     # inputs stay alive until the next call or a synchronization
+        return out_s, out_r
 
     def get_rank_stats(self, n_ranks: int) -> Dict[str, np.ndarray]:
         votes = np.zeros((n_ranks, 4), np.uint32); ops = np.zeros(n_ranks, np.uint32)

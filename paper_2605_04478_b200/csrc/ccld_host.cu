@@ -12,6 +12,7 @@
 #include <vector>
 
 #include "ccld_kernels.cuh"
+#include "ccld_rates.cuh"
 
 using namespace ccld;
 
@@ -613,6 +614,39 @@ int ccld_get_rank_stats(ccld_ctx* ctx, uint32_t n_ranks, uint32_t* votes, uint32
   CK(cudaMemcpyAsync(bw_cnt, ctx->reg.bw_cnt, (size_t)n * 4, cudaMemcpyDeviceToHost, st));
   CK(cudaMemcpyAsync(bw_sum, ctx->reg.bw_sum, (size_t)n * 8, cudaMemcpyDeviceToHost, st));
   CK(cudaStreamSynchronize(st));
+  return CCLD_OK;
+}
+
+int ccld_derive_rates(ccld_ctx* ctx, uint64_t n_rec, const uint32_t* rank, const int64_t* t_enter_ns, const int64_t* t_exit_ns,
+                      uint32_t n_ranks, uint64_t n_ticks, const uint64_t* tick_off, const int64_t* tick_ns,
+                      const uint32_t* send_count, const uint32_t* recv_count, uint32_t* send_chg, uint32_t* recv_chg) {
+  if (!ctx) return CCLD_ERR_ARG;
+  if (n_rec && (!rank || !t_enter_ns || !t_exit_ns || !send_chg || !recv_chg)) return fail(ctx, CCLD_ERR_ARG, "null record column");
+  if (n_ranks == 0 || !tick_off) return fail(ctx, CCLD_ERR_ARG, "tick_off is required (n_ranks + 1 entries)");
+  if (n_ticks && (!tick_ns || !send_count || !recv_count)) return fail(ctx, CCLD_ERR_ARG, "null tick column");
+  if (n_ticks >= 0xFFFFFFFFull) return fail(ctx, CCLD_ERR_CAPACITY, "too many ticks for 32-bit change counts");
+  if ((n_rec + RT_THREADS - 1) / RT_THREADS > 0x7FFFFFFFull) return fail(ctx, CCLD_ERR_CAPACITY, "too many records for one launch");
+  CK(cudaSetDevice(ctx->device));
+  if (n_rec == 0) return CCLD_OK;
+  cudaStream_t st = ctx->stream;
+  const u64 n_tiles = (n_ticks + RT_TILE - 1) / RT_TILE;
+  size_t off = 0;
+  auto take = [&](size_t b) { size_t o = off; off = align_up(off + b); return o; };
+  const size_t o_pre = take((n_ticks + 1) * 8), o_sum = take((n_tiles + 1) * 8);
+  cudaError_t e;
+  Block blk = ctx->pool.get(off, &e);
+  if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "scratch allocation failed");
+  TickArgs A; A.n_ticks = n_ticks; A.n_ranks = n_ranks; A.tick_off = tick_off; A.tick_ns = tick_ns; A.send = send_count; A.recv = recv_count;
+  A.prefix = (u64*)((char*)blk.p + o_pre); A.tile_sum = (u64*)((char*)blk.p + o_sum);
+  if (n_tiles) {
+    k_tick_sums<<<(u32)n_tiles, RT_THREADS, 0, st>>>(A);
+    k_tile_scan<<<1, RT_THREADS, 0, st>>>(A.tile_sum, n_tiles);
+    k_tick_prefix<<<(u32)n_tiles, RT_THREADS, 0, st>>>(A);
+  }
+  k_record_rates<<<(u32)((n_rec + RT_THREADS - 1) / RT_THREADS), RT_THREADS, 0, st>>>(A, n_rec, rank, t_enter_ns, t_exit_ns, send_chg, recv_chg);
+  const cudaError_t le = cudaGetLastError();
+  ctx->pool.put(blk);           // later work on this stream runs after these kernels: the block can be handed out again
+  if (le != cudaSuccess) return fail(ctx, CCLD_ERR_CUDA, std::string("rate kernels: ") + cudaGetErrorString(le));
   return CCLD_OK;
 }
 

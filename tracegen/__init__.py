@@ -14,4 +14,5 @@ from .core import (  # noqa: F401
     OP_ALLREDUCE, OP_ALLGATHER, OP_REDUCESCATTER, OP_ALLTOALL, OP_SENDRECV, OP_BROADCAST,
     Family, Fault, Hang, Spec, Window, gen_window, registry, records_per_window,
 )
+from .ticks import gen_ticks  # noqa: F401
 from .presets import cfg1, cfg2, cfg3, cfg4, cfg4w, cfg5, PRESETS  # noqa: F401
