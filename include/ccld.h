@@ -228,6 +228,20 @@ typedef struct {
 int ccld_locate_hang(ccld_ctx* ctx, uint32_t window_id, uint32_t comm, uint32_t seq, ccld_hang_verdict* out /* host */);
 
 /*
+ * Hang location for every alert of an analysed window in one kernel launch (Sec. 4.2.2, Fig. 6: the decision tree runs
+ * for each hang that detection reported; Sec. 4.2.1 raises the alerts). out[i] is what ccld_locate_hang returns for the
+ * i-th alert in the order ccld_get_verdict lists them (communicator registration order, then op counter).
+ *   alerts  host, cap entries, may be NULL: receives the (comm, seq, age) that out[i] belongs to
+ *   out     host, cap entries: the verdicts; out[i].roots is set to roots + i * roots_stride, out[i].roots_cap to
+ *           roots_stride (NULL and 0 when roots is NULL)
+ *   roots   host, cap * roots_stride rank ids, may be NULL
+ *   n_total the window's number of alerts; at most min(cap, CCLD_MAX_ALERTS_PER_WINDOW) are located
+ * Synchronizes the stream. Scratch comes from the context's block pool (CCLD_ERR_NOMEM if that fails).
+ */
+int ccld_locate_hangs(ccld_ctx* ctx, uint32_t window_id, ccld_hang_alert* alerts /* host */, ccld_hang_verdict* out /* host */,
+                      uint32_t cap, uint32_t* roots /* host */, uint32_t roots_stride, uint32_t* n_total);
+
+/*
  * Parity / inspection access to the per-op table of an analysed window. Device pointers, valid
  * until the window is released or the context reset. Groups are ordered by (communicator
  * registration order, seq); group g of communicator row r covers slots

@@ -9,7 +9,7 @@ from __future__ import annotations
 
 import ctypes as C
 import os
-from typing import Dict, Optional
+from typing import Dict, List, Optional
 
 import numpy as np
 
@@ -25,7 +25,7 @@ MAX_ALERTS_PER_WINDOW = 1024
 EXPORTS = ("ccld_params_default", "ccld_create", "ccld_destroy", "ccld_last_error", "ccld_comm_register",
            "ccld_trace_upload", "ccld_window_release", "ccld_analyze_window", "ccld_reset", "ccld_get_verdict",
            "ccld_locate_hang", "ccld_get_optable", "ccld_get_ranges", "ccld_get_rank_stats", "ccld_copy_to_host",
-           "ccld_timing_enable", "ccld_get_kernel_times", "ccld_ring_locate_static", "ccld_derive_rates")
+           "ccld_timing_enable", "ccld_get_kernel_times", "ccld_ring_locate_static", "ccld_derive_rates", "ccld_locate_hangs")
 STATIC_MAX_MEMBERS = 8192
 KERNEL_KINDS = ("k_seq_range", "k_plan", "k_slot_scatter", "k_reduce_fused", "k_reduce_mid", "k_reduce_large", "k_window_decide")
 
@@ -116,6 +116,7 @@ def load_library() -> C.CDLL:
         lib.ccld_reset.argtypes = [C.c_void_p]
         lib.ccld_get_verdict.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(Verdict)]
         lib.ccld_locate_hang.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.POINTER(HangVerdict)]
+        lib.ccld_locate_hangs.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.POINTER(C.c_uint32)]
         lib.ccld_get_optable.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(OpTable)]
         lib.ccld_get_ranges.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.POINTER(C.c_uint32)]
         lib.ccld_get_rank_stats.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
@@ -303,6 +304,25 @@ class Analyzer:
                                                                  "n_missing_frames", "stuck_step", "n_members", "min_total")}
         out["roots"] = np.array(roots[:min(hv.n_roots_total, roots_cap)], dtype=np.uint32)
         return out
+
+    def locate_hangs(self, window_id: int, cap: int = 1024, roots_stride: int = 64) -> List[Dict[str, object]]:
+        """ccld_locate_hangs: the hang verdict of every alert of the window, one launch; each dict also carries the alert's
+        comm, seq and age_ns."""
+        n = C.c_uint32(0)
+        cap = max(cap, 1)
+        hv = (HangVerdict * cap)(); al = (HangAlert * cap)()
+        roots = (C.c_uint32 * (cap * max(roots_stride, 1)))()
+        self._check(self.lib.ccld_locate_hangs(self.h, window_id, C.cast(al, C.c_void_p), C.cast(hv, C.c_void_p), cap,
+                                               C.cast(roots, C.c_void_p), roots_stride, C.byref(n)))
+        res = []
+        for i in range(min(n.value, cap)):
+            d: Dict[str, object] = {k: int(getattr(hv[i], k)) for k in ("cls", "n_roots_total", "n_not_entered", "n_hung", "n_not_hung",
+                                                                      "n_missing_frames", "stuck_step", "n_members", "min_total")}
+            k = min(hv[i].n_roots_total, roots_stride)
+            d["roots"] = np.array(roots[i * roots_stride:i * roots_stride + k], dtype=np.uint32)
+            d["comm"], d["seq"], d["age_ns"] = int(al[i].comm), int(al[i].seq), int(al[i].age_ns)
+            res.append(d)
+        return res
 
     def get_ranges(self, window_id: int) -> Dict[str, np.ndarray]:
         n = C.c_uint32(0)

@@ -565,6 +565,82 @@ int ccld_locate_hang(ccld_ctx* ctx, uint32_t window_id, uint32_t comm, uint32_t 
   return CCLD_OK;
 }
 
+int ccld_locate_hangs(ccld_ctx* ctx, uint32_t window_id, ccld_hang_alert* alerts, ccld_hang_verdict* out, uint32_t cap,
+                      uint32_t* roots, uint32_t roots_stride, uint32_t* n_total) {
+  if (!ctx || !n_total) return CCLD_ERR_ARG;
+  if (cap && !out) return fail(ctx, CCLD_ERR_ARG, "out is null");
+  WindowHost* w;
+  { int rc = find_analysed(ctx, window_id, &w); if (rc != CCLD_OK) return rc; }
+  CK(cudaSetDevice(ctx->device));
+  cudaStream_t st = ctx->stream;
+  u64 n_al64 = 0;
+  CK(cudaMemcpyAsync(&n_al64, w->d.counters + C_ALERTS, 8, cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  *n_total = (u32)std::min<u64>(n_al64, 0xFFFFFFFFull);
+  const u32 n_dev = (u32)std::min<u64>(n_al64, CCLD_MAX_ALERTS_PER_WINDOW), n = std::min<u32>(n_dev, cap);
+  if (n == 0) return CCLD_OK;
+  // the alerts in the order ccld_get_verdict lists them
+  char* m = (char*)ctx->misc_blk.p;
+  const MiscLayout L = misc_layout(ctx->n_ranks, ctx->max_n);
+  ccld_hang_alert* al_b = (ccld_hang_alert*)(m + L.alerts);
+  k_rank_sort_alerts<<<(n_dev + 127) / 128, 128, 0, st>>>(w->d.alerts, n_dev, al_b, ctx->reg);
+  CK(cudaGetLastError());
+  std::vector<ccld_hang_alert> al(n);
+  CK(cudaMemcpyAsync(al.data(), al_b, n * sizeof(ccld_hang_alert), cudaMemcpyDeviceToHost, st));
+  CK(cudaStreamSynchronize(st));
+  // per alert: scratch over the communicator's members, a root list and a verdict
+  std::vector<HangArgs> ha(n);
+  std::vector<size_t> o_roots(n);
+  std::vector<u32> members(n);
+  size_t off = 0;
+  auto take = [&](size_t b) { size_t o = off; off = align_up(off + b); return o; };
+  const size_t o_args = take(n * sizeof(HangArgs)), o_out = take(n * sizeof(ccld_hang_verdict));
+  std::vector<size_t> o_ent(n), o_done(n), o_frame(n), o_tot(n);
+  for (u32 i = 0; i < n; ++i) {
+    auto ci = ctx->comm_idx.find(al[i].comm);
+    if (ci == ctx->comm_idx.end()) return fail(ctx, CCLD_ERR_CUDA, "internal: alert names an unknown communicator");
+    const u32 nm = (u32)ctx->comms[ci->second].ranks.size();
+    members[i] = nm; ha[i].c = ci->second;
+    o_ent[i] = take(nm); o_done[i] = take(nm); o_frame[i] = take(nm * 4ull); o_tot[i] = take(nm * 8ull); o_roots[i] = take(nm * 4ull);
+  }
+  cudaError_t e;
+  Block blk = ctx->pool.get(off, &e);
+  if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "scratch allocation failed");
+  char* b = (char*)blk.p;
+  for (u32 i = 0; i < n; ++i) {
+    HangArgs& A = ha[i];
+    A.seq = al[i].seq; A.n_frames = w->n_frames; A.n_channels = w->n_channels;
+    A.f_rank = w->f_rank; A.f_comm = w->f_comm; A.f_seq = w->f_seq; A.progress = w->progress;
+    A.entered = (u8*)(b + o_ent[i]); A.done = (u8*)(b + o_done[i]); A.frame = (u32*)(b + o_frame[i]); A.tot = (u64*)(b + o_tot[i]);
+    A.roots = (u32*)(b + o_roots[i]); A.roots_cap = members[i];
+    A.out = (ccld_hang_verdict*)(b + o_out) + i;
+  }
+  std::vector<ccld_hang_verdict> hv(n);
+  std::vector<char> host_blk;
+  int rc = CCLD_OK;
+  do {
+    if (cudaMemcpyAsync(b + o_args, ha.data(), n * sizeof(HangArgs), cudaMemcpyHostToDevice, st) != cudaSuccess) { rc = CCLD_ERR_CUDA; break; }
+    k_hang_locate_many<<<n, 1024, 0, st>>>(w->d_desc, ctx->reg, (const HangArgs*)(b + o_args));
+    if (cudaGetLastError() != cudaSuccess) { rc = CCLD_ERR_CUDA; break; }
+    host_blk.resize(off);
+    // verdicts and root lists come back in one copy (they follow each other in the block)
+    if (cudaMemcpyAsync(host_blk.data() + o_out, b + o_out, off - o_out, cudaMemcpyDeviceToHost, st) != cudaSuccess) { rc = CCLD_ERR_CUDA; break; }
+    if (cudaStreamSynchronize(st) != cudaSuccess) { rc = CCLD_ERR_CUDA; break; }
+  } while (0);
+  ctx->pool.put(blk);
+  if (rc != CCLD_OK) return fail(ctx, rc, "hang sweep failed");
+  for (u32 i = 0; i < n; ++i) {
+    ccld_hang_verdict v;
+    std::memcpy(&v, host_blk.data() + o_out + i * sizeof(ccld_hang_verdict), sizeof v);
+    v.roots = roots ? roots + (size_t)i * roots_stride : nullptr; v.roots_cap = roots ? roots_stride : 0;
+    const u32 n_copy = std::min<u32>(std::min<u32>(v.n_roots_total, members[i]), v.roots_cap);
+    if (n_copy) std::memcpy(v.roots, host_blk.data() + o_roots[i], n_copy * 4ull);
+    out[i] = v;
+    if (alerts) alerts[i] = al[i];
+  }
+  return CCLD_OK;
+}
+
 int ccld_get_optable(ccld_ctx* ctx, uint32_t window_id, ccld_optable* out) {
   if (!ctx || !out) return CCLD_ERR_ARG;
   WindowHost* w;

@@ -1841,11 +1841,10 @@ struct HangArgs {
   ccld_hang_verdict* out;    // device copy of the struct (pointer fields unused)
 };
 
-__global__ void __launch_bounds__(1024) k_hang_locate(const WinDesc* __restrict__ wd, Registry R, HangArgs A) {
+__device__ __forceinline__ void hang_locate_cta(const WinDesc& D, const Registry& R, const HangArgs& A) {
   __shared__ u64 s_red64[32];
   __shared__ u32 s_red32[32];
   __shared__ u32 s_base;
-  const WinDesc& D = wd[0];
   const u32 c = A.c, n = R.comm_n[c], cid = R.comm_id[c];
   const u32* mem = R.members + R.comm_moff[c];
   const RangeRow row = D.ranges[c];
@@ -1937,6 +1936,14 @@ __global__ void __launch_bounds__(1024) k_hang_locate(const WinDesc* __restrict_
     v.roots = nullptr; v.roots_cap = 0;
     *A.out = v;
   }
+}
+
+__global__ void __launch_bounds__(1024) k_hang_locate(const WinDesc* __restrict__ wd, Registry R, HangArgs A) { hang_locate_cta(wd[0], R, A); }
+
+// every alert of a window in one launch: one CTA per alert, each with its own scratch and output
+__global__ void __launch_bounds__(1024) k_hang_locate_many(const WinDesc* __restrict__ wd, Registry R, const HangArgs* __restrict__ args) {
+  const HangArgs A = args[blockIdx.x];
+  hang_locate_cta(wd[0], R, A);
 }
 
 // ------------------------------------------------------------------------------------------------

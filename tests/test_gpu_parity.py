@@ -318,3 +318,41 @@ def test_reset_reproduces_the_same_results():
     for w in range(2):
         compare_window(an, o, w)
     compare_cumulative(an, o, spec.n_ranks, 1)
+
+
+def test_hang_sweep_locates_every_alert_in_one_launch():
+    """Several hung communicators of different sizes, one per leaf of the decision tree (plus ties and missing frames):
+    ccld_locate_hangs returns, alert by alert, what the oracle and ccld_locate_hang return."""
+    C_ = 2
+    recs, comms, entries, r0 = [], [], [], 0
+    plan = [(6, "h1"), (40, "h3"), (8, "h2"), (130, "h3"), (5, "ok"), (12, "h3tie"), (9, "h1")]
+    for cid, (n, kind) in enumerate(plan):
+        ranks = list(range(r0, r0 + n)); r0 += n
+        comms.append((cid + 3, ranks, 0))
+        entered = set(range(n)) - ({1, n - 1} if kind == "h1" else set())
+        done = {2, 3} if kind == "h2" else (set(range(n)) if kind == "ok" else set())
+        for r in hang_records(n, 2 + cid, entered, done, ranks):
+            r["comm"] = cid + 3
+            recs.append(r)
+        if kind.startswith("h3"):
+            for i in range(n):
+                if kind == "h3" and i == n // 2: continue                      # a member without a frame counts as zero
+                v = 4 if (kind == "h3tie" and i in (3, 4, 5)) else 7
+                entries.append((ranks[i], cid + 3, 2 + cid, [(v, v - 1)] * C_))
+    an, o = hand_pair(recs, comms, frames=frames_from(entries, C_), n_channels=C_, now=10**9 + 400 * 10**9)
+    al = an.get_verdict(0)["alerts"]
+    assert len(al["comm"]) == 6                                                # every communicator but the completed one
+    sweep = an.locate_hangs(0, cap=16, roots_stride=256)
+    assert [(d["comm"], d["seq"]) for d in sweep] == list(zip(al["comm"].tolist(), al["seq"].tolist()))
+    for d in sweep:
+        b = o.locate_hang(0, d["comm"], d["seq"])
+        assert d["cls"] == b["cls"] and d["n_roots_total"] == b["n_roots"], (d, b)
+        for k in ("n_not_entered", "n_hung", "n_not_hung", "n_missing_frames", "stuck_step", "n_members", "min_total"):
+            assert d[k] == b[k], (k, d[k], b[k])
+        assert np.array_equal(d["roots"], b["roots"])
+        a = an.locate_hang(0, d["comm"], d["seq"])
+        assert a["cls"] == d["cls"] and np.array_equal(a["roots"], d["roots"])
+    assert sorted(d["cls"] for d in sweep) == [1, 1, 2, 3, 3, 3]
+    # truncation: fewer verdicts than alerts, short root lists
+    few = an.locate_hangs(0, cap=2, roots_stride=1)
+    assert len(few) == 2 and all(len(d["roots"]) <= 1 for d in few) and few[0]["n_roots_total"] == sweep[0]["n_roots_total"]
