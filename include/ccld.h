@@ -284,6 +284,21 @@ int ccld_get_ranges(ccld_ctx* ctx, uint32_t window_id, ccld_comm_range* rows /* 
 int ccld_get_rank_stats(ccld_ctx* ctx, uint32_t n_ranks, uint32_t* votes, uint32_t* ops, uint32_t* bw_cnt, double* bw_sum);
 
 /*
+ * Cumulative analyzer state as a host blob: per communicator the Eq. 1 baseline state (rounds seen, first enter time, sum of
+ * the first m T_max, m) and the repetition counter of slow detections (Sec. 4.2.1), per rank the vote counters, analysed-op
+ * counts and bus-bandwidth sums. An analyzer service that restarts, or hands a job to another GPU, exports the state and
+ * imports it into a context with the same communicators registered in the same order (ids, sizes and first counters are
+ * checked; member lists are the caller's responsibility), then goes on with the next window as if nothing had happened.
+ *   ccld_state_export: *n_bytes receives the blob size; with buf = NULL only the size is returned. cap < size with a
+ *     buffer gives CCLD_ERR_CAPACITY. Synchronizes the stream.
+ *   ccld_state_import: replaces the context's cumulative state; CCLD_ERR_ARG if the blob is malformed or belongs to
+ *     another set of communicators. Synchronizes the stream.
+ * Both fix the set of communicators (like the first ccld_analyze_window). Windows and their results are not part of it.
+ */
+int ccld_state_export(ccld_ctx* ctx, void* buf /* host */, uint64_t cap, uint64_t* n_bytes);
+int ccld_state_import(ccld_ctx* ctx, const void* buf /* host */, uint64_t n_bytes);
+
+/*
  * SendRate / RecvRate inputs from raw probe samples (Sec. 4.1.2: the rate is the reciprocal of the number of changes of
  * SendCount / RecvCount seen by a probe that samples at a fixed period; Sec. 5.2 step 2 has the host's diagnostic
  * thread derive it). This call does that step on the GPU and produces the send_chg / recv_chg columns that

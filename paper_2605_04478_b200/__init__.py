@@ -25,7 +25,7 @@ MAX_ALERTS_PER_WINDOW = 1024
 EXPORTS = ("ccld_params_default", "ccld_create", "ccld_destroy", "ccld_last_error", "ccld_comm_register",
            "ccld_trace_upload", "ccld_window_release", "ccld_analyze_window", "ccld_reset", "ccld_get_verdict",
            "ccld_locate_hang", "ccld_get_optable", "ccld_get_ranges", "ccld_get_rank_stats", "ccld_copy_to_host",
-           "ccld_timing_enable", "ccld_get_kernel_times", "ccld_ring_locate_static", "ccld_derive_rates", "ccld_locate_hangs")
+           "ccld_timing_enable", "ccld_get_kernel_times", "ccld_ring_locate_static", "ccld_derive_rates", "ccld_locate_hangs", "ccld_state_export", "ccld_state_import")
 STATIC_MAX_MEMBERS = 8192
 KERNEL_KINDS = ("k_seq_range", "k_plan", "k_slot_scatter", "k_reduce_fused", "k_reduce_mid", "k_reduce_large", "k_window_decide")
 
@@ -116,6 +116,8 @@ def load_library() -> C.CDLL:
         lib.ccld_reset.argtypes = [C.c_void_p]
         lib.ccld_get_verdict.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(Verdict)]
         lib.ccld_locate_hang.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.POINTER(HangVerdict)]
+        lib.ccld_state_export.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.POINTER(C.c_uint64)]
+        lib.ccld_state_import.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
         lib.ccld_locate_hangs.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.POINTER(C.c_uint32)]
         lib.ccld_get_optable.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(OpTable)]
         lib.ccld_get_ranges.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.POINTER(C.c_uint32)]
@@ -323,6 +325,18 @@ class Analyzer:
             d["comm"], d["seq"], d["age_ns"] = int(al[i].comm), int(al[i].seq), int(al[i].age_ns)
             res.append(d)
         return res
+
+    def state_export(self) -> bytes:
+        """ccld_state_export: the cumulative state (Eq. 1 baselines, repetition counters, per-rank votes and sums) as bytes."""
+        n = C.c_uint64(0)
+        self._check(self.lib.ccld_state_export(self.h, None, 0, C.byref(n)))
+        buf = (C.c_char * n.value)()
+        self._check(self.lib.ccld_state_export(self.h, C.cast(buf, C.c_void_p), n.value, C.byref(n)))
+        return bytes(buf)
+
+    def state_import(self, blob: bytes) -> None:
+        buf = (C.c_char * len(blob)).from_buffer_copy(blob)
+        self._check(self.lib.ccld_state_import(self.h, C.cast(buf, C.c_void_p), len(blob)))
 
     def get_ranges(self, window_id: int) -> Dict[str, np.ndarray]:
         n = C.c_uint32(0)

@@ -693,6 +693,51 @@ int ccld_get_rank_stats(ccld_ctx* ctx, uint32_t n_ranks, uint32_t* votes, uint32
   return CCLD_OK;
 }
 
+namespace {
+struct StateHeader { u64 magic; u32 version, n_comms, n_ranks, pad; u64 stats_bytes; };
+constexpr u64 STATE_MAGIC = 0x3130545344434343ull;    // "CCCDST01"
+}  // namespace
+
+int ccld_state_export(ccld_ctx* ctx, void* buf, uint64_t cap, uint64_t* n_bytes) {
+  if (!ctx || !n_bytes) return CCLD_ERR_ARG;
+  CK(cudaSetDevice(ctx->device));
+  { int rc = finalize_registry(ctx); if (rc != CCLD_OK) return rc; }
+  const u32 nc = ctx->reg.n_comms;
+  const u64 need = sizeof(StateHeader) + (u64)nc * 12 + ctx->stats_bytes;
+  *n_bytes = need;
+  if (!buf || cap < need) return buf ? fail(ctx, CCLD_ERR_CAPACITY, "state buffer too small") : CCLD_OK;
+  char* p = (char*)buf;
+  StateHeader h{STATE_MAGIC, 1u, nc, ctx->n_ranks, 0u, (u64)ctx->stats_bytes};
+  std::memcpy(p, &h, sizeof h); p += sizeof h;
+  for (u32 c = 0; c < nc; ++c) { const u32 row[3] = {ctx->comms[c].id, (u32)ctx->comms[c].ranks.size(), ctx->comms[c].seq0}; std::memcpy(p, row, 12); p += 12; }
+  CK(cudaMemcpyAsync(p, (char*)ctx->reg_blk.p + ctx->stats_off, ctx->stats_bytes, cudaMemcpyDeviceToHost, ctx->stream));
+  CK(cudaStreamSynchronize(ctx->stream));
+  return CCLD_OK;
+}
+
+int ccld_state_import(ccld_ctx* ctx, const void* buf, uint64_t n_bytes) {
+  if (!ctx || !buf) return CCLD_ERR_ARG;
+  CK(cudaSetDevice(ctx->device));
+  { int rc = finalize_registry(ctx); if (rc != CCLD_OK) return rc; }
+  const u32 nc = ctx->reg.n_comms;
+  StateHeader h;
+  if (n_bytes < sizeof h) return fail(ctx, CCLD_ERR_ARG, "state blob too short");
+  std::memcpy(&h, buf, sizeof h);
+  if (h.magic != STATE_MAGIC || h.version != 1) return fail(ctx, CCLD_ERR_ARG, "not a state blob of this library version");
+  if (h.n_comms != nc || h.n_ranks != ctx->n_ranks || h.stats_bytes != ctx->stats_bytes || n_bytes != sizeof h + (u64)nc * 12 + h.stats_bytes)
+    return fail(ctx, CCLD_ERR_ARG, "state blob belongs to another set of communicators");
+  const char* p = (const char*)buf + sizeof h;
+  for (u32 c = 0; c < nc; ++c) {
+    u32 row[3]; std::memcpy(row, p, 12); p += 12;
+    if (row[0] != ctx->comms[c].id || row[1] != (u32)ctx->comms[c].ranks.size() || row[2] != ctx->comms[c].seq0)
+      return fail(ctx, CCLD_ERR_ARG, "state blob belongs to another set of communicators");
+  }
+  CK(cudaStreamSynchronize(ctx->stream));
+  CK(cudaMemcpyAsync((char*)ctx->reg_blk.p + ctx->stats_off, p, ctx->stats_bytes, cudaMemcpyHostToDevice, ctx->stream));
+  CK(cudaStreamSynchronize(ctx->stream));
+  return CCLD_OK;
+}
+
 int ccld_derive_rates(ccld_ctx* ctx, uint64_t n_rec, const uint32_t* rank, const int64_t* t_enter_ns, const int64_t* t_exit_ns,
                       uint32_t n_ranks, uint64_t n_ticks, const uint64_t* tick_off, const int64_t* tick_ns,
                       const uint32_t* send_count, const uint32_t* recv_count, uint32_t* send_chg, uint32_t* recv_chg) {

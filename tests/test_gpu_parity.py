@@ -7,6 +7,8 @@ import numpy as np
 import pytest
 import torch
 
+import oracle as orc
+import paper_2605_04478_b200 as ccld
 import tracegen as tg
 from helpers import ALLGATHER, MiB, frames_from, group_trace, make_cols
 from parity import compare_cumulative, compare_hang, compare_window, make_pair
@@ -356,3 +358,35 @@ def test_hang_sweep_locates_every_alert_in_one_launch():
     # truncation: fewer verdicts than alerts, short root lists
     few = an.locate_hangs(0, cap=2, roots_stride=1)
     assert len(few) == 2 and all(len(d["roots"]) <= 1 for d in few) and few[0]["n_roots_total"] == sweep[0]["n_roots_total"]
+
+
+def test_state_export_import_continues_on_another_context():
+    """Two windows on one analyzer, its state exported and imported into a fresh one, two more windows there: the second
+    analyzer's windows, cumulative votes and suspects equal an oracle that saw all four windows in one life."""
+    spec = tg.cfg2(reps=30, n_windows=4, tp=8, pp=2, dp=4)
+    an_a, an_b, o = ccld.Analyzer(), ccld.Analyzer(), orc.Oracle()
+    for cid, ranks, seq0 in tg.registry(spec):
+        an_a.comm_register(cid, ranks, 0, seq0); an_b.comm_register(cid, ranks, 0, seq0); o.comm_register(cid, ranks, seq0)
+    wins = [tg.gen_window(spec, w, device="cuda") for w in range(4)]
+    for w in range(4):
+        (an_a if w < 2 else an_b).trace_upload(w, wins[w].cols)
+        o.upload(w, wins[w].cols)
+    now = wins[-1].now_ns
+    an_a.analyze_window(0, 2, now)
+    blob = an_a.state_export()
+    an_b.state_import(blob)
+    an_b.analyze_window(2, 2, now)
+    o.analyze(0, 4, now)
+    for w in (0, 1):
+        compare_window(an_a, o, w)
+    for w in (2, 3):
+        compare_window(an_b, o, w)
+    compare_cumulative(an_b, o, spec.n_ranks, 3)
+    assert an_b.state_export() != blob
+    # a blob of another set of communicators is refused
+    an_c = ccld.Analyzer()
+    an_c.comm_register(0, [0, 1, 2, 3], 0, 0)
+    with pytest.raises(ccld.CcldError):
+        an_c.state_import(blob)
+    with pytest.raises(ccld.CcldError):
+        an_b.state_import(blob[:-8])
