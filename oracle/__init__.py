@@ -43,7 +43,7 @@ def _load():
         _lib.orc_destroy.argtypes = [C.c_void_p]
         for name in ("orc_comm_register", "orc_upload", "orc_release", "orc_analyze", "orc_window_sizes",
                      "orc_copy_groups", "orc_copy_slots", "orc_copy_comm_rows", "orc_copy_alerts",
-                     "orc_copy_rank_stats", "orc_suspects", "orc_locate_hang"):
+                     "orc_copy_rank_stats", "orc_suspects", "orc_locate_hang", "orc_attach_opset", "orc_opset_check"):
             getattr(_lib, name).restype = C.c_int
         _lib.orc_derive_rates.restype = None
     return _lib
@@ -155,6 +155,19 @@ class Oracle:
         n = self.lib.orc_suspects(self.h, C.c_uint32(cap), _p(kind), _p(rank), _p(votes), _p(ops), _p(bw))
         m = min(n, cap)
         return {"n_total": n, "kind": kind[:m], "rank": rank[:m], "votes": votes[:m], "ops": ops[:m], "mean_busbw": bw[:m]}
+
+    def attach_opset(self, window_id: int, algo, proto) -> int:
+        a = _np(algo, np.uint8); b = _np(proto, np.uint8)
+        return self.lib.orc_attach_opset(self.h, C.c_uint32(window_id), _p(a), _p(b))
+
+    def opset_check(self, window_id: int, comm: int, seq: int, cap: int = 65536) -> Dict[str, object]:
+        out = np.zeros(7, np.uint32); by = np.zeros(1, np.uint64); ranks = np.zeros(cap, np.uint32)
+        rc = self.lib.orc_opset_check(self.h, C.c_uint32(window_id), C.c_uint32(comm), C.c_uint32(seq), _p(out), _p(by), C.c_uint32(cap), _p(ranks))
+        assert rc == 0
+        d = {k: int(v) for k, v in zip(("n_members", "n_present", "n_deviating_total", "majority_count", "op", "algo", "proto"), out)}
+        d["bytes"] = int(by[0])
+        d["ranks"] = ranks[:min(d["n_deviating_total"], cap)].copy()
+        return d
 
     def locate_hang(self, window_id: int, comm: int, seq: int, cap: int = 65536) -> Dict[str, object]:
         out = np.zeros(8, np.uint32); mn = np.zeros(1, np.uint64); roots = np.zeros(cap, np.uint32)

@@ -15,6 +15,8 @@
 // decision tree, brute-force order statistics by counting, and invariants.
 // orc_derive_rates (counter changes per op from raw probe samples) is pinned to the same worked example, to closed
 // forms for a counter that advances every tick, to additivity over adjacent ops and to a numpy restatement.
+// orc_opset_check (majority Operation Type Set of an op and the ranks that deviate) is pinned to hand cases and to a
+// collections.Counter restatement.
 // "Parity unpinned" against the paper: the bus-bandwidth factor and the median/MAD convention,
 // because the paper defines neither (they are this repository's conventions, pinned only to
 // closed forms and hand values).
@@ -77,7 +79,7 @@ struct RankStat { u32 v[4] = {0, 0, 0, 0}; u32 ops = 0, bw_cnt = 0; double bw_su
 
 struct Window {
   u64 n = 0;
-  std::vector<u32> rank, comm, seq, send_chg, recv_chg; std::vector<u8> op; std::vector<u64> bytes; std::vector<i64> t_enter, t_exit;
+  std::vector<u32> rank, comm, seq, send_chg, recv_chg; std::vector<u8> op, algo, proto; std::vector<u64> bytes; std::vector<i64> t_enter, t_exit;
   u32 n_frames = 0, n_channels = 0; std::vector<u32> f_rank, f_comm, f_seq, progress;
   bool analysed = false;
   // results
@@ -485,6 +487,53 @@ int orc_locate_hang(void* h, u32 wid, u32 comm, u32 seq, u32* out, u64* min_tota
   }
   out[0] = cls; out[1] = (u32)r.size(); out[2] = n_ne; out[3] = n_hung; out[4] = n_ok; out[5] = n_missing; out[6] = stuck; out[7] = n;
   for (size_t i = 0; i < r.size() && i < cap; ++i) roots[i] = r[i];
+  return 0;
+}
+
+// Operation Type Set (Sec. 4.1.2: algorithm, protocol, data size and operation name, constant during a communication;
+// Sec. 4.2.2: inconsistent operations are what the not-hung ranks of leaf H2 point at). The two extra columns are
+// attached per record; without them algorithm and protocol count as 0.
+int orc_attach_opset(void* h, u32 wid, const u8* algo, const u8* proto) {
+  Oracle* o = (Oracle*)h;
+  auto wi = o->windows.find(wid);
+  if (wi == o->windows.end()) return -1;
+  Window& w = wi->second;
+  w.algo.assign(algo, algo + w.n); w.proto.assign(proto, proto + w.n);
+  return 0;
+}
+
+// For op (comm, seq): the most frequent (op, bytes, algo, proto) among the members that reported it - ties go to the
+// tuple whose first holder stands earliest in the ring - and the members that carry another tuple, in ring order.
+// out = {n_members, n_present, n_deviating, majority_count, op, algo, proto}; the first record of a member counts.
+int orc_opset_check(void* h, u32 wid, u32 comm, u32 seq, u32* out, u64* bytes_out, u32 cap, u32* ranks) {
+  Oracle* o = (Oracle*)h;
+  auto wi = o->windows.find(wid); auto ci = o->comm_idx.find(comm);
+  if (wi == o->windows.end() || ci == o->comm_idx.end()) return -1;
+  Window& w = wi->second; Comm& c = o->comms[ci->second];
+  const u32 n = (u32)c.ranks.size();
+  std::vector<long> rec(n, -1);
+  for (u64 i = 0; i < w.n; ++i) {
+    if (w.comm[i] != comm || w.seq[i] != seq) continue;
+    auto pi = c.pos.find(w.rank[i]);
+    if (pi != c.pos.end() && rec[pi->second] < 0) rec[pi->second] = (long)i;
+  }
+  auto same = [&](long a, long b) {
+    return w.op[a] == w.op[b] && w.bytes[a] == w.bytes[b] && (w.algo.empty() || (w.algo[a] == w.algo[b] && w.proto[a] == w.proto[b]));
+  };
+  u32 n_present = 0, best_cnt = 0; long best = -1;
+  for (u32 p = 0; p < n; ++p) {
+    if (rec[p] < 0) continue;
+    ++n_present;
+    u32 cnt = 0;
+    for (u32 q = 0; q < n; ++q) if (rec[q] >= 0 && same(rec[p], rec[q])) ++cnt;
+    if (cnt > best_cnt) { best_cnt = cnt; best = rec[p]; }      // positions ascend: the earliest holder wins ties
+  }
+  std::vector<u32> dev;
+  for (u32 p = 0; p < n; ++p) if (rec[p] >= 0 && !same(rec[p], best)) dev.push_back(c.ranks[p]);
+  out[0] = n; out[1] = n_present; out[2] = (u32)dev.size(); out[3] = best_cnt;
+  out[4] = best >= 0 ? w.op[best] : 0; out[5] = best >= 0 && !w.algo.empty() ? w.algo[best] : 0; out[6] = best >= 0 && !w.proto.empty() ? w.proto[best] : 0;
+  *bytes_out = best >= 0 ? w.bytes[best] : 0;
+  for (size_t i = 0; i < dev.size() && i < cap; ++i) ranks[i] = dev[i];
   return 0;
 }
 

@@ -570,3 +570,67 @@ def test_derived_rates_against_a_numpy_restatement():
         inside = (t[1:] > te[i]) & ((t[1:] <= tx[i]) | (tx[i] == -1))
         assert s[i] == int((np.diff(sc[lo:hi].astype(np.int64))[inside] != 0).sum())
         assert r[i] == int((np.diff(rc[lo:hi].astype(np.int64))[inside] != 0).sum())
+
+
+# ---------------------------------------------------------------- Operation Type Set consistency (Sec. 4.1.2, Sec. 4.2.2)
+def _opset_oracle(recs, comms, algo=None, proto=None):
+    o = orc.Oracle()
+    for cid, ranks, seq0 in comms:
+        assert o.comm_register(cid, ranks, seq0) == 0
+    assert o.upload(0, make_cols(recs)) == 0
+    if algo is not None:
+        assert o.attach_opset(0, algo, proto) == 0
+    return o
+
+
+def test_opset_majority_hand_cases():
+    ranks = [20, 21, 22, 23, 24, 25]
+    recs = group_trace([[5] * 6] * 3, ranks=ranks)                                 # three ops, everyone agrees
+    o = _opset_oracle(recs, [(0, ranks, 0)])
+    r = o.opset_check(0, 0, 1)
+    assert (r["n_members"], r["n_present"], r["n_deviating_total"], r["majority_count"]) == (6, 6, 0, 6) and r["bytes"] == 16 * MiB
+    # one rank issues another size, one another operation, one has not reported: two deviants, ring order
+    recs2 = [dict(x) for x in recs if not (x["seq"] == 1 and x["rank"] == 25)]
+    for x in recs2:
+        if x["seq"] == 1 and x["rank"] == 23: x["bytes"] = 8 * MiB
+        if x["seq"] == 1 and x["rank"] == 21: x["op"] = ALLGATHER
+    r = _opset_oracle(recs2, [(0, ranks, 0)]).opset_check(0, 0, 1)
+    assert (r["n_present"], r["n_deviating_total"], r["majority_count"], r["op"]) == (5, 2, 3, ALLREDUCE) and list(r["ranks"]) == [21, 23]
+    # algorithm / protocol columns: same op and size, two ranks on another protocol
+    algo = np.zeros(len(recs), np.uint8); proto = np.zeros(len(recs), np.uint8)
+    for i, x in enumerate(recs):
+        if x["seq"] == 2 and x["rank"] in (20, 24): proto[i] = 2
+    r = _opset_oracle(recs, [(0, ranks, 0)], algo, proto).opset_check(0, 0, 2)
+    assert r["n_deviating_total"] == 2 and list(r["ranks"]) == [20, 24] and r["proto"] == 0 and r["majority_count"] == 4
+    # a tie goes to the tuple whose first holder stands earliest in the ring: positions 0-2 against 3-5
+    for i, x in enumerate(recs):
+        proto[i] = 1 if (x["seq"] == 0 and x["rank"] >= 23) else proto[i]
+    r = _opset_oracle(recs, [(0, ranks, 0)], algo, proto).opset_check(0, 0, 0)
+    assert r["majority_count"] == 3 and r["proto"] == 0 and list(r["ranks"]) == [23, 24, 25]
+    # an op nobody reported
+    r = o.opset_check(0, 0, 9)
+    assert (r["n_present"], r["n_deviating_total"], r["majority_count"]) == (0, 0, 0)
+
+
+def test_opset_majority_against_a_counter_restatement():
+    from collections import Counter
+    rng = np.random.default_rng(31)
+    n = 40
+    ranks = list(rng.permutation(200)[:n].astype(int))
+    recs = group_trace([[5] * n] * 6, ranks=ranks)
+    for x in recs:
+        x["op"] = int(rng.integers(0, 2)); x["bytes"] = int(rng.choice([4, 8])) * MiB
+    keep = rng.random(len(recs)) > 0.1
+    recs = [x for x, k in zip(recs, keep) if k]
+    algo = rng.integers(0, 2, len(recs)).astype(np.uint8); proto = rng.integers(0, 2, len(recs)).astype(np.uint8)
+    o = _opset_oracle(recs, [(0, ranks, 0)], algo, proto)
+    for s in range(6):
+        tup = {}
+        for i, x in enumerate(recs):
+            if x["seq"] == s: tup[x["rank"]] = (x["op"], x["bytes"], int(algo[i]), int(proto[i]))
+        cnt = Counter(tup.values())
+        top = max(cnt.values())
+        maj = next(tup[r] for r in ranks if r in tup and cnt[tup[r]] == top)
+        r = o.opset_check(0, 0, s)
+        assert (r["op"], r["bytes"], r["algo"], r["proto"]) == maj and r["majority_count"] == top and r["n_present"] == len(tup)
+        assert list(r["ranks"]) == [q for q in ranks if q in tup and tup[q] != maj]
