@@ -284,6 +284,28 @@ int ccld_get_ranges(ccld_ctx* ctx, uint32_t window_id, ccld_comm_range* rows /* 
 int ccld_get_rank_stats(ccld_ctx* ctx, uint32_t n_ranks, uint32_t* votes, uint32_t* ops, uint32_t* bw_cnt, double* bw_sum);
 
 /*
+ * Operation Type Set consistency (Sec. 4.1.2: each rank records the communication algorithm, protocol, data size and
+ * operation name of an op, which stay constant during the communication; Sec. 4.2.2: inconsistent operations are the
+ * cause that the not-hung ranks of hang leaf H2 point at).
+ *   ccld_trace_attach_opset adds the two columns that ccld_trace_upload does not take - algorithm and protocol codes per
+ *     record, in the order of the uploaded columns, n_rec entries each; host memory is copied, device memory borrowed
+ *     until the window is released. Without it both count as 0. The window must have been uploaded.
+ *   ccld_opset_check, for op (comm, seq) of an analysed window: the most frequent (op, bytes, algo, proto) among the
+ *     members that reported the op - ties go to the tuple whose first holder stands earliest in the ring - how many
+ *     members carry it, and the ranks that carry another tuple, in ring order, up to ranks_cap of them into out->ranks
+ *     (host, caller-allocated, may be NULL). Synchronizes the stream.
+ */
+typedef struct {
+  uint32_t n_members, n_present, n_deviating_total, majority_count;
+  uint8_t op, algo, proto, pad;  /* the majority tuple (zeros if no member reported the op) */
+  uint64_t bytes;
+  uint32_t* ranks; uint32_t ranks_cap;
+} ccld_opset_verdict;
+
+int ccld_trace_attach_opset(ccld_ctx* ctx, uint32_t window_id, int mem_kind, const uint8_t* algo, const uint8_t* proto);
+int ccld_opset_check(ccld_ctx* ctx, uint32_t window_id, uint32_t comm, uint32_t seq, ccld_opset_verdict* out /* host */);
+
+/*
  * Cumulative analyzer state as a host blob: per communicator the Eq. 1 baseline state (rounds seen, first enter time, sum of
  * the first m T_max, m) and the repetition counter of slow detections (Sec. 4.2.1), per rank the vote counters, analysed-op
  * counts and bus-bandwidth sums. An analyzer service that restarts, or hands a job to another GPU, exports the state and

@@ -25,7 +25,7 @@ MAX_ALERTS_PER_WINDOW = 1024
 EXPORTS = ("ccld_params_default", "ccld_create", "ccld_destroy", "ccld_last_error", "ccld_comm_register",
            "ccld_trace_upload", "ccld_window_release", "ccld_analyze_window", "ccld_reset", "ccld_get_verdict",
            "ccld_locate_hang", "ccld_get_optable", "ccld_get_ranges", "ccld_get_rank_stats", "ccld_copy_to_host",
-           "ccld_timing_enable", "ccld_get_kernel_times", "ccld_ring_locate_static", "ccld_derive_rates", "ccld_locate_hangs", "ccld_state_export", "ccld_state_import")
+           "ccld_timing_enable", "ccld_get_kernel_times", "ccld_ring_locate_static", "ccld_derive_rates", "ccld_locate_hangs", "ccld_state_export", "ccld_state_import", "ccld_trace_attach_opset", "ccld_opset_check")
 STATIC_MAX_MEMBERS = 8192
 KERNEL_KINDS = ("k_seq_range", "k_plan", "k_slot_scatter", "k_reduce_fused", "k_reduce_mid", "k_reduce_large", "k_window_decide")
 
@@ -78,6 +78,12 @@ OPTABLE_I64 = ("e_min", "arrival_skew", "t_max", "t_min", "span", "med_skew", "m
 OPTABLE_U32 = ("rank_tmin", "rank_tmax", "max_chg", "rank_max_chg", "n_present", "gflags")
 
 
+class OpsetVerdict(C.Structure):
+    _fields_ = [(k, C.c_uint32) for k in ("n_members", "n_present", "n_deviating_total", "majority_count")] + \
+               [(k, C.c_uint8) for k in ("op", "algo", "proto", "pad")] + \
+               [("bytes", C.c_uint64), ("ranks", C.POINTER(C.c_uint32)), ("ranks_cap", C.c_uint32)]
+
+
 class OpTable(C.Structure):
     _fields_ = [("n_groups", C.c_uint64), ("n_slots", C.c_uint64)] + [(k, C.c_void_p) for k in OPTABLE_I64] + \
                [(k, C.c_void_p) for k in OPTABLE_U32] + [("busbw", C.c_void_p), ("flags", C.c_void_p), ("perm", C.c_void_p)]
@@ -116,6 +122,8 @@ def load_library() -> C.CDLL:
         lib.ccld_reset.argtypes = [C.c_void_p]
         lib.ccld_get_verdict.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(Verdict)]
         lib.ccld_locate_hang.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.POINTER(HangVerdict)]
+        lib.ccld_trace_attach_opset.argtypes = [C.c_void_p, C.c_uint32, C.c_int, C.c_void_p, C.c_void_p]
+        lib.ccld_opset_check.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.POINTER(OpsetVerdict)]
         lib.ccld_state_export.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.POINTER(C.c_uint64)]
         lib.ccld_state_import.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64]
         lib.ccld_locate_hangs.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.POINTER(C.c_uint32)]
@@ -265,6 +273,7 @@ class Analyzer:
     def window_release(self, window_id: int) -> None:
         self._check(self.lib.ccld_window_release(self.h, window_id))
         self._keep.pop(window_id, None)
+        self._keep.pop(("opset", window_id), None)
 
     def analyze_window(self, first_window: int, n_windows: int, now_ns: int) -> None:
         self._check(self.lib.ccld_analyze_window(self.h, first_window, n_windows, now_ns))
@@ -325,6 +334,26 @@ class Analyzer:
             d["comm"], d["seq"], d["age_ns"] = int(al[i].comm), int(al[i].seq), int(al[i].age_ns)
             res.append(d)
         return res
+
+    def trace_attach_opset(self, window_id: int, algo, proto) -> None:
+        """ccld_trace_attach_opset: algorithm and protocol codes per record (uint8), host (copied) or this GPU (borrowed)."""
+        torch = self.torch
+        a = _as_tensor(torch, algo, "uint8").contiguous(); b = _as_tensor(torch, proto, "uint8").contiguous()
+        assert a.device.type == b.device.type
+        self._check(self.lib.ccld_trace_attach_opset(self.h, window_id, 1 if a.device.type == "cuda" else 0,
+                                                     C.c_void_p(a.data_ptr()), C.c_void_p(b.data_ptr())))
+        self._keep.setdefault(("opset", window_id), []).append((a, b))
+
+    def opset_check(self, window_id: int, comm: int, seq: int, ranks_cap: int = MAX_COMM_SIZE) -> Dict[str, object]:
+        """ccld_opset_check: majority Operation Type Set of op (comm, seq) and the ranks that deviate from it."""
+        ranks = (C.c_uint32 * max(ranks_cap, 1))()
+        v = OpsetVerdict()
+        v.ranks = C.cast(ranks, C.POINTER(C.c_uint32)); v.ranks_cap = ranks_cap
+        self._check(self.lib.ccld_opset_check(self.h, window_id, comm, seq, C.byref(v)))
+        out: Dict[str, object] = {k: int(getattr(v, k)) for k in ("n_members", "n_present", "n_deviating_total", "majority_count",
+                                                                "op", "algo", "proto", "bytes")}
+        out["ranks"] = np.array(ranks[:min(v.n_deviating_total, ranks_cap)], dtype=np.uint32)
+        return out
 
     def state_export(self) -> bytes:
         """ccld_state_export: the cumulative state (Eq. 1 baselines, repetition counters, per-rank votes and sums) as bytes."""

@@ -13,6 +13,7 @@
 
 #include "ccld_kernels.cuh"
 #include "ccld_rates.cuh"
+#include "ccld_opset.cuh"
 
 using namespace ccld;
 
@@ -59,6 +60,7 @@ struct WindowHost {
   WinDesc d;                                    // device pointers
   u32 n_frames = 0, n_channels = 0;
   const u32 *f_rank = nullptr, *f_comm = nullptr, *f_seq = nullptr, *progress = nullptr;
+  const u8 *algo = nullptr, *proto = nullptr; bool owns_opset = false; Block opset_own;   // Operation Type Set columns
   bool analysed = false;
   std::shared_ptr<Shared> plan_blk, res_blk;
   WinDesc* d_desc = nullptr;                    // this window's descriptor on the device
@@ -361,6 +363,7 @@ int ccld_window_release(ccld_ctx* ctx, uint32_t window_id) {
   CK(cudaStreamSynchronize(ctx->stream));     // nothing in flight may still read the blocks we recycle
   drop_results(it->second);
   if (it->second.owns) ctx->pool.put(it->second.own);
+  if (it->second.owns_opset) ctx->pool.put(it->second.opset_own);
   ctx->windows.erase(it);
   return CCLD_OK;
 }
@@ -690,6 +693,63 @@ int ccld_get_rank_stats(ccld_ctx* ctx, uint32_t n_ranks, uint32_t* votes, uint32
   CK(cudaMemcpyAsync(bw_cnt, ctx->reg.bw_cnt, (size_t)n * 4, cudaMemcpyDeviceToHost, st));
   CK(cudaMemcpyAsync(bw_sum, ctx->reg.bw_sum, (size_t)n * 8, cudaMemcpyDeviceToHost, st));
   CK(cudaStreamSynchronize(st));
+  return CCLD_OK;
+}
+
+int ccld_trace_attach_opset(ccld_ctx* ctx, uint32_t window_id, int mem_kind, const uint8_t* algo, const uint8_t* proto) {
+  if (!ctx) return CCLD_ERR_ARG;
+  if (mem_kind != 0 && mem_kind != 1) return fail(ctx, CCLD_ERR_ARG, "mem_kind must be 0 (host) or 1 (device)");
+  auto it = ctx->windows.find(window_id);
+  if (it == ctx->windows.end()) return fail(ctx, CCLD_ERR_NO_WINDOW, "unknown window id");
+  WindowHost& w = it->second;
+  if (w.n_rec > 0 && (!algo || !proto)) return fail(ctx, CCLD_ERR_ARG, "null column");
+  CK(cudaSetDevice(ctx->device));
+  if (w.owns_opset) { CK(cudaStreamSynchronize(ctx->stream)); ctx->pool.put(w.opset_own); w.owns_opset = false; }
+  if (mem_kind == 1 || w.n_rec == 0) { w.algo = algo; w.proto = proto; return CCLD_OK; }
+  cudaError_t e;
+  const size_t half = align_up(w.n_rec);
+  w.opset_own = ctx->pool.get(2 * half, &e);
+  if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "window allocation failed");
+  w.owns_opset = true;
+  char* b = (char*)w.opset_own.p;
+  CK(cudaMemcpyAsync(b, algo, w.n_rec, cudaMemcpyHostToDevice, ctx->stream));
+  CK(cudaMemcpyAsync(b + half, proto, w.n_rec, cudaMemcpyHostToDevice, ctx->stream));
+  CK(cudaStreamSynchronize(ctx->stream));       // the caller's host arrays are free again
+  w.algo = (const u8*)b; w.proto = (const u8*)(b + half);
+  return CCLD_OK;
+}
+
+int ccld_opset_check(ccld_ctx* ctx, uint32_t window_id, uint32_t comm, uint32_t seq, ccld_opset_verdict* out) {
+  if (!ctx || !out) return CCLD_ERR_ARG;
+  WindowHost* w;
+  { int rc = find_analysed(ctx, window_id, &w); if (rc != CCLD_OK) return rc; }
+  auto ci = ctx->comm_idx.find(comm);
+  if (ci == ctx->comm_idx.end()) return fail(ctx, CCLD_ERR_UNKNOWN_COMM, "unknown communicator");
+  CK(cudaSetDevice(ctx->device));
+  cudaStream_t st = ctx->stream;
+  const u32 n = (u32)ctx->comms[ci->second].ranks.size();
+  size_t off = 0;
+  auto take = [&](size_t b) { size_t o = off; off = align_up(off + b); return o; };
+  const size_t o_hi = take(n * 8ull), o_lo = take(n * 4ull), o_rk = take(n * 4ull), o_out = take(sizeof(ccld_opset_verdict));
+  cudaError_t e;
+  Block blk = ctx->pool.get(off, &e);
+  if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "scratch allocation failed");
+  char* b = (char*)blk.p;
+  OpsetArgs A; A.c = ci->second; A.seq = seq; A.algo = w->algo; A.proto = w->proto;
+  A.key_hi = (u64*)(b + o_hi); A.key_lo = (u32*)(b + o_lo); A.ranks = (u32*)(b + o_rk); A.ranks_cap = n; A.out = (ccld_opset_verdict*)(b + o_out);
+  k_opset_check<<<1, 1024, 0, st>>>(w->d_desc, ctx->reg, A);
+  ccld_opset_verdict v;
+  u32* ranks = out->ranks; const u32 cap = ranks ? out->ranks_cap : 0;
+  int rc = CCLD_OK;
+  if (cudaGetLastError() != cudaSuccess || cudaMemcpyAsync(&v, A.out, sizeof v, cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) rc = CCLD_ERR_CUDA;
+  if (rc == CCLD_OK) {
+    *out = v; out->ranks = ranks; out->ranks_cap = cap;
+    const u32 n_copy = std::min<u32>(std::min<u32>(v.n_deviating_total, n), cap);
+    if (n_copy && (cudaMemcpyAsync(ranks, A.ranks, n_copy * 4ull, cudaMemcpyDeviceToHost, st) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess)) rc = CCLD_ERR_CUDA;
+  }
+  ctx->pool.put(blk);
+  if (rc != CCLD_OK) return fail(ctx, rc, "op-set check failed");
   return CCLD_OK;
 }
 

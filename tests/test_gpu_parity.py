@@ -390,3 +390,43 @@ def test_state_export_import_continues_on_another_context():
         an_c.state_import(blob)
     with pytest.raises(ccld.CcldError):
         an_b.state_import(blob[:-8])
+
+
+def test_opset_consistency_against_the_oracle():
+    """Majority Operation Type Set and deviating ranks for groups of every kernel class, with and without the algorithm /
+    protocol columns, with missing members, ties, an op nobody reported and an op outside the window's range."""
+    rng = np.random.default_rng(41)
+    recs, comms, r0 = [], [], 0
+    for cid, n in enumerate((6, 40, 130, 1100)):
+        ranks = list(range(r0, r0 + n)); r0 += n
+        comms.append((cid, ranks, 0))
+        g = group_trace([[5] * n] * 5, comm=cid, ranks=ranks)
+        for x in g:
+            if x["seq"] >= 1:
+                x["op"] = int(rng.choice([0, 0, 0, 1])); x["bytes"] = int(rng.choice([4, 4, 4, 8])) * MiB
+        if cid == 0:
+            for x in g:
+                if x["seq"] == 4: x["bytes"] = (4 if x["rank"] < ranks[3] else 8) * MiB       # a three-against-three tie
+        keep = rng.random(len(g)) > 0.05
+        recs += [x for x, k in zip(g, keep) if k or x["seq"] == 0]
+    recs = [x for x in recs if not (x["comm"] == 1 and x["seq"] == 3)]                        # an op nobody reported
+    an, o = hand_pair(recs, comms)
+    keys = ("n_members", "n_present", "n_deviating_total", "majority_count", "op", "algo", "proto", "bytes")
+
+    def check():
+        for cid, ranks, _ in comms:
+            for s in (0, 1, 2, 3, 4, 9):
+                a, b = an.opset_check(0, cid, s), o.opset_check(0, cid, s)
+                assert [a[k] for k in keys] == [b[k] for k in keys], (cid, s, a, b)
+                assert np.array_equal(a["ranks"], b["ranks"]), (cid, s)
+        short = an.opset_check(0, 3, 2, ranks_cap=3)
+        assert len(short["ranks"]) == 3 and short["n_deviating_total"] == o.opset_check(0, 3, 2)["n_deviating_total"]
+
+    check()
+    assert an.opset_check(0, 0, 0)["n_deviating_total"] == 0 and an.opset_check(0, 3, 1)["n_deviating_total"] > 100
+    algo = rng.integers(0, 2, len(recs)).astype(np.uint8); proto = (rng.random(len(recs)) < 0.1).astype(np.uint8)
+    an.trace_attach_opset(0, algo, proto); assert o.attach_opset(0, algo, proto) == 0
+    check()
+    an.trace_attach_opset(0, torch.from_numpy(proto).cuda(), torch.from_numpy(algo).cuda())   # device columns, swapped
+    assert o.attach_opset(0, proto, algo) == 0
+    check()
