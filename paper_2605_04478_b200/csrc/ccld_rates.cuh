@@ -106,12 +106,15 @@ __global__ void __launch_bounds__(RT_THREADS) k_tick_sums(TickArgs A) {
 __global__ void __launch_bounds__(RT_THREADS) k_tile_scan(u64* __restrict__ tile_sum, u64 n_tiles) {
   __shared__ u64 s_warp[RT_THREADS / 32 + 1];
   u64 carry = 0;
-  for (u64 base = 0; base < n_tiles; base += RT_THREADS) {
-    const u64 i = base + threadIdx.x;
-    const u64 v = i < n_tiles ? tile_sum[i] : 0;
+  for (u64 base = 0; base < n_tiles; base += RT_TILE) {          // RT_PER consecutive sums per thread and round
+    const u64 i0 = base + (u64)threadIdx.x * RT_PER;
+    u64 v[RT_PER], sum = 0;
+#pragma unroll
+    for (int k = 0; k < RT_PER; ++k) { v[k] = i0 + k < n_tiles ? tile_sum[i0 + k] : 0; sum += v[k]; }
     u64 total;
-    const u64 ex = cta_exclusive_scan(v, &total, s_warp);
-    if (i < n_tiles) tile_sum[i] = carry + ex;
+    u64 run = carry + cta_exclusive_scan(sum, &total, s_warp);
+#pragma unroll
+    for (int k = 0; k < RT_PER; ++k) { if (i0 + k < n_tiles) tile_sum[i0 + k] = run; run += v[k]; }
     carry += total;
   }
 }
@@ -142,6 +145,14 @@ __device__ __forceinline__ u64 ticks_upto(const i64* __restrict__ tn, u64 lo, u6
   return a - lo;
 }
 
+// the same count when it is expected to be small (an op spans a few ticks): doubling steps from lo, then bisection
+__device__ __forceinline__ u64 ticks_upto_near(const i64* __restrict__ tn, u64 lo, u64 hi, i64 t) {
+  u64 pos = lo, bound = 1;                          // every tick of [lo, pos) is at or before t
+  for (int step = 0; step < 64 && pos + bound - 1 < hi && __ldg(tn + pos + bound - 1) <= t; ++step) { pos += bound; bound <<= 1; }
+  const u64 end = pos + bound - 1 < hi ? pos + bound - 1 : hi;
+  return (pos - lo) + ticks_upto(tn, pos, end, t);
+}
+
 __global__ void __launch_bounds__(RT_THREADS) k_record_rates(TickArgs A, u64 n_rec, const u32* __restrict__ rank, const i64* __restrict__ t_enter,
                                                            const i64* __restrict__ t_exit, u32* __restrict__ send_chg, u32* __restrict__ recv_chg) {
   const u64 i = (u64)blockIdx.x * RT_THREADS + threadIdx.x;
@@ -152,7 +163,8 @@ __global__ void __launch_bounds__(RT_THREADS) k_record_rates(TickArgs A, u64 n_r
     const u64 lo = A.tick_off[r], hi = A.tick_off[r + 1];
     if (hi > lo) {
       const i64 a = t_enter[i], b = t_exit[i];
-      const u64 ca = ticks_upto(A.tick_ns, lo, hi, a), cb = b == -1 ? hi - lo : ticks_upto(A.tick_ns, lo, hi, b);
+      const u64 ca = ticks_upto(A.tick_ns, lo, hi, a);
+      const u64 cb = b == -1 ? hi - lo : (b < a ? 0 : ca + ticks_upto_near(A.tick_ns, lo + ca, hi, b));
       // a rank's first tick has no indicator, so the prefix "before the first tick" equals the prefix at it
       const u64 ia = lo + (ca ? ca - 1 : 0), ib = lo + (cb ? cb - 1 : 0);
       if (ib > ia) {
