@@ -31,7 +31,7 @@ HBM_FALLBACK_GBS = 6650.0
 # DRAM traffic per record (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture divided by the records of the
 # captured launch; 5-window case, 20.48 M records, see profiles/). Traffic grows in proportion to the records, so a
 # launch's traffic is this figure times its records. Set an entry to None whenever its kernel changes.
-NCU_TRAFFIC_PER_RECORD = {"k_reduce_fused": (782.503424e6 + 228.286208e6) / 20.48e6}
+NCU_TRAFFIC_PER_RECORD = {"k_reduce_fused": (782.953216e6 + 229.746688e6) / 20.48e6}
 
 
 def parse():

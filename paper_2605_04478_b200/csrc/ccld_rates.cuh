@@ -6,7 +6,8 @@
 //                   same rank (a rank's first tick never counts)
 //   k_tile_scan     exclusive prefix over the tile sums (one CTA)
 //   k_tick_prefix   inclusive prefix of the change indicators per tick: low word send, high word recv
-//   k_record_rates  per record: two binary searches in its rank's tick times, then a difference of prefixes
+//   k_record_rates  per record: two searches in its rank's tick times (the first starts from an even-spacing guess,
+//                   the second from the first), then a difference of prefixes
 //
 // No kernel waits on another CTA: the prefix is three plain launches.
 #pragma once
@@ -153,6 +154,33 @@ __device__ __forceinline__ u64 ticks_upto_near(const i64* __restrict__ tn, u64 l
   return (pos - lo) + ticks_upto(tn, pos, end, t);
 }
 
+// The same count, started from where t would sit if the ticks were evenly spaced (probes sample at a fixed period, so
+// the guess is usually within a tick or two); doubling steps up or down from the guess, then bisection. Any spacing
+// gives the right count: the guess only decides where the search starts.
+__device__ __forceinline__ u64 ticks_upto_guess(const i64* __restrict__ tn, u64 lo, u64 hi, i64 t) {
+  const u64 n = hi - lo;
+  if (n == 0) return 0;
+  const i64 t0 = __ldg(tn + lo), t1 = __ldg(tn + hi - 1);
+  if (t < t0) return 0;
+  if (t >= t1) return n;
+  // tn[lo] <= t < tn[hi - 1]: the first tick after t has index j in [1, n - 1]
+  u64 g = (u64)((double)(t - t0) / (double)(t1 - t0) * (double)(n - 1));
+  g = g > n - 2 ? n - 2 : g;
+  u64 j;
+  if (__ldg(tn + lo + g) <= t) {
+    u64 pos = g, step = 1;                          // tn[lo + pos] <= t
+    for (int it = 0; it < 64 && pos + step < n && __ldg(tn + lo + pos + step) <= t; ++it) { pos += step; step <<= 1; }
+    const u64 end = pos + step < n - 1 ? pos + step : n - 1;          // tn[lo + end] > t
+    j = pos + 1 + ticks_upto(tn, lo + pos + 1, lo + end, t);
+  } else {
+    u64 pos = g, step = 1;                          // tn[lo + pos] > t
+    for (int it = 0; it < 64 && pos >= step && __ldg(tn + lo + pos - step) > t; ++it) { pos -= step; step <<= 1; }
+    const u64 start = pos >= step ? pos - step : 0;                   // tn[lo + start] <= t
+    j = start + 1 + ticks_upto(tn, lo + start + 1, lo + pos, t);
+  }
+  return j;
+}
+
 __global__ void __launch_bounds__(RT_THREADS) k_record_rates(TickArgs A, u64 n_rec, const u32* __restrict__ rank, const i64* __restrict__ t_enter,
                                                            const i64* __restrict__ t_exit, u32* __restrict__ send_chg, u32* __restrict__ recv_chg) {
   const u64 i = (u64)blockIdx.x * RT_THREADS + threadIdx.x;
@@ -163,7 +191,7 @@ __global__ void __launch_bounds__(RT_THREADS) k_record_rates(TickArgs A, u64 n_r
     const u64 lo = A.tick_off[r], hi = A.tick_off[r + 1];
     if (hi > lo) {
       const i64 a = t_enter[i], b = t_exit[i];
-      const u64 ca = ticks_upto(A.tick_ns, lo, hi, a);
+      const u64 ca = ticks_upto_guess(A.tick_ns, lo, hi, a);
       const u64 cb = b == -1 ? hi - lo : (b < a ? 0 : ca + ticks_upto_near(A.tick_ns, lo + ca, hi, b));
       // a rank's first tick has no indicator, so the prefix "before the first tick" equals the prefix at it
       const u64 ia = lo + (ca ? ca - 1 : 0), ib = lo + (cb ? cb - 1 : 0);
