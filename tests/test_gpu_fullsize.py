@@ -83,3 +83,37 @@ def test_cfg4_full_size_in_the_bench_configuration():
     for k in ("votes", "ops", "bw_cnt"):
         same(a[k], b[k], k)
     close(a["bw_sum"], b["bw_sum"], "bw_sum")
+
+
+def test_derive_rates_full_window_in_the_bench_configuration():
+    """One cfg4 window with its raw probe samples (4.1 M records, 21 M ticks), derived in one call as bench.py does.
+    The oracle recomputes a sample of the records (it walks every tick of a record's rank); properties that hold at any
+    size are checked on all of them."""
+    import paper_2605_04478_b200 as ccld
+    spec = tg.cfg4(n_windows=1)
+    win = tg.gen_window(spec, 0, device="cuda")
+    ticks = tg.gen_ticks(win.cols, spec.n_ranks)
+    an = ccld.Analyzer()
+    s, r = an.derive_rates(win.cols["rank"], win.cols["t_enter"], win.cols["t_exit"], ticks["tick_off"], ticks["tick_ns"],
+                           ticks["send_count"], ticks["recv_count"])
+    torch.cuda.synchronize()
+    n = win.n_rec
+    assert n == 4_096_000 and int(ticks["tick_ns"].numel()) > 20_000_000
+    s = s.cpu().numpy().view(np.uint32); r = r.cpu().numpy().view(np.uint32)
+    c = {k: v.cpu().numpy() for k, v in win.cols.items() if k in ("rank", "t_enter", "t_exit")}
+    k = {k: v.cpu().numpy() for k, v in ticks.items()}
+    # sampled records, spread over every rank and the whole window, plus the first and last of the upload
+    rng = np.random.default_rng(7)
+    pick = np.unique(np.concatenate([rng.integers(0, n, 6000), np.arange(0, 64), np.arange(n - 64, n)]))
+    es, er = orc.derive_rates(c["rank"][pick], c["t_enter"][pick], c["t_exit"][pick], k["tick_off"], k["tick_ns"], k["send_count"], k["recv_count"])
+    same(s[pick], es, "send_chg"); same(r[pick], er, "recv_chg")
+    # a count never exceeds the ticks inside the op, and an op of this trace (8 sends spread over its duration) that
+    # covers at least one tick shows at least one change of the counter that rounds up
+    per = (c["t_exit"] - c["t_enter"]) // 1_000_000 + 1
+    assert (s <= per).all() and (r <= per).all()
+    assert (r[per >= 3] >= 1).all()
+    # the same call again gives the same columns (the scratch block is reused)
+    s2, r2 = an.derive_rates(win.cols["rank"], win.cols["t_enter"], win.cols["t_exit"], ticks["tick_off"], ticks["tick_ns"],
+                             ticks["send_count"], ticks["recv_count"])
+    torch.cuda.synchronize()
+    assert np.array_equal(s2.cpu().numpy().view(np.uint32), s) and np.array_equal(r2.cpu().numpy().view(np.uint32), r)
