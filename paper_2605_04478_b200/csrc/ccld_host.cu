@@ -450,6 +450,10 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   const size_t o_fcta = take(n_list[B_FCTA] * sizeof(FusedCta)), o_fwt = take(n_list[B_FWT] * sizeof(WarpTile)),
                o_fsum = take(n_list[B_FSUM] * sizeof(TileSum)), o_t2 = take(n_list[B_T2] * sizeof(Tile)), o_s2 = take(n_list[B_T2] * sizeof(TileSum)),
                o_t3 = take(n_list[B_T3] * sizeof(Tile)), o_s3 = take(n_list[B_T3] * sizeof(TileSum));
+  // groups the fused kernel may set aside for the deferred kernel: at most every group of the batch
+  u64 total_groups = 0;
+  for (u32 k = 0; k < B; ++k) total_groups += ctx->h_pinned[(size_t)k * T_COUNT + T_GROUPS];
+  const size_t o_defn = take(8), o_def = take(n_list[B_FCTA] ? total_groups * 8 : 0);
   Block rb = ctx->pool.get(off, &e);
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "result allocation failed");
   auto res_blk = std::make_shared<Shared>(&ctx->pool, rb);
@@ -468,7 +472,13 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   PlanLists pl; pl.fcta = (FusedCta*)(rbase + o_fcta); pl.fwt = (WarpTile*)(rbase + o_fwt); pl.t2 = (Tile*)(rbase + o_t2); pl.t3 = (Tile*)(rbase + o_t3);
   { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, pl, 1); }
   if (cta > 0) { TimedLaunch tl(ts, 2, st); k_slot_scatter<<<(u32)cta, SCAT_THREADS, 0, st>>>(d_desc, B, ctx->reg); }
-  if (n_list[B_FCTA]) { TimedLaunch tl(ts, 3, st); k_reduce_fused<<<(u32)n_list[B_FCTA], SMALL_SEQS, 0, st>>>(d_desc, pl.fcta, pl.fwt, (TileSum*)(rbase + o_fsum), ctx->reg, ctx->dp, now_ns); }
+  if (n_list[B_FCTA]) {
+    const DeferList dl{(u64*)(rbase + o_def), (u32*)(rbase + o_defn)};
+    CK(cudaMemsetAsync(rbase + o_defn, 0, 8, st));
+    TimedLaunch tl(ts, 3, st);
+    k_reduce_fused<<<(u32)n_list[B_FCTA], SMALL_SEQS, 0, st>>>(d_desc, pl.fcta, pl.fwt, (TileSum*)(rbase + o_fsum), ctx->reg, ctx->dp, dl);
+    k_reduce_deferred<<<DEF_GRID, DEF_WARPS * 32, 0, st>>>(d_desc, dl, ctx->reg, ctx->dp, now_ns);
+  }
   if (n_list[B_T2]) { TimedLaunch tl(ts, 4, st); k_reduce_mid<<<(u32)n_list[B_T2], MID_THREADS, mid_smem_bytes(2 * WARP_N), st>>>(d_desc, pl.t2, (TileSum*)(rbase + o_s2), ctx->reg, ctx->dp, now_ns); }
   if (n_list[B_T3]) { TimedLaunch tl(ts, 5, st); k_reduce_large<<<(u32)n_list[B_T3], LARGE_THREADS, 16ull * ctx->max_large_n, st>>>(d_desc, pl.t3, (TileSum*)(rbase + o_s3), ctx->reg, ctx->dp, now_ns); }
   { TimedLaunch tl(ts, 6, st); k_window_decide<<<(nc + 3) / 4, 128, 0, st>>>(d_desc, B, ctx->reg, ctx->dp); }

@@ -6,7 +6,9 @@
 //                   and the work list for the reduction kernels
 //   k_slot_scatter  group-by, part 3: perm[slot] = record index
 //   k_reduce_fused  per-op reductions + median/MAD + flags + votes for n <= 128, chunk-major work list:
-//                   n <= 8 one thread per group (warp-tiles), 9 <= n <= 128 one warp per group (register bitonic sort)
+//                   n <= 8 one thread per group (warp-tiles), 9 <= n <= 128 n_pad / 8 lanes per group (register /
+//                   shuffle bitonic network); complete groups whose times fit 32-bit offsets
+//   k_reduce_deferred  the groups k_reduce_fused sets aside (incomplete, in flight, 64-bit spreads)
 //   k_reduce_mid    same, 129 <= n <= 1024 (shared-memory bitonic sort, several groups per CTA)
 //   k_reduce_large  same, n > 1024 (one CTA per group, radix select)
 //   k_window_decide Eq. 1-4 per communicator and window, slow location
@@ -529,359 +531,11 @@ __global__ void __launch_bounds__(SCAT_THREADS) k_slot_scatter(const WinDesc* __
   }
 }
 
-// ------------------------------------------------------------------------------------------------
-// per-op reductions, n <= 8: one thread per group, lanes run along consecutive op counters so the
-// gathers of one member's records coalesce
-// ------------------------------------------------------------------------------------------------
-template <class K> __device__ __forceinline__ void cswap(K& a, K& b) { const K lo = a < b ? a : b; const K hi = a < b ? b : a; a = lo; b = hi; }
+}  // namespace ccld
 
-// 19-exchange sorting network for 8 keys
-template <class K> __device__ __forceinline__ void sort8(K (&v)[8]) {
-  cswap(v[0], v[2]); cswap(v[1], v[3]); cswap(v[4], v[6]); cswap(v[5], v[7]);
-  cswap(v[0], v[4]); cswap(v[1], v[5]); cswap(v[2], v[6]); cswap(v[3], v[7]);
-  cswap(v[0], v[1]); cswap(v[2], v[3]); cswap(v[4], v[5]); cswap(v[6], v[7]);
-  cswap(v[2], v[4]); cswap(v[3], v[5]);
-  cswap(v[1], v[4]); cswap(v[3], v[6]);
-  cswap(v[1], v[2]); cswap(v[3], v[4]); cswap(v[5], v[6]);
-}
-// bitonic merge: sorts 8 keys that first fall and then rise
-template <class K> __device__ __forceinline__ void merge8(K (&v)[8]) {
-  cswap(v[0], v[4]); cswap(v[1], v[5]); cswap(v[2], v[6]); cswap(v[3], v[7]);
-  cswap(v[0], v[2]); cswap(v[1], v[3]); cswap(v[4], v[6]); cswap(v[5], v[7]);
-  cswap(v[0], v[1]); cswap(v[2], v[3]); cswap(v[4], v[5]); cswap(v[6], v[7]);
-}
-template <class K> __device__ __forceinline__ K pick4(const K (&v)[8], u32 k) {
-  K r = v[0];
-  r = k == 1 ? v[1] : r; r = k == 2 ? v[2] : r; r = k == 3 ? v[3] : r;
-  return r;
-}
+#include "ccld_fused.cuh"
 
-template <class K> struct KeyMax;
-template <> struct KeyMax<u32> { static __device__ __forceinline__ u32 v() { return 0xFFFFFFFFu; } };
-template <> struct KeyMax<u64> { static __device__ __forceinline__ u64 v() { return U64_MAX_; } };
-
-// lower median and lower-median absolute deviation of x[0..n), n <= 8 (x[p] = maximum key for p >= n)
-template <class K> __device__ __forceinline__ void median_mad8(const K (&x)[8], u32 n, K* med, K* mad) {
-  K s[8];
-#pragma unroll
-  for (int p = 0; p < 8; ++p) s[p] = x[p];
-  sort8(s);
-  const u32 k = (n - 1) >> 1;
-  const K m = pick4(s, k);
-#pragma unroll
-  for (int p = 0; p < 8; ++p) s[p] = (u32)p < n ? (s[p] >= m ? s[p] - m : m - s[p]) : KeyMax<K>::v();   // falls to 0 at k, then rises
-  merge8(s);
-  *med = m; *mad = pick4(s, k);
-}
-
-// 1 / x for x >= 1 to within a few ulp: single-precision seed and two Newton steps
-__device__ __forceinline__ double rcp_newton(double x) {
-  double r = (double)__frcp_rn((float)x);
-  double e = fma(-x, r, 1.0); r = fma(r, e, r);
-  e = fma(-x, r, 1.0); r = fma(r, e, r);
-  return r;
-}
-__device__ __forceinline__ double busbw_fast(double bytes_num, double den, i64 t) {
-  return t > 0 ? bytes_num * rcp_newton((double)t * den) : 0.0;
-}
-
-// Sums v[m] over the warp for m = 0..7 with 9 shuffles; lane l ends up with the total of member
-// m = 4 * bit4(l) + 2 * bit3(l) + bit2(l).
-__device__ __forceinline__ double warp_sum8(double (&v)[8], u32 lane) {
-#pragma unroll
-  for (int w = 4, bit = 16; w >= 1; w >>= 1, bit >>= 1) {
-    const bool hi = (lane & bit) != 0;
-#pragma unroll
-    for (int i = 0; i < w; ++i) {
-      const double send = hi ? v[i] : v[i + w], keep = hi ? v[i + w] : v[i];
-      v[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, send, bit);
-    }
-  }
-  v[0] += __shfl_xor_sync(0xFFFFFFFFu, v[0], 2);
-  v[0] += __shfl_xor_sync(0xFFFFFFFFu, v[0], 1);
-  return v[0];
-}
-
-// A complete group whose skews or durations do not fit 32-bit keys (a spread of more than 4.29 s inside
-// one op): gathered again and handled here, out of line, so that the common path stays in 32 bits.
-// Returns the four order statistics, the packed flag bytes, and adds the members' bus bandwidths.
-__device__ __noinline__ u64 small_group64(const WinDesc& D, const Registry& R, const u32* mem, u64 pslot, u32 pstride, u32 n, u64 e_min, u32 k_milli,
-                                          bool analysed, bool add_bw, double bn, double den, u64* out4) {
-  u64 sk[8], du[8];
-#pragma unroll
-  for (int p = 0; p < 8; ++p) {
-    sk[p] = U64_MAX_; du[p] = U64_MAX_;
-    if ((u32)p < n) { const u32 idx = D.perm[pslot + (u64)p * pstride]; const i64 a = D.t_enter[idx], b = D.t_exit[idx]; sk[p] = (u64)a - e_min; du[p] = (u64)(b - a); }
-  }
-  if (add_bw)
-    for (u32 p = 0; p < n; ++p) atomicAdd(&R.bw_sum[mem[p]], busbw_fast(bn, den, (i64)du[p]));
-  u64 packed = 0;
-  out4[0] = out4[1] = out4[2] = out4[3] = 0;
-  if (analysed) {
-    u64 med_s, mad_s, med_d, mad_d;
-    median_mad8<u64>(sk, n, &med_s, &mad_s);
-    median_mad8<u64>(du, n, &med_d, &mad_d);
-    out4[0] = med_s; out4[1] = mad_s; out4[2] = med_d; out4[3] = mad_d;
-#pragma unroll
-    for (int p = 0; p < 8; ++p) {
-      if ((u32)p < n) {
-        const bool so = mul_gt(absdiff(sk[p], med_s), 1000u, mad_s, k_milli), sh = sk[p] > med_s;
-        const bool dq = mul_gt(absdiff(du[p], med_d), 1000u, mad_d, k_milli), dh = du[p] > med_d;
-        const u32 f = (so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0);
-        packed |= (u64)f << (8 * p);
-      }
-    }
-  } else {
-    for (u32 p = 0; p < n; ++p) packed |= (u64)CCLD_F_NOT_ANALYSED << (8 * p);
-  }
-  return packed;
-}
-
-enum { SC_COMP = 0, SC_INC, SC_BAR, SC_AN, SC_MIS, SC_BWC, SC_PRES, SC_FS, SC_FD, SC_COUNT };
-
-// One warp-tile: up to 32 consecutive op counters of one communicator, one lane per group.
-template <bool FULL>
-__device__ __forceinline__ void reduce_small_warp(const WinDesc& D, const WarpTile& t, TileSum* __restrict__ sums, const Registry& R, const Params& P,
-                                                  i64 now, u32 n_rt, double (*s_bw)[SMALL_N], u32* s_rounds, u32* s_cnt) {
-  const u32 n = FULL ? (u32)SMALL_N : n_rt;
-  const u32 c = t.c;
-  const RangeRow& row = t.row;
-  const u32* mem = R.members + t.moff;
-  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5, j = lane;
-  const bool active = j < t.count;
-  const u32 k_milli = P.k_milli;
-
-  double bw[SMALL_N];
-#pragma unroll
-  for (int p = 0; p < SMALL_N; ++p) bw[p] = 0.0;
-  bool complete = false, barrier = false, analysed = false, mismatch = false;
-  u32 n_present = 0, n_fs = 0, n_fd = 0;
-  u64 my_rng = 0;
-
-  if (active) {
-    const u64 g = row.group0 + t.seq_off + j;
-    const u64 slot = row.slot0 + (u64)(t.seq_off + j) * n;
-    u32 idx[SMALL_N];
-    {
-      const u32* __restrict__ pm = D.perm + perm_at(row, t.seq_off + j, 0);
-#pragma unroll
-      for (int p = 0; p < SMALL_N; ++p) idx[p] = (FULL || (u32)p < n) ? pm[(u64)p * row.n_seq] : NONE;
-    }
-    // Two batches of gathers, each issued in full before any of it is used (a missing member reads record 0 and
-    // is masked out): first the times, which are reduced to 32-bit keys, then the op-set and rate columns.
-    u32 safe[SMALL_N];
-#pragma unroll
-    for (int p = 0; p < SMALL_N; ++p) safe[p] = idx[p] == NONE ? 0u : idx[p];
-    i64 x_max = INT64_MIN, age = -1;
-    bool inflight = false, bad_time = false;
-    u32 miss = 0;
-    u64 e_min = 0, e_max = 0, tmax = 0, tmin = 0; u32 pmax = 0, pmin = 0;
-    u32 sk[SMALL_N], dd[SMALL_N];
-    bool fast = false;
-    {
-      const i64* __restrict__ c_te = D.t_enter; const i64* __restrict__ c_tx = D.t_exit;
-      i64 ld_a[SMALL_N], ld_b[SMALL_N];
-#pragma unroll
-      for (int p = 0; p < SMALL_N; ++p) { ld_a[p] = c_te[safe[p]]; ld_b[p] = c_tx[safe[p]]; }
-#pragma unroll
-      for (int p = 0; p < SMALL_N; ++p) {
-        if (FULL || (u32)p < n) {
-          if (idx[p] == NONE) miss |= 1u << p;
-          else {
-            ++n_present;
-            const i64 a = ld_a[p], b = ld_b[p];
-            if (b == -1) { inflight = true; const i64 ag = now - a; age = ag > age ? ag : age; }
-            else if (a < 0 || b < a) bad_time = true;
-            x_max = b > x_max ? b : x_max;
-          }
-        }
-      }
-      complete = miss == 0 && !inflight && !bad_time;
-      if (complete) {
-        e_min = (u64)ld_a[0]; e_max = e_min; tmax = (u64)(ld_b[0] - ld_a[0]); tmin = tmax;
-#pragma unroll
-        for (int p = 1; p < SMALL_N; ++p) {
-          if (FULL || (u32)p < n) {
-            const u64 te = (u64)ld_a[p], du = (u64)(ld_b[p] - ld_a[p]);
-            e_min = te < e_min ? te : e_min; e_max = te > e_max ? te : e_max;
-            if (du > tmax) { tmax = du; pmax = p; }
-            if (du < tmin) { tmin = du; pmin = p; }
-          }
-        }
-        fast = e_max - e_min < 0xFFFFFFFFull && tmax - tmin < 0xFFFFFFFFull;
-#pragma unroll
-        for (int p = 0; p < SMALL_N; ++p) {
-          const bool in = FULL || (u32)p < n;
-          sk[p] = in ? (u32)((u64)ld_a[p] - e_min) : 0xFFFFFFFFu; dd[p] = in ? (u32)((u64)(ld_b[p] - ld_a[p]) - tmin) : 0xFFFFFFFFu;
-        }
-      }
-    }
-    u64 gbytes = 0; u32 gop = 0; bool have_first = false;
-    u32 max_chg = 0, pos_chg = 0; bool have_chg = false;
-    {
-      const u64* __restrict__ c_by = D.bytes; const u8* __restrict__ c_op = D.op;
-      const u32* __restrict__ c_sc = D.send_chg; const u32* __restrict__ c_rc = D.recv_chg;
-      u64 ld_by[SMALL_N]; u32 ld_op[SMALL_N], ld_ch[SMALL_N];
-#pragma unroll
-      for (int p = 0; p < SMALL_N; ++p) {
-        ld_by[p] = c_by[safe[p]]; ld_op[p] = c_op[safe[p]]; ld_ch[p] = 0;
-        if (c_sc != nullptr) { const u32 sc = c_sc[safe[p]], rc = c_rc[safe[p]]; ld_ch[p] = sc > rc ? sc : rc; }
-      }
-#pragma unroll
-      for (int p = 0; p < SMALL_N; ++p) {
-        if ((FULL || (u32)p < n) && idx[p] != NONE) {
-          if (!have_first) { gbytes = ld_by[p]; gop = ld_op[p]; have_first = true; }
-          else if (ld_op[p] != gop || ld_by[p] != gbytes) mismatch = true;
-          if (!have_chg || ld_ch[p] > max_chg) { max_chg = ld_ch[p]; pos_chg = p; have_chg = true; }
-        }
-      }
-    }
-    barrier = have_first && gop == CCLD_OP_ALLREDUCE && gbytes < P.barrier_bytes;
-    u32 gfl = (mismatch ? CCLD_G_OPSET_MISMATCH : 0) | (barrier ? CCLD_G_BARRIER : 0) | (inflight ? CCLD_G_INFLIGHT : 0) |
-              (bad_time ? CCLD_G_BAD_TIME : 0);
-    u64 o_emin = 0, o_askew = 0, o_tmax = 0, o_tmin = 0, med_s = 0, mad_s = 0, med_d = 0, mad_d = 0; i64 o_span = 0;
-    u32 r_tmin = 0, r_tmax = 0, r_chg = 0; double gbw = 0.0;
-    u64 packed = 0;                                        // the group's flag bytes, member p in byte p
-#pragma unroll
-    for (int p = 0; p < SMALL_N; ++p)
-      if (FULL || (u32)p < n) packed |= (u64)(CCLD_F_NOT_ANALYSED | ((miss >> p) & 1u ? CCLD_F_MISSING : 0)) << (8 * p);
-
-    if (!complete) {
-      gfl |= CCLD_G_INCOMPLETE;
-      max_chg = 0;
-      if (inflight && age > P.hang_ns && !barrier) { gfl |= CCLD_G_HANG_ALERT; raise_alert(D, R.comm_id[c], row.seq_lo + t.seq_off + j, age); }
-    } else {
-      gfl |= CCLD_G_COMPLETE;
-      const u64 askew = e_max - e_min;
-      const i64 span = x_max - (i64)e_min;
-      double num, den; bus_factor(gop, n, &num, &den);
-      const double bn = (double)gbytes * num;
-      gbw = busbw_fast(bn, den, span);
-      o_emin = e_min; o_askew = askew; o_tmax = tmax; o_tmin = tmin; o_span = span;
-      my_rng = tmax - tmin;
-      r_tmin = mem[pmin]; r_tmax = mem[pmax]; r_chg = mem[pos_chg];
-      analysed = !barrier && n >= P.min_group;
-      if (analysed) gfl |= CCLD_G_ANALYSED;
-      if (fast) {
-        // 32-bit keys: skew, and duration minus the shortest duration
-        if (analysed) {
-          u32 ms, ds, md, dm;
-          median_mad8<u32>(sk, n, &ms, &ds);
-          median_mad8<u32>(dd, n, &md, &dm);
-          med_s = ms; mad_s = ds; med_d = tmin + md; mad_d = dm;
-          // |x - med| * 1000 > k * MAD  <=>  |x - med| > floor(k * MAD / 1000); deviations are below 2^32
-          const u64 qs = (u64)ds * k_milli / 1000u, qd = (u64)dm * k_milli / 1000u;
-          const u32 ts = qs > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)qs, td = qd > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)qd;
-          packed = 0;
-#pragma unroll
-          for (int p = 0; p < SMALL_N; ++p) {
-            if (FULL || (u32)p < n) {
-              const u32 a = sk[p] >= ms ? sk[p] - ms : ms - sk[p], b = dd[p] >= md ? dd[p] - md : md - dd[p];
-              const bool so = a > ts, sh = sk[p] > ms, dq = b > td, dh = dd[p] > md;
-              packed |= (u64)((so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0)) << (8 * p);
-            }
-          }
-        }
-        if (!barrier) {
-#pragma unroll
-          for (int p = 0; p < SMALL_N; ++p) if (FULL || (u32)p < n) bw[p] = busbw_fast(bn, den, (i64)(tmin + dd[p]));
-        }
-      } else {
-        u64 o4[4];
-        packed = small_group64(D, R, mem, perm_at(row, t.seq_off + j, 0), row.n_seq, n, e_min, k_milli, analysed, !barrier, bn, den, o4);
-        med_s = o4[0]; mad_s = o4[1]; med_d = o4[2]; mad_d = o4[3];
-      }
-      if (analysed) {
-#pragma unroll
-        for (int p = 0; p < SMALL_N; ++p) {
-          if (FULL || (u32)p < n) {
-            const u32 f = (u32)(packed >> (8 * p));
-            if (f & CCLD_F_SKEW_OUT) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p] * 4 + ((f & CCLD_F_SKEW_HI) ? 0 : 1)], 1u); }
-            if (f & CCLD_F_DUR_OUT) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p] * 4 + ((f & CCLD_F_DUR_HI) ? 2 : 3)], 1u); }
-          }
-        }
-      }
-    }
-    // ---- outputs ----
-    const u64 G = D.n_groups;
-    D.gi64[(u64)GI_E_MIN * G + g] = (i64)o_emin; D.gi64[(u64)GI_ARRIVAL_SKEW * G + g] = (i64)o_askew;
-    D.gi64[(u64)GI_T_MAX * G + g] = (i64)o_tmax; D.gi64[(u64)GI_T_MIN * G + g] = (i64)o_tmin; D.gi64[(u64)GI_SPAN * G + g] = o_span;
-    D.gi64[(u64)GI_MED_SKEW * G + g] = (i64)med_s; D.gi64[(u64)GI_MAD_SKEW * G + g] = (i64)mad_s;
-    D.gi64[(u64)GI_MED_DUR * G + g] = (i64)med_d; D.gi64[(u64)GI_MAD_DUR * G + g] = (i64)mad_d;
-    D.gu32[(u64)GU_RANK_TMIN * G + g] = r_tmin; D.gu32[(u64)GU_RANK_TMAX * G + g] = r_tmax;
-    D.gu32[(u64)GU_MAX_CHG * G + g] = max_chg; D.gu32[(u64)GU_RANK_MAX_CHG * G + g] = r_chg;
-    D.gu32[(u64)GU_N_PRESENT * G + g] = n_present; D.gu32[(u64)GU_GFLAGS * G + g] = gfl;
-    D.gbw[g] = gbw;
-    if (FULL && (slot & 7) == 0) {
-      *reinterpret_cast<u64*>(D.flags + slot) = packed;
-    } else {
-#pragma unroll
-      for (int p = 0; p < SMALL_N; ++p) if (FULL || (u32)p < n) D.flags[slot + p] = (u8)(packed >> (8 * p));
-    }
-  }
-
-  // ---- per-warp accumulation: counters (CTA shared memory), Eq. 2 candidate, per-rank bandwidth sums ----
-  const bool is_round = active && complete && !barrier;
-  const u32 b_comp = __ballot_sync(0xFFFFFFFFu, active && complete), b_inc = __ballot_sync(0xFFFFFFFFu, active && !complete);
-  const u32 b_bar = __ballot_sync(0xFFFFFFFFu, active && barrier), b_an = __ballot_sync(0xFFFFFFFFu, active && analysed);
-  const u32 b_mis = __ballot_sync(0xFFFFFFFFu, active && mismatch), b_bwc = __ballot_sync(0xFFFFFFFFu, is_round);
-  const u32 pres = __reduce_add_sync(0xFFFFFFFFu, n_present), fs = __reduce_add_sync(0xFFFFFFFFu, n_fs), fd = __reduce_add_sync(0xFFFFFFFFu, n_fd);
-  u64 brng = is_round ? my_rng : 0; u32 bk = is_round ? t.seq_off + j : NONE;
-  best_warp_reduce(brng, bk);
-  const double tot = warp_sum8(bw, lane);
-  if ((lane & 3) == 0) s_bw[wid][lane >> 2] = tot;
-  if (lane == 0) {
-    s_rounds[wid] = (u32)__popc(b_bwc);
-    TileSum ts; ts.best_rng = brng; ts.best_k = bk; ts.n_rounds = (u32)__popc(b_bwc); ts.n_an = (u32)__popc(b_an); ts.pad = 0;
-    sums[t.sum_idx] = ts;
-    if (b_comp) atomicAdd(&s_cnt[SC_COMP], (u32)__popc(b_comp));
-    if (b_inc) atomicAdd(&s_cnt[SC_INC], (u32)__popc(b_inc));
-    if (b_bar) atomicAdd(&s_cnt[SC_BAR], (u32)__popc(b_bar));
-    if (b_an) atomicAdd(&s_cnt[SC_AN], (u32)__popc(b_an));
-    if (b_mis) atomicAdd(&s_cnt[SC_MIS], (u32)__popc(b_mis));
-    if (pres) atomicAdd(&s_cnt[SC_PRES], pres);
-    if (fs) atomicAdd(&s_cnt[SC_FS], fs);
-    if (fd) atomicAdd(&s_cnt[SC_FD], fd);
-  }
-}
-
-// Class-0 CTA of the fused kernel: eight warp-tiles of one window and one time chunk.
-__device__ __forceinline__ void reduce_small_cta(const WinDesc& D, const FusedCta& t, const WarpTile* __restrict__ wts, TileSum* __restrict__ sums,
-                                                 const Registry& R, const Params& P, i64 now) {
-  __shared__ double s_bw[SMALL_SEQS / 32][SMALL_N];
-  __shared__ u32 s_comm[SMALL_SEQS / 32], s_rounds[SMALL_SEQS / 32];
-  __shared__ u32 s_cnt[SC_COUNT];
-  const u32 wid = threadIdx.x >> 5;
-  if (threadIdx.x < SC_COUNT) s_cnt[threadIdx.x] = 0;
-  if (threadIdx.x < SMALL_SEQS / 32) { s_comm[threadIdx.x] = NONE; s_rounds[threadIdx.x] = 0; }
-  __syncthreads();
-  if (wid < t.wt_count) {
-    const WarpTile wt = wts[t.wt_first + wid];
-    const u32 n = wt.row.n;
-    if ((threadIdx.x & 31) == 0) s_comm[wid] = wt.c;
-    if (n == SMALL_N) reduce_small_warp<true>(D, wt, sums, R, P, now, n, s_bw, s_rounds, s_cnt);
-    else reduce_small_warp<false>(D, wt, sums, R, P, now, n, s_bw, s_rounds, s_cnt);
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    count_add(D.counters, C_COMPLETE, s_cnt[SC_COMP]); count_add(D.counters, C_INCOMPLETE, s_cnt[SC_INC]);
-    count_add(D.counters, C_BARRIER, s_cnt[SC_BAR]); count_add(D.counters, C_ANALYSED, s_cnt[SC_AN]);
-    count_add(D.counters, C_MISMATCH, s_cnt[SC_MIS]); count_add(D.counters, C_PRESENT, s_cnt[SC_PRES]);
-    count_add(D.counters, C_FLAG_SKEW, s_cnt[SC_FS]); count_add(D.counters, C_FLAG_DUR, s_cnt[SC_FD]);
-  }
-  // per-rank bandwidth: consecutive warp-tiles of one communicator are summed before the atomics
-  if (threadIdx.x < (SMALL_SEQS / 32) * SMALL_N) {
-    const u32 q0 = threadIdx.x >> 3, m = threadIdx.x & 7, c = s_comm[q0];
-    if (c != NONE && (q0 == 0 || s_comm[q0 - 1] != c) && m < R.comm_n[c]) {
-      double v = 0.0; u32 rounds = 0;
-      for (u32 q = q0; q < SMALL_SEQS / 32 && s_comm[q] == c; ++q) { v += s_bw[q][m]; rounds += s_rounds[q]; }
-      if (rounds) {
-        const u32 rank = R.members[R.comm_moff[c] + m];
-        atomicAdd(&R.bw_sum[rank], v); atomicAdd(&R.bw_cnt[rank], rounds);
-      }
-    }
-  }
-}
+namespace ccld {
 
 // ------------------------------------------------------------------------------------------------
 // per-op reductions, 129 <= n <= 1024: a tile of S groups is staged in shared memory ([group][member],
@@ -1145,383 +799,6 @@ inline size_t mid_smem_bytes(u32 n_pad_min) {
 }
 
 // ------------------------------------------------------------------------------------------------
-// per-op reductions, 9 <= n <= 128: L = n_pad / 8 lanes per group, eight ring positions per lane
-// (lane s of a group holds positions 8 s .. 8 s + 7), 32 / L consecutive op counters per warp. Each
-// lane gathers, reduces and sorts its eight values in registers exactly like the n <= 8 path; the
-// lanes of a group meet through xor shuffles: log2 L rounds for the extrema, and a merge network
-// whose cross-lane steps move eight independent keys each. 32-bit keys whenever the group's value
-// range fits; other groups go through an out-of-line 64-bit routine. No shared-memory staging.
-// ------------------------------------------------------------------------------------------------
-template <class K> __device__ __forceinline__ K pick8(const K (&v)[8], u32 r) {
-  K x = v[0];
-#pragma unroll
-  for (int i = 1; i < 8; ++i) x = r == (u32)i ? v[i] : x;
-  return x;
-}
-
-// One cross-lane step of a merge network: element r of this lane against element r (MIRROR: 7 - r) of lane ^ mask;
-// the lane with keep_low set keeps the smaller key of each pair.
-template <class K, bool MIRROR>
-__device__ __forceinline__ void sub_exchange(K (&v)[8], int mask, bool keep_low) {
-  K o[8];
-#pragma unroll
-  for (int r = 0; r < 8; ++r) o[r] = __shfl_xor_sync(0xFFFFFFFFu, v[MIRROR ? 7 - r : r], mask);
-#pragma unroll
-  for (int r = 0; r < 8; ++r) { const bool lt = v[r] < o[r]; v[r] = (lt == keep_low) ? v[r] : o[r]; }
-}
-
-// Sorts the 8 L keys of a group ascending; element i lives in lane i / 8 (of the group), register i % 8.
-template <int L, class K>
-__device__ __forceinline__ void sub_sort(K (&v)[8], u32 s) {
-  sort8(v);
-#pragma unroll
-  for (int m = 1; m < L; m <<= 1) {
-    // two ascending runs of m lanes each: the mirror step leaves every key of the low run <= every key of the high
-    // run and both runs bitonic; half-cleaners across lanes and then inside the lane finish the merge
-    sub_exchange<K, true>(v, 2 * m - 1, (s & m) == 0);
-#pragma unroll
-    for (int h = m >> 1; h >= 1; h >>= 1) sub_exchange<K, false>(v, h, (s & h) == 0);
-    merge8(v);
-  }
-}
-// Sorts 8 L keys that fall and then rise.
-template <int L, class K>
-__device__ __forceinline__ void sub_merge(K (&v)[8], u32 s) {
-#pragma unroll
-  for (int h = L >> 1; h >= 1; h >>= 1) sub_exchange<K, false>(v, h, (s & h) == 0);
-  merge8(v);
-}
-
-// Lower median and lower-median absolute deviation of a group's keys (x[q] = maximum key where the position does
-// not exist or the group is not sorted at all). Every lane of the warp must call it.
-template <int L, class K>
-__device__ __forceinline__ void sub_median_mad(const K (&x)[8], u32 n, u32 s, u32 lane, K* med, K* mad) {
-  K v[8];
-#pragma unroll
-  for (int q = 0; q < 8; ++q) v[q] = x[q];
-  sub_sort<L, K>(v, s);
-  const u32 k = (n - 1) >> 1, src = (lane & ~(u32)(L - 1)) | (k >> 3);
-  const K m = __shfl_sync(0xFFFFFFFFu, pick8(v, k & 7), src);
-#pragma unroll
-  for (int r = 0; r < 8; ++r) v[r] = s * 8 + r < n ? (v[r] >= m ? v[r] - m : m - v[r]) : KeyMax<K>::v();   // falls to 0 at k, then rises
-  sub_merge<L, K>(v, s);
-  *med = m; *mad = __shfl_sync(0xFFFFFFFFu, pick8(v, k & 7), src);
-}
-
-// Groups whose skews or durations do not fit 32-bit keys: the whole warp comes here (shuffles), lanes with `mine`
-// set gather their times again and get the order statistics and flag bytes of their group in 64 bits; their
-// members' bus bandwidths are added straight to the per-rank sums.
-template <int L>
-__device__ __noinline__ void sub_group64(const WinDesc& D, const Registry& R, const u32* mem, u64 pslot, u32 pstride, u32 n, u32 s, u32 lane, bool mine,
-                                         u64 e_min, u32 k_milli, bool analysed, bool add_bw, double bn, double den, u64* out4, u64* packed_io) {
-  u64 sk[8], du[8];
-#pragma unroll
-  for (int q = 0; q < 8; ++q) {
-    sk[q] = U64_MAX_; du[q] = U64_MAX_;
-    if (mine && s * 8 + q < n) { const u32 idx = D.perm[pslot + (u64)q * pstride]; const i64 a = D.t_enter[idx], b = D.t_exit[idx]; sk[q] = (u64)a - e_min; du[q] = (u64)(b - a); }
-  }
-  if (mine && add_bw)
-    for (u32 q = 0; q < 8 && s * 8 + q < n; ++q) atomicAdd(&R.bw_sum[mem[s * 8 + q]], busbw_fast(bn, den, (i64)du[q]));
-  u64 med_s, mad_s, med_d, mad_d;
-  sub_median_mad<L, u64>(sk, n, s, lane, &med_s, &mad_s);
-  sub_median_mad<L, u64>(du, n, s, lane, &med_d, &mad_d);
-  if (mine && analysed) {
-    out4[0] = med_s; out4[1] = mad_s; out4[2] = med_d; out4[3] = mad_d;
-    u64 packed = 0;
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      if (s * 8 + q < n) {
-        const bool so = mul_gt(absdiff(sk[q], med_s), 1000u, mad_s, k_milli), sh = sk[q] > med_s;
-        const bool dq = mul_gt(absdiff(du[q], med_d), 1000u, mad_d, k_milli), dh = du[q] > med_d;
-        packed |= (u64)((so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0)) << (8 * q);
-      }
-    }
-    *packed_io = packed;
-  }
-}
-
-struct SubShared {
-  double bw[MID_THREADS / 32][WARP_N];
-  u64 brng[MID_THREADS / 32];
-  u32 bk[MID_THREADS / 32], rounds[MID_THREADS / 32], n_an[MID_THREADS / 32];
-  u32 cnt[SC_COUNT];
-};
-
-// One warp: 32 / L consecutive op counters of the tile, L lanes each.
-template <int L>
-__device__ __forceinline__ void reduce_sub_warp(const WinDesc& D, const FusedCta& t, const Registry& R, const Params& P, i64 now, SubShared& sh) {
-  constexpr int GW = 32 / L;                                  // groups per warp
-  constexpr u32 FULLM = 0xFFFFFFFFu;
-  const RangeRow& row = t.row;
-  const u32 n = row.n, c = t.c;
-  const u32* mem = R.members + t.moff;
-  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  const u32 s = lane % L, j = wid * GW + lane / L, p0 = s * 8;
-  const bool active = j < t.count, lead = active && s == 0;
-  const u32 gmask = ((1u << L) - 1u) << (lane & ~(u32)(L - 1));   // the lanes of my group
-  const u32 k_milli = P.k_milli;
-
-  // ---- batch 0: record indices of my eight positions (member-major permutation: stride n_seq) ----
-  u32 idx[8];
-  const u64 pslot = perm_at(row, t.seq_off + (active ? j : 0u), p0);
-  {
-    const u32* __restrict__ pm = D.perm + pslot;
-#pragma unroll
-    for (int q = 0; q < 8; ++q) idx[q] = (active && p0 + q < n) ? pm[(u64)q * row.n_seq] : NONE;
-  }
-  // ---- batch 1: times (a missing member reads record 0 and is masked out) ----
-  u32 npres = 0, miss = 0, stb = 0;                           // stb: 1 in flight, 2 bad time
-  i64 x_max = INT64_MIN, age = -1;
-  u64 e_min = U64_MAX_, e_max = 0, tmax = 0, tmin = U64_MAX_; u32 pmax = NONE, pmin = NONE;
-  i64 ld_a[8], ld_b[8];
-  {
-    const i64* __restrict__ c_te = D.t_enter; const i64* __restrict__ c_tx = D.t_exit;
-#pragma unroll
-    for (int q = 0; q < 8; ++q) { const u32 ix = idx[q] == NONE ? 0u : idx[q]; ld_a[q] = c_te[ix]; ld_b[q] = c_tx[ix]; }
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      if (idx[q] != NONE) {
-        ++npres;
-        const i64 a = ld_a[q], b = ld_b[q];
-        if (b == -1) { stb |= 1; const i64 ag = now - a; age = ag > age ? ag : age; }
-        else if (a < 0 || b < a) stb |= 2;
-        x_max = b > x_max ? b : x_max;
-        const u64 te = (u64)a, du = (u64)(b - a);
-        e_min = te < e_min ? te : e_min; e_max = te > e_max ? te : e_max;
-        if (pmax == NONE || du > tmax) { tmax = du; pmax = p0 + q; }
-        if (pmin == NONE || du < tmin) { tmin = du; pmin = p0 + q; }
-      } else if (active && p0 + q < n) miss = 1;
-    }
-  }
-  // ---- the lanes of a group meet ----
-  const u32 b_miss = __ballot_sync(FULLM, miss != 0), b_if = __ballot_sync(FULLM, (stb & 1) != 0), b_bt = __ballot_sync(FULLM, (stb & 2) != 0);
-  const bool inflight = (b_if & gmask) != 0, bad_time = (b_bt & gmask) != 0;
-  const bool complete = active && (b_miss & gmask) == 0 && !inflight && !bad_time;
-  if (b_miss) {
-#pragma unroll
-    for (int h = 1; h < L; h <<= 1) npres += __shfl_xor_sync(FULLM, npres, h);
-  } else npres = active ? n : 0u;
-  if (b_if) {
-#pragma unroll
-    for (int h = 1; h < L; h <<= 1) { const i64 o = (i64)shfl_xor64((u64)age, h); age = o > age ? o : age; }
-  }
-#pragma unroll
-  for (int h = 1; h < L; h <<= 1) {
-    { const i64 o = (i64)shfl_xor64((u64)x_max, h); x_max = o > x_max ? o : x_max; }
-    { const u64 o = shfl_xor64(e_min, h); e_min = o < e_min ? o : e_min; }
-    { const u64 o = shfl_xor64(e_max, h); e_max = o > e_max ? o : e_max; }
-    { const u64 ot = shfl_xor64(tmax, h); const u32 op = __shfl_xor_sync(FULLM, pmax, h);
-      if (op != NONE && (pmax == NONE || ot > tmax || (ot == tmax && op < pmax))) { tmax = ot; pmax = op; } }
-    { const u64 ot = shfl_xor64(tmin, h); const u32 op = __shfl_xor_sync(FULLM, pmin, h);
-      if (op != NONE && (pmin == NONE || ot < tmin || (ot == tmin && op < pmin))) { tmin = ot; pmin = op; } }
-  }
-  const bool fast = complete && e_max - e_min < 0xFFFFFFFFull && tmax - tmin < 0xFFFFFFFFull;
-  // 32-bit keys: skew, and duration minus the shortest duration (maximum key where there is nothing to sort)
-  u32 sk[8], dd[8];
-#pragma unroll
-  for (int q = 0; q < 8; ++q) {
-    const bool in = fast && p0 + q < n;
-    sk[q] = in ? (u32)((u64)ld_a[q] - e_min) : 0xFFFFFFFFu; dd[q] = in ? (u32)((u64)(ld_b[q] - ld_a[q]) - tmin) : 0xFFFFFFFFu;
-  }
-  // ---- batch 2: op-set and rate columns ----
-  u64 gbytes = 0, chk = 0; u32 gop = 0; bool have_first = false, mismatch = false;
-  {
-    const u64* __restrict__ c_by = D.bytes; const u8* __restrict__ c_op = D.op;
-    const u32* __restrict__ c_sc = D.send_chg; const u32* __restrict__ c_rc = D.recv_chg;
-    u64 ld_by[8]; u32 ld_op[8], ld_ch[8];
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      const u32 ix = idx[q] == NONE ? 0u : idx[q];
-      ld_by[q] = c_by[ix]; ld_op[q] = c_op[ix]; ld_ch[q] = 0;
-      if (c_sc != nullptr) { const u32 sc = c_sc[ix], rc = c_rc[ix]; ld_ch[q] = sc > rc ? sc : rc; }
-    }
-    // the group's first present member: mine, then the lowest lane that has one
-    u64 fby = 0; u32 fop = 0; bool fhave = false;
-#pragma unroll
-    for (int q = 7; q >= 0; --q) if (idx[q] != NONE) { fby = ld_by[q]; fop = ld_op[q]; fhave = true; }
-    const u32 b_have = __ballot_sync(FULLM, fhave) & gmask;
-    have_first = b_have != 0;
-    const u32 src = have_first ? (u32)__ffs(b_have) - 1u : lane;
-    gbytes = __shfl_sync(FULLM, fby, src); gop = __shfl_sync(FULLM, fop, src);
-    bool mism = false;
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      if (idx[q] != NONE) {
-        if (ld_op[q] != gop || ld_by[q] != gbytes) mism = true;
-        const u64 ck = ((u64)ld_ch[q] << 32) | (u64)(NONE - (p0 + q));     // most changes, then lowest position
-        chk = ck > chk ? ck : chk;
-      }
-    }
-    mismatch = (__ballot_sync(FULLM, mism) & gmask) != 0;
-#pragma unroll
-    for (int h = 1; h < L; h <<= 1) { const u64 o = shfl_xor64(chk, h); chk = o > chk ? o : chk; }
-  }
-  const bool barrier = have_first && gop == CCLD_OP_ALLREDUCE && gbytes < P.barrier_bytes;
-  const bool analysed = complete && !barrier && n >= P.min_group;
-  const bool add_bw = complete && !barrier;
-  const bool hang = active && !complete && inflight && age > P.hang_ns && !barrier;
-  u32 gfl = (mismatch ? CCLD_G_OPSET_MISMATCH : 0) | (barrier ? CCLD_G_BARRIER : 0) | (inflight ? CCLD_G_INFLIGHT : 0) |
-            (bad_time ? CCLD_G_BAD_TIME : 0) | (complete ? CCLD_G_COMPLETE : CCLD_G_INCOMPLETE) | (analysed ? CCLD_G_ANALYSED : 0) |
-            (hang ? CCLD_G_HANG_ALERT : 0);
-
-  // ---- order statistics, flags, bandwidths ----
-  u64 med_s = 0, mad_s = 0, med_d = 0, mad_d = 0;
-  u64 packed = 0;                                            // my eight flag bytes
-#pragma unroll
-  for (int q = 0; q < 8; ++q)
-    if (p0 + q < n) packed |= (u64)(CCLD_F_NOT_ANALYSED | (idx[q] == NONE ? CCLD_F_MISSING : 0)) << (8 * q);
-  double bw[8];
-#pragma unroll
-  for (int q = 0; q < 8; ++q) bw[q] = 0.0;
-  double num = 1.0, den = 1.0; bus_factor(gop, n, &num, &den);
-  const double bn = (double)gbytes * num;
-  if (__any_sync(FULLM, analysed && fast)) {
-    u32 ms, ds, md, dm;
-    sub_median_mad<L, u32>(sk, n, s, lane, &ms, &ds);
-    sub_median_mad<L, u32>(dd, n, s, lane, &md, &dm);
-    if (analysed && fast) {
-      med_s = ms; mad_s = ds; med_d = tmin + md; mad_d = dm;
-      // |x - med| * 1000 > k * MAD  <=>  |x - med| > floor(k * MAD / 1000); deviations are below 2^32
-      const u64 qs = (u64)ds * k_milli / 1000u, qd = (u64)dm * k_milli / 1000u;
-      const u32 ts = qs > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)qs, td = qd > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)qd;
-      packed = 0;
-#pragma unroll
-      for (int q = 0; q < 8; ++q) {
-        if (p0 + q < n) {
-          const u32 a = sk[q] >= ms ? sk[q] - ms : ms - sk[q], b = dd[q] >= md ? dd[q] - md : md - dd[q];
-          const bool so = a > ts, sh = sk[q] > ms, dq = b > td, dh = dd[q] > md;
-          packed |= (u64)((so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0)) << (8 * q);
-        }
-      }
-    }
-  }
-  if (add_bw && fast) {
-#pragma unroll
-    for (int q = 0; q < 8; ++q) if (p0 + q < n) bw[q] = busbw_fast(bn, den, (i64)(tmin + dd[q]));
-  }
-  if (__any_sync(FULLM, complete && !fast)) {
-    u64 o4[4] = {0, 0, 0, 0};
-    sub_group64<L>(D, R, mem, pslot, row.n_seq, n, s, lane, complete && !fast, e_min, k_milli, analysed, add_bw, bn, den, o4, &packed);
-    if (analysed && !fast) { med_s = o4[0]; mad_s = o4[1]; med_d = o4[2]; mad_d = o4[3]; }
-  }
-  u32 n_fs = 0, n_fd = 0;
-  if (analysed) {
-#pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      if (p0 + q < n) {
-        const u32 f = (u32)(packed >> (8 * q));
-        if (f & CCLD_F_SKEW_OUT) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p0 + q] * 4 + ((f & CCLD_F_SKEW_HI) ? 0 : 1)], 1u); }
-        if (f & CCLD_F_DUR_OUT) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p0 + q] * 4 + ((f & CCLD_F_DUR_HI) ? 2 : 3)], 1u); }
-      }
-    }
-  }
-  // ---- outputs: every lane its flag bytes, the group's first lane the row ----
-  if (active) {
-    const u64 slot = row.slot0 + (u64)(t.seq_off + j) * n + p0;
-    if (p0 + 8 <= n && (slot & 7) == 0) *reinterpret_cast<u64*>(D.flags + slot) = packed;
-    else {
-#pragma unroll
-      for (int q = 0; q < 8; ++q) if (p0 + q < n) D.flags[slot + q] = (u8)(packed >> (8 * q));
-    }
-  }
-  if (lead) {
-    const u64 g = row.group0 + t.seq_off + j, G = D.n_groups;
-    if (hang) raise_alert(D, R.comm_id[c], row.seq_lo + t.seq_off + j, age);
-    const i64 span = complete ? x_max - (i64)e_min : 0;
-    D.gi64[(u64)GI_E_MIN * G + g] = complete ? (i64)e_min : 0; D.gi64[(u64)GI_ARRIVAL_SKEW * G + g] = complete ? (i64)(e_max - e_min) : 0;
-    D.gi64[(u64)GI_T_MAX * G + g] = complete ? (i64)tmax : 0; D.gi64[(u64)GI_T_MIN * G + g] = complete ? (i64)tmin : 0;
-    D.gi64[(u64)GI_SPAN * G + g] = span;
-    D.gi64[(u64)GI_MED_SKEW * G + g] = (i64)med_s; D.gi64[(u64)GI_MAD_SKEW * G + g] = (i64)mad_s;
-    D.gi64[(u64)GI_MED_DUR * G + g] = (i64)med_d; D.gi64[(u64)GI_MAD_DUR * G + g] = (i64)mad_d;
-    D.gu32[(u64)GU_RANK_TMIN * G + g] = complete ? mem[pmin] : 0; D.gu32[(u64)GU_RANK_TMAX * G + g] = complete ? mem[pmax] : 0;
-    D.gu32[(u64)GU_MAX_CHG * G + g] = complete ? (u32)(chk >> 32) : 0;
-    D.gu32[(u64)GU_RANK_MAX_CHG * G + g] = complete ? mem[NONE - (u32)chk] : 0;
-    D.gu32[(u64)GU_N_PRESENT * G + g] = npres; D.gu32[(u64)GU_GFLAGS * G + g] = gfl;
-    D.gbw[g] = complete ? busbw_fast(bn, den, span) : 0.0;
-  }
-
-  // ---- per-warp accumulation ----
-  const bool is_round = lead && add_bw;
-  const u32 b_comp = __ballot_sync(FULLM, lead && complete), b_inc = __ballot_sync(FULLM, lead && !complete);
-  const u32 b_bar = __ballot_sync(FULLM, lead && barrier), b_an = __ballot_sync(FULLM, lead && analysed);
-  const u32 b_mis = __ballot_sync(FULLM, lead && mismatch), b_bwc = __ballot_sync(FULLM, is_round);
-  const u32 pres = __reduce_add_sync(FULLM, lead ? npres : 0u), fs = __reduce_add_sync(FULLM, n_fs), fd = __reduce_add_sync(FULLM, n_fd);
-  u64 brng = is_round ? tmax - tmin : 0; u32 bk = is_round ? t.seq_off + j : NONE;
-  best_warp_reduce(brng, bk);
-  // bandwidth sums over the warp's groups: each round halves the values a lane carries
-  u32 off = 0;
-#pragma unroll
-  for (int bit = 16, w = 4; bit >= L; bit >>= 1, w >>= 1) {
-    const bool hi = (lane & bit) != 0;
-#pragma unroll
-    for (int i = 0; i < w; ++i) {
-      const double send = hi ? bw[i] : bw[i + w], keep = hi ? bw[i + w] : bw[i];
-      bw[i] = keep + __shfl_xor_sync(FULLM, send, bit);
-    }
-    off += hi ? (u32)w : 0u;
-  }
-#pragma unroll
-  for (int i = 0; i < 8 / GW; ++i) sh.bw[wid][p0 + off + i] = bw[i];
-  if (lane == 0) {
-    sh.brng[wid] = brng; sh.bk[wid] = bk; sh.rounds[wid] = (u32)__popc(b_bwc); sh.n_an[wid] = (u32)__popc(b_an);
-    if (b_comp) atomicAdd(&sh.cnt[SC_COMP], (u32)__popc(b_comp));
-    if (b_inc) atomicAdd(&sh.cnt[SC_INC], (u32)__popc(b_inc));
-    if (b_bar) atomicAdd(&sh.cnt[SC_BAR], (u32)__popc(b_bar));
-    if (b_an) atomicAdd(&sh.cnt[SC_AN], (u32)__popc(b_an));
-    if (b_mis) atomicAdd(&sh.cnt[SC_MIS], (u32)__popc(b_mis));
-    if (pres) atomicAdd(&sh.cnt[SC_PRES], pres);
-    if (fs) atomicAdd(&sh.cnt[SC_FS], fs);
-    if (fd) atomicAdd(&sh.cnt[SC_FD], fd);
-  }
-}
-
-// Class-1 CTA of the fused kernel: one tile of 2048 / n_pad consecutive op counters of one communicator.
-__device__ __forceinline__ void reduce_sub_cta(const WinDesc& D, const FusedCta& t, TileSum* __restrict__ sums, const Registry& R, const Params& P, i64 now) {
-  __shared__ SubShared sh;
-  const u32 n = t.row.n, n_pad = mid_npad(n);
-  if (threadIdx.x < SC_COUNT) sh.cnt[threadIdx.x] = 0;
-  __syncthreads();
-  if (n_pad == 32) reduce_sub_warp<4>(D, t, R, P, now, sh);
-  else if (n_pad == 64) reduce_sub_warp<8>(D, t, R, P, now, sh);
-  else reduce_sub_warp<16>(D, t, R, P, now, sh);
-  __syncthreads();
-  u32 rounds = 0;
-#pragma unroll
-  for (int q = 0; q < MID_THREADS / 32; ++q) rounds += sh.rounds[q];
-  if (rounds) {
-    const u32* mem = R.members + t.moff;
-    for (u32 p = threadIdx.x; p < n; p += MID_THREADS) {
-      double v = 0.0;
-#pragma unroll
-      for (int q = 0; q < MID_THREADS / 32; ++q) v += sh.bw[q][p];
-      atomicAdd(&R.bw_sum[mem[p]], v);
-      atomicAdd(&R.bw_cnt[mem[p]], rounds);
-    }
-  }
-  if (threadIdx.x == 0) {
-    u64 brng = sh.brng[0]; u32 bk = sh.bk[0], n_an = sh.n_an[0];
-    for (int q = 1; q < MID_THREADS / 32; ++q) { best_merge(brng, bk, sh.brng[q], sh.bk[q]); n_an += sh.n_an[q]; }
-    TileSum ts; ts.best_rng = brng; ts.best_k = bk; ts.n_rounds = rounds; ts.n_an = n_an; ts.pad = 0;
-    sums[t.sum_idx] = ts;
-    count_add(D.counters, C_COMPLETE, sh.cnt[SC_COMP]); count_add(D.counters, C_INCOMPLETE, sh.cnt[SC_INC]); count_add(D.counters, C_BARRIER, sh.cnt[SC_BAR]);
-    count_add(D.counters, C_ANALYSED, sh.cnt[SC_AN]); count_add(D.counters, C_MISMATCH, sh.cnt[SC_MIS]); count_add(D.counters, C_PRESENT, sh.cnt[SC_PRES]);
-    count_add(D.counters, C_FLAG_SKEW, sh.cnt[SC_FS]); count_add(D.counters, C_FLAG_DUR, sh.cnt[SC_FD]);
-  }
-}
-
-// ------------------------------------------------------------------------------------------------
-// fused reduce kernel for communicators of up to 128 ranks: the work list is chunk-major, so CTAs that
-// run together gather from the same stretch of every rank's records
-// ------------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(SMALL_SEQS, 2) k_reduce_fused(const WinDesc* __restrict__ wd, const FusedCta* __restrict__ ctas,
-                                                             const WarpTile* __restrict__ wts, TileSum* __restrict__ sums, Registry R, Params P, i64 now) {
-  const FusedCta t = ctas[blockIdx.x];
-  const WinDesc& D = wd[t.w];
-  if (t.cls == 0) reduce_small_cta(D, t, wts, sums, R, P, now);
-  else reduce_sub_cta(D, t, sums, R, P, now);
-}
-
-// ------------------------------------------------------------------------------------------------
 // per-op reductions, n > 1024: one CTA per group; enter times and durations live in shared memory,
 // order statistics by most-significant-byte-first radix select
 // ------------------------------------------------------------------------------------------------
@@ -1763,10 +1040,22 @@ __global__ void __launch_bounds__(128) k_window_decide(const WinDesc* __restrict
     const u32 nt = row.n_units;
     u32 n_rounds = 0, n_an = 0;
     u64 best_rng = 0; u32 best_k = NONE;
+    bool redo = false;                                     // a unit left groups to the deferred kernel: its summary is partial
     for (u32 q = lane; q < nt; q += 32) {
       const TileSum x = ts[q];
       n_rounds += x.n_rounds; n_an += x.n_an;
       best_merge(best_rng, best_k, x.best_rng, x.best_k);
+      redo = redo || x.pad != 0;
+    }
+    if (__any_sync(0xFFFFFFFFu, redo)) {
+      // recount the communicator's window from the per-op rows
+      const u32* gfl = D.gu32 + (u64)GU_GFLAGS * G + row.group0;
+      n_rounds = 0; n_an = 0; best_rng = 0; best_k = NONE;
+      for (u32 k = lane; k < row.n_seq; k += 32) {
+        const u32 f = gfl[k];
+        if ((f & CCLD_G_COMPLETE) && !(f & CCLD_G_BARRIER)) { ++n_rounds; best_merge(best_rng, best_k, (u64)(t_max[k] - t_min[k]), k); }
+        if (f & CCLD_G_ANALYSED) ++n_an;
+      }
     }
     n_rounds = __reduce_add_sync(0xFFFFFFFFu, n_rounds); n_an = __reduce_add_sync(0xFFFFFFFFu, n_an);
     best_warp_reduce(best_rng, best_k);
