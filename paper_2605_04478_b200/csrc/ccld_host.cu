@@ -396,7 +396,8 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   size_t off = 0;
   auto take = [&](size_t b) { size_t o = off; off = align_up(off + b); return o; };
   const size_t o_desc = take(B * sizeof(WinDesc)), o_rmin = take((size_t)B * nc * 4), o_rmax = take((size_t)B * nc * 4),
-               o_rng = take((size_t)B * nc * sizeof(RangeRow)), o_srow = take((size_t)B * nc * sizeof(uint4)), o_tot = take((size_t)B * T_COUNT * 8), o_cnt = take((size_t)B * C_COUNT * 8);
+               o_rng = take((size_t)B * nc * sizeof(RangeRow)), o_srow = take((size_t)B * nc * sizeof(uint4)), o_tot = take((size_t)B * T_COUNT * 8), o_cnt = take((size_t)B * C_COUNT * 8),
+               o_cta0 = take((size_t)B * 4);
   cudaError_t e;
   Block pb = ctx->pool.get(off, &e);
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "plan allocation failed");
@@ -422,8 +423,12 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   CK(cudaMemsetAsync(pbase, 0, off, st));
   CK(cudaMemsetAsync(pbase + o_rmin, 0xFF, (size_t)B * nc * 4, st));
   CK(cudaMemcpyAsync(d_desc, hd.data(), B * sizeof(WinDesc), cudaMemcpyHostToDevice, st));
+  std::vector<u32> h_cta0(B);
+  for (u32 k = 0; k < B; ++k) h_cta0[k] = hd[k].cta0;
+  u32* d_cta0 = (u32*)(pbase + o_cta0);
+  CK(cudaMemcpyAsync(d_cta0, h_cta0.data(), B * 4ull, cudaMemcpyHostToDevice, st));
   TimerSlot* ts = timer_begin(ctx);
-  if (cta > 0) { TimedLaunch tl(ts, 0, st); k_seq_range<<<(u32)cta, REC_THREADS, 0, st>>>(d_desc, B, ctx->reg); }
+  if (cta > 0) { TimedLaunch tl(ts, 0, st); k_seq_range<<<(u32)cta, REC_THREADS, 0, st>>>(d_desc, d_cta0, B, ctx->reg); }
   { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, PlanLists{nullptr, nullptr, nullptr, nullptr}, 0); }
   CK(cudaGetLastError());
   { int rc = ensure_pinned(ctx, (size_t)B * T_COUNT * 8); if (rc != CCLD_OK) return rc; }
@@ -471,7 +476,7 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   if (total_slots) CK(cudaMemsetAsync(rbase + o_perm, 0xFF, total_slots * 4, st));
   PlanLists pl; pl.fcta = (FusedCta*)(rbase + o_fcta); pl.fwt = (WarpTile*)(rbase + o_fwt); pl.t2 = (Tile*)(rbase + o_t2); pl.t3 = (Tile*)(rbase + o_t3);
   { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, pl, 1); }
-  if (cta > 0) { TimedLaunch tl(ts, 2, st); k_slot_scatter<<<(u32)cta, SCAT_THREADS, 0, st>>>(d_desc, B, ctx->reg); }
+  if (cta > 0) { TimedLaunch tl(ts, 2, st); k_slot_scatter<<<(u32)cta, SCAT_THREADS, 0, st>>>(d_desc, d_cta0, B, ctx->reg); }
   if (n_list[B_FCTA]) {
     const DeferList dl{(u64*)(rbase + o_def), (u32*)(rbase + o_defn)};
     CK(cudaMemsetAsync(rbase + o_defn, 0, 8, st));

@@ -45,11 +45,14 @@ __device__ __forceinline__ u32 pos_lookup(const Registry& R, u32 rank, u32 c) {
   return NONE;
 }
 
-__device__ __forceinline__ u32 find_window(const WinDesc* wd, u32 nw, u32 cta) {
+// Which window of the batch a CTA of the record-streaming grids works on: the last window whose first CTA is <= cta.
+// cta0 is a compact copy of the descriptors' first-CTA fields (a few cache lines that every CTA hits in L1 / L2; the
+// descriptors themselves are a line apart each, and a search through them costs a chain of memory round trips per CTA).
+__device__ __forceinline__ u32 find_window(const u32* __restrict__ cta0, u32 nw, u32 cta) {
   u32 lo = 0, hi = nw - 1;
   while (lo < hi) {
     u32 mid = (lo + hi + 1) >> 1;
-    if (wd[mid].cta0 <= cta) lo = mid; else hi = mid - 1;
+    if (__ldg(cta0 + mid) <= cta) lo = mid; else hi = mid - 1;
   }
   return lo;
 }
@@ -150,47 +153,51 @@ __device__ __forceinline__ void range_note(const WinDesc& D, u32* t_key, u32* t_
 }
 
 // ---- group-by, part 1: which op counters does every communicator cover in every window ----
-__global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __restrict__ wd, u32 nw, Registry R) {
+__global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __restrict__ wd, const u32* __restrict__ cta0, u32 nw, Registry R) {
   __shared__ u32 s_comm[REC_THREADS * REC_PITCH], s_seq[REC_THREADS * REC_PITCH];
   __shared__ u32 t_key[RANGE_TAB], t_mn[RANGE_TAB], t_mx[RANGE_TAB];
   if (threadIdx.x < RANGE_TAB) { t_key[threadIdx.x] = NONE; t_mn[threadIdx.x] = NONE; t_mx[threadIdx.x] = 0; }
-  const u32 w = find_window(wd, nw, blockIdx.x);
+  const u32 w = find_window(cta0, nw, blockIdx.x);
   const WinDesc& D = wd[w];
   const u64 first = (u64)(blockIdx.x - D.cta0) * REC_PER_CTA;
   const u32 n_valid = D.n_rec - first < REC_PER_CTA ? (u32)(D.n_rec - first) : (u32)REC_PER_CTA;
   stage_column(D.comm, first, n_valid, s_comm);
   stage_column(D.seq, first, n_valid, s_seq);
   __syncthreads();
-  // cached communicators: id, index (NONE = unregistered), seq0, smallest / largest counter seen (empty: mn > mx)
-  u32 e_cid[RC], e_c[RC], e_s0[RC], e_mn[RC], e_mx[RC]; int cn = 0;
+  // Cached communicators: id, index (NONE = unregistered or empty entry), first valid counter, smallest / largest counter
+  // seen (empty: mn > mx). The walk itself is branch-free: a record updates the entry whose id it carries if its counter
+  // is valid; an empty entry has id NONE and index NONE, so a record that names communicator NONE lands nowhere.
+  u32 e_cid[RC], e_c[RC], e_s0[RC], e_mn[RC], e_mx[RC]; u32 next = 0;
+#pragma unroll
+  for (int e = 0; e < RC; ++e) { e_cid[e] = NONE; e_c[e] = NONE; e_s0[e] = NONE; e_mn[e] = NONE; e_mx[e] = 0; }
   const u32 r0 = threadIdx.x * REC_RUN;
   const u32 len = r0 >= n_valid ? 0u : (n_valid - r0 < REC_RUN ? n_valid - r0 : (u32)REC_RUN);
   const u32* pc = s_comm + threadIdx.x * REC_PITCH; const u32* ps = s_seq + threadIdx.x * REC_PITCH;
+#pragma unroll 4
   for (u32 k = 0; k < len; ++k) {
     const u32 cid = pc[k], sq = ps[k];
     bool hit = false;
 #pragma unroll
     for (int e = 0; e < RC; ++e) {
-      if (e < cn && e_cid[e] == cid) {
-        hit = true;
-        if (e_c[e] != NONE && sq >= e_s0[e]) { e_mn[e] = sq < e_mn[e] ? sq : e_mn[e]; e_mx[e] = sq > e_mx[e] ? sq : e_mx[e]; }
-      }
+      const bool h = e_cid[e] == cid, upd = h && sq >= e_s0[e];
+      e_mn[e] = upd ? min(e_mn[e], sq) : e_mn[e]; e_mx[e] = upd ? max(e_mx[e], sq) : e_mx[e];
+      hit = hit || h;
     }
     if (!hit) {
-      if (cn == RC) {
+      // the oldest entry makes room (its extremes go to the CTA's table)
+      u32 o_c = NONE, o_mn = NONE, o_mx = 0;
 #pragma unroll
-        for (int e = 0; e < RC; ++e) if (e_c[e] != NONE && e_mn[e] <= e_mx[e]) range_note(D, t_key, t_mn, t_mx, e_c[e], e_mn[e], e_mx[e]);
-        cn = 0;
-      }
+      for (int e = 0; e < RC; ++e) if ((u32)e == next) { o_c = e_c[e]; o_mn = e_mn[e]; o_mx = e_mx[e]; }
+      if (o_c != NONE && o_mn <= o_mx) range_note(D, t_key, t_mn, t_mx, o_c, o_mn, o_mx);
       const uint4 h = comm_find(R, cid, R.hash[hash_home(R, cid)]);
       const bool ok = h.y != NONE && sq >= h.z;
 #pragma unroll
-      for (int e = 0; e < RC; ++e) if (e == cn) { e_cid[e] = cid; e_c[e] = h.y; e_s0[e] = h.z; e_mn[e] = ok ? sq : NONE; e_mx[e] = ok ? sq : 0u; }
-      ++cn;
+      for (int e = 0; e < RC; ++e) if ((u32)e == next) { e_cid[e] = cid; e_c[e] = h.y; e_s0[e] = h.y != NONE ? h.z : NONE; e_mn[e] = ok ? sq : NONE; e_mx[e] = ok ? sq : 0u; }
+      next = (next + 1) & (RC - 1);
     }
   }
 #pragma unroll
-  for (int e = 0; e < RC; ++e) if (e < cn && e_c[e] != NONE && e_mn[e] <= e_mx[e]) range_note(D, t_key, t_mn, t_mx, e_c[e], e_mn[e], e_mx[e]);
+  for (int e = 0; e < RC; ++e) if (e_c[e] != NONE && e_mn[e] <= e_mx[e]) range_note(D, t_key, t_mn, t_mx, e_c[e], e_mn[e], e_mx[e]);
   __syncthreads();
   if (threadIdx.x < RANGE_TAB && t_key[threadIdx.x] != NONE) range_widen(D, t_key[threadIdx.x], t_mn[threadIdx.x], t_mx[threadIdx.x]);
 }
@@ -463,8 +470,9 @@ __device__ __noinline__ u64 resolve_slow(const Registry& R, u32 rank, u32 cid) {
   return (c << RANK_TAB_POS_BITS) | pos;
 }
 
-__global__ void __launch_bounds__(SCAT_THREADS) k_slot_scatter(const WinDesc* __restrict__ wd, u32 nw, Registry R) {
-  const u32 w = find_window(wd, nw, blockIdx.x);
+// four CTAs per SM (64 registers): the kernel waits on its dependent table loads, so resident warps are what it needs
+__global__ void __launch_bounds__(SCAT_THREADS, 4) k_slot_scatter(const WinDesc* __restrict__ wd, const u32* __restrict__ cta0, u32 nw, Registry R) {
+  const u32 w = find_window(cta0, nw, blockIdx.x);
   const WinDesc& D = wd[w];
   const u64 base = (u64)(blockIdx.x - D.cta0) * REC_PER_CTA;
   u32 err = 0, rej = 0, internal = 0;
