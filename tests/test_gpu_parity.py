@@ -430,3 +430,25 @@ def test_opset_consistency_against_the_oracle():
     an.trace_attach_opset(0, torch.from_numpy(proto).cuda(), torch.from_numpy(algo).cuda())   # device columns, swapped
     assert o.attach_opset(0, proto, algo) == 0
     check()
+
+
+def test_a_silent_rank_sends_every_group_of_its_communicators_to_the_general_path():
+    """One rank reports nothing and another one's ops are all in flight: every group of their communicators is incomplete,
+    so whole work units of the fused kernel are handed to the kernel for irregular groups, next to communicators that
+    stay on the fast path. Windows start 30 s apart, so op times also cross many 2^32 ns boundaries."""
+    spec = tg.cfg2(reps=40, n_windows=2, tp=8, pp=2, dp=16)
+    spec.t0_ns = 30_000_000_000
+    an, o = make_pair(tg.registry(spec))
+    silent, stuck = 5, 77
+    for w in range(2):
+        win = tg.gen_window(spec, w, device="cuda")
+        keep = win.cols["rank"] != silent
+        cols = {k: v[keep].clone() for k, v in win.cols.items()}
+        cols["t_exit"][cols["rank"] == stuck] = -1
+        an.trace_upload(w, cols); assert o.upload(w, cols) == 0
+        now = win.now_ns
+    an.analyze_window(0, 2, now); assert o.analyze(0, 2, now) == 0
+    for w in range(2):
+        v, _ = compare_window(an, o, w)
+        assert v["n_incomplete"] > 0 and v["n_complete"] > 0
+    compare_cumulative(an, o, spec.n_ranks, 1)
