@@ -810,24 +810,31 @@ inline size_t mid_smem_bytes(u32 n_pad_min) {
 // per-op reductions, n > 1024: one CTA per group; enter times and durations live in shared memory,
 // order statistics by most-significant-byte-first radix select
 // ------------------------------------------------------------------------------------------------
+// Reduction over the CTA (all threads call; blockDim.x a multiple of 32): warps reduce by shuffles, the first warp
+// reduces the warps' partial results the same way, everyone reads the result from s_red[0].
 template <class T, class Op>
 __device__ T block_reduce(T v, Op op, T* s_red /*[32]*/) {
-  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
 #pragma unroll
   for (int d = 16; d > 0; d >>= 1) { T o = __shfl_xor_sync(0xFFFFFFFFu, v, d); v = op(v, o); }
   __syncthreads();
   if (lane == 0) s_red[wid] = v;
   __syncthreads();
-  T r = s_red[0];
-  for (u32 q = 1; q < blockDim.x / 32; ++q) r = op(r, s_red[q]);
-  return r;
+  if (wid == 0) {
+    T x = lane < nw ? s_red[lane] : Op::identity();
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) { T o = __shfl_xor_sync(0xFFFFFFFFu, x, d); x = op(x, o); }
+    if (lane == 0) s_red[0] = x;
+  }
+  __syncthreads();
+  return s_red[0];
 }
-struct OpMinU64 { __device__ u64 operator()(u64 a, u64 b) const { return a < b ? a : b; } };
-struct OpMaxU64 { __device__ u64 operator()(u64 a, u64 b) const { return a > b ? a : b; } };
-struct OpMaxI64 { __device__ i64 operator()(i64 a, i64 b) const { return a > b ? a : b; } };
-struct OpAddU32 { __device__ u32 operator()(u32 a, u32 b) const { return a + b; } };
-struct OpOrU32 { __device__ u32 operator()(u32 a, u32 b) const { return a | b; } };
-struct OpMinU32 { __device__ u32 operator()(u32 a, u32 b) const { return a < b ? a : b; } };
+struct OpMinU64 { __device__ u64 operator()(u64 a, u64 b) const { return a < b ? a : b; } static __device__ u64 identity() { return U64_MAX_; } };
+struct OpMaxU64 { __device__ u64 operator()(u64 a, u64 b) const { return a > b ? a : b; } static __device__ u64 identity() { return 0; } };
+struct OpMaxI64 { __device__ i64 operator()(i64 a, i64 b) const { return a > b ? a : b; } static __device__ i64 identity() { return INT64_MIN; } };
+struct OpAddU32 { __device__ u32 operator()(u32 a, u32 b) const { return a + b; } static __device__ u32 identity() { return 0; } };
+struct OpOrU32 { __device__ u32 operator()(u32 a, u32 b) const { return a | b; } static __device__ u32 identity() { return 0; } };
+struct OpMinU32 { __device__ u32 operator()(u32 a, u32 b) const { return a < b ? a : b; } static __device__ u32 identity() { return NONE; } };
 
 // k-th smallest (0-based) of key(i), i < n; max_key bounds the keys. All threads of the CTA call it.
 template <class F>
