@@ -43,13 +43,19 @@ def parse():
     ap.add_argument("--windows", type=int, default=100, help="windows of 1,000 ops per rank resident on the GPU")
     ap.add_argument("--e2e-windows", type=int, default=10, help="windows per end-to-end step (host buffers)")
     ap.add_argument("--cpu-windows", type=int, default=10, help="windows the CPU oracle is timed on")
+    ap.add_argument("--mix", default="all", choices=sorted(MIXES), help="all: the cfg4 workload; tp_pp / dp: only its 8-rank or only its 64-rank "
+                    "communicators (timing one path of the fused kernel; the headline number is --mix all)")
     ap.add_argument("--rate-windows", type=int, default=2, help="windows whose raw probe samples are turned into rate columns (0 = skip)")
     return ap.parse_args()
 
 
-def workload(n_windows, rank=0):
+MIXES = {"all": ((0, 0, 1, 0, 2), 200), "tp_pp": ((0, 0, 1, 0), 250), "dp": ((2,), 200)}   # op pattern (0 TP, 1 PP, 2 DP), repetitions
+
+
+def workload(n_windows, rank=0, mix="all"):
     import tracegen as tg
-    spec = tg.cfg4(n_windows=n_windows)
+    pattern, reps = MIXES[mix]
+    spec = tg.cfg4(reps=reps, n_windows=n_windows, pattern=pattern)
     spec.seed += 1000 * rank
     return spec
 
@@ -183,12 +189,12 @@ def run_ours(args, rank, world, local_rank):
 
     cpu_base = None
     if rank == 0 and world == 1 and args.cpu_windows > 0:
-        spec0 = workload(args.windows)
+        spec0 = workload(args.windows, 0, args.mix)
         r, t = time_oracle(spec0, list(range(min(args.cpu_windows, spec0.n_windows))), gen_device=dev)
         cpu_base = {"value": r / t, "unit": UNIT, "cores": 1, "kind": "oracle",
                     "sample": "%d of %d windows (%.3f M records), single thread" % (min(args.cpu_windows, spec0.n_windows), spec0.n_windows, r / 1e6)}
 
-    spec = workload(args.windows, rank)
+    spec = workload(args.windows, rank, args.mix)
     NW = spec.n_windows
     an = ccld.Analyzer(device=local_rank)
     for cid, ranks, seq0 in tg.registry(spec):
@@ -335,7 +341,8 @@ def run_ours(args, rank, world, local_rank):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int64", "data": "synthetic",
-            "config": {"workload": "cfg4 streaming slow mix: 4,096 ranks (TP8 x PP8 x DP64), %d windows of 1,000 ops per rank, rank-major upload order" % NW,
+            "config": {"workload": "cfg4 streaming slow mix: 4,096 ranks (TP8 x PP8 x DP64), %d windows of %s ops per rank, rank-major upload order%s"
+                                   % (NW, format(spec.ops_per_window, ","), "" if args.mix == "all" else " (--mix %s: one communicator class only)" % args.mix),
                        "records_per_gpu": n_rec, "bytes_per_record": REC_BYTES, "l2": "inputs larger than L2 (%.1f GB of columns per GPU)" % (n_rec * REC_BYTES / 1e9),
                        "injected_ranks_recovered": recovered},
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu_base,

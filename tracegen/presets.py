@@ -71,8 +71,9 @@ def cfg3(n_rings: int = 16, ring: int = 256, n_done: int = 100, hung_ring: int =
     return s
 
 
-def cfg4(reps: int = 200, n_windows: int = 100, tp: int = 8, pp: int = 8, dp: int = 64) -> Spec:
-    s = _three_d("cfg4", 3, tp, pp, dp, [0, 0, 1, 0, 2], reps, n_windows)
+def cfg4(reps: int = 200, n_windows: int = 100, tp: int = 8, pp: int = 8, dp: int = 64, pattern=(0, 0, 1, 0, 2)) -> Spec:
+    """pattern: communicator family of each op slot (0 TP, 1 PP, 2 DP); other patterns single out one kernel path."""
+    s = _three_d("cfg4", 3, tp, pp, dp, list(pattern), reps, n_windows)
     r = _pick(s.seed, 1, s.n_ranks, 7)
     s.faults = ([Fault(x, "delay_exp", 200, 500_000) for x in r[:4]]
                 + [Fault(x, "bw", factor_milli=500) for x in r[4:6]]
