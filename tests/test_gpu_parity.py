@@ -452,3 +452,48 @@ def test_a_silent_rank_sends_every_group_of_its_communicators_to_the_general_pat
         v, _ = compare_window(an, o, w)
         assert v["n_incomplete"] > 0 and v["n_complete"] > 0
     compare_cumulative(an, o, spec.n_ranks, 1)
+
+
+@pytest.mark.parametrize("seed", [101, 102, 103])
+def test_randomized_groups_with_random_damage(seed):
+    """Seeded random communicators of 2 to 128 ranks over two windows with every kind of irregularity sprinkled in at random
+    - missing records, ops in flight, exits before enters, negative times, spreads beyond 2^32 ns, barriers, differing
+    sizes and ops - so that regular and irregular groups share warps and work units of the fused kernel."""
+    rng = np.random.default_rng(seed)
+    sizes = [int(x) for x in rng.choice([2, 3, 5, 8, 8, 8, 9, 16, 24, 32, 33, 64, 64, 100, 128], size=9)]
+    recs, comms, r0 = [[], []], [], 0
+    for cid, n in enumerate(sizes):
+        ranks = [int(x) for x in (r0 + rng.permutation(n))]; r0 += n
+        comms.append((cid * 3 + 1, ranks, 5))
+        n_seq = int(rng.integers(20, 90))
+        for w in range(2):
+            durs = rng.integers(900_000, 1_300_000, size=(n_seq, n)).tolist()
+            ents = rng.integers(0, 60_000, size=(n_seq, n)).tolist()
+            g = group_trace(durs, ents, comm=cid * 3 + 1, ranks=ranks, seq0=5 + w * n_seq, t0=3_000_000_000 + w * 40_000_000_000,
+                            spacing=int(rng.choice([7_000_000, 900_000_000])), bytes=4 * MiB)
+            for r in g:
+                u = rng.random()
+                if u < 0.010: r["drop"] = True
+                elif u < 0.015: r["t_exit"] = -1
+                elif u < 0.020: r["t_exit"] = r["t_enter"] - 7
+                elif u < 0.023: r["t_enter"] = -r["t_enter"]
+                elif u < 0.028: r["t_exit"] += 6_000_000_000
+                elif u < 0.033: r["t_enter"] -= 2_500_000_000
+                elif u < 0.040: r["bytes"] = 8 * MiB
+                elif u < 0.045: r["op"] = ALLGATHER
+                r["send_chg"] = int(rng.integers(0, 9)); r["recv_chg"] = int(rng.integers(0, 9))
+            for s in rng.choice(n_seq, size=2, replace=False):
+                for r in g:
+                    if r["seq"] == 5 + w * n_seq + int(s): r["bytes"] = 2          # a barrier
+            recs[w] += [r for r in g if not r.pop("drop", False)]
+    an, o = make_pair(comms)
+    for w in range(2):
+        order = rng.permutation(len(recs[w]))
+        cols = make_cols([recs[w][i] for i in order])
+        an.trace_upload(w, cols); assert o.upload(w, cols) == 0
+    now = 3_000_000_000 + 500 * 10**9
+    an.analyze_window(0, 2, now); assert o.analyze(0, 2, now) == 0
+    for w in range(2):
+        v, _ = compare_window(an, o, w)
+        assert v["n_incomplete"] > 0 and v["n_complete"] > 0 and v["n_alerts_total"] > 0
+    compare_cumulative(an, o, r0, 1)
