@@ -43,7 +43,7 @@ def _load():
         _lib.orc_destroy.argtypes = [C.c_void_p]
         for name in ("orc_comm_register", "orc_upload", "orc_release", "orc_analyze", "orc_window_sizes",
                      "orc_copy_groups", "orc_copy_slots", "orc_copy_comm_rows", "orc_copy_alerts",
-                     "orc_copy_rank_stats", "orc_suspects", "orc_locate_hang", "orc_attach_opset", "orc_opset_check"):
+                     "orc_copy_rank_stats", "orc_suspects", "orc_locate_hang", "orc_attach_opset", "orc_opset_check", "orc_comm_set_layers"):
             getattr(_lib, name).restype = C.c_int
         _lib.orc_derive_rates.restype = None
     return _lib
@@ -82,6 +82,10 @@ class Oracle:
     def comm_register(self, comm: int, ranks, seq0: int = 0) -> int:
         r = _np(np.asarray(ranks), np.uint32)
         return self.lib.orc_comm_register(self.h, C.c_uint32(comm), _p(r), C.c_uint32(len(r)), C.c_uint32(seq0))
+
+    def comm_set_layers(self, comm: int, layers) -> int:
+        a = _np(layers, np.uint32)
+        return self.lib.orc_comm_set_layers(self.h, C.c_uint32(comm), _p(a))
 
     def upload(self, window_id: int, cols, frames=None, n_channels: int = 0) -> int:
         a = {

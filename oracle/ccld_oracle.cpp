@@ -17,6 +17,8 @@
 // forms for a counter that advances every tick, to additivity over adjacent ops and to a numpy restatement.
 // orc_opset_check (majority Operation Type Set of an op and the ranks that deviate) is pinned to hand cases and to a
 // collections.Counter restatement.
+// Tree communicators: the same-layer restriction is the paper's (Sec. 4.2.1); which lagging member is named is this
+// repository's rule ("parity unpinned"), pinned to hand cases.
 // "Parity unpinned" against the paper: the bus-bandwidth factor and the median/MAD convention,
 // because the paper defines neither (they are this repository's conventions, pinned only to
 // closed forms and hand values).
@@ -55,6 +57,7 @@ struct Params {
 
 struct Comm {
   u32 id; u32 seq0; std::vector<u32> ranks; std::unordered_map<u32, u32> pos;
+  std::vector<u32> layer;   // tree communicators: layer id of each member (empty: ring)
   // Eq. 1 state, carried across windows
   u64 rounds = 0; i64 t_first = 0; i64 sum_m = 0; u64 m = 0; u64 slow_count = 0;
 };
@@ -315,6 +318,17 @@ int orc_comm_register(void* h, u32 comm, const u32* ranks, u32 n, u32 seq0) {
   return 0;
 }
 
+// Tree communicators (Sec. 4.2.1: only ranks of the same tree layer show consistent SendCount / RecvCount, so
+// diagnostics that compare them are restricted to same-layer ranks). layer[i] belongs to the i-th registered member.
+int orc_comm_set_layers(void* h, u32 comm, const u32* layer) {
+  Oracle* o = (Oracle*)h;
+  auto ci = o->comm_idx.find(comm);
+  if (ci == o->comm_idx.end()) return -1;
+  Comm& c = o->comms[ci->second];
+  c.layer.assign(layer, layer + c.ranks.size());
+  return 0;
+}
+
 int orc_upload(void* h, u32 wid, u64 n, const u32* rank, const u32* comm, const u32* seq, const u8* op, const u64* bytes,
                const i64* t_enter, const i64* t_exit, const u32* send_chg, const u32* recv_chg,
                u32 n_frames, const u32* f_rank, const u32* f_comm, const u32* f_seq, u32 n_channels, const u32* progress) {
@@ -471,15 +485,27 @@ int orc_locate_hang(void* h, u32 wid, u32 comm, u32 seq, u32* out, u64* min_tota
     for (u32 q = 0; q < n; ++q) if (frame[q] < 0) ++n_missing;
     u64 mn = *std::min_element(tot.begin(), tot.end());
     long root = -1, first_min = -1;
-    for (u32 q = 0; q < n; ++q) {
-      if (tot[q] != mn) continue;
-      if (first_min < 0) first_min = q;
-      if (root < 0 && tot[(q + n - 1) % n] > mn) root = q;        // most upstream rank of a run of minima
+    if (c.layer.empty()) {
+      for (u32 q = 0; q < n; ++q) {
+        if (tot[q] != mn) continue;
+        if (first_min < 0) first_min = q;
+        if (root < 0 && tot[(q + n - 1) % n] > mn) root = q;      // most upstream rank of a run of minima
+      }
+      if (root < 0) root = first_min;
+    } else {
+      // tree: a member is compared with its own layer only. Among the members that hold their layer's minimum while
+      // another member of the layer is ahead, the one furthest behind its layer's maximum; ties: the lowest position.
+      u64 best_lag = 0;
+      for (u32 q = 0; q < n; ++q) {
+        u64 lmn = tot[q], lmx = tot[q];
+        for (u32 x = 0; x < n; ++x) if (c.layer[x] == c.layer[q]) { lmn = std::min(lmn, tot[x]); lmx = std::max(lmx, tot[x]); }
+        if (tot[q] == lmn && lmx - lmn > best_lag) { best_lag = lmx - lmn; root = q; }
+      }
+      mn = root >= 0 ? tot[root] : 0;
     }
-    if (root < 0) root = first_min;
-    r.push_back(c.ranks[root]);
+    if (root >= 0) r.push_back(c.ranks[root]);
     *min_total = mn;
-    if (frame[root] >= 0) {
+    if (root >= 0 && frame[root] >= 0) {
       stuck = 0xFFFFFFFFu;
       for (u32 ch = 0; ch < w.n_channels; ++ch) stuck = std::min(stuck, w.progress[((u64)frame[root] * w.n_channels + ch) * 2 + 1]);
       if (w.n_channels == 0) stuck = 0;

@@ -634,3 +634,42 @@ def test_opset_majority_against_a_counter_restatement():
         r = o.opset_check(0, 0, s)
         assert (r["op"], r["bytes"], r["algo"], r["proto"]) == maj and r["majority_count"] == top and r["n_present"] == len(tup)
         assert list(r["ranks"]) == [q for q in ranks if q in tup and tup[q] != maj]
+
+
+# ---------------------------------------------------------------- tree communicators: same-layer comparison (Sec. 4.2.1)
+def _tree_hang(tots, layers, ring=False, drop_frame=None):
+    n = len(tots)
+    ranks = list(range(50, 50 + n))
+    recs = [dict(rank=r, comm=0, seq=0, t_enter=10**9, t_exit=-1) for r in ranks]
+    entries = [(ranks[i], 0, 0, [(tots[i] // 2, tots[i] - tots[i] // 2)]) for i in range(n) if i != drop_frame]
+    o = orc.Oracle()
+    assert o.comm_register(0, ranks, 0) == 0
+    if not ring:
+        assert o.comm_set_layers(0, layers) == 0
+    assert o.upload(0, make_cols(recs), frames_from(entries, 1), 1) == 0
+    assert o.analyze(0, 1, 10**9 + 400 * 10**9) == 0
+    return o.locate_hang(0, 0, 0), ranks
+
+
+def test_tree_hang_root_is_compared_with_its_own_layer_only():
+    layers = [0, 1, 1, 2, 2, 2, 2]
+    # the tree's root forwards little (3) and every leaf agrees (10): a ring would blame position 0, the tree names the
+    # layer-1 member that is 8 behind its peer
+    tots = [3, 20, 12, 10, 10, 10, 10]
+    h, ranks = _tree_hang(tots, layers, ring=True)
+    assert h["cls"] == 3 and list(h["roots"]) == [ranks[0]]
+    h, ranks = _tree_hang(tots, layers)
+    assert h["cls"] == 3 and list(h["roots"]) == [ranks[2]] and h["min_total"] == 12 and h["stuck_step"] == 6
+    # the largest gap inside a layer wins; equal gaps: the lowest position
+    h, ranks = _tree_hang([3, 20, 12, 10, 1, 10, 10], layers)
+    assert list(h["roots"]) == [ranks[4]] and h["min_total"] == 1
+    h, ranks = _tree_hang([3, 20, 12, 10, 2, 10, 10], layers)
+    assert list(h["roots"]) == [ranks[2]]
+    h, ranks = _tree_hang([3, 12, 20, 10, 10, 2, 10], layers)
+    assert list(h["roots"]) == [ranks[1]]
+    # every layer agrees with itself: the counters name nobody
+    h, ranks = _tree_hang([3, 20, 20, 10, 10, 10, 10], layers)
+    assert h["cls"] == 3 and h["n_roots"] == 0 and len(h["roots"]) == 0 and h["min_total"] == 0
+    # a member without a frame counts as zero and so lags its layer
+    h, ranks = _tree_hang([3, 20, 20, 10, 10, 10, 10], layers, drop_frame=5)
+    assert list(h["roots"]) == [ranks[5]] and h["n_missing_frames"] == 1 and h["stuck_step"] == 0
