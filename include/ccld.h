@@ -103,11 +103,28 @@ const char* ccld_last_error(ccld_ctx* ctx);
 /*
  * Communicator registration (the "domain initialization" of Sec. 2.1): `ranks` (host, n entries,
  * copied) lists the members in ring order - position p sends to position p+1 mod n -, which the
- * hang localizer uses. `algo` 0 = ring; 1 = tree is not supported yet (CCLD_ERR_ARG). `seq0` is
- * the communicator's first operation counter. All communicators must be registered before the
- * first ccld_analyze_window (later calls return CCLD_ERR_STATE). 1 <= n <= CCLD_MAX_COMM_SIZE.
+ * hang localizer uses. `algo` 0 = ring, 1 = tree (other values: CCLD_ERR_ARG); a tree communicator
+ * also needs ccld_comm_set_layers before its hangs can be located. `seq0` is the communicator's
+ * first operation counter. All communicators must be registered before the first
+ * ccld_analyze_window (later calls return CCLD_ERR_STATE). 1 <= n <= CCLD_MAX_COMM_SIZE.
  */
 int ccld_comm_register(ccld_ctx* ctx, uint32_t comm, const uint32_t* ranks, uint32_t n, uint8_t algo, uint32_t seq0);
+
+/*
+ * Tree communicators (Sec. 4.2.1): the SendCount / RecvCount of two members are comparable only
+ * when both sit in the same layer of the tree, so the diagnosis that compares them - branch H3 of
+ * the hang decision tree - is restricted to same-layer members. `layer` (host, one entry per
+ * member in the order given to ccld_comm_register, copied) names each member's layer; the ids are
+ * arbitrary, equal id = same layer. For such a communicator ccld_locate_hang / ccld_locate_hangs
+ * answer H3 like this: in every layer take the gap between the largest and the smallest counter
+ * total; the root is the member holding the minimum of the layer with the widest gap (equal gaps,
+ * or several holders: the lowest position); if no layer disagrees with itself n_roots_total = 0
+ * and min_total = 0. H1, H2 and the per-operation statistics (which compare times, not counters)
+ * treat a tree communicator like a ring. Errors: CCLD_ERR_STATE after the first analysis,
+ * CCLD_ERR_UNKNOWN_COMM, CCLD_ERR_ARG for a ring communicator or a null pointer. Locating a hang
+ * on a tree communicator whose layers were never set returns CCLD_ERR_STATE.
+ */
+int ccld_comm_set_layers(ccld_ctx* ctx, uint32_t comm, const uint32_t* layer);
 
 /*
  * Hands one window of trace records to the analyzer - what the rank probes push on kernel

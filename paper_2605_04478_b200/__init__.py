@@ -25,7 +25,8 @@ MAX_ALERTS_PER_WINDOW = 1024
 EXPORTS = ("ccld_params_default", "ccld_create", "ccld_destroy", "ccld_last_error", "ccld_comm_register",
            "ccld_trace_upload", "ccld_window_release", "ccld_analyze_window", "ccld_reset", "ccld_get_verdict",
            "ccld_locate_hang", "ccld_get_optable", "ccld_get_ranges", "ccld_get_rank_stats", "ccld_copy_to_host",
-           "ccld_timing_enable", "ccld_get_kernel_times", "ccld_ring_locate_static", "ccld_derive_rates", "ccld_locate_hangs", "ccld_state_export", "ccld_state_import", "ccld_trace_attach_opset", "ccld_opset_check")
+           "ccld_timing_enable", "ccld_get_kernel_times", "ccld_ring_locate_static", "ccld_derive_rates", "ccld_locate_hangs", "ccld_state_export", "ccld_state_import", "ccld_trace_attach_opset", "ccld_opset_check",
+           "ccld_comm_set_layers")
 STATIC_MAX_MEMBERS = 8192
 KERNEL_KINDS = ("k_seq_range", "k_plan", "k_slot_scatter", "k_reduce_fused", "k_reduce_mid", "k_reduce_large", "k_window_decide")
 
@@ -115,6 +116,7 @@ def load_library() -> C.CDLL:
         lib.ccld_create.argtypes = [C.POINTER(C.c_void_p), C.POINTER(Params), C.c_int, C.c_void_p]
         lib.ccld_destroy.argtypes = [C.c_void_p]
         lib.ccld_comm_register.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p, C.c_uint32, C.c_uint8, C.c_uint32]
+        lib.ccld_comm_set_layers.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
         lib.ccld_trace_upload.argtypes = [C.c_void_p, C.c_uint32, C.c_uint64, C.c_int] + [C.c_void_p] * 9 + \
                                          [C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p]
         lib.ccld_window_release.argtypes = [C.c_void_p, C.c_uint32]
@@ -239,6 +241,10 @@ class Analyzer:
     def comm_register(self, comm: int, ranks, algo: int = 0, seq0: int = 0) -> None:
         r = np.ascontiguousarray(np.asarray(ranks, dtype=np.uint32))
         self._check(self.lib.ccld_comm_register(self.h, comm, r.ctypes.data, len(r), algo, seq0))
+
+    def comm_set_layers(self, comm: int, layers) -> None:
+        a = np.ascontiguousarray(np.asarray(layers, dtype=np.uint32))
+        self._check(self.lib.ccld_comm_set_layers(self.h, comm, a.ctypes.data))
 
     def trace_upload(self, window_id: int, cols, frames=None, n_channels: int = 0) -> None:
         """cols: dict of torch tensors or numpy arrays, all on the CPU (copied) or all on this GPU (borrowed)."""

@@ -24,7 +24,12 @@ inline size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Block { void* p = nullptr; size_t bytes = 0; };
 
-struct CommHost { u32 id, seq0; std::vector<u32> ranks; };
+struct CommHost {
+  u32 id, seq0; std::vector<u32> ranks;
+  u8 algo = 0;                      // 0 ring, 1 tree
+  std::vector<u32> head;            // tree: lowest position of a member's layer (empty until the layers are set)
+  const u32* d_head = nullptr;      // device copy inside the registry block
+};
 
 // Device blocks are recycled through a free list so that steady-state analysis allocates nothing.
 struct Pool {
@@ -191,6 +196,8 @@ int finalize_registry(ccld_ctx* ctx) {
   auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes); return o; };
   const size_t o_hash = take(hsize * sizeof(uint4)), o_rtab = take(rank_tab.size() * 4), o_id = take(nc * 4), o_n = take(nc * 4), o_s0 = take(nc * 4), o_moff = take(nc * 8),
                o_mem = take(sum_n * 4), o_ptr = take((nr + 1) * 4ull), o_ec = take(sum_n * 4), o_ep = take(sum_n * 4);
+  std::vector<size_t> o_head(nc, 0);
+  for (u32 i = 0; i < nc; ++i) if (!ctx->comms[i].head.empty()) o_head[i] = take(ctx->comms[i].head.size() * 4);
   const size_t o_stats = off;
   const size_t o_state = take(nc * sizeof(CommState)), o_votes = take(nr * 16ull), o_ops = take(nr * 4ull), o_cnt = take(nr * 4ull), o_bw = take(nr * 8ull);
   cudaError_t e;
@@ -208,6 +215,12 @@ int finalize_registry(ccld_ctx* ctx) {
   CK(cudaMemcpyAsync(base + o_ptr, rank_ptr.data(), (nr + 1) * 4ull, cudaMemcpyHostToDevice, st));
   CK(cudaMemcpyAsync(base + o_ec, ent_comm.data(), sum_n * 4, cudaMemcpyHostToDevice, st));
   CK(cudaMemcpyAsync(base + o_ep, ent_pos.data(), sum_n * 4, cudaMemcpyHostToDevice, st));
+  for (u32 i = 0; i < nc; ++i) {
+    CommHost& c = ctx->comms[i];
+    if (c.head.empty()) continue;
+    CK(cudaMemcpyAsync(base + o_head[i], c.head.data(), c.head.size() * 4, cudaMemcpyHostToDevice, st));
+    c.d_head = (const u32*)(base + o_head[i]);
+  }
   CK(cudaMemsetAsync(base + o_stats, 0, off - o_stats, st));
   CK(cudaStreamSynchronize(st));              // the host vectors above go out of scope
   Registry& R = ctx->reg;
@@ -293,15 +306,30 @@ int ccld_comm_register(ccld_ctx* ctx, uint32_t comm, const uint32_t* ranks, uint
   if (!ctx) return CCLD_ERR_ARG;
   if (ctx->finalized) return fail(ctx, CCLD_ERR_STATE, "communicators must be registered before the first analysis");
   if (!ranks || n == 0) return fail(ctx, CCLD_ERR_ARG, "empty communicator");
-  if (algo != 0) return fail(ctx, CCLD_ERR_ARG, "only ring communicators (algo 0) are supported");
+  if (algo > 1) return fail(ctx, CCLD_ERR_ARG, "algo must be 0 (ring) or 1 (tree)");
   if (n > CCLD_MAX_COMM_SIZE) return fail(ctx, CCLD_ERR_CAPACITY, "communicator larger than CCLD_MAX_COMM_SIZE");
   if (ctx->comm_idx.count(comm)) return fail(ctx, CCLD_ERR_ARG, "communicator id registered twice");
-  CommHost c; c.id = comm; c.seq0 = seq0; c.ranks.assign(ranks, ranks + n);
+  CommHost c; c.id = comm; c.seq0 = seq0; c.algo = algo; c.ranks.assign(ranks, ranks + n);
   std::vector<u32> sorted(c.ranks); std::sort(sorted.begin(), sorted.end());
   if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return fail(ctx, CCLD_ERR_ARG, "rank listed twice in a communicator");
   if (sorted.back() >= CCLD_MAX_RANK_ID) return fail(ctx, CCLD_ERR_CAPACITY, "rank id not below CCLD_MAX_RANK_ID");
   ctx->comm_idx[comm] = (u32)ctx->comms.size();
   ctx->comms.push_back(std::move(c));
+  return CCLD_OK;
+}
+
+int ccld_comm_set_layers(ccld_ctx* ctx, uint32_t comm, const uint32_t* layer) {
+  if (!ctx) return CCLD_ERR_ARG;
+  if (ctx->finalized) return fail(ctx, CCLD_ERR_STATE, "layers must be set before the first analysis");
+  if (!layer) return fail(ctx, CCLD_ERR_ARG, "layer is null");
+  auto ci = ctx->comm_idx.find(comm);
+  if (ci == ctx->comm_idx.end()) return fail(ctx, CCLD_ERR_UNKNOWN_COMM, "unknown communicator");
+  CommHost& c = ctx->comms[ci->second];
+  if (c.algo != 1) return fail(ctx, CCLD_ERR_ARG, "layers belong to tree communicators (algo 1)");
+  const u32 n = (u32)c.ranks.size();
+  std::unordered_map<u32, u32> first;       // layer id -> lowest position that carries it
+  c.head.resize(n);
+  for (u32 p = 0; p < n; ++p) c.head[p] = first.emplace(layer[p], p).first->second;
   return CCLD_OK;
 }
 
@@ -554,6 +582,15 @@ int ccld_get_verdict(ccld_ctx* ctx, uint32_t window_id, ccld_verdict* out) {
   return CCLD_OK;
 }
 
+// Tree communicators compare progress counters inside a layer; the kernel needs the layer table for that.
+static int hang_layers(ccld_ctx* ctx, const CommHost& c, HangArgs* A) {
+  A->head = nullptr;
+  if (c.algo == 0) return CCLD_OK;
+  if (!c.d_head) return fail(ctx, CCLD_ERR_STATE, "tree communicator without layers (ccld_comm_set_layers)");
+  A->head = c.d_head;
+  return CCLD_OK;
+}
+
 int ccld_locate_hang(ccld_ctx* ctx, uint32_t window_id, uint32_t comm, uint32_t seq, ccld_hang_verdict* out) {
   if (!ctx || !out) return CCLD_ERR_ARG;
   WindowHost* w;
@@ -571,6 +608,7 @@ int ccld_locate_hang(ccld_ctx* ctx, uint32_t window_id, uint32_t comm, uint32_t 
   A.entered = (u8*)(m + L.entered); A.done = (u8*)(m + L.done); A.frame = (u32*)(m + L.frame); A.roots = (u32*)(m + L.roots);
   A.tot = (u64*)(m + L.tot); A.out = (ccld_hang_verdict*)(m + L.hang_out);
   A.roots_cap = n;
+  { int rc = hang_layers(ctx, ctx->comms[ci->second], &A); if (rc != CCLD_OK) return rc; }
   k_hang_locate<<<1, 1024, 0, st>>>(w->d_desc, ctx->reg, A);
   CK(cudaGetLastError());
   ccld_hang_verdict v;
@@ -619,6 +657,7 @@ int ccld_locate_hangs(ccld_ctx* ctx, uint32_t window_id, ccld_hang_alert* alerts
     if (ci == ctx->comm_idx.end()) return fail(ctx, CCLD_ERR_CUDA, "internal: alert names an unknown communicator");
     const u32 nm = (u32)ctx->comms[ci->second].ranks.size();
     members[i] = nm; ha[i].c = ci->second;
+    { int rc = hang_layers(ctx, ctx->comms[ci->second], &ha[i]); if (rc != CCLD_OK) return rc; }
     o_ent[i] = take(nm); o_done[i] = take(nm); o_frame[i] = take(nm * 4ull); o_tot[i] = take(nm * 8ull); o_roots[i] = take(nm * 4ull);
   }
   cudaError_t e;

@@ -1143,6 +1143,7 @@ struct HangArgs {
   u64* tot;                  // [n] scratch
   u32* roots; u32 roots_cap; // device list
   ccld_hang_verdict* out;    // device copy of the struct (pointer fields unused)
+  const u32* head;           // [n] tree communicators: lowest position of each member's layer; null for a ring
 };
 
 __device__ __forceinline__ void hang_locate_cta(const WinDesc& D, const Registry& R, const HangArgs& A) {
@@ -1190,7 +1191,39 @@ __device__ __forceinline__ void hang_locate_cta(const WinDesc& D, const Registry
   __syncthreads();
   const u32 cls = n_ne > 0 ? 1u : (n_ok > 0 ? 2u : 3u);
   u32 n_roots = 0, stuck = 0; u64 min_total = 0;
-  if (cls == 3) {
+  if (cls == 3 && A.head != nullptr) {
+    // tree (Sec. 4.2.1): counters are comparable inside a layer only. The lowest position of a layer walks the layer:
+    // its minimum, the first member that holds it, its maximum. The layer whose minimum is furthest behind its maximum
+    // names the root; equal gaps: the lowest position; no gap anywhere: nobody.
+    u64 lag = 0; u32 cand = NONE;
+    for (u32 p = threadIdx.x; p < n; p += blockDim.x) {
+      if (A.head[p] != p) continue;
+      u64 lmn = A.tot[p], lmx = lmn; u32 at = p;
+      for (u32 x = p + 1; x < n; ++x) {
+        if (A.head[x] != p) continue;
+        const u64 t = A.tot[x];
+        if (t < lmn) { lmn = t; at = x; }
+        lmx = t > lmx ? t : lmx;
+      }
+      const u64 g = lmx - lmn;
+      if (g > lag || (g == lag && g > 0 && at < cand)) { lag = g; cand = at; }
+    }
+    const u64 best = block_reduce(lag, OpMaxU64(), s_red64);
+    if (lag != best || best == 0) cand = NONE;
+    const u32 root = block_reduce(cand, OpMinU32(), s_red32);
+    if (root != NONE) {
+      n_roots = 1; min_total = A.tot[root];
+      if (threadIdx.x == 0) {
+        if (A.roots_cap > 0) A.roots[0] = mem[root];
+        const u32 f = A.frame[root];
+        if (f != NONE && A.n_channels > 0) {
+          u32 s = NONE;
+          for (u32 ch = 0; ch < A.n_channels; ++ch) { const u32 r = A.progress[((u64)f * A.n_channels + ch) * 2 + 1]; s = r < s ? r : s; }
+          stuck = s;
+        }
+      }
+    }
+  } else if (cls == 3) {
     // fewest counters; among equals the most upstream of a run (predecessor ahead), then the lowest position
     u32 up = NONE, any = NONE;
     for (u32 p = threadIdx.x; p < n; p += blockDim.x) {

@@ -497,3 +497,89 @@ def test_randomized_groups_with_random_damage(seed):
         v, _ = compare_window(an, o, w)
         assert v["n_incomplete"] > 0 and v["n_complete"] > 0 and v["n_alerts_total"] > 0
     compare_cumulative(an, o, r0, 1)
+
+
+# ---------------------------------------------------------------- tree communicators (Sec. 4.2.1: same-layer comparison)
+@pytest.mark.gpu
+def test_tree_communicators_compare_progress_within_a_layer():
+    """Hung tree communicators of several sizes, layers as the depth of a binary tree or as random ids, counter totals
+    that differ from layer to layer with random laggards, ties and missing frames: H3 names the same member as the
+    oracle, through ccld_locate_hang and through the sweep; H1 / H2 and the per-op results do not depend on the layers."""
+    rng = np.random.default_rng(77)
+    C_ = 2
+    an, o = ccld.Analyzer(), orc.Oracle()
+    recs, entries, r0 = [], [], 0
+    plan = [(7, "depth", "lag"), (7, "depth", "even"), (40, "rand", "lag"), (130, "depth", "tie"), (1500, "rand", "lag"),
+            (3000, "depth", "lag"), (9, "depth", "h1"), (12, "rand", "h2"), (33, "one", "lag"), (20, "each", "lag")]
+    for cid, (n, lay, kind) in enumerate(plan):
+        ranks = (r0 + rng.permutation(n)).tolist(); r0 += n
+        layers = {"depth": np.floor(np.log2(np.arange(n) + 1)).astype(np.uint32), "rand": rng.integers(0, 5, n).astype(np.uint32) * 1000 + 7,
+                  "one": np.zeros(n, np.uint32), "each": np.arange(n, dtype=np.uint32)[::-1].copy()}[lay]
+        an.comm_register(cid, ranks, 1, 0); assert o.comm_register(cid, ranks, 0) == 0
+        an.comm_set_layers(cid, layers); assert o.comm_set_layers(cid, layers) == 0
+        entered = set(range(n)) - ({1, n - 1} if kind == "h1" else set())
+        done = {2, 3} if kind == "h2" else set()
+        for r in hang_records(n, 1 + cid % 3, entered, done, ranks):
+            r["comm"] = cid
+            recs.append(r)
+        tot = 50 + 10 * (layers % 13).astype(np.int64)                           # every layer has its own level
+        if kind in ("lag", "tie", "h1", "h2"):
+            k = max(1, n // 10)
+            who = rng.choice(n, k, replace=False)
+            tot[who] -= 9 if kind == "tie" else rng.integers(1, 40, k)           # "tie": the same gap in several layers
+        for i in range(n):
+            if n > 100 and i == n // 3: continue                                 # no frame: counts as zero
+            entries.append((ranks[i], cid, 1 + cid % 3, [(int(tot[i]) // 2, int(tot[i]) - int(tot[i]) // 2)] * C_))
+    cols = make_cols(recs)
+    fr = frames_from(entries, C_)
+    an.trace_upload(0, cols, fr, C_); assert o.upload(0, cols, fr, C_) == 0
+    now = 10**9 + 400 * 10**9
+    an.analyze_window(0, 1, now); assert o.analyze(0, 1, now) == 0
+    compare_window(an, o, 0)
+    sweep = an.locate_hangs(0, cap=32, roots_stride=16)
+    assert len(sweep) == len(plan)
+    seen = {}
+    for d in sweep:
+        b = o.locate_hang(0, d["comm"], d["seq"])
+        a = an.locate_hang(0, d["comm"], d["seq"])
+        for v in (d, a):
+            assert v["cls"] == b["cls"] and v["n_roots_total"] == b["n_roots"], (v, b)
+            for k in ("n_not_entered", "n_hung", "n_not_hung", "n_missing_frames", "stuck_step", "n_members", "min_total"):
+                assert v[k] == b[k], (d["comm"], k, v[k], b[k])
+            assert np.array_equal(v["roots"][:16], b["roots"][:16])
+        seen[d["comm"]] = (b["cls"], b["n_roots"])
+    assert seen[1] == (3, 0) and seen[9] == (3, 0)                              # layers that agree / of one member each: nobody
+    assert seen[6][0] == 1 and seen[7][0] == 2 and all(seen[c] == (3, 1) for c in (0, 2, 3, 4, 5, 8))
+
+
+@pytest.mark.gpu
+def test_tree_communicator_call_order_and_errors():
+    an = ccld.Analyzer()
+    an.comm_register(0, [0, 1, 2], 0, 0); an.comm_register(1, [3, 4, 5], 1, 0); an.comm_register(2, [6, 7, 8], 1, 0)
+    with pytest.raises(ccld.CcldError) as e:
+        an.comm_register(3, [9, 10], 2, 0)
+    assert e.value.code == -1
+    with pytest.raises(ccld.CcldError) as e:
+        an.comm_set_layers(0, [0, 1, 1])                                         # a ring has no layers
+    assert e.value.code == -1
+    with pytest.raises(ccld.CcldError) as e:
+        an.comm_set_layers(9, [0])
+    assert e.value.code == -4
+    an.comm_set_layers(1, [0, 1, 1])
+    recs = []
+    for cid, ranks in ((1, [3, 4, 5]), (2, [6, 7, 8])):
+        for r in hang_records(3, 0, {0, 1, 2}, set(), ranks):
+            r["comm"] = cid; recs.append(r)
+    an.trace_upload(0, make_cols(recs), frames_from([(4, 1, 0, [(5, 5)]), (5, 1, 0, [(2, 2)])], 1), 1)
+    an.analyze_window(0, 1, 10**9 + 400 * 10**9)
+    v = an.locate_hang(0, 1, 0)
+    assert v["cls"] == 3 and list(v["roots"]) == [5] and v["min_total"] == 4 and v["stuck_step"] == 2
+    with pytest.raises(ccld.CcldError) as e:
+        an.locate_hang(0, 2, 0)                                                  # a tree whose layers were never set
+    assert e.value.code == -9
+    with pytest.raises(ccld.CcldError) as e:
+        an.locate_hangs(0, cap=8, roots_stride=4)
+    assert e.value.code == -9
+    with pytest.raises(ccld.CcldError) as e:
+        an.comm_set_layers(2, [0, 1, 1])                                         # too late
+    assert e.value.code == -9
