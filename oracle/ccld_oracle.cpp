@@ -17,8 +17,9 @@
 // forms for a counter that advances every tick, to additivity over adjacent ops and to a numpy restatement.
 // orc_opset_check (majority Operation Type Set of an op and the ranks that deviate) is pinned to hand cases and to a
 // collections.Counter restatement.
-// Tree communicators: the same-layer restriction is the paper's (Sec. 4.2.1); which lagging member is named is this
-// repository's rule ("parity unpinned"), pinned to hand cases.
+// Tree communicators: the same-layer restriction is the paper's (Sec. 4.2.1); which member is named - the one lagging its
+// layer's counters in a hang, the one changing more often than its layer in a slowdown - is this repository's rule
+// ("parity unpinned"), pinned to hand cases.
 // "Parity unpinned" against the paper: the bus-bandwidth factor and the median/MAD convention,
 // because the paper defines neither (they are this repository's conventions, pinned only to
 // closed forms and hand values).
@@ -288,6 +289,22 @@ void analyze_one(Oracle& o, Window& w, i64 now) {
         cr.root_comp = sel->rank_tmin;                  // minimal communication time
         if (sel->max_chg > 0) { cr.root_comm = sel->rank_max_chg; cr.rate_source = 0; }  // minimal rate = most changes
         else { cr.root_comm = sel->rank_tmax; cr.rate_source = 1; }
+        if (!c.layer.empty()) {
+          // tree (Sec. 4.2.1): update frequencies are comparable inside a layer only. The member with the most changes
+          // above its layer's fewest; ties: the lowest position; every layer uniform: the rates name nobody.
+          const u32 n = (u32)c.ranks.size();
+          const u32* rec = &w.perm[sel->slot0];
+          std::vector<u32> ch(n, 0);
+          if (!w.send_chg.empty()) for (u32 q = 0; q < n; ++q) ch[q] = std::max(w.send_chg[rec[q]], w.recv_chg[rec[q]]);
+          u32 best = 0; long at = -1;
+          for (u32 q = 0; q < n; ++q) {
+            u32 lmn = ch[q];
+            for (u32 x = 0; x < n; ++x) if (c.layer[x] == c.layer[q]) lmn = std::min(lmn, ch[x]);
+            if (ch[q] - lmn > best) { best = ch[q] - lmn; at = q; }
+          }
+          if (at >= 0) { cr.root_comm = c.ranks[at]; cr.rate_source = 0; }
+          else { cr.root_comm = sel->rank_tmax; cr.rate_source = 1; }
+        }
       }
     }
     cr.slow_count = c.slow_count;

@@ -673,3 +673,36 @@ def test_tree_hang_root_is_compared_with_its_own_layer_only():
     # a member without a frame counts as zero and so lags its layer
     h, ranks = _tree_hang([3, 20, 20, 10, 10, 10, 10], layers, drop_frame=5)
     assert list(h["roots"]) == [ranks[5]] and h["n_missing_frames"] == 1 and h["stuck_step"] == 0
+
+
+def _tree_slow(chg, layers, durs=None, with_rates=True):
+    n = len(chg)
+    ranks = list(range(70, 70 + n))
+    durs = durs or [10 * MS] * n
+    recs = [dict(rank=ranks[i], comm=0, seq=0, t_enter=10**9, t_exit=10**9 + durs[i], send_chg=chg[i], recv_chg=1) for i in range(n)]
+    o = orc.Oracle(dict(tbase_init_ns=2 * MS))
+    assert o.comm_register(0, ranks, 0) == 0
+    if layers is not None:
+        assert o.comm_set_layers(0, layers) == 0
+    assert o.upload(0, make_cols(recs, with_rates)) == 0
+    assert o.analyze(0, 1, 10**12) == 0
+    r = o.comm_rows(0)
+    assert r["slow_detected"][0] == 1
+    return int(r["root_comm"][0]) - 70, int(r["rate_source"][0])
+
+
+def test_tree_slow_root_compares_update_frequencies_within_a_layer():
+    layers = [0, 1, 1, 2, 2, 2, 2]
+    # the tree's root relays everything and changes most often (12): a ring would name it; inside the layers only
+    # position 5 (6 changes against its layer's 3) stands out
+    chg = [12, 6, 6, 3, 3, 6, 3]
+    assert _tree_slow(chg, None) == (0, 0)
+    assert _tree_slow(chg, layers) == (5, 0)
+    # the larger excess wins; equal excesses: the lowest position
+    assert _tree_slow([12, 6, 10, 3, 3, 6, 3], layers) == (2, 0)
+    assert _tree_slow([12, 6, 9, 3, 3, 6, 3], layers) == (2, 0)
+    assert _tree_slow([12, 9, 6, 3, 3, 3, 6], layers) == (1, 0)
+    # every layer uniform: the rates name nobody and the longest duration stands in, as it does without rate columns
+    durs = [10 * MS] * 7; durs[4] = 12 * MS
+    assert _tree_slow([12, 6, 6, 3, 3, 3, 3], layers, durs) == (4, 1)
+    assert _tree_slow(chg, layers, durs, with_rates=False) == (4, 1)
