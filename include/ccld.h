@@ -119,8 +119,13 @@ int ccld_comm_register(ccld_ctx* ctx, uint32_t comm, const uint32_t* ranks, uint
  * answer H3 like this: in every layer take the gap between the largest and the smallest counter
  * total; the root is the member holding the minimum of the layer with the widest gap (equal gaps,
  * or several holders: the lowest position); if no layer disagrees with itself n_roots_total = 0
- * and min_total = 0. H1, H2 and the per-operation statistics (which compare times, not counters)
- * treat a tree communicator like a ring. Errors: CCLD_ERR_STATE after the first analysis,
+ * and min_total = 0. The same restriction holds for the update frequencies: the root_comm of a
+ * slowed tree communicator (ccld_comm_verdict) is the member whose change count in the selected
+ * round - the larger of its two rate columns - lies furthest above the smallest of its layer
+ * (equal excesses: the lowest position); if no layer disagrees with itself, or the window has no
+ * rate columns, the member with the longest duration stands in (rate_source = 1). H1, H2 and the
+ * per-operation statistics (which compare times, not counters) treat a tree communicator like a
+ * ring; so does root_comm while the layers are not set. Errors: CCLD_ERR_STATE after the first analysis,
  * CCLD_ERR_UNKNOWN_COMM, CCLD_ERR_ARG for a ring communicator or a null pointer. Locating a hang
  * on a tree communicator whose layers were never set returns CCLD_ERR_STATE.
  */

@@ -84,6 +84,7 @@ struct ccld_ctx {
   std::vector<CommHost> comms; std::unordered_map<u32, u32> comm_idx;
   bool finalized = false; u32 n_ranks = 0, max_n = 0, max_large_n = 0; u64 sum_n = 0;
   Block reg_blk, misc_blk; Registry reg; size_t stats_off = 0, stats_bytes = 0;
+  const TreeRef* d_trees = nullptr; u32 n_trees = 0;     // tree communicators whose layers are known
   std::map<u32, WindowHost> windows;
   Pool pool; std::string err;
   u64* h_pinned = nullptr; size_t h_pinned_bytes = 0;
@@ -197,7 +198,9 @@ int finalize_registry(ccld_ctx* ctx) {
   const size_t o_hash = take(hsize * sizeof(uint4)), o_rtab = take(rank_tab.size() * 4), o_id = take(nc * 4), o_n = take(nc * 4), o_s0 = take(nc * 4), o_moff = take(nc * 8),
                o_mem = take(sum_n * 4), o_ptr = take((nr + 1) * 4ull), o_ec = take(sum_n * 4), o_ep = take(sum_n * 4);
   std::vector<size_t> o_head(nc, 0);
-  for (u32 i = 0; i < nc; ++i) if (!ctx->comms[i].head.empty()) o_head[i] = take(ctx->comms[i].head.size() * 4);
+  u32 n_trees = 0;
+  for (u32 i = 0; i < nc; ++i) if (!ctx->comms[i].head.empty()) { o_head[i] = take(ctx->comms[i].head.size() * 4); ++n_trees; }
+  const size_t o_trees = take(std::max<u32>(n_trees, 1) * sizeof(TreeRef));
   const size_t o_stats = off;
   const size_t o_state = take(nc * sizeof(CommState)), o_votes = take(nr * 16ull), o_ops = take(nr * 4ull), o_cnt = take(nr * 4ull), o_bw = take(nr * 8ull);
   cudaError_t e;
@@ -221,6 +224,10 @@ int finalize_registry(ccld_ctx* ctx) {
     CK(cudaMemcpyAsync(base + o_head[i], c.head.data(), c.head.size() * 4, cudaMemcpyHostToDevice, st));
     c.d_head = (const u32*)(base + o_head[i]);
   }
+  std::vector<TreeRef> trees;
+  for (u32 i = 0; i < nc; ++i) if (ctx->comms[i].d_head) { TreeRef t; t.c = i; t.pad = 0; t.head = ctx->comms[i].d_head; trees.push_back(t); }
+  if (n_trees) CK(cudaMemcpyAsync(base + o_trees, trees.data(), n_trees * sizeof(TreeRef), cudaMemcpyHostToDevice, st));
+  ctx->d_trees = (const TreeRef*)(base + o_trees); ctx->n_trees = n_trees;
   CK(cudaMemsetAsync(base + o_stats, 0, off - o_stats, st));
   CK(cudaStreamSynchronize(st));              // the host vectors above go out of scope
   Registry& R = ctx->reg;
@@ -514,7 +521,11 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   }
   if (n_list[B_T2]) { TimedLaunch tl(ts, 4, st); k_reduce_mid<<<(u32)n_list[B_T2], MID_THREADS, mid_smem_bytes(2 * WARP_N), st>>>(d_desc, pl.t2, (TileSum*)(rbase + o_s2), ctx->reg, ctx->dp, now_ns); }
   if (n_list[B_T3]) { TimedLaunch tl(ts, 5, st); k_reduce_large<<<(u32)n_list[B_T3], LARGE_THREADS, 16ull * ctx->max_large_n, st>>>(d_desc, pl.t3, (TileSum*)(rbase + o_s3), ctx->reg, ctx->dp, now_ns); }
-  { TimedLaunch tl(ts, 6, st); k_window_decide<<<(nc + 3) / 4, 128, 0, st>>>(d_desc, B, ctx->reg, ctx->dp); }
+  {
+    TimedLaunch tl(ts, 6, st);
+    k_window_decide<<<(nc + 3) / 4, 128, 0, st>>>(d_desc, B, ctx->reg, ctx->dp);
+    if (ctx->n_trees) k_tree_root_comm<<<dim3(ctx->n_trees, B), TREE_THREADS, 0, st>>>(d_desc, ctx->d_trees, ctx->reg);
+  }
   CK(cudaGetLastError());
   for (u32 k = 0; k < B; ++k) {
     WindowHost& w = *ws[k];

@@ -1283,6 +1283,10 @@ __global__ void __launch_bounds__(1024) k_hang_locate_many(const WinDesc* __rest
   hang_locate_cta(wd[0], R, A);
 }
 
+}  // namespace ccld
+#include "ccld_tree.cuh"
+namespace ccld {
+
 // ------------------------------------------------------------------------------------------------
 // suspects and ordered lists
 // ------------------------------------------------------------------------------------------------

@@ -583,3 +583,52 @@ def test_tree_communicator_call_order_and_errors():
     with pytest.raises(ccld.CcldError) as e:
         an.comm_set_layers(2, [0, 1, 1])                                         # too late
     assert e.value.code == -9
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("with_rates", [True, False])
+def test_tree_communicators_slow_root_compares_rates_within_a_layer(with_rates):
+    """Slowed tree communicators of every kernel class over a batch of two windows: the communication root is the member
+    that changes most often above its own layer's fewest changes (or the longest duration when no layer disagrees with
+    itself, or without rate columns), identical to the oracle; a ring in the same batch keeps the ring rule."""
+    rng = np.random.default_rng(5)
+    params = dict(tbase_init_ns=2 * 10**6)
+    an, o = ccld.Analyzer(params), orc.Oracle(params)
+    plan = [(7, "depth", "lag"), (8, "rand", "even"), (40, "rand", "lag"), (130, "depth", "tie"), (1500, "rand", "lag"),
+            (3000, "depth", "lag"), (33, "one", "lag"), (20, "each", "lag"), (16, None, "lag")]
+    regs, r0 = [], 0
+    for cid, (n, lay, kind) in enumerate(plan):
+        ranks = (r0 + rng.permutation(n)).tolist(); r0 += n
+        an.comm_register(cid, ranks, 0 if lay is None else 1, 0); assert o.comm_register(cid, ranks, 0) == 0
+        layers = None
+        if lay is not None:
+            layers = {"depth": np.floor(np.log2(np.arange(n) + 1)).astype(np.uint32), "rand": rng.integers(0, 5, n).astype(np.uint32) * 1000 + 7,
+                      "one": np.zeros(n, np.uint32), "each": np.arange(n, dtype=np.uint32)[::-1].copy()}[lay]
+            an.comm_set_layers(cid, layers); assert o.comm_set_layers(cid, layers) == 0
+        regs.append((ranks, layers, kind))
+    wins = []
+    for w in range(2):
+        recs = []
+        for cid, (ranks, layers, kind) in enumerate(regs):
+            n = len(ranks)
+            lv = (layers % 13).astype(np.int64) if layers is not None else np.zeros(n, np.int64)
+            for s in range(3):
+                chg = 3 + 2 * lv                                                # every layer has its own level
+                if kind in ("lag", "tie"):
+                    who = rng.choice(n, max(1, n // 10), replace=False)
+                    chg = chg.copy(); chg[who] += 4 if kind == "tie" else rng.integers(1, 30, len(who))
+                dur = 10**7 + rng.integers(0, 10**5, n) + (s == 1) * rng.integers(0, 10**6, n)   # op 1 has the widest range
+                t0 = 10**9 * (1 + w) + s * 10**8
+                for i in range(n):
+                    recs.append(dict(rank=ranks[i], comm=cid, seq=3 * w + s, t_enter=t0, t_exit=t0 + int(dur[i]),
+                                     send_chg=int(chg[i]) if i % 2 else 1, recv_chg=1 if i % 2 else int(chg[i])))
+        wins.append(make_cols(recs, with_rates))
+    for w in range(2):
+        an.trace_upload(w, wins[w]); assert o.upload(w, wins[w]) == 0
+    an.analyze_window(0, 2, 10**12); assert o.analyze(0, 2, 10**12) == 0
+    for w in range(2):
+        compare_window(an, o, w)
+        rows = o.comm_rows(w)
+        assert rows["slow_detected"].all() and (rows["sel_seq"] == 3 * w + 1).all()
+        src = rows["rate_source"].tolist()
+        assert src == ([0, 1, 0, 0, 0, 0, 0, 1, 0] if with_rates else [1] * 9)
