@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libccld.so")
 SOURCES = [os.path.join(CSRC, "ccld_host.cu"), os.path.join(CSRC, "ccld_static.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, f) for f in ("ccld_kernels.cuh", "ccld_device.cuh")] + [
+DEPS = SOURCES + [os.path.join(CSRC, f) for f in sorted(os.listdir(CSRC)) if f.endswith(".cuh")] + [
     os.path.join(os.path.dirname(HERE), "include", "ccld.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
