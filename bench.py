@@ -264,7 +264,8 @@ def run_ours(args, rank, world, local_rank):
                 "kernels_ms_per_step": {k: kt[k]["ms"] / args.steps for k in kt},
                 "whole_path": {"algorithmic_bytes_per_step": path_bytes, "achieved": path_gbs, "frac": path_gbs / peak}}
     # every launch of the fused reduce kernel is followed by one of k_reduce_deferred (timed inside the same event pair)
-    launches = sum(x["launches"] for x in kt.values()) + kt["k_reduce_fused"]["launches"]
+    # and every launch of k_window_decide is preceded by one of k_window_rounds
+    launches = sum(x["launches"] for x in kt.values()) + kt["k_reduce_fused"]["launches"] + kt["k_window_decide"]["launches"]
 
     # ---- end to end: host buffers -> upload -> analyse -> verdict ----
     NE = min(args.e2e_windows, NW)

@@ -170,7 +170,8 @@ int ccld_window_release(ccld_ctx* ctx, uint32_t window_id);
  * clock for the hang test. Work is enqueued on the context's stream; the call returns after
  * one short device round trip that sizes the result buffers.
  * A window is refused (CCLD_E_CAPACITY in its verdict, nothing analysed) if the op counters seen
- * in it would need more than 2 * n_rec + (sum of communicator sizes) slots.
+ * in it would need more than 2 * n_rec + (sum of communicator sizes) slots. A batch holds at most
+ * 65,535 windows (CCLD_ERR_CAPACITY beyond).
  */
 int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows, int64_t now_ns);
 

@@ -415,6 +415,7 @@ int ccld_reset(ccld_ctx* ctx) {
 int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows, int64_t now_ns) {
   if (!ctx) return CCLD_ERR_ARG;
   if (n_windows == 0) return fail(ctx, CCLD_ERR_ARG, "n_windows is zero");
+  if (n_windows > 65535) return fail(ctx, CCLD_ERR_CAPACITY, "more than 65,535 windows in one batch");
   CK(cudaSetDevice(ctx->device));
   std::vector<WindowHost*> ws(n_windows);
   for (u32 k = 0; k < n_windows; ++k) {
@@ -523,6 +524,7 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   if (n_list[B_T3]) { TimedLaunch tl(ts, 5, st); k_reduce_large<<<(u32)n_list[B_T3], LARGE_THREADS, 16ull * ctx->max_large_n, st>>>(d_desc, pl.t3, (TileSum*)(rbase + o_s3), ctx->reg, ctx->dp, now_ns); }
   {
     TimedLaunch tl(ts, 6, st);
+    k_window_rounds<<<dim3((nc + 3) / 4, B), 128, 0, st>>>(d_desc, ctx->reg);
     k_window_decide<<<(nc + 3) / 4, 128, 0, st>>>(d_desc, B, ctx->reg, ctx->dp);
     if (ctx->n_trees) k_tree_root_comm<<<dim3(ctx->n_trees, B), TREE_THREADS, 0, st>>>(d_desc, ctx->d_trees, ctx->reg);
   }

@@ -11,7 +11,8 @@
 //   k_reduce_deferred  the groups k_reduce_fused sets aside (incomplete, in flight, 64-bit spreads)
 //   k_reduce_mid    same, 129 <= n <= 1024 (shared-memory bitonic sort, several groups per CTA)
 //   k_reduce_large  same, n > 1024 (one CTA per group, radix select)
-//   k_window_decide Eq. 1-4 per communicator and window, slow location
+//   k_window_rounds Eq. 2 per (communicator, window): round counts, selected round, location candidates
+//   k_window_decide Eq. 1, 3, 4 per communicator, windows in order: baseline state, class, slow location
 //   k_hang_locate   hang decision tree over presence / completion / progress counters
 //   k_suspects, k_rank_sort_*  suspect list and ordered output lists
 #pragma once
@@ -1037,48 +1038,103 @@ __global__ void __launch_bounds__(LARGE_THREADS) k_reduce_large(const WinDesc* _
 // window decision per communicator (Sec. 4.2.1 Eq. 1-3, Sec. 4.2.2 Eq. 4): one warp per
 // communicator walks the windows of the batch in order
 // ------------------------------------------------------------------------------------------------
+// Stage 1, one warp per (communicator, window), all windows at once: everything of the window decision that does not
+// depend on the state carried from window to window - the round and analysed-op counts, the round Eq. 2 selects with its
+// T_max / T_min and the ranks the location step would name - goes into the communicator's verdict row.
+__global__ void __launch_bounds__(128) k_window_rounds(const WinDesc* __restrict__ wd, Registry R) {
+  const u32 c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (c >= R.n_comms) return;
+  const WinDesc& D = wd[blockIdx.y];
+  const RangeRow row = D.ranges[c];
+  if (row.n_seq == 0) return;
+  const u32 n = R.comm_n[c], cls = comm_class(n);
+  const u32* mem = R.members + R.comm_moff[c];
+  const u64 G = D.n_groups;
+  const i64* t_max = D.gi64 + (u64)GI_T_MAX * G + row.group0;
+  const i64* t_min = D.gi64 + (u64)GI_T_MIN * G + row.group0;
+  // round counts and the Eq. 2 candidate come from the tile summaries the reduce kernels left behind
+  const TileSum* ts = D.tsum[cls <= 1 ? 0 : cls - 1] + row.tile0;
+  const u32 nt = row.n_units;
+  u32 n_rounds = 0, n_an = 0;
+  u64 best_rng = 0; u32 best_k = NONE;
+  bool redo = false;                                     // a unit left groups to the deferred kernel: its summary is partial
+  for (u32 q = lane; q < nt; q += 32) {
+    const TileSum x = ts[q];
+    n_rounds += x.n_rounds; n_an += x.n_an;
+    best_merge(best_rng, best_k, x.best_rng, x.best_k);
+    redo = redo || x.pad != 0;
+  }
+  if (__any_sync(0xFFFFFFFFu, redo)) {
+    // recount the communicator's window from the per-op rows
+    const u32* gfl = D.gu32 + (u64)GU_GFLAGS * G + row.group0;
+    n_rounds = 0; n_an = 0; best_rng = 0; best_k = NONE;
+    for (u32 k = lane; k < row.n_seq; k += 32) {
+      const u32 f = gfl[k];
+      if ((f & CCLD_G_COMPLETE) && !(f & CCLD_G_BARRIER)) { ++n_rounds; best_merge(best_rng, best_k, (u64)(t_max[k] - t_min[k]), k); }
+      if (f & CCLD_G_ANALYSED) ++n_an;
+    }
+  }
+  n_rounds = __reduce_add_sync(0xFFFFFFFFu, n_rounds); n_an = __reduce_add_sync(0xFFFFFFFFu, n_an);
+  best_warp_reduce(best_rng, best_k);
+  // analysed ops of this window count towards every member's denominator
+  if (n_an) for (u32 p = lane; p < n; p += 32) atomicAdd(&R.ops[mem[p]], n_an);
+  if (lane == 0) {
+    ccld_comm_verdict v;
+    v.comm = R.comm_id[c]; v.n_rounds = n_rounds; v.sel_seq = NONE; v.cls = 0; v.slow_detected = 0; v.located = 0;
+    v.baseline_static = 0; v.rate_source = 0; v.root_comp = NONE; v.root_comm = NONE;
+    v.t_max = 0; v.t_min = 0; v.R = 0.0; v.P = 0.0; v.t_base = 0; v.rounds_total = 0; v.m = 0; v.slow_count = 0;
+    if (best_k != NONE) {
+      v.sel_seq = row.seq_lo + best_k; v.t_max = t_max[best_k]; v.t_min = t_min[best_k];
+      const u64 gq = row.group0 + best_k;
+      v.root_comp = D.gu32[(u64)GU_RANK_TMIN * G + gq];
+      const u32 mc = D.gu32[(u64)GU_MAX_CHG * G + gq];
+      if (mc > 0) { v.root_comm = D.gu32[(u64)GU_RANK_MAX_CHG * G + gq]; v.rate_source = 0; }
+      else { v.root_comm = D.gu32[(u64)GU_RANK_TMAX * G + gq]; v.rate_source = 1; }
+    }
+    D.comm_rows[row.row_idx] = v;
+  }
+}
+
+// Stage 2, one warp per communicator, windows in order: the recurrences - Eq. 1's baseline, which reads the per-op rows
+// until m is fixed, and the repetition counter - and with them Eq. 3, Eq. 4 and the location rule, which complete the
+// row stage 1 wrote. What a window needs is fetched ahead (range rows two windows, the stage-1 row and the result
+// pointers one window), so the walk waits for arithmetic only.
 __global__ void __launch_bounds__(128) k_window_decide(const WinDesc* __restrict__ wd, u32 nw, Registry R, Params P) {
   const u32 c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (c >= R.n_comms) return;
-  const u32 n = R.comm_n[c], cls = comm_class(n);
-  const u32* mem = R.members + R.comm_moff[c];
   CommState st = R.state[c];
+  struct Res { u64 n_groups; const i64* gi64; const u32* gu32; ccld_comm_verdict* comm_rows; };   // result pointers of a window
+  struct Part { u32 n_rounds, sel_seq, root_comp, root_comm, rate_source; i64 t_max, t_min; };    // what stage 1 left in the row
+  auto load_row = [&](u32 w) { RangeRow r = {0, 0, 0, 0, 0, 0, 0, 0}; if (w < nw) r = wd[w].ranges[c]; return r; };
+  auto load_res = [&](u32 w) {
+    Res r = {0, nullptr, nullptr, nullptr};
+    if (w < nw) { r.n_groups = wd[w].n_groups; r.gi64 = wd[w].gi64; r.gu32 = wd[w].gu32; r.comm_rows = wd[w].comm_rows; }
+    return r;
+  };
+  auto load_part = [&](const Res& r, const RangeRow& row) {
+    Part x = {0, NONE, NONE, NONE, 0, 0, 0};
+    if (r.comm_rows != nullptr && row.n_seq != 0) {
+      const ccld_comm_verdict* v = r.comm_rows + row.row_idx;
+      x.n_rounds = v->n_rounds; x.sel_seq = v->sel_seq; x.root_comp = v->root_comp; x.root_comm = v->root_comm;
+      x.rate_source = v->rate_source; x.t_max = v->t_max; x.t_min = v->t_min;
+    }
+    return x;
+  };
+  RangeRow row_a = load_row(0), row_b = load_row(1);
+  Res res_a = load_res(0), res_b = load_res(1);
+  Part part_a = load_part(res_a, row_a);
   for (u32 w = 0; w < nw; ++w) {
-    const WinDesc& D = wd[w];
-    const RangeRow row = D.ranges[c];
+    const RangeRow row = row_a; const Res D = res_a; const Part pt = part_a;
+    row_a = row_b; res_a = res_b; row_b = load_row(w + 2); res_b = load_res(w + 2); part_a = load_part(res_a, row_a);
     if (row.n_seq == 0) continue;
     const u64 G = D.n_groups;
-    const i64* t_max = D.gi64 + (u64)GI_T_MAX * G + row.group0;
-    const i64* t_min = D.gi64 + (u64)GI_T_MIN * G + row.group0;
-    // round counts and the Eq. 2 candidate come from the tile summaries the reduce kernels left behind
-    const TileSum* ts = D.tsum[cls <= 1 ? 0 : cls - 1] + row.tile0;
-    const u32 nt = row.n_units;
-    u32 n_rounds = 0, n_an = 0;
-    u64 best_rng = 0; u32 best_k = NONE;
-    bool redo = false;                                     // a unit left groups to the deferred kernel: its summary is partial
-    for (u32 q = lane; q < nt; q += 32) {
-      const TileSum x = ts[q];
-      n_rounds += x.n_rounds; n_an += x.n_an;
-      best_merge(best_rng, best_k, x.best_rng, x.best_k);
-      redo = redo || x.pad != 0;
-    }
-    if (__any_sync(0xFFFFFFFFu, redo)) {
-      // recount the communicator's window from the per-op rows
-      const u32* gfl = D.gu32 + (u64)GU_GFLAGS * G + row.group0;
-      n_rounds = 0; n_an = 0; best_rng = 0; best_k = NONE;
-      for (u32 k = lane; k < row.n_seq; k += 32) {
-        const u32 f = gfl[k];
-        if ((f & CCLD_G_COMPLETE) && !(f & CCLD_G_BARRIER)) { ++n_rounds; best_merge(best_rng, best_k, (u64)(t_max[k] - t_min[k]), k); }
-        if (f & CCLD_G_ANALYSED) ++n_an;
-      }
-    }
-    n_rounds = __reduce_add_sync(0xFFFFFFFFu, n_rounds); n_an = __reduce_add_sync(0xFFFFFFFFu, n_an);
-    best_warp_reduce(best_rng, best_k);
+    const u32 n_rounds = pt.n_rounds;
     // Eq. 1: rounds feed the baseline, in op-counter order, until m is fixed
     u32 walked = 0;
     if (st.m == 0 && n_rounds > 0) {
       const u32* gfl = D.gu32 + (u64)GU_GFLAGS * G + row.group0;
       const i64* e_min = D.gi64 + (u64)GI_E_MIN * G + row.group0;
+      const i64* t_max = D.gi64 + (u64)GI_T_MAX * G + row.group0;
       for (u32 k0 = 0; k0 < row.n_seq && st.m == 0; k0 += 32) {
         const u32 k = k0 + lane;
         const u32 f = k < row.n_seq ? gfl[k] : 0;
@@ -1097,17 +1153,14 @@ __global__ void __launch_bounds__(128) k_window_decide(const WinDesc* __restrict
       }
     }
     st.rounds += n_rounds - walked;
-    // analysed ops of this window count towards every member's denominator
-    if (n_an) for (u32 p = lane; p < n; p += 32) atomicAdd(&R.ops[mem[p]], n_an);
     if (lane == 0) {
       ccld_comm_verdict v;
-      v.comm = R.comm_id[c]; v.n_rounds = n_rounds; v.sel_seq = NONE; v.cls = 0; v.slow_detected = 0; v.located = 0;
+      v.comm = R.comm_id[c]; v.n_rounds = n_rounds; v.sel_seq = pt.sel_seq; v.cls = 0; v.slow_detected = 0; v.located = 0;
       v.baseline_static = st.m == 0; v.rate_source = 0; v.root_comp = NONE; v.root_comm = NONE;
-      v.t_max = 0; v.t_min = 0; v.R = 0.0; v.P = 0.0;
+      v.t_max = pt.t_max; v.t_min = pt.t_min; v.R = 0.0; v.P = 0.0;
       v.t_base = st.m > 0 ? st.sum_m / (i64)st.m : P.tbase_init_ns;
       v.rounds_total = st.rounds; v.m = st.m;
-      if (best_k != NONE) {
-        v.sel_seq = row.seq_lo + best_k; v.t_max = t_max[best_k]; v.t_min = t_min[best_k];
+      if (pt.sel_seq != NONE) {
         v.R = (double)(v.t_max - v.t_base) / (double)v.t_base;                                     // Eq. 3
         const bool slow = v.t_max > v.t_base && mul_gt((u64)(v.t_max - v.t_base), 1000u, (u64)v.t_base, P.theta_slow_milli);
         v.slow_detected = slow;
@@ -1117,11 +1170,7 @@ __global__ void __launch_bounds__(128) k_window_decide(const WinDesc* __restrict
           const u64 num = (u64)(v.t_max - v.t_min), den = (u64)(v.t_max - v.t_base);
           v.P = (double)num / (double)den;                                                         // Eq. 4
           v.cls = mul_gt(num, 1000u, den, P.beta_milli) ? 1u : (mul_lt(num, 1000u, den, P.alpha_milli) ? 2u : 3u);
-          const u64 gq = row.group0 + best_k;
-          v.root_comp = D.gu32[(u64)GU_RANK_TMIN * G + gq];
-          const u32 mc = D.gu32[(u64)GU_MAX_CHG * G + gq];
-          if (mc > 0) { v.root_comm = D.gu32[(u64)GU_RANK_MAX_CHG * G + gq]; v.rate_source = 0; }
-          else { v.root_comm = D.gu32[(u64)GU_RANK_TMAX * G + gq]; v.rate_source = 1; }
+          v.root_comp = pt.root_comp; v.root_comm = pt.root_comm; v.rate_source = pt.rate_source;
         }
       }
       v.slow_count = st.slow_count;
