@@ -1103,14 +1103,15 @@ __global__ void __launch_bounds__(128) k_window_decide(const WinDesc* __restrict
   const u32 c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
   if (c >= R.n_comms) return;
   CommState st = R.state[c];
-  struct Res { u64 n_groups; const i64* gi64; const u32* gu32; ccld_comm_verdict* comm_rows; };   // result pointers of a window
+  struct Res { const RangeRow* ranges; u64 n_groups; const i64* gi64; const u32* gu32; ccld_comm_verdict* comm_rows; };   // pointers of a window
   struct Part { u32 n_rounds, sel_seq, root_comp, root_comm, rate_source; i64 t_max, t_min; };    // what stage 1 left in the row
-  auto load_row = [&](u32 w) { RangeRow r = {0, 0, 0, 0, 0, 0, 0, 0}; if (w < nw) r = wd[w].ranges[c]; return r; };
+  // three steps, each on values fetched during an earlier window: descriptor -> range row -> stage-1 row
   auto load_res = [&](u32 w) {
-    Res r = {0, nullptr, nullptr, nullptr};
-    if (w < nw) { r.n_groups = wd[w].n_groups; r.gi64 = wd[w].gi64; r.gu32 = wd[w].gu32; r.comm_rows = wd[w].comm_rows; }
+    Res r = {nullptr, 0, nullptr, nullptr, nullptr};
+    if (w < nw) { r.ranges = wd[w].ranges; r.n_groups = wd[w].n_groups; r.gi64 = wd[w].gi64; r.gu32 = wd[w].gu32; r.comm_rows = wd[w].comm_rows; }
     return r;
   };
+  auto load_row = [&](const Res& r) { RangeRow x = {0, 0, 0, 0, 0, 0, 0, 0}; if (r.ranges != nullptr) x = r.ranges[c]; return x; };
   auto load_part = [&](const Res& r, const RangeRow& row) {
     Part x = {0, NONE, NONE, NONE, 0, 0, 0};
     if (r.comm_rows != nullptr && row.n_seq != 0) {
@@ -1120,12 +1121,14 @@ __global__ void __launch_bounds__(128) k_window_decide(const WinDesc* __restrict
     }
     return x;
   };
-  RangeRow row_a = load_row(0), row_b = load_row(1);
-  Res res_a = load_res(0), res_b = load_res(1);
+  Res res_a = load_res(0), res_b = load_res(1), res_c = load_res(2);
+  RangeRow row_a = load_row(res_a), row_b = load_row(res_b);
   Part part_a = load_part(res_a, row_a);
   for (u32 w = 0; w < nw; ++w) {
     const RangeRow row = row_a; const Res D = res_a; const Part pt = part_a;
-    row_a = row_b; res_a = res_b; row_b = load_row(w + 2); res_b = load_res(w + 2); part_a = load_part(res_a, row_a);
+    part_a = load_part(res_b, row_b);                    // window w + 1
+    row_a = row_b; row_b = load_row(res_c);              // window w + 2
+    res_a = res_b; res_b = res_c; res_c = load_res(w + 3);
     if (row.n_seq == 0) continue;
     const u64 G = D.n_groups;
     const u32 n_rounds = pt.n_rounds;
