@@ -76,3 +76,52 @@ def test_paper_example_and_pipeline_input():
     an.analyze_window(0, 1, win.now_ns); o.analyze(0, 1, win.now_ns)
     t, g = an.get_optable(0), o.groups(0)
     assert np.array_equal(t["max_chg"], g["max_chg"]) and np.array_equal(t["rank_max_chg"], g["rank_max_chg"])
+
+
+def _series(rng, n_ranks, n_ticks, period_ms=1):
+    off = np.arange(n_ranks + 1) * n_ticks
+    tn = np.concatenate([np.arange(n_ticks) * period_ms * MS + rng.integers(0, MS) for _ in range(n_ranks)])
+    sc = np.concatenate([np.cumsum(rng.integers(0, 2, n_ticks)) for _ in range(n_ranks)])
+    rc = np.concatenate([np.cumsum(rng.integers(0, 3, n_ticks) // 2) for _ in range(n_ranks)])
+    return off, tn, sc, rc
+
+
+def test_ops_of_29_to_36_ticks_at_every_place_in_the_table():
+    """Ops that span 29 to 36 ticks (around a warp's width), from before a rank's first tick, after it, in the middle of
+    its ticks, up to its last tick and in flight with as many ticks left, each ending on a tick and between two."""
+    rng = np.random.default_rng(3)
+    off, tn, sc, rc = _series(rng, 3, 200)
+    rank, te, tx = [], [], []
+    for r in range(3):
+        t = tn[off[r]:off[r + 1]]
+        for span in range(29, 37):
+            for first in (0, 1, 57, 200 - span):                    # from before the first tick, after it, mid-table, to the last tick
+                a = t[first] - 1 if first else t[0] - 5
+                rank.append(r); te.append(a); tx.append(t[first + span - 1])           # `span` ticks in (a, b]
+                rank.append(r); te.append(a); tx.append(t[first + span - 1] + MS // 2)
+            rank.append(r); te.append(t[200 - span] - 1); tx.append(-1)                 # in flight, `span` ticks left
+    _check(ccld.Analyzer(), np.array(rank), np.array(te), np.array(tx), off, tn, sc, rc)
+
+
+def test_a_few_long_ops_among_short_ones():
+    """Thousands of ops of a few ticks and ten that span hundreds to thousands of ticks (two of them in flight)."""
+    rng = np.random.default_rng(4)
+    off, tn, sc, rc = _series(rng, 4, 20_000)
+    n = 3000
+    rank = rng.integers(0, 4, n); te = rng.integers(0, 19_900 * MS, n); tx = te + rng.integers(0, 6 * MS, n)
+    long_ = rng.choice(n, 10, replace=False)
+    tx[long_] = te[long_] + rng.integers(100 * MS, 9_000 * MS, 10)
+    tx[long_[:2]] = -1
+    es, _ = _check(ccld.Analyzer(), rank, te, tx, off, tn, sc, rc)
+    assert es[long_].min() > 20 and np.median(es) <= 4
+
+
+def test_every_op_spans_hundreds_of_ticks():
+    """Every op spans 200 to 300 of its rank's 400 ticks, a tenth of them in flight."""
+    rng = np.random.default_rng(5)
+    off, tn, sc, rc = _series(rng, 50, 400)
+    n = 3000
+    rank = rng.integers(0, 50, n); te = rng.integers(-10 * MS, 150 * MS, n); tx = te + rng.integers(200 * MS, 300 * MS, n)
+    tx[rng.random(n) < 0.1] = -1
+    es, _ = _check(ccld.Analyzer(), rank, te, tx, off, tn, sc, rc)
+    assert np.median(es) > 50
