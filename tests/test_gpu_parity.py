@@ -286,6 +286,9 @@ def test_empty_window_capacity_and_call_order():
     with pytest.raises(ccld.CcldError) as e:
         an.get_verdict(7)
     assert e.value.code == -7
+    with pytest.raises(ccld.CcldError) as e:
+        an.analyze_window(0, 65536, 10**12)                  # more windows than one batch takes
+    assert e.value.code == -8
     # op counters 0 and 4,000,000,000 in one window: the slot space would be absurd, the window is refused
     far = group_trace([[5, 6, 7, 8]]) + group_trace([[5, 6, 7, 8]], seq0=4_000_000_000)
     an.trace_upload(2, make_cols(far))
