@@ -880,16 +880,16 @@ int ccld_derive_rates(ccld_ctx* ctx, uint64_t n_rec, const uint32_t* rank, const
   const u64 n_tiles = (n_ticks + RT_TILE - 1) / RT_TILE;
   size_t off = 0;
   auto take = [&](size_t b) { size_t o = off; off = align_up(off + b); return o; };
-  const size_t o_pre = take((n_ticks + 1) * 8), o_sum = take((n_tiles + 1) * 8);
+  const size_t o_blk = take(((n_ticks + 31) / 32 + 1) * sizeof(TickBlock)), o_sum = take((n_tiles + 1) * 8);
   cudaError_t e;
   Block blk = ctx->pool.get(off, &e);
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "scratch allocation failed");
   TickArgs A; A.n_ticks = n_ticks; A.n_ranks = n_ranks; A.tick_off = tick_off; A.tick_ns = tick_ns; A.send = send_count; A.recv = recv_count;
-  A.prefix = (u64*)((char*)blk.p + o_pre); A.tile_sum = (u64*)((char*)blk.p + o_sum);
+  A.blk = (TickBlock*)((char*)blk.p + o_blk); A.tile_sum = (u64*)((char*)blk.p + o_sum);
   if (n_tiles) {
-    k_tick_sums<<<(u32)n_tiles, RT_THREADS, 0, st>>>(A);
+    k_tick_blocks<<<(u32)n_tiles, RT_THREADS, 0, st>>>(A);
     k_tile_scan<<<1, RT_THREADS, 0, st>>>(A.tile_sum, n_tiles);
-    k_tick_prefix<<<(u32)n_tiles, RT_THREADS, 0, st>>>(A);
+    k_block_prefix<<<(u32)n_tiles, RB_PER_TILE, 0, st>>>(A);
   }
   k_record_rates<<<(u32)((n_rec + RT_THREADS - 1) / RT_THREADS), RT_THREADS, 0, st>>>(A, n_rec, rank, t_enter_ns, t_exit_ns, send_chg, recv_chg);
   const cudaError_t le = cudaGetLastError();

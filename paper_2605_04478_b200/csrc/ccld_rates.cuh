@@ -1,13 +1,16 @@
 // Counter changes per op from raw probe samples (Sec. 4.1.2: SendRate / RecvRate are reciprocals of the number of
 // changes of SendCount / RecvCount seen by a probe that samples at a fixed period; Sec. 5.2 step 2 does this on the
-// host's diagnostic thread). For sm_100a, streaming and HBM-bound:
+// host's diagnostic thread). For sm_100a, streaming and HBM-bound. The prefix of the change indicators is kept per
+// block of 32 ticks - the count before the block plus one bit per tick - so the counters are read once and what is
+// written is half a byte per tick:
 //
-//   k_tick_sums     per tile of ticks: how many ticks changed SendCount / RecvCount against the previous tick of the
-//                   same rank (a rank's first tick never counts)
+//   k_tick_blocks   per block of 32 ticks: which ticks changed SendCount / RecvCount against the previous tick of the
+//                   same rank (a rank's first tick never counts), as two 32-bit masks with their bit counts; per tile
+//                   of 64 blocks the sum of the counts
 //   k_tile_scan     exclusive prefix over the tile sums (one CTA)
-//   k_tick_prefix   inclusive prefix of the change indicators per tick: low word send, high word recv
+//   k_block_prefix  exclusive prefix of the counts inside each tile plus the tile's offset
 //   k_record_rates  per record: two searches in its rank's tick times (the first starts from an even-spacing guess,
-//                   the second from the first), then a difference of prefixes
+//                   the second from the first), then a difference of prefixes, each a block entry and a bit count
 //
 // No kernel waits on another CTA: the prefix is three plain launches.
 #pragma once
@@ -16,14 +19,20 @@
 namespace ccld {
 
 constexpr int RT_THREADS = 256;
-constexpr int RT_PER = 8;                          // consecutive ticks per thread
-constexpr int RT_TILE = RT_THREADS * RT_PER;
+constexpr int RT_PER = 8;                          // tile sums per thread and round in k_tile_scan
+constexpr int RT_TILE = RT_THREADS * RT_PER;       // ticks per CTA of k_tick_blocks: 8 warps x RB_PER_WARP blocks x 32
+constexpr int RB_PER_WARP = 8;
+constexpr int RB_PER_TILE = RT_TILE / 32;          // 64 blocks
+
+// x: changes before the block (send in the low word, recv in the high word; while k_tick_blocks runs: inside the block);
+// y: change bits of the block's ticks (send low, recv high)
+typedef ulonglong2 TickBlock;
 
 struct TickArgs {
   u64 n_ticks; u32 n_ranks;
   const u64* tick_off;                             // [n_ranks + 1]
   const i64* tick_ns; const u32 *send, *recv;      // [n_ticks], a rank's ticks contiguous and in time order
-  u64* prefix;                                     // [n_ticks]
+  TickBlock* blk;                                  // [ceil(n_ticks / 32)]
   u64* tile_sum;                                   // [tiles]
 };
 
@@ -32,47 +41,6 @@ __device__ __forceinline__ u32 tick_owner(const u64* __restrict__ off, u32 n_ran
   u32 lo = 0, hi = n_ranks - 1;
   while (lo < hi) { const u32 mid = (lo + hi + 1) >> 1; if (off[mid] <= i) lo = mid; else hi = mid - 1; }
   return lo;
-}
-
-// Change indicators of the thread's RT_PER consecutive ticks, packed (send | recv << 32); returns their sum.
-__device__ __forceinline__ u64 tick_indicators(const TickArgs& A, u64 i0, u64 (&ind)[RT_PER]) {
-  u64 sum = 0;
-#pragma unroll
-  for (int k = 0; k < RT_PER; ++k) ind[k] = 0;
-  if (i0 >= A.n_ticks) return 0;
-  u32 s[RT_PER], r[RT_PER];
-  const bool full = i0 + RT_PER <= A.n_ticks;
-  if (full && ((reinterpret_cast<uintptr_t>(A.send + i0) | reinterpret_cast<uintptr_t>(A.recv + i0)) & 15) == 0) {
-#pragma unroll
-    for (int q = 0; q < RT_PER / 4; ++q) {
-      const uint4 a = __ldg(reinterpret_cast<const uint4*>(A.send + i0) + q), b = __ldg(reinterpret_cast<const uint4*>(A.recv + i0) + q);
-      s[4 * q] = a.x; s[4 * q + 1] = a.y; s[4 * q + 2] = a.z; s[4 * q + 3] = a.w;
-      r[4 * q] = b.x; r[4 * q + 1] = b.y; r[4 * q + 2] = b.z; r[4 * q + 3] = b.w;
-    }
-  } else {
-#pragma unroll
-    for (int k = 0; k < RT_PER; ++k) { const bool in = i0 + k < A.n_ticks; s[k] = in ? __ldg(A.send + i0 + k) : 0u; r[k] = in ? __ldg(A.recv + i0 + k) : 0u; }
-  }
-  u32 ps = i0 ? __ldg(A.send + i0 - 1) : 0u, pr = i0 ? __ldg(A.recv + i0 - 1) : 0u;
-  // where the current rank's ticks end, and whether tick i0 opens a rank
-  u32 rk = tick_owner(A.tick_off, A.n_ranks, i0);
-  u64 seg_end = A.tick_off[rk + 1];
-  bool first = A.tick_off[rk] == i0;
-#pragma unroll
-  for (int k = 0; k < RT_PER; ++k) {
-    const u64 i = i0 + k;
-    if (i < A.n_ticks) {
-      if (i == seg_end) {                          // the next rank that has ticks starts here
-        first = true;
-        for (u32 step = 0; step <= A.n_ranks && A.tick_off[rk + 1] <= i; ++step) ++rk;
-        seg_end = A.tick_off[rk + 1];
-      }
-      if (!first) ind[k] = (u64)(s[k] != ps ? 1u : 0u) | ((u64)(r[k] != pr ? 1u : 0u) << 32);
-      first = false; ps = s[k]; pr = r[k];
-      sum += ind[k];
-    }
-  }
-  return sum;
 }
 
 // exclusive prefix of v over the CTA (all threads call); *total = the CTA's sum
@@ -95,13 +63,49 @@ __device__ __forceinline__ u64 cta_exclusive_scan(u64 v, u64* total, u64* s_warp
   return r;
 }
 
-__global__ void __launch_bounds__(RT_THREADS) k_tick_sums(TickArgs A) {
-  __shared__ u64 s_warp[RT_THREADS / 32 + 1];
-  u64 ind[RT_PER];
-  const u64 v = tick_indicators(A, (u64)blockIdx.x * RT_TILE + (u64)threadIdx.x * RT_PER, ind);
-  u64 total;
-  cta_exclusive_scan(v, &total, s_warp);
-  if (threadIdx.x == 0) A.tile_sum[blockIdx.x] = total;
+// One warp per RB_PER_WARP consecutive blocks, one lane per tick: the predecessor's counters come from the lane below
+// (from the previous block's last lane, or from memory, for lane 0). Where the ranks' segments start is found once per
+// warp by a search in the offset table and then followed from block to block.
+__global__ void __launch_bounds__(RT_THREADS) k_tick_blocks(TickArgs A) {
+  __shared__ u64 s_cnt[RT_THREADS / 32];
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const u64 t0 = (u64)blockIdx.x * RT_TILE + (u64)wid * (RB_PER_WARP * 32);
+  u64 wsum = 0;
+  if (t0 < A.n_ticks) {
+    u32 rk = tick_owner(A.tick_off, A.n_ranks, t0);             // a rank that has ticks: t0 < n_ticks
+    u64 seg_start = A.tick_off[rk], seg_end = A.tick_off[rk + 1];
+    u32 carry_s = t0 ? __ldg(A.send + t0 - 1) : 0u, carry_r = t0 ? __ldg(A.recv + t0 - 1) : 0u;
+#pragma unroll 2
+    for (int q = 0; q < RB_PER_WARP; ++q) {
+      const u64 bstart = t0 + (u64)q * 32;
+      if (bstart >= A.n_ticks) break;                           // the same in every lane
+      const u64 bend = bstart + 32 < A.n_ticks ? bstart + 32 : A.n_ticks;
+      const u64 i = bstart + lane;
+      const bool in = i < A.n_ticks;
+      const u32 sv = in ? __ldg(A.send + i) : 0u, rv = in ? __ldg(A.recv + i) : 0u;
+      u32 ps = __shfl_up_sync(0xFFFFFFFFu, sv, 1), pr = __shfl_up_sync(0xFFFFFFFFu, rv, 1);
+      if (lane == 0) { ps = carry_s; pr = carry_r; }
+      carry_s = __shfl_sync(0xFFFFFFFFu, sv, 31); carry_r = __shfl_sync(0xFFFFFFFFu, rv, 31);
+      // first ticks of ranks inside [bstart, bend): the current segment's, if it starts here, and those of the segments
+      // that start before the block ends (a rank without ticks has an empty segment and no first tick)
+      bool first = seg_start >= bstart && i == seg_start;
+      for (u32 step = 0; step <= A.n_ranks && seg_end < bend; ++step) {
+        ++rk; seg_start = seg_end; seg_end = A.tick_off[rk + 1];
+        if (seg_end > seg_start) first = first || i == seg_start;
+      }
+      const u32 ms = __ballot_sync(0xFFFFFFFFu, in && !first && sv != ps), mr = __ballot_sync(0xFFFFFFFFu, in && !first && rv != pr);
+      const u64 cnt = (u64)__popc(ms) | ((u64)__popc(mr) << 32);
+      if (lane == 0) A.blk[bstart >> 5] = make_ulonglong2(cnt, (u64)ms | ((u64)mr << 32));
+      wsum += cnt;
+    }
+  }
+  if (lane == 0) s_cnt[wid] = wsum;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    u64 t = 0;
+    for (int q = 0; q < RT_THREADS / 32; ++q) t += s_cnt[q];
+    A.tile_sum[blockIdx.x] = t;
+  }
 }
 
 __global__ void __launch_bounds__(RT_THREADS) k_tile_scan(u64* __restrict__ tile_sum, u64 n_tiles) {
@@ -120,23 +124,27 @@ __global__ void __launch_bounds__(RT_THREADS) k_tile_scan(u64* __restrict__ tile
   }
 }
 
-__global__ void __launch_bounds__(RT_THREADS) k_tick_prefix(TickArgs A) {
-  __shared__ u64 s_warp[RT_THREADS / 32 + 1];
-  u64 ind[RT_PER];
-  const u64 i0 = (u64)blockIdx.x * RT_TILE + (u64)threadIdx.x * RT_PER;
-  const u64 v = tick_indicators(A, i0, ind);
-  u64 total;
-  u64 run = A.tile_sum[blockIdx.x] + cta_exclusive_scan(v, &total, s_warp);
+// 64 threads: the counts of a tile's blocks become the changes before each block
+__global__ void __launch_bounds__(RB_PER_TILE) k_block_prefix(TickArgs A) {
+  __shared__ u64 s_half;
+  const u64 n_blocks = (A.n_ticks + 31) >> 5;
+  const u64 b = (u64)blockIdx.x * RB_PER_TILE + threadIdx.x;
+  const u32 lane = threadIdx.x & 31;
+  const u64 v = b < n_blocks ? A.blk[b].x : 0;
+  u64 inc = v;
 #pragma unroll
-  for (int k = 0; k < RT_PER; ++k) { run += ind[k]; ind[k] = run; }
-  if (i0 + RT_PER <= A.n_ticks) {
-    ulonglong2* dst = reinterpret_cast<ulonglong2*>(A.prefix + i0);          // i0 is a multiple of 8: 64-byte aligned
-#pragma unroll
-    for (int q = 0; q < RT_PER / 2; ++q) dst[q] = make_ulonglong2(ind[2 * q], ind[2 * q + 1]);
-  } else {
-#pragma unroll
-    for (int k = 0; k < RT_PER; ++k) if (i0 + k < A.n_ticks) A.prefix[i0 + k] = ind[k];
-  }
+  for (int d = 1; d < 32; d <<= 1) { const u64 o = __shfl_up_sync(0xFFFFFFFFu, inc, d); if (lane >= (u32)d) inc += o; }
+  if (threadIdx.x == 31) s_half = inc;
+  __syncthreads();
+  const u64 ex = A.tile_sum[blockIdx.x] + (threadIdx.x >= 32 ? s_half : 0) + inc - v;
+  if (b < n_blocks) A.blk[b].x = ex;
+}
+
+// changes up to and including tick i (send in the low word, recv in the high word)
+__device__ __forceinline__ u64 changes_upto(const TickBlock* __restrict__ blk, u64 i) {
+  const TickBlock e = blk[i >> 5];
+  const u32 keep = 0xFFFFFFFFu >> (31 - (u32)(i & 31));
+  return e.x + (u64)__popc((u32)e.y & keep) + ((u64)__popc((u32)(e.y >> 32) & keep) << 32);
 }
 
 // ticks of [lo, hi) at or before t
@@ -196,7 +204,7 @@ __global__ void __launch_bounds__(RT_THREADS) k_record_rates(TickArgs A, u64 n_r
       // a rank's first tick has no indicator, so the prefix "before the first tick" equals the prefix at it
       const u64 ia = lo + (ca ? ca - 1 : 0), ib = lo + (cb ? cb - 1 : 0);
       if (ib > ia) {
-        const u64 pa = A.prefix[ia], pb = A.prefix[ib];
+        const u64 pa = changes_upto(A.blk, ia), pb = changes_upto(A.blk, ib);
         s = (u32)pb - (u32)pa; q = (u32)(pb >> 32) - (u32)(pa >> 32);
       }
     }
