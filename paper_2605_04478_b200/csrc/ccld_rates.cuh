@@ -75,14 +75,21 @@ __global__ void __launch_bounds__(RT_THREADS) k_tick_blocks(TickArgs A) {
     u32 rk = tick_owner(A.tick_off, A.n_ranks, t0);             // a rank that has ticks: t0 < n_ticks
     u64 seg_start = A.tick_off[rk], seg_end = A.tick_off[rk + 1];
     u32 carry_s = t0 ? __ldg(A.send + t0 - 1) : 0u, carry_r = t0 ? __ldg(A.recv + t0 - 1) : 0u;
-#pragma unroll 2
+    u32 sv_[RB_PER_WARP], rv_[RB_PER_WARP];                     // all loads of the warp's blocks are issued before the first is used
+#pragma unroll
+    for (int q = 0; q < RB_PER_WARP; ++q) {
+      const u64 i = t0 + (u64)q * 32 + lane;
+      const bool in = i < A.n_ticks;
+      sv_[q] = in ? __ldg(A.send + i) : 0u; rv_[q] = in ? __ldg(A.recv + i) : 0u;
+    }
+#pragma unroll
     for (int q = 0; q < RB_PER_WARP; ++q) {
       const u64 bstart = t0 + (u64)q * 32;
       if (bstart >= A.n_ticks) break;                           // the same in every lane
       const u64 bend = bstart + 32 < A.n_ticks ? bstart + 32 : A.n_ticks;
       const u64 i = bstart + lane;
       const bool in = i < A.n_ticks;
-      const u32 sv = in ? __ldg(A.send + i) : 0u, rv = in ? __ldg(A.recv + i) : 0u;
+      const u32 sv = sv_[q], rv = rv_[q];
       u32 ps = __shfl_up_sync(0xFFFFFFFFu, sv, 1), pr = __shfl_up_sync(0xFFFFFFFFu, rv, 1);
       if (lane == 0) { ps = carry_s; pr = carry_r; }
       carry_s = __shfl_sync(0xFFFFFFFFu, sv, 31); carry_r = __shfl_sync(0xFFFFFFFFu, rv, 31);
