@@ -76,6 +76,23 @@ __global__ void __launch_bounds__(RT_THREADS) k_tick_blocks(TickArgs A) {
     u64 seg_start = A.tick_off[rk], seg_end = A.tick_off[rk + 1];
     u32 carry_s = t0 ? __ldg(A.send + t0 - 1) : 0u, carry_r = t0 ? __ldg(A.recv + t0 - 1) : 0u;
     u32 sv_[RB_PER_WARP], rv_[RB_PER_WARP];                     // all loads of the warp's blocks are issued before the first is used
+    if (t0 + RB_PER_WARP * 32 <= A.n_ticks && seg_start < t0 && seg_end >= t0 + RB_PER_WARP * 32) {
+      // the usual case: all of the warp's ticks exist and lie inside one rank's segment, after its first tick
+      const u32 *ps_ = A.send + t0 + lane, *pr_ = A.recv + t0 + lane;
+#pragma unroll
+      for (int q = 0; q < RB_PER_WARP; ++q) { sv_[q] = __ldg(ps_ + q * 32); rv_[q] = __ldg(pr_ + q * 32); }
+      TickBlock* out = A.blk + (t0 >> 5);
+#pragma unroll
+      for (int q = 0; q < RB_PER_WARP; ++q) {
+        u32 ps = __shfl_up_sync(0xFFFFFFFFu, sv_[q], 1), pr = __shfl_up_sync(0xFFFFFFFFu, rv_[q], 1);
+        if (lane == 0) { ps = carry_s; pr = carry_r; }
+        carry_s = __shfl_sync(0xFFFFFFFFu, sv_[q], 31); carry_r = __shfl_sync(0xFFFFFFFFu, rv_[q], 31);
+        const u32 ms = __ballot_sync(0xFFFFFFFFu, sv_[q] != ps), mr = __ballot_sync(0xFFFFFFFFu, rv_[q] != pr);
+        const u64 cnt = (u64)__popc(ms) | ((u64)__popc(mr) << 32);
+        if (lane == 0) out[q] = make_ulonglong2(cnt, (u64)ms | ((u64)mr << 32));
+        wsum += cnt;
+      }
+    } else {
 #pragma unroll
     for (int q = 0; q < RB_PER_WARP; ++q) {
       const u64 i = t0 + (u64)q * 32 + lane;
@@ -104,6 +121,7 @@ __global__ void __launch_bounds__(RT_THREADS) k_tick_blocks(TickArgs A) {
       const u64 cnt = (u64)__popc(ms) | ((u64)__popc(mr) << 32);
       if (lane == 0) A.blk[bstart >> 5] = make_ulonglong2(cnt, (u64)ms | ((u64)mr << 32));
       wsum += cnt;
+    }
     }
   }
   if (lane == 0) s_cnt[wid] = wsum;
