@@ -444,6 +444,140 @@ def test_hang_tree_h3_fewest_counts_and_ring_tie_break():
     assert list(h["roots"]) == [12] and h["n_missing_frames"] == 1 and h["min_total"] == 0
 
 
+# ---------------------------------------------------------------- branches of the grouping, hand cases
+def test_invalid_times_make_the_group_incomplete():
+    # op 0: rank 1 reports a negative enter time; op 1: rank 2 leaves before it entered; op 2 is healthy.
+    recs = group_trace([[5, 5, 5, 5]] * 3)
+    for r in recs:
+        if r["seq"] == 0 and r["rank"] == 1:
+            r["t_enter"], r["t_exit"] = -7, 3
+        if r["seq"] == 1 and r["rank"] == 2:
+            r["t_exit"] = r["t_enter"] - 1
+    o = run(recs, [(0, [0, 1, 2, 3], 0)])
+    s, g = o.sizes(0), o.groups(0)
+    assert s["n_complete"] == 1 and s["n_incomplete"] == 2 and s["n_analysed"] == 1 and s["n_rejected"] == 0 and s["n_alerts"] == 0
+    # bit 7 of the group word = invalid time, bit 1 = incomplete, bit 0 = complete; every member is present
+    assert [int(f) & (1 | 2 | 64 | 128) for f in g["gflags"]] == [2 | 128, 2 | 128, 1]
+    assert list(g["n_present"]) == [4, 4, 4]
+    # an incomplete group carries no statistics, its records are present but not analysed, and it is no round of Eq. 1
+    for k in ("e_min", "t_max", "t_min", "span", "med_dur", "arrival_skew"):
+        assert list(g[k][:2]) == [0, 0], k
+    flags, perm = o.slots(0)
+    assert list(flags[:8]) == [128] * 8 and list(flags[8:]) == [0] * 4 and (perm != 0xFFFFFFFF).all()
+    assert o.comm_rows(0)["n_rounds"][0] == 1 and o.comm_rows(0)["sel_seq"][0] == 2
+    st = o.rank_stats(4)
+    assert list(st["ops"]) == [1] * 4 and list(st["bw_cnt"]) == [1] * 4
+
+
+def test_duplicate_record_keeps_the_first_and_counts_one_rejection():
+    # rank 2 reports op 0 twice: 40 ns first, 900 ns second. The first one stands.
+    recs = group_trace([[10, 20, 40, 30]])
+    recs.append(dict(rank=2, comm=0, seq=0, t_enter=recs[2]["t_enter"], t_exit=recs[2]["t_enter"] + 900))
+    o = run(recs, [(0, [0, 1, 2, 3], 0)])
+    s, g = o.sizes(0), o.groups(0)
+    assert s["n_rejected"] == 1 and s["error_bits"] == 8 and s["n_complete"] == 1 and s["n_slots"] == 4
+    assert g["t_max"][0] == 40 and g["rank_tmax"][0] == 2 and g["n_present"][0] == 4
+    assert list(o.slots(0)[1]) == [0, 1, 2, 3]
+    # the other way round: the 900 ns record comes first in the upload and is the one kept
+    recs = [recs[4]] + recs[:4]
+    o = run(recs, [(0, [0, 1, 2, 3], 0)])
+    assert o.groups(0)["t_max"][0] == 900 and o.sizes(0)["n_rejected"] == 1 and list(o.slots(0)[1]) == [1, 2, 0, 4]
+
+
+def test_counter_range_comes_from_trace_ids_not_from_membership():
+    # The Trace ID (Sec. 5.1) is communicator id + operation counter and carries no rank, so which operations a
+    # communicator issued in a window is read off the Trace IDs alone. A record of rank 77, which is not a member,
+    # names communicator 0 with counter 14 while the members report 10..11: the record is rejected, the operations
+    # 12..14 exist and nobody reported them (incomplete, no member present). A counter below the communicator's first
+    # (3 < 10) names no operation and widens nothing.
+    recs = group_trace([[5, 5, 5, 5], [5, 5, 5, 5]], seq0=10)
+    recs.append(dict(rank=77, comm=0, seq=14, t_enter=1, t_exit=2))
+    recs.append(dict(rank=77, comm=0, seq=3, t_enter=1, t_exit=2))
+    o = run(recs, [(0, [0, 1, 2, 3], 10)])
+    s, g = o.sizes(0), o.groups(0)
+    assert s["n_rejected"] == 2 and s["error_bits"] == 2
+    assert list(g["seq"]) == [10, 11, 12, 13, 14] and s["n_slots"] == 20
+    assert list(g["n_present"]) == [4, 4, 0, 0, 0] and s["n_complete"] == 2 and s["n_incomplete"] == 3
+    assert [int(f) & 3 for f in g["gflags"]] == [1, 1, 2, 2, 2]
+    flags, perm = o.slots(0)
+    assert list(flags[8:]) == [64 | 128] * 12 and (perm[8:] == 0xFFFFFFFF).all()
+    assert o.comm_rows(0)["n_rounds"][0] == 2
+    # the same record from a member would have been accepted into op 14
+    recs[-2]["rank"] = 1
+    o = run(recs, [(0, [0, 1, 2, 3], 10)])
+    assert list(o.groups(0)["n_present"]) == [4, 4, 0, 0, 1] and o.sizes(0)["n_rejected"] == 1
+
+
+def test_barrier_groups_add_nothing_to_the_bandwidth_sums():
+    # op 0: a 3-byte AllReduce (barrier), op 1: 16 MiB in 2 ms over 4 ranks: 16 MiB * 2*3/4 / 2e6 ns = 12.582912 GB/s
+    recs = group_trace([[1000] * 4], bytes=3) + group_trace([[2 * MS] * 4], seq0=1, t0=2 * 10**9)
+    o = run(recs, [(0, [0, 1, 2, 3], 0)])
+    st = o.rank_stats(4)
+    assert list(st["bw_cnt"]) == [1] * 4 and list(st["ops"]) == [1] * 4
+    assert st["bw_sum"] == pytest.approx([16 * MiB * 6 / 4 / (2 * MS)] * 4, rel=1e-15)
+    g = o.groups(0)
+    assert g["busbw"][1] == pytest.approx(12.582912, rel=1e-15)
+    assert g["busbw"][0] == pytest.approx(3 * 6 / 4 / 1000, rel=1e-15)      # the group value is still reported
+    assert o.comm_rows(0)["n_rounds"][0] == 1                               # and a barrier is no round of Eq. 1 / Eq. 2
+
+
+def test_eq1_two_minute_rule_at_the_boundary():
+    # "all rounds within the first two minutes" (Sec. 4.2.1): a round that starts exactly 120 s after the first is
+    # outside, one nanosecond earlier it is inside (and m stays open: 2 rounds < 100).
+    for gap, m, base, static in ((120 * 10**9, 1, 10, 0), (120 * 10**9 - 1, 0, 2 * MS, 1)):
+        recs = []
+        for s, (t, d) in enumerate([(0, 10), (gap, 50)]):
+            for rk in (0, 1):
+                recs.append(dict(rank=rk, comm=0, seq=s, t_enter=10**9 + t, t_exit=10**9 + t + d))
+        o = run(recs, [(0, [0, 1], 0)])
+        r = o.comm_rows(0)
+        assert (r["m"][0], r["t_base"][0], r["baseline_static"][0], r["rounds_total"][0]) == (m, base, static, 2), gap
+
+
+def test_suspect_threshold_order_and_mean_bandwidth():
+    # 8 ranks, 10 identical AllReduces of 16 MiB in 2 ms; late arrivals: rank 6 twice, ranks 3 and 1 once each;
+    # rank 0 takes 4 ms once. Skews and durations are otherwise equal, so MAD = 0 and every deviation is flagged.
+    durs = [[2 * MS] * 8 for _ in range(10)]
+    ents = [[0] * 8 for _ in range(10)]
+    ents[0][6] = ents[5][6] = 500_000
+    ents[2][3] = 500_000
+    ents[7][1] = 500_000
+    durs[4][0] = 4 * MS
+    o = run(group_trace(durs, ents), [(0, list(range(8)), 0)])
+    st = o.rank_stats(8)
+    assert list(st["votes"][:, 0]) == [0, 1, 0, 1, 0, 0, 2, 0] and list(st["votes"][:, 2]) == [1] + [0] * 7
+    assert list(st["ops"]) == [10] * 8
+    # votes * 1000 >= vote_rep_milli * ops with vote_rep_milli = 100: one vote in ten ops is exactly on the boundary
+    sus = o.suspects()
+    assert sus["n_total"] == 4
+    assert list(sus["kind"]) == [1, 1, 1, 2]                 # stragglers first,
+    assert list(sus["rank"]) == [6, 1, 3, 0]                 # more votes first, equal votes by rank
+    assert list(sus["votes"]) == [2, 1, 1, 1] and list(sus["ops"]) == [10] * 4
+    full = 16 * MiB * 14 / 8 / (2 * MS)                      # 14.680064 GB/s
+    assert full == pytest.approx(14.680064, rel=1e-15)
+    assert list(sus["mean_busbw"][:3]) == pytest.approx([full] * 3, rel=1e-12)
+    assert sus["mean_busbw"][3] == pytest.approx((9 * full + full / 2) / 10, rel=1e-12)
+    # one milli above the boundary the single-vote ranks drop out
+    o = run(group_trace(durs, ents), [(0, list(range(8)), 0)], params=dict(vote_rep_milli=101))
+    sus = o.suspects()
+    assert list(sus["kind"]) == [1] and list(sus["rank"]) == [6]
+
+
+def test_hang_tree_h1_counts_a_later_operation_counter_as_entered():
+    # Leaf H1 names the members whose operation counter did not advance to the hung op (Sec. 4.2.2). Op 3 hangs:
+    # ranks 0 and 1 are inside it, rank 2 has no record of op 3 but reports op 4 (its counter is past 3), rank 3 reports
+    # nothing from op 3 on. Only rank 3 is named.
+    recs = hang_records(4, 3, {0, 1}, set())
+    recs.append(dict(rank=2, comm=0, seq=4, t_enter=10**9 + 10, t_exit=-1))
+    o = run(recs, [(0, [0, 1, 2, 3], 0)])
+    h = o.locate_hang(0, 0, 3)
+    assert h["cls"] == 1 and list(h["roots"]) == [3] and h["n_not_entered"] == 1
+    assert h["n_hung"] == 4 and h["n_not_hung"] == 0
+    # asked about op 4 instead, ranks 0, 1 and 3 have not reached it
+    h = o.locate_hang(0, 0, 4)
+    assert h["cls"] == 1 and list(h["roots"]) == [0, 1, 3]
+
+
 # ---------------------------------------------------------------- the benchmark configurations
 def test_cfg1_rank5_is_the_sole_suspect():
     import tracegen as tg
