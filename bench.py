@@ -1,17 +1,22 @@
 """Benchmark of the CCL-D analyzer hot path: trace records analysed per second at 4,096 ranks.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--windows NW]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config cfg4|cfg4w|cfg5]
 
 A step is one pass of the whole hot path (group-by, per-op reductions, median/MAD flags, votes,
-window decision) over the streaming slow-mix workload: 4,096 ranks (TP8 x PP8 x DP64), NW windows
-of 1,000 ops per rank (NW = 100: 409.6 M records, 18.4 GB of SoA columns resident in HBM).
+window decision) over every window of the workload, which is resident in HBM before the timed
+region starts. The headline workload (--config cfg4) is the streaming slow mix: 4,096 ranks
+(TP8 x PP8 x DP64), 100 windows of 1,000 ops per rank, 409.6 M records, 18.4 GB of SoA columns.
+At one GPU the same JSON line also carries, as extra keys, the same step on arrival-ordered
+uploads, on the one-communicator reading of the workload (cfg4w: 4,096 ranks in one ring) and
+on the 16,384-rank scale stress (cfg5), each with its dominant kernel and roofline fraction.
 For N > 1 (under torch.distributed.run) every rank analyses its own trace on its own GPU: the path
 has no exchange step, so the ranks only meet at the timing barrier.
 
---impl reference times the CPU oracle (one host core) on a bounded sample of the same workload.
+--impl reference times the CPU oracle on a bounded sample of the same workload.
 Rank 0 prints one JSON line.
 """
 import argparse
+import hashlib
 import json
 import os
 import statistics
@@ -26,12 +31,23 @@ if ROOT not in sys.path:
 METRIC = "trace records analyzed/sec at 4,096 ranks"
 UNIT = "records/s"
 REC_BYTES = 45            # 3 x u32 keys, u8 op, u64 bytes, 2 x i64 times, 2 x u32 rate columns
+VAL_BYTES = 33            # what a reduce kernel reads of a record: op, bytes, two times, two rate columns
+FLAG_BYTES = 1
+INDEX_BYTES = 4           # the record index a reduce kernel reads per slot: regrouping overhead, not method bytes
 ROW_BYTES = 104           # one per-op row
 HBM_FALLBACK_GBS = 6650.0
-# DRAM traffic per record (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture divided by the records of the
-# captured launch; 5-window case, 20.48 M records, see profiles/). Traffic grows in proportion to the records, so a
-# launch's traffic is this figure times its records. Set an entry to None whenever its kernel changes.
-NCU_TRAFFIC_PER_RECORD = {"k_reduce_fused": (784.674560e6 + 243.086848e6) / 20.48e6}
+CSRC = os.path.join(ROOT, "paper_2605_04478_b200", "csrc")
+
+# DRAM traffic per record of a kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu capture divided by the
+# records of the captured launch; the capture and its command are under profiles/). Traffic grows in proportion to the
+# records, so a launch's traffic is this figure times its records. Each entry names the source files of its kernel and
+# their hash at capture time: once a file changes the figure is stale and the bench reports null.
+NCU_TRAFFIC = {
+    "k_reduce_fused": {"bytes_per_record": (784.674560e6 + 243.086848e6) / 20.48e6, "files": ("ccld_fused.cuh",),
+                       "sha16": "782164e361d25351"},
+}
+
+MIXES = {"all": ((0, 0, 1, 0, 2), 200), "tp_pp": ((0, 0, 1, 0), 250), "dp": ((2,), 200)}   # op pattern (0 TP, 1 PP, 2 DP), repetitions
 
 
 def parse():
@@ -40,22 +56,33 @@ def parse():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--windows", type=int, default=100, help="windows of 1,000 ops per rank resident on the GPU")
+    ap.add_argument("--config", default="cfg4", choices=["cfg4", "cfg4w", "cfg5"], help="headline workload")
+    ap.add_argument("--windows", type=int, default=0, help="windows resident on the GPU (0: the configuration's own count)")
     ap.add_argument("--e2e-windows", type=int, default=10, help="windows per end-to-end step (host buffers)")
-    ap.add_argument("--cpu-windows", type=int, default=10, help="windows the CPU oracle is timed on")
-    ap.add_argument("--mix", default="all", choices=sorted(MIXES), help="all: the cfg4 workload; tp_pp / dp: only its 8-rank or only its 64-rank "
-                    "communicators (timing one path of the fused kernel; the headline number is --mix all)")
+    ap.add_argument("--cpu-windows", type=int, default=10, help="windows the single-thread CPU oracle is timed on (0 = skip both oracle legs)")
+    ap.add_argument("--mix", default="all", choices=sorted(MIXES), help="cfg4 only. all: the whole workload; tp_pp / dp: only its 8-rank or only "
+                    "its 64-rank communicators (timing one path of the fused kernel; the headline number is --mix all)")
     ap.add_argument("--rate-windows", type=int, default=2, help="windows whose raw probe samples are turned into rate columns (0 = skip)")
+    ap.add_argument("--extra", default="arrival,cfg4w,cfg5", help="comma list of extra measurements at one GPU (arrival, cfg4w, cfg5; empty = none)")
     return ap.parse_args()
 
 
-MIXES = {"all": ((0, 0, 1, 0, 2), 200), "tp_pp": ((0, 0, 1, 0), 250), "dp": ((2,), 200)}   # op pattern (0 TP, 1 PP, 2 DP), repetitions
+WORKLOAD_TEXT = {
+    "cfg4": "cfg4 streaming slow mix: 4,096 ranks (TP8 x PP8 x DP64), %d windows of %s ops per rank",
+    "cfg4w": "cfg4w, the streaming workload as one 4,096-rank ring communicator: %d windows of %s AllReduces",
+    "cfg5": "cfg5 scale stress: 16,384 ranks (TP8, 128-rank blocks, DP2048, one 1,024-rank ring that hangs in window 25), %d windows of %s ops per rank",
+}
 
 
-def workload(n_windows, rank=0, mix="all"):
+def workload(config, n_windows=0, rank=0, mix="all"):
     import tracegen as tg
-    pattern, reps = MIXES[mix]
-    spec = tg.cfg4(reps=reps, n_windows=n_windows, pattern=pattern)
+    if config == "cfg4":
+        pattern, reps = MIXES[mix]
+        spec = tg.cfg4(reps=reps, n_windows=n_windows or 100, pattern=pattern)
+    elif config == "cfg4w":
+        spec = tg.cfg4w(n_windows=n_windows or 100)
+    else:
+        spec = tg.cfg5(n_windows=n_windows or 50, hang_window=min(25, max((n_windows or 50) - 1, 0)))
     spec.seed += 1000 * rank
     return spec
 
@@ -72,12 +99,53 @@ def class_units(spec):
     return out
 
 
+def kernel_units(spec):
+    """Records and groups per window each kernel of the path handles."""
+    u = class_units(spec)
+    allr, allg = sum(x[0] for x in u.values()), sum(x[1] for x in u.values())
+    return {"k_seq_range": (allr, allg), "k_slot_scatter": (allr, allg),
+            "k_reduce_fused": (u["small"][0] + u["warp"][0], u["small"][1] + u["warp"][1]),
+            "k_reduce_mid": tuple(u["mid"]), "k_reduce_large": tuple(u["large"])}
+
+
+def algorithmic_bytes(kernel, recs, groups):
+    """Bytes one launch must move for `recs` records in `groups` groups: (method bytes, regrouping overhead)."""
+    if kernel == "k_seq_range":
+        return 8 * recs, 0                                     # communicator id and op counter
+    if kernel == "k_slot_scatter":
+        return 12 * recs, 4 * recs                             # three key columns read; the record index written per slot
+    if kernel.startswith("k_reduce"):
+        return (VAL_BYTES + FLAG_BYTES) * recs + ROW_BYTES * groups, INDEX_BYTES * recs
+    return 0, 0
+
+
 def peak_hbm():
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
             return float(json.load(f)["hbm_gbs"]), "measured"
     except Exception:
         return HBM_FALLBACK_GBS, "fallback"
+
+
+def sources_sha16(files):
+    h = hashlib.sha256()
+    for name in files:
+        with open(os.path.join(CSRC, name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def ncu_traffic(kernel, recs):
+    """DRAM traffic of one launch from the committed ncu capture, or None when the kernel's sources changed since."""
+    ent = NCU_TRAFFIC.get(kernel)
+    if ent is None:
+        return None
+    try:
+        if sources_sha16(ent["files"]) != ent["sha16"]:
+            return None
+    except OSError:
+        return None
+    return ent["bytes_per_record"] * recs
 
 
 def max_over_ranks(ms, device):
@@ -92,7 +160,7 @@ def max_over_ranks(ms, device):
 
 
 class ClockSampler:
-    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    """Samples SM clocks and throttle reasons of one GPU with nvidia-smi (query mode) while the timed region runs."""
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -131,8 +199,18 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
+# ------------------------------------------------------------------------------------------------
+# the CPU oracle, timed as it stands
+# ------------------------------------------------------------------------------------------------
+def host_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
 def time_oracle(spec, windows, gen_device="cpu"):
-    """CPU oracle (single thread) on the given windows of the workload: records, seconds."""
+    """CPU oracle (one instance, one thread, windows in order) on the given windows: records, seconds."""
     import oracle as orc
     import tracegen as tg
     o = orc.Oracle()
@@ -152,10 +230,41 @@ def time_oracle(spec, windows, gen_device="cpu"):
     return n_rec, secs
 
 
+def time_oracle_all_cores(spec, windows, threads, gen_device="cpu"):
+    """The same oracle, one fresh instance per window, `threads` windows at a time on as many host cores."""
+    import oracle as orc
+    import tracegen as tg
+    items = []
+    for w in windows:
+        win = tg.gen_window(spec, w, device=gen_device)
+        items.append((w, {k: v.cpu().numpy() for k, v in win.cols.items()}, win.now_ns))
+    t0 = time.perf_counter()
+    _, _, n_rec = orc.analyze_windows_independently(tg.registry(spec), iter(items), spec.n_ranks, threads=threads)
+    return n_rec, time.perf_counter() - t0
+
+
+def cpu_baseline(spec, n_single, gen_device):
+    """One-core and all-core oracle legs on a bounded sample (about 10 to 30 s of CPU work in all)."""
+    NW = spec.n_windows
+    n1 = min(n_single, NW)
+    r1, t1 = time_oracle(spec, list(range(n1)), gen_device)
+    cores = host_cores()
+    threads = max(1, min(cores, 32))                  # a window in flight holds about 0.6 GB of host memory
+    per_window = t1 / max(n1, 1)
+    # two rounds of windows per thread, fewer if a window takes long (the 16.4 M-record windows of the scale stress)
+    n_all = max(1, min(NW, 2 * threads if per_window < 3.0 else threads))
+    ra, ta = time_oracle_all_cores(spec, list(range(n_all)), threads, gen_device)
+    return {"value": ra / ta, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": "%d of %d windows (%.3f M records), one oracle instance per window, %d at a time (host has %d cores)"
+                      % (n_all, NW, ra / 1e6, threads, cores),
+            "single_thread": {"value": r1 / t1, "unit": UNIT, "cores": 1,
+                              "sample": "%d of %d windows (%.3f M records), one instance, windows in order" % (n1, NW, r1 / 1e6)}}
+
+
 def run_reference(args, rank):
     if rank != 0:
         return
-    spec = workload(args.windows)
+    spec = workload(args.config, args.windows)
     n_rec = secs = 0
     for s in range(args.warmup + args.steps):
         r, t = time_oracle(spec, [s % spec.n_windows])
@@ -166,14 +275,108 @@ def run_reference(args, rank):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": 1e3 * secs / args.steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "int64", "data": "synthetic",
-        "config": {"workload": "cfg4 streaming slow mix: 4,096 ranks (TP8 x PP8 x DP64), windows of 1,000 ops per rank",
+        "config": {"workload": WORKLOAD_TEXT[args.config] % (spec.n_windows, format(spec.ops_per_window, ",")),
                    "records_per_step": n_rec // args.steps},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
-                         "sample": "one window (4.096 M records) of the workload per step"},
+                         "sample": "one window (%.3f M records) of the workload per step" % (n_rec / args.steps / 1e6)},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------------
+# the CUDA path
+# ------------------------------------------------------------------------------------------------
+def measure(spec, order, steps, warmup, local_rank, world, sample_clocks):
+    """Uploads every window of `spec` (device-resident), then times `steps` passes of the whole path."""
+    import torch
+    import torch.distributed as dist
+    import paper_2605_04478_b200 as ccld
+    import tracegen as tg
+    dev = torch.device("cuda", local_rank)
+    NW = spec.n_windows
+    an = ccld.Analyzer(device=local_rank)
+    for cid, ranks, seq0 in tg.registry(spec):
+        an.comm_register(cid, ranks, 0, seq0)
+    n_rec, now = 0, 0
+    for w in range(NW):
+        win = tg.gen_window(spec, w, device=dev, order=order)
+        an.trace_upload(w, win.cols, win.frames, win.n_channels)
+        n_rec += win.n_rec
+        now = win.now_ns
+    del win
+    torch.cuda.synchronize()
+
+    def step():
+        an.reset()
+        an.analyze_window(0, NW, now)
+
+    for _ in range(warmup):
+        step()
+    an.timing_enable(True)
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    sampler = ClockSampler(local_rank) if sample_clocks else None
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    for i in range(steps):
+        ev[i].record()
+        step()
+    ev[steps].record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    clocks = sampler.stop() if sampler else None
+    ms = max_over_ranks(ev[0].elapsed_time(ev[steps]), dev)
+    per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+    kt = an.get_kernel_times()
+    an.timing_enable(False)
+
+    # sanity: the injected ranks are the suspects
+    v = an.get_verdict(NW - 1, check=False)
+    sus = v["suspects"]
+    found = {"stragglers": sorted(set(int(r) for r in sus["rank"][sus["kind"] == 1])),
+             "slow_links": sorted(set(int(r) for r in sus["rank"][sus["kind"] == 2]))}
+    recovered = found["stragglers"] == spec.truth["stragglers"] and found["slow_links"] == spec.truth["slow_links"]
+    an.close()
+    del an
+    torch.cuda.empty_cache()
+
+    peak, peak_kind = peak_hbm()
+    ku = kernel_units(spec)
+    dom = max(kt, key=lambda k: kt[k]["ms"])
+    d_ms = kt[dom]["ms"] / max(kt[dom]["launches"], 1)
+    recs, groups = ku.get(dom, (0, 0))
+    d_alg, d_over = algorithmic_bytes(dom, NW * recs, NW * groups)
+    achieved = d_alg / (d_ms * 1e-3) / 1e9 if d_ms > 0 else 0.0
+    n_groups = NW * sum(x[1] for x in class_units(spec).values())
+    path_bytes = (REC_BYTES + FLAG_BYTES) * n_rec + ROW_BYTES * n_groups
+    path_gbs = path_bytes * steps / (ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": ncu_traffic(dom, NW * recs), "peak_source": peak_kind, "ms_per_launch": d_ms,
+                "algorithmic_bytes_per_launch": d_alg,
+                "regrouping_bytes_per_launch": d_over,
+                "achieved_with_regrouping_bytes": (d_alg + d_over) / (d_ms * 1e-3) / 1e9 if d_ms > 0 else 0.0,
+                "kernels_ms_per_step": {k: kt[k]["ms"] / steps for k in kt},
+                "whole_path": {"algorithmic_bytes_per_step": path_bytes, "achieved": path_gbs, "frac": path_gbs / peak}}
+    # every launch of the fused reduce kernel is followed by one of k_reduce_deferred (timed inside the same event pair),
+    # likewise k_reduce_large and its deferred kernel, and every launch of k_window_decide is preceded by one of k_window_rounds
+    launches = (sum(x["launches"] for x in kt.values()) + kt["k_reduce_fused"]["launches"] + kt["k_reduce_large"]["launches"]
+                + kt["k_window_decide"]["launches"])
+    return {"n_rec": n_rec, "now": now, "ms_total": ms, "ms_per_step": ms / steps, "ms_best": min(per_step), "ms_median": statistics.median(per_step),
+            "value": world * n_rec * steps / (ms * 1e-3), "value_best": world * n_rec / (min(per_step) * 1e-3),
+            "value_median": world * n_rec / (statistics.median(per_step) * 1e-3),
+            "clocks": clocks, "roofline": roofline, "launches": launches, "recovered": recovered, "n_groups": n_groups}
+
+
+def brief(m, spec, config, order):
+    r = m["roofline"]
+    return {"workload": WORKLOAD_TEXT[config] % (spec.n_windows, format(spec.ops_per_window, ",")) + ", %s upload order" % order.replace("_", "-"),
+            "records_per_step": m["n_rec"], "value": m["value"], "unit": UNIT, "ms_per_step": m["ms_per_step"], "ms_best": m["ms_best"],
+            "ms_median": m["ms_median"], "dominant_kernel": r["kernel"], "dominant_ms_per_launch": r["ms_per_launch"], "dominant_frac": r["frac"],
+            "whole_path_gbs": r["whole_path"]["achieved"], "whole_path_frac": r["whole_path"]["frac"],
+            "kernels_ms_per_step": r["kernels_ms_per_step"], "injected_ranks_recovered": m["recovered"]}
 
 
 def run_ours(args, rank, world, local_rank):
@@ -189,83 +392,23 @@ def run_ours(args, rank, world, local_rank):
 
     cpu_base = None
     if rank == 0 and world == 1 and args.cpu_windows > 0:
-        spec0 = workload(args.windows, 0, args.mix)
-        r, t = time_oracle(spec0, list(range(min(args.cpu_windows, spec0.n_windows))), gen_device=dev)
-        cpu_base = {"value": r / t, "unit": UNIT, "cores": 1, "kind": "oracle",
-                    "sample": "%d of %d windows (%.3f M records), single thread" % (min(args.cpu_windows, spec0.n_windows), spec0.n_windows, r / 1e6)}
+        cpu_base = cpu_baseline(workload(args.config, args.windows, 0, args.mix), args.cpu_windows, dev)
 
-    spec = workload(args.windows, rank, args.mix)
+    spec = workload(args.config, args.windows, rank, args.mix)
     NW = spec.n_windows
-    an = ccld.Analyzer(device=local_rank)
-    for cid, ranks, seq0 in tg.registry(spec):
-        an.comm_register(cid, ranks, 0, seq0)
-    n_rec = 0
-    now = 0
-    for w in range(NW):
-        win = tg.gen_window(spec, w, device=dev)
-        an.trace_upload(w, win.cols)
-        n_rec += win.n_rec
-        now = win.now_ns
-    torch.cuda.synchronize()
+    m = measure(spec, "rank_major", args.steps, args.warmup, local_rank, world, True)
+    n_rec, now = m["n_rec"], m["now"]
+    peak = m["roofline"]["peak"]
 
-    def step():
-        an.reset()
-        an.analyze_window(0, NW, now)
-
-    for _ in range(args.warmup):
-        step()
-    an.timing_enable(True)
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    sampler = ClockSampler(local_rank)
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    for _ in range(args.steps):
-        step()
-    ev1.record()
-    torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
-    clocks = sampler.stop()
-    ms = ev0.elapsed_time(ev1)
-    kt = an.get_kernel_times()
-    an.timing_enable(False)
-    ms = max_over_ranks(ms, dev)
-    value = world * n_rec * args.steps / (ms * 1e-3)
-
-    # sanity: the injected ranks are the suspects
-    v = an.get_verdict(NW - 1)
-    sus = v["suspects"]
-    found = {"stragglers": sorted(set(int(r) for r in sus["rank"][sus["kind"] == 1])),
-             "slow_links": sorted(set(int(r) for r in sus["rank"][sus["kind"] == 2]))}
-    recovered = found["stragglers"] == spec.truth["stragglers"] and found["slow_links"] == spec.truth["slow_links"]
-
-    # ---- roofline of the dominant kernel ----
-    units = class_units(spec)
-    alg = {   # algorithmic bytes one launch moves (per window: records, groups of the class)
-        "k_seq_range": lambda: NW * 8 * sum(u[0] for u in units.values()),
-        "k_slot_scatter": lambda: NW * (12 + 4) * sum(u[0] for u in units.values()),
-        "k_reduce_fused": lambda: NW * ((4 + 33 + 1) * (units["small"][0] + units["warp"][0]) + ROW_BYTES * (units["small"][1] + units["warp"][1])),
-        "k_reduce_mid": lambda: NW * ((4 + 33 + 1) * units["mid"][0] + ROW_BYTES * units["mid"][1]),
-        "k_reduce_large": lambda: NW * ((4 + 33 + 1) * units["large"][0] + ROW_BYTES * units["large"][1]),
-    }
-    dom = max(kt, key=lambda k: kt[k]["ms"])
-    peak, peak_kind = peak_hbm()
-    d_ms = kt[dom]["ms"] / max(kt[dom]["launches"], 1)
-    d_bytes = alg.get(dom, lambda: 0)()
-    achieved = d_bytes / (d_ms * 1e-3) / 1e9 if d_ms > 0 else 0.0
-    path_bytes = REC_BYTES * n_rec + n_rec + ROW_BYTES * NW * sum(u[1] for u in units.values())
-    path_gbs = path_bytes * args.steps / (ms * 1e-3) / 1e9
-    tpr = NCU_TRAFFIC_PER_RECORD.get(dom)
-    traffic = tpr * NW * (units["small"][0] + units["warp"][0]) if tpr is not None else None   # records of the kernel's classes
-    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": traffic, "peak_source": peak_kind, "ms_per_launch": d_ms, "algorithmic_bytes_per_launch": d_bytes,
-                "kernels_ms_per_step": {k: kt[k]["ms"] / args.steps for k in kt},
-                "whole_path": {"algorithmic_bytes_per_step": path_bytes, "achieved": path_gbs, "frac": path_gbs / peak}}
-    # every launch of the fused reduce kernel is followed by one of k_reduce_deferred (timed inside the same event pair)
-    # and every launch of k_window_decide is preceded by one of k_window_rounds
-    launches = sum(x["launches"] for x in kt.values()) + kt["k_reduce_fused"]["launches"] + kt["k_window_decide"]["launches"]
+    extras = [x for x in args.extra.split(",") if x] if (world == 1 and args.mix == "all") else []
+    other = {}
+    x_steps, x_warm = max(3, min(args.steps, 5)), max(3, min(args.warmup, 3))
+    if "arrival" in extras:
+        other["arrival_order"] = brief(measure(spec, "arrival", x_steps, x_warm, local_rank, world, False), spec, args.config, "arrival")
+    for cfg in ("cfg4", "cfg4w", "cfg5"):
+        if cfg in extras and cfg != args.config:
+            xs = workload(cfg, 0, rank)
+            other[cfg] = brief(measure(xs, "rank_major", x_steps, x_warm, local_rank, world, False), xs, cfg, "rank_major")
 
     # ---- end to end: host buffers -> upload -> analyse -> verdict ----
     NE = min(args.e2e_windows, NW)
@@ -312,15 +455,17 @@ def run_ours(args, rank, world, local_rank):
         e2e = {"value": world * e_rec * e_steps / (e_ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                "windows_per_step": NE, "steps": e_steps, "ms_per_step": e_ms / e_steps}
         an_e.close()
+        del host
 
     # ---- counter changes per op from raw probe samples (the step before the path), timed on its own ----
     rates = None
     NR = min(args.rate_windows, NW)
-    if NR > 0:
+    if NR > 0 and args.config == "cfg4":
+        an_r = ccld.Analyzer(device=local_rank)
         win = tg.gen_window(spec, 0, device=dev)
         ticks = tg.gen_ticks(win.cols, spec.n_ranks)
-        call = lambda: an.derive_rates(win.cols["rank"], win.cols["t_enter"], win.cols["t_exit"], ticks["tick_off"], ticks["tick_ns"],
-                                       ticks["send_count"], ticks["recv_count"])
+        call = lambda: an_r.derive_rates(win.cols["rank"], win.cols["t_enter"], win.cols["t_exit"], ticks["tick_off"], ticks["tick_ns"],
+                                         ticks["send_count"], ticks["recv_count"])
         for _ in range(3):
             call()
         torch.cuda.synchronize()
@@ -335,20 +480,24 @@ def run_ours(args, rank, world, local_rank):
         r_bytes = 16 * n_t + 28 * win.n_rec              # ticks read once (time, two counters); rank and times read, two counts written
         rates = {"records": win.n_rec, "ticks": n_t, "ms_per_window": r_ms, "algorithmic_bytes": r_bytes,
                  "achieved": r_bytes / (r_ms * 1e-3) / 1e9, "unit": "GB/s", "frac": r_bytes / (r_ms * 1e-3) / 1e9 / peak, "launches_per_window": 4}
+        an_r.close()
         del win, ticks
 
     if rank == 0:
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "metric": METRIC, "value": m["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": m["ms_per_step"], "ms_best": m["ms_best"], "ms_median": m["ms_median"],
+            "value_best": m["value_best"], "value_median": m["value_median"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "int64", "data": "synthetic",
-            "config": {"workload": "cfg4 streaming slow mix: 4,096 ranks (TP8 x PP8 x DP64), %d windows of %s ops per rank, rank-major upload order%s"
-                                   % (NW, format(spec.ops_per_window, ","), "" if args.mix == "all" else " (--mix %s: one communicator class only)" % args.mix),
+            "config": {"workload": WORKLOAD_TEXT[args.config] % (NW, format(spec.ops_per_window, ",")) + ", rank-major upload order"
+                                   + ("" if args.mix == "all" else " (--mix %s: one communicator class only)" % args.mix),
                        "records_per_gpu": n_rec, "bytes_per_record": REC_BYTES, "l2": "inputs larger than L2 (%.1f GB of columns per GPU)" % (n_rec * REC_BYTES / 1e9),
-                       "injected_ranks_recovered": recovered},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "cpu_baseline": cpu_base,
+                       "injected_ranks_recovered": m["recovered"]},
+            "clocks": m["clocks"], "e2e": e2e, "gpu_launches": m["launches"], "roofline": m["roofline"], "cpu_baseline": cpu_base,
             "derive_rates": rates,
         }
+        line.update(other)
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -379,12 +379,21 @@ int ccld_get_kernel_times(ccld_ctx* ctx, double* ms /* host [CCLD_K_KINDS] */, u
 /*
  * Hang location for one ring without any allocation. The paper has no counterpart to this entry
  * point; it exists for callers that cannot allocate device memory when they need a diagnosis: a
- * watchdog or signal handler looking at a job whose memory is exhausted or whose allocator sits
- * behind the hang itself, a plugin hosted inside another process that must leave that process's
- * memory pool alone, or a monitoring loop in which an allocation could stall the device. It needs
- * no context and calls no cudaMalloc, cudaFree or allocating library routine; its working memory is
- * one fixed array of CCLD_STATIC_SCRATCH_BYTES bytes that is part of the library image, so every GPU
- * that loads the library holds that much from load to exit.
+ * watchdog thread looking at a job whose memory is exhausted or whose allocator sits behind the
+ * hang itself, a plugin hosted inside another process that must leave that process's memory pool
+ * alone, or a monitoring loop in which an allocation could stall the device. It needs no context and
+ * calls no cudaMalloc, cudaFree or allocating library routine; its working memory is one fixed array
+ * of CCLD_STATIC_SCRATCH_BYTES bytes inside the library's device image, so every GPU on which the
+ * library has been used holds that much until the process exits.
+ *
+ * Set-up call. The CUDA runtime creates a device's primary context and loads the library's device
+ * image (the array and the kernel) lazily, the first time a call names that device; that one-time
+ * step does take device memory and fails with CCLD_ERR_NOMEM or CCLD_ERR_CUDA when none is left.
+ * The first call on a device also looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current) and caches it. So make one call per device at start-up, while memory is
+ * still available and before any stream capture begins (a one-member ring is enough); only the
+ * calls after it allocate nothing. This is an ordinary host function: call it from a thread, not
+ * from a signal handler.
  *
  * Inputs (all device memory on `device`, owned by the caller), indexed by ring position p < n_members:
  *   ranks[p]       rank id of the member at position p (position p sends to p+1 mod n)
@@ -397,12 +406,10 @@ int ccld_get_kernel_times(ccld_ctx* ctx, double* ms /* host [CCLD_K_KINDS] */, u
  * `cuda_stream` and synchronizes that stream before it returns.
  *
  * Limits and rules: n_members <= CCLD_STATIC_MAX_MEMBERS, else CCLD_ERR_CAPACITY and nothing runs.
- * `err` (host, may be NULL) receives a message of at most err_cap bytes on failure. The first call on
- * a device looks up the array's device address (cudaGetSymbolAddress, with that device current) and
- * caches it; make that first call before any stream capture begins. All calls on a device share the
- * array, which keeps the previous call's contents; the kernel rewrites every entry it reads, but calls
- * whose kernels overlap on the GPU (other streams or host threads) race and must be serialized by the
- * caller. The caller's current device is restored on return.
+ * `err` (host, may be NULL) receives a message of at most err_cap bytes on failure. All calls on a
+ * device share the array, which keeps the previous call's contents; the kernel rewrites every entry it
+ * reads, but calls whose kernels overlap on the GPU (other streams or host threads) race and must be
+ * serialized by the caller. The caller's current device is restored on return.
  */
 #define CCLD_STATIC_MAX_MEMBERS 8192u
 #define CCLD_STATIC_SCRATCH_BYTES (CCLD_STATIC_MAX_MEMBERS * 12u + 256u)

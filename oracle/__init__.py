@@ -43,7 +43,7 @@ def _load():
         _lib.orc_destroy.argtypes = [C.c_void_p]
         for name in ("orc_comm_register", "orc_upload", "orc_release", "orc_analyze", "orc_window_sizes",
                      "orc_copy_groups", "orc_copy_slots", "orc_copy_comm_rows", "orc_copy_alerts",
-                     "orc_copy_rank_stats", "orc_suspects", "orc_locate_hang", "orc_attach_opset", "orc_opset_check", "orc_comm_set_layers"):
+                     "orc_copy_rank_stats", "orc_add_rank_stats", "orc_suspects", "orc_locate_hang", "orc_attach_opset", "orc_opset_check", "orc_comm_set_layers"):
             getattr(_lib, name).restype = C.c_int
         _lib.orc_derive_rates.restype = None
     return _lib
@@ -153,6 +153,11 @@ class Oracle:
         self.lib.orc_copy_rank_stats(self.h, C.c_uint32(n_ranks), _p(votes), _p(ops), _p(cnt), _p(bw))
         return {"votes": votes, "ops": ops, "bw_cnt": cnt, "bw_sum": bw}
 
+    def add_rank_stats(self, st: Dict[str, np.ndarray]) -> int:
+        """Adds the per-rank statistics another instance returned from rank_stats() to this instance's."""
+        v = _np(st["votes"], np.uint32); ops = _np(st["ops"], np.uint32); cnt = _np(st["bw_cnt"], np.uint32); bw = _np(st["bw_sum"], np.float64)
+        return self.lib.orc_add_rank_stats(self.h, C.c_uint32(len(ops)), _p(v), _p(ops), _p(cnt), _p(bw))
+
     def suspects(self, cap: int = 65536) -> Dict[str, np.ndarray]:
         kind = np.zeros(cap, np.uint32); rank = np.zeros(cap, np.uint32); votes = np.zeros(cap, np.uint32)
         ops = np.zeros(cap, np.uint32); bw = np.zeros(cap, np.float64)
@@ -195,3 +200,45 @@ def derive_rates(rank, t_enter, t_exit, tick_off, tick_ns, send_count, recv_coun
     lib.orc_derive_rates(C.c_uint64(n), _p(rank), _p(te), _p(tx), C.c_uint32(len(off) - 1), _p(off), _p(tn), _p(sc), _p(rc),
                          _p(out_s), _p(out_r))
     return out_s, out_r
+
+
+def analyze_windows_independently(registry, windows, n_ranks: int, threads: int = 1, params=None, keep=None):
+    """Each window on a fresh Oracle of its own (one instance per thread at a time; ctypes calls release the GIL, so
+    `threads` host cores work side by side). `windows` yields (window_id, cols, now_ns) with CPU columns. Returns the
+    summed per-rank statistics, the per-window size dictionaries and the number of records analysed. Per-window results
+    that depend on earlier windows (the Eq. 1 baseline, the repetition counter) are not meaningful here; the per-op
+    table, flags, counts and the per-rank sums are. keep(window_id, oracle) is called before an instance is dropped.
+    """
+    from concurrent.futures import ThreadPoolExecutor
+
+    def one(item):
+        wid, cols, now = item
+        o = Oracle(params)
+        for cid, ranks, seq0 in registry:
+            o.comm_register(cid, ranks, seq0)
+        o.upload(wid, cols)
+        o.analyze(wid, 1, now)
+        sz = o.sizes(wid)
+        st = o.rank_stats(n_ranks)
+        if keep is not None:
+            keep(wid, o)
+        return wid, sz, st
+
+    total = {"votes": np.zeros((n_ranks, 4), np.uint32), "ops": np.zeros(n_ranks, np.uint32),
+             "bw_cnt": np.zeros(n_ranks, np.uint32), "bw_sum": np.zeros(n_ranks, np.float64)}
+    sizes, n_rec = {}, 0
+    with ThreadPoolExecutor(max_workers=max(1, threads)) as ex:
+        # windows are pulled lazily, at most 2 x threads in flight, so host memory stays bounded
+        import itertools
+        it = iter(windows)
+        pending = [ex.submit(one, item) for item in itertools.islice(it, 2 * max(1, threads))]
+        while pending:
+            wid, sz, st = pending.pop(0).result()
+            for k in total:
+                total[k] += st[k]
+            sizes[wid] = sz
+            n_rec += sz["n_records"]
+            nxt = next(it, None)
+            if nxt is not None:
+                pending.append(ex.submit(one, nxt))
+    return total, sizes, n_rec

@@ -1,9 +1,11 @@
 // CCL-D decision-analyzer oracle: TEST INFRASTRUCTURE ONLY.
 //
-// A plain, single-threaded, sort-based C++17 statement of what the analyzer hot path computes,
+// A plain, sort-based C++17 statement of what the analyzer hot path computes,
 // written from the paper's definitions (Sec. 4.1.2, Sec. 4.2.1 Eq. 1-3, Sec. 4.2.2 Eq. 4 and the
 // hang decision tree of Fig. 6) and from the per-op statistics this repository adds to them
 // (arrival skew, duration, bus bandwidth, lower-median / MAD outlier test, per-rank votes).
+// One instance runs on one thread; independent instances (one per window) may run side by side on several host cores
+// and their per-rank statistics add up (orc_add_rank_stats).
 // It shares no code, header, table or helper with the CUDA library and must never be called by
 // the product path: only the tests, the smoke check and the benchmark's CPU-baseline leg use it.
 //
@@ -440,6 +442,20 @@ int orc_copy_rank_stats(void* h, u32 n_ranks, u32* votes /*[n][4]*/, u32* ops, u
     RankStat s; if (it != o->stats.end()) s = it->second;
     for (int k = 0; k < 4; ++k) votes[r * 4 + k] = s.v[k];
     ops[r] = s.ops; bw_cnt[r] = s.bw_cnt; bw_sum[r] = s.bw_sum;
+  }
+  return 0;
+}
+
+// Adds per-rank statistics gathered elsewhere (another oracle instance that analysed other windows) to this one's:
+// votes, analysed-op counts and bandwidth sums are plain sums over windows, so windows analysed independently - each by
+// its own single-threaded instance, possibly at the same time on different host cores - combine by addition.
+int orc_add_rank_stats(void* h, u32 n_ranks, const u32* votes /*[n][4]*/, const u32* ops, const u32* bw_cnt, const double* bw_sum) {
+  Oracle* o = (Oracle*)h;
+  for (u32 r = 0; r < n_ranks; ++r) {
+    if (ops[r] == 0 && bw_cnt[r] == 0 && !(votes[r * 4] | votes[r * 4 + 1] | votes[r * 4 + 2] | votes[r * 4 + 3])) continue;
+    RankStat& s = o->stats[r];
+    for (int k = 0; k < 4; ++k) s.v[k] += votes[r * 4 + k];
+    s.ops += ops[r]; s.bw_cnt += bw_cnt[r]; s.bw_sum += bw_sum[r];
   }
   return 0;
 }

@@ -1,15 +1,24 @@
 // ccld_ring_locate_static: the hang decision tree over one ring, for callers that may not allocate.
 //
-// Who needs this: code that runs where device allocation is off the table - a watchdog or signal
-// path that must diagnose a job whose memory is exhausted or whose allocator is wedged behind the
-// very hang being diagnosed, a plugin that lives inside another process (a CCL profiler hook, a
-// framework extension) and is forbidden to touch that process's memory pool, or a tight monitoring
-// loop where an allocation could synchronize the device. Everything this entry point needs beyond
-// the caller's own buffers sits in one fixed array that is part of the loaded library image.
+// Who needs this: code that runs where device allocation is off the table - a watchdog thread that
+// must diagnose a job whose memory is exhausted or whose allocator is wedged behind the very hang
+// being diagnosed, a plugin that lives inside another process (a CCL profiler hook, a framework
+// extension) and is forbidden to touch that process's memory pool, or a tight monitoring loop where
+// an allocation could synchronize the device. Everything this entry point needs beyond the caller's
+// own buffers sits in one fixed array that is part of the library's device image.
+//
+// What "allocates nothing" covers: the entry point itself never calls cudaMalloc, cudaFree or an
+// allocating library routine. The CUDA runtime, however, creates a device's primary context and loads
+// this library's device image (array and kernel) lazily, on the first call that names that device, and
+// that one-time step takes device memory and can fail when none is left. So the first call on a
+// device is the set-up call: make it once at start-up, while memory is still available (any small
+// ring will do), and only the calls after it are free of allocation. It is an ordinary host function
+// (runtime calls, snprintf): call it from a thread, never from a signal handler.
 //
 // The scratch array is shared by every call on a device and keeps whatever the last call left in it.
 // The kernel overwrites every byte it later reads, so stale contents are harmless, but two calls
 // whose kernels overlap on the GPU (different streams, different host threads) race on it.
+#include <atomic>
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
@@ -33,12 +42,15 @@ constexpr size_t OFF_OUT = OFF_ROOTS + (size_t)MAX_N * 4;
 constexpr size_t SCRATCH_BYTES = OFF_OUT + 256;
 static_assert(SCRATCH_BYTES == CCLD_STATIC_SCRATCH_BYTES, "header and implementation disagree on the scratch size");
 
-// Lives in every GPU's copy of the library image from load to exit. In host code this name is only a
-// handle for cudaGetSymbolAddress; it is never passed to a kernel as if it were a device address.
+// Lives in every GPU's copy of the library's device image from the moment the runtime loads it there (the first call
+// on that device) until exit. In host code this name is only a handle for cudaGetSymbolAddress; it is never passed
+// to a kernel as if it were a device address.
 static __device__ __align__(256) unsigned char g_ring_scratch[SCRATCH_BYTES];
 
 constexpr int MAX_DEVICES = 64;
-void* g_scratch_addr[MAX_DEVICES];          // device address of g_ring_scratch on each device, once looked up
+// Device address of g_ring_scratch on each device, once looked up. Host threads may race to fill an entry; they all
+// store the same address, and the atomic makes the publication well defined.
+std::atomic<void*> g_scratch_addr[MAX_DEVICES];
 
 template <class T, class Op>
 __device__ T cta_reduce(T v, Op op, T* s_red /*[32]*/) {
@@ -153,14 +165,16 @@ extern "C" int ccld_ring_locate_static(int device, void* cuda_stream, uint32_t n
   int rc = CCLD_OK;
   cudaStream_t st = (cudaStream_t)cuda_stream;
   // set-up, once per device and with that device current: ask the runtime where the array lives there
-  if (g_scratch_addr[device] == nullptr) {
+  if (g_scratch_addr[device].load(std::memory_order_acquire) == nullptr) {
     void* p = nullptr;
     cudaError_t e = cudaGetSymbolAddress(&p, g_ring_scratch);
-    if (e != cudaSuccess || p == nullptr) { rc = say(err, err_cap, CCLD_ERR_CUDA, cudaGetErrorString(e)); goto done; }
-    g_scratch_addr[device] = p;
+    if (e != cudaSuccess || p == nullptr) {
+      rc = say(err, err_cap, e == cudaErrorMemoryAllocation ? CCLD_ERR_NOMEM : CCLD_ERR_CUDA, cudaGetErrorString(e)); goto done;
+    }
+    g_scratch_addr[device].store(p, std::memory_order_release);
   }
   {
-    unsigned char* scratch = (unsigned char*)g_scratch_addr[device];
+    unsigned char* scratch = (unsigned char*)g_scratch_addr[device].load(std::memory_order_acquire);
     k_ring_locate_static<<<1, 1024, 0, st>>>(n_members, ranks, state, n_channels, progress, scratch);
     cudaError_t e = cudaGetLastError();
     ccld_hang_verdict v;

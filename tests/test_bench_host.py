@@ -16,7 +16,7 @@ import bench
 rank = int(os.environ["RANK"])
 dist.init_process_group("gloo")
 ms = bench.max_over_ranks(10.0 + 5.0 * rank, torch.device("cpu"))
-spec = bench.workload(3, rank)
+spec = bench.workload("cfg4", 3, rank)
 print("RESULT", rank, ms, spec.seed, flush=True)
 dist.destroy_process_group()
 """
@@ -25,12 +25,43 @@ dist.destroy_process_group()
 def test_class_units_of_the_bench_workload():
     sys.path.insert(0, ROOT)
     import bench
-    spec = bench.workload(100)
+    spec = bench.workload("cfg4", 100)
     u = bench.class_units(spec)
     assert u["small"] == [4096 * 800, 512 * 600 + 512 * 200] and u["warp"] == [4096 * 200, 64 * 200]
     assert u["mid"] == [0, 0] and u["large"] == [0, 0]
     assert sum(x[0] for x in u.values()) == 4_096_000
-    assert bench.workload(3, 1).seed != bench.workload(3, 0).seed
+    assert bench.workload("cfg4", 3, 1).seed != bench.workload("cfg4", 3, 0).seed
+
+
+def test_units_and_bytes_of_the_other_workloads():
+    sys.path.insert(0, ROOT)
+    import bench
+    w = bench.workload("cfg4w")
+    assert w.n_windows == 100 and bench.class_units(w)["large"] == [4_096_000, 1000]
+    assert bench.kernel_units(w)["k_reduce_large"] == (4_096_000, 1000) and bench.kernel_units(w)["k_reduce_fused"] == (0, 0)
+    s = bench.workload("cfg5")
+    u = bench.class_units(s)
+    assert s.n_windows == 50 and s.hang.window == 25
+    assert u["small"] == [16_384 * 500, 2048 * 500] and u["warp"] == [16_384 * 250, 128 * 250]
+    assert u["large"] == [16_384 * 250, 8 * 250] and u["mid"] == [1024 * 10, 10]
+    # a reduce kernel's method bytes: values and flag per record, one row per group; the record index it also reads is overhead
+    assert bench.algorithmic_bytes("k_reduce_fused", 1000, 10) == (34 * 1000 + 104 * 10, 4 * 1000)
+    assert bench.algorithmic_bytes("k_seq_range", 1000, 10) == (8000, 0)
+    assert bench.algorithmic_bytes("k_slot_scatter", 1000, 10) == (12000, 4000)
+
+
+def test_ncu_traffic_goes_stale_with_the_kernel_source(monkeypatch):
+    sys.path.insert(0, ROOT)
+    import bench
+    ent = bench.NCU_TRAFFIC["k_reduce_fused"]
+    fresh = bench.sources_sha16(ent["files"]) == ent["sha16"]
+    t = bench.ncu_traffic("k_reduce_fused", 1_000_000)
+    assert (t is not None) == fresh
+    if fresh:
+        assert t == ent["bytes_per_record"] * 1_000_000
+    monkeypatch.setitem(bench.NCU_TRAFFIC, "k_reduce_fused", dict(ent, sha16="0" * 16))
+    assert bench.ncu_traffic("k_reduce_fused", 1_000_000) is None
+    assert bench.ncu_traffic("k_plan", 5) is None
 
 
 def test_max_over_ranks_with_two_gloo_ranks(tmp_path):

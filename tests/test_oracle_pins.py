@@ -444,6 +444,37 @@ def test_hang_tree_h3_fewest_counts_and_ring_tie_break():
     assert list(h["roots"]) == [12] and h["n_missing_frames"] == 1 and h["min_total"] == 0
 
 
+def test_windows_analysed_independently_add_up_to_the_sequential_run():
+    """Votes, analysed-op counts and bandwidth sums are sums over windows: one fresh instance per window, four at a
+    time, merged by addition, gives the statistics and the suspect list of one instance that saw the windows in order."""
+    import tracegen as tg
+    spec = tg.cfg2(reps=40, n_windows=5)
+    reg = tg.registry(spec)
+    wins = [tg.gen_window(spec, w) for w in range(spec.n_windows)]
+    now = wins[-1].now_ns
+    o = orc.Oracle()
+    for cid, ranks, seq0 in reg:
+        o.comm_register(cid, ranks, seq0)
+    for w, win in enumerate(wins):
+        o.upload(w, win.cols)
+    o.analyze(0, len(wins), now)
+    tot, sizes, n_rec = orc.analyze_windows_independently(reg, ((w, win.cols, now) for w, win in enumerate(wins)), spec.n_ranks, threads=4)
+    assert n_rec == sum(w.n_rec for w in wins) and sorted(sizes) == list(range(5))
+    ref = o.rank_stats(spec.n_ranks)
+    for k in ("votes", "ops", "bw_cnt"):
+        assert np.array_equal(ref[k], tot[k]), k
+    assert np.allclose(ref["bw_sum"], tot["bw_sum"], rtol=1e-12, atol=0)
+    for w in range(5):
+        assert sizes[w]["n_flag_skew"] == o.sizes(w)["n_flag_skew"] and sizes[w]["n_groups"] == o.sizes(w)["n_groups"]
+    merged = orc.Oracle()
+    merged.add_rank_stats(tot)
+    a, b = o.suspects(), merged.suspects()
+    assert a["n_total"] == b["n_total"] > 0
+    for k in ("kind", "rank", "votes", "ops"):
+        assert np.array_equal(a[k], b[k]), k
+    assert np.allclose(a["mean_busbw"], b["mean_busbw"], rtol=1e-12, atol=0)
+
+
 # ---------------------------------------------------------------- branches of the grouping, hand cases
 def test_invalid_times_make_the_group_incomplete():
     # op 0: rank 1 reports a negative enter time; op 1: rank 2 leaves before it entered; op 2 is healthy.
