@@ -88,7 +88,7 @@ def built_ring(n, kind, rng, n_channels):
     done = set(rng.choice(n, size=max(1, n // 5), replace=False).tolist()) if kind == "h2" else set()
     for p, r in enumerate(ranks):
         if p in skipped:
-            if p % 2 == 0 and n > 1:                                   # some of them are already past the op
+            if p % 2 == 0 and p != min(skipped):                       # some of them are already past the op
                 recs.append(dict(rank=int(r), comm=9, seq=3, t_enter=5000, t_exit=-1))
             continue
         recs.append(dict(rank=int(r), comm=9, seq=2, t_enter=4000, t_exit=(4100 if p in done else -1)))
