@@ -26,9 +26,11 @@ constexpr int WARP_N = 128;            // up to 128 ranks: one warp per group, b
 constexpr int MID_N = 1024;            // up to 1024 ranks: shared-memory bitonic sort, several groups per CTA
 constexpr int MID_THREADS = 256;
 constexpr int MID_ELEMS = 2048;        //   padded records per tile
-constexpr int LARGE_THREADS = 1024;    // above: one CTA walks a few consecutive groups, radix select
-constexpr int LARGE_SEQS = 8;
-constexpr int LARGE_MAXP = CCLD_MAX_COMM_SIZE / LARGE_THREADS;
+constexpr int LARGE_SEQS = 8;          // above: tiles of up to 8 consecutive op counters (as many as fit shared memory), radix select
+constexpr int LG_THREADS = 512;
+constexpr int LG_WARPS = LG_THREADS / 32;
+constexpr int LG_KEYS = 16;            //   (member, group) pairs a thread of the kernel holds at most
+constexpr u32 LG_BUDGET = 104 * 1024;  //   dynamic shared memory per CTA below which two CTAs fit one SM
 
 struct Params {
   i64 tbase_init_ns, m_max_ns, hang_ns;
@@ -124,10 +126,26 @@ enum { GU_RANK_TMIN = 0, GU_RANK_TMAX, GU_MAX_CHG, GU_RANK_MAX_CHG, GU_N_PRESENT
 __host__ __device__ inline u32 next_pow2(u32 n) { u32 p = 1; while (p < n) p <<= 1; return p; }
 __host__ __device__ inline u32 comm_class(u32 n) { return n <= SMALL_N ? 0u : (n <= WARP_N ? 1u : (n <= MID_N ? 2u : 3u)); }
 __host__ __device__ inline u32 mid_npad(u32 n) { u32 p = next_pow2(n); return p < 32 ? 32 : p; }
+// Communicators of more than MID_N ranks: G groups (consecutive op counters) are worked on side by side, their 32-bit
+// keys in shared memory next to the tile's per-member bandwidth sums, one histogram per group and the partial extrema.
+__host__ __device__ inline u32 large_npad(u32 n) { return (n + 31u) & ~31u; }
+__host__ __device__ inline u32 large_pitch(u32 n, u32 G) { return large_npad(n) + 32u / G; }    // lanes g, g + 1, ... of one member hit distinct banks
+__host__ __device__ inline size_t large_smem(u32 n, u32 G) {
+  return (size_t)8 * G * large_pitch(n, G)            // enter-time offsets and durations, u32 each, [G][pitch]
+       + (size_t)8 * large_npad(n)                    // per-member bandwidth sums
+       + (size_t)G * 256 * 4                          // one histogram per group
+       + (size_t)LG_WARPS * G * 40                    // per-warp partial extrema (LargePart)
+       + (size_t)G * 48;                              // per-group totals (LargeLead), select state
+}
+__host__ __device__ inline u32 large_g(u32 n) {
+  for (u32 G = LARGE_SEQS; G > 1; G >>= 1)
+    if (large_smem(n, G) <= LG_BUDGET && (u64)G * large_npad(n) <= (u64)LG_KEYS * LG_THREADS) return G;
+  return 1;
+}
 // op counters per work unit: a warp-tile (class 0) or a CTA tile (classes 1 to 3)
 __host__ __device__ inline u32 tile_seqs(u32 n) {
   u32 c = comm_class(n);
-  return c == 0 ? 32u : (c <= 2 ? MID_ELEMS / mid_npad(n) : (u32)LARGE_SEQS);
+  return c == 0 ? 32u : (c <= 2 ? MID_ELEMS / mid_npad(n) : large_g(n));
 }
 __host__ __device__ inline u32 ceil_div(u32 a, u32 b) { return (a + b - 1) / b; }
 // chunking of a fused-class communicator with n_seq op counters in a window of T chunks

@@ -82,7 +82,7 @@ struct TimerSlot { cudaEvent_t a[TIMER_PAIRS], b[TIMER_PAIRS]; int kind[TIMER_PA
 struct ccld_ctx {
   ccld_params params; Params dp; int device = 0; cudaStream_t stream = nullptr;
   std::vector<CommHost> comms; std::unordered_map<u32, u32> comm_idx;
-  bool finalized = false; u32 n_ranks = 0, max_n = 0, max_large_n = 0; u64 sum_n = 0;
+  bool finalized = false; u32 n_ranks = 0, max_n = 0, max_large_n = 0; u64 sum_n = 0; size_t large_smem = 0; u32 n_sms = 148;
   Block reg_blk, misc_blk; Registry reg; size_t stats_off = 0, stats_bytes = 0;
   const TreeRef* d_trees = nullptr; u32 n_trees = 0;     // tree communicators whose layers are known
   std::map<u32, WindowHost> windows;
@@ -245,7 +245,13 @@ int finalize_registry(ccld_ctx* ctx) {
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "scratch allocation failed");
 
   CK(cudaFuncSetAttribute(k_reduce_mid, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mid_smem_bytes(2 * WARP_N)));
-  if (max_large) CK(cudaFuncSetAttribute(k_reduce_large, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(16ull * max_large)));
+  if (max_large) {
+    size_t need = 0;                       // the largest tile layout among the registered communicators
+    for (auto& c : ctx->comms) if (c.ranks.size() > MID_N) need = std::max(need, large_smem((u32)c.ranks.size(), large_g((u32)c.ranks.size())));
+    ctx->large_smem = need;
+    CK(cudaFuncSetAttribute(k_reduce_large, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need));
+    CK(cudaFuncSetAttribute(k_reduce_large_deferred, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(16ull * max_large)));
+  }
   ctx->finalized = true;
   return CCLD_OK;
 }
@@ -284,6 +290,7 @@ int ccld_create(ccld_ctx** out, const ccld_params* params, int device, void* cud
   ccld_ctx* ctx = new (std::nothrow) ccld_ctx();
   if (!ctx) return CCLD_ERR_NOMEM;
   ctx->params = *params; ctx->device = device; ctx->stream = (cudaStream_t)cuda_stream;
+  { int sms = 0; if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) == cudaSuccess && sms > 0) ctx->n_sms = (u32)sms; }
   Params& d = ctx->dp;
   d.tbase_init_ns = params->tbase_init_ns; d.m_max_ns = params->m_max_ns; d.hang_ns = params->hang_ns; d.barrier_bytes = params->barrier_bytes;
   d.theta_slow_milli = params->theta_slow_milli; d.alpha_milli = params->alpha_milli; d.beta_milli = params->beta_milli;
@@ -494,7 +501,8 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   // groups the fused kernel may set aside for the deferred kernel: at most every group of the batch
   u64 total_groups = 0;
   for (u32 k = 0; k < B; ++k) total_groups += ctx->h_pinned[(size_t)k * T_COUNT + T_GROUPS];
-  const size_t o_defn = take(8), o_def = take(n_list[B_FCTA] ? total_groups * 8 : 0);
+  const size_t o_defn = take(16), o_def = take(n_list[B_FCTA] ? total_groups * 8 : 0),
+               o_def3 = take(n_list[B_T3] * (size_t)LARGE_SEQS * 8);          // likewise for the kernel of the largest communicators
   Block rb = ctx->pool.get(off, &e);
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "result allocation failed");
   auto res_blk = std::make_shared<Shared>(&ctx->pool, rb);
@@ -513,15 +521,21 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   PlanLists pl; pl.fcta = (FusedCta*)(rbase + o_fcta); pl.fwt = (WarpTile*)(rbase + o_fwt); pl.t2 = (Tile*)(rbase + o_t2); pl.t3 = (Tile*)(rbase + o_t3);
   { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, pl, 1); }
   if (cta > 0) { TimedLaunch tl(ts, 2, st); k_slot_scatter<<<(u32)cta, SCAT_THREADS, 0, st>>>(d_desc, d_cta0, B, ctx->reg); }
+  CK(cudaMemsetAsync(rbase + o_defn, 0, 16, st));
   if (n_list[B_FCTA]) {
     const DeferList dl{(u64*)(rbase + o_def), (u32*)(rbase + o_defn)};
-    CK(cudaMemsetAsync(rbase + o_defn, 0, 8, st));
     TimedLaunch tl(ts, 3, st);
     k_reduce_fused<<<(u32)n_list[B_FCTA], SMALL_SEQS, 0, st>>>(d_desc, pl.fcta, pl.fwt, (TileSum*)(rbase + o_fsum), ctx->reg, ctx->dp, dl);
     k_reduce_deferred<<<DEF_GRID, DEF_WARPS * 32, 0, st>>>(d_desc, dl, ctx->reg, ctx->dp, now_ns);
   }
   if (n_list[B_T2]) { TimedLaunch tl(ts, 4, st); k_reduce_mid<<<(u32)n_list[B_T2], MID_THREADS, mid_smem_bytes(2 * WARP_N), st>>>(d_desc, pl.t2, (TileSum*)(rbase + o_s2), ctx->reg, ctx->dp, now_ns); }
-  if (n_list[B_T3]) { TimedLaunch tl(ts, 5, st); k_reduce_large<<<(u32)n_list[B_T3], LARGE_THREADS, 16ull * ctx->max_large_n, st>>>(d_desc, pl.t3, (TileSum*)(rbase + o_s3), ctx->reg, ctx->dp, now_ns); }
+  if (n_list[B_T3]) {
+    const DeferList dl{(u64*)(rbase + o_def3), (u32*)(rbase + o_defn) + 2};
+    TimedLaunch tl(ts, 5, st);
+    const u32 grid = (u32)std::min<u64>(n_list[B_T3], 2ull * ctx->n_sms);      // persistent: two CTAs per SM take the tiles in turn
+    k_reduce_large<<<grid, LG_THREADS, ctx->large_smem, st>>>(d_desc, pl.t3, (u32)n_list[B_T3], (TileSum*)(rbase + o_s3), ctx->reg, ctx->dp, dl);
+    k_reduce_large_deferred<<<LARGE_DEF_GRID, LARGE_DEF_THREADS, 16ull * ctx->max_large_n, st>>>(d_desc, dl, ctx->reg, ctx->dp, now_ns);
+  }
   {
     TimedLaunch tl(ts, 6, st);
     k_window_rounds<<<dim3((nc + 3) / 4, B), 128, 0, st>>>(d_desc, ctx->reg);

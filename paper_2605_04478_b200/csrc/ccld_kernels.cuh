@@ -10,7 +10,8 @@
 //                   shuffle bitonic network); complete groups whose times fit 32-bit offsets
 //   k_reduce_deferred  the groups k_reduce_fused sets aside (incomplete, in flight, 64-bit spreads)
 //   k_reduce_mid    same, 129 <= n <= 1024 (shared-memory bitonic sort, several groups per CTA)
-//   k_reduce_large  same, n > 1024 (one CTA per group, radix select)
+//   k_reduce_large  same, n > 1024 (ccld_large.cuh: a CTA per tile of 8 op counters, several groups side by side, radix select)
+//   k_reduce_large_deferred  the groups k_reduce_large sets aside
 //   k_window_rounds Eq. 2 per (communicator, window): round counts, selected round, location candidates
 //   k_window_decide Eq. 1, 3, 4 per communicator, windows in order: baseline state, class, slow location
 //   k_hang_locate   hang decision tree over presence / completion / progress counters
@@ -543,6 +544,7 @@ __global__ void __launch_bounds__(SCAT_THREADS, 4) k_slot_scatter(const WinDesc*
 }  // namespace ccld
 
 #include "ccld_fused.cuh"
+#include "ccld_large.cuh"
 
 namespace ccld {
 
@@ -805,233 +807,6 @@ inline size_t mid_smem_bytes(u32 n_pad_min) {
   // cap = (MID_ELEMS / n_pad) * (n_pad + 1) is largest for the smallest n_pad
   size_t cap = (size_t)(MID_ELEMS / n_pad_min) * (n_pad_min + 1);
   return cap * (4 * 8 + 2 * 4 + 2) + 16 + (MID_ELEMS / n_pad_min) * sizeof(MidGroup);
-}
-
-// ------------------------------------------------------------------------------------------------
-// per-op reductions, n > 1024: one CTA per group; enter times and durations live in shared memory,
-// order statistics by most-significant-byte-first radix select
-// ------------------------------------------------------------------------------------------------
-// Reduction over the CTA (all threads call; blockDim.x a multiple of 32): warps reduce by shuffles, the first warp
-// reduces the warps' partial results the same way, everyone reads the result from s_red[0].
-template <class T, class Op>
-__device__ T block_reduce(T v, Op op, T* s_red /*[32]*/) {
-  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
-#pragma unroll
-  for (int d = 16; d > 0; d >>= 1) { T o = __shfl_xor_sync(0xFFFFFFFFu, v, d); v = op(v, o); }
-  __syncthreads();
-  if (lane == 0) s_red[wid] = v;
-  __syncthreads();
-  if (wid == 0) {
-    T x = lane < nw ? s_red[lane] : Op::identity();
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) { T o = __shfl_xor_sync(0xFFFFFFFFu, x, d); x = op(x, o); }
-    if (lane == 0) s_red[0] = x;
-  }
-  __syncthreads();
-  return s_red[0];
-}
-struct OpMinU64 { __device__ u64 operator()(u64 a, u64 b) const { return a < b ? a : b; } static __device__ u64 identity() { return U64_MAX_; } };
-struct OpMaxU64 { __device__ u64 operator()(u64 a, u64 b) const { return a > b ? a : b; } static __device__ u64 identity() { return 0; } };
-struct OpMaxI64 { __device__ i64 operator()(i64 a, i64 b) const { return a > b ? a : b; } static __device__ i64 identity() { return INT64_MIN; } };
-struct OpAddU32 { __device__ u32 operator()(u32 a, u32 b) const { return a + b; } static __device__ u32 identity() { return 0; } };
-struct OpOrU32 { __device__ u32 operator()(u32 a, u32 b) const { return a | b; } static __device__ u32 identity() { return 0; } };
-struct OpMinU32 { __device__ u32 operator()(u32 a, u32 b) const { return a < b ? a : b; } static __device__ u32 identity() { return NONE; } };
-
-// k-th smallest (0-based) of key(i), i < n; max_key bounds the keys. All threads of the CTA call it.
-template <class F>
-__device__ u64 radix_select(F key, u32 n, u32 k, u64 max_key, u32* hist /*[256]*/, u32* s_pick /*[2]*/) {
-  int top = max_key == 0 ? 0 : (63 - __clzll((long long)max_key)) >> 3;
-  u64 prefix = 0, mask = 0; u32 krem = k;
-  for (int b = top; b >= 0; --b) {
-    for (u32 i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
-    __syncthreads();
-    for (u32 i = threadIdx.x; i < n; i += blockDim.x) {
-      const u64 v = key(i);
-      if ((v & mask) == prefix) {
-        const u32 bin = (u32)(v >> (8 * b)) & 255u;
-        const u32 m = __match_any_sync(__activemask(), bin);       // one atomic per distinct bin in the warp
-        if ((threadIdx.x & 31) == (u32)(__ffs(m) - 1)) atomicAdd(&hist[bin], (u32)__popc(m));
-      }
-    }
-    __syncthreads();
-    if (threadIdx.x < 32) {
-      u32 loc[8], sum = 0;
-#pragma unroll
-      for (int q = 0; q < 8; ++q) { loc[q] = hist[threadIdx.x * 8 + q]; sum += loc[q]; }
-      u32 inc = sum;
-#pragma unroll
-      for (int d = 1; d < 32; d <<= 1) { u32 o = __shfl_up_sync(0xFFFFFFFFu, inc, d); if ((threadIdx.x & 31) >= (u32)d) inc += o; }
-      u32 ex = inc - sum;
-      if (krem >= ex && krem < inc) {
-        u32 cum = ex;
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          if (krem >= cum && krem < cum + loc[q]) { s_pick[0] = threadIdx.x * 8 + q; s_pick[1] = krem - cum; }
-          cum += loc[q];
-        }
-      }
-    }
-    __syncthreads();
-    prefix |= (u64)s_pick[0] << (8 * b); mask |= 0xFFull << (8 * b); krem = s_pick[1];
-    __syncthreads();
-  }
-  return prefix;
-}
-
-__global__ void __launch_bounds__(LARGE_THREADS) k_reduce_large(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles,
-                                                                 TileSum* __restrict__ sums, Registry R, Params P, i64 now) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
-  __shared__ u64 s_red64[32];
-  __shared__ u32 s_red32[32];
-  __shared__ u32 s_hist[256];
-  __shared__ u32 s_pick[2];
-  const Tile t = tiles[blockIdx.x];
-  const WinDesc& D = wd[t.w];
-  const u32 c = t.c, n = R.comm_n[c];
-  const RangeRow row = D.ranges[c];
-  const u32* mem = R.members + R.comm_moff[c];
-  u64* s_te = (u64*)smem_raw;
-  u64* s_du = s_te + n;
-  const u64 G = D.n_groups;
-  double bwacc[LARGE_MAXP];               // member p = threadIdx.x + q * LARGE_THREADS
-#pragma unroll
-  for (int q = 0; q < LARGE_MAXP; ++q) bwacc[q] = 0.0;
-  u32 n_bwc = 0, n_an_tile = 0;
-  u64 t_brng = 0; u32 t_bk = NONE;
-
-  for (u32 jg = 0; jg < t.count; ++jg) {
-    __syncthreads();
-    const u64 g = row.group0 + t.seq_off + jg, slot = row.slot0 + (u64)(t.seq_off + jg) * n;      // slot: flags, group-major
-    const u32 seq = row.seq_lo + t.seq_off + jg;
-    const u32* __restrict__ pm = D.perm + perm_at(row, t.seq_off + jg, 0);                          // member p at pm[p * n_seq]
-    const u64 pst = row.n_seq;
-    // pass 1: gather, presence, first present member
-    u32 npres = 0, first = NONE, stor = 0;
-    for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS) {
-      const u32 idx = pm[p * pst];
-      u64 te = 0, du = 0; u32 st = 0;
-      if (idx != NONE) {
-        const i64 x = D.t_enter[idx], y = D.t_exit[idx];
-        st = 1 | (y == -1 ? 2 : ((x < 0 || y < x) ? 4 : 0));
-        te = (u64)x; du = (u64)(y - x);
-        ++npres; first = first == NONE ? p : first;
-      }
-      stor |= st; s_te[p] = te; s_du[p] = du;
-    }
-    npres = block_reduce(npres, OpAddU32(), s_red32);
-    first = block_reduce(first, OpMinU32(), s_red32);
-    stor = block_reduce(stor, OpOrU32(), s_red32);
-    const bool have_first = first != NONE;
-    u64 gbytes = 0; u32 gop = 0;
-    if (have_first) { const u32 idx = pm[first * pst]; gbytes = D.bytes[idx]; gop = D.op[idx]; }
-    const bool inflight = stor & 2, bad_time = stor & 4, complete = npres == n && !inflight && !bad_time;
-    const bool barrier = have_first && gop == CCLD_OP_ALLREDUCE && gbytes < P.barrier_bytes;
-    // pass 2: op-set check, rate column, in-flight age, extrema
-    u32 mism = 0; i64 age = -1; u64 chk = 0;
-    u64 e_min = U64_MAX_, tmax = 0, tmin = U64_MAX_; i64 x_max = INT64_MIN;
-    for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS) {
-      const u32 idx = pm[p * pst];
-      if (idx == NONE) continue;
-      if (D.op[idx] != gop || D.bytes[idx] != gbytes) mism = 1;
-      u32 ch = 0;
-      if (D.send_chg != nullptr) { const u32 sc = D.send_chg[idx], rc = D.recv_chg[idx]; ch = sc > rc ? sc : rc; }
-      const u64 ck = ((u64)ch << 32) | (u64)(NONE - p); chk = ck > chk ? ck : chk;
-      const u64 te = s_te[p], du = s_du[p];
-      if (D.t_exit[idx] == -1) { const i64 ag = now - (i64)te; age = ag > age ? ag : age; }
-      e_min = te < e_min ? te : e_min; tmax = du > tmax ? du : tmax; tmin = du < tmin ? du : tmin;
-      const i64 tx = (i64)(te + du); x_max = tx > x_max ? tx : x_max;
-    }
-    mism = block_reduce(mism, OpOrU32(), s_red32);
-    age = block_reduce(age, OpMaxI64(), (i64*)s_red64);
-    chk = block_reduce(chk, OpMaxU64(), s_red64);
-    e_min = block_reduce(e_min, OpMinU64(), s_red64);
-    tmax = block_reduce(tmax, OpMaxU64(), s_red64);
-    tmin = block_reduce(tmin, OpMinU64(), s_red64);
-    x_max = block_reduce(x_max, OpMaxI64(), (i64*)s_red64);
-    u32 gfl = (mism ? CCLD_G_OPSET_MISMATCH : 0) | (barrier ? CCLD_G_BARRIER : 0) | (inflight ? CCLD_G_INFLIGHT : 0) |
-              (bad_time ? CCLD_G_BAD_TIME : 0) | (complete ? CCLD_G_COMPLETE : CCLD_G_INCOMPLETE);
-    const bool analysed = complete && !barrier && n >= P.min_group;
-    const bool hang = !complete && inflight && age > P.hang_ns && !barrier;
-    if (analysed) gfl |= CCLD_G_ANALYSED;
-    if (hang) gfl |= CCLD_G_HANG_ALERT;
-
-    if (!complete) {
-      for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS)
-        D.flags[slot + p] = pm[p * pst] == NONE ? (CCLD_F_NOT_ANALYSED | CCLD_F_MISSING) : CCLD_F_NOT_ANALYSED;
-      if (threadIdx.x == 0) {
-        if (hang) raise_alert(D, R.comm_id[c], seq, age);
-        for (int q = 0; q < GI_COUNT; ++q) D.gi64[(u64)q * G + g] = 0;
-        for (int q = 0; q < GU_COUNT; ++q) D.gu32[(u64)q * G + g] = 0;
-        D.gu32[(u64)GU_N_PRESENT * G + g] = npres; D.gu32[(u64)GU_GFLAGS * G + g] = gfl; D.gbw[g] = 0.0;
-        count_add(D.counters, C_INCOMPLETE, 1); count_add(D.counters, C_BARRIER, barrier); count_add(D.counters, C_MISMATCH, mism);
-        count_add(D.counters, C_PRESENT, npres);
-      }
-      continue;
-    }
-    // positions of the extrema: lowest ring position among equals
-    u32 pmax = NONE, pmin = NONE; u64 askew = 0;
-    for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS) {
-      if (s_du[p] == tmax && p < pmax) pmax = p;
-      if (s_du[p] == tmin && p < pmin) pmin = p;
-      const u64 sk = s_te[p] - e_min; askew = sk > askew ? sk : askew;
-    }
-    pmax = block_reduce(pmax, OpMinU32(), s_red32);
-    pmin = block_reduce(pmin, OpMinU32(), s_red32);
-    askew = block_reduce(askew, OpMaxU64(), s_red64);
-    const i64 span = x_max - (i64)e_min;
-    double num, den; bus_factor(gop, n, &num, &den);
-    const double bn = (double)gbytes * num;
-    if (!barrier) {
-      ++n_bwc; n_an_tile += analysed ? 1u : 0u;
-      best_merge(t_brng, t_bk, tmax - tmin, t.seq_off + jg);
-#pragma unroll
-      for (int q = 0; q < LARGE_MAXP; ++q) { const u32 p = threadIdx.x + q * LARGE_THREADS; if (p < n) bwacc[q] += busbw(bn, den, (i64)s_du[p]); }
-    }
-
-    u64 med_s = 0, mad_s = 0, med_d = 0, mad_d = 0; u32 n_fs = 0, n_fd = 0;
-    if (analysed) {
-      const u32 k = (n - 1) >> 1;
-      med_s = radix_select([&](u32 i) { return s_te[i] - e_min; }, n, k, askew, s_hist, s_pick);
-      { const u64 m = med_s, dmax = m > askew - m ? m : askew - m;
-        mad_s = radix_select([&](u32 i) { return absdiff(s_te[i] - e_min, m); }, n, k, dmax, s_hist, s_pick); }
-      med_d = tmin + radix_select([&](u32 i) { return s_du[i] - tmin; }, n, k, tmax - tmin, s_hist, s_pick);
-      { const u64 m = med_d, dmax = (m - tmin) > (tmax - m) ? (m - tmin) : (tmax - m);
-        mad_d = radix_select([&](u32 i) { return absdiff(s_du[i], m); }, n, k, dmax, s_hist, s_pick); }
-      for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS) {
-        const u64 sk = s_te[p] - e_min, du = s_du[p];
-        const bool so = mul_gt(absdiff(sk, med_s), 1000u, mad_s, P.k_milli), sh = sk > med_s;
-        const bool dq = mul_gt(absdiff(du, med_d), 1000u, mad_d, P.k_milli), dh = du > med_d;
-        D.flags[slot + p] = (so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0);
-        if (so) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p] * 4 + (sh ? 0 : 1)], 1u); }
-        if (dq) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p] * 4 + (dh ? 2 : 3)], 1u); }
-      }
-      n_fs = block_reduce(n_fs, OpAddU32(), s_red32);
-      n_fd = block_reduce(n_fd, OpAddU32(), s_red32);
-    } else {
-      for (u32 p = threadIdx.x; p < n; p += LARGE_THREADS) D.flags[slot + p] = CCLD_F_NOT_ANALYSED;
-    }
-    if (threadIdx.x == 0) {
-      D.gi64[(u64)GI_E_MIN * G + g] = (i64)e_min; D.gi64[(u64)GI_ARRIVAL_SKEW * G + g] = (i64)askew;
-      D.gi64[(u64)GI_T_MAX * G + g] = (i64)tmax; D.gi64[(u64)GI_T_MIN * G + g] = (i64)tmin; D.gi64[(u64)GI_SPAN * G + g] = span;
-      D.gi64[(u64)GI_MED_SKEW * G + g] = (i64)med_s; D.gi64[(u64)GI_MAD_SKEW * G + g] = (i64)mad_s;
-      D.gi64[(u64)GI_MED_DUR * G + g] = (i64)med_d; D.gi64[(u64)GI_MAD_DUR * G + g] = (i64)mad_d;
-      D.gu32[(u64)GU_RANK_TMIN * G + g] = mem[pmin]; D.gu32[(u64)GU_RANK_TMAX * G + g] = mem[pmax];
-      D.gu32[(u64)GU_MAX_CHG * G + g] = (u32)(chk >> 32); D.gu32[(u64)GU_RANK_MAX_CHG * G + g] = mem[NONE - (u32)chk];
-      D.gu32[(u64)GU_N_PRESENT * G + g] = npres; D.gu32[(u64)GU_GFLAGS * G + g] = gfl;
-      D.gbw[g] = busbw(bn, den, span);
-      count_add(D.counters, C_COMPLETE, 1); count_add(D.counters, C_BARRIER, barrier); count_add(D.counters, C_ANALYSED, analysed);
-      count_add(D.counters, C_MISMATCH, mism); count_add(D.counters, C_PRESENT, npres);
-      count_add(D.counters, C_FLAG_SKEW, n_fs); count_add(D.counters, C_FLAG_DUR, n_fd);
-    }
-  }  // groups of the tile
-  if (threadIdx.x == 0) { TileSum ts; ts.best_rng = t_brng; ts.best_k = t_bk; ts.n_rounds = n_bwc; ts.n_an = n_an_tile; ts.pad = 0; sums[blockIdx.x] = ts; }
-  if (n_bwc) {
-#pragma unroll
-    for (int q = 0; q < LARGE_MAXP; ++q) {
-      const u32 p = threadIdx.x + q * LARGE_THREADS;
-      if (p < n) { atomicAdd(&R.bw_sum[mem[p]], bwacc[q]); atomicAdd(&R.bw_cnt[mem[p]], n_bwc); }
-    }
-  }
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -1,0 +1,517 @@
+// Per-op reductions, median / MAD, flags and votes for communicators of more than 1,024 ranks (sm_100a).
+//
+//   k_reduce_large           the common case: every member reported, nothing in flight, all times of a group within
+//                            2^31 ns of its first member's enter time. A tile is G consecutive op counters of one
+//                            communicator (G = 8, 4, 2 or 1: as many as fit the shared-memory budget that still lets two
+//                            CTAs share an SM). Lanes run along the op counter first: the G record indices of one member
+//                            are neighbours in the member-major permutation, and in a rank-major upload so are the
+//                            records themselves, so the gathers of a warp touch 32 / G short contiguous stretches.
+//                            Enter-time offsets and durations of the G groups wait in shared memory as 32-bit keys;
+//                            every CTA-wide step - the extrema, the four radix selects, the flag pass - runs once for
+//                            all G groups side by side, so a tile costs the barriers of one group. During a select a
+//                            thread keeps its keys in registers. The grid is persistent: CTA b takes tiles b, b + grid,
+//                            ..., so CTAs that run at the same time work on neighbouring op counters (what one fetches
+//                            of a 64-byte line, its neighbours find in L2) and a CTA's tiles of one communicator and
+//                            window add their per-member bandwidth sums in shared memory before they go to global memory.
+//   k_reduce_large_deferred  the groups the fast kernel sets aside (a missing member, a record in flight, invalid
+//                            times, spreads beyond 32 bits): one CTA per listed group, 64-bit throughout, hang alerts.
+#pragma once
+#include "ccld_device.cuh"
+
+namespace ccld {
+
+struct LargePart { u64 kmax, kmin, ck; u32 emin, emax, xmax, bits; };      // bits: 1 = some record disqualifies the group, 2 = op set differs
+struct LargeLead { u64 brng; u32 bk, rounds, an, def, pad; };
+static_assert(sizeof(LargePart) == 40 && sizeof(LargeLead) == 32, "large_smem() counts these sizes");
+
+__device__ __forceinline__ int top_byte(u32 bound) { return bound == 0 ? 0 : (31 - __clz(bound)) >> 3; }
+
+// The k-th smallest (0-based) of a group's keys, for every group of the tile at once. A thread holds up to LG_KEYS keys
+// of its own group lane g in registers (bit q of `have` says whether slot q holds one); `act` says whether the group takes
+// part. Digits of 8 bits, most significant first, starting at byte `top` (the same for all groups). A thread counts the
+// keys that share the digit of its first candidate itself and adds them once - in the passes over high bytes nearly all
+// keys of a group agree - and adds the others one by one. Histograms must be zero on entry and are zero again on
+// return. All threads of the CTA call it.
+__device__ __forceinline__ u32 large_select(const u32 (&v)[LG_KEYS], u32 have, bool act, u32 k, int top, u32 G, u32 g,
+                                            u32* __restrict__ s_hist, u32* __restrict__ s_pick, u32* __restrict__ s_krem) {
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  if (threadIdx.x < G) s_krem[threadIdx.x] = k;
+  u32 prefix = 0, mask = 0;
+  u32* __restrict__ hist = s_hist + g * 256;
+  for (int b = top; b >= 0; --b) {
+    const u32 sh = 8u * (u32)b;
+    if (act) {
+      u32 cm = 0;
+#pragma unroll
+      for (int q = 0; q < LG_KEYS; ++q) cm |= ((v[q] & mask) == prefix ? 1u : 0u) << q;
+      cm &= have;
+      if (cm) {
+        u32 d0 = 0;
+#pragma unroll
+        for (int q = LG_KEYS - 1; q >= 0; --q) d0 = (cm >> q) & 1u ? (v[q] >> sh) & 255u : d0;      // digit of the first candidate
+        u32 c0 = 0;
+#pragma unroll
+        for (int q = 0; q < LG_KEYS; ++q) {
+          const u32 d = (v[q] >> sh) & 255u;
+          if ((cm >> q) & 1u) { if (d == d0) ++c0; else atomicAdd(&hist[d], 1u); }
+        }
+        atomicAdd(&hist[d0], c0);
+      }
+    }
+    __syncthreads();
+    if (wid < G) {                                                               // warp w scans and clears group w's histogram
+      u32 loc[8], sum = 0;
+      const u32 kr = s_krem[wid];
+#pragma unroll
+      for (int q = 0; q < 8; ++q) { loc[q] = s_hist[wid * 256 + lane * 8 + q]; sum += loc[q]; s_hist[wid * 256 + lane * 8 + q] = 0; }
+      u32 inc = sum;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) { const u32 o = __shfl_up_sync(0xFFFFFFFFu, inc, d); if (lane >= (u32)d) inc += o; }
+      const u32 ex = inc - sum;
+      if (kr >= ex && kr < inc) {
+        u32 cum = ex;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          if (kr >= cum && kr < cum + loc[q]) { s_pick[wid] = lane * 8 + q; s_krem[wid] = kr - cum; }
+          cum += loc[q];
+        }
+      }
+    }
+    __syncthreads();
+    prefix |= s_pick[g] << sh; mask |= 0xFFu << sh;
+  }
+  return prefix;
+}
+
+__global__ void __launch_bounds__(LG_THREADS, 2) k_reduce_large(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles, u32 n_tiles,
+                                                                 TileSum* __restrict__ sums, Registry R, Params P, DeferList DL) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ u32 s_cnt[SC_COUNT];
+  __shared__ u32 s_bound[2][LARGE_SEQS];
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  u32 cur_w = NONE, cur_c = NONE, cur_rounds = 0;            // whose bandwidth sums shared memory holds
+  const u32* cur_mem = nullptr; u32 cur_n = 0;
+  double* s_bw = nullptr;
+
+  for (u32 ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
+    const Tile t = tiles[ti];
+    const WinDesc& D = wd[t.w];
+    const u32 c = t.c, n = R.comm_n[c];
+    const RangeRow row = D.ranges[c];
+    const u32* __restrict__ mem = R.members + R.comm_moff[c];
+    const u32 n_pad = large_npad(n), G = large_g(n), pitch = large_pitch(n, G), lgG = 31 - __clz(G);
+    u32* s_sk = (u32*)smem_raw;                               // enter time minus (first member's enter time - 2^31)
+    u32* s_du = s_sk + (size_t)G * pitch;                     // duration
+    double* bw_here = (double*)(s_du + (size_t)G * pitch);
+    u32* s_hist = (u32*)(bw_here + n_pad);
+    LargePart* s_part = (LargePart*)(s_hist + G * 256);
+    LargeLead* s_lead = (LargeLead*)(s_part + LG_WARPS * G);
+    u32* s_pick = (u32*)(s_lead + G);
+    u32* s_krem = s_pick + G;
+    const u32 g = threadIdx.x & (G - 1), pl = threadIdx.x >> lgG, MP = LG_THREADS >> lgG;
+    const bool lead = pl == 0;                                // threads 0 .. G-1: one per group lane
+
+    __syncthreads();                                          // the previous tile is done with shared memory
+    if (t.w != cur_w || c != cur_c) {
+      // another communicator or window: what shared memory holds goes out, and the layout may change
+      if (cur_rounds) for (u32 p = threadIdx.x; p < cur_n; p += LG_THREADS) { atomicAdd(&R.bw_sum[cur_mem[p]], s_bw[p]); atomicAdd(&R.bw_cnt[cur_mem[p]], cur_rounds); }
+      __syncthreads();
+      cur_w = t.w; cur_c = c; cur_rounds = 0; cur_mem = mem; cur_n = n; s_bw = bw_here;
+      for (u32 p = threadIdx.x; p < n_pad; p += LG_THREADS) s_bw[p] = 0.0;
+      for (u32 i = threadIdx.x; i < G * 256; i += LG_THREADS) s_hist[i] = 0;
+    }
+    if (threadIdx.x < SC_COUNT) s_cnt[threadIdx.x] = 0;
+    const u32* __restrict__ perm = D.perm + row.slot0;
+    const i64* __restrict__ c_te = D.t_enter; const i64* __restrict__ c_tx = D.t_exit;
+    const u64* __restrict__ c_by = D.bytes; const u8* __restrict__ c_op = D.op;
+    const u32* __restrict__ c_sc = D.send_chg; const u32* __restrict__ c_rc = D.recv_chg;
+    const u64 G_all = D.n_groups;
+    const bool gvalid = g < t.count;
+    const u32 so = t.seq_off + (gvalid ? g : 0u);             // op-counter offset of my group inside the range
+
+    // ---- gather: the group's first member gives the time base and the op set (every thread of the group lane loads it:
+    //      one address per lane group, served by one transaction) ----
+    u32 bits = 0;
+    i64 te0 = 0; u64 by0 = 0; u32 op0 = 0;
+    {
+      const u32 i0 = gvalid ? __ldg(perm + so) : NONE;
+      if (i0 != NONE) { te0 = c_te[i0]; by0 = c_by[i0]; op0 = c_op[i0]; } else bits = 1;
+    }
+    const u64 base = (u64)te0 - 0x80000000ull;
+    u32 emin = 0xFFFFFFFFu, emax = 0, xmax = 0; u64 kmax = 0, kmin = U64_MAX_, ck = 0;
+    for (u32 p0 = pl; p0 < n; p0 += 4 * MP) {
+      u32 idx[4]; i64 x[4], y[4]; u64 by[4]; u32 op[4], ch[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) { const u32 p = p0 + q * MP; idx[q] = (gvalid && p < n) ? __ldg(perm + (u64)p * row.n_seq + so) : NONE; }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const u32 ix = idx[q] == NONE ? 0u : idx[q];
+        x[q] = c_te[ix]; y[q] = c_tx[ix]; by[q] = c_by[ix]; op[q] = c_op[ix]; ch[q] = 0;
+        if (c_sc != nullptr) { const u32 sc = c_sc[ix], rc = c_rc[ix]; ch[q] = sc > rc ? sc : rc; }
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const u32 p = p0 + q * MP;
+        if (p < n) {
+          u32 a_lo = 0, d = 0;
+          if (idx[q] == NONE) { if (gvalid) bits |= 1; }
+          else {
+            const u64 ra = (u64)x[q] - base, rb = (u64)y[q] - base;
+            a_lo = (u32)ra; const u32 b_lo = (u32)rb; d = b_lo - a_lo;
+            if (((ra | rb) >> 32) != 0 || (x[q] | y[q]) < 0 || b_lo < a_lo) bits |= 1;     // beyond 32 bits, negative or in flight, exit before enter
+            if (op[q] != op0 || by[q] != by0) bits |= 2;
+            emin = min(emin, a_lo); emax = max(emax, a_lo); xmax = max(xmax, b_lo);
+            const u64 k1 = ((u64)d << 32) | (u64)(NONE - p); kmax = k1 > kmax ? k1 : kmax;   // longest, then the lowest position
+            const u64 k2 = ((u64)d << 32) | (u64)p; kmin = k2 < kmin ? k2 : kmin;            // shortest, then the lowest position
+            const u64 k3 = ((u64)ch[q] << 32) | (u64)(NONE - p); ck = k3 > ck ? k3 : ck;     // most changes, then the lowest position
+          }
+          s_sk[g * pitch + p] = a_lo; s_du[g * pitch + p] = d;
+        }
+      }
+    }
+    // ---- extrema of the G groups: lanes of one group lane meet by shuffles, warps through shared memory ----
+    for (u32 h = G; h < 32; h <<= 1) {
+      emin = min(emin, __shfl_xor_sync(0xFFFFFFFFu, emin, h)); emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, h));
+      xmax = max(xmax, __shfl_xor_sync(0xFFFFFFFFu, xmax, h)); bits |= __shfl_xor_sync(0xFFFFFFFFu, bits, h);
+      const u64 a = shfl_xor64(kmax, h); kmax = a > kmax ? a : kmax;
+      const u64 b = shfl_xor64(kmin, h); kmin = b < kmin ? b : kmin;
+      const u64 e = shfl_xor64(ck, h); ck = e > ck ? e : ck;
+    }
+    if (lane < G) { LargePart x; x.kmax = kmax; x.kmin = kmin; x.ck = ck; x.emin = emin; x.emax = emax; x.xmax = xmax; x.bits = bits; s_part[wid * G + lane] = x; }
+    __syncthreads();
+#pragma unroll 4
+    for (u32 w = 0; w < LG_WARPS; ++w) {
+      const LargePart x = s_part[w * G + g];
+      emin = min(emin, x.emin); emax = max(emax, x.emax); xmax = max(xmax, x.xmax); bits |= x.bits;
+      kmax = x.kmax > kmax ? x.kmax : kmax; kmin = x.kmin < kmin ? x.kmin : kmin; ck = x.ck > ck ? x.ck : ck;
+    }
+    const bool gok = gvalid && !(bits & 1);
+    const u32 tmx = (u32)(kmax >> 32), tmn = (u32)(kmin >> 32);
+    const bool barrier = op0 == CCLD_OP_ALLREDUCE && by0 < P.barrier_bytes;
+    const bool analysed = gok && !barrier && n >= P.min_group;
+    double num, den; bus_factor(op0, n, &num, &den);
+    const double bn = (double)by0 * num;
+    if (lead) {
+      s_bound[0][g] = analysed ? emax - emin : 0u; s_bound[1][g] = analysed ? tmx - tmn : 0u;
+      LargeLead mine = {0, NONE, 0, 0, 0, 0};
+      if (gvalid && !gok) {                                   // set aside for the 64-bit kernel
+        const u32 e = atomicAdd(DL.count, 1u);
+        DL.entries[e] = ((u64)t.w << 32) | (u64)(row.group0 + so);
+        mine.def = 1;
+      }
+      if (gok) {
+        // everything of the per-op row that needs no order statistic goes out now, so that it occupies no registers during the selects
+        const u64 gi_ = row.group0 + so;
+        i64* __restrict__ gi = D.gi64 + gi_; u32* __restrict__ gu = D.gu32 + gi_;
+        const u32 span = xmax - emin;
+        gi[(u64)GI_E_MIN * G_all] = (i64)(base + emin); gi[(u64)GI_ARRIVAL_SKEW * G_all] = (i64)(u64)(emax - emin);
+        gi[(u64)GI_T_MAX * G_all] = (i64)(u64)tmx; gi[(u64)GI_T_MIN * G_all] = (i64)(u64)tmn; gi[(u64)GI_SPAN * G_all] = (i64)(u64)span;
+        gu[(u64)GU_RANK_TMIN * G_all] = mem[(u32)kmin]; gu[(u64)GU_RANK_TMAX * G_all] = mem[NONE - (u32)kmax];
+        gu[(u64)GU_MAX_CHG * G_all] = (u32)(ck >> 32); gu[(u64)GU_RANK_MAX_CHG * G_all] = mem[NONE - (u32)ck];
+        gu[(u64)GU_N_PRESENT * G_all] = n;
+        const bool mismatch = (bits & 2) != 0;
+        gu[(u64)GU_GFLAGS * G_all] = CCLD_G_COMPLETE | (barrier ? CCLD_G_BARRIER : 0) | (mismatch ? CCLD_G_OPSET_MISMATCH : 0) | (analysed ? CCLD_G_ANALYSED : 0);
+        D.gbw[gi_] = span ? bn * rcp_newton((double)span * den) : 0.0;
+        atomicAdd(&s_cnt[SC_COMP], 1u); atomicAdd(&s_cnt[SC_PRES], n);
+        if (barrier) atomicAdd(&s_cnt[SC_BAR], 1u);
+        if (analysed) { atomicAdd(&s_cnt[SC_AN], 1u); mine.an = 1; }
+        if (mismatch) atomicAdd(&s_cnt[SC_MIS], 1u);
+        if (!barrier) { mine.rounds = 1; mine.brng = (u64)(tmx - tmn); mine.bk = so; }
+      }
+      s_lead[g] = mine;
+    }
+    __syncthreads();
+    u32 bs = 0, bd = 0;
+    for (u32 q = 0; q < G; ++q) { bs = max(bs, s_bound[0][q]); bd = max(bd, s_bound[1][q]); }
+
+    // ---- order statistics, all groups of the tile side by side; a thread's keys sit in registers during a select ----
+    u32 ms = 0, ds = 0, md = 0, dm = 0;
+    u32 have = 0;
+#pragma unroll
+    for (int q = 0; q < LG_KEYS; ++q) have |= (pl + (u32)q * MP < n ? 1u : 0u) << q;
+    if (__syncthreads_or(analysed)) {
+      const u32 k = (n - 1) >> 1;
+      u32 v[LG_KEYS];
+#pragma unroll
+      for (int q = 0; q < LG_KEYS; ++q) v[q] = (have >> q) & 1u ? s_sk[g * pitch + pl + (u32)q * MP] - emin : 0u;
+      ms = large_select(v, have, analysed, k, top_byte(bs), G, g, s_hist, s_pick, s_krem);
+#pragma unroll
+      for (int q = 0; q < LG_KEYS; ++q) v[q] = __usad(v[q], ms, 0u);
+      ds = large_select(v, have, analysed, k, top_byte(bs), G, g, s_hist, s_pick, s_krem);
+#pragma unroll
+      for (int q = 0; q < LG_KEYS; ++q) v[q] = (have >> q) & 1u ? s_du[g * pitch + pl + (u32)q * MP] - tmn : 0u;
+      md = large_select(v, have, analysed, k, top_byte(bd), G, g, s_hist, s_pick, s_krem);
+#pragma unroll
+      for (int q = 0; q < LG_KEYS; ++q) v[q] = __usad(v[q], md, 0u);
+      dm = large_select(v, have, analysed, k, top_byte(bd), G, g, s_hist, s_pick, s_krem);
+      if (!analysed) { ms = ds = md = dm = 0; }
+    }
+
+    // ---- flags, votes, per-member bandwidth ----
+    u32 n_fs = 0, n_fd = 0;
+    {
+      const u64 ts = (u64)ds * P.k_milli, td = (u64)dm * P.k_milli;          // |x - med| * 1000 > k * MAD: both sides below 2^64
+      u8* __restrict__ fp = D.flags + row.slot0 + (u64)so * n;
+      for (u32 p0 = 0; p0 < n; p0 += MP) {                                   // the same trip count for every thread: shuffles inside
+        const u32 p = p0 + pl;
+        double bwv = 0.0;
+        if (gok && p < n) {
+          const u32 d = s_du[g * pitch + p];
+          u32 f = CCLD_F_NOT_ANALYSED;
+          if (analysed) {
+            const u32 skw = s_sk[g * pitch + p] - emin, dd = d - tmn;
+            const bool so_ = (u64)__usad(skw, ms, 0u) * 1000u > ts, shi = skw > ms;
+            const bool dq = (u64)__usad(dd, md, 0u) * 1000u > td, dhi = dd > md;
+            f = (so_ ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (shi ? CCLD_F_SKEW_HI : 0) | (dhi ? CCLD_F_DUR_HI : 0);
+            if (so_) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p] * 4 + (shi ? 0 : 1)], 1u); }
+            if (dq) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p] * 4 + (dhi ? 2 : 3)], 1u); }
+          }
+          fp[p] = (u8)f;
+          if (!barrier && d != 0) bwv = bn * rcp_newton1((double)d * den);
+        }
+        for (u32 h = 1; h < G; h <<= 1) bwv += __shfl_xor_sync(0xFFFFFFFFu, bwv, h);   // the G group lanes of member p are neighbours
+        if (g == 0 && p < n) s_bw[p] += bwv;
+      }
+    }
+    n_fs = __reduce_add_sync(0xFFFFFFFFu, n_fs); n_fd = __reduce_add_sync(0xFFFFFFFFu, n_fd);
+    if (lane == 0) { if (n_fs) atomicAdd(&s_cnt[SC_FS], n_fs); if (n_fd) atomicAdd(&s_cnt[SC_FD], n_fd); }
+    if (lead && gok) {
+      i64* __restrict__ gi = D.gi64 + row.group0 + so;
+      gi[(u64)GI_MED_SKEW * G_all] = (i64)(u64)ms; gi[(u64)GI_MAD_SKEW * G_all] = (i64)(u64)ds;
+      gi[(u64)GI_MED_DUR * G_all] = analysed ? (i64)((u64)tmn + md) : 0; gi[(u64)GI_MAD_DUR * G_all] = (i64)(u64)dm;
+    }
+    __syncthreads();
+    for (u32 q = 0; q < G; ++q) cur_rounds += s_lead[q].rounds;
+    if (threadIdx.x == 0) {
+      TileSum ts; ts.best_rng = 0; ts.best_k = NONE; ts.n_rounds = 0; ts.n_an = 0; ts.pad = 0;
+      for (u32 q = 0; q < G; ++q) { best_merge(ts.best_rng, ts.best_k, s_lead[q].brng, s_lead[q].bk); ts.n_rounds += s_lead[q].rounds; ts.n_an += s_lead[q].an; ts.pad += s_lead[q].def; }
+      sums[ti] = ts;
+      count_add(D.counters, C_COMPLETE, s_cnt[SC_COMP]); count_add(D.counters, C_BARRIER, s_cnt[SC_BAR]); count_add(D.counters, C_ANALYSED, s_cnt[SC_AN]);
+      count_add(D.counters, C_MISMATCH, s_cnt[SC_MIS]); count_add(D.counters, C_PRESENT, s_cnt[SC_PRES]);
+      count_add(D.counters, C_FLAG_SKEW, s_cnt[SC_FS]); count_add(D.counters, C_FLAG_DUR, s_cnt[SC_FD]);
+    }
+  }  // tiles of this CTA
+  __syncthreads();
+  if (cur_rounds) for (u32 p = threadIdx.x; p < cur_n; p += LG_THREADS) { atomicAdd(&R.bw_sum[cur_mem[p]], s_bw[p]); atomicAdd(&R.bw_cnt[cur_mem[p]], cur_rounds); }
+}
+
+// ------------------------------------------------------------------------------------------------
+// the groups k_reduce_large set aside: one CTA per listed group; enter times and durations live in
+// shared memory as 64-bit values, order statistics by most-significant-byte-first radix select
+// ------------------------------------------------------------------------------------------------
+constexpr int LARGE_DEF_THREADS = 1024;
+constexpr int LARGE_DEF_GRID = 148;         // grid-stride over the list: one CTA per SM of a B200
+
+// Reduction over the CTA (all threads call; blockDim.x a multiple of 32): warps reduce by shuffles, the first warp
+// reduces the warps' partial results the same way, everyone reads the result from s_red[0].
+template <class T, class Op>
+__device__ T block_reduce(T v, Op op, T* s_red /*[32]*/) {
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
+#pragma unroll
+  for (int d = 16; d > 0; d >>= 1) { T o = __shfl_xor_sync(0xFFFFFFFFu, v, d); v = op(v, o); }
+  __syncthreads();
+  if (lane == 0) s_red[wid] = v;
+  __syncthreads();
+  if (wid == 0) {
+    T x = lane < nw ? s_red[lane] : Op::identity();
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) { T o = __shfl_xor_sync(0xFFFFFFFFu, x, d); x = op(x, o); }
+    if (lane == 0) s_red[0] = x;
+  }
+  __syncthreads();
+  return s_red[0];
+}
+struct OpMinU64 { __device__ u64 operator()(u64 a, u64 b) const { return a < b ? a : b; } static __device__ u64 identity() { return U64_MAX_; } };
+struct OpMaxU64 { __device__ u64 operator()(u64 a, u64 b) const { return a > b ? a : b; } static __device__ u64 identity() { return 0; } };
+struct OpMaxI64 { __device__ i64 operator()(i64 a, i64 b) const { return a > b ? a : b; } static __device__ i64 identity() { return INT64_MIN; } };
+struct OpAddU32 { __device__ u32 operator()(u32 a, u32 b) const { return a + b; } static __device__ u32 identity() { return 0; } };
+struct OpOrU32 { __device__ u32 operator()(u32 a, u32 b) const { return a | b; } static __device__ u32 identity() { return 0; } };
+struct OpMinU32 { __device__ u32 operator()(u32 a, u32 b) const { return a < b ? a : b; } static __device__ u32 identity() { return NONE; } };
+
+// k-th smallest (0-based) of key(i), i < n; max_key bounds the keys. All threads of the CTA call it.
+template <class F>
+__device__ u64 radix_select(F key, u32 n, u32 k, u64 max_key, u32* hist /*[256]*/, u32* s_pick /*[2]*/) {
+  int top = max_key == 0 ? 0 : (63 - __clzll((long long)max_key)) >> 3;
+  u64 prefix = 0, mask = 0; u32 krem = k;
+  for (int b = top; b >= 0; --b) {
+    for (u32 i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
+    __syncthreads();
+    for (u32 i = threadIdx.x; i < n; i += blockDim.x) {
+      const u64 v = key(i);
+      if ((v & mask) == prefix) {
+        const u32 bin = (u32)(v >> (8 * b)) & 255u;
+        const u32 m = __match_any_sync(__activemask(), bin);       // one atomic per distinct bin in the warp
+        if ((threadIdx.x & 31) == (u32)(__ffs(m) - 1)) atomicAdd(&hist[bin], (u32)__popc(m));
+      }
+    }
+    __syncthreads();
+    if (threadIdx.x < 32) {
+      u32 loc[8], sum = 0;
+#pragma unroll
+      for (int q = 0; q < 8; ++q) { loc[q] = hist[threadIdx.x * 8 + q]; sum += loc[q]; }
+      u32 inc = sum;
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) { u32 o = __shfl_up_sync(0xFFFFFFFFu, inc, d); if ((threadIdx.x & 31) >= (u32)d) inc += o; }
+      u32 ex = inc - sum;
+      if (krem >= ex && krem < inc) {
+        u32 cum = ex;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          if (krem >= cum && krem < cum + loc[q]) { s_pick[0] = threadIdx.x * 8 + q; s_pick[1] = krem - cum; }
+          cum += loc[q];
+        }
+      }
+    }
+    __syncthreads();
+    prefix |= (u64)s_pick[0] << (8 * b); mask |= 0xFFull << (8 * b); krem = s_pick[1];
+    __syncthreads();
+  }
+  return prefix;
+}
+
+__global__ void __launch_bounds__(LARGE_DEF_THREADS) k_reduce_large_deferred(const WinDesc* __restrict__ wd, DeferList DL, Registry R, Params P, i64 now) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  __shared__ u64 s_red64[32];
+  __shared__ u32 s_red32[32];
+  __shared__ u32 s_hist[256];
+  __shared__ u32 s_pick[2];
+  const u32 total = *DL.count;
+  for (u32 e = blockIdx.x; e < total; e += gridDim.x) {
+    const u64 ent = DL.entries[e];
+    const WinDesc& D = wd[(u32)(ent >> 32)];
+    const u64 g = (u32)ent;
+    u32 c;
+    { // owner: the last communicator whose first group is <= g (communicators without groups share their successor's start)
+      u32 lo = 0, hi = R.n_comms - 1;
+      while (lo < hi) { const u32 mid = (lo + hi + 1) >> 1; if (D.ranges[mid].group0 <= g) lo = mid; else hi = mid - 1; }
+      c = lo;
+    }
+    const RangeRow row = D.ranges[c];
+    const u32 n = row.n, so = (u32)(g - row.group0);
+    const u32* mem = R.members + R.comm_moff[c];
+    u64* s_te = (u64*)smem_raw;
+    u64* s_du = s_te + n;
+    const u64 G = D.n_groups;
+    __syncthreads();
+    const u64 slot = row.slot0 + (u64)so * n;                      // flags, group-major
+    const u32 seq = row.seq_lo + so;
+    const u32* __restrict__ pm = D.perm + perm_at(row, so, 0);     // member p at pm[p * n_seq]
+    const u64 pst = row.n_seq;
+    // pass 1: gather, presence, first present member
+    u32 npres = 0, first = NONE, stor = 0;
+    for (u32 p = threadIdx.x; p < n; p += LARGE_DEF_THREADS) {
+      const u32 idx = pm[p * pst];
+      u64 te = 0, du = 0; u32 st = 0;
+      if (idx != NONE) {
+        const i64 x = D.t_enter[idx], y = D.t_exit[idx];
+        st = 1 | (y == -1 ? 2 : ((x < 0 || y < x) ? 4 : 0));
+        te = (u64)x; du = (u64)(y - x);
+        ++npres; first = first == NONE ? p : first;
+      }
+      stor |= st; s_te[p] = te; s_du[p] = du;
+    }
+    npres = block_reduce(npres, OpAddU32(), s_red32);
+    first = block_reduce(first, OpMinU32(), s_red32);
+    stor = block_reduce(stor, OpOrU32(), s_red32);
+    const bool have_first = first != NONE;
+    u64 gbytes = 0; u32 gop = 0;
+    if (have_first) { const u32 idx = pm[first * pst]; gbytes = D.bytes[idx]; gop = D.op[idx]; }
+    const bool inflight = stor & 2, bad_time = stor & 4, complete = npres == n && !inflight && !bad_time;
+    const bool barrier = have_first && gop == CCLD_OP_ALLREDUCE && gbytes < P.barrier_bytes;
+    // pass 2: op-set check, rate column, in-flight age, extrema
+    u32 mism = 0; i64 age = -1; u64 chk = 0;
+    u64 e_min = U64_MAX_, tmax = 0, tmin = U64_MAX_; i64 x_max = INT64_MIN;
+    for (u32 p = threadIdx.x; p < n; p += LARGE_DEF_THREADS) {
+      const u32 idx = pm[p * pst];
+      if (idx == NONE) continue;
+      if (D.op[idx] != gop || D.bytes[idx] != gbytes) mism = 1;
+      u32 ch = 0;
+      if (D.send_chg != nullptr) { const u32 sc = D.send_chg[idx], rc = D.recv_chg[idx]; ch = sc > rc ? sc : rc; }
+      const u64 ck = ((u64)ch << 32) | (u64)(NONE - p); chk = ck > chk ? ck : chk;
+      const u64 te = s_te[p], du = s_du[p];
+      if (D.t_exit[idx] == -1) { const i64 ag = now - (i64)te; age = ag > age ? ag : age; }
+      e_min = te < e_min ? te : e_min; tmax = du > tmax ? du : tmax; tmin = du < tmin ? du : tmin;
+      const i64 tx = (i64)(te + du); x_max = tx > x_max ? tx : x_max;
+    }
+    mism = block_reduce(mism, OpOrU32(), s_red32);
+    age = block_reduce(age, OpMaxI64(), (i64*)s_red64);
+    chk = block_reduce(chk, OpMaxU64(), s_red64);
+    e_min = block_reduce(e_min, OpMinU64(), s_red64);
+    tmax = block_reduce(tmax, OpMaxU64(), s_red64);
+    tmin = block_reduce(tmin, OpMinU64(), s_red64);
+    x_max = block_reduce(x_max, OpMaxI64(), (i64*)s_red64);
+    u32 gfl = (mism ? CCLD_G_OPSET_MISMATCH : 0) | (barrier ? CCLD_G_BARRIER : 0) | (inflight ? CCLD_G_INFLIGHT : 0) |
+              (bad_time ? CCLD_G_BAD_TIME : 0) | (complete ? CCLD_G_COMPLETE : CCLD_G_INCOMPLETE);
+    const bool analysed = complete && !barrier && n >= P.min_group;
+    const bool hang = !complete && inflight && age > P.hang_ns && !barrier;
+    if (analysed) gfl |= CCLD_G_ANALYSED;
+    if (hang) gfl |= CCLD_G_HANG_ALERT;
+
+    if (!complete) {
+      for (u32 p = threadIdx.x; p < n; p += LARGE_DEF_THREADS)
+        D.flags[slot + p] = pm[p * pst] == NONE ? (CCLD_F_NOT_ANALYSED | CCLD_F_MISSING) : CCLD_F_NOT_ANALYSED;
+      if (threadIdx.x == 0) {
+        if (hang) raise_alert(D, R.comm_id[c], seq, age);
+        for (int q = 0; q < GI_COUNT; ++q) D.gi64[(u64)q * G + g] = 0;
+        for (int q = 0; q < GU_COUNT; ++q) D.gu32[(u64)q * G + g] = 0;
+        D.gu32[(u64)GU_N_PRESENT * G + g] = npres; D.gu32[(u64)GU_GFLAGS * G + g] = gfl; D.gbw[g] = 0.0;
+        count_add(D.counters, C_INCOMPLETE, 1); count_add(D.counters, C_BARRIER, barrier); count_add(D.counters, C_MISMATCH, mism);
+        count_add(D.counters, C_PRESENT, npres);
+      }
+      continue;
+    }
+    // positions of the extrema: lowest ring position among equals
+    u32 pmax = NONE, pmin = NONE; u64 askew = 0;
+    for (u32 p = threadIdx.x; p < n; p += LARGE_DEF_THREADS) {
+      if (s_du[p] == tmax && p < pmax) pmax = p;
+      if (s_du[p] == tmin && p < pmin) pmin = p;
+      const u64 sk = s_te[p] - e_min; askew = sk > askew ? sk : askew;
+    }
+    pmax = block_reduce(pmax, OpMinU32(), s_red32);
+    pmin = block_reduce(pmin, OpMinU32(), s_red32);
+    askew = block_reduce(askew, OpMaxU64(), s_red64);
+    const i64 span = x_max - (i64)e_min;
+    double num, den; bus_factor(gop, n, &num, &den);
+    const double bn = (double)gbytes * num;
+    if (!barrier) {
+      for (u32 p = threadIdx.x; p < n; p += LARGE_DEF_THREADS) { atomicAdd(&R.bw_sum[mem[p]], busbw(bn, den, (i64)s_du[p])); atomicAdd(&R.bw_cnt[mem[p]], 1u); }
+    }
+    u64 med_s = 0, mad_s = 0, med_d = 0, mad_d = 0; u32 n_fs = 0, n_fd = 0;
+    if (analysed) {
+      const u32 k = (n - 1) >> 1;
+      med_s = radix_select([&](u32 i) { return s_te[i] - e_min; }, n, k, askew, s_hist, s_pick);
+      { const u64 m = med_s, dmax = m > askew - m ? m : askew - m;
+        mad_s = radix_select([&](u32 i) { return absdiff(s_te[i] - e_min, m); }, n, k, dmax, s_hist, s_pick); }
+      med_d = tmin + radix_select([&](u32 i) { return s_du[i] - tmin; }, n, k, tmax - tmin, s_hist, s_pick);
+      { const u64 m = med_d, dmax = (m - tmin) > (tmax - m) ? (m - tmin) : (tmax - m);
+        mad_d = radix_select([&](u32 i) { return absdiff(s_du[i], m); }, n, k, dmax, s_hist, s_pick); }
+      for (u32 p = threadIdx.x; p < n; p += LARGE_DEF_THREADS) {
+        const u64 sk = s_te[p] - e_min, du = s_du[p];
+        const bool so_ = mul_gt(absdiff(sk, med_s), 1000u, mad_s, P.k_milli), sh = sk > med_s;
+        const bool dq = mul_gt(absdiff(du, med_d), 1000u, mad_d, P.k_milli), dh = du > med_d;
+        D.flags[slot + p] = (so_ ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (sh ? CCLD_F_SKEW_HI : 0) | (dh ? CCLD_F_DUR_HI : 0);
+        if (so_) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p] * 4 + (sh ? 0 : 1)], 1u); }
+        if (dq) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p] * 4 + (dh ? 2 : 3)], 1u); }
+      }
+      n_fs = block_reduce(n_fs, OpAddU32(), s_red32);
+      n_fd = block_reduce(n_fd, OpAddU32(), s_red32);
+    } else {
+      for (u32 p = threadIdx.x; p < n; p += LARGE_DEF_THREADS) D.flags[slot + p] = CCLD_F_NOT_ANALYSED;
+    }
+    if (threadIdx.x == 0) {
+      D.gi64[(u64)GI_E_MIN * G + g] = (i64)e_min; D.gi64[(u64)GI_ARRIVAL_SKEW * G + g] = (i64)askew;
+      D.gi64[(u64)GI_T_MAX * G + g] = (i64)tmax; D.gi64[(u64)GI_T_MIN * G + g] = (i64)tmin; D.gi64[(u64)GI_SPAN * G + g] = span;
+      D.gi64[(u64)GI_MED_SKEW * G + g] = (i64)med_s; D.gi64[(u64)GI_MAD_SKEW * G + g] = (i64)mad_s;
+      D.gi64[(u64)GI_MED_DUR * G + g] = (i64)med_d; D.gi64[(u64)GI_MAD_DUR * G + g] = (i64)mad_d;
+      D.gu32[(u64)GU_RANK_TMIN * G + g] = mem[pmin]; D.gu32[(u64)GU_RANK_TMAX * G + g] = mem[pmax];
+      D.gu32[(u64)GU_MAX_CHG * G + g] = (u32)(chk >> 32); D.gu32[(u64)GU_RANK_MAX_CHG * G + g] = mem[NONE - (u32)chk];
+      D.gu32[(u64)GU_N_PRESENT * G + g] = npres; D.gu32[(u64)GU_GFLAGS * G + g] = gfl;
+      D.gbw[g] = busbw(bn, den, span);
+      count_add(D.counters, C_COMPLETE, 1); count_add(D.counters, C_BARRIER, barrier); count_add(D.counters, C_ANALYSED, analysed);
+      count_add(D.counters, C_MISMATCH, mism); count_add(D.counters, C_PRESENT, npres);
+      count_add(D.counters, C_FLAG_SKEW, n_fs); count_add(D.counters, C_FLAG_DUR, n_fd);
+    }
+  }
+}
+
+}  // namespace ccld
