@@ -114,6 +114,8 @@ def algorithmic_bytes(kernel, recs, groups):
         return 8 * recs, 0                                     # communicator id and op counter
     if kernel == "k_slot_scatter":
         return 12 * recs, 4 * recs                             # three key columns read; the record index written per slot
+    if kernel == "k_reduce_large":                             # with its staging pass: 32-bit keys written once and read again
+        return (VAL_BYTES + FLAG_BYTES) * recs + ROW_BYTES * groups, (INDEX_BYTES + 16) * recs
     if kernel.startswith("k_reduce"):
         return (VAL_BYTES + FLAG_BYTES) * recs + ROW_BYTES * groups, INDEX_BYTES * recs
     return 0, 0
@@ -361,8 +363,9 @@ def measure(spec, order, steps, warmup, local_rank, world, sample_clocks):
                 "kernels_ms_per_step": {k: kt[k]["ms"] / steps for k in kt},
                 "whole_path": {"algorithmic_bytes_per_step": path_bytes, "achieved": path_gbs, "frac": path_gbs / peak}}
     # every launch of the fused reduce kernel is followed by one of k_reduce_deferred (timed inside the same event pair),
-    # likewise k_reduce_large and its deferred kernel, and every launch of k_window_decide is preceded by one of k_window_rounds
-    launches = (sum(x["launches"] for x in kt.values()) + kt["k_reduce_fused"]["launches"] + kt["k_reduce_large"]["launches"]
+    # k_reduce_large runs between k_large_stage and k_reduce_large_deferred, and every launch of k_window_decide is preceded by
+    # one of k_window_rounds
+    launches = (sum(x["launches"] for x in kt.values()) + kt["k_reduce_fused"]["launches"] + 2 * kt["k_reduce_large"]["launches"]
                 + kt["k_window_decide"]["launches"])
     return {"n_rec": n_rec, "now": now, "ms_total": ms, "ms_per_step": ms / steps, "ms_best": min(per_step), "ms_median": statistics.median(per_step),
             "value": world * n_rec * steps / (ms * 1e-3), "value_best": world * n_rec / (min(per_step) * 1e-3),

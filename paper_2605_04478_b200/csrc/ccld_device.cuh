@@ -30,7 +30,8 @@ constexpr int LARGE_SEQS = 8;          // above: tiles of up to 8 consecutive op
 constexpr int LG_THREADS = 512;
 constexpr int LG_WARPS = LG_THREADS / 32;
 constexpr int LG_KEYS = 16;            //   (member, group) pairs a thread of the kernel holds at most
-constexpr u32 LG_BUDGET = 104 * 1024;  //   dynamic shared memory per CTA below which two CTAs fit one SM
+constexpr int LS_THREADS = 256;        //   staging kernel: a CTA takes LS_MEMBERS members of a tile
+constexpr int LS_MEMBERS = 512;
 
 struct Params {
   i64 tbase_init_ns, m_max_ns, hang_ns;
@@ -110,6 +111,7 @@ struct WinDesc {
   u64 n_groups, n_slots;
   u32* perm;                         // [n_slots]
   u8* flags;                         // [n_slots]
+  u32 *skey, *dkey;                  // [n_slots] staged 32-bit keys of the largest communicators (null when the batch has none)
   i64* gi64;                         // [9][n_groups]
   u32* gu32;                         // [6][n_groups]
   double* gbw;                       // [n_groups]
@@ -126,26 +128,18 @@ enum { GU_RANK_TMIN = 0, GU_RANK_TMAX, GU_MAX_CHG, GU_RANK_MAX_CHG, GU_N_PRESENT
 __host__ __device__ inline u32 next_pow2(u32 n) { u32 p = 1; while (p < n) p <<= 1; return p; }
 __host__ __device__ inline u32 comm_class(u32 n) { return n <= SMALL_N ? 0u : (n <= WARP_N ? 1u : (n <= MID_N ? 2u : 3u)); }
 __host__ __device__ inline u32 mid_npad(u32 n) { u32 p = next_pow2(n); return p < 32 ? 32 : p; }
-// Communicators of more than MID_N ranks: G groups (consecutive op counters) are worked on side by side, their 32-bit
-// keys in shared memory next to the tile's per-member bandwidth sums, one histogram per group and the partial extrema.
+// Communicators of more than MID_N ranks: a tile is LARGE_SEQS consecutive op counters; the select kernel works on G of
+// them side by side, as many as let a thread keep its share of the keys (at most LG_KEYS) in registers.
 __host__ __device__ inline u32 large_npad(u32 n) { return (n + 31u) & ~31u; }
-__host__ __device__ inline u32 large_pitch(u32 n, u32 G) { return large_npad(n) + 32u / G; }    // lanes g, g + 1, ... of one member hit distinct banks
-__host__ __device__ inline size_t large_smem(u32 n, u32 G) {
-  return (size_t)8 * G * large_pitch(n, G)            // enter-time offsets and durations, u32 each, [G][pitch]
-       + (size_t)8 * large_npad(n)                    // per-member bandwidth sums
-       + (size_t)G * 256 * 4                          // one histogram per group
-       + (size_t)LG_WARPS * G * 40                    // per-warp partial extrema (LargePart)
-       + (size_t)G * 48;                              // per-group totals (LargeLead), select state
-}
 __host__ __device__ inline u32 large_g(u32 n) {
-  for (u32 G = LARGE_SEQS; G > 1; G >>= 1)
-    if (large_smem(n, G) <= LG_BUDGET && (u64)G * large_npad(n) <= (u64)LG_KEYS * LG_THREADS) return G;
-  return 1;
+  u32 G = LARGE_SEQS;
+  while (G > 1 && (u64)G * large_npad(n) > (u64)LG_KEYS * LG_THREADS) G >>= 1;
+  return G;
 }
 // op counters per work unit: a warp-tile (class 0) or a CTA tile (classes 1 to 3)
 __host__ __device__ inline u32 tile_seqs(u32 n) {
   u32 c = comm_class(n);
-  return c == 0 ? 32u : (c <= 2 ? MID_ELEMS / mid_npad(n) : large_g(n));
+  return c == 0 ? 32u : (c <= 2 ? MID_ELEMS / mid_npad(n) : (u32)LARGE_SEQS);
 }
 __host__ __device__ inline u32 ceil_div(u32 a, u32 b) { return (a + b - 1) / b; }
 // chunking of a fused-class communicator with n_seq op counters in a window of T chunks

@@ -246,10 +246,8 @@ int finalize_registry(ccld_ctx* ctx) {
 
   CK(cudaFuncSetAttribute(k_reduce_mid, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mid_smem_bytes(2 * WARP_N)));
   if (max_large) {
-    size_t need = 0;                       // the largest tile layout among the registered communicators
-    for (auto& c : ctx->comms) if (c.ranks.size() > MID_N) need = std::max(need, large_smem((u32)c.ranks.size(), large_g((u32)c.ranks.size())));
-    ctx->large_smem = need;
-    CK(cudaFuncSetAttribute(k_reduce_large, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)need));
+    ctx->large_smem = large_smem(max_large);
+    CK(cudaFuncSetAttribute(k_reduce_large, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->large_smem));
     CK(cudaFuncSetAttribute(k_reduce_large_deferred, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(16ull * max_large)));
   }
   ctx->finalized = true;
@@ -455,7 +453,7 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
     d.rmin = (u32*)(pbase + o_rmin) + (size_t)k * nc; d.rmax = (u32*)(pbase + o_rmax) + (size_t)k * nc;
     d.ranges = (RangeRow*)(pbase + o_rng) + (size_t)k * nc; d.srow = (uint4*)(pbase + o_srow) + (size_t)k * nc;
     d.totals = (u64*)(pbase + o_tot) + (size_t)k * T_COUNT; d.counters = (u64*)(pbase + o_cnt) + (size_t)k * C_COUNT;
-    d.n_groups = d.n_slots = 0; d.perm = nullptr; d.flags = nullptr; d.gi64 = nullptr; d.gu32 = nullptr; d.gbw = nullptr;
+    d.n_groups = d.n_slots = 0; d.perm = nullptr; d.flags = nullptr; d.skey = d.dkey = nullptr; d.gi64 = nullptr; d.gu32 = nullptr; d.gbw = nullptr;
     d.comm_rows = nullptr; d.alerts = nullptr;
     for (int q = 0; q < B_COUNT; ++q) d.base[q] = 0;
     d.pad = 0; d.tsum[0] = d.tsum[1] = d.tsum[2] = nullptr;
@@ -502,7 +500,9 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   u64 total_groups = 0;
   for (u32 k = 0; k < B; ++k) total_groups += ctx->h_pinned[(size_t)k * T_COUNT + T_GROUPS];
   const size_t o_defn = take(16), o_def = take(n_list[B_FCTA] ? total_groups * 8 : 0),
-               o_def3 = take(n_list[B_T3] * (size_t)LARGE_SEQS * 8);          // likewise for the kernel of the largest communicators
+               o_def3 = take(n_list[B_T3] * (size_t)LARGE_SEQS * 8),          // likewise for the kernel of the largest communicators
+               o_lgrp = take(n_list[B_T3] * (size_t)LARGE_SEQS * sizeof(LargeGroup)),
+               o_skey = take(n_list[B_T3] ? total_slots * 4 : 0), o_dkey = take(n_list[B_T3] ? total_slots * 4 : 0);
   Block rb = ctx->pool.get(off, &e);
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "result allocation failed");
   auto res_blk = std::make_shared<Shared>(&ctx->pool, rb);
@@ -512,6 +512,7 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
     WinDesc& d = hd[k];
     d.n_groups = t[T_GROUPS]; d.n_slots = t[T_SLOTS];
     d.perm = (u32*)(rbase + o_perm + perm_off[k]); d.flags = (u8*)(rbase + o_flags[k]);
+    if (n_list[B_T3]) { d.skey = (u32*)(rbase + o_skey + perm_off[k]); d.dkey = (u32*)(rbase + o_dkey + perm_off[k]); }
     d.gi64 = (i64*)(rbase + o_gi[k]); d.gu32 = (u32*)(rbase + o_gu[k]); d.gbw = (double*)(rbase + o_gb[k]);
     d.comm_rows = (ccld_comm_verdict*)(rbase + o_rows[k]); d.alerts = (ccld_hang_alert*)(rbase + o_al[k]);
     d.tsum[0] = (TileSum*)(rbase + o_fsum); d.tsum[1] = (TileSum*)(rbase + o_s2); d.tsum[2] = (TileSum*)(rbase + o_s3);
@@ -531,9 +532,12 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   if (n_list[B_T2]) { TimedLaunch tl(ts, 4, st); k_reduce_mid<<<(u32)n_list[B_T2], MID_THREADS, mid_smem_bytes(2 * WARP_N), st>>>(d_desc, pl.t2, (TileSum*)(rbase + o_s2), ctx->reg, ctx->dp, now_ns); }
   if (n_list[B_T3]) {
     const DeferList dl{(u64*)(rbase + o_def3), (u32*)(rbase + o_defn) + 2};
+    LargeGroup* lgrp = (LargeGroup*)(rbase + o_lgrp);
+    CK(cudaMemsetAsync(lgrp, 0, n_list[B_T3] * (size_t)LARGE_SEQS * sizeof(LargeGroup), st));
     TimedLaunch tl(ts, 5, st);
+    k_large_stage<<<dim3((u32)n_list[B_T3], (ctx->max_large_n + LS_MEMBERS - 1) / LS_MEMBERS), LS_THREADS, 0, st>>>(d_desc, pl.t3, lgrp, ctx->reg);
     const u32 grid = (u32)std::min<u64>(n_list[B_T3], 2ull * ctx->n_sms);      // persistent: two CTAs per SM take the tiles in turn
-    k_reduce_large<<<grid, LG_THREADS, ctx->large_smem, st>>>(d_desc, pl.t3, (u32)n_list[B_T3], (TileSum*)(rbase + o_s3), ctx->reg, ctx->dp, dl);
+    k_reduce_large<<<grid, LG_THREADS, ctx->large_smem, st>>>(d_desc, pl.t3, (u32)n_list[B_T3], lgrp, (TileSum*)(rbase + o_s3), ctx->reg, ctx->dp, dl);
     k_reduce_large_deferred<<<LARGE_DEF_GRID, LARGE_DEF_THREADS, 16ull * ctx->max_large_n, st>>>(d_desc, dl, ctx->reg, ctx->dp, now_ns);
   }
   {

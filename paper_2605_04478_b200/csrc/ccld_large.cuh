@@ -1,36 +1,132 @@
 // Per-op reductions, median / MAD, flags and votes for communicators of more than 1,024 ranks (sm_100a).
 //
-//   k_reduce_large           the common case: every member reported, nothing in flight, all times of a group within
-//                            2^31 ns of its first member's enter time. A tile is G consecutive op counters of one
-//                            communicator (G = 8, 4, 2 or 1: as many as fit the shared-memory budget that still lets two
-//                            CTAs share an SM). Lanes run along the op counter first: the G record indices of one member
-//                            are neighbours in the member-major permutation, and in a rank-major upload so are the
-//                            records themselves, so the gathers of a warp touch 32 / G short contiguous stretches.
-//                            Enter-time offsets and durations of the G groups wait in shared memory as 32-bit keys;
-//                            every CTA-wide step - the extrema, the four radix selects, the flag pass - runs once for
-//                            all G groups side by side, so a tile costs the barriers of one group. During a select a
-//                            thread keeps its keys in registers. The grid is persistent: CTA b takes tiles b, b + grid,
-//                            ..., so CTAs that run at the same time work on neighbouring op counters (what one fetches
-//                            of a 64-byte line, its neighbours find in L2) and a CTA's tiles of one communicator and
-//                            window add their per-member bandwidth sums in shared memory before they go to global memory.
-//   k_reduce_large_deferred  the groups the fast kernel sets aside (a missing member, a record in flight, invalid
-//                            times, spreads beyond 32 bits): one CTA per listed group, 64-bit throughout, hang alerts.
+// A group of thousands of members has its records spread over as many places of the upload, and its order statistics
+// need every key several times. The work is therefore cut in two:
+//
+//   k_large_stage            one pass over the records of a tile (LARGE_SEQS consecutive op counters of one communicator,
+//                            LS_MEMBERS members per CTA). Lanes run along the op counter first: the eight record indices
+//                            of a member are one 32-byte sector of the member-major permutation, and in a rank-major
+//                            upload the eight records are neighbours too, so every gather of a warp fetches whole
+//                            sectors. Times become 32-bit keys (enter-time offset from the group's first member, duration)
+//                            and leave, transposed through shared memory, as two contiguous arrays per group; the extrema,
+//                            the op-set check and the rate column are reduced on the way and merged per group with atomics.
+//   k_reduce_large           the order statistics. A CTA works on G groups of a tile side by side (G = 8, 4, 2 or 1: a
+//                            thread keeps its share of a group's keys, at most LG_KEYS, in registers during a select);
+//                            every CTA-wide step runs once for all G groups, so a sub-tile costs the barriers of one
+//                            group. Keys are read from the staged arrays with coalesced loads; flags, votes and the
+//                            per-member bandwidth sums follow, the sums gathered in shared memory over all tiles a CTA
+//                            handles of one communicator and window (the grid is persistent).
+//   k_reduce_large_deferred  the groups that are not complete and 32-bit clean (a missing member, a record in flight,
+//                            invalid times, spreads beyond 32 bits): one CTA per listed group, 64-bit throughout, hang alerts.
 #pragma once
 #include "ccld_device.cuh"
 
 namespace ccld {
 
-struct LargePart { u64 kmax, kmin, ck; u32 emin, emax, xmax, bits; };      // bits: 1 = some record disqualifies the group, 2 = op set differs
+// What k_large_stage leaves per group; every field is a maximum (minima are stored complemented), so zero is the
+// neutral start. bits: 1 = some record disqualifies the group for the 32-bit path, 2 = the op set differs inside it.
+struct LargeGroup { u64 kmax, n_kmin, ck; u32 n_emin, emax, xmax, bits; };
 struct LargeLead { u64 brng; u32 bk, rounds, an, def, pad; };
-static_assert(sizeof(LargePart) == 40 && sizeof(LargeLead) == 32, "large_smem() counts these sizes");
+// per-group values the flag pass reads back from shared memory
+struct LargeScal { u64 ts, td; double bn, den; u32 emin, tmn, ms, md; u32 state, pad; };       // state: 1 group handled here, 2 analysed, 4 barrier
+
+constexpr u32 LS_PITCH = LS_MEMBERS + 4;     // lanes (op counter 0..7, member 0..3) hit 32 distinct banks
+
+__global__ void __launch_bounds__(LS_THREADS) k_large_stage(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles, LargeGroup* __restrict__ grp, Registry R) {
+  __shared__ u32 s_a[LARGE_SEQS * LS_PITCH], s_d[LARGE_SEQS * LS_PITCH];
+  __shared__ LargeGroup s_part[LS_THREADS / 32][LARGE_SEQS];
+  const Tile t = tiles[blockIdx.x];
+  const WinDesc& D = wd[t.w];
+  const u32 n = R.comm_n[t.c], m0 = blockIdx.y * LS_MEMBERS;
+  if (m0 >= n) return;
+  const RangeRow row = D.ranges[t.c];
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  const u32 j = lane & 7, pq = lane >> 3;                     // op counter of the tile, member of the quad
+  const bool jvalid = j < t.count;
+  const u32 so = t.seq_off + (jvalid ? j : 0u);
+  const u32* __restrict__ perm = D.perm + row.slot0;
+  const i64* __restrict__ c_te = D.t_enter; const i64* __restrict__ c_tx = D.t_exit;
+  const u64* __restrict__ c_by = D.bytes; const u8* __restrict__ c_op = D.op;
+  const u32* __restrict__ c_sc = D.send_chg; const u32* __restrict__ c_rc = D.recv_chg;
+  // the group's first member gives the time base and the op set
+  u32 bits = 0;
+  i64 te0 = 0; u64 by0 = 0; u32 op0 = 0;
+  {
+    const u32 i0 = jvalid ? __ldg(perm + so) : NONE;
+    if (i0 != NONE) { te0 = c_te[i0]; by0 = c_by[i0]; op0 = c_op[i0]; } else bits = 1;
+  }
+  const u64 base = (u64)te0 - 0x80000000ull;
+  u32 emin = 0xFFFFFFFFu, emax = 0, xmax = 0; u64 kmax = 0, kmin = U64_MAX_, ck = 0;
+  constexpr u32 PER_WARP = LS_MEMBERS / (LS_THREADS / 32);    // 64 members per warp, four at a time
+  for (u32 it = 0; it < PER_WARP / 4; it += 4) {
+    u32 idx[4]; i64 x[4], y[4]; u64 by[4]; u32 op[4], ch[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) { const u32 p = m0 + wid * PER_WARP + (it + q) * 4 + pq; idx[q] = (jvalid && p < n) ? __ldg(perm + (u64)p * row.n_seq + so) : NONE; }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const u32 ix = idx[q] == NONE ? 0u : idx[q];
+      x[q] = c_te[ix]; y[q] = c_tx[ix]; by[q] = c_by[ix]; op[q] = c_op[ix]; ch[q] = 0;
+      if (c_sc != nullptr) { const u32 sc = c_sc[ix], rc = c_rc[ix]; ch[q] = sc > rc ? sc : rc; }
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const u32 pm = wid * PER_WARP + (it + q) * 4 + pq, p = m0 + pm;
+      u32 a_lo = 0, d = 0;
+      if (p < n) {
+        if (idx[q] == NONE) { if (jvalid) bits |= 1; }
+        else {
+          const u64 ra = (u64)x[q] - base, rb = (u64)y[q] - base;
+          a_lo = (u32)ra; const u32 b_lo = (u32)rb; d = b_lo - a_lo;
+          if (((ra | rb) >> 32) != 0 || (x[q] | y[q]) < 0 || b_lo < a_lo) bits |= 1;     // beyond 32 bits, negative or in flight, exit before enter
+          if (op[q] != op0 || by[q] != by0) bits |= 2;
+          emin = min(emin, a_lo); emax = max(emax, a_lo); xmax = max(xmax, b_lo);
+          const u64 k1 = ((u64)d << 32) | (u64)(NONE - p); kmax = k1 > kmax ? k1 : kmax;   // longest, then the lowest position
+          const u64 k2 = ((u64)d << 32) | (u64)p; kmin = k2 < kmin ? k2 : kmin;            // shortest, then the lowest position
+          const u64 k3 = ((u64)ch[q] << 32) | (u64)(NONE - p); ck = k3 > ck ? k3 : ck;     // most changes, then the lowest position
+        }
+      }
+      s_a[j * LS_PITCH + pm] = a_lo; s_d[j * LS_PITCH + pm] = d;
+    }
+  }
+  // the four members of a warp step meet by shuffles, the warps through shared memory; one thread per op counter merges
+  // the CTA's part into the group's record
+#pragma unroll
+  for (int h = 8; h < 32; h <<= 1) {
+    emin = min(emin, __shfl_xor_sync(0xFFFFFFFFu, emin, h)); emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, h));
+    xmax = max(xmax, __shfl_xor_sync(0xFFFFFFFFu, xmax, h)); bits |= __shfl_xor_sync(0xFFFFFFFFu, bits, h);
+    const u64 a = shfl_xor64(kmax, h); kmax = a > kmax ? a : kmax;
+    const u64 b = shfl_xor64(kmin, h); kmin = b < kmin ? b : kmin;
+    const u64 e = shfl_xor64(ck, h); ck = e > ck ? e : ck;
+  }
+  if (lane < LARGE_SEQS) { LargeGroup x; x.kmax = kmax; x.n_kmin = ~kmin; x.ck = ck; x.n_emin = ~emin; x.emax = emax; x.xmax = xmax; x.bits = bits; s_part[wid][lane] = x; }
+  __syncthreads();
+  if (threadIdx.x < t.count) {
+    LargeGroup a = s_part[0][threadIdx.x];
+    for (u32 w = 1; w < LS_THREADS / 32; ++w) {
+      const LargeGroup x = s_part[w][threadIdx.x];
+      a.kmax = x.kmax > a.kmax ? x.kmax : a.kmax; a.n_kmin = x.n_kmin > a.n_kmin ? x.n_kmin : a.n_kmin; a.ck = x.ck > a.ck ? x.ck : a.ck;
+      a.n_emin = max(a.n_emin, x.n_emin); a.emax = max(a.emax, x.emax); a.xmax = max(a.xmax, x.xmax); a.bits |= x.bits;
+    }
+    LargeGroup* o = grp + (u64)blockIdx.x * LARGE_SEQS + threadIdx.x;
+    atomicMax((ull*)&o->kmax, (ull)a.kmax); atomicMax((ull*)&o->n_kmin, (ull)a.n_kmin); atomicMax((ull*)&o->ck, (ull)a.ck);
+    atomicMax(&o->n_emin, a.n_emin); atomicMax(&o->emax, a.emax); atomicMax(&o->xmax, a.xmax);
+    if (a.bits) atomicOr(&o->bits, a.bits);
+  }
+  // keys leave group by group, members contiguous
+  const u32 cnt = n - m0 < LS_MEMBERS ? n - m0 : (u32)LS_MEMBERS;
+  for (u32 q = 0; q < t.count; ++q) {
+    const u64 o = row.slot0 + (u64)(t.seq_off + q) * n + m0;
+    for (u32 pm = threadIdx.x; pm < cnt; pm += LS_THREADS) { D.skey[o + pm] = s_a[q * LS_PITCH + pm]; D.dkey[o + pm] = s_d[q * LS_PITCH + pm]; }
+  }
+}
 
 __device__ __forceinline__ int top_byte(u32 bound) { return bound == 0 ? 0 : (31 - __clz(bound)) >> 3; }
 
-// The k-th smallest (0-based) of a group's keys, for every group of the tile at once. A thread holds up to LG_KEYS keys
-// of its own group lane g in registers (bit q of `have` says whether slot q holds one); `act` says whether the group takes
-// part. Digits of 8 bits, most significant first, starting at byte `top` (the same for all groups). A thread counts the
-// keys that share the digit of its first candidate itself and adds them once - in the passes over high bytes nearly all
-// keys of a group agree - and adds the others one by one. Histograms must be zero on entry and are zero again on
+// The k-th smallest (0-based) of a group's keys, for every group of the sub-tile at once. A thread holds up to LG_KEYS
+// keys of its own group g in registers (bit q of `have` says whether slot q holds one); `act` says whether the group
+// takes part. Digits of 8 bits, most significant first, starting at byte `top` (the same for all groups). A thread counts
+// the keys that share the digit of its first candidate itself and adds them once - in the passes over high bytes nearly
+// all keys of a group agree - and adds the others one by one. Histograms must be zero on entry and are zero again on
 // return. All threads of the CTA call it.
 __device__ __forceinline__ u32 large_select(const u32 (&v)[LG_KEYS], u32 have, bool act, u32 k, int top, u32 G, u32 g,
                                             u32* __restrict__ s_hist, u32* __restrict__ s_pick, u32* __restrict__ s_krem) {
@@ -83,15 +179,23 @@ __device__ __forceinline__ u32 large_select(const u32 (&v)[LG_KEYS], u32 have, b
   return prefix;
 }
 
+inline size_t large_smem(u32 max_n) { return (size_t)8 * large_npad(max_n); }     // per-member bandwidth sums
+
 __global__ void __launch_bounds__(LG_THREADS, 2) k_reduce_large(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles, u32 n_tiles,
-                                                                 TileSum* __restrict__ sums, Registry R, Params P, DeferList DL) {
+                                                                 const LargeGroup* __restrict__ grp, TileSum* __restrict__ sums,
+                                                                 Registry R, Params P, DeferList DL) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
+  double* s_bw = (double*)smem_raw;
+  __shared__ u32 s_hist[LARGE_SEQS * 256];
+  __shared__ LargeScal s_sc[LARGE_SEQS];
+  __shared__ LargeLead s_lead[LARGE_SEQS];
   __shared__ u32 s_cnt[SC_COUNT];
   __shared__ u32 s_bound[2][LARGE_SEQS];
+  __shared__ u32 s_pick[LARGE_SEQS], s_krem[LARGE_SEQS];
   const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   u32 cur_w = NONE, cur_c = NONE, cur_rounds = 0;            // whose bandwidth sums shared memory holds
   const u32* cur_mem = nullptr; u32 cur_n = 0;
-  double* s_bw = nullptr;
+  for (u32 i = threadIdx.x; i < LARGE_SEQS * 256; i += LG_THREADS) s_hist[i] = 0;
 
   for (u32 ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
     const Tile t = tiles[ti];
@@ -99,192 +203,137 @@ __global__ void __launch_bounds__(LG_THREADS, 2) k_reduce_large(const WinDesc* _
     const u32 c = t.c, n = R.comm_n[c];
     const RangeRow row = D.ranges[c];
     const u32* __restrict__ mem = R.members + R.comm_moff[c];
-    const u32 n_pad = large_npad(n), G = large_g(n), pitch = large_pitch(n, G), lgG = 31 - __clz(G);
-    u32* s_sk = (u32*)smem_raw;                               // enter time minus (first member's enter time - 2^31)
-    u32* s_du = s_sk + (size_t)G * pitch;                     // duration
-    double* bw_here = (double*)(s_du + (size_t)G * pitch);
-    u32* s_hist = (u32*)(bw_here + n_pad);
-    LargePart* s_part = (LargePart*)(s_hist + G * 256);
-    LargeLead* s_lead = (LargeLead*)(s_part + LG_WARPS * G);
-    u32* s_pick = (u32*)(s_lead + G);
-    u32* s_krem = s_pick + G;
-    const u32 g = threadIdx.x & (G - 1), pl = threadIdx.x >> lgG, MP = LG_THREADS >> lgG;
-    const bool lead = pl == 0;                                // threads 0 .. G-1: one per group lane
+    const u32 G = large_g(n), lgG = 31 - __clz(G);
+    const u32 g = wid & (G - 1), pl = (wid >> lgG) * 32 + lane, MP = (LG_WARPS >> lgG) * 32;      // a warp works on one group, lanes on consecutive members
+    const bool lead = pl == 0;
+    const u64 G_all = D.n_groups;
 
     __syncthreads();                                          // the previous tile is done with shared memory
     if (t.w != cur_w || c != cur_c) {
-      // another communicator or window: what shared memory holds goes out, and the layout may change
+      // another communicator or window: the sums shared memory holds go out
       if (cur_rounds) for (u32 p = threadIdx.x; p < cur_n; p += LG_THREADS) { atomicAdd(&R.bw_sum[cur_mem[p]], s_bw[p]); atomicAdd(&R.bw_cnt[cur_mem[p]], cur_rounds); }
-      __syncthreads();
-      cur_w = t.w; cur_c = c; cur_rounds = 0; cur_mem = mem; cur_n = n; s_bw = bw_here;
-      for (u32 p = threadIdx.x; p < n_pad; p += LG_THREADS) s_bw[p] = 0.0;
-      for (u32 i = threadIdx.x; i < G * 256; i += LG_THREADS) s_hist[i] = 0;
+      cur_w = t.w; cur_c = c; cur_rounds = 0; cur_mem = mem; cur_n = n;
+      for (u32 p = threadIdx.x; p < n; p += LG_THREADS) s_bw[p] = 0.0;
     }
     if (threadIdx.x < SC_COUNT) s_cnt[threadIdx.x] = 0;
-    const u32* __restrict__ perm = D.perm + row.slot0;
-    const i64* __restrict__ c_te = D.t_enter; const i64* __restrict__ c_tx = D.t_exit;
-    const u64* __restrict__ c_by = D.bytes; const u8* __restrict__ c_op = D.op;
-    const u32* __restrict__ c_sc = D.send_chg; const u32* __restrict__ c_rc = D.recv_chg;
-    const u64 G_all = D.n_groups;
-    const bool gvalid = g < t.count;
-    const u32 so = t.seq_off + (gvalid ? g : 0u);             // op-counter offset of my group inside the range
-
-    // ---- gather: the group's first member gives the time base and the op set (every thread of the group lane loads it:
-    //      one address per lane group, served by one transaction) ----
-    u32 bits = 0;
-    i64 te0 = 0; u64 by0 = 0; u32 op0 = 0;
-    {
-      const u32 i0 = gvalid ? __ldg(perm + so) : NONE;
-      if (i0 != NONE) { te0 = c_te[i0]; by0 = c_by[i0]; op0 = c_op[i0]; } else bits = 1;
-    }
-    const u64 base = (u64)te0 - 0x80000000ull;
-    u32 emin = 0xFFFFFFFFu, emax = 0, xmax = 0; u64 kmax = 0, kmin = U64_MAX_, ck = 0;
-    for (u32 p0 = pl; p0 < n; p0 += 4 * MP) {
-      u32 idx[4]; i64 x[4], y[4]; u64 by[4]; u32 op[4], ch[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) { const u32 p = p0 + q * MP; idx[q] = (gvalid && p < n) ? __ldg(perm + (u64)p * row.n_seq + so) : NONE; }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const u32 ix = idx[q] == NONE ? 0u : idx[q];
-        x[q] = c_te[ix]; y[q] = c_tx[ix]; by[q] = c_by[ix]; op[q] = c_op[ix]; ch[q] = 0;
-        if (c_sc != nullptr) { const u32 sc = c_sc[ix], rc = c_rc[ix]; ch[q] = sc > rc ? sc : rc; }
-      }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        const u32 p = p0 + q * MP;
-        if (p < n) {
-          u32 a_lo = 0, d = 0;
-          if (idx[q] == NONE) { if (gvalid) bits |= 1; }
-          else {
-            const u64 ra = (u64)x[q] - base, rb = (u64)y[q] - base;
-            a_lo = (u32)ra; const u32 b_lo = (u32)rb; d = b_lo - a_lo;
-            if (((ra | rb) >> 32) != 0 || (x[q] | y[q]) < 0 || b_lo < a_lo) bits |= 1;     // beyond 32 bits, negative or in flight, exit before enter
-            if (op[q] != op0 || by[q] != by0) bits |= 2;
-            emin = min(emin, a_lo); emax = max(emax, a_lo); xmax = max(xmax, b_lo);
-            const u64 k1 = ((u64)d << 32) | (u64)(NONE - p); kmax = k1 > kmax ? k1 : kmax;   // longest, then the lowest position
-            const u64 k2 = ((u64)d << 32) | (u64)p; kmin = k2 < kmin ? k2 : kmin;            // shortest, then the lowest position
-            const u64 k3 = ((u64)ch[q] << 32) | (u64)(NONE - p); ck = k3 > ck ? k3 : ck;     // most changes, then the lowest position
-          }
-          s_sk[g * pitch + p] = a_lo; s_du[g * pitch + p] = d;
-        }
-      }
-    }
-    // ---- extrema of the G groups: lanes of one group lane meet by shuffles, warps through shared memory ----
-    for (u32 h = G; h < 32; h <<= 1) {
-      emin = min(emin, __shfl_xor_sync(0xFFFFFFFFu, emin, h)); emax = max(emax, __shfl_xor_sync(0xFFFFFFFFu, emax, h));
-      xmax = max(xmax, __shfl_xor_sync(0xFFFFFFFFu, xmax, h)); bits |= __shfl_xor_sync(0xFFFFFFFFu, bits, h);
-      const u64 a = shfl_xor64(kmax, h); kmax = a > kmax ? a : kmax;
-      const u64 b = shfl_xor64(kmin, h); kmin = b < kmin ? b : kmin;
-      const u64 e = shfl_xor64(ck, h); ck = e > ck ? e : ck;
-    }
-    if (lane < G) { LargePart x; x.kmax = kmax; x.kmin = kmin; x.ck = ck; x.emin = emin; x.emax = emax; x.xmax = xmax; x.bits = bits; s_part[wid * G + lane] = x; }
-    __syncthreads();
-#pragma unroll 4
-    for (u32 w = 0; w < LG_WARPS; ++w) {
-      const LargePart x = s_part[w * G + g];
-      emin = min(emin, x.emin); emax = max(emax, x.emax); xmax = max(xmax, x.xmax); bits |= x.bits;
-      kmax = x.kmax > kmax ? x.kmax : kmax; kmin = x.kmin < kmin ? x.kmin : kmin; ck = x.ck > ck ? x.ck : ck;
-    }
-    const bool gok = gvalid && !(bits & 1);
-    const u32 tmx = (u32)(kmax >> 32), tmn = (u32)(kmin >> 32);
-    const bool barrier = op0 == CCLD_OP_ALLREDUCE && by0 < P.barrier_bytes;
-    const bool analysed = gok && !barrier && n >= P.min_group;
-    double num, den; bus_factor(op0, n, &num, &den);
-    const double bn = (double)by0 * num;
-    if (lead) {
-      s_bound[0][g] = analysed ? emax - emin : 0u; s_bound[1][g] = analysed ? tmx - tmn : 0u;
-      LargeLead mine = {0, NONE, 0, 0, 0, 0};
-      if (gvalid && !gok) {                                   // set aside for the 64-bit kernel
-        const u32 e = atomicAdd(DL.count, 1u);
-        DL.entries[e] = ((u64)t.w << 32) | (u64)(row.group0 + so);
-        mine.def = 1;
-      }
-      if (gok) {
-        // everything of the per-op row that needs no order statistic goes out now, so that it occupies no registers during the selects
-        const u64 gi_ = row.group0 + so;
-        i64* __restrict__ gi = D.gi64 + gi_; u32* __restrict__ gu = D.gu32 + gi_;
-        const u32 span = xmax - emin;
-        gi[(u64)GI_E_MIN * G_all] = (i64)(base + emin); gi[(u64)GI_ARRIVAL_SKEW * G_all] = (i64)(u64)(emax - emin);
-        gi[(u64)GI_T_MAX * G_all] = (i64)(u64)tmx; gi[(u64)GI_T_MIN * G_all] = (i64)(u64)tmn; gi[(u64)GI_SPAN * G_all] = (i64)(u64)span;
-        gu[(u64)GU_RANK_TMIN * G_all] = mem[(u32)kmin]; gu[(u64)GU_RANK_TMAX * G_all] = mem[NONE - (u32)kmax];
-        gu[(u64)GU_MAX_CHG * G_all] = (u32)(ck >> 32); gu[(u64)GU_RANK_MAX_CHG * G_all] = mem[NONE - (u32)ck];
-        gu[(u64)GU_N_PRESENT * G_all] = n;
-        const bool mismatch = (bits & 2) != 0;
-        gu[(u64)GU_GFLAGS * G_all] = CCLD_G_COMPLETE | (barrier ? CCLD_G_BARRIER : 0) | (mismatch ? CCLD_G_OPSET_MISMATCH : 0) | (analysed ? CCLD_G_ANALYSED : 0);
-        D.gbw[gi_] = span ? bn * rcp_newton((double)span * den) : 0.0;
-        atomicAdd(&s_cnt[SC_COMP], 1u); atomicAdd(&s_cnt[SC_PRES], n);
-        if (barrier) atomicAdd(&s_cnt[SC_BAR], 1u);
-        if (analysed) { atomicAdd(&s_cnt[SC_AN], 1u); mine.an = 1; }
-        if (mismatch) atomicAdd(&s_cnt[SC_MIS], 1u);
-        if (!barrier) { mine.rounds = 1; mine.brng = (u64)(tmx - tmn); mine.bk = so; }
-      }
-      s_lead[g] = mine;
-    }
-    __syncthreads();
-    u32 bs = 0, bd = 0;
-    for (u32 q = 0; q < G; ++q) { bs = max(bs, s_bound[0][q]); bd = max(bd, s_bound[1][q]); }
-
-    // ---- order statistics, all groups of the tile side by side; a thread's keys sit in registers during a select ----
-    u32 ms = 0, ds = 0, md = 0, dm = 0;
+    if (threadIdx.x < LARGE_SEQS) { LargeLead z = {0, NONE, 0, 0, 0, 0}; s_lead[threadIdx.x] = z; }
     u32 have = 0;
 #pragma unroll
     for (int q = 0; q < LG_KEYS; ++q) have |= (pl + (u32)q * MP < n ? 1u : 0u) << q;
-    if (__syncthreads_or(analysed)) {
-      const u32 k = (n - 1) >> 1;
-      u32 v[LG_KEYS];
-#pragma unroll
-      for (int q = 0; q < LG_KEYS; ++q) v[q] = (have >> q) & 1u ? s_sk[g * pitch + pl + (u32)q * MP] - emin : 0u;
-      ms = large_select(v, have, analysed, k, top_byte(bs), G, g, s_hist, s_pick, s_krem);
-#pragma unroll
-      for (int q = 0; q < LG_KEYS; ++q) v[q] = __usad(v[q], ms, 0u);
-      ds = large_select(v, have, analysed, k, top_byte(bs), G, g, s_hist, s_pick, s_krem);
-#pragma unroll
-      for (int q = 0; q < LG_KEYS; ++q) v[q] = (have >> q) & 1u ? s_du[g * pitch + pl + (u32)q * MP] - tmn : 0u;
-      md = large_select(v, have, analysed, k, top_byte(bd), G, g, s_hist, s_pick, s_krem);
-#pragma unroll
-      for (int q = 0; q < LG_KEYS; ++q) v[q] = __usad(v[q], md, 0u);
-      dm = large_select(v, have, analysed, k, top_byte(bd), G, g, s_hist, s_pick, s_krem);
-      if (!analysed) { ms = ds = md = dm = 0; }
-    }
 
-    // ---- flags, votes, per-member bandwidth ----
-    u32 n_fs = 0, n_fd = 0;
-    {
-      const u64 ts = (u64)ds * P.k_milli, td = (u64)dm * P.k_milli;          // |x - med| * 1000 > k * MAD: both sides below 2^64
-      u8* __restrict__ fp = D.flags + row.slot0 + (u64)so * n;
-      for (u32 p0 = 0; p0 < n; p0 += MP) {                                   // the same trip count for every thread: shuffles inside
-        const u32 p = p0 + pl;
-        double bwv = 0.0;
-        if (gok && p < n) {
-          const u32 d = s_du[g * pitch + p];
-          u32 f = CCLD_F_NOT_ANALYSED;
-          if (analysed) {
-            const u32 skw = s_sk[g * pitch + p] - emin, dd = d - tmn;
-            const bool so_ = (u64)__usad(skw, ms, 0u) * 1000u > ts, shi = skw > ms;
-            const bool dq = (u64)__usad(dd, md, 0u) * 1000u > td, dhi = dd > md;
-            f = (so_ ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (shi ? CCLD_F_SKEW_HI : 0) | (dhi ? CCLD_F_DUR_HI : 0);
-            if (so_) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p] * 4 + (shi ? 0 : 1)], 1u); }
-            if (dq) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p] * 4 + (dhi ? 2 : 3)], 1u); }
-          }
-          fp[p] = (u8)f;
-          if (!barrier && d != 0) bwv = bn * rcp_newton1((double)d * den);
+    for (u32 j0 = 0; j0 < t.count; j0 += G) {
+      const bool gvalid = j0 + g < t.count;
+      const u32 so = t.seq_off + j0 + (gvalid ? g : 0u);      // op-counter offset of my group inside the range
+      const u64 slot = row.slot0 + (u64)so * n;               // first slot of my group (keys and flags, group-major)
+      __syncthreads();                                        // the previous sub-tile's shared-memory values are no longer read
+      // ---- what the staging pass left for the group; op and size of its first member ----
+      const LargeGroup x = grp[(u64)ti * LARGE_SEQS + j0 + (gvalid ? g : 0u)];
+      const u32 emin = ~x.n_emin, tmx = (u32)(x.kmax >> 32), tmn = (u32)(~x.n_kmin >> 32);
+      u64 by0 = 0; u32 op0 = 0; i64 te0 = 0;
+      const bool gok = gvalid && !(x.bits & 1);
+      if (gok) { const u32 i0 = __ldg(D.perm + row.slot0 + so); by0 = D.bytes[i0]; op0 = D.op[i0]; te0 = D.t_enter[i0]; }
+      const bool barrier = op0 == CCLD_OP_ALLREDUCE && by0 < P.barrier_bytes;
+      const bool analysed = gok && !barrier && n >= P.min_group;
+      double num, den; bus_factor(op0, n, &num, &den);
+      const double bn = (double)by0 * num;
+      if (lead) {
+        s_bound[0][g] = analysed ? x.emax - emin : 0u; s_bound[1][g] = analysed ? tmx - tmn : 0u;
+        if (gvalid && !gok) {                                 // set aside for the 64-bit kernel
+          const u32 e = atomicAdd(DL.count, 1u);
+          DL.entries[e] = ((u64)t.w << 32) | (u64)(row.group0 + so);
+          s_lead[g].def += 1;
         }
-        for (u32 h = 1; h < G; h <<= 1) bwv += __shfl_xor_sync(0xFFFFFFFFu, bwv, h);   // the G group lanes of member p are neighbours
-        if (g == 0 && p < n) s_bw[p] += bwv;
+        if (gok) {
+          // everything of the per-op row that needs no order statistic
+          const u64 kmin = ~x.n_kmin;
+          const u64 gi_ = row.group0 + so;
+          i64* __restrict__ gi = D.gi64 + gi_; u32* __restrict__ gu = D.gu32 + gi_;
+          const u32 span = x.xmax - emin;
+          gi[(u64)GI_E_MIN * G_all] = (i64)((u64)te0 - 0x80000000ull + emin); gi[(u64)GI_ARRIVAL_SKEW * G_all] = (i64)(u64)(x.emax - emin);
+          gi[(u64)GI_T_MAX * G_all] = (i64)(u64)tmx; gi[(u64)GI_T_MIN * G_all] = (i64)(u64)tmn; gi[(u64)GI_SPAN * G_all] = (i64)(u64)span;
+          gu[(u64)GU_RANK_TMIN * G_all] = mem[(u32)kmin]; gu[(u64)GU_RANK_TMAX * G_all] = mem[NONE - (u32)x.kmax];
+          gu[(u64)GU_MAX_CHG * G_all] = (u32)(x.ck >> 32); gu[(u64)GU_RANK_MAX_CHG * G_all] = mem[NONE - (u32)x.ck];
+          gu[(u64)GU_N_PRESENT * G_all] = n;
+          const bool mismatch = (x.bits & 2) != 0;
+          gu[(u64)GU_GFLAGS * G_all] = CCLD_G_COMPLETE | (barrier ? CCLD_G_BARRIER : 0) | (mismatch ? CCLD_G_OPSET_MISMATCH : 0) | (analysed ? CCLD_G_ANALYSED : 0);
+          D.gbw[gi_] = span ? bn * rcp_newton((double)span * den) : 0.0;
+          atomicAdd(&s_cnt[SC_COMP], 1u); atomicAdd(&s_cnt[SC_PRES], n);
+          if (barrier) atomicAdd(&s_cnt[SC_BAR], 1u);
+          if (analysed) { atomicAdd(&s_cnt[SC_AN], 1u); s_lead[g].an += 1; }
+          if (mismatch) atomicAdd(&s_cnt[SC_MIS], 1u);
+          if (!barrier) { LargeLead m = s_lead[g]; m.rounds += 1; best_merge(m.brng, m.bk, (u64)(tmx - tmn), so); s_lead[g] = m; }
+        }
       }
-    }
-    n_fs = __reduce_add_sync(0xFFFFFFFFu, n_fs); n_fd = __reduce_add_sync(0xFFFFFFFFu, n_fd);
-    if (lane == 0) { if (n_fs) atomicAdd(&s_cnt[SC_FS], n_fs); if (n_fd) atomicAdd(&s_cnt[SC_FD], n_fd); }
-    if (lead && gok) {
-      i64* __restrict__ gi = D.gi64 + row.group0 + so;
-      gi[(u64)GI_MED_SKEW * G_all] = (i64)(u64)ms; gi[(u64)GI_MAD_SKEW * G_all] = (i64)(u64)ds;
-      gi[(u64)GI_MED_DUR * G_all] = analysed ? (i64)((u64)tmn + md) : 0; gi[(u64)GI_MAD_DUR * G_all] = (i64)(u64)dm;
-    }
+      __syncthreads();
+      u32 bs = 0, bd = 0;
+      for (u32 q = 0; q < G; ++q) { bs = max(bs, s_bound[0][q]); bd = max(bd, s_bound[1][q]); }
+
+      // ---- order statistics, all groups of the sub-tile side by side; a thread's keys sit in registers during a select ----
+      u32 ms = 0, ds = 0, md = 0, dm = 0;
+      if (__syncthreads_or(analysed)) {
+        const u32 k = (n - 1) >> 1;
+        u32 v[LG_KEYS];
+        const u32* __restrict__ sk = D.skey + slot + pl; const u32* __restrict__ du = D.dkey + slot + pl;
+#pragma unroll
+        for (int q = 0; q < LG_KEYS; ++q) v[q] = (analysed && ((have >> q) & 1u)) ? sk[(u32)q * MP] - emin : 0u;
+        ms = large_select(v, have, analysed, k, top_byte(bs), G, g, s_hist, s_pick, s_krem);
+#pragma unroll
+        for (int q = 0; q < LG_KEYS; ++q) v[q] = __usad(v[q], ms, 0u);
+        ds = large_select(v, have, analysed, k, top_byte(bs), G, g, s_hist, s_pick, s_krem);
+#pragma unroll
+        for (int q = 0; q < LG_KEYS; ++q) v[q] = (analysed && ((have >> q) & 1u)) ? du[(u32)q * MP] - tmn : 0u;
+        md = large_select(v, have, analysed, k, top_byte(bd), G, g, s_hist, s_pick, s_krem);
+#pragma unroll
+        for (int q = 0; q < LG_KEYS; ++q) v[q] = __usad(v[q], md, 0u);
+        dm = large_select(v, have, analysed, k, top_byte(bd), G, g, s_hist, s_pick, s_krem);
+        if (!analysed) { ms = ds = md = dm = 0; }
+      }
+      if (lead) {
+        LargeScal z; z.ts = (u64)ds * P.k_milli; z.td = (u64)dm * P.k_milli; z.bn = bn; z.den = den;   // |x - med| * 1000 > k * MAD: both sides below 2^64
+        z.emin = emin; z.tmn = tmn; z.ms = ms; z.md = md; z.state = (gok ? 1u : 0u) | (analysed ? 2u : 0u) | (barrier ? 4u : 0u); z.pad = 0;
+        s_sc[g] = z;
+        if (gok) {
+          i64* __restrict__ gi = D.gi64 + row.group0 + so;
+          gi[(u64)GI_MED_SKEW * G_all] = (i64)(u64)ms; gi[(u64)GI_MAD_SKEW * G_all] = (i64)(u64)ds;
+          gi[(u64)GI_MED_DUR * G_all] = analysed ? (i64)((u64)tmn + md) : 0; gi[(u64)GI_MAD_DUR * G_all] = (i64)(u64)dm;
+        }
+      }
+      __syncthreads();
+
+      // ---- flags, votes, per-member bandwidth: a thread takes a member through the G groups ----
+      u32 n_fs = 0, n_fd = 0;
+      const u32 gcnt = t.count - j0 < G ? t.count - j0 : G;
+      const u64 slot0 = row.slot0 + (u64)(t.seq_off + j0) * n;
+      for (u32 p = threadIdx.x; p < n; p += LG_THREADS) {
+        double bwv = 0.0;
+        const u32 rank4 = mem[p] * 4;
+        for (u32 q = 0; q < gcnt; ++q) {
+          const LargeScal& z = s_sc[q];
+          if (!(z.state & 1)) continue;
+          const u64 o = slot0 + (u64)q * n + p;
+          const u32 d = D.dkey[o];
+          u32 f = CCLD_F_NOT_ANALYSED;
+          if (z.state & 2) {
+            const u32 skw = D.skey[o] - z.emin, dd = d - z.tmn;
+            const bool so_ = (u64)__usad(skw, z.ms, 0u) * 1000u > z.ts, shi = skw > z.ms;
+            const bool dq = (u64)__usad(dd, z.md, 0u) * 1000u > z.td, dhi = dd > z.md;
+            f = (so_ ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (shi ? CCLD_F_SKEW_HI : 0) | (dhi ? CCLD_F_DUR_HI : 0);
+            if (so_) { ++n_fs; atomicAdd(&R.votes[rank4 + (shi ? 0 : 1)], 1u); }
+            if (dq) { ++n_fd; atomicAdd(&R.votes[rank4 + (dhi ? 2 : 3)], 1u); }
+          }
+          D.flags[o] = (u8)f;
+          if (!(z.state & 4) && d != 0) bwv += z.bn * rcp_newton1((double)d * z.den);
+        }
+        s_bw[p] += bwv;
+      }
+      n_fs = __reduce_add_sync(0xFFFFFFFFu, n_fs); n_fd = __reduce_add_sync(0xFFFFFFFFu, n_fd);
+      if (lane == 0) { if (n_fs) atomicAdd(&s_cnt[SC_FS], n_fs); if (n_fd) atomicAdd(&s_cnt[SC_FD], n_fd); }
+    }  // sub-tiles
     __syncthreads();
-    for (u32 q = 0; q < G; ++q) cur_rounds += s_lead[q].rounds;
+    for (u32 q = 0; q < LARGE_SEQS; ++q) cur_rounds += s_lead[q].rounds;
     if (threadIdx.x == 0) {
       TileSum ts; ts.best_rng = 0; ts.best_k = NONE; ts.n_rounds = 0; ts.n_an = 0; ts.pad = 0;
-      for (u32 q = 0; q < G; ++q) { best_merge(ts.best_rng, ts.best_k, s_lead[q].brng, s_lead[q].bk); ts.n_rounds += s_lead[q].rounds; ts.n_an += s_lead[q].an; ts.pad += s_lead[q].def; }
+      for (u32 q = 0; q < LARGE_SEQS; ++q) { best_merge(ts.best_rng, ts.best_k, s_lead[q].brng, s_lead[q].bk); ts.n_rounds += s_lead[q].rounds; ts.n_an += s_lead[q].an; ts.pad += s_lead[q].def; }
       sums[ti] = ts;
       count_add(D.counters, C_COMPLETE, s_cnt[SC_COMP]); count_add(D.counters, C_BARRIER, s_cnt[SC_BAR]); count_add(D.counters, C_ANALYSED, s_cnt[SC_AN]);
       count_add(D.counters, C_MISMATCH, s_cnt[SC_MIS]); count_add(D.counters, C_PRESENT, s_cnt[SC_PRES]);
