@@ -245,6 +245,7 @@ int finalize_registry(ccld_ctx* ctx) {
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "scratch allocation failed");
 
   CK(cudaFuncSetAttribute(k_reduce_mid, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)mid_smem_bytes(2 * WARP_N)));
+  CK(cudaFuncSetAttribute(k_seq_range, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)range_smem_bytes(RANGE_DIRECT)));
   if (max_large) {
     ctx->large_smem = large_smem(max_large);
     CK(cudaFuncSetAttribute(k_reduce_large, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ctx->large_smem));
@@ -438,7 +439,7 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   auto take = [&](size_t b) { size_t o = off; off = align_up(off + b); return o; };
   const size_t o_desc = take(B * sizeof(WinDesc)), o_rmin = take((size_t)B * nc * 4), o_rmax = take((size_t)B * nc * 4),
                o_rng = take((size_t)B * nc * sizeof(RangeRow)), o_srow = take((size_t)B * nc * sizeof(uint4)), o_tot = take((size_t)B * T_COUNT * 8), o_cnt = take((size_t)B * C_COUNT * 8),
-               o_cta0 = take((size_t)B * 4);
+               o_end = take(0);
   cudaError_t e;
   Block pb = ctx->pool.get(off, &e);
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "plan allocation failed");
@@ -449,7 +450,7 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   for (u32 k = 0; k < B; ++k) {
     WinDesc d = ws[k]->d;
     d.slot_cap = 2 * d.n_rec + ctx->sum_n;
-    d.n_cta = (u32)((d.n_rec + REC_PER_CTA - 1) / REC_PER_CTA); d.cta0 = (u32)cta; cta += d.n_cta;
+    d.n_cta = (u32)((d.n_rec + REC_PER_CTA - 1) / REC_PER_CTA); d.cta0 = 0; cta = std::max<u64>(cta, d.n_cta);
     d.rmin = (u32*)(pbase + o_rmin) + (size_t)k * nc; d.rmax = (u32*)(pbase + o_rmax) + (size_t)k * nc;
     d.ranges = (RangeRow*)(pbase + o_rng) + (size_t)k * nc; d.srow = (uint4*)(pbase + o_srow) + (size_t)k * nc;
     d.totals = (u64*)(pbase + o_tot) + (size_t)k * T_COUNT; d.counters = (u64*)(pbase + o_cnt) + (size_t)k * C_COUNT;
@@ -464,12 +465,9 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   CK(cudaMemsetAsync(pbase, 0, off, st));
   CK(cudaMemsetAsync(pbase + o_rmin, 0xFF, (size_t)B * nc * 4, st));
   CK(cudaMemcpyAsync(d_desc, hd.data(), B * sizeof(WinDesc), cudaMemcpyHostToDevice, st));
-  std::vector<u32> h_cta0(B);
-  for (u32 k = 0; k < B; ++k) h_cta0[k] = hd[k].cta0;
-  u32* d_cta0 = (u32*)(pbase + o_cta0);
-  CK(cudaMemcpyAsync(d_cta0, h_cta0.data(), B * 4ull, cudaMemcpyHostToDevice, st));
+  (void)o_end;
   TimerSlot* ts = timer_begin(ctx);
-  if (cta > 0) { TimedLaunch tl(ts, 0, st); k_seq_range<<<(u32)cta, REC_THREADS, 0, st>>>(d_desc, d_cta0, B, ctx->reg); }
+  if (cta > 0) { TimedLaunch tl(ts, 0, st); k_seq_range<<<dim3((u32)cta, B), REC_THREADS, range_smem_bytes(nc), st>>>(d_desc, ctx->reg); }
   { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, PlanLists{nullptr, nullptr, nullptr, nullptr}, 0); }
   CK(cudaGetLastError());
   { int rc = ensure_pinned(ctx, (size_t)B * T_COUNT * 8); if (rc != CCLD_OK) return rc; }
@@ -521,7 +519,7 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   if (total_slots) CK(cudaMemsetAsync(rbase + o_perm, 0xFF, total_slots * 4, st));
   PlanLists pl; pl.fcta = (FusedCta*)(rbase + o_fcta); pl.fwt = (WarpTile*)(rbase + o_fwt); pl.t2 = (Tile*)(rbase + o_t2); pl.t3 = (Tile*)(rbase + o_t3);
   { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, pl, 1); }
-  if (cta > 0) { TimedLaunch tl(ts, 2, st); k_slot_scatter<<<(u32)cta, SCAT_THREADS, 0, st>>>(d_desc, d_cta0, B, ctx->reg); }
+  if (cta > 0) { TimedLaunch tl(ts, 2, st); k_slot_scatter<<<dim3((u32)cta, B), SCAT_THREADS, 0, st>>>(d_desc, ctx->reg); }
   CK(cudaMemsetAsync(rbase + o_defn, 0, 16, st));
   if (n_list[B_FCTA]) {
     const DeferList dl{(u64*)(rbase + o_def), (u32*)(rbase + o_defn)};

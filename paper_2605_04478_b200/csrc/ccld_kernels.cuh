@@ -47,18 +47,6 @@ __device__ __forceinline__ u32 pos_lookup(const Registry& R, u32 rank, u32 c) {
   return NONE;
 }
 
-// Which window of the batch a CTA of the record-streaming grids works on: the last window whose first CTA is <= cta.
-// cta0 is a compact copy of the descriptors' first-CTA fields (a few cache lines that every CTA hits in L1 / L2; the
-// descriptors themselves are a line apart each, and a search through them costs a chain of memory round trips per CTA).
-__device__ __forceinline__ u32 find_window(const u32* __restrict__ cta0, u32 nw, u32 cta) {
-  u32 lo = 0, hi = nw - 1;
-  while (lo < hi) {
-    u32 mid = (lo + hi + 1) >> 1;
-    if (__ldg(cta0 + mid) <= cta) lo = mid; else hi = mid - 1;
-  }
-  return lo;
-}
-
 // a * ka > b * kb in exact 128-bit arithmetic
 __device__ __forceinline__ bool mul_gt(u64 a, u32 ka, u64 b, u32 kb) {
   u64 alo = a * ka, ahi = __umul64hi(a, (u64)ka);
@@ -142,66 +130,118 @@ __device__ __forceinline__ void range_widen(const WinDesc& D, u32 c, u32 mn, u32
   if (mx > __ldcg(&D.rmax[c])) atomicMax(&D.rmax[c], mx);
 }
 
-constexpr u32 RANGE_TAB = 64;           // per-CTA table of the communicators met; overflow goes straight to global memory
+// A CTA keeps the op-counter extremes of every communicator it meets in a shared-memory table indexed by the
+// communicator's registry index (registries of up to RANGE_DIRECT communicators; beyond that updates go to global
+// memory, checked before each atomic) and merges the entries it touched into the window's global ranges at the end.
+constexpr u32 RANGE_DIRECT = 4096;
+inline size_t range_smem_bytes(u32 n_comms) { return n_comms <= RANGE_DIRECT ? (size_t)8 * n_comms : 0; }
 
-__device__ __forceinline__ void range_note(const WinDesc& D, u32* t_key, u32* t_mn, u32* t_mx, u32 c, u32 mn, u32 mx) {
-  u32 h = c & (RANGE_TAB - 1);
-  for (u32 probe = 0; probe < RANGE_TAB; ++probe) {
-    const u32 old = atomicCAS(&t_key[h], NONE, c);
-    if (old == NONE || old == c) { atomicMin(&t_mn[h], mn); atomicMax(&t_mx[h], mx); return; }
-    h = (h + 1) & (RANGE_TAB - 1);
-  }
-  range_widen(D, c, mn, mx);
+__device__ __forceinline__ void range_put(const WinDesc& D, u32* s_mn, u32* s_mx, u32 c, u32 mn, u32 mx) {
+  if (s_mn != nullptr) { atomicMin(&s_mn[c], mn); atomicMax(&s_mx[c], mx); }
+  else range_widen(D, c, mn, mx);
 }
 
 // ---- group-by, part 1: which op counters does every communicator cover in every window ----
-__global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __restrict__ wd, const u32* __restrict__ cta0, u32 nw, Registry R) {
-  __shared__ u32 s_comm[REC_THREADS * REC_PITCH], s_seq[REC_THREADS * REC_PITCH];
-  __shared__ u32 t_key[RANGE_TAB], t_mn[RANGE_TAB], t_mx[RANGE_TAB];
-  if (threadIdx.x < RANGE_TAB) { t_key[threadIdx.x] = NONE; t_mn[threadIdx.x] = NONE; t_mx[threadIdx.x] = 0; }
-  const u32 w = find_window(cta0, nw, blockIdx.x);
-  const WinDesc& D = wd[w];
-  const u64 first = (u64)(blockIdx.x - D.cta0) * REC_PER_CTA;
+// A thread takes a run of REC_RUN consecutive records. A rank's stream alternates between a handful of communicators, so
+// the thread folds its run in registers, one distinct communicator at a time (up to RANGE_FOLDS of them), and the warp
+// then merges what its lanes found - in a rank-major upload all lanes meet the same few communicators - so that one lane
+// updates the CTA's table per communicator. Records left over after the folds (an upload in arrival or random order)
+// look their communicator up and update the table themselves: one registry lookup and two shared-memory atomics per
+// record at worst.
+constexpr int RANGE_FOLDS = 4;
+
+__global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __restrict__ wd, Registry R) {
+  extern __shared__ u32 s_dyn[];
+  u32* const s_mn = R.n_comms <= RANGE_DIRECT ? s_dyn : nullptr;
+  u32* const s_mx = R.n_comms <= RANGE_DIRECT ? s_dyn + R.n_comms : nullptr;
+  const WinDesc& D = wd[blockIdx.y];                          // grid: (CTAs of the largest window, windows)
+  if (blockIdx.x >= D.n_cta) return;
+  const u64 first = (u64)blockIdx.x * REC_PER_CTA;
   const u32 n_valid = D.n_rec - first < REC_PER_CTA ? (u32)(D.n_rec - first) : (u32)REC_PER_CTA;
-  stage_column(D.comm, first, n_valid, s_comm);
-  stage_column(D.seq, first, n_valid, s_seq);
-  __syncthreads();
-  // Cached communicators: id, index (NONE = unregistered or empty entry), first valid counter, smallest / largest counter
-  // seen (empty: mn > mx). The walk itself is branch-free: a record updates the entry whose id it carries if its counter
-  // is valid; an empty entry has id NONE and index NONE, so a record that names communicator NONE lands nowhere.
-  u32 e_cid[RC], e_c[RC], e_s0[RC], e_mn[RC], e_mx[RC]; u32 next = 0;
-#pragma unroll
-  for (int e = 0; e < RC; ++e) { e_cid[e] = NONE; e_c[e] = NONE; e_s0[e] = NONE; e_mn[e] = NONE; e_mx[e] = 0; }
+  const u32 lane = threadIdx.x & 31;
   const u32 r0 = threadIdx.x * REC_RUN;
   const u32 len = r0 >= n_valid ? 0u : (n_valid - r0 < REC_RUN ? n_valid - r0 : (u32)REC_RUN);
-  const u32* pc = s_comm + threadIdx.x * REC_PITCH; const u32* ps = s_seq + threadIdx.x * REC_PITCH;
-#pragma unroll 4
-  for (u32 k = 0; k < len; ++k) {
-    const u32 cid = pc[k], sq = ps[k];
-    bool hit = false;
+  // the run goes straight into registers: four 128-bit loads per column where the column allows it
+  u32 cid[REC_RUN], sq[REC_RUN];
+  {
+    const u32* __restrict__ pc = D.comm + first + r0; const u32* __restrict__ ps = D.seq + first + r0;
+    if (len == REC_RUN && ((reinterpret_cast<uintptr_t>(pc) | reinterpret_cast<uintptr_t>(ps)) & 15) == 0) {
 #pragma unroll
-    for (int e = 0; e < RC; ++e) {
-      const bool h = e_cid[e] == cid, upd = h && sq >= e_s0[e];
-      e_mn[e] = upd ? min(e_mn[e], sq) : e_mn[e]; e_mx[e] = upd ? max(e_mx[e], sq) : e_mx[e];
-      hit = hit || h;
-    }
-    if (!hit) {
-      // the oldest entry makes room (its extremes go to the CTA's table)
-      u32 o_c = NONE, o_mn = NONE, o_mx = 0;
+      for (int q = 0; q < REC_RUN / 4; ++q) {
+        const uint4 a = __ldg(reinterpret_cast<const uint4*>(pc) + q), b = __ldg(reinterpret_cast<const uint4*>(ps) + q);
+        cid[4 * q] = a.x; cid[4 * q + 1] = a.y; cid[4 * q + 2] = a.z; cid[4 * q + 3] = a.w;
+        sq[4 * q] = b.x; sq[4 * q + 1] = b.y; sq[4 * q + 2] = b.z; sq[4 * q + 3] = b.w;
+      }
+    } else {
 #pragma unroll
-      for (int e = 0; e < RC; ++e) if ((u32)e == next) { o_c = e_c[e]; o_mn = e_mn[e]; o_mx = e_mx[e]; }
-      if (o_c != NONE && o_mn <= o_mx) range_note(D, t_key, t_mn, t_mx, o_c, o_mn, o_mx);
-      const uint4 h = comm_find(R, cid, R.hash[hash_home(R, cid)]);
-      const bool ok = h.y != NONE && sq >= h.z;
-#pragma unroll
-      for (int e = 0; e < RC; ++e) if ((u32)e == next) { e_cid[e] = cid; e_c[e] = h.y; e_s0[e] = h.y != NONE ? h.z : NONE; e_mn[e] = ok ? sq : NONE; e_mx[e] = ok ? sq : 0u; }
-      next = (next + 1) & (RC - 1);
+      for (int k = 0; k < REC_RUN; ++k) { cid[k] = (u32)k < len ? pc[k] : NONE; sq[k] = (u32)k < len ? ps[k] : 0u; }
     }
   }
+  if (s_mn != nullptr) {
+    for (u32 c = threadIdx.x; c < R.n_comms; c += REC_THREADS) { s_mn[c] = NONE; s_mx[c] = 0; }
+    __syncthreads();
+  }
+  // records of the run not yet accounted for; a run cut short by the end of the window skips the folds (its padding
+  // would match a record that names communicator 0xFFFFFFFF) and goes record by record
+  const u32 tail = len < REC_RUN ? (1u << len) - 1u : 0u;
+  u32 left = len < REC_RUN ? 0u : (1u << REC_RUN) - 1u;
+  // folds: the communicator of the first record still left takes every record of the run that names it
+  for (int f = 0; f < RANGE_FOLDS && __any_sync(0xFFFFFFFFu, left != 0); ++f) {
+    const bool act = left != 0;
+    u32 id = NONE;
 #pragma unroll
-  for (int e = 0; e < RC; ++e) if (e_c[e] != NONE && e_mn[e] <= e_mx[e]) range_note(D, t_key, t_mn, t_mx, e_c[e], e_mn[e], e_mx[e]);
+    for (int k = REC_RUN - 1; k >= 0; --k) id = (left >> k) & 1u ? cid[k] : id;
+    uint4 h = make_uint4(0, NONE, 0, 0);                      // (id, index, first counter, members); index NONE: unregistered
+    if (act) h = comm_find(R, id, R.hash[hash_home(R, id)]);
+    const u32 s0 = h.y != NONE ? h.z : NONE;                  // no counter passes an unregistered communicator's test
+    u32 m = 0, mn = NONE, mx = 0;
+#pragma unroll
+    for (int k = 0; k < REC_RUN; ++k) {
+      const bool e = ((left >> k) & 1u) && cid[k] == id;
+      m |= (e ? 1u : 0u) << k;
+      const bool ok = e && sq[k] >= s0;
+      mn = ok ? min(mn, sq[k]) : mn; mx = ok ? max(mx, sq[k]) : mx;
+    }
+    left &= ~m;
+    // lanes that hold the same communicator merge: a few rounds, each led by the lowest lane still waiting
+    bool mine = act && h.y != NONE && mn <= mx;
+    u32 pend = __ballot_sync(0xFFFFFFFFu, mine);
+    for (int it = 0; it < RANGE_FOLDS && pend; ++it) {
+      const u32 leader = (u32)__ffs(pend) - 1u;
+      const u32 lid = __shfl_sync(0xFFFFFFFFu, h.y, leader);
+      const bool same = mine && h.y == lid;
+      const u32 a = __reduce_min_sync(0xFFFFFFFFu, same ? mn : NONE), b = __reduce_max_sync(0xFFFFFFFFu, same ? mx : 0u);
+      if (lane == leader) range_put(D, s_mn, s_mx, lid, a, b);
+      if (same) mine = false;
+      pend &= ~__ballot_sync(0xFFFFFFFFu, same);
+    }
+    if (mine) range_put(D, s_mn, s_mx, h.y, mn, mx);
+  }
+  // every record still left: one lookup each, four in flight
+  left |= tail;
+  if (left != 0) {
+#pragma unroll
+    for (int k0 = 0; k0 < REC_RUN; k0 += 4) {
+      uint4 h[4]; bool need[4];
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        need[q] = ((left >> (k0 + q)) & 1u) != 0;
+        h[q] = need[q] ? R.hash[hash_home(R, cid[k0 + q])] : make_uint4(0, NONE, 0, 0);
+      }
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        if (!need[q]) continue;
+        const uint4 e = comm_find(R, cid[k0 + q], h[q]);
+        if (e.y != NONE && sq[k0 + q] >= e.z) range_put(D, s_mn, s_mx, e.y, sq[k0 + q], sq[k0 + q]);
+      }
+    }
+  }
+  if (s_mn == nullptr) return;
   __syncthreads();
-  if (threadIdx.x < RANGE_TAB && t_key[threadIdx.x] != NONE) range_widen(D, t_key[threadIdx.x], t_mn[threadIdx.x], t_mx[threadIdx.x]);
+  for (u32 c = threadIdx.x; c < R.n_comms; c += REC_THREADS) {
+    const u32 mn = s_mn[c];
+    if (mn != NONE) range_widen(D, c, mn, s_mx[c]);
+  }
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -472,63 +512,98 @@ __device__ __noinline__ u64 resolve_slow(const Registry& R, u32 rank, u32 cid) {
   return (c << RANK_TAB_POS_BITS) | pos;
 }
 
-// four CTAs per SM (64 registers): the kernel waits on its dependent table loads, so resident warps are what it needs
-__global__ void __launch_bounds__(SCAT_THREADS, 4) k_slot_scatter(const WinDesc* __restrict__ wd, const u32* __restrict__ cta0, u32 nw, Registry R) {
-  const u32 w = find_window(cta0, nw, blockIdx.x);
-  const WinDesc& D = wd[w];
-  const u64 base = (u64)(blockIdx.x - D.cta0) * REC_PER_CTA;
+// Where the record (rank, communicator id, op counter) goes, given the communicator's index c, the member's position
+// and the scatter row of c. Returns false if nothing is stored; *err / *rej / *internal collect what went wrong.
+__device__ __forceinline__ bool scatter_slot(const Registry& R, u32 c, u32 ns, u32 lo, u64 base_pos, u32 sq, u64 n_slots, u64* slot,
+                                             u32* err, u32* rej, u32* internal) {
+  if (ns == 0 || sq < lo) {
+    if (sq < R.comm_seq0[c]) { *err |= CCLD_E_SEQ_RANGE; ++*rej; }
+    else if (ns != 0) *internal = 1;
+    return false;
+  }
+  *slot = base_pos + (sq - lo);
+  if (sq - lo >= ns || *slot >= n_slots) { *internal = 1; return false; }
+  return true;
+}
+
+constexpr u32 SCAT_LOCAL = 4;     // ranks, counted from the rank of the CTA's first record, whose table rows a CTA resolves once
+
+// A CTA's records mostly belong to a few neighbouring ranks (a rank-major upload: one or two), so the CTA first resolves
+// the inline table rows of SCAT_LOCAL ranks - communicator id -> (counters covered, first counter, slot of the member's
+// first counter) - into shared memory; a record of those ranks then needs no global table at all and, in windows of
+// fewer than 2^32 slots, only 32-bit arithmetic. Any other record (another rank, a communicator beyond the inline pairs,
+// a counter outside the range, a rejected record) takes the two dependent table loads and the full checks.
+__global__ void __launch_bounds__(SCAT_THREADS, 4) k_slot_scatter(const WinDesc* __restrict__ wd, Registry R) {
+  __shared__ uint4 s_ent[SCAT_LOCAL * RANK_TAB_K];       // (communicator id, counters covered, first counter, first slot); counters covered 0: unused
+  const WinDesc& D = wd[blockIdx.y];                          // grid: (CTAs of the largest window, windows)
+  if (blockIdx.x >= D.n_cta) return;
+  const u64 base = (u64)blockIdx.x * REC_PER_CTA;
   u32 err = 0, rej = 0, internal = 0;
   // descriptor fields in registers: the stores below could alias the descriptor as far as the compiler knows
   u32* const perm = D.perm; const u64 n_slots = D.n_slots; const uint4* const srow = D.srow; const u64 n_rec = D.n_rec;
   const u32 *c_rank = D.rank, *c_comm = D.comm, *c_seq = D.seq;
-  constexpr int HALF = SCAT_PER_THREAD / 2;
+  // the records first: their loads are in flight while the table rows are resolved
+  u32 rk[SCAT_PER_THREAD], cid[SCAT_PER_THREAD], sq[SCAT_PER_THREAD];
+  u32 todo = 0;                                             // records that still need placing
 #pragma unroll
-  for (int h = 0; h < 2; ++h) {
-    u32 rk[HALF], cid[HALF], sq[HALF]; bool in[HALF];
-#pragma unroll
-    for (int k = 0; k < HALF; ++k) {
-      const u64 i = base + (u64)(h * HALF + k) * SCAT_THREADS + threadIdx.x;
-      in[k] = i < n_rec;
-      rk[k] = in[k] ? c_rank[i] : 0u; cid[k] = in[k] ? c_comm[i] : 0u; sq[k] = in[k] ? c_seq[i] : 0u;
+  for (int k = 0; k < SCAT_PER_THREAD; ++k) {
+    const u64 i = base + (u64)k * SCAT_THREADS + threadIdx.x;
+    const bool in = i < n_rec;
+    rk[k] = in ? c_rank[i] : 0u; cid[k] = in ? c_comm[i] : 0u; sq[k] = in ? c_seq[i] : 0u;
+    if (in) todo |= 1u << k;
+  }
+  const u32 r_first = c_rank[base];
+  if (threadIdx.x < SCAT_LOCAL * RANK_TAB_K) {
+    const u32 r = r_first + threadIdx.x / RANK_TAB_K, k = threadIdx.x % RANK_TAB_K;
+    uint4 e = make_uint4(NONE, 0, 0, 0);
+    if (n_slots <= 0xFFFFFFFFull && r_first < R.n_ranks && r < R.n_ranks) {
+      const uint4 t = R.rank_tab[(u64)r * 2 + (k >> 1)];
+      const u32 id = (k & 1) ? t.z : t.x, cp = (k & 1) ? t.w : t.y;
+      if (id != NONE && cp != NONE && cp != RANK_TAB_OVERFLOW) {
+        const uint4 sr = srow[cp >> RANK_TAB_POS_BITS];
+        const u64 b = ((u64)sr.x | ((u64)sr.y << 32)) + (u64)(cp & ((1u << RANK_TAB_POS_BITS) - 1)) * sr.z;
+        if (b + sr.z <= n_slots) e = make_uint4(id, sr.z, sr.w, (u32)b);    // the member's whole column lies inside the table
+      }
     }
-    uint4 ta[HALF], tb[HALF];
+    s_ent[threadIdx.x] = e;
+  }
+  __syncthreads();
 #pragma unroll
-    for (int k = 0; k < HALF; ++k) {
-      const u32 r = rk[k] < R.n_ranks ? rk[k] : 0u;
-      ta[k] = R.rank_tab[(u64)r * 2]; tb[k] = R.rank_tab[(u64)r * 2 + 1];
+  for (int k = 0; k < SCAT_PER_THREAD; ++k) {
+    const u32 dr = rk[k] - r_first;
+    if (dr < SCAT_LOCAL) {
+      const uint4* ent = s_ent + dr * RANK_TAB_K;
+      uint4 e = ent[0];
+#pragma unroll
+      for (int q = 1; q < RANK_TAB_K; ++q) { const uint4 x = ent[q]; if (x.x == cid[k]) e = x; }
+      const u32 off = sq[k] - e.z;                            // below the first counter: wraps to a huge value
+      if (e.x == cid[k] && off < e.y && ((todo >> k) & 1u)) {
+        perm[e.w + off] = (u32)base + (u32)k * SCAT_THREADS + threadIdx.x;
+        todo &= ~(1u << k);
+      }
     }
-    u32 cp[HALF];                              // index << 13 | position, NONE if the record is rejected
+  }
+  if (__any_sync(0xFFFFFFFFu, todo != 0)) {
 #pragma unroll
-    for (int k = 0; k < HALF; ++k) {
+    for (int k = 0; k < SCAT_PER_THREAD; ++k) {
+      if (!((todo >> k) & 1u)) continue;
       u32 v = NONE;
       if (rk[k] < R.n_ranks) {
-        v = ta[k].x == cid[k] ? ta[k].y : v; v = ta[k].z == cid[k] ? ta[k].w : v;
-        v = tb[k].x == cid[k] ? tb[k].y : v; v = tb[k].z == cid[k] ? tb[k].w : v;
+        const uint4 ta = R.rank_tab[(u64)rk[k] * 2], tb = R.rank_tab[(u64)rk[k] * 2 + 1];
+        v = ta.x == cid[k] ? ta.y : v; v = ta.z == cid[k] ? ta.w : v;
+        v = tb.x == cid[k] ? tb.y : v; v = tb.z == cid[k] ? tb.w : v;
       }
-      if (in[k] && (v == NONE || cid[k] == NONE)) {
+      if (v == NONE || v == RANK_TAB_OVERFLOW || cid[k] == NONE) {
         const u64 rs = resolve_slow(R, rk[k], cid[k]);
         v = (u32)rs;
         if (rs >> 32) { err |= (u32)(rs >> 32); ++rej; }
       }
-      cp[k] = in[k] ? v : NONE;
-    }
-    uint4 sr[HALF];
-#pragma unroll
-    for (int k = 0; k < HALF; ++k) sr[k] = cp[k] != NONE ? srow[cp[k] >> RANK_TAB_POS_BITS] : make_uint4(0, 0, 0, 0);
-#pragma unroll
-    for (int k = 0; k < HALF; ++k) {
-      if (cp[k] != NONE) {
-        const u32 ns = sr[k].z, lo = sr[k].w;
-        if (ns == 0 || sq[k] < lo) {
-          if (sq[k] < R.comm_seq0[cp[k] >> RANK_TAB_POS_BITS]) { err |= CCLD_E_SEQ_RANGE; ++rej; }
-          else if (ns != 0) internal = 1;
-        } else {
-          const u64 sb = (u64)sr[k].x | ((u64)sr[k].y << 32);
-          const u64 slot = sb + (u64)(cp[k] & ((1u << RANK_TAB_POS_BITS) - 1)) * ns + (sq[k] - lo);
-          if (sq[k] - lo >= ns || slot >= n_slots) internal = 1;
-          else perm[slot] = (u32)(base + (u64)(h * HALF + k) * SCAT_THREADS + threadIdx.x);
-        }
-      }
+      if (v == NONE) continue;
+      const u32 c = v >> RANK_TAB_POS_BITS;
+      const uint4 sr = srow[c];
+      u64 slot;
+      if (scatter_slot(R, c, sr.z, sr.w, ((u64)sr.x | ((u64)sr.y << 32)) + (u64)(v & ((1u << RANK_TAB_POS_BITS) - 1)) * sr.z, sq[k], n_slots, &slot, &err, &rej, &internal))
+        perm[slot] = (u32)(base + (u64)k * SCAT_THREADS + threadIdx.x);
     }
   }
   err = __reduce_or_sync(0xFFFFFFFFu, err);
