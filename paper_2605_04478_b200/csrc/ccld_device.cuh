@@ -21,7 +21,11 @@ constexpr int REC_THREADS = 128;       // record-streaming kernels: threads per 
 constexpr int REC_PER_THREAD = 16;     //   each walks a run of consecutive records
 constexpr int REC_PER_CTA = REC_THREADS * REC_PER_THREAD;
 constexpr int SMALL_N = 8;             // communicators of up to 8 ranks: one thread per group
-constexpr int SMALL_SEQS = 256;        //   threads per CTA: eight warp-tiles of up to 32 op counters
+constexpr int SMALL_SEQS = 256;        //   threads per CTA: eight warps, each on a warp-tile of up to 32 op counters at a time
+#ifndef CCLD_FUSED_WT_PER_CTA
+#define CCLD_FUSED_WT_PER_CTA 16
+#endif
+constexpr u32 FUSED_WT_PER_CTA = CCLD_FUSED_WT_PER_CTA;   //   warp-tiles a CTA works through (a multiple of its eight warps)
 constexpr int WARP_N = 128;            // up to 128 ranks: one warp per group, bitonic sort in registers
 constexpr int MID_N = 1024;            // up to 1024 ranks: shared-memory bitonic sort, several groups per CTA
 constexpr int MID_THREADS = 256;

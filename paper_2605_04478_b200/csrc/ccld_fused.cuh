@@ -176,21 +176,118 @@ struct FusedShared {
   u32 comm[SMALL_SEQS / 32], rounds[SMALL_SEQS / 32], n_an[SMALL_SEQS / 32], n_def[SMALL_SEQS / 32], brng[SMALL_SEQS / 32], bk[SMALL_SEQS / 32];
   u32 cnt[SC_COUNT];
   OutPtrs out;
-  u32 stage[16][SMALL_SEQS];   // per thread (column): eight enter-time offsets, eight durations
+  // n <= 32: per thread (column) eight enter-time offsets and eight durations. 33 <= n <= 128: the tile's keys as
+  // [metric][member][op counter], pitch S + 1 (S = op counters per tile), written by the staging phase of the tile.
+  u32 stage[2 * (MID_ELEMS + WARP_N)];
+  u64 t_base[32], t_gby[32], t_ck[SMALL_SEQS / 32][32];       // staged tiles, per op counter: time base, size of the op, most changes per warp
+  u32 t_gop[32], t_bits[32];                                  //   op code; 1 = some record disqualifies the group, 2 = the op set differs
 };
+constexpr u32 STAGE_ROWS = SMALL_SEQS;                        // row pitch of the per-thread layout
+
+// Staging phase of a tile of a communicator of 33 to 128 ranks (S = 2048 / n_pad op counters, S <= 32): the CTA's warps
+// share the members, lanes run along the op counter, so the record indices of a warp step are one contiguous piece of
+// the member-major permutation and - in a rank-major upload - the records themselves lie in one short stretch of a
+// rank's stream instead of one sector per lane. Times become 32-bit keys against the group's first member (whose enter
+// time, size and op code every thread loads for its own op counter), the op-set check and the rate column are reduced on
+// the way; the keys land in shared memory as [metric][member][op counter].
+template <int L>
+__device__ __forceinline__ void stage_tile(const WinDesc& D, const RangeRow& row, u32 seq0, u32 count, FusedShared& sh) {
+  constexpr u32 S = 32 / L * (SMALL_SEQS / 32), PITCH = S + 1, NW = SMALL_SEQS / 32;     // S op counters per tile: 32 (n_pad 64), 16 (n_pad 128)
+  constexpr u32 MPS = 32 / S;                                  // members a warp step covers
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5, n = row.n;
+  const u32 sq = lane & (S - 1), ml = lane / S;
+  const bool sv = sq < count;
+  const u32* __restrict__ perm = D.perm + row.slot0 + seq0 + (sv ? sq : 0u);
+  const i64* __restrict__ c_te = D.t_enter; const i64* __restrict__ c_tx = D.t_exit;
+  const u64* __restrict__ c_by = D.bytes; const u8* __restrict__ c_op = D.op;
+  const u32* __restrict__ c_sc = D.send_chg; const u32* __restrict__ c_rc = D.recv_chg;
+  u32 bits = 0; i64 te0 = 0; u64 by0 = 0; u32 op0 = 0;
+  {
+    const u32 i0 = sv ? __ldg(perm) : NONE;
+    if (i0 != NONE) { te0 = c_te[i0]; by0 = c_by[i0]; op0 = c_op[i0]; } else bits = 1;
+  }
+  const u64 base = (u64)te0 - 0x80000000ull;
+  u64 ck = 0;
+  u32* __restrict__ k_a = sh.stage; u32* __restrict__ k_d = sh.stage + (MID_ELEMS + WARP_N);
+  // member of warp step i: wid * MPS + ml + i * NW * MPS
+  for (u32 p0 = wid * MPS + ml; p0 < n; p0 += 4 * NW * MPS) {
+    u32 idx[4]; i64 x[4], y[4]; u64 by[4]; u32 op[4], ch[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) { const u32 p = p0 + q * NW * MPS; idx[q] = (sv && p < n) ? __ldg(perm + (u64)p * row.n_seq) : NONE; }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const u32 ix = idx[q] == NONE ? 0u : idx[q];
+      x[q] = c_te[ix]; y[q] = c_tx[ix]; by[q] = c_by[ix]; op[q] = c_op[ix]; ch[q] = 0;
+      if (c_sc != nullptr) { const u32 sc = c_sc[ix], rc = c_rc[ix]; ch[q] = max(sc, rc); }
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      const u32 p = p0 + q * NW * MPS;
+      if (p < n) {
+        u32 a_lo = 0, d = 0;
+        if (idx[q] == NONE) { if (sv) bits |= 1; }
+        else {
+          const u64 ra = (u64)x[q] - base, rb = (u64)y[q] - base;
+          a_lo = (u32)ra; const u32 b_lo = (u32)rb; d = b_lo - a_lo;
+          if (((ra | rb) >> 32) != 0 || (x[q] | y[q]) < 0 || b_lo < a_lo) bits |= 1;     // beyond 32 bits, negative or in flight, exit before enter
+          if (op[q] != op0 || by[q] != by0) bits |= 2;
+          const u64 k2 = ((u64)ch[q] << 32) | (u64)(NONE - p); ck = k2 > ck ? k2 : ck;     // most changes, then the lowest position
+        }
+        k_a[p * PITCH + sq] = a_lo; k_d[p * PITCH + sq] = d;
+      }
+    }
+  }
+  if (MPS > 1) {                                              // the lanes that share an op counter
+#pragma unroll
+    for (u32 h = S; h < 32; h <<= 1) { bits |= __shfl_xor_sync(FULLM, bits, h); const u64 o = shfl_xor64(ck, h); ck = o > ck ? o : ck; }
+  }
+  if (lane < S) {
+    sh.t_ck[wid][lane] = ck;
+    if (bits) atomicOr(&sh.t_bits[lane], bits);
+    if (wid == 0) { sh.t_base[lane] = base; sh.t_gby[lane] = by0; sh.t_gop[lane] = op0; }
+  }
+}
 
 // One group per L lanes, eight ring positions per lane (position s * 8 + q in lane s of the group); the warp takes
 // 32 / L consecutive op counters starting at offset seq0 of the communicator's range, `count` of them valid.
-// FULL: the communicator fills every position (n = 8 L).
-template <int L, bool FULL>
+// FULL: the communicator fills every position (n = 8 L). STAGED: the tile's keys and per-op values wait in shared memory
+// (stage_tile); jt0 = the warp's first op counter inside the tile.
+template <int L, bool FULL, bool STAGED = false>
 __device__ __forceinline__ void fast_groups(const WinDesc& D, u32 w_idx, const RangeRow& row, const u32* __restrict__ mem, u32 seq0, u32 count,
-                                            const Registry& R, const Params& P, const DeferList& DL, FusedShared& sh, FastAcc& acc, double (&bw)[8]) {
+                                            const Registry& R, const Params& P, const DeferList& DL, FusedShared& sh, FastAcc& acc, double (&bw)[8],
+                                            u32 jt0 = 0) {
   const u32 lane = threadIdx.x & 31, s = lane % L, j = lane / L, base_lane = lane - s, p0 = s * 8;
   const u32 gmask = L == 32 ? FULLM : (((1u << (L & 31)) - 1u) << base_lane);
   const u32 n = FULL ? (u32)(L * 8) : row.n;
   const bool active = j < count, lead = s == 0;
-  u32* __restrict__ my = &sh.stage[0][threadIdx.x];          // my[q * SMALL_SEQS]: offset of position q, my[(8 + q) * SMALL_SEQS]: duration
+  constexpr u32 S_T = STAGED ? 32 / L * (SMALL_SEQS / 32) : 1, PITCH = S_T + 1;
+  // where the keys of my eight positions are: a column of the per-thread layout, or rows of the staged tile
+  const u32 jt = STAGED ? (active ? jt0 + j : jt0) : 0u;
+  const u32* __restrict__ ka = STAGED ? sh.stage + p0 * PITCH + jt : &sh.stage[threadIdx.x];
+  const u32* __restrict__ kd = STAGED ? sh.stage + (MID_ELEMS + WARP_N) + p0 * PITCH + jt : &sh.stage[8 * STAGE_ROWS + threadIdx.x];
+  constexpr u32 KSTEP = STAGED ? PITCH : STAGE_ROWS;
+  u32* __restrict__ my = &sh.stage[threadIdx.x];              // my[q * SMALL_SEQS]: offset of position q, my[(8 + q) * SMALL_SEQS]: duration
 
+  bool ok = true;
+  u32 emin = 0xFFFFFFFFu, emax = 0, xmax = 0, tmx = 0, tmn = 0xFFFFFFFFu;
+  u64 base;
+  bool mm = false;
+  u64 gby, ck = 0; u32 gop;
+  if (STAGED) {
+    base = sh.t_base[jt]; gby = sh.t_gby[jt]; gop = sh.t_gop[jt];
+    const u32 bits = sh.t_bits[jt];
+    ok = !(bits & 1); mm = (bits & 2) != 0;
+#pragma unroll
+    for (int w = 0; w < SMALL_SEQS / 32; ++w) { const u64 o = sh.t_ck[w][jt]; ck = o > ck ? o : ck; }
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      if (FULL || p0 + q < n) {
+        const u32 a_lo = ka[q * KSTEP], d = kd[q * KSTEP];
+        emin = min(emin, a_lo); emax = max(emax, a_lo); xmax = max(xmax, a_lo + d);
+        tmx = max(tmx, d); tmn = min(tmn, d);
+      }
+    }
+  } else {
   // ---- record indices of my eight positions (member-major permutation: stride n_seq) ----
   u32 idx[8];
   {
@@ -198,13 +295,10 @@ __device__ __forceinline__ void fast_groups(const WinDesc& D, u32 w_idx, const R
 #pragma unroll
     for (int q = 0; q < 8; ++q) idx[q] = (active && (FULL || p0 + q < n)) ? __ldg(pm + (u64)q * row.n_seq) : NONE;
   }
-  bool ok = true;
 #pragma unroll
   for (int q = 0; q < 8; ++q) if ((FULL || p0 + q < n) && idx[q] == NONE) ok = false;      // a missing member: the group is deferred
 
   // ---- batch 1: times, turned into 32-bit offsets from (first member's enter time - 2^31 ns) as they arrive ----
-  u32 emin = 0xFFFFFFFFu, emax = 0, xmax = 0, tmx = 0, tmn = 0xFFFFFFFFu;
-  u64 base;
   {
     const i64* __restrict__ c_te = D.t_enter; const i64* __restrict__ c_tx = D.t_exit;
     i64 ta[8], tb[8];
@@ -228,8 +322,6 @@ __device__ __forceinline__ void fast_groups(const WinDesc& D, u32 w_idx, const R
     if (hx != 0 || (int)neg < 0) ok = false;       // beyond 32 bits, negative, or in flight (t_exit = -1)
   }
   // ---- batch 2: op set (every member against the group's first) and rate column ----
-  bool mm = false;
-  u64 gby, ck = 0; u32 gop;
   {
     const u64* __restrict__ c_by = D.bytes; const u8* __restrict__ c_op = D.op;
     const u32* __restrict__ c_sc = D.send_chg; const u32* __restrict__ c_rc = D.recv_chg;
@@ -251,6 +343,7 @@ __device__ __forceinline__ void fast_groups(const WinDesc& D, u32 w_idx, const R
       }
     }
   }
+  }
   // ---- the lanes of a group meet ----
   bool gok = active && ok;
   if (L > 1) { const u32 b_ok = __ballot_sync(FULLM, ok); gok = active && (b_ok & gmask) == gmask; }     // every lane votes
@@ -268,20 +361,20 @@ __device__ __forceinline__ void fast_groups(const WinDesc& D, u32 w_idx, const R
       emin = min(emin, __shfl_xor_sync(FULLM, emin, h)); emax = max(emax, __shfl_xor_sync(FULLM, emax, h));
       xmax = max(xmax, __shfl_xor_sync(FULLM, xmax, h));
       tmx = max(tmx, __shfl_xor_sync(FULLM, tmx, h)); tmn = min(tmn, __shfl_xor_sync(FULLM, tmn, h));
-      const u64 o = shfl_xor64(ck, h); ck = o > ck ? o : ck;
+      if (!STAGED) { const u64 o = shfl_xor64(ck, h); ck = o > ck ? o : ck; }
     }
   }
   // lowest position that holds the longest / shortest duration
   u32 pmax = NONE, pmin = NONE;
 #pragma unroll
   for (int q = 7; q >= 0; --q) {
-    if (FULL || p0 + q < n) { const u32 d = my[(8 + q) * SMALL_SEQS]; if (d == tmx) pmax = p0 + q; if (d == tmn) pmin = p0 + q; }
+    if (FULL || p0 + q < n) { const u32 d = kd[q * KSTEP]; if (d == tmx) pmax = p0 + q; if (d == tmn) pmin = p0 + q; }
   }
   bool mismatch = mm;
   if (L > 1) {
 #pragma unroll
     for (int h = 1; h < L; h <<= 1) { pmax = min(pmax, __shfl_xor_sync(FULLM, pmax, h)); pmin = min(pmin, __shfl_xor_sync(FULLM, pmin, h)); }
-    mismatch = (__ballot_sync(FULLM, mm) & gmask) != 0;
+    if (!STAGED) mismatch = (__ballot_sync(FULLM, mm) & gmask) != 0;
   }
   const bool barrier = gop == CCLD_OP_ALLREDUCE && gby < P.barrier_bytes;
   const bool analysed = gok && !barrier && n >= P.min_group;
@@ -291,10 +384,10 @@ __device__ __forceinline__ void fast_groups(const WinDesc& D, u32 w_idx, const R
   if (__any_sync(FULLM, analysed)) {
     u32 v[8];
 #pragma unroll
-    for (int q = 0; q < 8; ++q) v[q] = (FULL || p0 + q < n) ? my[q * SMALL_SEQS] - emin : 0xFFFFFFFFu;
+    for (int q = 0; q < 8; ++q) v[q] = (FULL || p0 + q < n) ? ka[q * KSTEP] - emin : 0xFFFFFFFFu;
     if (L == 1) median_mad8<u32>(v, n, &ms, &ds); else sub_median_mad<L, u32>(v, n, s, lane, &ms, &ds);
 #pragma unroll
-    for (int q = 0; q < 8; ++q) v[q] = (FULL || p0 + q < n) ? my[(8 + q) * SMALL_SEQS] - tmn : 0xFFFFFFFFu;
+    for (int q = 0; q < 8; ++q) v[q] = (FULL || p0 + q < n) ? kd[q * KSTEP] - tmn : 0xFFFFFFFFu;
     if (L == 1) median_mad8<u32>(v, n, &md, &dm); else sub_median_mad<L, u32>(v, n, s, lane, &md, &dm);
     if (!analysed) { ms = ds = md = dm = 0; }
   }
@@ -305,17 +398,19 @@ __device__ __forceinline__ void fast_groups(const WinDesc& D, u32 w_idx, const R
   const double bn = (double)gby * num;
   u32 f_lo = 0, f_hi = 0;                                   // my eight flag bytes
   {
-    // |x - med| * 1000 > k * MAD, exact in 64 bits: deviations and MADs are below 2^32
-    const u64 ts = (u64)ds * P.k_milli, td = (u64)dm * P.k_milli;
+    // |x - med| * 1000 > k * MAD, exact: deviations and MADs are below 2^32, so both sides fit 64 bits, and for whole
+    // numbers a * 1000 > T is a > floor(T / 1000); a quotient of 2^32 - 1 or more can never be exceeded
+    const u64 qs = (u64)ds * P.k_milli / 1000u, qd = (u64)dm * P.k_milli / 1000u;
+    const u32 ts = qs > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)qs, td = qd > 0xFFFFFFFFull ? 0xFFFFFFFFu : (u32)qd;
 #pragma unroll
     for (int q = 0; q < 8; ++q) {
       if (FULL || p0 + q < n) {
-        const u32 d = my[(8 + q) * SMALL_SEQS];
+        const u32 d = kd[q * KSTEP];
         u32 f = CCLD_F_NOT_ANALYSED;
         if (analysed) {
-          const u32 sk = my[q * SMALL_SEQS] - emin, dd = d - tmn;
-          const bool so = (u64)__usad(sk, ms, 0u) * 1000u > ts, shi = sk > ms;
-          const bool dq = (u64)__usad(dd, md, 0u) * 1000u > td, dhi = dd > md;
+          const u32 sk = ka[q * KSTEP] - emin, dd = d - tmn;
+          const bool so = __usad(sk, ms, 0u) > ts, shi = sk > ms;
+          const bool dq = __usad(dd, md, 0u) > td, dhi = dd > md;
           f = (so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (shi ? CCLD_F_SKEW_HI : 0) | (dhi ? CCLD_F_DUR_HI : 0);
           if (so) { acc.flagged += 1u; atomicAdd(&R.votes[(u64)mem[p0 + q] * 4 + (shi ? 0 : 1)], 1u); }
           if (dq) { acc.flagged += 1u << 16; atomicAdd(&R.votes[(u64)mem[p0 + q] * 4 + (dhi ? 2 : 3)], 1u); }
@@ -404,40 +499,34 @@ __device__ __forceinline__ void flush_counters(const WinDesc& D, const FusedShar
   count_add(D.counters, C_FLAG_SKEW, sh.cnt[SC_FS]); count_add(D.counters, C_FLAG_DUR, sh.cnt[SC_FD]);
 }
 
-// Class-0 CTA (n <= 8): eight warp-tiles of one window and one time chunk, each up to 32 consecutive op counters of
-// one communicator with its own summary entry.
+// Class-0 CTA (n <= 8): up to FUSED_WT_PER_CTA warp-tiles of one window and one time chunk, each up to 32 consecutive op
+// counters of one communicator with its own summary entry. A warp takes every eighth tile and meets the other warps
+// only at the end, so the warps of a CTA drift apart and one warp's gathers overlap another's arithmetic.
 __device__ __forceinline__ void fused_small_cta(const WinDesc& D, const FusedCta& t, const WarpTile* __restrict__ wts, TileSum* __restrict__ sums,
                                                 const Registry& R, const Params& P, const DeferList& DL, FusedShared& sh) {
   const u32 wid = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  if (threadIdx.x < SMALL_SEQS / 32) sh.comm[threadIdx.x] = NONE;
-  __syncthreads();
-  if (wid < t.wt_count) {
-    const WarpTile wt = wts[t.wt_first + wid];
+  __syncthreads();                                          // the CTA's counters are zero
+  for (u32 i = wid; i < t.wt_count; i += SMALL_SEQS / 32) {
+    const WarpTile wt = wts[t.wt_first + i];
     FastAcc acc; double bw[8];
     if (wt.row.n == SMALL_N) fast_groups<1, true>(D, t.w, wt.row, R.members + wt.moff, wt.seq_off, wt.count, R, P, DL, sh, acc, bw);
     else fast_groups<1, false>(D, t.w, wt.row, R.members + wt.moff, wt.seq_off, wt.count, R, P, DL, sh, acc, bw);
     warp_fold<1>(acc, bw, wt.row.n, sh);
     __syncwarp();
     if (lane == 0) {
-      sh.comm[wid] = wt.c;
       TileSum ts; ts.best_rng = sh.brng[wid]; ts.best_k = sh.bk[wid]; ts.n_rounds = sh.rounds[wid]; ts.n_an = sh.n_an[wid]; ts.pad = sh.n_def[wid];
       sums[wt.sum_idx] = ts;
     }
+    // per-rank bandwidth of the tile: lane m < n adds member m's sum
+    const u32 rounds = sh.rounds[wid];
+    if (lane < wt.row.n && rounds) {
+      const u32 rank = R.members[wt.moff + lane];
+      atomicAdd(&R.bw_sum[rank], sh.bw[wid][lane]); atomicAdd(&R.bw_cnt[rank], rounds);
+    }
+    __syncwarp();
   }
   __syncthreads();
   if (threadIdx.x == 0) flush_counters(D, sh);
-  // per-rank bandwidth: consecutive warp-tiles of one communicator are summed before the atomics
-  if (threadIdx.x < (SMALL_SEQS / 32) * SMALL_N) {
-    const u32 q0 = threadIdx.x >> 3, m = threadIdx.x & 7, c = sh.comm[q0];
-    if (c != NONE && (q0 == 0 || sh.comm[q0 - 1] != c) && m < R.comm_n[c]) {
-      double v = 0.0; u32 rounds = 0;
-      for (u32 q = q0; q < SMALL_SEQS / 32 && sh.comm[q] == c; ++q) { v += sh.bw[q][m]; rounds += sh.rounds[q]; }
-      if (rounds) {
-        const u32 rank = R.members[R.comm_moff[c] + m];
-        atomicAdd(&R.bw_sum[rank], v); atomicAdd(&R.bw_cnt[rank], rounds);
-      }
-    }
-  }
 }
 
 // Class-1 CTA (9 <= n <= 128): one tile of 2048 / n_pad consecutive op counters of one communicator, 32 / L per warp;
@@ -450,7 +539,15 @@ __device__ __forceinline__ void fused_sub_cta(const WinDesc& D, const FusedCta& 
   const u32 first = wid * GW;
   const u32 cnt = first < t.count ? (t.count - first < GW ? t.count - first : GW) : 0u;
   FastAcc acc; double bw[8];
-  if (n == (u32)(L * 8)) fast_groups<L, true>(D, t.w, t.row, R.members + t.moff, t.seq_off + first, cnt, R, P, DL, sh, acc, bw);
+  if (L >= 8) {
+    // the tile's records are gathered with lanes along the op counter and wait in shared memory as 32-bit keys
+    if (threadIdx.x < 32) sh.t_bits[threadIdx.x] = 0;
+    __syncthreads();
+    stage_tile<L>(D, t.row, t.seq_off, t.count, sh);
+    __syncthreads();
+    if (n == (u32)(L * 8)) fast_groups<L, true, true>(D, t.w, t.row, R.members + t.moff, t.seq_off + first, cnt, R, P, DL, sh, acc, bw, first);
+    else fast_groups<L, false, true>(D, t.w, t.row, R.members + t.moff, t.seq_off + first, cnt, R, P, DL, sh, acc, bw, first);
+  } else if (n == (u32)(L * 8)) fast_groups<L, true>(D, t.w, t.row, R.members + t.moff, t.seq_off + first, cnt, R, P, DL, sh, acc, bw);
   else fast_groups<L, false>(D, t.w, t.row, R.members + t.moff, t.seq_off + first, cnt, R, P, DL, sh, acc, bw);
   warp_fold<L>(acc, bw, n, sh);
   __syncthreads();

@@ -408,7 +408,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
         if (comm_class(n) == 0) wt += u; else c1 += u;
       }
       uint2 tot; plan_scan2(make_uint2(wt, c1), &tot, s_pair);
-      n_cta += ceil_div(tot.x, 8) + tot.y; n_wt += tot.x;
+      n_cta += ceil_div(tot.x, FUSED_WT_PER_CTA) + tot.y; n_wt += tot.x;
     }
     if (threadIdx.x == 0) {
       // op counters further apart than 2^31, or more slots than the cap: refuse the window
@@ -465,7 +465,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
       uint2 tot; plan_scan2(make_uint2(wt, 0), &tot, s_pair);
       wt_total = tot.x;
     }
-    const u32 n0 = ceil_div(wt_total, 8);
+    const u32 n0 = ceil_div(wt_total, FUSED_WT_PER_CTA);
     for (u32 c0 = 0; c0 < R.n_comms; c0 += PLAN_THREADS) {
       const u32 c = c0 + threadIdx.x;
       const u32 ns = plan_nseq(D, R, c), n = c < R.n_comms ? R.comm_n[c] : 1u, cls = comm_class(n);
@@ -487,7 +487,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
     for (u32 j = threadIdx.x; j < n0; j += PLAN_THREADS) {
       FusedCta x; x.w = blockIdx.x; x.cls = 0; x.c = 0; x.seq_off = 0; x.count = 0; x.sum_idx = 0; x.moff = 0;
       x.row = RangeRow{0, 0, 0, 0, 0, 0, 0, 0};
-      x.wt_first = wt_base + 8 * j; x.wt_count = wt_total - 8 * j < 8 ? wt_total - 8 * j : 8;
+      x.wt_first = wt_base + FUSED_WT_PER_CTA * j; x.wt_count = wt_total - FUSED_WT_PER_CTA * j < FUSED_WT_PER_CTA ? wt_total - FUSED_WT_PER_CTA * j : FUSED_WT_PER_CTA;
       L.fcta[cta_base + j] = x;
     }
     cta_base += n0 + c1_run; wt_base += wt_total;
