@@ -193,15 +193,20 @@ __global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __rest
     for (int k = REC_RUN - 1; k >= 0; --k) id = (left >> k) & 1u ? cid[k] : id;
     uint4 h = make_uint4(0, NONE, 0, 0);                      // (id, index, first counter, members); index NONE: unregistered
     if (act) h = comm_find(R, id, R.hash[hash_home(R, id)]);
-    const u32 s0 = h.y != NONE ? h.z : NONE;                  // no counter passes an unregistered communicator's test
+    // a record folded earlier carries another id, so matching the id is enough (the run is complete: no padding)
     u32 m = 0, mn = NONE, mx = 0;
 #pragma unroll
     for (int k = 0; k < REC_RUN; ++k) {
-      const bool e = ((left >> k) & 1u) && cid[k] == id;
-      m |= (e ? 1u : 0u) << k;
-      const bool ok = e && sq[k] >= s0;
-      mn = ok ? min(mn, sq[k]) : mn; mx = ok ? max(mx, sq[k]) : mx;
+      if (cid[k] == id) { m |= 1u << k; mn = min(mn, sq[k]); mx = max(mx, sq[k]); }
     }
+    m &= left;
+    if (h.y != NONE && m != 0 && mn < h.z) {
+      // counters below the communicator's first name no operation: fold again without them
+      mn = NONE; mx = 0;
+#pragma unroll
+      for (int k = 0; k < REC_RUN; ++k) if (((m >> k) & 1u) && sq[k] >= h.z) { mn = min(mn, sq[k]); mx = max(mx, sq[k]); }
+    }
+    if (m == 0) { mn = NONE; mx = 0; }
     left &= ~m;
     // lanes that hold the same communicator merge: a few rounds, each led by the lowest lane still waiting
     bool mine = act && h.y != NONE && mn <= mx;
