@@ -32,7 +32,7 @@ struct LargeScal { u64 ts, td; double bn, den; u32 emin, tmn, ms, md; u32 state,
 
 constexpr u32 LS_PITCH = LS_MEMBERS + 4;     // lanes (op counter 0..7, member 0..3) hit 32 distinct banks
 
-__global__ void __launch_bounds__(LS_THREADS) k_large_stage(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles, LargeGroup* __restrict__ grp, Registry R) {
+__global__ void __launch_bounds__(LS_THREADS, 4) k_large_stage(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles, LargeGroup* __restrict__ grp, Registry R) {
   __shared__ u32 s_a[LARGE_SEQS * LS_PITCH], s_d[LARGE_SEQS * LS_PITCH];
   __shared__ LargeGroup s_part[LS_THREADS / 32][LARGE_SEQS];
   const Tile t = tiles[blockIdx.x];
@@ -120,38 +120,37 @@ __global__ void __launch_bounds__(LS_THREADS) k_large_stage(const WinDesc* __res
   }
 }
 
-__device__ __forceinline__ int top_byte(u32 bound) { return bound == 0 ? 0 : (31 - __clz(bound)) >> 3; }
+constexpr u32 LG_DIGIT = 8, LG_BINS = 1u << LG_DIGIT;      // radix digit of the selects; one histogram of LG_BINS bins per group
 
-// The k-th smallest (0-based) of a group's keys, for every group of the sub-tile at once. A thread holds up to LG_KEYS
-// keys of its own group g in registers (bit q of `have` says whether slot q holds one); `act` says whether the group
-// takes part. Digits of 8 bits, most significant first, starting at byte `top` (the same for all groups). A thread counts
-// the keys that share the digit of its first candidate itself and adds them once - in the passes over high bytes nearly
-// all keys of a group agree - and adds the others one by one. Histograms must be zero on entry and are zero again on
-// return. All threads of the CTA call it.
-__device__ __forceinline__ u32 large_select(const u32 (&v)[LG_KEYS], u32 have, bool act, u32 k, int top, u32 G, u32 g,
+// The k-th smallest (0-based) of a group's keys, for every group of the sub-tile at once. A thread holds up to LG_KEYS keys
+// of its own group g in registers (bit q of `have` says whether slot q holds one); `act` says whether the group takes
+// part. Digits of LG_DIGIT bits, most significant first; the first digit starts at the highest bit of `bound`, the
+// largest key of any group, so that it splits the keys as finely as 256 bins can, and a key that drops out of the
+// running costs its thread next to nothing in the passes that follow. After a pass warp w scans and clears group w's
+// histogram and names the digit that holds the k-th key. Histograms must be zero on entry and are zero again on return.
+// All threads of the CTA call it.
+__device__ __forceinline__ u32 large_select(const u32 (&v)[LG_KEYS], u32 have, bool act, u32 k, u32 bound, u32 G, u32 g,
                                             u32* __restrict__ s_hist, u32* __restrict__ s_pick, u32* __restrict__ s_krem) {
   const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   if (threadIdx.x < G) s_krem[threadIdx.x] = k;
-  u32 prefix = 0, mask = 0;
-  u32* __restrict__ hist = s_hist + g * 256;
-  for (int b = top; b >= 0; --b) {
-    const u32 sh = 8u * (u32)b;
+  u32* __restrict__ hist = s_hist + g * LG_BINS;
+  u32 hi = 32 - (u32)__clz(bound | 1u);                      // bits still undecided: the result lies below 2^hi
+  u32 prefix = 0;                                            // the decided bits, already in place
+  while (hi > 0) {
+    const u32 sh = hi > LG_DIGIT ? hi - LG_DIGIT : 0u, w = hi - sh;       // this pass decides bits [sh, hi)
+    const u32 dmask = (1u << w) - 1u;
     if (act) {
       u32 cm = 0;
+      if (hi >= 32) cm = have;
+      else {
+        const u32 want = prefix >> hi;
 #pragma unroll
-      for (int q = 0; q < LG_KEYS; ++q) cm |= ((v[q] & mask) == prefix ? 1u : 0u) << q;
-      cm &= have;
+        for (int q = 0; q < LG_KEYS; ++q) cm |= ((v[q] >> hi) == want ? 1u : 0u) << q;
+        cm &= have;
+      }
       if (cm) {
-        u32 d0 = 0;
 #pragma unroll
-        for (int q = LG_KEYS - 1; q >= 0; --q) d0 = (cm >> q) & 1u ? (v[q] >> sh) & 255u : d0;      // digit of the first candidate
-        u32 c0 = 0;
-#pragma unroll
-        for (int q = 0; q < LG_KEYS; ++q) {
-          const u32 d = (v[q] >> sh) & 255u;
-          if ((cm >> q) & 1u) { if (d == d0) ++c0; else atomicAdd(&hist[d], 1u); }
-        }
-        atomicAdd(&hist[d0], c0);
+        for (int q = 0; q < LG_KEYS; ++q) if ((cm >> q) & 1u) atomicAdd(&hist[(v[q] >> sh) & dmask], 1u);
       }
     }
     __syncthreads();
@@ -159,7 +158,7 @@ __device__ __forceinline__ u32 large_select(const u32 (&v)[LG_KEYS], u32 have, b
       u32 loc[8], sum = 0;
       const u32 kr = s_krem[wid];
 #pragma unroll
-      for (int q = 0; q < 8; ++q) { loc[q] = s_hist[wid * 256 + lane * 8 + q]; sum += loc[q]; s_hist[wid * 256 + lane * 8 + q] = 0; }
+      for (int q = 0; q < 8; ++q) { loc[q] = s_hist[wid * LG_BINS + lane * 8 + q]; sum += loc[q]; s_hist[wid * LG_BINS + lane * 8 + q] = 0; }
       u32 inc = sum;
 #pragma unroll
       for (int d = 1; d < 32; d <<= 1) { const u32 o = __shfl_up_sync(0xFFFFFFFFu, inc, d); if (lane >= (u32)d) inc += o; }
@@ -174,19 +173,21 @@ __device__ __forceinline__ u32 large_select(const u32 (&v)[LG_KEYS], u32 have, b
       }
     }
     __syncthreads();
-    prefix |= s_pick[g] << sh; mask |= 0xFFu << sh;
+    prefix |= s_pick[g] << sh;
+    hi = sh;
   }
   return prefix;
 }
 
-inline size_t large_smem(u32 max_n) { return (size_t)8 * large_npad(max_n); }     // per-member bandwidth sums
+// dynamic shared memory of k_reduce_large: per-member bandwidth sums of the largest communicator
+inline size_t large_smem(u32 max_n) { return (size_t)8 * large_npad(max_n); }
 
 __global__ void __launch_bounds__(LG_THREADS, 2) k_reduce_large(const WinDesc* __restrict__ wd, const Tile* __restrict__ tiles, u32 n_tiles,
                                                                  const LargeGroup* __restrict__ grp, TileSum* __restrict__ sums,
                                                                  Registry R, Params P, DeferList DL) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   double* s_bw = (double*)smem_raw;
-  __shared__ u32 s_hist[LARGE_SEQS * 256];
+  __shared__ u32 s_hist[LARGE_SEQS * LG_BINS];
   __shared__ LargeScal s_sc[LARGE_SEQS];
   __shared__ LargeLead s_lead[LARGE_SEQS];
   __shared__ u32 s_cnt[SC_COUNT];
@@ -195,8 +196,7 @@ __global__ void __launch_bounds__(LG_THREADS, 2) k_reduce_large(const WinDesc* _
   const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   u32 cur_w = NONE, cur_c = NONE, cur_rounds = 0;            // whose bandwidth sums shared memory holds
   const u32* cur_mem = nullptr; u32 cur_n = 0;
-  for (u32 i = threadIdx.x; i < LARGE_SEQS * 256; i += LG_THREADS) s_hist[i] = 0;
-
+  for (u32 i = threadIdx.x; i < LARGE_SEQS * LG_BINS; i += LG_THREADS) s_hist[i] = 0;
   for (u32 ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
     const Tile t = tiles[ti];
     const WinDesc& D = wd[t.w];
@@ -212,6 +212,7 @@ __global__ void __launch_bounds__(LG_THREADS, 2) k_reduce_large(const WinDesc* _
     if (t.w != cur_w || c != cur_c) {
       // another communicator or window: the sums shared memory holds go out
       if (cur_rounds) for (u32 p = threadIdx.x; p < cur_n; p += LG_THREADS) { atomicAdd(&R.bw_sum[cur_mem[p]], s_bw[p]); atomicAdd(&R.bw_cnt[cur_mem[p]], cur_rounds); }
+      __syncthreads();
       cur_w = t.w; cur_c = c; cur_rounds = 0; cur_mem = mem; cur_n = n;
       for (u32 p = threadIdx.x; p < n; p += LG_THREADS) s_bw[p] = 0.0;
     }
@@ -276,16 +277,16 @@ __global__ void __launch_bounds__(LG_THREADS, 2) k_reduce_large(const WinDesc* _
         const u32* __restrict__ sk = D.skey + slot + pl; const u32* __restrict__ du = D.dkey + slot + pl;
 #pragma unroll
         for (int q = 0; q < LG_KEYS; ++q) v[q] = (analysed && ((have >> q) & 1u)) ? sk[(u32)q * MP] - emin : 0u;
-        ms = large_select(v, have, analysed, k, top_byte(bs), G, g, s_hist, s_pick, s_krem);
+        ms = large_select(v, have, analysed, k, bs, G, g, s_hist, s_pick, s_krem);
 #pragma unroll
         for (int q = 0; q < LG_KEYS; ++q) v[q] = __usad(v[q], ms, 0u);
-        ds = large_select(v, have, analysed, k, top_byte(bs), G, g, s_hist, s_pick, s_krem);
+        ds = large_select(v, have, analysed, k, bs, G, g, s_hist, s_pick, s_krem);
 #pragma unroll
         for (int q = 0; q < LG_KEYS; ++q) v[q] = (analysed && ((have >> q) & 1u)) ? du[(u32)q * MP] - tmn : 0u;
-        md = large_select(v, have, analysed, k, top_byte(bd), G, g, s_hist, s_pick, s_krem);
+        md = large_select(v, have, analysed, k, bd, G, g, s_hist, s_pick, s_krem);
 #pragma unroll
         for (int q = 0; q < LG_KEYS; ++q) v[q] = __usad(v[q], md, 0u);
-        dm = large_select(v, have, analysed, k, top_byte(bd), G, g, s_hist, s_pick, s_krem);
+        dm = large_select(v, have, analysed, k, bd, G, g, s_hist, s_pick, s_krem);
         if (!analysed) { ms = ds = md = dm = 0; }
       }
       if (lead) {
