@@ -167,13 +167,29 @@ int ccld_window_release(ccld_ctx* ctx, uint32_t window_id);
  * in that order: grouping by (communicator, op counter) (Sec. 4.2.1), per-op cross-rank
  * reductions, median/MAD flags, votes, then per communicator the window rules of Eq. 1-4 whose
  * state (baseline rounds, slow counter) carries from window to window. `now_ns` is the analyzer's
- * clock for the hang test. Work is enqueued on the context's stream; the call returns after
- * one short device round trip that sizes the result buffers.
+ * clock for the hang test. Work is enqueued on the context's stream.
+ * The first batch of a shape (the same record count in every window) waits, in the middle of the
+ * call, for one short device round trip that sizes the result buffers. A later batch of the same
+ * shape does not wait at all: its buffers are sized from the totals the shape had before, the
+ * call only enqueues and returns, and the layout pass checks the totals on the device. If they
+ * differ, that batch and every batch enqueued after it give up on the device without touching any
+ * state, and the next call that synchronizes anyway (ccld_get_verdict and the other result
+ * accessors, ccld_window_release, ccld_state_export, a batch of a new shape) analyses them again
+ * in order, this time waiting - results and their order are the same either way, only the time
+ * differs. ccld_set_speculation(ctx, 0) makes every call wait.
  * A window is refused (CCLD_E_CAPACITY in its verdict, nothing analysed) if the op counters seen
  * in it would need more than 2 * n_rec + (sum of communicator sizes) slots. A batch holds at most
  * 65,535 windows (CCLD_ERR_CAPACITY beyond).
  */
 int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows, int64_t now_ns);
+
+/*
+ * Whether ccld_analyze_window may size a batch from the totals its shape had before instead of
+ * waiting for the layout pass (Sec. 4.2.1 analyses one window per minute: a monitoring loop sees
+ * the same shape over and over). on = 0: always wait; on = 1 (the default): wait only for shapes
+ * not seen before. Batches still in doubt are settled first.
+ */
+int ccld_set_speculation(ccld_ctx* ctx, int on);
 
 /* Clears votes, per-communicator state and all window results (records stay uploaded). */
 int ccld_reset(ccld_ctx* ctx);

@@ -25,7 +25,7 @@ MAX_ALERTS_PER_WINDOW = 1024
 EXPORTS = ("ccld_params_default", "ccld_create", "ccld_destroy", "ccld_last_error", "ccld_comm_register",
            "ccld_trace_upload", "ccld_window_release", "ccld_analyze_window", "ccld_reset", "ccld_get_verdict",
            "ccld_locate_hang", "ccld_get_optable", "ccld_get_ranges", "ccld_get_rank_stats", "ccld_copy_to_host",
-           "ccld_timing_enable", "ccld_get_kernel_times", "ccld_ring_locate_static", "ccld_derive_rates", "ccld_locate_hangs", "ccld_state_export", "ccld_state_import", "ccld_trace_attach_opset", "ccld_opset_check",
+           "ccld_timing_enable", "ccld_get_kernel_times", "ccld_set_speculation", "ccld_ring_locate_static", "ccld_derive_rates", "ccld_locate_hangs", "ccld_state_export", "ccld_state_import", "ccld_trace_attach_opset", "ccld_opset_check",
            "ccld_comm_set_layers")
 STATIC_MAX_MEMBERS = 8192
 KERNEL_KINDS = ("k_seq_range", "k_plan", "k_slot_scatter", "k_reduce_fused", "k_reduce_mid", "k_reduce_large", "k_window_decide")
@@ -122,6 +122,7 @@ def load_library() -> C.CDLL:
         lib.ccld_window_release.argtypes = [C.c_void_p, C.c_uint32]
         lib.ccld_analyze_window.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_int64]
         lib.ccld_reset.argtypes = [C.c_void_p]
+        lib.ccld_set_speculation.argtypes = [C.c_void_p, C.c_int]
         lib.ccld_get_verdict.argtypes = [C.c_void_p, C.c_uint32, C.POINTER(Verdict)]
         lib.ccld_locate_hang.argtypes = [C.c_void_p, C.c_uint32, C.c_uint32, C.c_uint32, C.POINTER(HangVerdict)]
         lib.ccld_trace_attach_opset.argtypes = [C.c_void_p, C.c_uint32, C.c_int, C.c_void_p, C.c_void_p]
@@ -286,6 +287,9 @@ class Analyzer:
 
     def reset(self) -> None:
         self._check(self.lib.ccld_reset(self.h))
+
+    def set_speculation(self, on: bool) -> None:
+        self._check(self.lib.ccld_set_speculation(self.h, 1 if on else 0))
 
     @staticmethod
     def _records(buf, struct, count, cap):

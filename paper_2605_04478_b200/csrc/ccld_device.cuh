@@ -85,6 +85,7 @@ constexpr int N_CLASSES = 4;           // reduction code paths: n <= 8, <= 128, 
 constexpr u32 CHUNK_REF = 96;          // op counters per chunk of the busiest communicator of a window
 constexpr u32 CHUNK_MAX = 64;          // at most this many chunks per window (longer chunks beyond)
 enum { T_GROUPS = 0, T_SLOTS, T_FCTA, T_FWT, T_FSUM, T_TILES2, T_TILES3, T_ROWS, T_FAILED, T_CHUNKS, T_COUNT = 12 };
+constexpr u64 FAILED_CAPACITY = 1, FAILED_EXPECT = 2;      // T_FAILED: the window needs too many slots / its layout is not the expected one
 enum { B_FCTA = 0, B_FWT, B_FSUM, B_T2, B_T3, B_COUNT };
 
 struct Tile { u32 w, c, seq_off, count; };                 // classes 2 and 3: one CTA each; summary index = tile index
@@ -110,6 +111,8 @@ struct WinDesc {
   RangeRow* ranges;                  // [n_comms]
   uint4* srow;                       // [n_comms] scatter rows: (slot0 - seq_lo * n) low, high, n (0 = nothing to place), seq_lo
   u64* totals;                       // [T_COUNT]
+  const u64* expect;                 // [T_COUNT] totals the host sized this window's results for without waiting (null: it waited)
+  u32* poison;                       // set once a window's layout differs from what the host expected: every window planned later gives up too
   u64* counters;                     // [C_COUNT]
   // sized after the plan:
   u64 n_groups, n_slots;

@@ -73,6 +73,13 @@ struct WindowHost {
   WindowHost() { std::memset(&d, 0, sizeof d); std::memset(totals, 0, sizeof totals); }
 };
 
+// A batch that was enqueued on totals the host expected instead of waiting for the plan: its actual totals arrive in
+// pinned memory behind the batch's kernels and are checked at the next call that synchronizes anyway.
+struct PendingBatch { u32 first = 0, n = 0; i64 now = 0; u64* h_tot = nullptr; size_t h_bytes = 0; };
+// Totals of the last batches that were planned with a wait, by shape (record count of every window).
+struct ShapeEntry { std::vector<u64> n_rec; std::vector<u64> totals; };
+constexpr size_t SHAPE_CACHE = 4;
+
 constexpr u32 TIMER_RING = 32;
 constexpr int TIMER_PAIRS = CCLD_K_KINDS + 1;          // the layout kernel runs twice per call
 struct TimerSlot { cudaEvent_t a[TIMER_PAIRS], b[TIMER_PAIRS]; int kind[TIMER_PAIRS]; int n = 0; };
@@ -88,6 +95,8 @@ struct ccld_ctx {
   std::map<u32, WindowHost> windows;
   Pool pool; std::string err;
   u64* h_pinned = nullptr; size_t h_pinned_bytes = 0;
+  std::vector<PendingBatch> pending; std::vector<std::pair<u64*, size_t>> pinned_free; std::vector<ShapeEntry> shapes;
+  u32* d_poison = nullptr; int speculate = 1;
   // optional per-kernel timing: a ring of event pairs, harvested lazily
   bool timing = false; std::vector<TimerSlot> ring; u32 ring_next = 0;
   double t_ms[CCLD_K_KINDS]; u64 t_launches[CCLD_K_KINDS];
@@ -203,6 +212,7 @@ int finalize_registry(ccld_ctx* ctx) {
   const size_t o_trees = take(std::max<u32>(n_trees, 1) * sizeof(TreeRef));
   const size_t o_stats = off;
   const size_t o_state = take(nc * sizeof(CommState)), o_votes = take(nr * 16ull), o_ops = take(nr * 4ull), o_cnt = take(nr * 4ull), o_bw = take(nr * 8ull);
+  const size_t stats_end = off, o_poison = take(256);
   cudaError_t e;
   ctx->reg_blk = ctx->pool.get(off, &e);
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "registry allocation failed");
@@ -237,7 +247,7 @@ int finalize_registry(ccld_ctx* ctx) {
   R.rank_ptr = (const u32*)(base + o_ptr); R.ent_comm = (const u32*)(base + o_ec); R.ent_pos = (const u32*)(base + o_ep);
   R.state = (CommState*)(base + o_state); R.votes = (u32*)(base + o_votes); R.ops = (u32*)(base + o_ops);
   R.bw_cnt = (u32*)(base + o_cnt); R.bw_sum = (double*)(base + o_bw);
-  ctx->stats_off = o_stats; ctx->stats_bytes = off - o_stats;
+  ctx->stats_off = o_stats; ctx->stats_bytes = stats_end - o_stats; ctx->d_poison = (u32*)(base + o_poison);
   ctx->n_ranks = nr; ctx->max_n = max_n; ctx->max_large_n = max_large; ctx->sum_n = sum_n;
 
   // scratch for suspects, alert ordering and hang location
@@ -260,7 +270,62 @@ void drop_results(WindowHost& w) {
   std::memset(w.totals, 0, sizeof w.totals);
 }
 
+int analyze_batch(ccld_ctx* ctx, u32 first_window, u32 n_windows, i64 now_ns, bool may_speculate);
+
+u64* pinned_get(ccld_ctx* ctx, size_t bytes, size_t* got) {
+  for (size_t i = 0; i < ctx->pinned_free.size(); ++i)
+    if (ctx->pinned_free[i].second >= bytes) { auto p = ctx->pinned_free[i]; ctx->pinned_free.erase(ctx->pinned_free.begin() + i); *got = p.second; return p.first; }
+  u64* p = nullptr;
+  if (cudaMallocHost((void**)&p, bytes) != cudaSuccess) return nullptr;
+  *got = bytes;
+  return p;
+}
+
+// Brings the batches that were enqueued on expected totals to a definite state: waits for the stream, reads the totals
+// their plans really found, and analyses again - this time waiting for the plan - every batch from the first one whose
+// expectation failed (that batch and all later ones gave up on the device without touching any state, so the order of
+// the windows is kept). Every call that hands out results or changes state goes through here first.
+int settle(ccld_ctx* ctx) {
+  if (ctx->pending.empty()) return CCLD_OK;
+  CK(cudaSetDevice(ctx->device));
+  CK(cudaStreamSynchronize(ctx->stream));
+  std::vector<PendingBatch> todo;
+  todo.swap(ctx->pending);
+  bool failed = false;
+  int rc = CCLD_OK;
+  for (PendingBatch& b : todo) {
+    for (u32 k = 0; k < b.n && !failed; ++k) if (b.h_tot[(size_t)k * T_COUNT + T_FAILED] == FAILED_EXPECT) failed = true;
+    ctx->pinned_free.emplace_back(b.h_tot, b.h_bytes);
+    if (!failed) {
+      // a window may still have been refused for its size, which the expectation cannot have foreseen: keep what the plan found
+      for (u32 k = 0; k < b.n; ++k) {
+        auto it = ctx->windows.find(b.first + k);
+        if (it != ctx->windows.end() && it->second.analysed) std::memcpy(it->second.totals, b.h_tot + (size_t)k * T_COUNT, sizeof it->second.totals);
+      }
+      continue;
+    }
+  }
+  if (!failed) return CCLD_OK;
+  CK(cudaMemsetAsync(ctx->d_poison, 0, 4, ctx->stream));
+  failed = false;
+  for (PendingBatch& b : todo) {
+    if (!failed) { for (u32 k = 0; k < b.n && !failed; ++k) if (b.h_tot[(size_t)k * T_COUNT + T_FAILED] == FAILED_EXPECT) failed = true; }
+    if (!failed) continue;
+    bool present = true;
+    for (u32 k = 0; k < b.n; ++k) {
+      auto it = ctx->windows.find(b.first + k);
+      if (it == ctx->windows.end()) { present = false; continue; }
+      drop_results(it->second);
+    }
+    if (!present) continue;                                // released in the meantime: nothing to analyse
+    const int r = analyze_batch(ctx, b.first, b.n, b.now, false);
+    if (r != CCLD_OK && rc == CCLD_OK) rc = r;
+  }
+  return rc;
+}
+
 int find_analysed(ccld_ctx* ctx, u32 wid, WindowHost** out) {
+  { int rc = settle(ctx); if (rc != CCLD_OK) return rc; }
   auto it = ctx->windows.find(wid);
   if (it == ctx->windows.end()) return fail(ctx, CCLD_ERR_NO_WINDOW, "unknown window id");
   if (!it->second.analysed) return fail(ctx, CCLD_ERR_NO_WINDOW, "window not analysed");
@@ -308,6 +373,8 @@ int ccld_destroy(ccld_ctx* ctx) {
   ctx->pool.put(ctx->reg_blk); ctx->pool.put(ctx->misc_blk);
   ctx->pool.clear();
   if (ctx->h_pinned) cudaFreeHost(ctx->h_pinned);
+  for (auto& b : ctx->pending) cudaFreeHost(b.h_tot);
+  for (auto& f : ctx->pinned_free) cudaFreeHost(f.first);
   for (auto& sl : ctx->ring) for (int i = 0; i < TIMER_PAIRS; ++i) { cudaEventDestroy(sl.a[i]); cudaEventDestroy(sl.b[i]); }
   delete ctx;
   return CCLD_OK;
@@ -398,6 +465,7 @@ int ccld_trace_upload(ccld_ctx* ctx, uint32_t window_id, uint64_t n_rec, int mem
 
 int ccld_window_release(ccld_ctx* ctx, uint32_t window_id) {
   if (!ctx) return CCLD_ERR_ARG;
+  { int rc = settle(ctx); if (rc != CCLD_OK) return rc; }
   auto it = ctx->windows.find(window_id);
   if (it == ctx->windows.end()) return fail(ctx, CCLD_ERR_NO_WINDOW, "unknown window id");
   CK(cudaSetDevice(ctx->device));
@@ -413,8 +481,14 @@ int ccld_reset(ccld_ctx* ctx) {
   if (!ctx) return CCLD_ERR_ARG;
   CK(cudaSetDevice(ctx->device));
   CK(cudaStreamSynchronize(ctx->stream));
+  // batches still in doubt need no second analysis: their results are dropped with all the others
+  for (auto& b : ctx->pending) ctx->pinned_free.emplace_back(b.h_tot, b.h_bytes);
+  ctx->pending.clear();
   for (auto& kv : ctx->windows) drop_results(kv.second);
-  if (ctx->finalized) CK(cudaMemsetAsync((char*)ctx->reg_blk.p + ctx->stats_off, 0, ctx->stats_bytes, ctx->stream));
+  if (ctx->finalized) {
+    CK(cudaMemsetAsync((char*)ctx->reg_blk.p + ctx->stats_off, 0, ctx->stats_bytes, ctx->stream));
+    CK(cudaMemsetAsync(ctx->d_poison, 0, 4, ctx->stream));
+  }
   return CCLD_OK;
 }
 
@@ -422,6 +496,21 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   if (!ctx) return CCLD_ERR_ARG;
   if (n_windows == 0) return fail(ctx, CCLD_ERR_ARG, "n_windows is zero");
   if (n_windows > 65535) return fail(ctx, CCLD_ERR_CAPACITY, "more than 65,535 windows in one batch");
+  return analyze_batch(ctx, first_window, n_windows, now_ns, ctx->speculate != 0);
+}
+
+int ccld_set_speculation(ccld_ctx* ctx, int on) {
+  if (!ctx) return CCLD_ERR_ARG;
+  { int rc = settle(ctx); if (rc != CCLD_OK) return rc; }
+  ctx->speculate = on != 0;
+  return CCLD_OK;
+}
+
+}  // extern "C"
+
+namespace {
+
+int analyze_batch(ccld_ctx* ctx, u32 first_window, u32 n_windows, i64 now_ns, bool may_speculate) {
   CK(cudaSetDevice(ctx->device));
   std::vector<WindowHost*> ws(n_windows);
   for (u32 k = 0; k < n_windows; ++k) {
@@ -434,12 +523,25 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   const u32 B = n_windows, nc = ctx->reg.n_comms;
   cudaStream_t st = ctx->stream;
 
+  // A batch of a shape seen before (the same record count in every window) is enqueued without waiting for its plan:
+  // the results are sized from the totals that shape had last time, and the plan checks them on the device.
+  const ShapeEntry* expect = nullptr;
+  if (may_speculate) {
+    for (const ShapeEntry& e : ctx->shapes) {
+      if (e.n_rec.size() != B) continue;
+      bool same = true;
+      for (u32 k = 0; k < B && same; ++k) same = e.n_rec[k] == ws[k]->n_rec;
+      if (same) { expect = &e; break; }
+    }
+  }
+  if (!expect) { int rc = settle(ctx); if (rc != CCLD_OK) return rc; }    // the waiting path runs with nothing in doubt before it
+
   // ---- plan block: descriptors, op-counter ranges, layout rows, totals, counters ----
   size_t off = 0;
   auto take = [&](size_t b) { size_t o = off; off = align_up(off + b); return o; };
   const size_t o_desc = take(B * sizeof(WinDesc)), o_rmin = take((size_t)B * nc * 4), o_rmax = take((size_t)B * nc * 4),
                o_rng = take((size_t)B * nc * sizeof(RangeRow)), o_srow = take((size_t)B * nc * sizeof(uint4)), o_tot = take((size_t)B * T_COUNT * 8), o_cnt = take((size_t)B * C_COUNT * 8),
-               o_end = take(0);
+               o_zero_end = off, o_exp = take(expect ? (size_t)B * T_COUNT * 8 : 0);
   cudaError_t e;
   Block pb = ctx->pool.get(off, &e);
   if (e != cudaSuccess) return fail(ctx, CCLD_ERR_NOMEM, "plan allocation failed");
@@ -454,6 +556,7 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
     d.rmin = (u32*)(pbase + o_rmin) + (size_t)k * nc; d.rmax = (u32*)(pbase + o_rmax) + (size_t)k * nc;
     d.ranges = (RangeRow*)(pbase + o_rng) + (size_t)k * nc; d.srow = (uint4*)(pbase + o_srow) + (size_t)k * nc;
     d.totals = (u64*)(pbase + o_tot) + (size_t)k * T_COUNT; d.counters = (u64*)(pbase + o_cnt) + (size_t)k * C_COUNT;
+    d.expect = expect ? (const u64*)(pbase + o_exp) + (size_t)k * T_COUNT : nullptr; d.poison = ctx->d_poison;
     d.n_groups = d.n_slots = 0; d.perm = nullptr; d.flags = nullptr; d.skey = d.dkey = nullptr; d.gi64 = nullptr; d.gu32 = nullptr; d.gbw = nullptr;
     d.comm_rows = nullptr; d.alerts = nullptr;
     for (int q = 0; q < B_COUNT; ++q) d.base[q] = 0;
@@ -462,28 +565,36 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   }
   if (cta > 0x7FFFFFFFull) return fail(ctx, CCLD_ERR_CAPACITY, "batch too large for one launch");
   WinDesc* d_desc = (WinDesc*)(pbase + o_desc);
-  CK(cudaMemsetAsync(pbase, 0, off, st));
-  CK(cudaMemsetAsync(pbase + o_rmin, 0xFF, (size_t)B * nc * 4, st));
-  CK(cudaMemcpyAsync(d_desc, hd.data(), B * sizeof(WinDesc), cudaMemcpyHostToDevice, st));
-  (void)o_end;
   TimerSlot* ts = timer_begin(ctx);
-  if (cta > 0) { TimedLaunch tl(ts, 0, st); k_seq_range<<<dim3((u32)cta, B), REC_THREADS, range_smem_bytes(nc), st>>>(d_desc, ctx->reg); }
-  { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, PlanLists{nullptr, nullptr, nullptr, nullptr}, 0); }
-  CK(cudaGetLastError());
-  { int rc = ensure_pinned(ctx, (size_t)B * T_COUNT * 8); if (rc != CCLD_OK) return rc; }
-  CK(cudaMemcpyAsync(ctx->h_pinned, pbase + o_tot, (size_t)B * T_COUNT * 8, cudaMemcpyDeviceToHost, st));
-  CK(cudaStreamSynchronize(st));
+  auto start_plan = [&]() -> cudaError_t {               // clears the plan block, uploads the descriptors, runs the range pass and the layout
+    cudaError_t r = cudaMemsetAsync(pbase, 0, o_zero_end, st);
+    if (r == cudaSuccess) r = cudaMemsetAsync(pbase + o_rmin, 0xFF, (size_t)B * nc * 4, st);
+    if (r == cudaSuccess && expect) r = cudaMemcpyAsync(pbase + o_exp, expect->totals.data(), (size_t)B * T_COUNT * 8, cudaMemcpyHostToDevice, st);
+    if (r == cudaSuccess) r = cudaMemcpyAsync(d_desc, hd.data(), B * sizeof(WinDesc), cudaMemcpyHostToDevice, st);
+    if (r != cudaSuccess) return r;
+    if (cta > 0) { TimedLaunch tl(ts, 0, st); k_seq_range<<<dim3((u32)cta, B), REC_THREADS, range_smem_bytes(nc), st>>>(d_desc, ctx->reg); }
+    { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, PlanLists{nullptr, nullptr, nullptr, nullptr}, 0); }
+    return cudaGetLastError();
+  };
+  const u64* tot = nullptr;                                // [B][T_COUNT] totals the results are sized from
+  if (!expect) {
+    CK(start_plan());
+    { int rc = ensure_pinned(ctx, (size_t)B * T_COUNT * 8); if (rc != CCLD_OK) return rc; }
+    CK(cudaMemcpyAsync(ctx->h_pinned, pbase + o_tot, (size_t)B * T_COUNT * 8, cudaMemcpyDeviceToHost, st));
+    CK(cudaStreamSynchronize(st));
+    tot = ctx->h_pinned;
+  } else tot = expect->totals.data();
 
-  // ---- result block: sized from the plan ----
+  // ---- result block: sized from the totals ----
   off = 0;
   u64 total_slots = 0, n_list[B_COUNT] = {0, 0, 0, 0, 0};       // batch-wide list lengths (B_*)
   const int t_of[B_COUNT] = {T_FCTA, T_FWT, T_FSUM, T_TILES2, T_TILES3};
-  for (u32 k = 0; k < B; ++k) { const u64* t = ctx->h_pinned + (size_t)k * T_COUNT; total_slots += t[T_SLOTS]; }
+  for (u32 k = 0; k < B; ++k) { const u64* t = tot + (size_t)k * T_COUNT; total_slots += t[T_SLOTS]; }
   const size_t o_perm = take(total_slots * 4 + ALIGN);
   std::vector<size_t> o_flags(B), o_gi(B), o_gu(B), o_gb(B), o_rows(B), o_al(B), perm_off(B);
   { size_t po = 0;
     for (u32 k = 0; k < B; ++k) {
-      const u64* t = ctx->h_pinned + (size_t)k * T_COUNT;
+      const u64* t = tot + (size_t)k * T_COUNT;
       perm_off[k] = po; po += t[T_SLOTS] * 4;
       o_flags[k] = take(t[T_SLOTS]); o_gi[k] = take(t[T_GROUPS] * 8 * GI_COUNT); o_gu[k] = take(t[T_GROUPS] * 4 * GU_COUNT);
       o_gb[k] = take(t[T_GROUPS] * 8); o_rows[k] = take(t[T_ROWS] * sizeof(ccld_comm_verdict));
@@ -496,7 +607,7 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
                o_t3 = take(n_list[B_T3] * sizeof(Tile)), o_s3 = take(n_list[B_T3] * sizeof(TileSum));
   // groups the fused kernel may set aside for the deferred kernel: at most every group of the batch
   u64 total_groups = 0;
-  for (u32 k = 0; k < B; ++k) total_groups += ctx->h_pinned[(size_t)k * T_COUNT + T_GROUPS];
+  for (u32 k = 0; k < B; ++k) total_groups += tot[(size_t)k * T_COUNT + T_GROUPS];
   const size_t o_defn = take(16), o_def = take(n_list[B_FCTA] ? total_groups * 8 : 0),
                o_def3 = take(n_list[B_T3] * (size_t)LARGE_SEQS * 8),          // likewise for the kernel of the largest communicators
                o_lgrp = take(n_list[B_T3] * (size_t)LARGE_SEQS * sizeof(LargeGroup)),
@@ -506,7 +617,7 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   auto res_blk = std::make_shared<Shared>(&ctx->pool, rb);
   char* rbase = (char*)rb.p;
   for (u32 k = 0; k < B; ++k) {
-    const u64* t = ctx->h_pinned + (size_t)k * T_COUNT;
+    const u64* t = tot + (size_t)k * T_COUNT;
     WinDesc& d = hd[k];
     d.n_groups = t[T_GROUPS]; d.n_slots = t[T_SLOTS];
     d.perm = (u32*)(rbase + o_perm + perm_off[k]); d.flags = (u8*)(rbase + o_flags[k]);
@@ -515,7 +626,8 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
     d.comm_rows = (ccld_comm_verdict*)(rbase + o_rows[k]); d.alerts = (ccld_hang_alert*)(rbase + o_al[k]);
     d.tsum[0] = (TileSum*)(rbase + o_fsum); d.tsum[1] = (TileSum*)(rbase + o_s2); d.tsum[2] = (TileSum*)(rbase + o_s3);
   }
-  CK(cudaMemcpyAsync(d_desc, hd.data(), B * sizeof(WinDesc), cudaMemcpyHostToDevice, st));
+  if (expect) CK(start_plan());                            // descriptors already complete: nothing was waited for
+  else CK(cudaMemcpyAsync(d_desc, hd.data(), B * sizeof(WinDesc), cudaMemcpyHostToDevice, st));
   if (total_slots) CK(cudaMemsetAsync(rbase + o_perm, 0xFF, total_slots * 4, st));
   PlanLists pl; pl.fcta = (FusedCta*)(rbase + o_fcta); pl.fwt = (WarpTile*)(rbase + o_fwt); pl.t2 = (Tile*)(rbase + o_t2); pl.t3 = (Tile*)(rbase + o_t3);
   { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, pl, 1); }
@@ -548,10 +660,33 @@ int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows
   for (u32 k = 0; k < B; ++k) {
     WindowHost& w = *ws[k];
     w.analysed = true; w.plan_blk = plan_blk; w.res_blk = res_blk; w.d_desc = d_desc + k; w.d = hd[k];
-    std::memcpy(w.totals, ctx->h_pinned + (size_t)k * T_COUNT, sizeof w.totals);
+    std::memcpy(w.totals, tot + (size_t)k * T_COUNT, sizeof w.totals);
+  }
+  if (expect) {
+    // what the plan really found follows the batch into pinned memory; settle() reads it
+    PendingBatch pbatch; pbatch.first = first_window; pbatch.n = B; pbatch.now = now_ns;
+    pbatch.h_tot = pinned_get(ctx, (size_t)B * T_COUNT * 8, &pbatch.h_bytes);
+    if (!pbatch.h_tot) { cudaStreamSynchronize(st); return fail(ctx, CCLD_ERR_NOMEM, "pinned allocation failed"); }
+    CK(cudaMemcpyAsync(pbatch.h_tot, pbase + o_tot, (size_t)B * T_COUNT * 8, cudaMemcpyDeviceToHost, st));
+    ctx->pending.push_back(pbatch);
+  } else {
+    // remember the totals of this shape, unless a window was refused
+    bool clean = true;
+    for (u32 k = 0; k < B && clean; ++k) clean = tot[(size_t)k * T_COUNT + T_FAILED] == 0;
+    if (clean) {
+      ShapeEntry se; se.n_rec.resize(B); se.totals.assign(tot, tot + (size_t)B * T_COUNT);
+      for (u32 k = 0; k < B; ++k) se.n_rec[k] = ws[k]->n_rec;
+      for (size_t i = 0; i < ctx->shapes.size(); ++i) if (ctx->shapes[i].n_rec == se.n_rec) { ctx->shapes.erase(ctx->shapes.begin() + i); break; }
+      if (ctx->shapes.size() >= SHAPE_CACHE) ctx->shapes.erase(ctx->shapes.begin());
+      ctx->shapes.push_back(std::move(se));
+    }
   }
   return CCLD_OK;
 }
+
+}  // namespace
+
+extern "C" {
 
 int ccld_get_verdict(ccld_ctx* ctx, uint32_t window_id, ccld_verdict* out) {
   if (!ctx || !out) return CCLD_ERR_ARG;
@@ -766,6 +901,7 @@ int ccld_get_ranges(ccld_ctx* ctx, uint32_t window_id, ccld_comm_range* rows, ui
 int ccld_get_rank_stats(ccld_ctx* ctx, uint32_t n_ranks, uint32_t* votes, uint32_t* ops, uint32_t* bw_cnt, double* bw_sum) {
   if (!ctx || !votes || !ops || !bw_cnt || !bw_sum) return CCLD_ERR_ARG;
   if (!ctx->finalized) return fail(ctx, CCLD_ERR_STATE, "nothing analysed yet");
+  { int rc = settle(ctx); if (rc != CCLD_OK) return rc; }
   CK(cudaSetDevice(ctx->device));
   std::memset(votes, 0, (size_t)n_ranks * 16); std::memset(ops, 0, (size_t)n_ranks * 4);
   std::memset(bw_cnt, 0, (size_t)n_ranks * 4); std::memset(bw_sum, 0, (size_t)n_ranks * 8);
@@ -845,6 +981,7 @@ int ccld_state_export(ccld_ctx* ctx, void* buf, uint64_t cap, uint64_t* n_bytes)
   if (!ctx || !n_bytes) return CCLD_ERR_ARG;
   CK(cudaSetDevice(ctx->device));
   { int rc = finalize_registry(ctx); if (rc != CCLD_OK) return rc; }
+  { int rc = settle(ctx); if (rc != CCLD_OK) return rc; }
   const u32 nc = ctx->reg.n_comms;
   const u64 need = sizeof(StateHeader) + (u64)nc * 12 + ctx->stats_bytes;
   *n_bytes = need;
@@ -862,6 +999,7 @@ int ccld_state_import(ccld_ctx* ctx, const void* buf, uint64_t n_bytes) {
   if (!ctx || !buf) return CCLD_ERR_ARG;
   CK(cudaSetDevice(ctx->device));
   { int rc = finalize_registry(ctx); if (rc != CCLD_OK) return rc; }
+  { int rc = settle(ctx); if (rc != CCLD_OK) return rc; }
   const u32 nc = ctx->reg.n_comms;
   StateHeader h;
   if (n_bytes < sizeof h) return fail(ctx, CCLD_ERR_ARG, "state blob too short");

@@ -357,8 +357,22 @@ __device__ __forceinline__ u32 comm_units(u32 ns, u32 n, u32 T) {
 
 struct PlanLists { FusedCta* fcta; WarpTile* fwt; Tile* t2; Tile* t3; };
 
+// A window that is given up leaves no work behind: zero ranges and scatter rows, zero totals.
+__device__ __forceinline__ void plan_give_up(WinDesc& D, const Registry& R, u64 why) {
+  for (u32 c = threadIdx.x; c < R.n_comms; c += PLAN_THREADS) { RangeRow z = {0, 0, 0, R.comm_n[c], 0, 0, 0, 0}; D.ranges[c] = z; D.srow[c] = make_uint4(0, 0, 0, 0); }
+  if (threadIdx.x == 0) {
+    for (int q = 0; q < T_COUNT; ++q) D.totals[q] = 0;
+    D.totals[T_FAILED] = why; D.totals[T_CHUNKS] = 1;
+  }
+}
+
 // emit == 0: ranges, scatter rows and totals (the window is refused if it needs more than slot_cap slots).
 // emit == 1: the work lists (base[] filled by the host from the totals).
+// When the host sized the results from totals it expected (D.expect) instead of waiting for these, a window whose totals
+// differ gives up and raises the poison flag; so does every window planned after the flag went up - in the same batch
+// (seen here at emit == 1) or in a later one - so that windows are never analysed out of order. A window that gave up
+// fills its stretch of the work lists with entries that hold no work, because the kernels that follow are launched
+// over the expected lengths.
 __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd, Registry R, PlanLists L, int emit) {
   __shared__ PlanAcc s_warp[33];
   __shared__ uint2 s_pair[33];
@@ -366,7 +380,22 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
   __shared__ int s_failed;
   WinDesc& D = wd[blockIdx.x];
   const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  if (emit && D.totals[T_FAILED]) return;
+  if (emit) {
+    if (D.expect != nullptr) {
+      if (!D.totals[T_FAILED] && *(volatile u32*)D.poison != 0) { __syncthreads(); plan_give_up(D, R, FAILED_EXPECT); __syncthreads(); }
+      if (D.totals[T_FAILED]) {
+        const u64 n_cta = D.expect[T_FCTA], n2 = D.expect[T_TILES2], n3 = D.expect[T_TILES3];
+        for (u64 j = threadIdx.x; j < n_cta; j += PLAN_THREADS) {
+          FusedCta x; x.w = blockIdx.x; x.cls = 0; x.c = 0; x.seq_off = 0; x.count = 0; x.sum_idx = 0; x.wt_first = 0; x.wt_count = 0; x.moff = 0;
+          x.row = RangeRow{0, 0, 0, 0, 0, 0, 0, 0};
+          L.fcta[D.base[B_FCTA] + j] = x;
+        }
+        for (u64 j = threadIdx.x; j < n2; j += PLAN_THREADS) { Tile t; t.w = blockIdx.x; t.c = 0; t.seq_off = 0; t.count = 0; L.t2[D.base[B_T2] + j] = t; }
+        for (u64 j = threadIdx.x; j < n3; j += PLAN_THREADS) { Tile t; t.w = blockIdx.x; t.c = 0; t.seq_off = 0; t.count = 0; L.t3[D.base[B_T3] + j] = t; }
+        return;
+      }
+    } else if (D.totals[T_FAILED]) return;
+  }
 
   if (!emit) {
     // 1. layout: groups, slots, rows; tiles of the two big classes; busiest fused-class communicator
@@ -417,13 +446,19 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
     }
     if (threadIdx.x == 0) {
       // op counters further apart than 2^31, or more slots than the cap: refuse the window
-      const int failed = run.slots > D.slot_cap || run.groups > 0x7FFFFFFFull || n_cta > 0x7FFFFFFFull || n_wt > 0x7FFFFFFFull;
-      s_failed = failed;
+      u64 failed = (run.slots > D.slot_cap || run.groups > 0x7FFFFFFFull || n_cta > 0x7FFFFFFFull || n_wt > 0x7FFFFFFFull) ? FAILED_CAPACITY : 0;
+      if (!failed && D.expect != nullptr) {
+        const u64* e = D.expect;
+        const bool same = e[T_GROUPS] == run.groups && e[T_SLOTS] == run.slots && e[T_FCTA] == n_cta && e[T_FWT] == n_wt && e[T_FSUM] == urun &&
+                          e[T_TILES2] == run.t2 && e[T_TILES3] == run.t3 && e[T_ROWS] == run.rows && e[T_CHUNKS] == T;
+        if (!same || *(volatile u32*)D.poison != 0) { failed = FAILED_EXPECT; atomicExch(D.poison, 1u); }
+      }
+      s_failed = failed != 0;
       D.totals[T_GROUPS] = failed ? 0 : run.groups; D.totals[T_SLOTS] = failed ? 0 : run.slots;
       D.totals[T_FCTA] = failed ? 0 : n_cta; D.totals[T_FWT] = failed ? 0 : n_wt; D.totals[T_FSUM] = failed ? 0 : urun;
       D.totals[T_TILES2] = failed ? 0 : run.t2; D.totals[T_TILES3] = failed ? 0 : run.t3;
       D.totals[T_ROWS] = failed ? 0 : run.rows; D.totals[T_FAILED] = failed; D.totals[T_CHUNKS] = T;
-      if (failed) atomicOr((unsigned*)&D.counters[C_ERR], (unsigned)CCLD_E_CAPACITY);
+      if (failed == FAILED_CAPACITY) atomicOr((unsigned*)&D.counters[C_ERR], (unsigned)CCLD_E_CAPACITY);
     }
     __syncthreads();
     if (s_failed)
@@ -541,7 +576,7 @@ constexpr u32 SCAT_LOCAL = 4;     // ranks, counted from the rank of the CTA's f
 __global__ void __launch_bounds__(SCAT_THREADS, 4) k_slot_scatter(const WinDesc* __restrict__ wd, Registry R) {
   __shared__ uint4 s_ent[SCAT_LOCAL * RANK_TAB_K];       // (communicator id, counters covered, first counter, first slot); counters covered 0: unused
   const WinDesc& D = wd[blockIdx.y];                          // grid: (CTAs of the largest window, windows)
-  if (blockIdx.x >= D.n_cta) return;
+  if (blockIdx.x >= D.n_cta) return;                          // (a window that was given up has empty scatter rows: nothing is stored)
   const u64 base = (u64)blockIdx.x * REC_PER_CTA;
   u32 err = 0, rej = 0, internal = 0;
   // descriptor fields in registers: the stores below could alias the descriptor as far as the compiler knows

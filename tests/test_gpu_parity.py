@@ -635,3 +635,64 @@ def test_tree_communicators_slow_root_compares_rates_within_a_layer(with_rates):
         assert rows["slow_detected"].all() and (rows["sel_seq"] == 3 * w + 1).all()
         src = rows["rate_source"].tolist()
         assert src == ([0, 1, 0, 0, 0, 0, 0, 1, 0] if with_rates else [1] * 9)
+
+
+# ---------------------------------------------------------------- batches enqueued without waiting for their plan
+def test_repeated_shape_is_enqueued_without_waiting_and_stays_in_order():
+    """Windows analysed one call at a time: from the second call on the shape is known, the call sizes its buffers from
+    the earlier totals and only enqueues. Results, and the state that carries from window to window (Eq. 1 baseline going
+    dynamic, the repetition counter), are those of the oracle walking the windows in order."""
+    spec = tg.cfg2(reps=60, n_windows=6, tp=8, pp=2, dp=16)
+    params = dict(m_max_rounds=150, tbase_init_ns=100_000)       # the baseline freezes in the second window, slow rounds repeat
+    reg = tg.registry(spec)
+    an, o = make_pair(reg, params)
+    wins = [tg.gen_window(spec, w, device="cuda") for w in range(spec.n_windows)]
+    for w, win in enumerate(wins):
+        an.trace_upload(w, win.cols); assert o.upload(w, win.cols) == 0
+    now = wins[-1].now_ns
+    for w in range(spec.n_windows):
+        an.analyze_window(w, 1, now)                             # nothing is read back in between
+    assert o.analyze(0, spec.n_windows, now) == 0
+    for w in range(spec.n_windows):
+        compare_window(an, o, w)
+    rows = o.comm_rows(spec.n_windows - 1)
+    assert (rows["baseline_static"] == 0).any() and (rows["slow_count"] > 1).any()
+    compare_cumulative(an, o, spec.n_ranks, spec.n_windows - 1)
+
+
+@pytest.mark.parametrize("speculate", [True, False])
+def test_a_batch_that_does_not_match_its_expected_layout_is_analysed_again_in_order(speculate):
+    """Window 2 has the record count of its predecessors but one record with a far later op counter, so its layout (more
+    groups, more slots) is not the one the call expected; windows 3 and 4 are enqueued behind it before anything is read
+    back. All of them must come out as if every call had waited: same rows, same cumulative state, same order."""
+    spec = tg.cfg2(reps=40, n_windows=5, tp=8, pp=2, dp=16)
+    params = dict(m_max_rounds=100, tbase_init_ns=100_000)
+    reg = tg.registry(spec)
+    an, o = make_pair(reg, params)
+    an.set_speculation(speculate)
+    cols = []
+    for w in range(spec.n_windows):
+        c = {k: v.clone() for k, v in tg.gen_window(spec, w, device="cpu").cols.items()}
+        if w == 2:
+            c["seq"][7] += 500                                   # a rank far ahead: 500 groups nobody else reported
+        cols.append(c)
+    for w, c in enumerate(cols):
+        an.trace_upload(w, c); assert o.upload(w, c) == 0
+    now = tg.gen_window(spec, spec.n_windows - 1).now_ns
+    an.timing_enable(True)
+    for w in range(spec.n_windows):
+        an.analyze_window(w, 1, now)
+    assert o.analyze(0, spec.n_windows, now) == 0
+    v2 = an.get_verdict(2, check=False)
+    # the layout kernel runs twice per analysed batch: five calls, and - when calls do not wait - windows 2, 3 and 4 once more
+    assert an.get_kernel_times()["k_plan"]["launches"] == (16 if speculate else 10)
+    an.timing_enable(False)
+    assert v2["n_incomplete"] == o.sizes(2)["n_incomplete"] > 400 and v2["n_groups"] == o.sizes(2)["n_groups"] > o.sizes(1)["n_groups"] + 400
+    for w in range(spec.n_windows):
+        compare_window(an, o, w)
+    compare_cumulative(an, o, spec.n_ranks, spec.n_windows - 1)
+    # the library keeps working in the same context: a reset and the same windows once more, now all as one batch
+    an.reset()
+    an.analyze_window(0, spec.n_windows, now)
+    for w in range(spec.n_windows):
+        compare_window(an, o, w)
