@@ -574,7 +574,9 @@ constexpr u32 SCAT_LOCAL = 4;     // ranks, counted from the rank of the CTA's f
 // fewer than 2^32 slots, only 32-bit arithmetic. Any other record (another rank, a communicator beyond the inline pairs,
 // a counter outside the range, a rejected record) takes the two dependent table loads and the full checks.
 __global__ void __launch_bounds__(SCAT_THREADS, 4) k_slot_scatter(const WinDesc* __restrict__ wd, Registry R) {
-  __shared__ uint4 s_ent[SCAT_LOCAL * RANK_TAB_K];       // (communicator id, counters covered, first counter, first slot); counters covered 0: unused
+  // (communicator id, counters covered, first counter, first slot) per resolved pair; counters covered 0: unused. Every
+  // warp resolves its own copy, so no warp waits for another.
+  __shared__ uint4 s_ent_all[SCAT_THREADS / 32][SCAT_LOCAL * RANK_TAB_K];
   const WinDesc& D = wd[blockIdx.y];                          // grid: (CTAs of the largest window, windows)
   if (blockIdx.x >= D.n_cta) return;                          // (a window that was given up has empty scatter rows: nothing is stored)
   const u64 base = (u64)blockIdx.x * REC_PER_CTA;
@@ -592,9 +594,11 @@ __global__ void __launch_bounds__(SCAT_THREADS, 4) k_slot_scatter(const WinDesc*
     rk[k] = in ? c_rank[i] : 0u; cid[k] = in ? c_comm[i] : 0u; sq[k] = in ? c_seq[i] : 0u;
     if (in) todo |= 1u << k;
   }
+  const u32 lane = threadIdx.x & 31;
+  uint4* const s_ent = s_ent_all[threadIdx.x >> 5];
   const u32 r_first = c_rank[base];
-  if (threadIdx.x < SCAT_LOCAL * RANK_TAB_K) {
-    const u32 r = r_first + threadIdx.x / RANK_TAB_K, k = threadIdx.x % RANK_TAB_K;
+  if (lane < SCAT_LOCAL * RANK_TAB_K) {
+    const u32 r = r_first + lane / RANK_TAB_K, k = lane % RANK_TAB_K;
     uint4 e = make_uint4(NONE, 0, 0, 0);
     if (n_slots <= 0xFFFFFFFFull && r_first < R.n_ranks && r < R.n_ranks) {
       const uint4 t = R.rank_tab[(u64)r * 2 + (k >> 1)];
@@ -605,9 +609,9 @@ __global__ void __launch_bounds__(SCAT_THREADS, 4) k_slot_scatter(const WinDesc*
         if (b + sr.z <= n_slots) e = make_uint4(id, sr.z, sr.w, (u32)b);    // the member's whole column lies inside the table
       }
     }
-    s_ent[threadIdx.x] = e;
+    s_ent[lane] = e;
   }
-  __syncthreads();
+  __syncwarp();
 #pragma unroll
   for (int k = 0; k < SCAT_PER_THREAD; ++k) {
     const u32 dr = rk[k] - r_first;
