@@ -136,22 +136,13 @@ __device__ __forceinline__ u32 large_select(const u32 (&v)[LG_KEYS], u32 have, b
   u32* __restrict__ hist = s_hist + g * LG_BINS;
   u32 hi = 32 - (u32)__clz(bound | 1u);                      // bits still undecided: the result lies below 2^hi
   u32 prefix = 0;                                            // the decided bits, already in place
+  u32 alive = act ? have : 0u;                               // my keys that still agree with the decided bits
   while (hi > 0) {
     const u32 sh = hi > LG_DIGIT ? hi - LG_DIGIT : 0u, w = hi - sh;       // this pass decides bits [sh, hi)
     const u32 dmask = (1u << w) - 1u;
-    if (act) {
-      u32 cm = 0;
-      if (hi >= 32) cm = have;
-      else {
-        const u32 want = prefix >> hi;
+    if (alive) {
 #pragma unroll
-        for (int q = 0; q < LG_KEYS; ++q) cm |= ((v[q] >> hi) == want ? 1u : 0u) << q;
-        cm &= have;
-      }
-      if (cm) {
-#pragma unroll
-        for (int q = 0; q < LG_KEYS; ++q) if ((cm >> q) & 1u) atomicAdd(&hist[(v[q] >> sh) & dmask], 1u);
-      }
+      for (int q = 0; q < LG_KEYS; ++q) if ((alive >> q) & 1u) atomicAdd(&hist[(v[q] >> sh) & dmask], 1u);
     }
     __syncthreads();
     if (wid < G) {                                                               // warp w scans and clears group w's histogram
@@ -173,7 +164,14 @@ __device__ __forceinline__ u32 large_select(const u32 (&v)[LG_KEYS], u32 have, b
       }
     }
     __syncthreads();
-    prefix |= s_pick[g] << sh;
+    const u32 pick = s_pick[g];
+    prefix |= pick << sh;
+    if (alive) {                                             // few keys survive the first pass: most threads are done here
+      u32 keep = 0;
+#pragma unroll
+      for (int q = 0; q < LG_KEYS; ++q) keep |= (((v[q] >> sh) & dmask) == pick ? 1u : 0u) << q;
+      alive &= keep;
+    }
     hi = sh;
   }
   return prefix;
@@ -305,27 +303,24 @@ __global__ void __launch_bounds__(LG_THREADS, 2) k_reduce_large(const WinDesc* _
       u32 n_fs = 0, n_fd = 0;
       const u32 gcnt = t.count - j0 < G ? t.count - j0 : G;
       const u64 slot0 = row.slot0 + (u64)(t.seq_off + j0) * n;
-      for (u32 p = threadIdx.x; p < n; p += LG_THREADS) {
-        double bwv = 0.0;
-        const u32 rank4 = mem[p] * 4;
-        for (u32 q = 0; q < gcnt; ++q) {
-          const LargeScal& z = s_sc[q];
-          if (!(z.state & 1)) continue;
-          const u64 o = slot0 + (u64)q * n + p;
-          const u32 d = D.dkey[o];
+      for (u32 q = 0; q < gcnt; ++q) {
+        const LargeScal z = s_sc[q];                                           // the group's values stay in registers over my members
+        if (!(z.state & 1)) continue;
+        const u64 o0 = slot0 + (u64)q * n;
+        for (u32 p = threadIdx.x; p < n; p += LG_THREADS) {                  // a member belongs to one thread: no two threads touch s_bw[p]
+          const u32 d = D.dkey[o0 + p];
           u32 f = CCLD_F_NOT_ANALYSED;
           if (z.state & 2) {
-            const u32 skw = D.skey[o] - z.emin, dd = d - z.tmn;
+            const u32 skw = D.skey[o0 + p] - z.emin, dd = d - z.tmn;
             const bool so_ = (u64)__usad(skw, z.ms, 0u) * 1000u > z.ts, shi = skw > z.ms;
             const bool dq = (u64)__usad(dd, z.md, 0u) * 1000u > z.td, dhi = dd > z.md;
             f = (so_ ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (shi ? CCLD_F_SKEW_HI : 0) | (dhi ? CCLD_F_DUR_HI : 0);
-            if (so_) { ++n_fs; atomicAdd(&R.votes[rank4 + (shi ? 0 : 1)], 1u); }
-            if (dq) { ++n_fd; atomicAdd(&R.votes[rank4 + (dhi ? 2 : 3)], 1u); }
+            if (so_) { ++n_fs; atomicAdd(&R.votes[(u64)mem[p] * 4 + (shi ? 0 : 1)], 1u); }
+            if (dq) { ++n_fd; atomicAdd(&R.votes[(u64)mem[p] * 4 + (dhi ? 2 : 3)], 1u); }
           }
-          D.flags[o] = (u8)f;
-          if (!(z.state & 4) && d != 0) bwv += z.bn * rcp_newton1((double)d * z.den);
+          D.flags[o0 + p] = (u8)f;
+          if (!(z.state & 4) && d != 0) s_bw[p] += z.bn * rcp_newton1((double)d * z.den);
         }
-        s_bw[p] += bwv;
       }
       n_fs = __reduce_add_sync(0xFFFFFFFFu, n_fs); n_fd = __reduce_add_sync(0xFFFFFFFFu, n_fd);
       if (lane == 0) { if (n_fs) atomicAdd(&s_cnt[SC_FS], n_fs); if (n_fd) atomicAdd(&s_cnt[SC_FD], n_fd); }
