@@ -149,6 +149,20 @@ __device__ __forceinline__ void range_put(const WinDesc& D, u32* s_mn, u32* s_mx
 // look their communicator up and update the table themselves: one registry lookup and two shared-memory atomics per
 // record at worst.
 constexpr int RANGE_FOLDS = 4;
+constexpr int RANGE_WARP_FOLDS = 8;
+
+// cid[i] for the lowest i with bit i of `left` set (any element if left is 0)
+__device__ __forceinline__ u32 first_left(const u32 (&cid)[REC_RUN], u32 left) {
+  static_assert(REC_RUN == 16, "selection tree over a run of 16");
+  const u32 b = (u32)__ffs(left) - 1u;
+  u32 x8[8], x4[4];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) x8[i] = (b & 8u) ? cid[8 + i] : cid[i];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) x4[i] = (b & 4u) ? x8[4 + i] : x8[i];
+  const u32 y0 = (b & 2u) ? x4[2] : x4[0], y1 = (b & 2u) ? x4[3] : x4[1];
+  return (b & 1u) ? y1 : y0;
+}
 
 __global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __restrict__ wd, Registry R) {
   extern __shared__ u32 s_dyn[];
@@ -185,6 +199,38 @@ __global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __rest
   // would match a record that names communicator 0xFFFFFFFF) and goes record by record
   const u32 tail = len < REC_RUN ? (1u << len) - 1u : 0u;
   u32 left = len < REC_RUN ? 0u : (1u << REC_RUN) - 1u;
+  // warp folds: in a rank-major upload the 32 runs of a warp belong to one or two ranks, so all lanes meet the same few
+  // communicators. One of them at a time - the communicator of the first record left in the lowest lane that has one -
+  // is folded by every lane and reduced over the warp, and lane 0 updates the table once. The stage ends as soon as a
+  // fold clears less than an eighth of what was left (an upload in another order): the lanes then fold on their own.
+  {
+    u32 remaining = __reduce_add_sync(0xFFFFFFFFu, (u32)__popc(left));
+    for (int f = 0; f < RANGE_WARP_FOLDS && remaining != 0; ++f) {
+      const u32 have = __ballot_sync(0xFFFFFFFFu, left != 0);
+      const u32 id = __shfl_sync(0xFFFFFFFFu, first_left(cid, left), (u32)__ffs(have) - 1u);
+      const uint4 h = comm_find(R, id, R.hash[hash_home(R, id)]);        // the same in every lane
+      u32 m = 0, mn = NONE, mx = 0;
+#pragma unroll
+      for (int k = 0; k < REC_RUN; ++k) {
+        if (cid[k] == id) { m |= 1u << k; mn = min(mn, sq[k]); mx = max(mx, sq[k]); }
+      }
+      m &= left;                                             // a run cut short holds padding and takes no part
+      u32 a = __reduce_min_sync(0xFFFFFFFFu, m ? mn : NONE), b = __reduce_max_sync(0xFFFFFFFFu, m ? mx : 0u);
+      if (h.y != NONE && a < h.z) {
+        // counters below the communicator's first name no operation: fold again without them
+        mn = NONE; mx = 0;
+#pragma unroll
+        for (int k = 0; k < REC_RUN; ++k) if (((m >> k) & 1u) && sq[k] >= h.z) { mn = min(mn, sq[k]); mx = max(mx, sq[k]); }
+        a = __reduce_min_sync(0xFFFFFFFFu, mn); b = __reduce_max_sync(0xFFFFFFFFu, mx);
+      }
+      if (lane == 0 && h.y != NONE && a <= b) range_put(D, s_mn, s_mx, h.y, a, b);
+      left &= ~m;
+      const u32 cleared = __reduce_add_sync(0xFFFFFFFFu, (u32)__popc(m));
+      const bool worth = cleared * 8u >= remaining;
+      remaining -= cleared;
+      if (!worth) break;
+    }
+  }
   // folds: the communicator of the first record still left takes every record of the run that names it
   for (int f = 0; f < RANGE_FOLDS && __any_sync(0xFFFFFFFFu, left != 0); ++f) {
     const bool act = left != 0;
