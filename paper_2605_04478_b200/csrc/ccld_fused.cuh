@@ -22,7 +22,9 @@ constexpr u32 FULLM = 0xFFFFFFFFu;
 #define CCLD_FUSED_MIN_CTAS 3
 #endif
 
-template <class K> __device__ __forceinline__ void cswap(K& a, K& b) { const K lo = a < b ? a : b; const K hi = a < b ? b : a; a = lo; b = hi; }
+template <class K> __device__ __forceinline__ void cswap(K& a, K& b) { const K lo = min(a, b), hi = max(a, b); a = lo; b = hi; }
+__device__ __forceinline__ u32 key_absdiff(u32 a, u32 b) { return __usad(a, b, 0u); }
+__device__ __forceinline__ u64 key_absdiff(u64 a, u64 b) { return a >= b ? a - b : b - a; }
 
 // 19-exchange sorting network for 8 keys
 template <class K> __device__ __forceinline__ void sort8(K (&v)[8]) {
@@ -58,19 +60,22 @@ template <class K> __device__ __forceinline__ void median_mad8(const K (&x)[8], 
   const u32 k = (n - 1) >> 1;
   const K m = pick4(s, k);
 #pragma unroll
-  for (int p = 0; p < 8; ++p) s[p] = (u32)p < n ? (s[p] >= m ? s[p] - m : m - s[p]) : KeyMax<K>::v();   // falls to 0 at k, then rises
+  for (int p = 0; p < 8; ++p) s[p] = (u32)p < n ? key_absdiff(s[p], m) : KeyMax<K>::v();   // falls to 0 at k, then rises
   merge8(s);
   *med = m; *mad = pick4(s, k);
 }
 
 // 1 / x for x >= 1 to within a few ulp: single-precision seed and two Newton steps
 // one Newton step on the single-precision seed: relative error near 2e-14
+__device__ __forceinline__ float rcp_seed(double x) {     // 1 <= x < 2^64: the approximate reciprocal is good to about 2^-22
+  float r; asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"((float)x)); return r;
+}
 __device__ __forceinline__ double rcp_newton1(double x) {
-  const double r = (double)__frcp_rn((float)x);
+  const double r = (double)rcp_seed(x);
   return fma(r, fma(-x, r, 1.0), r);
 }
 __device__ __forceinline__ double rcp_newton(double x) {
-  double r = (double)__frcp_rn((float)x);
+  double r = (double)rcp_seed(x);
   double e = fma(-x, r, 1.0); r = fma(r, e, r);
   e = fma(-x, r, 1.0); r = fma(r, e, r);
   return r;
@@ -111,7 +116,7 @@ __device__ __forceinline__ void sub_exchange(K (&v)[8], int mask, bool keep_low)
 #pragma unroll
   for (int r = 0; r < 8; ++r) o[r] = __shfl_xor_sync(0xFFFFFFFFu, v[MIRROR ? 7 - r : r], mask);
 #pragma unroll
-  for (int r = 0; r < 8; ++r) { const bool lt = v[r] < o[r]; v[r] = (lt == keep_low) ? v[r] : o[r]; }
+  for (int r = 0; r < 8; ++r) v[r] = keep_low ? min(v[r], o[r]) : max(v[r], o[r]);
 }
 
 // Sorts the 8 L keys of a group ascending; element i lives in lane i / 8 (of the group), register i % 8.
@@ -147,7 +152,7 @@ __device__ __forceinline__ void sub_median_mad(const K (&x)[8], u32 n, u32 s, u3
   const u32 k = (n - 1) >> 1, src = (lane & ~(u32)(L - 1)) | (k >> 3);
   const K m = __shfl_sync(0xFFFFFFFFu, pick8(v, k & 7), src);
 #pragma unroll
-  for (int r = 0; r < 8; ++r) v[r] = s * 8 + r < n ? (v[r] >= m ? v[r] - m : m - v[r]) : KeyMax<K>::v();   // falls to 0 at k, then rises
+  for (int r = 0; r < 8; ++r) v[r] = s * 8 + r < n ? key_absdiff(v[r], m) : KeyMax<K>::v();   // falls to 0 at k, then rises
   sub_merge<L, K>(v, s);
   *med = m; *mad = __shfl_sync(0xFFFFFFFFu, pick8(v, k & 7), src);
 }
@@ -406,19 +411,34 @@ __device__ __forceinline__ void fast_groups(const WinDesc& D, u32 w_idx, const R
     for (int q = 0; q < 8; ++q) {
       if (FULL || p0 + q < n) {
         const u32 d = kd[q * KSTEP];
-        u32 f = CCLD_F_NOT_ANALYSED;
-        if (analysed) {
-          const u32 sk = ka[q * KSTEP] - emin, dd = d - tmn;
-          const bool so = __usad(sk, ms, 0u) > ts, shi = sk > ms;
-          const bool dq = __usad(dd, md, 0u) > td, dhi = dd > md;
-          f = (so ? CCLD_F_SKEW_OUT : 0) | (dq ? CCLD_F_DUR_OUT : 0) | (shi ? CCLD_F_SKEW_HI : 0) | (dhi ? CCLD_F_DUR_HI : 0);
-          if (so) { acc.flagged += 1u; atomicAdd(&R.votes[(u64)mem[p0 + q] * 4 + (shi ? 0 : 1)], 1u); }
-          if (dq) { acc.flagged += 1u << 16; atomicAdd(&R.votes[(u64)mem[p0 + q] * 4 + (dhi ? 2 : 3)], 1u); }
-        }
+        const u32 sk = ka[q * KSTEP] - emin, dd = d - tmn;
+        const u32 f = (__usad(sk, ms, 0u) > ts ? (u32)CCLD_F_SKEW_OUT : 0u) | (__usad(dd, md, 0u) > td ? (u32)CCLD_F_DUR_OUT : 0u) |
+                      (sk > ms ? (u32)CCLD_F_SKEW_HI : 0u) | (dd > md ? (u32)CCLD_F_DUR_HI : 0u);
         if (q < 4) f_lo |= f << (8 * q); else f_hi |= f << (8 * (q - 4));
         if (!barrier && d != 0) bw[q] = bn * rcp_newton1((double)d * den);
       }
     }
+    if (!analysed) {
+      // every position that exists carries the not-analysed mark
+      const u32 cnt = FULL ? 8u : (n > p0 ? (n - p0 < 8u ? n - p0 : 8u) : 0u);
+      f_lo = 0x80808080u & (cnt >= 4 ? 0xFFFFFFFFu : (1u << (8 * cnt)) - 1u);
+      f_hi = cnt > 4 ? 0x80808080u & (cnt >= 8 ? 0xFFFFFFFFu : (1u << (8 * (cnt - 4))) - 1u) : 0u;
+    }
+    // votes: outliers are rare, so they are taken off the flag bytes afterwards, one set bit at a time
+    static_assert(CCLD_F_SKEW_OUT == 1 && CCLD_F_DUR_OUT == 2 && CCLD_F_SKEW_HI == 4 && CCLD_F_DUR_HI == 8, "flag bit layout");
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const u32 fw = half ? f_hi : f_lo;
+      u32 o = fw & 0x03030303u;
+      while (o) {
+        const u32 b = (u32)__ffs(o) - 1u, q = (b >> 3) + 4u * half, dur = b & 1u;
+        const u32 hi = (fw >> (b + 2u)) & 1u;               // the HI bit of the same metric sits two places up
+        atomicAdd(&R.votes[(u64)mem[p0 + q] * 4 + 2u * dur + (hi ? 0u : 1u)], 1u);
+        o &= o - 1u;
+      }
+    }
+    acc.flagged += (u32)__popc(f_lo & 0x01010101u) + (u32)__popc(f_hi & 0x01010101u) +
+                   (((u32)__popc(f_lo & 0x02020202u) + (u32)__popc(f_hi & 0x02020202u)) << 16);
   }
   {
     u8* __restrict__ fp = ld_volatile(sh.out.flags) + row.slot0 + (u64)(seq0 + j) * n + p0;
