@@ -37,8 +37,13 @@ struct TickArgs {
 };
 
 // the rank whose ticks contain tick i: the last r with tick_off[r] <= i
-__device__ __forceinline__ u32 tick_owner(const u64* __restrict__ off, u32 n_ranks, u64 i) {
+__device__ __forceinline__ u32 tick_owner(const u64* __restrict__ off, u32 n_ranks, u64 i, u64 n_ticks) {
+  // probes sample at one period, so the ranks' segments are about equally long: the proportional guess comes first
+  const u32 g = (u32)min((u64)(n_ranks - 1), (u64)((double)i * (double)n_ranks / (double)n_ticks));
+  const u64 g0 = off[g], g1 = off[g + 1];
+  if (g0 <= i && i < g1) return g;
   u32 lo = 0, hi = n_ranks - 1;
+  if (g0 <= i) lo = g; else hi = g ? g - 1 : 0;
   while (lo < hi) { const u32 mid = (lo + hi + 1) >> 1; if (off[mid] <= i) lo = mid; else hi = mid - 1; }
   return lo;
 }
@@ -65,14 +70,14 @@ __device__ __forceinline__ u64 cta_exclusive_scan(u64 v, u64* total, u64* s_warp
 
 // One warp per RB_PER_WARP consecutive blocks, one lane per tick: the predecessor's counters come from the lane below
 // (from the previous block's last lane, or from memory, for lane 0). Where the ranks' segments start is found once per
-// warp by a search in the offset table and then followed from block to block.
+// warp (a proportional guess, else a search in the offset table) and then followed from block to block.
 __global__ void __launch_bounds__(RT_THREADS) k_tick_blocks(TickArgs A) {
   __shared__ u64 s_cnt[RT_THREADS / 32];
   const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   const u64 t0 = (u64)blockIdx.x * RT_TILE + (u64)wid * (RB_PER_WARP * 32);
   u64 wsum = 0;
   if (t0 < A.n_ticks) {
-    u32 rk = tick_owner(A.tick_off, A.n_ranks, t0);             // a rank that has ticks: t0 < n_ticks
+    u32 rk = tick_owner(A.tick_off, A.n_ranks, t0, A.n_ticks);             // a rank that has ticks: t0 < n_ticks
     u64 seg_start = A.tick_off[rk], seg_end = A.tick_off[rk + 1];
     u32 carry_s = t0 ? __ldg(A.send + t0 - 1) : 0u, carry_r = t0 ? __ldg(A.recv + t0 - 1) : 0u;
     u32 sv_[RB_PER_WARP], rv_[RB_PER_WARP];                     // all loads of the warp's blocks are issued before the first is used
@@ -197,7 +202,7 @@ __device__ __forceinline__ u64 ticks_upto_guess(const i64* __restrict__ tn, u64 
   if (t < t0) return 0;
   if (t >= t1) return n;
   // tn[lo] <= t < tn[hi - 1]: the first tick after t has index j in [1, n - 1]
-  u64 g = (u64)((double)(t - t0) / (double)(t1 - t0) * (double)(n - 1));
+  u64 g = (u64)(__fdividef((float)(t - t0), (float)(t1 - t0)) * (float)(n - 1));   // single precision is plenty for a starting point
   g = g > n - 2 ? n - 2 : g;
   u64 j;
   if (__ldg(tn + lo + g) <= t) {
