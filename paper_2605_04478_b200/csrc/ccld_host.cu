@@ -1042,7 +1042,7 @@ int ccld_derive_rates(ccld_ctx* ctx, uint64_t n_rec, const uint32_t* rank, const
   A.blk = (TickBlock*)((char*)blk.p + o_blk); A.tile_sum = (u64*)((char*)blk.p + o_sum);
   if (n_tiles) {
     k_tick_blocks<<<(u32)n_tiles, RT_THREADS, 0, st>>>(A);
-    k_tile_scan<<<1, RT_THREADS, 0, st>>>(A.tile_sum, n_tiles);
+    k_tile_scan<<<1, TS_THREADS, 0, st>>>(A.tile_sum, n_tiles);
     k_block_prefix<<<(u32)n_tiles, RB_PER_TILE, 0, st>>>(A);
   }
   k_record_rates<<<(u32)((n_rec + RT_THREADS - 1) / RT_THREADS), RT_THREADS, 0, st>>>(A, n_rec, rank, t_enter_ns, t_exit_ns, send_chg, recv_chg);

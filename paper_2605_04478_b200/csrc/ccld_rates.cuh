@@ -19,7 +19,7 @@
 namespace ccld {
 
 constexpr int RT_THREADS = 256;
-constexpr int RT_PER = 8;                          // tile sums per thread and round in k_tile_scan
+constexpr int RT_PER = 8;
 constexpr int RT_TILE = RT_THREADS * RT_PER;       // ticks per CTA of k_tick_blocks: 8 warps x RB_PER_WARP blocks x 32
 constexpr int RB_PER_WARP = 8;
 constexpr int RB_PER_TILE = RT_TILE / 32;          // 64 blocks
@@ -46,26 +46,6 @@ __device__ __forceinline__ u32 tick_owner(const u64* __restrict__ off, u32 n_ran
   if (g0 <= i) lo = g; else hi = g ? g - 1 : 0;
   while (lo < hi) { const u32 mid = (lo + hi + 1) >> 1; if (off[mid] <= i) lo = mid; else hi = mid - 1; }
   return lo;
-}
-
-// exclusive prefix of v over the CTA (all threads call); *total = the CTA's sum
-__device__ __forceinline__ u64 cta_exclusive_scan(u64 v, u64* total, u64* s_warp /*[RT_THREADS / 32 + 1]*/) {
-  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-  u64 inc = v;
-#pragma unroll
-  for (int d = 1; d < 32; d <<= 1) { const u64 o = __shfl_up_sync(0xFFFFFFFFu, inc, d); if (lane >= (u32)d) inc += o; }
-  if (lane == 31) s_warp[wid] = inc;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    u64 run = 0;
-    for (int q = 0; q < RT_THREADS / 32; ++q) { const u64 x = s_warp[q]; s_warp[q] = run; run += x; }
-    s_warp[RT_THREADS / 32] = run;
-  }
-  __syncthreads();
-  const u64 r = s_warp[wid] + inc - v;
-  *total = s_warp[RT_THREADS / 32];
-  __syncthreads();
-  return r;
 }
 
 // One warp per RB_PER_WARP consecutive blocks, one lane per tick: the predecessor's counters come from the lane below
@@ -138,19 +118,33 @@ __global__ void __launch_bounds__(RT_THREADS) k_tick_blocks(TickArgs A) {
   }
 }
 
-__global__ void __launch_bounds__(RT_THREADS) k_tile_scan(u64* __restrict__ tile_sum, u64 n_tiles) {
-  __shared__ u64 s_warp[RT_THREADS / 32 + 1];
+// One CTA of 1,024 threads, 16 consecutive sums per thread and round: 16,384 tiles (33.5 M ticks) per round.
+constexpr int TS_THREADS = 1024;
+constexpr int TS_PER = 16;
+__global__ void __launch_bounds__(TS_THREADS) k_tile_scan(u64* __restrict__ tile_sum, u64 n_tiles) {
+  __shared__ u64 s_warp[TS_THREADS / 32];
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   u64 carry = 0;
-  for (u64 base = 0; base < n_tiles; base += RT_TILE) {          // RT_PER consecutive sums per thread and round
-    const u64 i0 = base + (u64)threadIdx.x * RT_PER;
-    u64 v[RT_PER], sum = 0;
+  for (u64 base = 0; base < n_tiles; base += (u64)TS_THREADS * TS_PER) {
+    const u64 i0 = base + (u64)threadIdx.x * TS_PER;
+    u64 v[TS_PER], sum = 0;
 #pragma unroll
-    for (int k = 0; k < RT_PER; ++k) { v[k] = i0 + k < n_tiles ? tile_sum[i0 + k] : 0; sum += v[k]; }
-    u64 total;
-    u64 run = carry + cta_exclusive_scan(sum, &total, s_warp);
+    for (int k = 0; k < TS_PER; ++k) { v[k] = i0 + k < n_tiles ? tile_sum[i0 + k] : 0; sum += v[k]; }
+    u64 inc = sum;
 #pragma unroll
-    for (int k = 0; k < RT_PER; ++k) { if (i0 + k < n_tiles) tile_sum[i0 + k] = run; run += v[k]; }
+    for (int d = 1; d < 32; d <<= 1) { const u64 o = __shfl_up_sync(0xFFFFFFFFu, inc, d); if (lane >= (u32)d) inc += o; }
+    if (lane == 31) s_warp[wid] = inc;
+    __syncthreads();
+    // every warp scans the 32 warp totals itself
+    u64 w = s_warp[lane], winc = w;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) { const u64 o = __shfl_up_sync(0xFFFFFFFFu, winc, d); if (lane >= (u32)d) winc += o; }
+    const u64 before = __shfl_sync(0xFFFFFFFFu, winc - w, wid), total = __shfl_sync(0xFFFFFFFFu, winc, 31);
+    u64 run = carry + before + inc - sum;
+#pragma unroll
+    for (int k = 0; k < TS_PER; ++k) { if (i0 + k < n_tiles) tile_sum[i0 + k] = run; run += v[k]; }
     carry += total;
+    __syncthreads();                                  // s_warp is written again in the next round
   }
 }
 
@@ -219,6 +213,37 @@ __device__ __forceinline__ u64 ticks_upto_guess(const i64* __restrict__ tn, u64 
   return j;
 }
 
+// The same three searches with 32-bit indices relative to the start of a rank's segment (segments of fewer than 2^32
+// ticks, which is every segment that fits a GPU's memory next to its records; longer ones take the 64-bit forms above).
+__device__ __forceinline__ u32 seg_upto(const i64* __restrict__ tn, u32 a, u32 b, i64 t) {      // first index of [a, b) whose tick is after t
+  for (int step = 0; step < 32 && a < b; ++step) { const u32 mid = a + ((b - a) >> 1); if (__ldg(tn + mid) <= t) a = mid + 1; else b = mid; }
+  return a;
+}
+__device__ __forceinline__ u32 seg_upto_near(const i64* __restrict__ tn, u32 from, u32 n, i64 t) {   // every tick of [0, from) is at or before t
+  u32 pos = from, bound = 1;
+  for (int step = 0; step < 32 && pos + bound - 1 < n && __ldg(tn + pos + bound - 1) <= t; ++step) { pos += bound; bound <<= 1; }
+  const u32 end = pos + bound - 1 < n ? pos + bound - 1 : n;
+  return seg_upto(tn, pos, end, t);
+}
+__device__ __forceinline__ u32 seg_upto_guess(const i64* __restrict__ tn, u32 n, i64 t) {
+  const i64 t0 = __ldg(tn), t1 = __ldg(tn + n - 1);
+  if (t < t0) return 0;
+  if (t >= t1) return n;
+  // tn[0] <= t < tn[n - 1]: the first tick after t has index j in [1, n - 1]
+  u32 g = (u32)(__fdividef((float)(t - t0), (float)(t1 - t0)) * (float)(n - 1));
+  g = g > n - 2 ? n - 2 : g;
+  if (__ldg(tn + g) <= t) {
+    u32 pos = g, step = 1;                          // tn[pos] <= t
+    for (int it = 0; it < 32 && pos + step < n && __ldg(tn + pos + step) <= t; ++it) { pos += step; step <<= 1; }
+    const u32 end = pos + step < n - 1 ? pos + step : n - 1;          // tn[end] > t
+    return seg_upto(tn, pos + 1, end, t);
+  }
+  u32 pos = g, step = 1;                            // tn[pos] > t
+  for (int it = 0; it < 32 && pos >= step && __ldg(tn + pos - step) > t; ++it) { pos -= step; step <<= 1; }
+  const u32 start = pos >= step ? pos - step : 0;                     // tn[start] <= t
+  return seg_upto(tn, start + 1, pos, t);
+}
+
 __global__ void __launch_bounds__(RT_THREADS) k_record_rates(TickArgs A, u64 n_rec, const u32* __restrict__ rank, const i64* __restrict__ t_enter,
                                                            const i64* __restrict__ t_exit, u32* __restrict__ send_chg, u32* __restrict__ recv_chg) {
   const u64 i = (u64)blockIdx.x * RT_THREADS + threadIdx.x;
@@ -229,8 +254,15 @@ __global__ void __launch_bounds__(RT_THREADS) k_record_rates(TickArgs A, u64 n_r
     const u64 lo = A.tick_off[r], hi = A.tick_off[r + 1];
     if (hi > lo) {
       const i64 a = t_enter[i], b = t_exit[i];
-      const u64 ca = ticks_upto_guess(A.tick_ns, lo, hi, a);
-      const u64 cb = b == -1 ? hi - lo : (b < a ? 0 : ca + ticks_upto_near(A.tick_ns, lo + ca, hi, b));
+      u64 ca, cb;
+      if (hi - lo < 0xFFFFFFFFull) {
+        const i64* __restrict__ tn = A.tick_ns + lo; const u32 n = (u32)(hi - lo);
+        const u32 xa = seg_upto_guess(tn, n, a);
+        ca = xa; cb = b == -1 ? n : (b < a ? 0u : seg_upto_near(tn, xa, n, b));
+      } else {
+        ca = ticks_upto_guess(A.tick_ns, lo, hi, a);
+        cb = b == -1 ? hi - lo : (b < a ? 0 : ca + ticks_upto_near(A.tick_ns, lo + ca, hi, b));
+      }
       // a rank's first tick has no indicator, so the prefix "before the first tick" equals the prefix at it
       const u64 ia = lo + (ca ? ca - 1 : 0), ib = lo + (cb ? cb - 1 : 0);
       if (ib > ia) {
