@@ -387,6 +387,9 @@ int ccld_derive_rates(ccld_ctx* ctx, uint64_t n_rec, const uint32_t* rank, const
  * launches since timing was last enabled. Kinds: 0 op-counter range, 1 slot layout and work lists
  * (two launches per call), 2 slot scatter, 3 reductions n <= 128 (fused), 4 reductions n <= 1024,
  * 5 reductions n > 1024, 6 window decision. Enabling (on = 1) clears the sums; on = 0 stops timing.
+ * Independently of this switch, every entry point and every stage of ccld_analyze_window opens a named NVTX range
+ * ("ccld_analyze_window", "ccld: slot scatter", ...) on the calling thread, which costs nothing unless a timeline
+ * tool is attached.
  */
 #define CCLD_K_KINDS 7
 int ccld_timing_enable(ccld_ctx* ctx, int on);

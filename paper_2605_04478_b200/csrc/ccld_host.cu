@@ -11,6 +11,8 @@
 #include <unordered_map>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "ccld_kernels.cuh"
 #include "ccld_rates.cuh"
 #include "ccld_opset.cuh"
@@ -137,9 +139,18 @@ TimerSlot* timer_begin(ccld_ctx* ctx) {
   timer_harvest(ctx, s);
   return &s;
 }
-struct TimedLaunch {                                     // records an event pair around one launch
-  TimerSlot* s; cudaStream_t st; int i;
-  TimedLaunch(TimerSlot* slot, int kind, cudaStream_t stream) : s(slot), st(stream), i(-1) {
+// A named range for timeline tools (a no-op unless one is attached).
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+  NvtxRange(const NvtxRange&) = delete; NvtxRange& operator=(const NvtxRange&) = delete;
+};
+const char* const STAGE_NAMES[CCLD_K_KINDS] = {"ccld: op-counter ranges", "ccld: layout", "ccld: slot scatter", "ccld: reduce (up to 128 ranks)",
+                                               "ccld: reduce (129 to 1024 ranks)", "ccld: reduce (more than 1024 ranks)", "ccld: window decision"};
+
+struct TimedLaunch {                                     // a named range and, when timing is on, an event pair around one launch
+  NvtxRange r; TimerSlot* s; cudaStream_t st; int i;
+  TimedLaunch(TimerSlot* slot, int kind, cudaStream_t stream) : r(STAGE_NAMES[kind]), s(slot), st(stream), i(-1) {
     if (s && s->n < TIMER_PAIRS) { i = s->n++; s->kind[i] = kind; cudaEventRecord(s->a[i], st); }
   }
   ~TimedLaunch() { if (i >= 0) cudaEventRecord(s->b[i], st); }
@@ -419,6 +430,7 @@ int ccld_trace_upload(ccld_ctx* ctx, uint32_t window_id, uint64_t n_rec, int mem
                       const uint32_t* send_chg, const uint32_t* recv_chg,
                       uint32_t n_frames, const uint32_t* f_rank, const uint32_t* f_comm, const uint32_t* f_seq,
                       uint32_t n_channels, const uint32_t* progress) {
+  NvtxRange nvtx_range("ccld_trace_upload");
   if (!ctx) return CCLD_ERR_ARG;
   if (mem_kind != 0 && mem_kind != 1) return fail(ctx, CCLD_ERR_ARG, "mem_kind must be 0 (host) or 1 (device)");
   if (n_rec >= 0xFFFFFFFFull) return fail(ctx, CCLD_ERR_CAPACITY, "window of 2^32 - 1 or more records");
@@ -493,6 +505,7 @@ int ccld_reset(ccld_ctx* ctx) {
 }
 
 int ccld_analyze_window(ccld_ctx* ctx, uint32_t first_window, uint32_t n_windows, int64_t now_ns) {
+  NvtxRange nvtx_range("ccld_analyze_window");
   if (!ctx) return CCLD_ERR_ARG;
   if (n_windows == 0) return fail(ctx, CCLD_ERR_ARG, "n_windows is zero");
   if (n_windows > 65535) return fail(ctx, CCLD_ERR_CAPACITY, "more than 65,535 windows in one batch");
@@ -689,6 +702,7 @@ int analyze_batch(ccld_ctx* ctx, u32 first_window, u32 n_windows, i64 now_ns, bo
 extern "C" {
 
 int ccld_get_verdict(ccld_ctx* ctx, uint32_t window_id, ccld_verdict* out) {
+  NvtxRange nvtx_range("ccld_get_verdict");
   if (!ctx || !out) return CCLD_ERR_ARG;
   WindowHost* w;
   { int rc = find_analysed(ctx, window_id, &w); if (rc != CCLD_OK) return rc; }
@@ -756,6 +770,7 @@ static int hang_layers(ccld_ctx* ctx, const CommHost& c, HangArgs* A) {
 }
 
 int ccld_locate_hang(ccld_ctx* ctx, uint32_t window_id, uint32_t comm, uint32_t seq, ccld_hang_verdict* out) {
+  NvtxRange nvtx_range("ccld_locate_hang");
   if (!ctx || !out) return CCLD_ERR_ARG;
   WindowHost* w;
   { int rc = find_analysed(ctx, window_id, &w); if (rc != CCLD_OK) return rc; }
