@@ -118,7 +118,9 @@ __global__ void __launch_bounds__(RT_THREADS) k_tick_blocks(TickArgs A) {
   }
 }
 
-// One CTA of 1,024 threads, 16 consecutive sums per thread and round: 16,384 tiles (33.5 M ticks) per round.
+// One CTA of 1,024 threads; a round covers 16,384 tiles (33.5 M ticks). A warp owns 512 consecutive sums of the round and
+// reads them 32 at a time, lanes on consecutive sums (coalesced, all sixteen loads issued before the first is used), scans
+// each 32 with shuffles and carries its running total from step to step; the warps' totals are scanned by every warp.
 constexpr int TS_THREADS = 1024;
 constexpr int TS_PER = 16;
 __global__ void __launch_bounds__(TS_THREADS) k_tile_scan(u64* __restrict__ tile_sum, u64 n_tiles) {
@@ -126,24 +128,28 @@ __global__ void __launch_bounds__(TS_THREADS) k_tile_scan(u64* __restrict__ tile
   const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
   u64 carry = 0;
   for (u64 base = 0; base < n_tiles; base += (u64)TS_THREADS * TS_PER) {
-    const u64 i0 = base + (u64)threadIdx.x * TS_PER;
-    u64 v[TS_PER], sum = 0;
+    const u64 i0 = base + (u64)wid * (32 * TS_PER) + lane;
+    u64 v[TS_PER];
 #pragma unroll
-    for (int k = 0; k < TS_PER; ++k) { v[k] = i0 + k < n_tiles ? tile_sum[i0 + k] : 0; sum += v[k]; }
-    u64 inc = sum;
+    for (int k = 0; k < TS_PER; ++k) v[k] = i0 + 32 * k < n_tiles ? tile_sum[i0 + 32 * k] : 0;
+    u64 run = 0;                                      // the warp's sums before step k
 #pragma unroll
-    for (int d = 1; d < 32; d <<= 1) { const u64 o = __shfl_up_sync(0xFFFFFFFFu, inc, d); if (lane >= (u32)d) inc += o; }
-    if (lane == 31) s_warp[wid] = inc;
+    for (int k = 0; k < TS_PER; ++k) {
+      u64 inc = v[k];
+#pragma unroll
+      for (int d = 1; d < 32; d <<= 1) { const u64 o = __shfl_up_sync(0xFFFFFFFFu, inc, d); if (lane >= (u32)d) inc += o; }
+      v[k] = run + inc - v[k];                        // exclusive inside the warp's span
+      run += __shfl_sync(0xFFFFFFFFu, inc, 31);
+    }
+    if (lane == 0) s_warp[wid] = run;
     __syncthreads();
-    // every warp scans the 32 warp totals itself
     u64 w = s_warp[lane], winc = w;
 #pragma unroll
     for (int d = 1; d < 32; d <<= 1) { const u64 o = __shfl_up_sync(0xFFFFFFFFu, winc, d); if (lane >= (u32)d) winc += o; }
-    const u64 before = __shfl_sync(0xFFFFFFFFu, winc - w, wid), total = __shfl_sync(0xFFFFFFFFu, winc, 31);
-    u64 run = carry + before + inc - sum;
+    const u64 before = carry + __shfl_sync(0xFFFFFFFFu, winc - w, wid);
+    carry += __shfl_sync(0xFFFFFFFFu, winc, 31);
 #pragma unroll
-    for (int k = 0; k < TS_PER; ++k) { if (i0 + k < n_tiles) tile_sum[i0 + k] = run; run += v[k]; }
-    carry += total;
+    for (int k = 0; k < TS_PER; ++k) if (i0 + 32 * k < n_tiles) tile_sum[i0 + 32 * k] = before + v[k];
     __syncthreads();                                  // s_warp is written again in the next round
   }
 }
