@@ -696,3 +696,65 @@ def test_a_batch_that_does_not_match_its_expected_layout_is_analysed_again_in_or
     an.analyze_window(0, spec.n_windows, now)
     for w in range(spec.n_windows):
         compare_window(an, o, w)
+
+
+def mismatching_windows(spec):
+    """The windows of `spec` on the CPU; window 2 keeps its record count but carries one record with a far later op counter."""
+    cols = []
+    for w in range(spec.n_windows):
+        c = {k: v.clone() for k, v in tg.gen_window(spec, w, device="cpu").cols.items()}
+        if w == 2:
+            c["seq"][7] += 500
+        cols.append(c)
+    return cols
+
+
+def test_state_exported_while_batches_wait_is_the_state_after_all_of_them():
+    """Calls that did not wait, one of them with a layout other than the expected one, and then - before any result is
+    read - the cumulative state is exported and carried to a fresh context together with one more window. What arrives
+    there must be the state after all five windows, in order: the export has to settle what is still waiting first."""
+    spec = tg.cfg2(reps=40, n_windows=6, tp=8, pp=2, dp=16)
+    params = dict(m_max_rounds=100, tbase_init_ns=100_000)
+    reg = tg.registry(spec)
+    an_a, o = make_pair(reg, params)
+    an_b, _ = make_pair(reg, params)
+    cols = mismatching_windows(spec)
+    for w in range(5):
+        an_a.trace_upload(w, cols[w]); assert o.upload(w, cols[w]) == 0
+    an_b.trace_upload(5, cols[5]); assert o.upload(5, cols[5]) == 0
+    now = tg.gen_window(spec, spec.n_windows - 1).now_ns
+    for w in range(5):
+        an_a.analyze_window(w, 1, now)
+    blob = an_a.state_export()                                   # nothing was read back before this
+    an_b.state_import(blob)
+    an_b.analyze_window(5, 1, now)
+    assert o.analyze(0, 6, now) == 0
+    compare_window(an_b, o, 5)
+    compare_cumulative(an_b, o, spec.n_ranks, 5)
+    for w in range(5):
+        compare_window(an_a, o, w)
+
+
+def test_reset_and_release_while_batches_wait():
+    """A reset right behind calls that did not wait discards them (also the one that would have had to be analysed again);
+    a window released while its batch waits is settled first and the windows of the same batch stay readable."""
+    spec = tg.cfg2(reps=40, n_windows=5, tp=8, pp=2, dp=16)
+    params = dict(m_max_rounds=100, tbase_init_ns=100_000)
+    reg = tg.registry(spec)
+    an, o = make_pair(reg, params)
+    cols = mismatching_windows(spec)
+    for w, c in enumerate(cols):
+        an.trace_upload(w, c); assert o.upload(w, c) == 0
+    now = tg.gen_window(spec, spec.n_windows - 1).now_ns
+    for w in range(spec.n_windows):
+        an.analyze_window(w, 1, now)
+    an.reset()                                                   # windows 2 to 4 were waiting to be analysed again
+    for w in range(spec.n_windows):
+        an.analyze_window(w, 1, now)
+    an.window_release(3)                                         # its batch gave up behind window 2 and is still waiting
+    assert o.analyze(0, spec.n_windows, now) == 0
+    for w in (0, 1, 2, 4):
+        compare_window(an, o, w)
+    compare_cumulative(an, o, spec.n_ranks, 4)
+    with pytest.raises(ccld.CcldError):
+        an.get_verdict(3)
