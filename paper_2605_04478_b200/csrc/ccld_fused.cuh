@@ -278,6 +278,10 @@ __device__ __forceinline__ void fast_groups(const WinDesc& D, u32 w_idx, const R
   u64 base;
   bool mm = false;
   u64 gby, ck = 0; u32 gop;
+  // thread per group: lane m fetches the rank of ring position m now, so that the ranks a row names are a shuffle away
+  // when the row is written instead of one more round trip to memory
+  u32 mem_l = 0;
+  if (L == 1) mem_l = lane < n ? __ldg(mem + lane) : 0u;
   if (STAGED) {
     base = sh.t_base[jt]; gby = sh.t_gby[jt]; gop = sh.t_gop[jt];
     const u32 bits = sh.t_bits[jt];
@@ -375,6 +379,10 @@ __device__ __forceinline__ void fast_groups(const WinDesc& D, u32 w_idx, const R
   for (int q = 7; q >= 0; --q) {
     if (FULL || p0 + q < n) { const u32 d = kd[q * KSTEP]; if (d == tmx) pmax = p0 + q; if (d == tmn) pmin = p0 + q; }
   }
+  u32 r_tmin = 0, r_tmax = 0, r_chg = 0;                      // ranks the row names
+  if (L == 1) {                                             // all lanes are still here
+    r_tmin = __shfl_sync(FULLM, mem_l, pmin & 31u); r_tmax = __shfl_sync(FULLM, mem_l, pmax & 31u); r_chg = __shfl_sync(FULLM, mem_l, (NONE - (u32)ck) & 31u);
+  }
   bool mismatch = mm;
   if (L > 1) {
 #pragma unroll
@@ -448,6 +456,7 @@ __device__ __forceinline__ void fast_groups(const WinDesc& D, u32 w_idx, const R
       for (int q = 0; q < 8; ++q) if (FULL || p0 + q < n) fp[q] = (u8)((q < 4 ? f_lo >> (8 * q) : f_hi >> (8 * (q - 4))) & 0xFFu);
     }
   }
+  if (L > 1) { r_tmin = mem[pmin]; r_tmax = mem[pmax]; r_chg = mem[NONE - (u32)ck]; }
   if (lead) {
     const u64 g = row.group0 + seq0 + j, G = ld_volatile(sh.out.G);
     i64* __restrict__ gi = ld_volatile(sh.out.gi64) + g; u32* __restrict__ gu = ld_volatile(sh.out.gu32) + g;
@@ -456,8 +465,8 @@ __device__ __forceinline__ void fast_groups(const WinDesc& D, u32 w_idx, const R
     gi[(u64)GI_T_MAX * G] = (i64)(u64)tmx; gi[(u64)GI_T_MIN * G] = (i64)(u64)tmn; gi[(u64)GI_SPAN * G] = (i64)(u64)span;
     gi[(u64)GI_MED_SKEW * G] = (i64)(u64)ms; gi[(u64)GI_MAD_SKEW * G] = (i64)(u64)ds;
     gi[(u64)GI_MED_DUR * G] = analysed ? (i64)((u64)tmn + md) : 0; gi[(u64)GI_MAD_DUR * G] = (i64)(u64)dm;
-    gu[(u64)GU_RANK_TMIN * G] = mem[pmin]; gu[(u64)GU_RANK_TMAX * G] = mem[pmax];
-    gu[(u64)GU_MAX_CHG * G] = (u32)(ck >> 32); gu[(u64)GU_RANK_MAX_CHG * G] = mem[NONE - (u32)ck];
+    gu[(u64)GU_RANK_TMIN * G] = r_tmin; gu[(u64)GU_RANK_TMAX * G] = r_tmax;
+    gu[(u64)GU_MAX_CHG * G] = (u32)(ck >> 32); gu[(u64)GU_RANK_MAX_CHG * G] = r_chg;
     gu[(u64)GU_N_PRESENT * G] = n;
     gu[(u64)GU_GFLAGS * G] = CCLD_G_COMPLETE | (barrier ? CCLD_G_BARRIER : 0) | (mismatch ? CCLD_G_OPSET_MISMATCH : 0) | (analysed ? CCLD_G_ANALYSED : 0);
     ld_volatile(sh.out.gbw)[g] = span ? bn * rcp_newton((double)span * den) : 0.0;
