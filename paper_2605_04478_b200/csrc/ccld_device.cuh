@@ -109,7 +109,9 @@ struct WinDesc {
   u32 cta0, n_cta;                   // this window's CTAs in the record-streaming grids
   u32 *rmin, *rmax;                  // [n_comms] op counter range seen
   RangeRow* ranges;                  // [n_comms]
-  uint4* srow;                       // [n_comms] scatter rows: (slot0 - seq_lo * n) low, high, n (0 = nothing to place), seq_lo
+  uint4* srow;                       // [n_comms] scatter rows: first slot low, high, op counters covered (0 = nothing to place), first op counter
+  uint4* rent;                       // [n_ranks][RANK_TAB_K] a rank's inline pairs resolved for this window: (communicator id, op counters
+                                     //   covered (0: unused), first op counter, first slot of the member's column); 32-bit slots only
   u64* totals;                       // [T_COUNT]
   const u64* expect;                 // [T_COUNT] totals the host sized this window's results for without waiting (null: it waited)
   u32* poison;                       // set once a window's layout differs from what the host expected: every window planned later gives up too

@@ -553,7 +553,7 @@ int analyze_batch(ccld_ctx* ctx, u32 first_window, u32 n_windows, i64 now_ns, bo
   size_t off = 0;
   auto take = [&](size_t b) { size_t o = off; off = align_up(off + b); return o; };
   const size_t o_desc = take(B * sizeof(WinDesc)), o_rmin = take((size_t)B * nc * 4), o_rmax = take((size_t)B * nc * 4),
-               o_rng = take((size_t)B * nc * sizeof(RangeRow)), o_srow = take((size_t)B * nc * sizeof(uint4)), o_tot = take((size_t)B * T_COUNT * 8), o_cnt = take((size_t)B * C_COUNT * 8),
+               o_rng = take((size_t)B * nc * sizeof(RangeRow)), o_srow = take((size_t)B * nc * sizeof(uint4)), o_rent = take((size_t)B * ctx->n_ranks * RANK_TAB_K * sizeof(uint4)), o_tot = take((size_t)B * T_COUNT * 8), o_cnt = take((size_t)B * C_COUNT * 8),
                o_zero_end = off, o_exp = take(expect ? (size_t)B * T_COUNT * 8 : 0);
   cudaError_t e;
   Block pb = ctx->pool.get(off, &e);
@@ -568,6 +568,7 @@ int analyze_batch(ccld_ctx* ctx, u32 first_window, u32 n_windows, i64 now_ns, bo
     d.n_cta = (u32)((d.n_rec + REC_PER_CTA - 1) / REC_PER_CTA); d.cta0 = 0; cta = std::max<u64>(cta, d.n_cta);
     d.rmin = (u32*)(pbase + o_rmin) + (size_t)k * nc; d.rmax = (u32*)(pbase + o_rmax) + (size_t)k * nc;
     d.ranges = (RangeRow*)(pbase + o_rng) + (size_t)k * nc; d.srow = (uint4*)(pbase + o_srow) + (size_t)k * nc;
+    d.rent = (uint4*)(pbase + o_rent) + (size_t)k * ctx->n_ranks * RANK_TAB_K;
     d.totals = (u64*)(pbase + o_tot) + (size_t)k * T_COUNT; d.counters = (u64*)(pbase + o_cnt) + (size_t)k * C_COUNT;
     d.expect = expect ? (const u64*)(pbase + o_exp) + (size_t)k * T_COUNT : nullptr; d.poison = ctx->d_poison;
     d.n_groups = d.n_slots = 0; d.perm = nullptr; d.flags = nullptr; d.skey = d.dkey = nullptr; d.gi64 = nullptr; d.gu32 = nullptr; d.gbw = nullptr;
@@ -644,7 +645,7 @@ int analyze_batch(ccld_ctx* ctx, u32 first_window, u32 n_windows, i64 now_ns, bo
   if (total_slots) CK(cudaMemsetAsync(rbase + o_perm, 0xFF, total_slots * 4, st));
   PlanLists pl; pl.fcta = (FusedCta*)(rbase + o_fcta); pl.fwt = (WarpTile*)(rbase + o_fwt); pl.t2 = (Tile*)(rbase + o_t2); pl.t3 = (Tile*)(rbase + o_t3);
   { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, pl, 1); }
-  if (cta > 0) { TimedLaunch tl(ts, 2, st); k_slot_scatter<<<dim3((u32)cta, B), SCAT_THREADS, 0, st>>>(d_desc, ctx->reg); }
+  if (cta > 0) { TimedLaunch tl(ts, 2, st); k_slot_scatter<<<dim3((u32)((cta * REC_PER_CTA + SCAT_PER_CTA - 1) / SCAT_PER_CTA), B), SCAT_THREADS, 0, st>>>(d_desc, ctx->reg); }
   CK(cudaMemsetAsync(rbase + o_defn, 0, 16, st));
   if (n_list[B_FCTA]) {
     const DeferList dl{(u64*)(rbase + o_def), (u32*)(rbase + o_defn)};

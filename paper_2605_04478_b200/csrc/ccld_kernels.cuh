@@ -404,8 +404,12 @@ __device__ __forceinline__ u32 comm_units(u32 ns, u32 n, u32 T) {
 struct PlanLists { FusedCta* fcta; WarpTile* fwt; Tile* t2; Tile* t3; };
 
 // A window that is given up leaves no work behind: zero ranges and scatter rows, zero totals.
-__device__ __forceinline__ void plan_give_up(WinDesc& D, const Registry& R, u64 why) {
+__device__ __forceinline__ void plan_clear_rows(WinDesc& D, const Registry& R) {
   for (u32 c = threadIdx.x; c < R.n_comms; c += PLAN_THREADS) { RangeRow z = {0, 0, 0, R.comm_n[c], 0, 0, 0, 0}; D.ranges[c] = z; D.srow[c] = make_uint4(0, 0, 0, 0); }
+  for (u64 i = threadIdx.x; i < (u64)R.n_ranks * RANK_TAB_K; i += PLAN_THREADS) D.rent[i] = make_uint4(0, 0, 0, 0);
+}
+__device__ __forceinline__ void plan_give_up(WinDesc& D, const Registry& R, u64 why) {
+  plan_clear_rows(D, R);
   if (threadIdx.x == 0) {
     for (int q = 0; q < T_COUNT; ++q) D.totals[q] = 0;
     D.totals[T_FAILED] = why; D.totals[T_CHUNKS] = 1;
@@ -507,8 +511,27 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
       if (failed == FAILED_CAPACITY) atomicOr((unsigned*)&D.counters[C_ERR], (unsigned)CCLD_E_CAPACITY);
     }
     __syncthreads();
-    if (s_failed)
-      for (u32 c = threadIdx.x; c < R.n_comms; c += PLAN_THREADS) { RangeRow z = {0, 0, 0, R.comm_n[c], 0, 0, 0, 0}; D.ranges[c] = z; D.srow[c] = make_uint4(0, 0, 0, 0); }
+    if (s_failed) { plan_clear_rows(D, R); return; }
+    // 4. every rank's inline (communicator, position) pairs resolved against this window's scatter rows, so that the
+    //    scatter pass finds (op counters covered, first op counter, first slot of the member's column) with one load.
+    //    Only where slots fit 32 bits and the member's whole column lies inside the table; other entries stay unused.
+    if (run.slots <= 0xFFFFFFFFull) {
+#pragma unroll 4
+      for (u64 i = threadIdx.x; i < (u64)R.n_ranks * 2; i += PLAN_THREADS) {
+        const uint4 t = R.rank_tab[i];
+        uint4 e[2] = {make_uint4(0, 0, 0, 0), make_uint4(0, 0, 0, 0)};
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const u32 id = h ? t.z : t.x, cp = h ? t.w : t.y;
+          if (id != NONE && cp != NONE && cp != RANK_TAB_OVERFLOW) {
+            const uint4 sr = D.srow[cp >> RANK_TAB_POS_BITS];
+            const u64 b = ((u64)sr.x | ((u64)sr.y << 32)) + (u64)(cp & ((1u << RANK_TAB_POS_BITS) - 1)) * sr.z;
+            if (sr.z != 0 && b + sr.z <= run.slots) e[h] = make_uint4(id, sr.z, sr.w, (u32)b);
+          }
+        }
+        D.rent[i * 2] = e[0]; D.rent[i * 2 + 1] = e[1];
+      }
+    }
     return;
   }
 
@@ -588,7 +611,8 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
 // Registry walk for a record whose (rank, communicator) pair is not inline: returns index << 13 | position in the
 // low word, or NONE there with the rejecting CCLD_E_* bit in the high word.
 constexpr int SCAT_THREADS = 256;     // lanes on consecutive records: the stores of a warp land close together
-constexpr int SCAT_PER_THREAD = REC_PER_CTA / SCAT_THREADS;
+constexpr int SCAT_PER_THREAD = 12;    // records per thread: enough to spread the two dependent table reads a warp starts with
+constexpr int SCAT_PER_CTA = SCAT_THREADS * SCAT_PER_THREAD;
 
 __device__ __noinline__ u64 resolve_slow(const Registry& R, u32 rank, u32 cid) {
   const u32 c = comm_lookup(R, cid);
@@ -612,11 +636,11 @@ __device__ __forceinline__ bool scatter_slot(const Registry& R, u32 c, u32 ns, u
   return true;
 }
 
-constexpr u32 SCAT_LOCAL = 4;     // ranks, counted from the rank of the CTA's first record, whose table rows a CTA resolves once
+constexpr u32 SCAT_LOCAL = 8;     // ranks, counted from the rank of the CTA's first record, whose table rows a CTA resolves once
 
-// A CTA's records mostly belong to a few neighbouring ranks (a rank-major upload: one or two), so the CTA first resolves
-// the inline table rows of SCAT_LOCAL ranks - communicator id -> (counters covered, first counter, slot of the member's
-// first counter) - into shared memory; a record of those ranks then needs no global table at all and, in windows of
+// A CTA's records mostly belong to a few neighbouring ranks (a rank-major upload: one or two), so each warp first copies
+// the resolved inline pairs of SCAT_LOCAL ranks - communicator id -> (counters covered, first counter, slot of the member's
+// first counter), which the layout pass wrote for this window - into shared memory; a record of those ranks then needs no global table at all and, in windows of
 // fewer than 2^32 slots, only 32-bit arithmetic. Any other record (another rank, a communicator beyond the inline pairs,
 // a counter outside the range, a rejected record) takes the two dependent table loads and the full checks.
 __global__ void __launch_bounds__(SCAT_THREADS, 4) k_slot_scatter(const WinDesc* __restrict__ wd, Registry R) {
@@ -624,8 +648,8 @@ __global__ void __launch_bounds__(SCAT_THREADS, 4) k_slot_scatter(const WinDesc*
   // warp resolves its own copy, so no warp waits for another.
   __shared__ uint4 s_ent_all[SCAT_THREADS / 32][SCAT_LOCAL * RANK_TAB_K];
   const WinDesc& D = wd[blockIdx.y];                          // grid: (CTAs of the largest window, windows)
-  if (blockIdx.x >= D.n_cta) return;                          // (a window that was given up has empty scatter rows: nothing is stored)
-  const u64 base = (u64)blockIdx.x * REC_PER_CTA;
+  const u64 base = (u64)blockIdx.x * SCAT_PER_CTA;
+  if (base >= D.n_rec) return;                                // (a window that was given up has empty scatter rows: nothing is stored)
   u32 err = 0, rej = 0, internal = 0;
   // descriptor fields in registers: the stores below could alias the descriptor as far as the compiler knows
   u32* const perm = D.perm; const u64 n_slots = D.n_slots; const uint4* const srow = D.srow; const u64 n_rec = D.n_rec;
@@ -644,17 +668,9 @@ __global__ void __launch_bounds__(SCAT_THREADS, 4) k_slot_scatter(const WinDesc*
   uint4* const s_ent = s_ent_all[threadIdx.x >> 5];
   const u32 r_first = c_rank[base];
   if (lane < SCAT_LOCAL * RANK_TAB_K) {
-    const u32 r = r_first + lane / RANK_TAB_K, k = lane % RANK_TAB_K;
+    const u32 r = r_first + lane / RANK_TAB_K;
     uint4 e = make_uint4(NONE, 0, 0, 0);
-    if (n_slots <= 0xFFFFFFFFull && r_first < R.n_ranks && r < R.n_ranks) {
-      const uint4 t = R.rank_tab[(u64)r * 2 + (k >> 1)];
-      const u32 id = (k & 1) ? t.z : t.x, cp = (k & 1) ? t.w : t.y;
-      if (id != NONE && cp != NONE && cp != RANK_TAB_OVERFLOW) {
-        const uint4 sr = srow[cp >> RANK_TAB_POS_BITS];
-        const u64 b = ((u64)sr.x | ((u64)sr.y << 32)) + (u64)(cp & ((1u << RANK_TAB_POS_BITS) - 1)) * sr.z;
-        if (b + sr.z <= n_slots) e = make_uint4(id, sr.z, sr.w, (u32)b);    // the member's whole column lies inside the table
-      }
-    }
+    if (r_first < R.n_ranks && r < R.n_ranks) e = D.rent[(u64)r * RANK_TAB_K + lane % RANK_TAB_K];
     s_ent[lane] = e;
   }
   __syncwarp();
