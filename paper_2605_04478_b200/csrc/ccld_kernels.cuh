@@ -671,6 +671,7 @@ __global__ void __launch_bounds__(SCAT_THREADS, 4) k_slot_scatter(const WinDesc*
     const u32 r = r_first + lane / RANK_TAB_K;
     uint4 e = make_uint4(NONE, 0, 0, 0);
     if (r_first < R.n_ranks && r < R.n_ranks) e = D.rent[(u64)r * RANK_TAB_K + lane % RANK_TAB_K];
+    if (e.y == 0) e.x = NONE;                                 // an unused pair must not shadow a record of communicator 0
     s_ent[lane] = e;
   }
   __syncwarp();
