@@ -291,7 +291,7 @@ __global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __rest
   __syncthreads();
   for (u32 c = threadIdx.x; c < R.n_comms; c += REC_THREADS) {
     const u32 mn = s_mn[c];
-    if (mn != NONE) range_widen(D, c, mn, s_mx[c]);
+    if (mn != NONE) { atomicMin(&D.rmin[c], mn); atomicMax(&D.rmax[c], s_mx[c]); }      // nothing waits for these
   }
 }
 
