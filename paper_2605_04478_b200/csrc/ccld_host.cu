@@ -586,7 +586,13 @@ int analyze_batch(ccld_ctx* ctx, u32 first_window, u32 n_windows, i64 now_ns, bo
     if (r == cudaSuccess && expect) r = cudaMemcpyAsync(pbase + o_exp, expect->totals.data(), (size_t)B * T_COUNT * 8, cudaMemcpyHostToDevice, st);
     if (r == cudaSuccess) r = cudaMemcpyAsync(d_desc, hd.data(), B * sizeof(WinDesc), cudaMemcpyHostToDevice, st);
     if (r != cudaSuccess) return r;
-    if (cta > 0) { TimedLaunch tl(ts, 0, st); k_seq_range<<<dim3((u32)cta, B), REC_THREADS, range_smem_bytes(nc), st>>>(d_desc, ctx->reg); }
+    if (cta > 0) {
+      // enough CTAs to fill the device several times over, then as many blocks per CTA as that leaves
+      const u64 want = 32ull * ctx->n_sms;
+      const u32 per = (u32)std::min<u64>(RANGE_BLOCKS_MAX, std::max<u64>(1, cta * B / want));
+      TimedLaunch tl(ts, 0, st);
+      k_seq_range<<<dim3((u32)((cta + per - 1) / per), B), REC_THREADS, range_smem_bytes(nc), st>>>(d_desc, ctx->reg, per);
+    }
     { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, PlanLists{nullptr, nullptr, nullptr, nullptr}, 0); }
     return cudaGetLastError();
   };

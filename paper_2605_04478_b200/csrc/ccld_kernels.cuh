@@ -150,6 +150,7 @@ __device__ __forceinline__ void range_put(const WinDesc& D, u32* s_mn, u32* s_mx
 // record at worst.
 constexpr int RANGE_FOLDS = 4;
 constexpr int RANGE_WARP_FOLDS = 8;
+constexpr u32 RANGE_BLOCKS_MAX = 16;                  // blocks of REC_PER_CTA records a CTA takes at most (the host takes fewer for small batches)
 
 // cid[i] for the lowest i with bit i of `left` set (any element if left is 0)
 __device__ __forceinline__ u32 first_left(const u32 (&cid)[REC_RUN], u32 left) {
@@ -164,126 +165,131 @@ __device__ __forceinline__ u32 first_left(const u32 (&cid)[REC_RUN], u32 left) {
   return (b & 1u) ? y1 : y0;
 }
 
-__global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __restrict__ wd, Registry R) {
+__global__ void __launch_bounds__(REC_THREADS) k_seq_range(const WinDesc* __restrict__ wd, Registry R, u32 blocks_per_cta) {
   extern __shared__ u32 s_dyn[];
   u32* const s_mn = R.n_comms <= RANGE_DIRECT ? s_dyn : nullptr;
   u32* const s_mx = R.n_comms <= RANGE_DIRECT ? s_dyn + R.n_comms : nullptr;
   const WinDesc& D = wd[blockIdx.y];                          // grid: (CTAs of the largest window, windows)
-  if (blockIdx.x >= D.n_cta) return;
-  const u64 first = (u64)blockIdx.x * REC_PER_CTA;
-  const u32 n_valid = D.n_rec - first < REC_PER_CTA ? (u32)(D.n_rec - first) : (u32)REC_PER_CTA;
+  if ((u64)blockIdx.x * blocks_per_cta * REC_PER_CTA >= D.n_rec) return;
   const u32 lane = threadIdx.x & 31;
-  const u32 r0 = threadIdx.x * REC_RUN;
-  const u32 len = r0 >= n_valid ? 0u : (n_valid - r0 < REC_RUN ? n_valid - r0 : (u32)REC_RUN);
-  // the run goes straight into registers: four 128-bit loads per column where the column allows it
-  u32 cid[REC_RUN], sq[REC_RUN];
-  {
-    const u32* __restrict__ pc = D.comm + first + r0; const u32* __restrict__ ps = D.seq + first + r0;
-    if (len == REC_RUN && ((reinterpret_cast<uintptr_t>(pc) | reinterpret_cast<uintptr_t>(ps)) & 15) == 0) {
-#pragma unroll
-      for (int q = 0; q < REC_RUN / 4; ++q) {
-        const uint4 a = __ldg(reinterpret_cast<const uint4*>(pc) + q), b = __ldg(reinterpret_cast<const uint4*>(ps) + q);
-        cid[4 * q] = a.x; cid[4 * q + 1] = a.y; cid[4 * q + 2] = a.z; cid[4 * q + 3] = a.w;
-        sq[4 * q] = b.x; sq[4 * q + 1] = b.y; sq[4 * q + 2] = b.z; sq[4 * q + 3] = b.w;
-      }
-    } else {
-#pragma unroll
-      for (int k = 0; k < REC_RUN; ++k) { cid[k] = (u32)k < len ? pc[k] : NONE; sq[k] = (u32)k < len ? ps[k] : 0u; }
-    }
-  }
   if (s_mn != nullptr) {
     for (u32 c = threadIdx.x; c < R.n_comms; c += REC_THREADS) { s_mn[c] = NONE; s_mx[c] = 0; }
     __syncthreads();
   }
-  // records of the run not yet accounted for; a run cut short by the end of the window skips the folds (its padding
-  // would match a record that names communicator 0xFFFFFFFF) and goes record by record
-  const u32 tail = len < REC_RUN ? (1u << len) - 1u : 0u;
-  u32 left = len < REC_RUN ? 0u : (1u << REC_RUN) - 1u;
-  // warp folds: in a rank-major upload the 32 runs of a warp belong to one or two ranks, so all lanes meet the same few
-  // communicators. One of them at a time - the communicator of the first record left in the lowest lane that has one -
-  // is folded by every lane and reduced over the warp, and lane 0 updates the table once. The stage ends as soon as a
-  // fold clears less than an eighth of what was left (an upload in another order): the lanes then fold on their own.
-  {
-    u32 remaining = __reduce_add_sync(0xFFFFFFFFu, (u32)__popc(left));
-    for (int f = 0; f < RANGE_WARP_FOLDS && remaining != 0; ++f) {
-      const u32 have = __ballot_sync(0xFFFFFFFFu, left != 0);
-      const u32 id = __shfl_sync(0xFFFFFFFFu, first_left(cid, left), (u32)__ffs(have) - 1u);
-      const uint4 h = comm_find(R, id, R.hash[hash_home(R, id)]);        // the same in every lane
+  // a CTA takes blocks_per_cta consecutive blocks of the window, one after the other, and keeps one table for them: the
+  // table's set-up, its barriers and its merge into the window's ranges are paid once
+  for (u32 blk = 0; blk < blocks_per_cta; ++blk) {
+    const u64 first = ((u64)blockIdx.x * blocks_per_cta + blk) * REC_PER_CTA;
+    if (first >= D.n_rec) break;
+    const u32 n_valid = D.n_rec - first < REC_PER_CTA ? (u32)(D.n_rec - first) : (u32)REC_PER_CTA;
+    const u32 r0 = threadIdx.x * REC_RUN;
+    const u32 len = r0 >= n_valid ? 0u : (n_valid - r0 < REC_RUN ? n_valid - r0 : (u32)REC_RUN);
+    // the run goes straight into registers: four 128-bit loads per column where the column allows it
+    u32 cid[REC_RUN], sq[REC_RUN];
+    {
+      const u32* __restrict__ pc = D.comm + first + r0; const u32* __restrict__ ps = D.seq + first + r0;
+      if (len == REC_RUN && ((reinterpret_cast<uintptr_t>(pc) | reinterpret_cast<uintptr_t>(ps)) & 15) == 0) {
+  #pragma unroll
+        for (int q = 0; q < REC_RUN / 4; ++q) {
+          const uint4 a = __ldg(reinterpret_cast<const uint4*>(pc) + q), b = __ldg(reinterpret_cast<const uint4*>(ps) + q);
+          cid[4 * q] = a.x; cid[4 * q + 1] = a.y; cid[4 * q + 2] = a.z; cid[4 * q + 3] = a.w;
+          sq[4 * q] = b.x; sq[4 * q + 1] = b.y; sq[4 * q + 2] = b.z; sq[4 * q + 3] = b.w;
+        }
+      } else {
+  #pragma unroll
+        for (int k = 0; k < REC_RUN; ++k) { cid[k] = (u32)k < len ? pc[k] : NONE; sq[k] = (u32)k < len ? ps[k] : 0u; }
+      }
+    }
+    // records of the run not yet accounted for; a run cut short by the end of the window skips the folds (its padding
+    // would match a record that names communicator 0xFFFFFFFF) and goes record by record
+    const u32 tail = len < REC_RUN ? (1u << len) - 1u : 0u;
+    u32 left = len < REC_RUN ? 0u : (1u << REC_RUN) - 1u;
+    // warp folds: in a rank-major upload the 32 runs of a warp belong to one or two ranks, so all lanes meet the same few
+    // communicators. One of them at a time - the communicator of the first record left in the lowest lane that has one -
+    // is folded by every lane and reduced over the warp, and lane 0 updates the table once. The stage ends as soon as a
+    // fold clears less than an eighth of what was left (an upload in another order): the lanes then fold on their own.
+    {
+      u32 remaining = __reduce_add_sync(0xFFFFFFFFu, (u32)__popc(left));
+      for (int f = 0; f < RANGE_WARP_FOLDS && remaining != 0; ++f) {
+        const u32 have = __ballot_sync(0xFFFFFFFFu, left != 0);
+        const u32 id = __shfl_sync(0xFFFFFFFFu, first_left(cid, left), (u32)__ffs(have) - 1u);
+        const uint4 h = comm_find(R, id, R.hash[hash_home(R, id)]);        // the same in every lane
+        u32 m = 0, mn = NONE, mx = 0;
+  #pragma unroll
+        for (int k = 0; k < REC_RUN; ++k) {
+          if (cid[k] == id) { m |= 1u << k; mn = min(mn, sq[k]); mx = max(mx, sq[k]); }
+        }
+        m &= left;                                             // a run cut short holds padding and takes no part
+        u32 a = __reduce_min_sync(0xFFFFFFFFu, m ? mn : NONE), b = __reduce_max_sync(0xFFFFFFFFu, m ? mx : 0u);
+        if (h.y != NONE && a < h.z) {
+          // counters below the communicator's first name no operation: fold again without them
+          mn = NONE; mx = 0;
+  #pragma unroll
+          for (int k = 0; k < REC_RUN; ++k) if (((m >> k) & 1u) && sq[k] >= h.z) { mn = min(mn, sq[k]); mx = max(mx, sq[k]); }
+          a = __reduce_min_sync(0xFFFFFFFFu, mn); b = __reduce_max_sync(0xFFFFFFFFu, mx);
+        }
+        if (lane == 0 && h.y != NONE && a <= b) range_put(D, s_mn, s_mx, h.y, a, b);
+        left &= ~m;
+        const u32 cleared = __reduce_add_sync(0xFFFFFFFFu, (u32)__popc(m));
+        const bool worth = cleared * 8u >= remaining;
+        remaining -= cleared;
+        if (!worth) break;
+      }
+    }
+    // folds: the communicator of the first record still left takes every record of the run that names it
+    for (int f = 0; f < RANGE_FOLDS && __any_sync(0xFFFFFFFFu, left != 0); ++f) {
+      const bool act = left != 0;
+      u32 id = NONE;
+  #pragma unroll
+      for (int k = REC_RUN - 1; k >= 0; --k) id = (left >> k) & 1u ? cid[k] : id;
+      uint4 h = make_uint4(0, NONE, 0, 0);                      // (id, index, first counter, members); index NONE: unregistered
+      if (act) h = comm_find(R, id, R.hash[hash_home(R, id)]);
+      // a record folded earlier carries another id, so matching the id is enough (the run is complete: no padding)
       u32 m = 0, mn = NONE, mx = 0;
-#pragma unroll
+  #pragma unroll
       for (int k = 0; k < REC_RUN; ++k) {
         if (cid[k] == id) { m |= 1u << k; mn = min(mn, sq[k]); mx = max(mx, sq[k]); }
       }
-      m &= left;                                             // a run cut short holds padding and takes no part
-      u32 a = __reduce_min_sync(0xFFFFFFFFu, m ? mn : NONE), b = __reduce_max_sync(0xFFFFFFFFu, m ? mx : 0u);
-      if (h.y != NONE && a < h.z) {
+      m &= left;
+      if (h.y != NONE && m != 0 && mn < h.z) {
         // counters below the communicator's first name no operation: fold again without them
         mn = NONE; mx = 0;
-#pragma unroll
+  #pragma unroll
         for (int k = 0; k < REC_RUN; ++k) if (((m >> k) & 1u) && sq[k] >= h.z) { mn = min(mn, sq[k]); mx = max(mx, sq[k]); }
-        a = __reduce_min_sync(0xFFFFFFFFu, mn); b = __reduce_max_sync(0xFFFFFFFFu, mx);
       }
-      if (lane == 0 && h.y != NONE && a <= b) range_put(D, s_mn, s_mx, h.y, a, b);
+      if (m == 0) { mn = NONE; mx = 0; }
       left &= ~m;
-      const u32 cleared = __reduce_add_sync(0xFFFFFFFFu, (u32)__popc(m));
-      const bool worth = cleared * 8u >= remaining;
-      remaining -= cleared;
-      if (!worth) break;
-    }
-  }
-  // folds: the communicator of the first record still left takes every record of the run that names it
-  for (int f = 0; f < RANGE_FOLDS && __any_sync(0xFFFFFFFFu, left != 0); ++f) {
-    const bool act = left != 0;
-    u32 id = NONE;
-#pragma unroll
-    for (int k = REC_RUN - 1; k >= 0; --k) id = (left >> k) & 1u ? cid[k] : id;
-    uint4 h = make_uint4(0, NONE, 0, 0);                      // (id, index, first counter, members); index NONE: unregistered
-    if (act) h = comm_find(R, id, R.hash[hash_home(R, id)]);
-    // a record folded earlier carries another id, so matching the id is enough (the run is complete: no padding)
-    u32 m = 0, mn = NONE, mx = 0;
-#pragma unroll
-    for (int k = 0; k < REC_RUN; ++k) {
-      if (cid[k] == id) { m |= 1u << k; mn = min(mn, sq[k]); mx = max(mx, sq[k]); }
-    }
-    m &= left;
-    if (h.y != NONE && m != 0 && mn < h.z) {
-      // counters below the communicator's first name no operation: fold again without them
-      mn = NONE; mx = 0;
-#pragma unroll
-      for (int k = 0; k < REC_RUN; ++k) if (((m >> k) & 1u) && sq[k] >= h.z) { mn = min(mn, sq[k]); mx = max(mx, sq[k]); }
-    }
-    if (m == 0) { mn = NONE; mx = 0; }
-    left &= ~m;
-    // lanes that hold the same communicator merge: a few rounds, each led by the lowest lane still waiting
-    bool mine = act && h.y != NONE && mn <= mx;
-    u32 pend = __ballot_sync(0xFFFFFFFFu, mine);
-    for (int it = 0; it < RANGE_FOLDS && pend; ++it) {
-      const u32 leader = (u32)__ffs(pend) - 1u;
-      const u32 lid = __shfl_sync(0xFFFFFFFFu, h.y, leader);
-      const bool same = mine && h.y == lid;
-      const u32 a = __reduce_min_sync(0xFFFFFFFFu, same ? mn : NONE), b = __reduce_max_sync(0xFFFFFFFFu, same ? mx : 0u);
-      if (lane == leader) range_put(D, s_mn, s_mx, lid, a, b);
-      if (same) mine = false;
-      pend &= ~__ballot_sync(0xFFFFFFFFu, same);
-    }
-    if (mine) range_put(D, s_mn, s_mx, h.y, mn, mx);
-  }
-  // every record still left: one lookup each, four in flight
-  left |= tail;
-  if (left != 0) {
-#pragma unroll
-    for (int k0 = 0; k0 < REC_RUN; k0 += 4) {
-      uint4 h[4]; bool need[4];
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        need[q] = ((left >> (k0 + q)) & 1u) != 0;
-        h[q] = need[q] ? R.hash[hash_home(R, cid[k0 + q])] : make_uint4(0, NONE, 0, 0);
+      // lanes that hold the same communicator merge: a few rounds, each led by the lowest lane still waiting
+      bool mine = act && h.y != NONE && mn <= mx;
+      u32 pend = __ballot_sync(0xFFFFFFFFu, mine);
+      for (int it = 0; it < RANGE_FOLDS && pend; ++it) {
+        const u32 leader = (u32)__ffs(pend) - 1u;
+        const u32 lid = __shfl_sync(0xFFFFFFFFu, h.y, leader);
+        const bool same = mine && h.y == lid;
+        const u32 a = __reduce_min_sync(0xFFFFFFFFu, same ? mn : NONE), b = __reduce_max_sync(0xFFFFFFFFu, same ? mx : 0u);
+        if (lane == leader) range_put(D, s_mn, s_mx, lid, a, b);
+        if (same) mine = false;
+        pend &= ~__ballot_sync(0xFFFFFFFFu, same);
       }
-#pragma unroll
-      for (int q = 0; q < 4; ++q) {
-        if (!need[q]) continue;
-        const uint4 e = comm_find(R, cid[k0 + q], h[q]);
-        if (e.y != NONE && sq[k0 + q] >= e.z) range_put(D, s_mn, s_mx, e.y, sq[k0 + q], sq[k0 + q]);
+      if (mine) range_put(D, s_mn, s_mx, h.y, mn, mx);
+    }
+    // every record still left: one lookup each, four in flight
+    left |= tail;
+    if (left != 0) {
+  #pragma unroll
+      for (int k0 = 0; k0 < REC_RUN; k0 += 4) {
+        uint4 h[4]; bool need[4];
+  #pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          need[q] = ((left >> (k0 + q)) & 1u) != 0;
+          h[q] = need[q] ? R.hash[hash_home(R, cid[k0 + q])] : make_uint4(0, NONE, 0, 0);
+        }
+  #pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          if (!need[q]) continue;
+          const uint4 e = comm_find(R, cid[k0 + q], h[q]);
+          if (e.y != NONE && sq[k0 + q] >= e.z) range_put(D, s_mn, s_mx, e.y, sq[k0 + q], sq[k0 + q]);
+        }
       }
     }
   }
