@@ -651,7 +651,12 @@ int analyze_batch(ccld_ctx* ctx, u32 first_window, u32 n_windows, i64 now_ns, bo
   if (total_slots) CK(cudaMemsetAsync(rbase + o_perm, 0xFF, total_slots * 4, st));
   PlanLists pl; pl.fcta = (FusedCta*)(rbase + o_fcta); pl.fwt = (WarpTile*)(rbase + o_fwt); pl.t2 = (Tile*)(rbase + o_t2); pl.t3 = (Tile*)(rbase + o_t3);
   { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, pl, 1); }
-  if (cta > 0) { TimedLaunch tl(ts, 2, st); k_slot_scatter<<<dim3((u32)((cta * REC_PER_CTA + SCAT_PER_CTA - 1) / SCAT_PER_CTA), B), SCAT_THREADS, 0, st>>>(d_desc, ctx->reg); }
+  if (cta > 0) {
+    const u64 blocks = (cta * REC_PER_CTA + SCAT_PER_CTA - 1) / SCAT_PER_CTA;      // of the largest window
+    const u32 per = (u32)std::min<u64>(SCAT_BLOCKS_MAX, std::max<u64>(1, blocks * B / (32ull * ctx->n_sms)));
+    TimedLaunch tl(ts, 2, st);
+    k_slot_scatter<<<dim3((u32)((blocks + per - 1) / per), B), SCAT_THREADS, 0, st>>>(d_desc, ctx->reg, per);
+  }
   CK(cudaMemsetAsync(rbase + o_defn, 0, 16, st));
   if (n_list[B_FCTA]) {
     const DeferList dl{(u64*)(rbase + o_def), (u32*)(rbase + o_defn)};

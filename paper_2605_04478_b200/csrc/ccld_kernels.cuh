@@ -619,6 +619,7 @@ __global__ void __launch_bounds__(PLAN_THREADS) k_plan(WinDesc* __restrict__ wd,
 constexpr int SCAT_THREADS = 256;     // lanes on consecutive records: the stores of a warp land close together
 constexpr int SCAT_PER_THREAD = 12;    // records per thread: enough to spread the two dependent table reads a warp starts with
 constexpr int SCAT_PER_CTA = SCAT_THREADS * SCAT_PER_THREAD;
+constexpr u32 SCAT_BLOCKS_MAX = 8;    // blocks of SCAT_PER_CTA records a CTA takes at most
 
 __device__ __noinline__ u64 resolve_slow(const Registry& R, u32 rank, u32 cid) {
   const u32 c = comm_lookup(R, cid);
@@ -649,75 +650,92 @@ constexpr u32 SCAT_LOCAL = 8;     // ranks, counted from the rank of the CTA's f
 // first counter), which the layout pass wrote for this window - into shared memory; a record of those ranks then needs no global table at all and, in windows of
 // fewer than 2^32 slots, only 32-bit arithmetic. Any other record (another rank, a communicator beyond the inline pairs,
 // a counter outside the range, a rejected record) takes the two dependent table loads and the full checks.
-__global__ void __launch_bounds__(SCAT_THREADS, 4) k_slot_scatter(const WinDesc* __restrict__ wd, Registry R) {
+__global__ void __launch_bounds__(SCAT_THREADS, 4) k_slot_scatter(const WinDesc* __restrict__ wd, Registry R, u32 blocks_per_cta) {
   // (communicator id, counters covered, first counter, first slot) per resolved pair; counters covered 0: unused. Every
-  // warp resolves its own copy, so no warp waits for another.
-  __shared__ uint4 s_ent_all[SCAT_THREADS / 32][SCAT_LOCAL * RANK_TAB_K];
+  // warp keeps its own copy, so no warp waits for another; two copies, because the entries of the next block are written
+  // while lanes may still read those of the current one.
+  __shared__ uint4 s_ent_all[2][SCAT_THREADS / 32][SCAT_LOCAL * RANK_TAB_K];
+  static_assert(SCAT_LOCAL * RANK_TAB_K == 32, "one resolved pair per lane");
   const WinDesc& D = wd[blockIdx.y];                          // grid: (CTAs of the largest window, windows)
-  const u64 base = (u64)blockIdx.x * SCAT_PER_CTA;
-  if (base >= D.n_rec) return;                                // (a window that was given up has empty scatter rows: nothing is stored)
+  const u64 base0 = (u64)blockIdx.x * blocks_per_cta * SCAT_PER_CTA;
+  if (base0 >= D.n_rec) return;                               // (a window that was given up has empty scatter rows: nothing is stored)
   u32 err = 0, rej = 0, internal = 0;
   // descriptor fields in registers: the stores below could alias the descriptor as far as the compiler knows
   u32* const perm = D.perm; const u64 n_slots = D.n_slots; const uint4* const srow = D.srow; const u64 n_rec = D.n_rec;
+  const uint4* const rent = D.rent;
   const u32 *c_rank = D.rank, *c_comm = D.comm, *c_seq = D.seq;
-  // the records first: their loads are in flight while the table rows are resolved
-  u32 rk[SCAT_PER_THREAD], cid[SCAT_PER_THREAD], sq[SCAT_PER_THREAD];
-  u32 todo = 0;                                             // records that still need placing
-#pragma unroll
-  for (int k = 0; k < SCAT_PER_THREAD; ++k) {
-    const u64 i = base + (u64)k * SCAT_THREADS + threadIdx.x;
-    const bool in = i < n_rec;
-    rk[k] = in ? c_rank[i] : 0u; cid[k] = in ? c_comm[i] : 0u; sq[k] = in ? c_seq[i] : 0u;
-    if (in) todo |= 1u << k;
-  }
-  const u32 lane = threadIdx.x & 31;
-  uint4* const s_ent = s_ent_all[threadIdx.x >> 5];
-  const u32 r_first = c_rank[base];
-  if (lane < SCAT_LOCAL * RANK_TAB_K) {
+  const u32 lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+  // the resolved pairs of the SCAT_LOCAL ranks that start at rank r_first, one per lane
+  auto pairs_of = [&](u32 r_first) {
     const u32 r = r_first + lane / RANK_TAB_K;
     uint4 e = make_uint4(NONE, 0, 0, 0);
-    if (r_first < R.n_ranks && r < R.n_ranks) e = D.rent[(u64)r * RANK_TAB_K + lane % RANK_TAB_K];
-    if (e.y == 0) e.x = NONE;                                 // an unused pair must not shadow a record of communicator 0
-    s_ent[lane] = e;
-  }
-  __syncwarp();
-#pragma unroll
-  for (int k = 0; k < SCAT_PER_THREAD; ++k) {
-    const u32 dr = rk[k] - r_first;
-    if (dr < SCAT_LOCAL) {
-      const uint4* ent = s_ent + dr * RANK_TAB_K;
-      uint4 e = ent[0];
-#pragma unroll
-      for (int q = 1; q < RANK_TAB_K; ++q) { const uint4 x = ent[q]; if (x.x == cid[k]) e = x; }
-      const u32 off = sq[k] - e.z;                            // below the first counter: wraps to a huge value
-      if (e.x == cid[k] && off < e.y && ((todo >> k) & 1u)) {
-        perm[e.w + off] = (u32)base + (u32)k * SCAT_THREADS + threadIdx.x;
-        todo &= ~(1u << k);
-      }
-    }
-  }
-  if (__any_sync(0xFFFFFFFFu, todo != 0)) {
+    if (r_first < R.n_ranks && r < R.n_ranks) e = rent[(u64)r * RANK_TAB_K + lane % RANK_TAB_K];
+    return e;
+  };
+  // A CTA takes blocks_per_cta consecutive blocks. The chain "first record's rank -> that rank's resolved pairs" of a
+  // block is started one block ahead, so a block waits for its records only.
+  u32 r_first = c_rank[base0];
+  uint4 e_mine = pairs_of(r_first);
+  for (u32 blk = 0; blk < blocks_per_cta; ++blk) {
+    const u64 base = base0 + (u64)blk * SCAT_PER_CTA;
+    if (base >= n_rec) break;
+    u32 rk[SCAT_PER_THREAD], cid[SCAT_PER_THREAD], sq[SCAT_PER_THREAD];
+    u32 todo = 0;                                             // records that still need placing
 #pragma unroll
     for (int k = 0; k < SCAT_PER_THREAD; ++k) {
-      if (!((todo >> k) & 1u)) continue;
-      u32 v = NONE;
-      if (rk[k] < R.n_ranks) {
-        const uint4 ta = R.rank_tab[(u64)rk[k] * 2], tb = R.rank_tab[(u64)rk[k] * 2 + 1];
-        v = ta.x == cid[k] ? ta.y : v; v = ta.z == cid[k] ? ta.w : v;
-        v = tb.x == cid[k] ? tb.y : v; v = tb.z == cid[k] ? tb.w : v;
-      }
-      if (v == NONE || v == RANK_TAB_OVERFLOW || cid[k] == NONE) {
-        const u64 rs = resolve_slow(R, rk[k], cid[k]);
-        v = (u32)rs;
-        if (rs >> 32) { err |= (u32)(rs >> 32); ++rej; }
-      }
-      if (v == NONE) continue;
-      const u32 c = v >> RANK_TAB_POS_BITS;
-      const uint4 sr = srow[c];
-      u64 slot;
-      if (scatter_slot(R, c, sr.z, sr.w, ((u64)sr.x | ((u64)sr.y << 32)) + (u64)(v & ((1u << RANK_TAB_POS_BITS) - 1)) * sr.z, sq[k], n_slots, &slot, &err, &rej, &internal))
-        perm[slot] = (u32)(base + (u64)k * SCAT_THREADS + threadIdx.x);
+      const u64 i = base + (u64)k * SCAT_THREADS + threadIdx.x;
+      const bool in = i < n_rec;
+      rk[k] = in ? c_rank[i] : 0u; cid[k] = in ? c_comm[i] : 0u; sq[k] = in ? c_seq[i] : 0u;
+      if (in) todo |= 1u << k;
     }
+    const u64 base_next = base + SCAT_PER_CTA;
+    const bool has_next = blk + 1 < blocks_per_cta && base_next < n_rec;
+    const u32 r_next = has_next ? c_rank[base_next] : 0u;     // in flight with the records
+    uint4* const s_ent = s_ent_all[blk & 1][wid];
+    if (e_mine.y == 0) e_mine.x = NONE;                       // an unused pair must not shadow a record of communicator 0
+    s_ent[lane] = e_mine;
+    __syncwarp();
+#pragma unroll
+    for (int k = 0; k < SCAT_PER_THREAD; ++k) {
+      const u32 dr = rk[k] - r_first;
+      if (dr < SCAT_LOCAL) {
+        const uint4* ent = s_ent + dr * RANK_TAB_K;
+        uint4 e = ent[0];
+#pragma unroll
+        for (int q = 1; q < RANK_TAB_K; ++q) { const uint4 x = ent[q]; if (x.x == cid[k]) e = x; }
+        const u32 off = sq[k] - e.z;                          // below the first counter: wraps to a huge value
+        if (e.x == cid[k] && off < e.y && ((todo >> k) & 1u)) {
+          perm[e.w + off] = (u32)base + (u32)k * SCAT_THREADS + threadIdx.x;
+          todo &= ~(1u << k);
+        }
+      }
+    }
+    // the next block's pairs: its first rank has arrived with this block's records
+    if (has_next) e_mine = pairs_of(r_next);
+    if (__any_sync(0xFFFFFFFFu, todo != 0)) {
+#pragma unroll
+      for (int k = 0; k < SCAT_PER_THREAD; ++k) {
+        if (!((todo >> k) & 1u)) continue;
+        u32 v = NONE;
+        if (rk[k] < R.n_ranks) {
+          const uint4 ta = R.rank_tab[(u64)rk[k] * 2], tb = R.rank_tab[(u64)rk[k] * 2 + 1];
+          v = ta.x == cid[k] ? ta.y : v; v = ta.z == cid[k] ? ta.w : v;
+          v = tb.x == cid[k] ? tb.y : v; v = tb.z == cid[k] ? tb.w : v;
+        }
+        if (v == NONE || v == RANK_TAB_OVERFLOW || cid[k] == NONE) {
+          const u64 rs = resolve_slow(R, rk[k], cid[k]);
+          v = (u32)rs;
+          if (rs >> 32) { err |= (u32)(rs >> 32); ++rej; }
+        }
+        if (v == NONE) continue;
+        const u32 c = v >> RANK_TAB_POS_BITS;
+        const uint4 sr = srow[c];
+        u64 slot;
+        if (scatter_slot(R, c, sr.z, sr.w, ((u64)sr.x | ((u64)sr.y << 32)) + (u64)(v & ((1u << RANK_TAB_POS_BITS) - 1)) * sr.z, sq[k], n_slots, &slot, &err, &rej, &internal))
+          perm[slot] = (u32)(base + (u64)k * SCAT_THREADS + threadIdx.x);
+      }
+    }
+    r_first = r_next;
   }
   err = __reduce_or_sync(0xFFFFFFFFu, err);
   rej = __reduce_add_sync(0xFFFFFFFFu, rej);
