@@ -653,7 +653,7 @@ int analyze_batch(ccld_ctx* ctx, u32 first_window, u32 n_windows, i64 now_ns, bo
   { TimedLaunch tl(ts, 1, st); k_plan<<<B, PLAN_THREADS, 0, st>>>(d_desc, ctx->reg, pl, 1); }
   if (cta > 0) {
     const u64 blocks = (cta * REC_PER_CTA + SCAT_PER_CTA - 1) / SCAT_PER_CTA;      // of the largest window
-    const u32 per = (u32)std::min<u64>(SCAT_BLOCKS_MAX, std::max<u64>(1, blocks * B / (32ull * ctx->n_sms)));
+    const u32 per = (u32)std::min<u64>(SCAT_BLOCKS_MAX, std::max<u64>(1, blocks * B / (16ull * ctx->n_sms)));
     TimedLaunch tl(ts, 2, st);
     k_slot_scatter<<<dim3((u32)((blocks + per - 1) / per), B), SCAT_THREADS, 0, st>>>(d_desc, ctx->reg, per);
   }
